@@ -1,0 +1,234 @@
+/*
+ * speca.h -- C ABI of the SpeCa speculative feature-cache hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the data-parallel arithmetic of "forecast-then-verify" sampling
+ * for diffusion transformers (SpeCa, arXiv 2509.11628):
+ *
+ *   - the per-layer derivative table that the TaylorSeer draft model keeps (Eq. 3, Section 3.3),
+ *     rewritten in place at every fully computed reference step,
+ *   - the Taylor extrapolation of every cached block output to a speculative step (Eq. 2),
+ *   - the relative L2 error between the forecast and the freshly computed feature of the
+ *     verification layer, reduced to one accept/reject decision per sample (Eq. 4 and the
+ *     sequential validation rule of Section 3.4.2),
+ *   - per-sample masks so that rejected samples of a batch stop forecasting (the
+ *     sample-adaptive computation allocation of Sections 1 and 4).
+ *
+ * Conventions shared by every entry point
+ *   - Every function returns a speca_status_t. Nothing throws, aborts or prints.
+ *   - "host" pointers are read during the call and may be freed on return. "device" pointers
+ *     must be valid on the cache's CUDA device until the work enqueued on `stream` has run.
+ *   - All device work is enqueued on the caller's stream (a cudaStream_t passed as void*, NULL =
+ *     the legacy default stream) and the call returns without synchronising.
+ *   - Arguments are validated on the host before anything is launched: a call that returns an
+ *     error has enqueued nothing and has not changed the cache's state.
+ *   - Tensors are dense, row-major [B, N_e, D] in the cache's storage dtype; sample b of an entry
+ *     starts at element b*N_e*D. Device tensor pointers must be aligned to the element size;
+ *     16-byte aligned pointers (with N_e*D*sizeof(element) a multiple of 16) take the fast
+ *     vectorised / bulk-copy path, anything else a slower element-wise path with equal results.
+ *   - A handle is not thread safe: use one handle from one host thread at a time.
+ *   - There is no CPU fallback: without a usable CUDA device speca_cache_create fails.
+ */
+#ifndef SPECA_H_
+#define SPECA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPECA_MAX_ORDER   4     /* highest Taylor order m */
+#define SPECA_MAX_BATCH   64    /* most samples B in one cache */
+#define SPECA_MAX_ENTRIES 512   /* most cached tensors (block outputs) in one cache */
+
+typedef struct speca_cache speca_cache_t; /* opaque, owned by the library */
+
+typedef enum {
+    SPECA_OK = 0,
+    SPECA_ERR_INVALID_ARG = 1, /* null pointer, value out of range, non-finite time */
+    SPECA_ERR_SHAPE = 2,       /* entry list / batch / order outside the supported limits */
+    SPECA_ERR_ALIGNMENT = 3,   /* pointer not aligned as the call requires */
+    SPECA_ERR_STATE = 4,       /* call order violated (forecast before an update, double update ...) */
+    SPECA_ERR_ZERO_GAP = 5,    /* a reference time equals one it must differ from */
+    SPECA_ERR_NOMEM = 6,       /* arena too small, or host allocation failed */
+    SPECA_ERR_CUDA = 7,        /* a CUDA runtime call failed; see speca_last_error */
+    SPECA_ERR_UNSUPPORTED = 8  /* device is not an sm_100 part, or feature not built */
+} speca_status_t;
+
+typedef enum { SPECA_F32 = 0, SPECA_BF16 = 1 } speca_dtype_t;
+
+/*
+ * Which polynomial basis the derivative table holds.
+ *  SPECA_BASIS_TAYLOR  Eq. 2-3 as printed: plane i holds the i-th backward difference quotient
+ *                      (Delta^i F / N^i on a uniform grid of spacing N), the forecast is
+ *                      sum_i plane_i * x^i / i! with x = t_target - t_last. For non-uniform
+ *                      reference times every quotient divides by the latest gap. Exact for
+ *                      features that are polynomials of degree <= 1 in t.
+ *  SPECA_BASIS_NEWTON  Newton divided differences over the true reference times, evaluated in
+ *                      Newton form. Exact for polynomials of degree <= m at any gaps. Same
+ *                      kernels, different host-computed scalars.
+ */
+typedef enum { SPECA_BASIS_TAYLOR = 0, SPECA_BASIS_NEWTON = 1 } speca_basis_t;
+
+/* Which kernel variant moves the data. Results are identical; only speed differs. */
+typedef enum {
+    SPECA_PATH_AUTO = 0,   /* library default */
+    SPECA_PATH_DIRECT = 1, /* vectorised global loads straight into registers */
+    SPECA_PATH_BULK = 2    /* cp.async.bulk (TMA) staging through a shared-memory ring */
+} speca_path_t;
+
+typedef struct {
+    int64_t tokens; /* N_e  >= 1 */
+    int32_t dim;    /* D    >= 1 */
+} speca_entry_desc_t;
+
+typedef struct {
+    int32_t n_entries;                 /* 1..SPECA_MAX_ENTRIES */
+    const speca_entry_desc_t* entries; /* host; copied by speca_cache_create */
+    int32_t batch;                     /* B, 1..SPECA_MAX_BATCH */
+    int32_t max_order;                 /* m, 0..SPECA_MAX_ORDER (0 = plain cache reuse) */
+    int32_t dtype;                     /* speca_dtype_t: storage type of tables, features, forecasts */
+    int32_t basis;                     /* speca_basis_t */
+    int32_t verify_entry;              /* index of the verification layer's entry; -1 = last entry */
+    float eps;                         /* epsilon of Eq. 4; <= 0 selects the paper's 1e-8 */
+    void* arena;                       /* device; caller-owned, 256-byte aligned, lives as long as the handle */
+    size_t arena_bytes;                /* >= speca_cache_arena_bytes() */
+    int32_t device;                    /* CUDA device ordinal that owns the arena */
+    int32_t path;                      /* speca_path_t */
+} speca_cache_config_t;
+
+/*
+ * Bytes of device memory a cache with this configuration needs (tables for every entry, sample
+ * and order 0..m, plus a few KB of descriptors and reduction scratch). `arena`, `arena_bytes`
+ * and `device` are ignored. Host only; touches no GPU.
+ * Errors: INVALID_ARG (null), SHAPE (limits exceeded, sizes overflow).
+ */
+speca_status_t speca_cache_arena_bytes(const speca_cache_config_t* cfg, size_t* out_bytes);
+
+/*
+ * Build a cache over the caller's arena (Section 3.3: one derivative table per cached block
+ * output). Writes the descriptor tables into the arena (synchronously) and returns a handle in
+ * *out. The arena's table region is not cleared: planes are defined only once an update has
+ * written them. Errors: INVALID_ARG, SHAPE, ALIGNMENT (arena), NOMEM (arena too small),
+ * CUDA, UNSUPPORTED (device is not compute capability 10.x).
+ */
+speca_status_t speca_cache_create(const speca_cache_config_t* cfg, speca_cache_t** out);
+
+/* Waits for the device to finish work that uses the handle, then frees host state. The arena
+ * stays with the caller. NULL is accepted. */
+speca_status_t speca_cache_destroy(speca_cache_t* cache);
+
+/* Forget the reference history of the samples with host_sample_mask[b] != 0 (NULL = all):
+ * their next update is a first update. Host state only. */
+speca_status_t speca_cache_reset(speca_cache_t* cache, const uint8_t* host_sample_mask);
+
+/*
+ * Reference step, Eq. 3 / workflow step 1 of Section 3.2: fold freshly computed features into
+ * the derivative tables, in place.
+ *   feats            host array of n_entries device pointers; feats[e] = [B, N_e, D] feature of
+ *                    entry e at the new reference time, NULL = entry e is not part of this call
+ *                    (a model hands over one block at a time; any subset per call is fine).
+ *   t_ref            host, B doubles: the reference time of each sample (any monotone or
+ *                    non-monotone coordinate; only differences are used).
+ *   host_sample_mask host, B bytes, NULL = all: samples that were fully computed. Other samples'
+ *                    tables are neither read nor written.
+ * For sample b with r = number of committed references: plane 0 <- f; for i < min(m, r):
+ * plane i+1 <- (new plane i - old plane i) / gap_i, the chain carried in fp32 and each plane
+ * rounded once to the storage dtype. gap_i is t_ref - t_last (TAYLOR) or t_ref - (i-th previous
+ * reference time) (NEWTON).
+ * All entries of one reference step must be updated (each exactly once per masked sample)
+ * before speca_cache_commit_step; t_ref and the mask must be the same in all of those calls.
+ * Errors: INVALID_ARG, ALIGNMENT, ZERO_GAP, STATE (entry updated twice in one step, or
+ * t_ref / mask differ from the step's first call), CUDA.
+ */
+speca_status_t speca_cache_update(speca_cache_t* cache, const void* const* feats, const double* t_ref,
+                                  const uint8_t* host_sample_mask, void* stream);
+
+/*
+ * Close a reference step: push t_ref into each masked sample's reference history and raise its
+ * reference count. Host state only. Errors: STATE if some entry has not been updated for
+ * exactly the masked samples since the last commit, or no update is pending.
+ */
+speca_status_t speca_cache_commit_step(speca_cache_t* cache);
+
+/*
+ * Speculative step, Eq. 2 / workflow step 2: extrapolate every cached block output to t_target.
+ *   t_target        host, B doubles.
+ *   dev_active_mask device, B bytes, NULL = all samples: samples with a zero byte are skipped
+ *                   (their planes are not read, their rows of outs are not written).
+ *   outs            host array of n_entries device pointers, outs[e] = [B, N_e, D], NULL = skip e.
+ * out = sum_{i=0..v} plane_i * prod-of-multipliers, evaluated by Horner's rule in fp32 and
+ * rounded once to the storage dtype; v = min(m, references - 1) per sample.
+ * Errors: INVALID_ARG, ALIGNMENT, STATE (a sample has no committed reference and the mask is
+ * NULL; with a device mask such samples must be inactive: they are skipped on the device), CUDA.
+ */
+speca_status_t speca_forecast(speca_cache_t* cache, const double* t_target, const uint8_t* dev_active_mask,
+                              void* const* outs, void* stream);
+
+/*
+ * Verification, Eq. 4 and the accept rule of Section 3.4.2, fused with the forecast of the
+ * verification entry:  e_b = ||p_b - f_b||_2 / (||f_b||_2 + eps),  accept_b = (e_b <= tau_b),
+ * with p the forecast rounded to the storage dtype and the norms taken over all N_v*D elements
+ * of sample b. Sums are accumulated in fp32 per thread and combined in a fixed order (warp
+ * shuffle, shared memory, cluster shared memory, then fp64 across clusters), so results are
+ * identical from run to run. A NaN anywhere in a sample rejects it.
+ *   fresh           device, [B, N_v, D]: the verification layer's feature computed by the model.
+ *   t_target, tau   host, B doubles / B floats.
+ *   dev_active_mask device, B bytes, NULL = all. Inactive samples: err, accept, out_pred untouched.
+ *   out_pred        device [B, N_v, D] or NULL: also store the forecast p.
+ *   dev_err         device, B floats.  dev_accept: device, B bytes (1 = accept).
+ * Uses a few KB of reduction scratch inside the arena: two verify calls on the same handle must
+ * not overlap on the GPU (enqueue them on one stream).
+ * Errors: INVALID_ARG, ALIGNMENT, STATE, CUDA.
+ */
+speca_status_t speca_verify(speca_cache_t* cache, const void* fresh, const double* t_target, const float* tau,
+                            const uint8_t* dev_active_mask, void* out_pred, float* dev_err,
+                            uint8_t* dev_accept, void* stream);
+
+/*
+ * Per-sample continuation of the speculative run (sequential validation of Section 3.4.2, the
+ * forced activation period N of Appendix A, sample-adaptive allocation):
+ *   for every active sample b: if accept_b then spec_count_b += 1
+ *   keep_b   = active_b && accept_b && spec_count_b < k_max
+ *   active'_b = AND of keep over the `group` consecutive samples that contain b
+ *               (group = 1: per sample; 2: a classifier-free-guidance pair shares its fate)
+ *   dev_active_idx = ascending list of the samples with active' = 1, dev_n_active = its length.
+ * All pointers are device pointers; dev_spec_count (B int32) and dev_active_mask (B bytes) are
+ * updated in place; dev_active_idx (B int32) and dev_n_active (1 int32) may be NULL.
+ * Errors: INVALID_ARG (null, k_max < 1, group < 1 or not dividing B), CUDA.
+ */
+speca_status_t speca_select_adaptive(speca_cache_t* cache, const uint8_t* dev_accept, int32_t k_max,
+                                     int32_t group, int32_t* dev_spec_count, uint8_t* dev_active_mask,
+                                     int32_t* dev_active_idx, int32_t* dev_n_active, void* stream);
+
+/* After a reference step: mark the samples with host_sample_mask[b] != 0 (NULL = all) active again
+ * and clear their speculative-step counters, on the stream. Errors: INVALID_ARG, CUDA. */
+speca_status_t speca_activate(speca_cache_t* cache, const uint8_t* host_sample_mask, int32_t* dev_spec_count,
+                              uint8_t* dev_active_mask, void* stream);
+
+/* Threshold schedule of Section 3.4.2: tau_t = tau0 * beta^((T - t) / T). Returns NaN for T <= 0. */
+double speca_tau(double tau0, double beta, double t, double T);
+
+/* Per-sample host state: committed reference count and latest reference time (NaN if none).
+ * Either output may be NULL. */
+speca_status_t speca_cache_state(const speca_cache_t* cache, int32_t* host_n_refs, double* host_t_last);
+
+/* Device address and byte stride of the table of (entry, sample): plane i starts at
+ * *plane0 + i * *plane_stride_bytes. For checkpointing and tests. */
+speca_status_t speca_cache_plane(const speca_cache_t* cache, int32_t entry, int32_t sample, void** plane0,
+                                 size_t* plane_stride_bytes);
+
+/* How many kernels the handle has launched since it was created. */
+speca_status_t speca_cache_launch_count(const speca_cache_t* cache, uint64_t* out);
+
+const char* speca_status_string(speca_status_t status);
+/* Human-readable detail of the most recent error on this handle ("" if none). */
+const char* speca_last_error(const speca_cache_t* cache);
+/* Library version string. */
+const char* speca_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECA_H_ */

@@ -1,0 +1,180 @@
+/*
+ * speca_oracle.c -- plain CPU statement of the SpeCa feature-cache arithmetic (arXiv 2509.11628).
+ *
+ * TEST INFRASTRUCTURE ONLY. This file is the yardstick the CUDA library is compared with. It is
+ * deliberately slow and literal: double arithmetic on values read back from storage, one loop per
+ * equation, no blocking, no fusion. It shares no code, header, table or helper with the CUDA
+ * path, and nothing in the product may call it.
+ *
+ * What each function follows
+ *   oracle_update_segment    Eq. 3 (finite differences of the cached feature), kept as difference
+ *                            quotients so that reference steps may be unevenly spaced
+ *   oracle_forecast_segment  Eq. 2 (TaylorSeer prediction), written as the printed sum
+ *   oracle_rel_l2            Eq. 4 (relative error, epsilon = 1e-8)
+ *   oracle_accept            Section 3.4.2, rule 1/2 (e <= tau accepts)
+ *   oracle_tau               Section 3.4.2, tau_t = tau0 * beta^((T-t)/T)
+ *   oracle_speedup           Eq. 8, S = 1 / (1 - alpha + alpha*gamma)
+ *
+ * Pins (tests/test_oracle_pins.py): exact-rational evaluation of Eq. 2-3 from the raw feature
+ * history; order 0 == reuse; exactness on polynomials (degree <= 1 Taylor basis, degree <= m
+ * Newton basis); closed-form quadratic residual; Eq. 4 special cases and brute force; the
+ * paper's worked speed-up number. Unpinned: nothing the paper prints numbers for exists beyond
+ * the speed-up example; uneven gaps in the Taylor basis are pinned only through the
+ * degree <= 1 exactness and the recursion's definition ("parity unpinned" for that case
+ * beyond those two properties).
+ *
+ * Storage types: 0 = IEEE binary32, 1 = bfloat16 (upper 16 bits of binary32, round to nearest
+ * even on store, NaN kept NaN).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#define ORACLE_MAX_ORDER 8
+
+enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
+enum { ORACLE_TAYLOR = 0, ORACLE_NEWTON = 1 };
+
+/* ---- storage <-> double ------------------------------------------------------------------ */
+
+static double bf16_bits_to_double(uint16_t h) {
+    uint32_t w = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &w, sizeof f);
+    return (double)f;
+}
+
+/* Round a double to the nearest bfloat16 (ties to even) and return its bits. bfloat16 has 8
+ * significant bits and binary32's exponent range, so: scale the value so that one unit in the
+ * last place becomes 1.0, round to an integer with the default rounding mode, scale back. */
+uint16_t oracle_double_to_bf16_bits(double v) {
+    if (isnan(v)) return 0x7FC0u;
+    if (isinf(v)) return v > 0 ? 0x7F80u : 0xFF80u;
+    if (v == 0.0) return signbit(v) ? 0x8000u : 0x0000u;
+    int e;
+    (void)frexp(v, &e); /* |v| = f * 2^e with f in [0.5, 1) -> leading bit has weight 2^(e-1) */
+    int lead = e - 1;
+    if (lead < -126) lead = -126; /* subnormal range: fixed quantum 2^-133 */
+    double q = nearbyint(ldexp(v, 7 - lead)); /* 7 fraction bits below the leading bit */
+    double r = ldexp(q, lead - 7);
+    if (fabs(r) >= ldexp(1.0, 128)) return r > 0 ? 0x7F80u : 0xFF80u;
+    float f = (float)r; /* exact: r has at most 8 significant bits */
+    uint32_t w;
+    memcpy(&w, &f, sizeof w);
+    return (uint16_t)(w >> 16);
+}
+
+static double load_elem(const void* p, int dtype, int64_t i) {
+    if (dtype == ORACLE_F32) return (double)((const float*)p)[i];
+    return bf16_bits_to_double(((const uint16_t*)p)[i]);
+}
+
+static void store_elem(void* p, int dtype, int64_t i, double v) {
+    if (dtype == ORACLE_F32)
+        ((float*)p)[i] = (float)v;
+    else
+        ((uint16_t*)p)[i] = oracle_double_to_bf16_bits(v);
+}
+
+/* ---- Eq. 3: table rewrite at a reference step ---------------------------------------------- */
+/*
+ * One (entry, sample) table of `n` elements, planes[i] at planes + i*plane_stride elements.
+ * n_refs  = references folded in so far (0 = empty table).
+ * t_hist  = their times, most recent first (t_hist[0] = t_last); min(n_refs, m) are read.
+ * The i-th finite difference of Eq. 3 over reference times t, t+N, ..., t+iN obeys
+ * Delta^i F(t) = Delta^(i-1) F(t) - Delta^(i-1) F(t+N); the table keeps Delta^i / N^i, so the
+ * new quotient of order i+1 is (new order-i quotient - old order-i quotient) / (t_new - t_last).
+ * Newton basis: the divisor is t_new - t_hist[i] instead (divided differences).
+ * The chain runs on unrounded values; each plane is rounded once when stored.
+ * Returns 0, or 1 if a divisor is zero (nothing is written then).
+ */
+int oracle_update_segment(int dtype, int64_t n, int m, int basis, int n_refs, const double* t_hist,
+                          double t_new, const void* feat, void* planes, int64_t plane_stride) {
+    int v_new = n_refs < m ? n_refs : m; /* highest order defined after this update */
+    double gap[ORACLE_MAX_ORDER];
+    for (int i = 0; i < v_new; ++i) {
+        gap[i] = t_new - (basis == ORACLE_NEWTON ? t_hist[i] : t_hist[0]);
+        if (gap[i] == 0.0) return 1;
+    }
+    size_t esz = dtype == ORACLE_F32 ? 4 : 2;
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < n; ++j) {
+        double c[ORACLE_MAX_ORDER + 1];
+        c[0] = load_elem(feat, dtype, j);
+        for (int i = 0; i < v_new; ++i) {
+            double old_i = load_elem((const char*)planes + (size_t)i * plane_stride * esz, dtype, j);
+            c[i + 1] = (c[i] - old_i) / gap[i];
+        }
+        for (int i = 0; i <= v_new; ++i)
+            store_elem((char*)planes + (size_t)i * plane_stride * esz, dtype, j, c[i]);
+    }
+    return 0;
+}
+
+/* ---- Eq. 2: forecast ------------------------------------------------------------------------ */
+/*
+ * v = min(m, n_refs - 1) orders are defined. With x = t_target - t_last (= -k on the paper's
+ * integer grid):
+ *   Taylor basis:  out = plane_0 + sum_{i=1..v} plane_i * x^i / i!
+ *   Newton basis:  out = plane_0 + sum_{i=1..v} plane_i * prod_{j<i} (t_target - t_hist[j])
+ * Returns 0, or 1 if the table is empty (n_refs < 1).
+ */
+int oracle_forecast_segment(int dtype, int64_t n, int m, int basis, int n_refs, const double* t_hist,
+                            double t_target, const void* planes, int64_t plane_stride, void* out) {
+    if (n_refs < 1) return 1;
+    int v = n_refs - 1 < m ? n_refs - 1 : m;
+    double w[ORACLE_MAX_ORDER + 1]; /* weight of plane i */
+    w[0] = 1.0;
+    if (basis == ORACLE_NEWTON) {
+        for (int i = 1; i <= v; ++i) w[i] = w[i - 1] * (t_target - t_hist[i - 1]);
+    } else {
+        double x = t_target - t_hist[0];
+        double fact = 1.0;
+        for (int i = 1; i <= v; ++i) {
+            fact *= (double)i;
+            w[i] = pow(x, (double)i) / fact;
+        }
+    }
+    size_t esz = dtype == ORACLE_F32 ? 4 : 2;
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < n; ++j) {
+        double s = load_elem(planes, dtype, j);
+        for (int i = 1; i <= v; ++i)
+            s += load_elem((const char*)planes + (size_t)i * plane_stride * esz, dtype, j) * w[i];
+        store_elem(out, dtype, j, s);
+    }
+    return 0;
+}
+
+/* ---- Eq. 4: relative error ------------------------------------------------------------------- */
+/* e = ||pred - fresh||_2 / (||fresh||_2 + eps), Euclidean norms over the n elements of a sample. */
+double oracle_rel_l2(int dtype, int64_t n, const void* pred, const void* fresh, double eps) {
+    double num = 0.0, den = 0.0;
+#pragma omp parallel for schedule(static) reduction(+ : num, den)
+    for (int64_t j = 0; j < n; ++j) {
+        double p = load_elem(pred, dtype, j);
+        double f = load_elem(fresh, dtype, j);
+        num += (p - f) * (p - f);
+        den += f * f;
+    }
+    return sqrt(num) / (sqrt(den) + eps);
+}
+
+/* Section 3.4.2: accepted iff e <= tau. A NaN error compares false and is rejected. */
+int oracle_accept(double err, double tau) { return err <= tau ? 1 : 0; }
+
+/* Section 3.4.2: tau_t = tau0 * beta^((T - t)/T). */
+double oracle_tau(double tau0, double beta, double t, double T) { return tau0 * pow(beta, (T - t) / T); }
+
+/* Eq. 8: speed-up for acceptance rate alpha and verification cost ratio gamma. */
+double oracle_speedup(double alpha, double gamma) { return 1.0 / (1.0 - alpha + alpha * gamma); }
+
+/* Number of threads the loops above use (1 when built without OpenMP). */
+#ifdef _OPENMP
+#include <omp.h>
+int oracle_threads(void) { return omp_get_max_threads(); }
+void oracle_set_threads(int n) { omp_set_num_threads(n); }
+#else
+int oracle_threads(void) { return 1; }
+void oracle_set_threads(int n) { (void)n; }
+#endif

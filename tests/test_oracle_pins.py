@@ -1,0 +1,448 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these tests retype the oracle's formulas in floating point: they use exact rational
+arithmetic on the raw feature history (Eq. 2-3 as printed), closed forms, invariants, special
+cases that reduce to a library routine (torch's bfloat16 conversion, Lagrange interpolation),
+hand-computed examples and the one worked number the paper prints.
+"""
+import math
+import os
+from fractions import Fraction
+from math import comb, factorial
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import speca_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def bf16_bits(x: torch.Tensor) -> np.ndarray:
+    return x.to(torch.bfloat16).contiguous().view(torch.int16).numpy().view(np.uint16).copy()
+
+
+def bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def run_history(dtype, m, basis, times, feats):
+    """Feed a raw feature history (oldest first) through the oracle; return planes and history."""
+    n = feats[0].size
+    planes = np.zeros((m + 1, n), dtype=O.np_dtype(dtype))
+    hist = []
+    for k, (t, f) in enumerate(zip(times, feats)):
+        O.update_segment(dtype, m, basis, k, hist, t, np.ascontiguousarray(f), planes)
+        hist = ([t] + hist)[: m + 1]
+    return planes, hist
+
+
+# ---------------------------------------------------------------------------------------------
+# Eq. 2-3 as printed, in exact rationals, from the raw features on a uniform grid
+# ---------------------------------------------------------------------------------------------
+
+def eq3_delta(i, hist_at):
+    """Delta^i F(x_t) = sum_j (-1)^(i-j) C(i,j) F(x_{t+jN}); hist_at(j) = F at t + j*N."""
+    return sum(Fraction((-1) ** (i - j) * comb(i, j)) * hist_at(j) for j in range(i + 1))
+
+
+def eq2_pred(m, N, k, hist_at):
+    """F_pred(x_{t-k}) = F(x_t) + sum_{i=1..m} Delta^i F / (i! N^i) * (-k)^i."""
+    s = Fraction(hist_at(0))
+    for i in range(1, m + 1):
+        s += eq3_delta(i, hist_at) * Fraction((-k) ** i, factorial(i) * N ** i)
+    return s
+
+
+@pytest.mark.parametrize("m", [1, 2, 3, 4])
+@pytest.mark.parametrize("N", [1, 2, 4])
+def test_taylor_basis_equals_printed_equations_in_rationals(m, N):
+    rng = np.random.default_rng(100 * m + N)
+    n = 37
+    t = 40  # current step index; references at t + m*N, ..., t + N, t (time runs downwards)
+    raw = {j: rng.integers(-50, 51, size=n) for j in range(m + 1)}  # F(x_{t+jN}), small integers
+    times = [float(t + j * N) for j in range(m, -1, -1)]
+    feats = [raw[j].astype(np.float32) for j in range(m, -1, -1)]
+    planes, hist = run_history(O.F32, m, O.TAYLOR, times, feats)
+    # stored planes are Delta^i / N^i (exact in binary for these N and integer features)
+    for i in range(m + 1):
+        for e in range(n):
+            want = eq3_delta(i, lambda j: Fraction(int(raw[j][e]))) / Fraction(N ** i)
+            assert Fraction(float(planes[i, e])) == want, (i, e)
+    for k in [1, 2, 3, 5]:
+        out = np.zeros(n, dtype=np.float32)
+        O.forecast_segment(O.F32, m, O.TAYLOR, m + 1, hist, float(t - k), planes, out)
+        for e in range(n):
+            want = eq2_pred(m, N, k, lambda j: Fraction(int(raw[j][e])))
+            got = float(out[e])
+            assert abs(got - float(want)) <= 1.2e-7 * max(1.0, abs(float(want))), (k, e, got, float(want))
+
+
+def test_counterexample_quadratic_is_not_reproduced_by_printed_equations():
+    """f(s) = s^2, t = 0, N = 1, m = 2: Eq. 3 gives Delta^1 = 1, Delta^2 = 2 and Eq. 2 gives
+    k^2 - k, not k^2. The oracle follows the printed equations."""
+    m = 2
+    times = [2.0, 1.0, 0.0]
+    feats = [np.array([s * s], dtype=np.float32) for s in times]
+    planes, hist = run_history(O.F32, m, O.TAYLOR, times, feats)
+    assert planes[:, 0].tolist() == [0.0, 1.0, 2.0]
+    for k in range(1, 6):
+        out = np.zeros(1, dtype=np.float32)
+        O.forecast_segment(O.F32, m, O.TAYLOR, 3, hist, float(-k), planes, out)
+        assert out[0] == k * k - k
+
+
+# ---------------------------------------------------------------------------------------------
+# special cases of the forecast
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype", [O.F32, O.BF16])
+def test_order_zero_is_plain_reuse_bit_for_bit(dtype):
+    g = torch.Generator().manual_seed(1)
+    x = torch.randn(4099, generator=g) * 7
+    f = bf16_bits(x) if dtype == O.BF16 else x.numpy().copy()
+    planes = np.zeros((1, f.size), dtype=f.dtype)
+    O.update_segment(dtype, 0, O.TAYLOR, 0, [], 0.7, f, planes)
+    assert np.array_equal(planes[0], f)
+    out = np.zeros_like(f)
+    O.forecast_segment(dtype, 0, O.TAYLOR, 1, [0.7], 0.3, planes, out)
+    assert np.array_equal(out, f)
+    # a later reference simply replaces the feature
+    f2 = f[::-1].copy()
+    O.update_segment(dtype, 0, O.TAYLOR, 1, [0.7], 0.6, f2, planes)
+    O.forecast_segment(dtype, 0, O.TAYLOR, 2, [0.6], 0.1, planes, out)
+    assert np.array_equal(out, f2)
+
+
+@pytest.mark.parametrize("basis", [O.TAYLOR, O.NEWTON])
+@pytest.mark.parametrize("m", [1, 2, 3])
+def test_warm_up_uses_only_defined_orders(basis, m):
+    """One reference -> reuse; two references -> straight line through them, whatever m is."""
+    f0 = np.array([3.0, -8.0, 0.5], dtype=np.float32)
+    f1 = np.array([5.0, -4.0, 0.25], dtype=np.float32)
+    planes = np.full((m + 1, 3), 777.0, dtype=np.float32)  # garbage above the defined orders
+    O.update_segment(O.F32, m, basis, 0, [], 8.0, f0, planes)
+    out = np.zeros(3, dtype=np.float32)
+    O.forecast_segment(O.F32, m, basis, 1, [8.0], 5.0, planes, out)
+    assert np.array_equal(out, f0)
+    O.update_segment(O.F32, m, basis, 1, [8.0], 6.0, f1, planes)
+    O.forecast_segment(O.F32, m, basis, 2, [6.0, 8.0], 5.0, planes, out)
+    assert out.tolist() == (f1 + (f1 - f0) / (6.0 - 8.0) * (5.0 - 6.0)).tolist()
+    if m >= 2:
+        assert np.all(planes[2] == 777.0)  # never written, never read
+
+
+@pytest.mark.parametrize("basis", [O.TAYLOR, O.NEWTON])
+@pytest.mark.parametrize("m", [1, 2, 3, 4])
+def test_exact_for_degree_one_at_any_gaps(basis, m):
+    rng = np.random.default_rng(5)
+    a0 = rng.integers(-20, 21, size=11).astype(np.float64)
+    a1 = rng.integers(-20, 21, size=11).astype(np.float64)
+    times = [4.0, 3.5, 3.375, 2.0, 1.75, 1.0]  # dyadic, uneven
+    feats = [(a0 + a1 * t).astype(np.float32) for t in times]
+    planes, hist = run_history(O.F32, m, basis, times, feats)
+    for tt in [0.5, 0.0, 1.0, 3.0, -2.25]:
+        out = np.zeros(11, dtype=np.float32)
+        O.forecast_segment(O.F32, m, basis, len(times), hist, tt, planes, out)
+        assert np.array_equal(out.astype(np.float64), a0 + a1 * tt), tt
+
+
+@pytest.mark.parametrize("m", [2, 3])
+def test_taylor_basis_quadratic_residual_closed_form(m):
+    """For f = a0 + a1 s + a2 s^2 and equal gaps g between the last references, backward
+    difference quotients give D1 = f'(t) - a2 g, D2 = f''(t), so the printed forecast misses
+    the truth by exactly -a2 * g * x (x = t_target - t_last)."""
+    a0, a1, a2 = 3.0, -2.0, 5.0
+    g = -0.25
+    t_last = 2.0
+    times = [t_last - j * g for j in range(m, -1, -1)]
+    feats = [np.array([a0 + a1 * t + a2 * t * t], dtype=np.float32) for t in times]
+    planes, hist = run_history(O.F32, m, O.TAYLOR, times, feats)
+    for x in [-0.25, -0.5, -1.0, 0.125]:
+        out = np.zeros(1, dtype=np.float32)
+        O.forecast_segment(O.F32, m, O.TAYLOR, m + 1, hist, t_last + x, planes, out)
+        tt = t_last + x
+        truth = a0 + a1 * tt + a2 * tt * tt
+        assert out[0] - truth == pytest.approx(-a2 * g * x, abs=1e-5)
+    # the residual shrinks linearly with the reference gap
+    res = []
+    for gg in [-0.5, -0.25, -0.125]:
+        ts = [t_last - j * gg for j in range(m, -1, -1)]
+        fs = [np.array([a0 + a1 * t + a2 * t * t], dtype=np.float32) for t in ts]
+        pl, hi = run_history(O.F32, m, O.TAYLOR, ts, fs)
+        out = np.zeros(1, dtype=np.float32)
+        O.forecast_segment(O.F32, m, O.TAYLOR, m + 1, hi, t_last - 0.5, pl, out)
+        tt = t_last - 0.5
+        res.append(float(out[0]) - (a0 + a1 * tt + a2 * tt * tt))
+    assert res[0] == pytest.approx(2 * res[1], rel=1e-4) and res[1] == pytest.approx(2 * res[2], rel=1e-4)
+
+
+@pytest.mark.parametrize("m", [1, 2, 3, 4])
+def test_newton_basis_exact_for_degree_m_at_any_gaps(m):
+    rng = np.random.default_rng(m)
+    coef = rng.integers(-4, 5, size=(m + 1, 9)).astype(np.float64)
+    times = [3.0, 2.5, 2.25, 1.5, 1.0, 0.875][: m + 2]
+
+    def poly(t):
+        return sum(coef[i] * t ** i for i in range(m + 1))
+
+    feats = [poly(t).astype(np.float32) for t in times]
+    planes, hist = run_history(O.F32, m, O.NEWTON, times, feats)
+    for tt in [0.5, 0.25, 0.0, 2.0]:
+        out = np.zeros(9, dtype=np.float32)
+        O.forecast_segment(O.F32, m, O.NEWTON, len(times), hist, tt, planes, out)
+        np.testing.assert_allclose(out.astype(np.float64), poly(tt), rtol=2e-6, atol=2e-5)
+
+
+@pytest.mark.parametrize("m", [1, 2, 3])
+def test_newton_basis_equals_lagrange_interpolation_in_rationals(m):
+    """The Newton-form forecast is the unique polynomial of degree <= m through the last m+1
+    references: compare with Lagrange's formula evaluated in exact rationals."""
+    rng = np.random.default_rng(17 + m)
+    times = [Fraction(8), Fraction(7), Fraction(11, 2), Fraction(5), Fraction(17, 4)][: m + 2]
+    raw = [rng.integers(-30, 31, size=5) for _ in times]
+    planes, hist = run_history(O.F32, m, O.NEWTON, [float(t) for t in times],
+                               [r.astype(np.float32) for r in raw])
+    nodes = times[-(m + 1):]
+    vals = raw[-(m + 1):]
+    for tt in [Fraction(4), Fraction(7, 2), Fraction(0)]:
+        out = np.zeros(5, dtype=np.float32)
+        O.forecast_segment(O.F32, m, O.NEWTON, len(times), hist, float(tt), planes, out)
+        for e in range(5):
+            want = Fraction(0)
+            for a, ta in enumerate(nodes):
+                w = Fraction(int(vals[a][e]))
+                for c, tc in enumerate(nodes):
+                    if c != a:
+                        w *= (tt - tc) / (ta - tc)
+                want += w
+            assert float(out[e]) == pytest.approx(float(want), rel=1e-5, abs=1e-4)
+
+
+def test_bases_coincide_up_to_order_one():
+    rng = np.random.default_rng(3)
+    times = [1.0, 0.9, 0.75]
+    feats = [rng.standard_normal(64).astype(np.float32) for _ in times]
+    pt, ht = run_history(O.F32, 1, O.TAYLOR, times, feats)
+    pn, hn = run_history(O.F32, 1, O.NEWTON, times, feats)
+    assert np.array_equal(pt, pn)
+    a, b = np.zeros(64, np.float32), np.zeros(64, np.float32)
+    O.forecast_segment(O.F32, 1, O.TAYLOR, 3, ht, 0.6, pt, a)
+    O.forecast_segment(O.F32, 1, O.NEWTON, 3, hn, 0.6, pn, b)
+    assert np.array_equal(a, b)
+
+
+@pytest.mark.parametrize("basis", [O.TAYLOR, O.NEWTON])
+@pytest.mark.parametrize("dtype", [O.F32, O.BF16])
+def test_forecast_at_the_reference_time_returns_the_feature(basis, dtype):
+    g = torch.Generator().manual_seed(9)
+    m = 3
+    times = [1.0, 0.8, 0.7, 0.65]
+    feats = []
+    for _ in times:
+        x = torch.randn(257, generator=g)
+        feats.append(bf16_bits(x) if dtype == O.BF16 else x.numpy().copy())
+    planes, hist = run_history(dtype, m, basis, times, feats)
+    out = np.zeros_like(feats[0])
+    O.forecast_segment(dtype, m, basis, 4, hist, times[-1], planes, out)
+    assert np.array_equal(out, feats[-1])
+
+
+def test_zero_gap_is_refused_and_leaves_table_untouched():
+    f = np.arange(8, dtype=np.float32)
+    planes = np.zeros((3, 8), dtype=np.float32)
+    O.update_segment(O.F32, 2, O.TAYLOR, 0, [], 1.0, f, planes)
+    before = planes.copy()
+    with pytest.raises(ZeroDivisionError):
+        O.update_segment(O.F32, 2, O.TAYLOR, 1, [1.0], 1.0, f + 1, planes)
+    assert np.array_equal(planes, before)
+    with pytest.raises(RuntimeError):
+        O.forecast_segment(O.F32, 2, O.TAYLOR, 0, [], 1.0, planes, np.zeros(8, np.float32))
+
+
+# ---------------------------------------------------------------------------------------------
+# storage rounding: bfloat16 round-to-nearest-even against torch's conversion
+# ---------------------------------------------------------------------------------------------
+
+def test_bf16_rounding_matches_library_conversion():
+    g = torch.Generator().manual_seed(4)
+    x = torch.cat([
+        torch.randn(20000, generator=g) * torch.exp(torch.randn(20000, generator=g) * 8),
+        torch.tensor([0.0, -0.0, 1.0, -1.0, 1.00390625, 1.01171875, 1.005859375, 3.3895314e38, -3.4e38,
+                      1e-40, -1e-40, 9.1835e-41, 4.6e-41, 1.17549435e-38, float("inf"), float("-inf")]),
+    ]).to(torch.float32)
+    want = bf16_bits(x)
+    got = np.array([O.to_bf16_bits(float(v)) for v in x.tolist()], dtype=np.uint16)
+    assert np.array_equal(got, want)
+    # exact ties go to even: 1 + 2^-8 is halfway between 1 and 1 + 2^-7
+    assert O.to_bf16_bits(1.0 + 2.0 ** -8) == 0x3F80
+    assert O.to_bf16_bits(1.0 + 3 * 2.0 ** -8) == 0x3F82
+    # a double just above the tie rounds up although its float32 rounding would be the tie itself
+    assert O.to_bf16_bits(1.0 + 2.0 ** -8 + 2.0 ** -40) == 0x3F81
+    assert O.to_bf16_bits(float("nan")) & 0x7FFF > 0x7F80
+
+
+def test_bf16_tables_round_once_per_stored_plane():
+    """The difference chain runs on unrounded values: plane 2 is the rounding of the exact
+    second quotient, not of a quotient of rounded first quotients."""
+    vals = [1.0, 1.0 + 2.0 ** -7, 1.0 + 3 * 2.0 ** -6]  # bf16-exact features
+    feats = [np.array([O.to_bf16_bits(v)], dtype=np.uint16) for v in vals]
+    times = [3.0, 2.0, 1.0]
+    planes, _ = run_history(O.BF16, 2, O.TAYLOR, times, feats)
+    d1_old = Fraction(vals[1]) - Fraction(vals[0])
+    d1_new = (Fraction(vals[2]) - Fraction(vals[1])) / Fraction(-1)
+    # at the second update the old plane 1 was stored rounded; the new plane 1 is used unrounded
+    d1_old_stored = Fraction(float(bits_to_f64(np.array([O.to_bf16_bits(float(d1_old / -1))], np.uint16))[0]))
+    d2 = (d1_new - d1_old_stored) / Fraction(-1)
+    assert int(planes[2, 0]) == O.to_bf16_bits(float(d2))
+    assert int(planes[1, 0]) == O.to_bf16_bits(float(d1_new))
+    assert int(planes[0, 0]) == O.to_bf16_bits(vals[2])
+
+
+# ---------------------------------------------------------------------------------------------
+# Eq. 4 and the accept rule
+# ---------------------------------------------------------------------------------------------
+
+def test_relative_error_hand_examples():
+    f = np.array([5.0, 12.0], dtype=np.float32)       # norm 13
+    p = f + np.array([3.0, 4.0], dtype=np.float32)    # difference norm 5
+    assert O.rel_l2(O.F32, p, f) == pytest.approx(5.0 / (13.0 + 1e-8), rel=1e-15)
+    assert O.rel_l2(O.F32, f, f) == 0.0
+    z = np.zeros(2, dtype=np.float32)
+    assert O.rel_l2(O.F32, z, f) == pytest.approx(13.0 / (13.0 + 1e-8), rel=1e-15)
+    assert O.rel_l2(O.F32, p - f, z) == pytest.approx(5.0 / 1e-8, rel=1e-12)  # zero feature: only eps
+    assert O.rel_l2(O.F32, z, z) == 0.0
+    assert O.rel_l2(O.F32, p, f, eps=1.0) == pytest.approx(5.0 / 14.0, rel=1e-15)
+
+
+def test_relative_error_properties():
+    g = torch.Generator().manual_seed(11)
+    f = torch.randn(5000, generator=g).numpy()
+    p = (torch.randn(5000, generator=g) * 0.1).numpy() + f
+    e = O.rel_l2(O.F32, p, f)
+    assert O.rel_l2(O.F32, (4 * p).astype(np.float32), (4 * f).astype(np.float32)) == pytest.approx(e, rel=1e-7)
+    delta = 2.0 ** -3
+    fs = torch.from_numpy(f).to(torch.bfloat16).to(torch.float32).numpy()  # 8 significant bits
+    pf = (fs * np.float32(1 + delta)).astype(np.float32)  # so that (1 + 2^-3) * f is exact in binary32
+    nf = math.sqrt(math.fsum(float(v) ** 2 for v in fs))
+    assert O.rel_l2(O.F32, pf, fs) == pytest.approx(delta * nf / (nf + 1e-8), rel=1e-12)
+    # sensitive to which operand is the denominator
+    assert O.rel_l2(O.F32, f, p) != pytest.approx(e, rel=1e-6)
+
+
+@pytest.mark.parametrize("dtype", [O.F32, O.BF16])
+def test_relative_error_brute_force_in_rationals(dtype):
+    g = torch.Generator().manual_seed(21)
+    for n in [1, 2, 7, 16]:
+        a, b = torch.randn(n, generator=g), torch.randn(n, generator=g)
+        if dtype == O.BF16:
+            p, f = bf16_bits(a), bf16_bits(b)
+            pv, fv = bits_to_f64(p), bits_to_f64(f)
+        else:
+            p, f = a.numpy().copy(), b.numpy().copy()
+            pv, fv = p.astype(np.float64), f.astype(np.float64)
+        num = sum((Fraction(float(x)) - Fraction(float(y))) ** 2 for x, y in zip(pv, fv))
+        den = sum(Fraction(float(y)) ** 2 for y in fv)
+        want = math.sqrt(num) / (math.sqrt(den) + 1e-8)
+        assert O.rel_l2(dtype, p, f) == pytest.approx(want, rel=1e-13)
+
+
+def test_accept_rule():
+    assert O.accept(0.5, 0.5)            # equality accepts
+    assert O.accept(0.0, 0.0)
+    assert not O.accept(math.nextafter(0.5, 1.0), 0.5)
+    assert O.accept(math.nextafter(0.5, 0.0), 0.5)
+    assert not O.accept(float("nan"), 0.5)
+    assert not O.accept(float("inf"), 1e30)
+    f = np.array([1.0, float("nan")], dtype=np.float32)
+    assert not O.accept(O.rel_l2(O.F32, f, f), 10.0)  # NaN anywhere rejects, even p == f
+
+
+def test_threshold_schedule():
+    assert O.tau_schedule(0.3, 0.5, 50, 50) == pytest.approx(0.3, rel=1e-15)       # t = T
+    assert O.tau_schedule(0.3, 0.5, 0, 50) == pytest.approx(0.15, rel=1e-15)       # t = 0
+    assert O.tau_schedule(0.1, 0.2, 25, 50) == pytest.approx(0.1 * math.sqrt(0.2), rel=1e-15)
+    ts = [O.tau_schedule(0.1, 0.2, t, 50) for t in range(50, -1, -1)]
+    assert all(a > b for a, b in zip(ts, ts[1:]))  # decays as t runs down
+    assert ts[0] == pytest.approx(0.1) and ts[-1] == pytest.approx(0.02)
+
+
+def test_speedup_matches_the_papers_worked_example():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "speedup_example.txt")) if l.strip() and l[0] != "#"]
+    assert len(rows) == 2
+    for alpha, gamma, denom, s, nd in rows:
+        alpha, gamma, denom, s, nd = float(alpha), float(gamma), float(denom), float(s), int(nd)
+        got = O.speedup(alpha, gamma)
+        assert 1.0 / got == pytest.approx(denom, rel=1e-12)
+        assert round(got, nd) == pytest.approx(s)
+
+
+def test_block_counts_match_printed_verification_ratios():
+    from paper_2509_11628_b200 import workloads as W
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "gamma_blocks.txt")) if l.strip() and l[0] != "#"]
+    for name, gamma, blocks in rows:
+        gamma, blocks = float(gamma), int(blocks)
+        assert 1.0 / blocks == pytest.approx(gamma, rel=0.03)
+        w = W.BY_NAME[name]()
+        if name == "dit_xl2":
+            assert len(w.entries) == 2 * blocks
+        else:
+            duals = sum(1 for l in w.labels if l.endswith(".main"))
+            singles = sum(1 for l in w.labels if l.startswith("S"))
+            assert duals + singles == blocks
+
+
+# ---------------------------------------------------------------------------------------------
+# per-sample continuation
+# ---------------------------------------------------------------------------------------------
+
+def test_select_adaptive_hand_cases():
+    # accept continues, reject stops, inactive stays inactive and is not counted
+    act, cnt, idx = O.select_adaptive([1, 0, 1, 1], 5, 1, [0, 0, 2, 0], [1, 1, 1, 0])
+    assert act == [1, 0, 1, 0] and cnt == [1, 0, 3, 0] and idx == [0, 2]
+    # the forced activation period caps consecutive speculative steps
+    act, cnt, idx = O.select_adaptive([1, 1], 3, 1, [1, 2], [1, 1])
+    assert act == [1, 0] and cnt == [2, 3] and idx == [0]
+    # a guidance pair shares its fate
+    act, cnt, idx = O.select_adaptive([1, 0, 1, 1], 9, 2, [0, 0, 0, 0], [1, 1, 1, 1])
+    assert act == [0, 0, 1, 1] and cnt == [1, 0, 1, 1] and idx == [2, 3]
+    # sequential validation: once rejected, later accepts do not revive the sample
+    act = [1]
+    cnt = [0]
+    trace = []
+    for a in [1, 1, 0, 1, 1]:
+        act, cnt, _ = O.select_adaptive([a], 99, 1, cnt, act)
+        trace.append(act[0])
+    assert trace == [1, 1, 0, 0, 0] and cnt == [2]
+
+
+# ---------------------------------------------------------------------------------------------
+# stateful wrapper: masks and per-sample histories
+# ---------------------------------------------------------------------------------------------
+
+def test_cache_masks_and_per_sample_history():
+    rng = np.random.default_rng(8)
+    B, m, n = 3, 2, 50
+    c = O.OracleCache([n, n], B, m, O.F32)
+    feats = lambda: [rng.standard_normal((B, n)).astype(np.float32) for _ in range(2)]
+    f0 = feats()
+    c.update(f0, [1.0, 1.0, 1.0]); c.commit_step()
+    f1 = feats()
+    c.update(f1, [0.9, 0.8, 0.9], mask=[1, 1, 0]); c.commit_step()
+    assert c.n_refs == [2, 2, 1]
+    assert c.t_hist[2] == [1.0] and c.t_hist[1] == [0.8, 1.0]
+    # sample 2 was masked out: its table still holds the first feature only
+    assert np.array_equal(c.planes[0][2, 0], f0[0][2])
+    out = c.forecast_entry(1, [0.7, 0.7, 0.7])
+    assert np.array_equal(out[2], f0[1][2])  # one reference: reuse
+    want1 = f1[1][1] + (f1[1][1].astype(np.float64) - f0[1][1]) / (0.8 - 1.0) * (0.7 - 0.8)
+    np.testing.assert_allclose(out[1], want1, rtol=1e-6, atol=1e-6)
+    # inactive samples are left alone by forecast and verify
+    sentinel = np.full((B, n), 42.0, dtype=np.float32)
+    out2 = c.forecast_entry(0, [0.7] * 3, active=[0, 1, 0], out=sentinel.copy())
+    assert np.all(out2[0] == 42.0) and np.all(out2[2] == 42.0) and not np.all(out2[1] == 42.0)
+    err, acc, pred = c.verify(c.forecast_entry(1, [0.7] * 3), [0.7] * 3, [0.1] * 3, active=[1, 0, 1])
+    assert err[0] == 0.0 and acc[0] == 1 and np.isnan(err[1]) and acc[1] == -1 and acc[2] == 1
+    c.reset([0, 1, 0])
+    assert c.n_refs == [2, 0, 1]
