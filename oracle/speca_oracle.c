@@ -25,6 +25,14 @@
  *
  * Storage types: 0 = IEEE binary32, 1 = bfloat16 (upper 16 bits of binary32, round to nearest
  * even on store, NaN kept NaN).
+ *
+ * Precision. Each formula is evaluated in double. The method's stated precision is "fp32
+ * accumulation, bf16 storage": the value that is quantised to the storage type is a binary32
+ * register. A stored result is therefore rounded double -> binary32 -> storage type, both to
+ * nearest even, so that the quantisation decision is taken in the kernel's precision. (Cached
+ * features have 8-bit significands and reciprocal gaps like 50 have few bits, so exact bfloat16
+ * ties are common in the difference quotients; rounding the double directly would break them by
+ * the 1e-16 representation error of the gap instead of by the ties-to-even rule.)
  */
 #include <math.h>
 #include <stdint.h>
@@ -70,10 +78,11 @@ static double load_elem(const void* p, int dtype, int64_t i) {
 }
 
 static void store_elem(void* p, int dtype, int64_t i, double v) {
+    float r = (float)v; /* the binary32 register that holds the result */
     if (dtype == ORACLE_F32)
-        ((float*)p)[i] = (float)v;
+        ((float*)p)[i] = r;
     else
-        ((uint16_t*)p)[i] = oracle_double_to_bf16_bits(v);
+        ((uint16_t*)p)[i] = oracle_double_to_bf16_bits((double)r);
 }
 
 /* ---- Eq. 3: table rewrite at a reference step ---------------------------------------------- */

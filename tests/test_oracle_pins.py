@@ -283,6 +283,21 @@ def test_bf16_rounding_matches_library_conversion():
     assert O.to_bf16_bits(float("nan")) & 0x7FFF > 0x7F80
 
 
+def test_stored_value_is_quantised_from_a_binary32_register():
+    """fp32 accumulation, bf16 storage: c - d = 11 and gap = 0.98 - 1.0 (not exactly -0.02) give a
+    quotient a hair below 550 in magnitude. 550 needs 9 significant bits, so it is an exact bfloat16
+    tie between 548 and 552; held in a binary32 register it IS 550 and ties-to-even gives 552.
+    Rounding the double directly would give 548."""
+    f0 = np.array([O.to_bf16_bits(0.0)], dtype=np.uint16)
+    f1 = np.array([O.to_bf16_bits(11.0)], dtype=np.uint16)
+    planes, _ = run_history(O.BF16, 1, O.TAYLOR, [1.0, 0.98], [f0, f1])
+    assert (0.98 - 1.0) != -0.02 and abs(11.0 / (0.98 - 1.0)) < 550.0
+    assert float(bits_to_f64(planes[1])[0]) == -552.0
+    # fp32 storage keeps the binary32 value itself
+    pf, _ = run_history(O.F32, 1, O.TAYLOR, [1.0, 0.98], [np.zeros(1, np.float32), np.full(1, 11.0, np.float32)])
+    assert float(pf[1, 0]) == float(np.float32(11.0 / (0.98 - 1.0))) == -550.0
+
+
 def test_bf16_tables_round_once_per_stored_plane():
     """The difference chain runs on unrounded values: plane 2 is the rounding of the exact
     second quotient, not of a quotient of rounded first quotients."""
