@@ -1,0 +1,315 @@
+"""ctypes binding of ``libspeca.so``: the same entry points as ``include/speca.h``.
+
+Argument marshalling only -- every arithmetic step runs in the CUDA kernels behind the C ABI.
+Device buffers are torch tensors (or raw integer addresses); host arrays are Python sequences.
+There is no fallback: if the library is missing or cannot be loaded, importing the entry points
+raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libspeca.so")
+
+SPECA_OK = 0
+SPECA_ERR_INVALID_ARG, SPECA_ERR_SHAPE, SPECA_ERR_ALIGNMENT, SPECA_ERR_STATE = 1, 2, 3, 4
+SPECA_ERR_ZERO_GAP, SPECA_ERR_NOMEM, SPECA_ERR_CUDA, SPECA_ERR_UNSUPPORTED = 5, 6, 7, 8
+SPECA_F32, SPECA_BF16 = 0, 1
+SPECA_BASIS_TAYLOR, SPECA_BASIS_NEWTON = 0, 1
+SPECA_PATH_AUTO, SPECA_PATH_DIRECT, SPECA_PATH_BULK = 0, 1, 2
+SPECA_MAX_ORDER, SPECA_MAX_BATCH, SPECA_MAX_ENTRIES = 4, 64, 512
+
+EXPORTS = [
+    "speca_cache_arena_bytes", "speca_cache_create", "speca_cache_destroy", "speca_cache_reset",
+    "speca_cache_update", "speca_cache_commit_step", "speca_forecast", "speca_verify",
+    "speca_select_adaptive", "speca_activate", "speca_tau", "speca_cache_state", "speca_cache_plane",
+    "speca_cache_launch_count", "speca_status_string", "speca_last_error", "speca_version",
+]
+
+
+class SpecaError(RuntimeError):
+    def __init__(self, status: int, detail: str = ""):
+        self.status = status
+        name = _lib().speca_status_string(status).decode()
+        super().__init__("speca status %d (%s)%s" % (status, name, (": " + detail) if detail else ""))
+
+
+class EntryDesc(ctypes.Structure):
+    _fields_ = [("tokens", ctypes.c_int64), ("dim", ctypes.c_int32)]
+
+
+class CacheConfig(ctypes.Structure):
+    _fields_ = [
+        ("n_entries", ctypes.c_int32), ("entries", ctypes.POINTER(EntryDesc)), ("batch", ctypes.c_int32),
+        ("max_order", ctypes.c_int32), ("dtype", ctypes.c_int32), ("basis", ctypes.c_int32),
+        ("verify_entry", ctypes.c_int32), ("eps", ctypes.c_float), ("arena", ctypes.c_void_p),
+        ("arena_bytes", ctypes.c_size_t), ("device", ctypes.c_int32), ("path", ctypes.c_int32),
+    ]
+
+
+_LIB = None
+
+
+def _lib() -> ctypes.CDLL:
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            "libspeca.so is not built (%s). Run `python -m paper_2509_11628_b200.build`; "
+            "there is no CPU fallback." % LIB_PATH)
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, dbl = ctypes.c_void_p, ctypes.c_int32, ctypes.c_double
+    cfgp = ctypes.POINTER(CacheConfig)
+    L.speca_cache_arena_bytes.argtypes = [cfgp, ctypes.POINTER(ctypes.c_size_t)]
+    L.speca_cache_create.argtypes = [cfgp, ctypes.POINTER(vp)]
+    L.speca_cache_destroy.argtypes = [vp]
+    L.speca_cache_reset.argtypes = [vp, vp]
+    L.speca_cache_update.argtypes = [vp, vp, vp, vp, vp]
+    L.speca_cache_commit_step.argtypes = [vp]
+    L.speca_forecast.argtypes = [vp, vp, vp, vp, vp]
+    L.speca_verify.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.speca_select_adaptive.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, vp]
+    L.speca_activate.argtypes = [vp, vp, vp, vp, vp]
+    L.speca_tau.argtypes = [dbl, dbl, dbl, dbl]
+    L.speca_tau.restype = dbl
+    L.speca_cache_state.argtypes = [vp, vp, vp]
+    L.speca_cache_plane.argtypes = [vp, i32, i32, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_size_t)]
+    L.speca_cache_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64)]
+    L.speca_status_string.argtypes = [i32]
+    L.speca_status_string.restype = ctypes.c_char_p
+    L.speca_last_error.argtypes = [vp]
+    L.speca_last_error.restype = ctypes.c_char_p
+    L.speca_version.restype = ctypes.c_char_p
+    for name in EXPORTS:
+        if getattr(L, name).restype is ctypes.c_int:  # default restype: status codes
+            getattr(L, name).restype = i32
+    _LIB = L
+    return L
+
+
+# ---- marshalling helpers -------------------------------------------------------------------------
+
+def _dev_ptr(x) -> Optional[int]:
+    """torch CUDA tensor / int address / None -> integer address or None."""
+    if x is None:
+        return None
+    if isinstance(x, torch.Tensor):
+        if not x.is_cuda:
+            raise TypeError("device buffer expected, got a CPU tensor")
+        if not x.is_contiguous():
+            raise TypeError("device buffers must be contiguous")
+        return x.data_ptr()
+    return int(x)
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream or None
+    if isinstance(stream, torch.cuda.Stream):
+        return stream.cuda_stream or None
+    return int(stream) or None
+
+
+def _doubles(xs: Sequence[float]):
+    return (ctypes.c_double * len(xs))(*[float(x) for x in xs])
+
+
+def _floats(xs: Sequence[float]):
+    return (ctypes.c_float * len(xs))(*[float(x) for x in xs])
+
+
+def _bytes(xs: Optional[Sequence[int]]):
+    if xs is None:
+        return None
+    return (ctypes.c_uint8 * len(xs))(*[1 if x else 0 for x in xs])
+
+
+def _ptr_array(xs: Sequence):
+    return (ctypes.c_void_p * len(xs))(*[_dev_ptr(x) for x in xs])
+
+
+def _check(status: int, handle=None):
+    if status != SPECA_OK:
+        detail = _lib().speca_last_error(handle).decode() if handle else ""
+        raise SpecaError(status, detail)
+
+
+def _config(entries, batch, max_order, dtype, basis, verify_entry, eps, arena, arena_bytes, device, path):
+    arr = (EntryDesc * len(entries))(*[EntryDesc(int(n), int(d)) for n, d in entries])
+    cfg = CacheConfig(len(entries), arr, batch, max_order, dtype, basis, verify_entry, eps,
+                      _dev_ptr(arena), arena_bytes, device, path)
+    cfg._keep = arr
+    return cfg
+
+
+# ---- the entry points, same names as the header ----------------------------------------------------
+
+def speca_cache_arena_bytes(entries, batch, max_order, dtype, basis=SPECA_BASIS_TAYLOR, verify_entry=-1,
+                            path=SPECA_PATH_AUTO) -> int:
+    cfg = _config(entries, batch, max_order, dtype, basis, verify_entry, 0.0, None, 0, 0, path)
+    out = ctypes.c_size_t(0)
+    _check(_lib().speca_cache_arena_bytes(ctypes.byref(cfg), ctypes.byref(out)))
+    return out.value
+
+
+def speca_cache_create(entries, batch, max_order, dtype, arena, basis=SPECA_BASIS_TAYLOR, verify_entry=-1,
+                       eps=0.0, device=None, path=SPECA_PATH_AUTO, arena_bytes=None) -> int:
+    """Returns the opaque handle (an integer address). ``arena`` is a CUDA uint8 tensor the caller
+    keeps alive, or a raw device address together with ``arena_bytes``."""
+    if isinstance(arena, torch.Tensor):
+        if device is None:
+            device = arena.device.index
+        if arena_bytes is None:
+            arena_bytes = arena.numel() * arena.element_size()
+    cfg = _config(entries, batch, max_order, dtype, basis, verify_entry, eps, arena, arena_bytes or 0,
+                  device or 0, path)
+    out = ctypes.c_void_p(None)
+    _check(_lib().speca_cache_create(ctypes.byref(cfg), ctypes.byref(out)))
+    return out.value
+
+
+def speca_cache_destroy(cache) -> None:
+    _check(_lib().speca_cache_destroy(cache))
+
+
+def speca_cache_reset(cache, host_sample_mask=None) -> None:
+    _check(_lib().speca_cache_reset(cache, _bytes(host_sample_mask)), cache)
+
+
+def speca_cache_update(cache, feats, t_ref, host_sample_mask=None, stream=None) -> None:
+    _check(_lib().speca_cache_update(cache, _ptr_array(feats), _doubles(t_ref), _bytes(host_sample_mask),
+                                     _stream_ptr(stream)), cache)
+
+
+def speca_cache_commit_step(cache) -> None:
+    _check(_lib().speca_cache_commit_step(cache), cache)
+
+
+def speca_forecast(cache, t_target, dev_active_mask, outs, stream=None) -> None:
+    _check(_lib().speca_forecast(cache, _doubles(t_target), _dev_ptr(dev_active_mask), _ptr_array(outs),
+                                 _stream_ptr(stream)), cache)
+
+
+def speca_verify(cache, fresh, t_target, tau, dev_active_mask, out_pred, dev_err, dev_accept, stream=None) -> None:
+    _check(_lib().speca_verify(cache, _dev_ptr(fresh), _doubles(t_target), _floats(tau), _dev_ptr(dev_active_mask),
+                               _dev_ptr(out_pred), _dev_ptr(dev_err), _dev_ptr(dev_accept), _stream_ptr(stream)),
+           cache)
+
+
+def speca_select_adaptive(cache, dev_accept, k_max, group, dev_spec_count, dev_active_mask, dev_active_idx=None,
+                          dev_n_active=None, stream=None) -> None:
+    _check(_lib().speca_select_adaptive(cache, _dev_ptr(dev_accept), int(k_max), int(group), _dev_ptr(dev_spec_count),
+                                        _dev_ptr(dev_active_mask), _dev_ptr(dev_active_idx), _dev_ptr(dev_n_active),
+                                        _stream_ptr(stream)), cache)
+
+
+def speca_activate(cache, host_sample_mask, dev_spec_count, dev_active_mask, stream=None) -> None:
+    _check(_lib().speca_activate(cache, _bytes(host_sample_mask), _dev_ptr(dev_spec_count), _dev_ptr(dev_active_mask),
+                                 _stream_ptr(stream)), cache)
+
+
+def speca_tau(tau0: float, beta: float, t: float, T: float) -> float:
+    return float(_lib().speca_tau(tau0, beta, t, T))
+
+
+def speca_cache_state(cache, batch: int):
+    n = (ctypes.c_int32 * batch)()
+    t = (ctypes.c_double * batch)()
+    _check(_lib().speca_cache_state(cache, n, t), cache)
+    return list(n), list(t)
+
+
+def speca_cache_plane(cache, entry: int, sample: int):
+    p = ctypes.c_void_p(None)
+    s = ctypes.c_size_t(0)
+    _check(_lib().speca_cache_plane(cache, entry, sample, ctypes.byref(p), ctypes.byref(s)), cache)
+    return p.value, s.value
+
+
+def speca_cache_launch_count(cache) -> int:
+    n = ctypes.c_uint64(0)
+    _check(_lib().speca_cache_launch_count(cache, ctypes.byref(n)), cache)
+    return n.value
+
+
+def speca_status_string(status: int) -> str:
+    return _lib().speca_status_string(status).decode()
+
+
+def speca_last_error(cache) -> str:
+    return _lib().speca_last_error(cache).decode()
+
+
+def speca_version() -> str:
+    return _lib().speca_version().decode()
+
+
+class SpecaCache:
+    """Owns an arena tensor and a handle; forwards to the entry points above."""
+
+    def __init__(self, entries, batch, max_order, dtype, device="cuda:0", basis=SPECA_BASIS_TAYLOR,
+                 verify_entry=-1, eps=0.0, path=SPECA_PATH_AUTO):
+        self.entries = [(int(n), int(d)) for n, d in entries]
+        self.batch, self.max_order, self.dtype, self.basis = batch, max_order, dtype, basis
+        self.device = torch.device(device)
+        self.verify_entry = verify_entry if verify_entry >= 0 else len(self.entries) - 1
+        nbytes = speca_cache_arena_bytes(self.entries, batch, max_order, dtype, basis, verify_entry, path)
+        self.arena = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        assert self.arena.data_ptr() % 256 == 0
+        self.handle = speca_cache_create(self.entries, batch, max_order, dtype, self.arena, basis, verify_entry,
+                                         eps, self.device.index or 0, path)
+
+    def close(self):
+        if self.handle:
+            speca_cache_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def update(self, feats, t_ref, mask=None, stream=None):
+        speca_cache_update(self.handle, feats, t_ref, mask, stream)
+
+    def commit_step(self):
+        speca_cache_commit_step(self.handle)
+
+    def forecast(self, t_target, outs, active=None, stream=None):
+        speca_forecast(self.handle, t_target, active, outs, stream)
+
+    def verify(self, fresh, t_target, tau, err, accept, active=None, out_pred=None, stream=None):
+        speca_verify(self.handle, fresh, t_target, tau, active, out_pred, err, accept, stream)
+
+    def select_adaptive(self, accept, k_max, group, spec_count, active, idx=None, n_active=None, stream=None):
+        speca_select_adaptive(self.handle, accept, k_max, group, spec_count, active, idx, n_active, stream)
+
+    def activate(self, mask, spec_count, active, stream=None):
+        speca_activate(self.handle, mask, spec_count, active, stream)
+
+    def reset(self, mask=None):
+        speca_cache_reset(self.handle, mask)
+
+    def state(self):
+        return speca_cache_state(self.handle, self.batch)
+
+    def plane_tensor(self, entry: int, sample: int) -> torch.Tensor:
+        """View of the (entry, sample) table as ``[m+1, n_elems]`` in the storage dtype."""
+        ptr, stride = speca_cache_plane(self.handle, entry, sample)
+        esz = 2 if self.dtype == SPECA_BF16 else 4
+        tdt = torch.bfloat16 if self.dtype == SPECA_BF16 else torch.float32
+        n = self.entries[entry][0] * self.entries[entry][1]
+        off = ptr - self.arena.data_ptr()
+        raw = self.arena[off: off + stride * (self.max_order + 1)].view(tdt).view(self.max_order + 1, stride // esz)
+        return raw[:, :n]
+
+    @property
+    def launches(self) -> int:
+        return speca_cache_launch_count(self.handle)

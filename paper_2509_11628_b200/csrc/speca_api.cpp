@@ -1,0 +1,573 @@
+// Host side of the C ABI declared in speca.h: handle, arena layout, per-sample reference
+// history, the host-computed scalars of Eq. 2-3, argument checks and kernel launches.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <limits>
+#include <new>
+#include <vector>
+
+#include "speca_internal.h"
+
+using namespace speca;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Layout {
+    size_t segs_off, tiles_direct_off, tiles_bulk_off, partials_off, ticket_off, tables_off, total;
+    std::vector<SegDesc> segs;
+    std::vector<uint32_t> tiles_direct, tiles_bulk;
+};
+
+// Shape checks and arena layout shared by speca_cache_arena_bytes and speca_cache_create.
+speca_status_t make_layout(const speca_cache_config_t* cfg, Layout* L) {
+    if (cfg == nullptr || cfg->entries == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (cfg->n_entries < 1 || cfg->n_entries > SPECA_MAX_ENTRIES) return SPECA_ERR_SHAPE;
+    if (cfg->batch < 1 || cfg->batch > SPECA_MAX_BATCH) return SPECA_ERR_SHAPE;
+    if (cfg->max_order < 0 || cfg->max_order > SPECA_MAX_ORDER) return SPECA_ERR_SHAPE;
+    if (cfg->dtype != SPECA_F32 && cfg->dtype != SPECA_BF16) return SPECA_ERR_INVALID_ARG;
+    if (cfg->basis != SPECA_BASIS_TAYLOR && cfg->basis != SPECA_BASIS_NEWTON) return SPECA_ERR_INVALID_ARG;
+    if (cfg->path != SPECA_PATH_AUTO && cfg->path != SPECA_PATH_DIRECT && cfg->path != SPECA_PATH_BULK)
+        return SPECA_ERR_INVALID_ARG;
+    if (cfg->verify_entry < -1 || cfg->verify_entry >= cfg->n_entries) return SPECA_ERR_INVALID_ARG;
+    const size_t esz = cfg->dtype == SPECA_BF16 ? 2 : 4;
+    const size_t n_segs = static_cast<size_t>(cfg->n_entries) * cfg->batch;
+    const int B = cfg->batch, m = cfg->max_order;
+
+    size_t off = 0;
+    L->segs_off = off;
+    off = align_up(off + n_segs * sizeof(SegDesc), kAlign);
+    L->tiles_direct_off = off;
+    off = align_up(off + (n_segs + 1) * sizeof(uint32_t), kAlign);
+    L->tiles_bulk_off = off;
+    off = align_up(off + (n_segs + 1) * sizeof(uint32_t), kAlign);
+    L->partials_off = off;
+    off = align_up(off + static_cast<size_t>(kMaxClusters) * B * 2 * sizeof(float), kAlign);
+    L->ticket_off = off;
+    off = align_up(off + 2 * sizeof(uint32_t), kAlign);
+    L->tables_off = off;
+
+    L->segs.resize(n_segs);
+    L->tiles_direct.assign(n_segs + 1, 0);
+    L->tiles_bulk.assign(n_segs + 1, 0);
+    const uint32_t td = tile_elems(cfg->dtype, SPECA_PATH_DIRECT), tb = tile_elems(cfg->dtype, SPECA_PATH_BULK);
+    uint64_t tiles_d = 0, tiles_b = 0;
+    for (int e = 0; e < cfg->n_entries; ++e) {
+        const int64_t tokens = cfg->entries[e].tokens;
+        const int64_t dim = cfg->entries[e].dim;
+        if (tokens < 1 || dim < 1) return SPECA_ERR_SHAPE;
+        if (tokens > (int64_t(1) << 31) / dim) return SPECA_ERR_SHAPE;  // n_elems must stay below 2^31
+        const uint64_t n = static_cast<uint64_t>(tokens) * dim;
+        if (n >= (uint64_t(1) << 31)) return SPECA_ERR_SHAPE;
+        const size_t stride = align_up(n * esz, kAlign);
+        for (int b = 0; b < B; ++b) {
+            SegDesc& s = L->segs[static_cast<size_t>(e) * B + b];
+            s.plane0_off = off;
+            s.plane_stride = stride;
+            s.io_off = static_cast<uint64_t>(b) * n * esz;
+            s.n_elems = static_cast<uint32_t>(n);
+            s.entry = static_cast<uint16_t>(e);
+            s.sample = static_cast<uint16_t>(b);
+            off += stride * (m + 1);
+            L->tiles_direct[static_cast<size_t>(e) * B + b] = static_cast<uint32_t>(tiles_d);
+            L->tiles_bulk[static_cast<size_t>(e) * B + b] = static_cast<uint32_t>(tiles_b);
+            tiles_d += (n + td - 1) / td;
+            tiles_b += (n + tb - 1) / tb;
+            if (tiles_b >= (uint64_t(1) << 32)) return SPECA_ERR_SHAPE;
+        }
+    }
+    L->tiles_direct[n_segs] = static_cast<uint32_t>(tiles_d);
+    L->tiles_bulk[n_segs] = static_cast<uint32_t>(tiles_b);
+    L->total = off;
+    return SPECA_OK;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+        if (prev != dev) ok = cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+struct speca_cache {
+    int n_entries, B, m, dtype, basis, verify_entry, device, path;
+    double eps;
+    char* arena;
+    Layout L;
+    int sm_count;
+    int grid_update, grid_forecast, grid_verify, cluster;
+    // per-sample reference history, most recent first
+    int32_t n_refs[SPECA_MAX_BATCH];
+    double t_hist[SPECA_MAX_BATCH][SPECA_MAX_ORDER + 1];
+    // reference step in progress
+    bool pending;
+    double pend_t[SPECA_MAX_BATCH];
+    uint8_t pend_mask[SPECA_MAX_BATCH];
+    std::vector<uint8_t> entry_updated;
+    uint64_t launches;
+    char last_error[256];
+};
+
+namespace {
+
+speca_status_t fail(speca_cache* c, speca_status_t st, const char* fmt, ...) {
+    if (c != nullptr) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(c->last_error, sizeof c->last_error, fmt, ap);
+        va_end(ap);
+    }
+    return st;
+}
+
+speca_status_t cuda_fail(speca_cache* c, cudaError_t err, const char* what) {
+    return fail(c, SPECA_ERR_CUDA, "%s: %s", what, cudaGetErrorString(err));
+}
+
+inline size_t elem_size(const speca_cache* c) { return c->dtype == SPECA_BF16 ? 2 : 4; }
+
+// An asynchronous error left by earlier work on this device surfaces here, before new work is queued.
+speca_status_t check_sticky(speca_cache* c) {
+    cudaError_t e = cudaPeekAtLastError();
+    if (e != cudaSuccess) return cuda_fail(c, e, "earlier CUDA error");
+    return SPECA_OK;
+}
+
+// Horner multipliers of Eq. 2 for sample b at time t: level i (1-based) multiplies by mu[i-1].
+void forecast_scalars(const speca_cache* c, int b, double t, int* order, float* mu) {
+    const int v = c->n_refs[b] < 1 ? -1 : (c->n_refs[b] - 1 < c->m ? c->n_refs[b] - 1 : c->m);
+    *order = v;
+    for (int i = 0; i < SPECA_MAX_ORDER; ++i) mu[i] = 0.f;
+    for (int i = 1; i <= v; ++i) {
+        const double x = (c->basis == SPECA_BASIS_NEWTON) ? (t - c->t_hist[b][i - 1]) : (t - c->t_hist[b][0]) / i;
+        mu[i - 1] = static_cast<float>(x);
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+speca_status_t speca_cache_arena_bytes(const speca_cache_config_t* cfg, size_t* out_bytes) {
+    if (out_bytes == nullptr) return SPECA_ERR_INVALID_ARG;
+    Layout L;
+    speca_status_t st = make_layout(cfg, &L);
+    if (st != SPECA_OK) return st;
+    *out_bytes = L.total;
+    return SPECA_OK;
+}
+
+speca_status_t speca_cache_create(const speca_cache_config_t* cfg, speca_cache_t** out) {
+    if (out == nullptr) return SPECA_ERR_INVALID_ARG;
+    *out = nullptr;
+    speca_cache* c = new (std::nothrow) speca_cache();
+    if (c == nullptr) return SPECA_ERR_NOMEM;
+    speca_status_t st = make_layout(cfg, &c->L);
+    if (st != SPECA_OK) {
+        delete c;
+        return st;
+    }
+    if (cfg->arena == nullptr) {
+        delete c;
+        return SPECA_ERR_INVALID_ARG;
+    }
+    if (reinterpret_cast<uintptr_t>(cfg->arena) % kAlign != 0) {
+        delete c;
+        return SPECA_ERR_ALIGNMENT;
+    }
+    if (cfg->arena_bytes < c->L.total) {
+        delete c;
+        return SPECA_ERR_NOMEM;
+    }
+    int n_dev = 0;
+    cudaError_t ce = cudaGetDeviceCount(&n_dev);
+    if (ce != cudaSuccess || cfg->device < 0 || cfg->device >= n_dev) {
+        delete c;
+        return ce != cudaSuccess ? SPECA_ERR_CUDA : SPECA_ERR_INVALID_ARG;
+    }
+    int major = 0;
+    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, cfg->device);
+    if (major != 10) {  // the kernels are built for sm_100a only
+        delete c;
+        return SPECA_ERR_UNSUPPORTED;
+    }
+    c->n_entries = cfg->n_entries;
+    c->B = cfg->batch;
+    c->m = cfg->max_order;
+    c->dtype = cfg->dtype;
+    c->basis = cfg->basis;
+    c->verify_entry = cfg->verify_entry < 0 ? cfg->n_entries - 1 : cfg->verify_entry;
+    c->device = cfg->device;
+    c->path = cfg->path == SPECA_PATH_AUTO ? SPECA_PATH_DIRECT : cfg->path;
+    c->eps = cfg->eps > 0.f ? static_cast<double>(cfg->eps) : 1e-8;  // Eq. 4
+    c->arena = static_cast<char*>(cfg->arena);
+    c->pending = false;
+    c->launches = 0;
+    c->last_error[0] = 0;
+    c->entry_updated.assign(c->n_entries, 0);
+    for (int b = 0; b < SPECA_MAX_BATCH; ++b) {
+        c->n_refs[b] = 0;
+        for (int i = 0; i <= SPECA_MAX_ORDER; ++i) c->t_hist[b][i] = std::numeric_limits<double>::quiet_NaN();
+    }
+    if (c->path == SPECA_PATH_BULK) {  // not built in this version of the library
+        delete c;
+        return SPECA_ERR_UNSUPPORTED;
+    }
+
+    DeviceGuard guard(c->device);
+    if (!guard.ok) {
+        delete c;
+        return SPECA_ERR_CUDA;
+    }
+    const Layout& L = c->L;
+    ce = cudaMemcpy(c->arena + L.segs_off, L.segs.data(), L.segs.size() * sizeof(SegDesc), cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess)
+        ce = cudaMemcpy(c->arena + L.tiles_direct_off, L.tiles_direct.data(), L.tiles_direct.size() * sizeof(uint32_t),
+                        cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess)
+        ce = cudaMemcpy(c->arena + L.tiles_bulk_off, L.tiles_bulk.data(), L.tiles_bulk.size() * sizeof(uint32_t),
+                        cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess) ce = cudaMemset(c->arena + L.ticket_off, 0, kAlign);
+    if (ce != cudaSuccess) {
+        delete c;
+        return SPECA_ERR_CUDA;
+    }
+    cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
+    c->grid_update = c->sm_count * ctas_per_sm_update(c->dtype, c->m);
+    c->grid_forecast = c->sm_count * ctas_per_sm_forecast(c->dtype, c->m);
+    c->cluster = 4;
+    int gv = c->sm_count * ctas_per_sm_verify(c->dtype, c->m);
+    gv = gv / c->cluster * c->cluster;
+    if (gv / c->cluster > kMaxClusters) gv = kMaxClusters * c->cluster;
+    c->grid_verify = gv;
+    *out = c;
+    return SPECA_OK;
+}
+
+speca_status_t speca_cache_destroy(speca_cache_t* c) {
+    if (c == nullptr) return SPECA_OK;
+    DeviceGuard guard(c->device);
+    cudaError_t ce = cudaDeviceSynchronize();
+    delete c;
+    return ce == cudaSuccess ? SPECA_OK : SPECA_ERR_CUDA;
+}
+
+speca_status_t speca_cache_reset(speca_cache_t* c, const uint8_t* host_sample_mask) {
+    if (c == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (c->pending) return fail(c, SPECA_ERR_STATE, "reset while a reference step is open");
+    for (int b = 0; b < c->B; ++b) {
+        if (host_sample_mask != nullptr && host_sample_mask[b] == 0) continue;
+        c->n_refs[b] = 0;
+        for (int i = 0; i <= SPECA_MAX_ORDER; ++i) c->t_hist[b][i] = std::numeric_limits<double>::quiet_NaN();
+    }
+    return SPECA_OK;
+}
+
+speca_status_t speca_cache_update(speca_cache_t* c, const void* const* feats, const double* t_ref,
+                                  const uint8_t* host_sample_mask, void* stream) {
+    if (c == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (feats == nullptr || t_ref == nullptr) return fail(c, SPECA_ERR_INVALID_ARG, "update: null argument");
+    uint8_t mask[SPECA_MAX_BATCH];
+    bool any_sample = false;
+    for (int b = 0; b < c->B; ++b) {
+        mask[b] = (host_sample_mask == nullptr || host_sample_mask[b] != 0) ? 1 : 0;
+        any_sample |= mask[b] != 0;
+        if (mask[b] && !std::isfinite(t_ref[b])) return fail(c, SPECA_ERR_INVALID_ARG, "update: t_ref[%d] not finite", b);
+    }
+    if (c->pending) {
+        for (int b = 0; b < c->B; ++b) {
+            if (mask[b] != c->pend_mask[b] || (mask[b] && std::memcmp(&t_ref[b], &c->pend_t[b], sizeof(double)) != 0))
+                return fail(c, SPECA_ERR_STATE, "update: mask or t_ref differ from the open reference step (sample %d)", b);
+        }
+    }
+    StreamParams p;
+    std::memset(&p, 0, sizeof p);
+    // scalars of Eq. 3: reciprocal gaps
+    for (int b = 0; b < c->B; ++b) {
+        p.order[b] = -1;
+        if (!mask[b]) continue;
+        const int v_new = c->n_refs[b] < c->m ? c->n_refs[b] : c->m;
+        for (int i = 0; i < v_new; ++i) {
+            const double gap = t_ref[b] - (c->basis == SPECA_BASIS_NEWTON ? c->t_hist[b][i] : c->t_hist[b][0]);
+            if (gap == 0.0) return fail(c, SPECA_ERR_ZERO_GAP, "update: sample %d repeats a reference time", b);
+            p.coef[b][i] = static_cast<float>(1.0 / gap);
+        }
+        p.order[b] = static_cast<int8_t>(v_new);
+    }
+    int e_lo = -1, e_hi = -1;
+    const size_t esz = elem_size(c);
+    for (int e = 0; e < c->n_entries; ++e) {
+        if (feats[e] == nullptr) continue;
+        if (c->entry_updated[e]) return fail(c, SPECA_ERR_STATE, "update: entry %d already updated in this step", e);
+        if (reinterpret_cast<uintptr_t>(feats[e]) % esz != 0)
+            return fail(c, SPECA_ERR_ALIGNMENT, "update: feats[%d] not aligned to the element size", e);
+        if (e_lo < 0) e_lo = e;
+        e_hi = e;
+        p.io[e] = const_cast<void*>(feats[e]);
+    }
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return fail(c, SPECA_ERR_CUDA, "cudaSetDevice failed");
+    speca_status_t st = check_sticky(c);
+    if (st != SPECA_OK) return st;
+    if (e_lo >= 0 && any_sample) {
+        const Layout& L = c->L;
+        const std::vector<uint32_t>& tiles = c->path == SPECA_PATH_BULK ? L.tiles_bulk : L.tiles_direct;
+        p.segs = reinterpret_cast<const SegDesc*>(c->arena + L.segs_off);
+        p.tile_start = reinterpret_cast<const uint32_t*>(
+            c->arena + (c->path == SPECA_PATH_BULK ? L.tiles_bulk_off : L.tiles_direct_off));
+        p.arena = c->arena;
+        p.dev_mask = nullptr;
+        p.err_flag = reinterpret_cast<uint32_t*>(c->arena + L.ticket_off) + 1;
+        p.seg_lo = static_cast<uint32_t>(e_lo) * c->B;
+        p.seg_hi = static_cast<uint32_t>(e_hi + 1) * c->B;
+        p.tile_lo = tiles[p.seg_lo];
+        p.tile_hi = tiles[p.seg_hi];
+        const uint32_t n_tiles = p.tile_hi - p.tile_lo;
+        const int grid = static_cast<int>(n_tiles < static_cast<uint32_t>(c->grid_update) ? n_tiles : c->grid_update);
+        cudaError_t ce = launch_update(p, c->dtype, c->path, grid, static_cast<cudaStream_t>(stream));
+        if (ce != cudaSuccess) return cuda_fail(c, ce, "update launch");
+        c->launches += 1;
+    }
+    if (!c->pending) {
+        c->pending = true;
+        for (int b = 0; b < c->B; ++b) {
+            c->pend_mask[b] = mask[b];
+            c->pend_t[b] = t_ref[b];
+        }
+    }
+    for (int e = 0; e < c->n_entries; ++e)
+        if (feats[e] != nullptr) c->entry_updated[e] = 1;
+    return SPECA_OK;
+}
+
+speca_status_t speca_cache_commit_step(speca_cache_t* c) {
+    if (c == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (!c->pending) return fail(c, SPECA_ERR_STATE, "commit: no reference step is open");
+    for (int e = 0; e < c->n_entries; ++e)
+        if (!c->entry_updated[e]) return fail(c, SPECA_ERR_STATE, "commit: entry %d was not updated in this step", e);
+    for (int b = 0; b < c->B; ++b) {
+        if (!c->pend_mask[b]) continue;
+        for (int i = SPECA_MAX_ORDER; i >= 1; --i) c->t_hist[b][i] = c->t_hist[b][i - 1];
+        c->t_hist[b][0] = c->pend_t[b];
+        c->n_refs[b] += 1;
+    }
+    c->pending = false;
+    std::fill(c->entry_updated.begin(), c->entry_updated.end(), 0);
+    return SPECA_OK;
+}
+
+speca_status_t speca_forecast(speca_cache_t* c, const double* t_target, const uint8_t* dev_active_mask,
+                              void* const* outs, void* stream) {
+    if (c == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (t_target == nullptr || outs == nullptr) return fail(c, SPECA_ERR_INVALID_ARG, "forecast: null argument");
+    if (c->pending) return fail(c, SPECA_ERR_STATE, "forecast: a reference step is open (commit it first)");
+    StreamParams p;
+    std::memset(&p, 0, sizeof p);
+    bool any_sample = false;
+    for (int b = 0; b < c->B; ++b) {
+        if (!std::isfinite(t_target[b])) return fail(c, SPECA_ERR_INVALID_ARG, "forecast: t_target[%d] not finite", b);
+        int order;
+        forecast_scalars(c, b, t_target[b], &order, p.coef[b]);
+        if (order < 0 && dev_active_mask == nullptr)
+            return fail(c, SPECA_ERR_STATE, "forecast: sample %d has no committed reference", b);
+        p.order[b] = static_cast<int8_t>(order);
+        any_sample |= order >= 0;
+    }
+    int e_lo = -1, e_hi = -1;
+    const size_t esz = elem_size(c);
+    for (int e = 0; e < c->n_entries; ++e) {
+        if (outs[e] == nullptr) continue;
+        if (reinterpret_cast<uintptr_t>(outs[e]) % esz != 0)
+            return fail(c, SPECA_ERR_ALIGNMENT, "forecast: outs[%d] not aligned to the element size", e);
+        if (e_lo < 0) e_lo = e;
+        e_hi = e;
+        p.io[e] = outs[e];
+    }
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return fail(c, SPECA_ERR_CUDA, "cudaSetDevice failed");
+    speca_status_t st = check_sticky(c);
+    if (st != SPECA_OK) return st;
+    if (e_lo < 0 || !any_sample) return SPECA_OK;
+    const Layout& L = c->L;
+    const std::vector<uint32_t>& tiles = c->path == SPECA_PATH_BULK ? L.tiles_bulk : L.tiles_direct;
+    p.segs = reinterpret_cast<const SegDesc*>(c->arena + L.segs_off);
+    p.tile_start =
+        reinterpret_cast<const uint32_t*>(c->arena + (c->path == SPECA_PATH_BULK ? L.tiles_bulk_off : L.tiles_direct_off));
+    p.arena = c->arena;
+    p.dev_mask = dev_active_mask;
+    p.err_flag = reinterpret_cast<uint32_t*>(c->arena + L.ticket_off) + 1;
+    p.seg_lo = static_cast<uint32_t>(e_lo) * c->B;
+    p.seg_hi = static_cast<uint32_t>(e_hi + 1) * c->B;
+    p.tile_lo = tiles[p.seg_lo];
+    p.tile_hi = tiles[p.seg_hi];
+    const uint32_t n_tiles = p.tile_hi - p.tile_lo;
+    const int grid = static_cast<int>(n_tiles < static_cast<uint32_t>(c->grid_forecast) ? n_tiles : c->grid_forecast);
+    cudaError_t ce = launch_forecast(p, c->dtype, c->path, grid, static_cast<cudaStream_t>(stream));
+    if (ce != cudaSuccess) return cuda_fail(c, ce, "forecast launch");
+    c->launches += 1;
+    return SPECA_OK;
+}
+
+speca_status_t speca_verify(speca_cache_t* c, const void* fresh, const double* t_target, const float* tau,
+                            const uint8_t* dev_active_mask, void* out_pred, float* dev_err, uint8_t* dev_accept,
+                            void* stream) {
+    if (c == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (fresh == nullptr || t_target == nullptr || tau == nullptr || dev_err == nullptr || dev_accept == nullptr)
+        return fail(c, SPECA_ERR_INVALID_ARG, "verify: null argument");
+    if (c->pending) return fail(c, SPECA_ERR_STATE, "verify: a reference step is open (commit it first)");
+    const size_t esz = elem_size(c);
+    if (reinterpret_cast<uintptr_t>(fresh) % esz != 0 || reinterpret_cast<uintptr_t>(out_pred) % esz != 0)
+        return fail(c, SPECA_ERR_ALIGNMENT, "verify: fresh / out_pred not aligned to the element size");
+    if (reinterpret_cast<uintptr_t>(dev_err) % sizeof(float) != 0)
+        return fail(c, SPECA_ERR_ALIGNMENT, "verify: dev_err not aligned");
+    VerifyParams p;
+    std::memset(&p, 0, sizeof p);
+    bool any_sample = false;
+    for (int b = 0; b < c->B; ++b) {
+        if (!std::isfinite(t_target[b])) return fail(c, SPECA_ERR_INVALID_ARG, "verify: t_target[%d] not finite", b);
+        if (std::isnan(tau[b])) return fail(c, SPECA_ERR_INVALID_ARG, "verify: tau[%d] is NaN", b);
+        int order;
+        forecast_scalars(c, b, t_target[b], &order, p.coef[b]);
+        if (order < 0 && dev_active_mask == nullptr)
+            return fail(c, SPECA_ERR_STATE, "verify: sample %d has no committed reference", b);
+        p.order[b] = static_cast<int8_t>(order);
+        p.tau[b] = tau[b];
+        any_sample |= order >= 0;
+    }
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return fail(c, SPECA_ERR_CUDA, "cudaSetDevice failed");
+    speca_status_t st = check_sticky(c);
+    if (st != SPECA_OK) return st;
+    if (!any_sample) return SPECA_OK;
+    const Layout& L = c->L;
+    const SegDesc& s0 = L.segs[static_cast<size_t>(c->verify_entry) * c->B];
+    const uint32_t te = tile_elems(c->dtype, SPECA_PATH_DIRECT);
+    p.segs = reinterpret_cast<const SegDesc*>(c->arena + L.segs_off) + static_cast<size_t>(c->verify_entry) * c->B;
+    p.arena = c->arena;
+    p.dev_mask = dev_active_mask;
+    p.fresh = static_cast<const char*>(fresh);
+    p.out_pred = static_cast<char*>(out_pred);
+    p.err = dev_err;
+    p.accept = dev_accept;
+    p.partials = reinterpret_cast<float*>(c->arena + L.partials_off);
+    p.ticket = reinterpret_cast<uint32_t*>(c->arena + L.ticket_off);
+    p.n_elems = s0.n_elems;
+    p.tiles_per_sample = (s0.n_elems + te - 1) / te;
+    p.units_per_sample = (p.tiles_per_sample + c->cluster - 1) / c->cluster;
+    p.batch = c->B;
+    p.eps = c->eps;
+    const uint64_t units = static_cast<uint64_t>(p.units_per_sample) * c->B;
+    int grid = c->grid_verify;
+    if (units * c->cluster < static_cast<uint64_t>(grid)) grid = static_cast<int>(units) * c->cluster;
+    cudaError_t ce = launch_verify(p, c->dtype, grid, c->cluster, static_cast<cudaStream_t>(stream));
+    if (ce != cudaSuccess) return cuda_fail(c, ce, "verify launch");
+    c->launches += 1;
+    return SPECA_OK;
+}
+
+speca_status_t speca_select_adaptive(speca_cache_t* c, const uint8_t* dev_accept, int32_t k_max, int32_t group,
+                                     int32_t* dev_spec_count, uint8_t* dev_active_mask, int32_t* dev_active_idx,
+                                     int32_t* dev_n_active, void* stream) {
+    if (c == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (dev_accept == nullptr || dev_spec_count == nullptr || dev_active_mask == nullptr)
+        return fail(c, SPECA_ERR_INVALID_ARG, "select: null argument");
+    if (k_max < 1 || group < 1 || c->B % group != 0)
+        return fail(c, SPECA_ERR_INVALID_ARG, "select: k_max >= 1 and group must divide the batch");
+    if (reinterpret_cast<uintptr_t>(dev_spec_count) % 4 != 0 || reinterpret_cast<uintptr_t>(dev_active_idx) % 4 != 0 ||
+        reinterpret_cast<uintptr_t>(dev_n_active) % 4 != 0)
+        return fail(c, SPECA_ERR_ALIGNMENT, "select: int32 buffers must be 4-byte aligned");
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return fail(c, SPECA_ERR_CUDA, "cudaSetDevice failed");
+    speca_status_t st = check_sticky(c);
+    if (st != SPECA_OK) return st;
+    cudaError_t ce = launch_select(dev_accept, k_max, group, c->B, dev_spec_count, dev_active_mask, dev_active_idx,
+                                   dev_n_active, static_cast<cudaStream_t>(stream));
+    if (ce != cudaSuccess) return cuda_fail(c, ce, "select launch");
+    c->launches += 1;
+    return SPECA_OK;
+}
+
+speca_status_t speca_activate(speca_cache_t* c, const uint8_t* host_sample_mask, int32_t* dev_spec_count,
+                              uint8_t* dev_active_mask, void* stream) {
+    if (c == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (dev_spec_count == nullptr || dev_active_mask == nullptr)
+        return fail(c, SPECA_ERR_INVALID_ARG, "activate: null argument");
+    if (reinterpret_cast<uintptr_t>(dev_spec_count) % 4 != 0)
+        return fail(c, SPECA_ERR_ALIGNMENT, "activate: dev_spec_count must be 4-byte aligned");
+    uint64_t bits = 0;
+    for (int b = 0; b < c->B; ++b)
+        if (host_sample_mask == nullptr || host_sample_mask[b] != 0) bits |= (uint64_t(1) << b);
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return fail(c, SPECA_ERR_CUDA, "cudaSetDevice failed");
+    speca_status_t st = check_sticky(c);
+    if (st != SPECA_OK) return st;
+    cudaError_t ce = launch_activate(bits, c->B, dev_spec_count, dev_active_mask, static_cast<cudaStream_t>(stream));
+    if (ce != cudaSuccess) return cuda_fail(c, ce, "activate launch");
+    c->launches += 1;
+    return SPECA_OK;
+}
+
+double speca_tau(double tau0, double beta, double t, double T) {
+    if (!(T > 0.0)) return std::numeric_limits<double>::quiet_NaN();
+    return tau0 * std::pow(beta, (T - t) / T);
+}
+
+speca_status_t speca_cache_state(const speca_cache_t* c, int32_t* host_n_refs, double* host_t_last) {
+    if (c == nullptr) return SPECA_ERR_INVALID_ARG;
+    for (int b = 0; b < c->B; ++b) {
+        if (host_n_refs != nullptr) host_n_refs[b] = c->n_refs[b];
+        if (host_t_last != nullptr) host_t_last[b] = c->t_hist[b][0];
+    }
+    return SPECA_OK;
+}
+
+speca_status_t speca_cache_plane(const speca_cache_t* c, int32_t entry, int32_t sample, void** plane0,
+                                 size_t* plane_stride_bytes) {
+    if (c == nullptr || plane0 == nullptr || plane_stride_bytes == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (entry < 0 || entry >= c->n_entries || sample < 0 || sample >= c->B) return SPECA_ERR_INVALID_ARG;
+    const SegDesc& s = c->L.segs[static_cast<size_t>(entry) * c->B + sample];
+    *plane0 = c->arena + s.plane0_off;
+    *plane_stride_bytes = s.plane_stride;
+    return SPECA_OK;
+}
+
+speca_status_t speca_cache_launch_count(const speca_cache_t* c, uint64_t* out) {
+    if (c == nullptr || out == nullptr) return SPECA_ERR_INVALID_ARG;
+    *out = c->launches;
+    return SPECA_OK;
+}
+
+const char* speca_status_string(speca_status_t status) {
+    switch (status) {
+        case SPECA_OK: return "ok";
+        case SPECA_ERR_INVALID_ARG: return "invalid argument";
+        case SPECA_ERR_SHAPE: return "shape outside supported limits";
+        case SPECA_ERR_ALIGNMENT: return "pointer alignment";
+        case SPECA_ERR_STATE: return "call order violated";
+        case SPECA_ERR_ZERO_GAP: return "reference time repeats (zero gap)";
+        case SPECA_ERR_NOMEM: return "out of memory / arena too small";
+        case SPECA_ERR_CUDA: return "CUDA error";
+        case SPECA_ERR_UNSUPPORTED: return "unsupported device or feature";
+    }
+    return "unknown status";
+}
+
+const char* speca_last_error(const speca_cache_t* c) { return c == nullptr ? "" : c->last_error; }
+
+const char* speca_version(void) { return "speca-b200 0.1 (sm_100a)"; }
+
+}  // extern "C"

@@ -1,0 +1,86 @@
+// Internal declarations shared by the host dispatch (speca_api.cpp) and the kernels
+// (speca_kernels.cu). Not part of the public ABI.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "speca.h"
+
+namespace speca {
+
+// Bytes of one plane that a tile covers. A tile is the unit a CTA picks up from the flattened
+// work list: kTileBytes / sizeof(element) consecutive elements of one (entry, sample) table.
+constexpr uint32_t kTileBytesDirect = 16384;  // 256 threads x 4 vectors x 16 B
+constexpr uint32_t kTileBytesBulk = 8192;     // one cp.async.bulk per plane per stage
+constexpr int kThreads = 256;
+constexpr int kMaxClusters = 1024;  // upper bound on verify clusters (reduction scratch rows)
+
+// One (entry, sample) table. Segments are ordered entry-major, sample-minor: seg = e * B + b.
+struct SegDesc {
+    uint64_t plane0_off;    // byte offset of plane 0 from the arena base (256-byte aligned)
+    uint64_t plane_stride;  // bytes between consecutive planes (multiple of 256)
+    uint64_t io_off;        // byte offset of this sample's row inside the entry's [B, N_e, D] tensor
+    uint32_t n_elems;       // N_e * D
+    uint16_t entry;
+    uint16_t sample;
+};
+static_assert(sizeof(SegDesc) == 32, "SegDesc layout");
+
+// Arguments of the streaming kernels (update, forecast), passed by value as one kernel parameter.
+struct StreamParams {
+    const SegDesc* segs;         // all segments of the cache
+    const uint32_t* tile_start;  // [n_segs + 1] prefix of tiles per segment, for this path's tile size
+    char* arena;
+    const uint8_t* dev_mask;  // device, per sample, may be null
+    uint32_t seg_lo, seg_hi;  // segment range this launch covers
+    uint32_t tile_lo, tile_hi;
+    uint32_t* err_flag;  // device word the bulk path sets if a wait gives up
+    // update:   order = highest plane written (v_new), coef[b][i] = 1 / gap_i
+    // forecast: order = highest plane read (v),        coef[b][i] = Horner multiplier of level i+1
+    // order < 0: sample is skipped
+    int8_t order[SPECA_MAX_BATCH];
+    float coef[SPECA_MAX_BATCH][SPECA_MAX_ORDER];
+    void* io[SPECA_MAX_ENTRIES];  // per entry: feature (update) or output (forecast); null = skip
+};
+
+// Arguments of the fused forecast + relative-L2 kernel over the verification entry.
+struct VerifyParams {
+    const SegDesc* segs;  // segments of the verify entry only (B of them)
+    char* arena;
+    const uint8_t* dev_mask;
+    const char* fresh;  // [B, N_v, D]
+    char* out_pred;     // may be null
+    float* err;
+    uint8_t* accept;
+    float* partials;     // [n_clusters][B][2]
+    uint32_t* ticket;    // arrival counter, zero between launches
+    uint32_t n_elems;    // per sample
+    uint32_t tiles_per_sample;
+    uint32_t units_per_sample;  // ceil(tiles_per_sample / cluster size)
+    int32_t batch;
+    double eps;
+    int8_t order[SPECA_MAX_BATCH];
+    float coef[SPECA_MAX_BATCH][SPECA_MAX_ORDER];
+    float tau[SPECA_MAX_BATCH];
+};
+
+// Launchers. `dtype` is a speca_dtype_t. All enqueue on `stream` and return the launch status.
+cudaError_t launch_update(const StreamParams& p, int dtype, int path, int grid, cudaStream_t stream);
+cudaError_t launch_forecast(const StreamParams& p, int dtype, int path, int grid, cudaStream_t stream);
+cudaError_t launch_verify(const VerifyParams& p, int dtype, int grid, int cluster, cudaStream_t stream);
+cudaError_t launch_select(const uint8_t* accept, int32_t k_max, int32_t group, int32_t batch, int32_t* spec_count,
+                          uint8_t* active, int32_t* idx, int32_t* n_active, cudaStream_t stream);
+cudaError_t launch_activate(uint64_t mask_bits, int32_t batch, int32_t* spec_count, uint8_t* active,
+                            cudaStream_t stream);
+
+// Resident CTAs per SM of each kernel family (occupancy query), for sizing persistent grids.
+int ctas_per_sm_update(int dtype, int order);
+int ctas_per_sm_forecast(int dtype, int order);
+int ctas_per_sm_verify(int dtype, int order);
+
+inline uint32_t tile_elems(int dtype, int path) {
+    uint32_t bytes = (path == SPECA_PATH_BULK) ? kTileBytesBulk : kTileBytesDirect;
+    return bytes / (dtype == SPECA_BF16 ? 2u : 4u);
+}
+
+}  // namespace speca
