@@ -1,0 +1,102 @@
+"""The multi-rank plumbing on CPU: two ``gloo`` processes shard the samples, each runs its own
+(oracle) cache on its shard with no exchange on the data path, and only the timing reduction and the
+optional decision gather cross ranks. Checks that the sharded decisions equal the unsharded ones."""
+import os
+import socket
+import sys
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port() -> int:
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def _inputs(B, n, seed=11):
+    g = torch.Generator().manual_seed(seed)
+    feats = [torch.randn(B, n, generator=g).numpy().copy() for _ in range(3)]
+    noise = torch.tensor([0.0, 0.01, 0.3, 1.0, 0.02])[:B].view(B, 1)
+    fresh_noise = (torch.randn(B, n, generator=g) * noise).numpy()
+    return feats, fresh_noise
+
+
+def _decisions(sample_ids, feats, fresh_noise, n):
+    from oracle import speca_oracle as O
+    B = len(sample_ids)
+    if B == 0:
+        return [], []
+    cache = O.OracleCache([n], B, 2, O.F32)
+    for k, t in enumerate([1.0, 0.9, 0.8]):
+        cache.update([feats[k][sample_ids]], [t] * B)
+        cache.commit_step()
+    pred = cache.forecast_entry(0, [0.75] * B)
+    fresh = (pred + fresh_noise[sample_ids]).astype(np.float32)
+    err, acc, _ = cache.verify(fresh, [0.75] * B, [0.05] * B)
+    return [float(e) for e in err], [int(a) for a in acc]
+
+
+def _worker(rank, world, port, out_dir):
+    if ROOT not in sys.path:
+        sys.path.insert(0, ROOT)
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    from paper_2509_11628_b200 import dist as D
+    info = D.init("gloo")
+    assert (info.rank, info.world) == (rank, world) and info.is_main == (rank == 0)
+    B, n = 5, 257
+    feats, fresh_noise = _inputs(B, n)
+    mine = D.shard_samples(B, world, rank)
+    D.barrier()
+    err, acc = _decisions(mine, feats, fresh_noise, n)
+    D.barrier()
+    slowest = D.max_over_ranks(10.0 + rank)
+    total = D.sum_over_ranks(len(mine))
+    everyone = D.gather_decisions(acc)
+    assert slowest == 10.0 + (world - 1)
+    assert total == B
+    flat = [a for part in everyone for a in part]
+    if rank == 0:
+        torch.save({"acc": flat, "err_rank0": err, "shard0": mine}, os.path.join(out_dir, "r0.pt"))
+    D.shutdown()
+
+
+def test_two_ranks_shard_samples_without_a_data_path_collective(tmp_path):
+    port = _free_port()
+    mp.spawn(_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    got = torch.load(os.path.join(str(tmp_path), "r0.pt"))
+    B, n = 5, 257
+    feats, fresh_noise = _inputs(B, n)
+    err_all, acc_all = _decisions(list(range(B)), feats, fresh_noise, n)
+    assert got["acc"] == acc_all            # per-sample decisions do not depend on the sharding
+    assert got["shard0"] == [0, 1, 2]
+    assert got["err_rank0"] == err_all[:3]  # bit-identical: a sample's error depends on that sample alone
+    assert acc_all[0] == 1 and acc_all[3] == 0
+
+
+def test_shard_samples_is_a_balanced_partition():
+    from paper_2509_11628_b200 import dist as D
+    for n in (1, 5, 8, 16, 64):
+        for world in (1, 2, 3, 4, 8):
+            parts = [D.shard_samples(n, world, r) for r in range(world)]
+            flat = [i for p in parts for i in p]
+            assert flat == list(range(n))
+            sizes = [len(p) for p in parts]
+            assert max(sizes) - min(sizes) <= 1
+
+
+def test_single_process_reductions_are_identities():
+    from paper_2509_11628_b200 import dist as D
+    assert not dist.is_initialized()
+    assert D.max_over_ranks(3.5) == 3.5 and D.sum_over_ranks(2.0) == 2.0
+    assert D.gather_decisions([1, 0]) == [[1, 0]]
+    D.barrier()
