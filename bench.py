@@ -186,18 +186,20 @@ class Harness:
             events[0].record()
         c.update(feats, t_ref)
         c.commit_step()
-        c.activate(None, self.spec, self.active)
         if events is not None:
             events[1].record()
-        c.forecast(t_tgt, self.outs, self.active)
+        c.activate(None, self.spec, self.active)
         if events is not None:
             events[2].record()
-        c.verify(fresh, t_tgt, tau, self.err, self.accept, self.active)
+        c.forecast(t_tgt, self.outs, self.active)
         if events is not None:
             events[3].record()
-        c.select_adaptive(self.accept, 1 << 30, 1, self.spec, self.active, self.idx, self.n_active)
+        c.verify(fresh, t_tgt, tau, self.err, self.accept, self.active)
         if events is not None:
             events[4].record()
+        c.select_adaptive(self.accept, 1 << 30, 1, self.spec, self.active, self.idx, self.n_active)
+        if events is not None:
+            events[5].record()
 
     def close(self):
         self.cache.close()
@@ -208,7 +210,7 @@ def time_device_resident(h: Harness, steps: int, warmup: int, info: D.RankInfo, 
     for _ in range(warmup):
         h.step()
     torch.cuda.synchronize(dev)
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(steps)]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(steps)]
     launches0 = h.cache.launches
     sampler = ClockSampler(physical_gpu_index(dev.index or 0)) if sample_clocks else None
     D.barrier()
@@ -230,9 +232,9 @@ def time_device_resident(h: Harness, steps: int, warmup: int, info: D.RankInfo, 
     per = {"update": 0.0, "forecast": 0.0, "verify": 0.0, "select": 0.0}
     for k in range(steps):
         per["update"] += ev[k][0].elapsed_time(ev[k][1])
-        per["forecast"] += ev[k][1].elapsed_time(ev[k][2])
-        per["verify"] += ev[k][2].elapsed_time(ev[k][3])
-        per["select"] += ev[k][3].elapsed_time(ev[k][4])
+        per["forecast"] += ev[k][2].elapsed_time(ev[k][3])
+        per["verify"] += ev[k][3].elapsed_time(ev[k][4])
+        per["select"] += ev[k][1].elapsed_time(ev[k][2]) + ev[k][4].elapsed_time(ev[k][5])  # activate + select
     per = {k: v / steps for k, v in per.items()}
     return total_ms, per, h.cache.launches - launches0, (sampler.summary() if sampler else None)
 
