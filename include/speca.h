@@ -207,6 +207,47 @@ speca_status_t speca_select_adaptive(speca_cache_t* cache, const uint8_t* dev_ac
 speca_status_t speca_activate(speca_cache_t* cache, const uint8_t* host_sample_mask, int32_t* dev_spec_count,
                               uint8_t* dev_active_mask, void* stream);
 
+/*
+ * Verification without a handle, an arena or any allocation. (The paper has no counterpart: this is
+ * Eq. 4 and the accept rule applied to a forecast tensor the caller already holds, offered for
+ * callers that cannot give the library memory.)
+ *
+ * Who needs it: code that runs where device memory can no longer be obtained -- a serving process
+ * whose framework pool took all of HBM at start-up, a plug-in that is only handed input and output
+ * tensors, a host thread that must not call cudaMalloc because that call synchronises the whole
+ * device. speca_verify keeps its reduction scratch in the caller's arena; this variant keeps it in
+ * a fixed array inside the library image instead, SPECA_STATIC_SCRATCH_BYTES (about 66 KB) that
+ * every GPU which loads the library holds until the process exits. The call path contains no
+ * cudaMalloc, cudaFree or other allocating routine.
+ *
+ *   e_b = ||pred_b - fresh_b||_2 / (||fresh_b||_2 + eps),  accept_b = (e_b <= tau_b)
+ *
+ *   pred, fresh     device, dense [batch, n_elems] in `dtype`; both 16-byte aligned, and
+ *                   n_elems * sizeof(element) a multiple of 16 when batch > 1 (every row must
+ *                   start on a 16-byte boundary). pred is typically an output of speca_forecast.
+ *   n_elems         1 .. SPECA_STATIC_MAX_ELEMS per sample; batch 1 .. SPECA_STATIC_MAX_BATCH.
+ *   tau             host, batch floats. eps <= 0 selects the paper's 1e-8.
+ *   dev_active_mask device, batch bytes, NULL = all; inactive samples' err / accept are untouched.
+ *   dev_err         device, batch floats.  dev_accept: device, batch bytes (1 = accept).
+ *   device          CUDA device ordinal that owns all the buffers; stream as everywhere else.
+ *
+ * The first call on a device looks up the scratch array's device address
+ * (cudaGetSymbolAddress, with that device current) and remembers it; make that first call before
+ * any stream capture begins. Every call on a device shares the one array, which keeps whatever the
+ * previous call left: each call re-initialises what it needs on the stream before the reduction
+ * runs, so calls in stream order are independent, but two calls whose kernels overlap on the GPU
+ * (different streams, no dependency between them) race on the scratch and give wrong results.
+ * Errors: INVALID_ARG (null, dtype, NaN tau, bad device), SHAPE (batch or n_elems beyond the
+ * maxima above), ALIGNMENT, UNSUPPORTED (not an sm_100 device), CUDA. On error nothing is enqueued.
+ */
+#define SPECA_STATIC_MAX_BATCH 64
+#define SPECA_STATIC_MAX_ELEMS 2147483647LL
+#define SPECA_STATIC_MAX_CLUSTERS 128
+#define SPECA_STATIC_SCRATCH_BYTES (32 * 64 + 8 * 64 * SPECA_STATIC_MAX_CLUSTERS + 256)
+speca_status_t speca_verify_pred_static(const void* pred, const void* fresh, int64_t n_elems, int32_t batch,
+                                        int32_t dtype, const float* tau, float eps, const uint8_t* dev_active_mask,
+                                        float* dev_err, uint8_t* dev_accept, int32_t device, void* stream);
+
 /* Threshold schedule of Section 3.4.2: tau_t = tau0 * beta^((T - t) / T). Returns NaN for T <= 0. */
 double speca_tau(double tau0, double beta, double t, double T);
 

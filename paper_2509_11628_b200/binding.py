@@ -29,6 +29,7 @@ EXPORTS = [
     "speca_cache_update", "speca_cache_commit_step", "speca_forecast", "speca_verify",
     "speca_select_adaptive", "speca_activate", "speca_tau", "speca_cache_state", "speca_cache_plane",
     "speca_cache_launch_count", "speca_status_string", "speca_last_error", "speca_version",
+    "speca_verify_pred_static",
 ]
 
 
@@ -76,6 +77,7 @@ def _lib() -> ctypes.CDLL:
     L.speca_verify.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.speca_select_adaptive.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, vp]
     L.speca_activate.argtypes = [vp, vp, vp, vp, vp]
+    L.speca_verify_pred_static.argtypes = [vp, vp, ctypes.c_int64, i32, i32, vp, ctypes.c_float, vp, vp, vp, i32, vp]
     L.speca_tau.argtypes = [dbl, dbl, dbl, dbl]
     L.speca_tau.restype = dbl
     L.speca_cache_state.argtypes = [vp, vp, vp]
@@ -212,6 +214,16 @@ def speca_select_adaptive(cache, dev_accept, k_max, group, dev_spec_count, dev_a
 def speca_activate(cache, host_sample_mask, dev_spec_count, dev_active_mask, stream=None) -> None:
     _check(_lib().speca_activate(cache, _bytes(host_sample_mask), _dev_ptr(dev_spec_count), _dev_ptr(dev_active_mask),
                                  _stream_ptr(stream)), cache)
+
+
+def speca_verify_pred_static(pred, fresh, n_elems, batch, dtype, tau, eps, dev_active_mask, dev_err, dev_accept,
+                             device=0, stream=None) -> None:
+    """Eq. 4 + accept rule on a forecast the caller holds, with the reduction scratch inside the
+    library image: for callers that cannot allocate device memory or hand over an arena. Calls
+    whose kernels overlap on the GPU race on that shared scratch; keep them in stream order."""
+    _check(_lib().speca_verify_pred_static(_dev_ptr(pred), _dev_ptr(fresh), int(n_elems), int(batch), int(dtype),
+                                           _floats(tau), float(eps), _dev_ptr(dev_active_mask), _dev_ptr(dev_err),
+                                           _dev_ptr(dev_accept), int(device), _stream_ptr(stream)))
 
 
 def speca_tau(tau0: float, beta: float, t: float, T: float) -> float:

@@ -14,7 +14,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libspeca.so")
-SOURCES = ["speca_kernels.cu", "speca_api.cpp"]
+SOURCES = ["speca_kernels.cu", "speca_static.cu", "speca_api.cpp"]
 HEADERS = [os.path.join(CSRC, "speca_internal.h"), os.path.join(ROOT, "include", "speca.h")]
 
 
