@@ -132,11 +132,11 @@ def physical_gpu_index(local_index: int) -> int:
 class Harness:
     """Device-resident state for one workload: cache, two alternating feature sets, outputs."""
 
-    def __init__(self, w: W.Workload, device: str, seed_offset: int = 0):
+    def __init__(self, w: W.Workload, device: str, seed_offset: int = 0, path: int = 0):
         from paper_2509_11628_b200 import binding as S
         self.S, self.w, self.device = S, w, torch.device(device)
         self.B, self.m = w.batch, w.max_order
-        self.cache = S.SpecaCache(w.entries, w.batch, w.max_order, w.dtype, device)
+        self.cache = S.SpecaCache(w.entries, w.batch, w.max_order, w.dtype, device, path=path)
         self.src = W.FeatureSource(w, device, seed_offset)
         ne = len(w.entries)
         # warm the tables with max_order + 1 fully computed steps of the generator
@@ -380,6 +380,8 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--also", default="dit_xl2,hunyuan_video",
                     help="comma list of further configs measured device-resident and reported under per_config")
+    ap.add_argument("--path", default="auto", choices=["auto", "direct", "wide"],
+                    help="kernel variant (speca_path_t); results are identical, only speed differs")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -402,7 +404,8 @@ def main():
     peak, peak_src = measured_peak()
 
     w = make_workload(args.config)
-    h = Harness(w, device, seed_offset=17 * info.rank)
+    path = {"auto": 0, "direct": 1, "wide": 3}[args.path]
+    h = Harness(w, device, seed_offset=17 * info.rank, path=path)
     total_ms, per_ms, launches, clocks = time_device_resident(h, args.steps, args.warmup, info, True)
     total_ms = D.max_over_ranks(total_ms, device)
     value, ms_step, kernels, extra = summarize(w, per_ms, total_ms, args.steps, info.world, peak)
@@ -426,7 +429,7 @@ def main():
         for name in [n for n in args.also.split(",") if n and n != args.config]:
             try:
                 w2 = make_workload(name)
-                h2 = Harness(w2, device)
+                h2 = Harness(w2, device, path=path)
                 k2 = max(5, min(args.steps, 2000 // max(1, len(w2.entries)) * 4))
                 t2, p2, _, _ = time_device_resident(h2, k2, 3, info, False)
                 v2, ms2, kern2, ex2 = summarize(w2, p2, t2, k2, 1, peak)

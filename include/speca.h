@@ -73,9 +73,10 @@ typedef enum { SPECA_BASIS_TAYLOR = 0, SPECA_BASIS_NEWTON = 1 } speca_basis_t;
 
 /* Which kernel variant moves the data. Results are identical; only speed differs. */
 typedef enum {
-    SPECA_PATH_AUTO = 0,   /* library default */
-    SPECA_PATH_DIRECT = 1, /* vectorised global loads straight into registers */
-    SPECA_PATH_BULK = 2    /* cp.async.bulk (TMA) staging through a shared-memory ring */
+    SPECA_PATH_AUTO = 0,   /* library default: the fastest measured (currently WIDE) */
+    SPECA_PATH_DIRECT = 1, /* 16-byte vector loads straight into registers, 256 threads x 4 deep */
+    SPECA_PATH_BULK = 2,   /* cp.async.bulk (TMA) staging through a shared-memory ring */
+    SPECA_PATH_WIDE = 3    /* 32-byte vector loads / stores, per-kernel launch shapes */
 } speca_path_t;
 
 typedef struct {
@@ -92,7 +93,8 @@ typedef struct {
     int32_t basis;                     /* speca_basis_t */
     int32_t verify_entry;              /* index of the verification layer's entry; -1 = last entry */
     float eps;                         /* epsilon of Eq. 4; <= 0 selects the paper's 1e-8 */
-    void* arena;                       /* device; caller-owned, 256-byte aligned, lives as long as the handle */
+    void* arena;                       /* device; caller-owned, 256-byte aligned (4 KB aligned for full speed:
+                                          planes then start on 4 KB boundaries), lives as long as the handle */
     size_t arena_bytes;                /* >= speca_cache_arena_bytes() */
     int32_t device;                    /* CUDA device ordinal that owns the arena */
     int32_t path;                      /* speca_path_t */

@@ -17,12 +17,16 @@ using namespace speca;
 namespace {
 
 constexpr size_t kAlign = 256;
+// Planes start on 4 KB boundaries (relative to the arena base). A warp moves 1 KB per 32-byte vector
+// instruction; streams whose starts differ by an odd multiple of 256 B split those across L2 / DRAM
+// interleave boundaries and measured 3-5 % slower on B200.
+constexpr size_t kPlaneAlign = 4096;
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-    size_t segs_off, tiles_direct_off, tiles_bulk_off, partials_off, ticket_off, tables_off, total;
+    size_t segs_off, tiles_off[kNumTileSizes], partials_off, ticket_off, tables_off, total;
     std::vector<SegDesc> segs;
-    std::vector<uint32_t> tiles_direct, tiles_bulk;
+    std::vector<uint32_t> tiles[kNumTileSizes];  // per tile size: first tile of each segment, then the total
 };
 
 // Shape checks and arena layout shared by speca_cache_arena_bytes and speca_cache_create.
@@ -33,7 +37,8 @@ speca_status_t make_layout(const speca_cache_config_t* cfg, Layout* L) {
     if (cfg->max_order < 0 || cfg->max_order > SPECA_MAX_ORDER) return SPECA_ERR_SHAPE;
     if (cfg->dtype != SPECA_F32 && cfg->dtype != SPECA_BF16) return SPECA_ERR_INVALID_ARG;
     if (cfg->basis != SPECA_BASIS_TAYLOR && cfg->basis != SPECA_BASIS_NEWTON) return SPECA_ERR_INVALID_ARG;
-    if (cfg->path != SPECA_PATH_AUTO && cfg->path != SPECA_PATH_DIRECT && cfg->path != SPECA_PATH_BULK)
+    if (cfg->path != SPECA_PATH_AUTO && cfg->path != SPECA_PATH_DIRECT && cfg->path != SPECA_PATH_BULK &&
+        cfg->path != SPECA_PATH_WIDE)
         return SPECA_ERR_INVALID_ARG;
     if (cfg->verify_entry < -1 || cfg->verify_entry >= cfg->n_entries) return SPECA_ERR_INVALID_ARG;
     const size_t esz = cfg->dtype == SPECA_BF16 ? 2 : 4;
@@ -43,21 +48,22 @@ speca_status_t make_layout(const speca_cache_config_t* cfg, Layout* L) {
     size_t off = 0;
     L->segs_off = off;
     off = align_up(off + n_segs * sizeof(SegDesc), kAlign);
-    L->tiles_direct_off = off;
-    off = align_up(off + (n_segs + 1) * sizeof(uint32_t), kAlign);
-    L->tiles_bulk_off = off;
-    off = align_up(off + (n_segs + 1) * sizeof(uint32_t), kAlign);
+    for (int k = 0; k < kNumTileSizes; ++k) {
+        L->tiles_off[k] = off;
+        off = align_up(off + (n_segs + 1) * sizeof(uint32_t), kAlign);
+    }
     L->partials_off = off;
     off = align_up(off + static_cast<size_t>(kMaxClusters) * B * 2 * sizeof(float), kAlign);
     L->ticket_off = off;
-    off = align_up(off + 2 * sizeof(uint32_t), kAlign);
+    off = align_up(off + 2 * sizeof(uint32_t), kPlaneAlign);
     L->tables_off = off;
 
     L->segs.resize(n_segs);
-    L->tiles_direct.assign(n_segs + 1, 0);
-    L->tiles_bulk.assign(n_segs + 1, 0);
-    const uint32_t td = tile_elems(cfg->dtype, SPECA_PATH_DIRECT), tb = tile_elems(cfg->dtype, SPECA_PATH_BULK);
-    uint64_t tiles_d = 0, tiles_b = 0;
+    uint64_t n_tiles[kNumTileSizes];
+    for (int k = 0; k < kNumTileSizes; ++k) {
+        L->tiles[k].assign(n_segs + 1, 0);
+        n_tiles[k] = 0;
+    }
     for (int e = 0; e < cfg->n_entries; ++e) {
         const int64_t tokens = cfg->entries[e].tokens;
         const int64_t dim = cfg->entries[e].dim;
@@ -65,7 +71,7 @@ speca_status_t make_layout(const speca_cache_config_t* cfg, Layout* L) {
         if (tokens > (int64_t(1) << 31) / dim) return SPECA_ERR_SHAPE;  // n_elems must stay below 2^31
         const uint64_t n = static_cast<uint64_t>(tokens) * dim;
         if (n >= (uint64_t(1) << 31)) return SPECA_ERR_SHAPE;
-        const size_t stride = align_up(n * esz, kAlign);
+        const size_t stride = align_up(n * esz, kPlaneAlign);
         for (int b = 0; b < B; ++b) {
             SegDesc& s = L->segs[static_cast<size_t>(e) * B + b];
             s.plane0_off = off;
@@ -75,15 +81,14 @@ speca_status_t make_layout(const speca_cache_config_t* cfg, Layout* L) {
             s.entry = static_cast<uint16_t>(e);
             s.sample = static_cast<uint16_t>(b);
             off += stride * (m + 1);
-            L->tiles_direct[static_cast<size_t>(e) * B + b] = static_cast<uint32_t>(tiles_d);
-            L->tiles_bulk[static_cast<size_t>(e) * B + b] = static_cast<uint32_t>(tiles_b);
-            tiles_d += (n + td - 1) / td;
-            tiles_b += (n + tb - 1) / tb;
-            if (tiles_b >= (uint64_t(1) << 32)) return SPECA_ERR_SHAPE;
+            for (int k = 0; k < kNumTileSizes; ++k) {
+                L->tiles[k][static_cast<size_t>(e) * B + b] = static_cast<uint32_t>(n_tiles[k]);
+                n_tiles[k] += (n * esz + kTileSizes[k] - 1) / kTileSizes[k];
+                if (n_tiles[k] >= (uint64_t(1) << 32)) return SPECA_ERR_SHAPE;
+            }
         }
     }
-    L->tiles_direct[n_segs] = static_cast<uint32_t>(tiles_d);
-    L->tiles_bulk[n_segs] = static_cast<uint32_t>(tiles_b);
+    for (int k = 0; k < kNumTileSizes; ++k) L->tiles[k][n_segs] = static_cast<uint32_t>(n_tiles[k]);
     L->total = off;
     return SPECA_OK;
 }
@@ -110,6 +115,7 @@ struct speca_cache {
     Layout L;
     int sm_count;
     int grid_update, grid_forecast, grid_verify, cluster;
+    int tile_update, tile_forecast;  // indices into kTileSizes
     // per-sample reference history, most recent first
     int32_t n_refs[SPECA_MAX_BATCH];
     double t_hist[SPECA_MAX_BATCH][SPECA_MAX_ORDER + 1];
@@ -212,7 +218,7 @@ speca_status_t speca_cache_create(const speca_cache_config_t* cfg, speca_cache_t
     c->basis = cfg->basis;
     c->verify_entry = cfg->verify_entry < 0 ? cfg->n_entries - 1 : cfg->verify_entry;
     c->device = cfg->device;
-    c->path = cfg->path == SPECA_PATH_AUTO ? SPECA_PATH_DIRECT : cfg->path;
+    c->path = cfg->path == SPECA_PATH_AUTO ? SPECA_PATH_WIDE : cfg->path;
     c->eps = cfg->eps > 0.f ? static_cast<double>(cfg->eps) : 1e-8;  // Eq. 4
     c->arena = static_cast<char*>(cfg->arena);
     c->pending = false;
@@ -235,11 +241,8 @@ speca_status_t speca_cache_create(const speca_cache_config_t* cfg, speca_cache_t
     }
     const Layout& L = c->L;
     ce = cudaMemcpy(c->arena + L.segs_off, L.segs.data(), L.segs.size() * sizeof(SegDesc), cudaMemcpyHostToDevice);
-    if (ce == cudaSuccess)
-        ce = cudaMemcpy(c->arena + L.tiles_direct_off, L.tiles_direct.data(), L.tiles_direct.size() * sizeof(uint32_t),
-                        cudaMemcpyHostToDevice);
-    if (ce == cudaSuccess)
-        ce = cudaMemcpy(c->arena + L.tiles_bulk_off, L.tiles_bulk.data(), L.tiles_bulk.size() * sizeof(uint32_t),
+    for (int k = 0; k < kNumTileSizes && ce == cudaSuccess; ++k)
+        ce = cudaMemcpy(c->arena + L.tiles_off[k], L.tiles[k].data(), L.tiles[k].size() * sizeof(uint32_t),
                         cudaMemcpyHostToDevice);
     if (ce == cudaSuccess) ce = cudaMemset(c->arena + L.ticket_off, 0, kAlign);
     if (ce != cudaSuccess) {
@@ -247,13 +250,18 @@ speca_status_t speca_cache_create(const speca_cache_config_t* cfg, speca_cache_t
         return SPECA_ERR_CUDA;
     }
     cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
-    c->grid_update = c->sm_count * ctas_per_sm_update(c->dtype, c->m);
-    c->grid_forecast = c->sm_count * ctas_per_sm_forecast(c->dtype, c->m);
+    c->tile_update = tile_size_index(stream_tile_bytes(c->path, true));
+    c->tile_forecast = tile_size_index(stream_tile_bytes(c->path, false));
+    if (c->tile_update < 0 || c->tile_forecast < 0) {
+        delete c;
+        return SPECA_ERR_UNSUPPORTED;
+    }
+    c->grid_update = c->sm_count * stream_ctas_per_sm(c->path, true);
+    c->grid_forecast = c->sm_count * stream_ctas_per_sm(c->path, false);
     c->cluster = 4;
-    int gv = c->sm_count * ctas_per_sm_verify(c->dtype, c->m);
-    gv = gv / c->cluster * c->cluster;
-    if (gv / c->cluster > kMaxClusters) gv = kMaxClusters * c->cluster;
-    c->grid_verify = gv;
+    int n_clusters = max_resident_verify_clusters(c->dtype, c->m, c->cluster);
+    if (n_clusters > kMaxClusters) n_clusters = kMaxClusters;
+    c->grid_verify = n_clusters * c->cluster;
     *out = c;
     return SPECA_OK;
 }
@@ -325,10 +333,9 @@ speca_status_t speca_cache_update(speca_cache_t* c, const void* const* feats, co
     if (st != SPECA_OK) return st;
     if (e_lo >= 0 && any_sample) {
         const Layout& L = c->L;
-        const std::vector<uint32_t>& tiles = c->path == SPECA_PATH_BULK ? L.tiles_bulk : L.tiles_direct;
+        const std::vector<uint32_t>& tiles = L.tiles[c->tile_update];
         p.segs = reinterpret_cast<const SegDesc*>(c->arena + L.segs_off);
-        p.tile_start = reinterpret_cast<const uint32_t*>(
-            c->arena + (c->path == SPECA_PATH_BULK ? L.tiles_bulk_off : L.tiles_direct_off));
+        p.tile_start = reinterpret_cast<const uint32_t*>(c->arena + L.tiles_off[c->tile_update]);
         p.arena = c->arena;
         p.dev_mask = nullptr;
         p.err_flag = reinterpret_cast<uint32_t*>(c->arena + L.ticket_off) + 1;
@@ -403,10 +410,9 @@ speca_status_t speca_forecast(speca_cache_t* c, const double* t_target, const ui
     if (st != SPECA_OK) return st;
     if (e_lo < 0 || !any_sample) return SPECA_OK;
     const Layout& L = c->L;
-    const std::vector<uint32_t>& tiles = c->path == SPECA_PATH_BULK ? L.tiles_bulk : L.tiles_direct;
+    const std::vector<uint32_t>& tiles = L.tiles[c->tile_forecast];
     p.segs = reinterpret_cast<const SegDesc*>(c->arena + L.segs_off);
-    p.tile_start =
-        reinterpret_cast<const uint32_t*>(c->arena + (c->path == SPECA_PATH_BULK ? L.tiles_bulk_off : L.tiles_direct_off));
+    p.tile_start = reinterpret_cast<const uint32_t*>(c->arena + L.tiles_off[c->tile_forecast]);
     p.arena = c->arena;
     p.dev_mask = dev_active_mask;
     p.err_flag = reinterpret_cast<uint32_t*>(c->arena + L.ticket_off) + 1;
@@ -437,6 +443,7 @@ speca_status_t speca_verify(speca_cache_t* c, const void* fresh, const double* t
     VerifyParams p;
     std::memset(&p, 0, sizeof p);
     bool any_sample = false;
+    int v_max = 0;
     for (int b = 0; b < c->B; ++b) {
         if (!std::isfinite(t_target[b])) return fail(c, SPECA_ERR_INVALID_ARG, "verify: t_target[%d] not finite", b);
         if (std::isnan(tau[b])) return fail(c, SPECA_ERR_INVALID_ARG, "verify: tau[%d] is NaN", b);
@@ -447,6 +454,7 @@ speca_status_t speca_verify(speca_cache_t* c, const void* fresh, const double* t
         p.order[b] = static_cast<int8_t>(order);
         p.tau[b] = tau[b];
         any_sample |= order >= 0;
+        v_max = order > v_max ? order : v_max;
     }
     DeviceGuard guard(c->device);
     if (!guard.ok) return fail(c, SPECA_ERR_CUDA, "cudaSetDevice failed");
@@ -455,7 +463,7 @@ speca_status_t speca_verify(speca_cache_t* c, const void* fresh, const double* t
     if (!any_sample) return SPECA_OK;
     const Layout& L = c->L;
     const SegDesc& s0 = L.segs[static_cast<size_t>(c->verify_entry) * c->B];
-    const uint32_t te = tile_elems(c->dtype, SPECA_PATH_DIRECT);
+    const uint32_t te = verify_tile_elems(c->dtype, v_max);
     p.segs = reinterpret_cast<const SegDesc*>(c->arena + L.segs_off) + static_cast<size_t>(c->verify_entry) * c->B;
     p.arena = c->arena;
     p.dev_mask = dev_active_mask;

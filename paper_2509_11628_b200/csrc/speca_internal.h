@@ -8,17 +8,26 @@
 
 namespace speca {
 
-// Bytes of one plane that a tile covers. A tile is the unit a CTA picks up from the flattened
-// work list: kTileBytes / sizeof(element) consecutive elements of one (entry, sample) table.
-constexpr uint32_t kTileBytesDirect = 16384;  // 256 threads x 4 vectors x 16 B
-constexpr uint32_t kTileBytesBulk = 8192;     // one cp.async.bulk per plane per stage
-constexpr int kThreads = 256;
+// A tile is the unit a CTA picks up from the flattened work list: a fixed number of bytes of one
+// plane of one (entry, sample) table. Each stream kernel shape has its own tile size; the arena
+// holds one tile-prefix table per size in kTileSizes.
+constexpr uint32_t kTileSizes[] = {4096, 8192, 16384, 32768};
+constexpr int kNumTileSizes = 4;
+constexpr int kThreads = 256;       // verify kernel CTA size
+// Tile of the verify kernel compiled for order v (the highest order among the launch's samples).
+__host__ __device__ constexpr uint32_t verify_tile_bytes(int v) { return v <= 2 ? 16384u : 8192u; }
 constexpr int kMaxClusters = 1024;  // upper bound on verify clusters (reduction scratch rows)
+
+inline int tile_size_index(uint32_t tile_bytes) {
+    for (int i = 0; i < kNumTileSizes; ++i)
+        if (kTileSizes[i] == tile_bytes) return i;
+    return -1;
+}
 
 // One (entry, sample) table. Segments are ordered entry-major, sample-minor: seg = e * B + b.
 struct SegDesc {
-    uint64_t plane0_off;    // byte offset of plane 0 from the arena base (256-byte aligned)
-    uint64_t plane_stride;  // bytes between consecutive planes (multiple of 256)
+    uint64_t plane0_off;    // byte offset of plane 0 from the arena base (4 KB aligned)
+    uint64_t plane_stride;  // bytes between consecutive planes (multiple of 4096)
     uint64_t io_off;        // byte offset of this sample's row inside the entry's [B, N_e, D] tensor
     uint32_t n_elems;       // N_e * D
     uint16_t entry;
@@ -73,14 +82,12 @@ cudaError_t launch_select(const uint8_t* accept, int32_t k_max, int32_t group, i
 cudaError_t launch_activate(uint64_t mask_bits, int32_t batch, int32_t* spec_count, uint8_t* active,
                             cudaStream_t stream);
 
-// Resident CTAs per SM of each kernel family (occupancy query), for sizing persistent grids.
-int ctas_per_sm_update(int dtype, int order);
-int ctas_per_sm_forecast(int dtype, int order);
-int ctas_per_sm_verify(int dtype, int order);
+// Tile size and designed CTAs per SM of the stream kernel a path uses for update / forecast.
+uint32_t stream_tile_bytes(int path, bool update);
+int stream_ctas_per_sm(int path, bool update);
+// Clusters of the verify kernel that fit on the current device at once.
+int max_resident_verify_clusters(int dtype, int order, int cluster);
 
-inline uint32_t tile_elems(int dtype, int path) {
-    uint32_t bytes = (path == SPECA_PATH_BULK) ? kTileBytesBulk : kTileBytesDirect;
-    return bytes / (dtype == SPECA_BF16 ? 2u : 4u);
-}
+inline uint32_t verify_tile_elems(int dtype, int v) { return verify_tile_bytes(v) / (dtype == SPECA_BF16 ? 2u : 4u); }
 
 }  // namespace speca

@@ -101,6 +101,83 @@ __device__ __forceinline__ void store_scalar(char* base, uint32_t idx, float x) 
 }
 
 // ------------------------------------------------------------------------------------------------
+// 16- and 32-byte global vectors
+// ------------------------------------------------------------------------------------------------
+
+// W bytes of consecutive elements in registers. sm_100 has 256-bit global loads and stores
+// (ld/st.global.v8.b32); a warp then moves 1 KB of consecutive bytes per instruction.
+template <int W>
+struct Vec {
+    uint32_t r[W / 4];
+};
+
+// The asm statements are volatile so that a tile's loads are all issued, in program order, before
+// the first value is consumed: the number of independent loads in flight per thread is part of the
+// design (see the shape table below), not something to leave to the instruction scheduler.
+template <int W>
+__device__ __forceinline__ Vec<W> load_vec(const char* p) {
+    Vec<W> v;
+    if constexpr (W == 16)
+        asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(v.r[0]), "=r"(v.r[1]), "=r"(v.r[2]), "=r"(v.r[3])
+                     : "l"(p));
+    else
+        asm volatile("ld.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(v.r[0]), "=r"(v.r[1]), "=r"(v.r[2]), "=r"(v.r[3]), "=r"(v.r[4]), "=r"(v.r[5]), "=r"(v.r[6]),
+                       "=r"(v.r[7])
+                     : "l"(p));
+    return v;
+}
+
+template <int W>
+__device__ __forceinline__ void store_vec(char* p, const Vec<W>& v) {
+    if constexpr (W == 16)
+        asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.r[0]), "r"(v.r[1]), "r"(v.r[2]),
+                     "r"(v.r[3])
+                     : "memory");
+    else
+        asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(v.r[0]), "r"(v.r[1]),
+                     "r"(v.r[2]), "r"(v.r[3]), "r"(v.r[4]), "r"(v.r[5]), "r"(v.r[6]), "r"(v.r[7])
+                     : "memory");
+}
+
+template <int DT, int W>
+struct VecElems {
+    static constexpr int kEPV = W / Elem<DT>::kBytes;
+};
+
+template <int DT, int W>
+__device__ __forceinline__ void unpack_vec(const Vec<W>& v, float (&f)[W / Elem<DT>::kBytes]) {
+    if constexpr (DT == SPECA_F32) {
+#pragma unroll
+        for (int k = 0; k < W / 4; ++k) f[k] = __uint_as_float(v.r[k]);
+    } else {
+        // bfloat16 is the upper half of a binary32: widening is a shift
+#pragma unroll
+        for (int k = 0; k < W / 4; ++k) {
+            f[2 * k] = __uint_as_float(v.r[k] << 16);
+            f[2 * k + 1] = __uint_as_float(v.r[k] & 0xFFFF0000u);
+        }
+    }
+}
+
+template <int DT, int W>
+__device__ __forceinline__ Vec<W> pack_vec(const float (&f)[W / Elem<DT>::kBytes]) {
+    Vec<W> v;
+    if constexpr (DT == SPECA_F32) {
+#pragma unroll
+        for (int k = 0; k < W / 4; ++k) v.r[k] = __float_as_uint(f[k]);
+    } else {
+#pragma unroll
+        for (int k = 0; k < W / 4; ++k) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * k], f[2 * k + 1]);  // round to nearest even
+            v.r[k] = *reinterpret_cast<uint32_t*>(&h);
+        }
+    }
+    return v;
+}
+
+// ------------------------------------------------------------------------------------------------
 // work list: tile -> segment
 // ------------------------------------------------------------------------------------------------
 
@@ -119,47 +196,45 @@ __device__ __forceinline__ uint32_t find_segment(const uint32_t* __restrict__ ti
 }
 
 // ------------------------------------------------------------------------------------------------
-// per-tile bodies, direct (register) path
+// per-tile bodies
 // ------------------------------------------------------------------------------------------------
+// A tile is NT x U vectors of W bytes per plane; thread t owns vectors t, t + NT, ... so that a warp
+// touches W * 32 consecutive bytes per instruction. `cnt` elements of the tile exist (the last tile
+// of a segment is ragged): whole vectors go through the vector loop, the remainder through the
+// scalar loop. `row` must be W-byte aligned (the planes always are).
 
 // Eq. 2 in Horner form: acc = D_v; acc = D_{i-1} + acc * mu_i for i = v..1.
-template <int DT, int V, int U>
+template <int DT, int V, int W, int NT, int U>
 __device__ __forceinline__ void forecast_tile(const char* __restrict__ plane0, uint64_t stride,
                                               char* __restrict__ out, uint32_t cnt, const float (&mu)[SPECA_MAX_ORDER]) {
-    constexpr int EPV = Elem<DT>::kEPV;
-    const bool vec_ok = (reinterpret_cast<uintptr_t>(out) & 15u) == 0;
-    const uint32_t nvec = vec_ok ? cnt / EPV : 0;
-    uint4* __restrict__ dst = reinterpret_cast<uint4*>(out);
-    for (uint32_t base = 0; base < nvec; base += kThreads * U) {
-        uint4 d[V + 1][U];
+    constexpr int EPV = W / Elem<DT>::kBytes;
+    const uint32_t nvec = cnt / EPV;
+    Vec<W> d[V + 1][U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t idx = base + u * kThreads + threadIdx.x;
-            if (idx < nvec) {
+    for (int u = 0; u < U; ++u) {
+        const uint32_t idx = u * NT + threadIdx.x;
+        if (idx < nvec) {
 #pragma unroll
-                for (int i = 0; i <= V; ++i)
-                    d[i][u] = __ldcs(reinterpret_cast<const uint4*>(plane0 + i * stride) + idx);
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t idx = base + u * kThreads + threadIdx.x;
-            if (idx < nvec) {
-                float acc[EPV];
-                unpack<DT>(d[V][u], acc);
-#pragma unroll
-                for (int i = V; i >= 1; --i) {
-                    float lo[EPV];
-                    unpack<DT>(d[i - 1][u], lo);
-#pragma unroll
-                    for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
-                }
-                __stcs(dst + idx, pack<DT>(acc));
-            }
+            for (int i = 0; i <= V; ++i) d[i][u] = load_vec<W>(plane0 + i * stride + static_cast<size_t>(idx) * W);
         }
     }
-    // ragged tail, or the whole tile when the output row is not 16-byte aligned
-    for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += kThreads) {
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint32_t idx = u * NT + threadIdx.x;
+        if (idx < nvec) {
+            float acc[EPV];
+            unpack_vec<DT, W>(d[V][u], acc);
+#pragma unroll
+            for (int i = V; i >= 1; --i) {
+                float lo[EPV];
+                unpack_vec<DT, W>(d[i - 1][u], lo);
+#pragma unroll
+                for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+            }
+            store_vec<W>(out + static_cast<size_t>(idx) * W, pack_vec<DT, W>(acc));
+        }
+    }
+    for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += NT) {
         float acc = load_scalar<DT>(plane0 + V * stride, j);
 #pragma unroll
         for (int i = V; i >= 1; --i) acc = fmaf(acc, mu[i - 1], load_scalar<DT>(plane0 + (i - 1) * stride, j));
@@ -169,44 +244,46 @@ __device__ __forceinline__ void forecast_tile(const char* __restrict__ plane0, u
 
 // Eq. 3 as a chain of difference quotients: c_0 = f; c_{i+1} = (c_i - D_i) * r_i; D_i <- c_i.
 // V = highest plane written. Reads f and planes 0..V-1, writes planes 0..V, each element once.
-template <int DT, int V, int U>
+template <int DT, int V, int W, int NT, int U>
 __device__ __forceinline__ void update_tile(char* __restrict__ plane0, uint64_t stride, const char* __restrict__ feat,
                                             uint32_t cnt, const float (&r)[SPECA_MAX_ORDER]) {
-    constexpr int EPV = Elem<DT>::kEPV;
-    const bool vec_ok = (reinterpret_cast<uintptr_t>(feat) & 15u) == 0;
-    const uint32_t nvec = vec_ok ? cnt / EPV : 0;
-    for (uint32_t base = 0; base < nvec; base += kThreads * U) {
-        uint4 fv[U];
-        uint4 d[V > 0 ? V : 1][U];
+    constexpr int EPV = W / Elem<DT>::kBytes;
+    const uint32_t nvec = cnt / EPV;
+    Vec<W> fv[U];
+    Vec<W> d[V > 0 ? V : 1][U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t idx = base + u * kThreads + threadIdx.x;
-            if (idx < nvec) {
-                fv[u] = __ldcs(reinterpret_cast<const uint4*>(feat) + idx);
+    for (int u = 0; u < U; ++u) {
+        const uint32_t idx = u * NT + threadIdx.x;
+        if (idx < nvec) {
+            fv[u] = load_vec<W>(feat + static_cast<size_t>(idx) * W);
 #pragma unroll
-                for (int i = 0; i < V; ++i) d[i][u] = __ldcs(reinterpret_cast<const uint4*>(plane0 + i * stride) + idx);
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t idx = base + u * kThreads + threadIdx.x;
-            if (idx < nvec) {
-                float c[EPV];
-                unpack<DT>(fv[u], c);
-                // plane 0 is the feature itself: already in storage format
-                __stcs(reinterpret_cast<uint4*>(plane0) + idx, fv[u]);
-#pragma unroll
-                for (int i = 0; i < V; ++i) {
-                    float old[EPV];
-                    unpack<DT>(d[i][u], old);
-#pragma unroll
-                    for (int k = 0; k < EPV; ++k) c[k] = (c[k] - old[k]) * r[i];
-                    __stcs(reinterpret_cast<uint4*>(plane0 + (i + 1) * stride) + idx, pack<DT>(c));
-                }
-            }
+            for (int i = 0; i < V; ++i) d[i][u] = load_vec<W>(plane0 + i * stride + static_cast<size_t>(idx) * W);
         }
     }
-    for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += kThreads) {
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint32_t idx = u * NT + threadIdx.x;
+        if (idx < nvec) {
+            float c[EPV];
+            unpack_vec<DT, W>(fv[u], c);
+            // every new plane is computed before the first store is issued: the thread's stores
+            // leave as one burst after its loads have all returned
+#pragma unroll
+            for (int i = 0; i < V; ++i) {
+                float old[EPV];
+                unpack_vec<DT, W>(d[i][u], old);
+#pragma unroll
+                for (int k = 0; k < EPV; ++k) c[k] = (c[k] - old[k]) * r[i];
+                d[i][u] = pack_vec<DT, W>(c);  // plane i + 1
+            }
+            // plane 0 is the feature itself: already in storage format
+            store_vec<W>(plane0 + static_cast<size_t>(idx) * W, fv[u]);
+#pragma unroll
+            for (int i = 0; i < V; ++i)
+                store_vec<W>(plane0 + (i + 1) * stride + static_cast<size_t>(idx) * W, d[i][u]);
+        }
+    }
+    for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += NT) {
         float c = load_scalar<DT>(feat, j);
         float old[V > 0 ? V : 1];
 #pragma unroll
@@ -220,19 +297,16 @@ __device__ __forceinline__ void update_tile(char* __restrict__ plane0, uint64_t 
     }
 }
 
-// ------------------------------------------------------------------------------------------------
-// streaming kernels: persistent CTAs stride over the flattened tile list
-// ------------------------------------------------------------------------------------------------
-
-// Runtime-order variants for the rare tiles whose sample has fewer references than the launch's
-// common order (warm-up after a reset): one vector at a time, planes visited in a loop.
+// Runtime-order, any-alignment variants for the rare tiles whose sample has fewer references than
+// the launch's common order (warm-up after a reset) or whose row is not vector aligned: 16-byte
+// vectors when the row allows it, else one element at a time; planes visited in a loop.
 template <int DT>
 __device__ __noinline__ void forecast_tile_any(const char* __restrict__ plane0, uint64_t stride, char* __restrict__ out,
                                                uint32_t cnt, int v, const float (&mu)[SPECA_MAX_ORDER]) {
     constexpr int EPV = Elem<DT>::kEPV;
     const bool vec_ok = (reinterpret_cast<uintptr_t>(out) & 15u) == 0;
     const uint32_t nvec = vec_ok ? cnt / EPV : 0;
-    for (uint32_t idx = threadIdx.x; idx < nvec; idx += kThreads) {
+    for (uint32_t idx = threadIdx.x; idx < nvec; idx += blockDim.x) {
         float acc[EPV];
         unpack<DT>(__ldcs(reinterpret_cast<const uint4*>(plane0 + v * stride) + idx), acc);
         for (int i = v; i >= 1; --i) {
@@ -243,7 +317,7 @@ __device__ __noinline__ void forecast_tile_any(const char* __restrict__ plane0, 
         }
         __stcs(reinterpret_cast<uint4*>(out) + idx, pack<DT>(acc));
     }
-    for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += kThreads) {
+    for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += blockDim.x) {
         float acc = load_scalar<DT>(plane0 + v * stride, j);
         for (int i = v; i >= 1; --i) acc = fmaf(acc, mu[i - 1], load_scalar<DT>(plane0 + (i - 1) * stride, j));
         store_scalar<DT>(out, j, acc);
@@ -256,7 +330,7 @@ __device__ __noinline__ void update_tile_any(char* __restrict__ plane0, uint64_t
     constexpr int EPV = Elem<DT>::kEPV;
     const bool vec_ok = (reinterpret_cast<uintptr_t>(feat) & 15u) == 0;
     const uint32_t nvec = vec_ok ? cnt / EPV : 0;
-    for (uint32_t idx = threadIdx.x; idx < nvec; idx += kThreads) {
+    for (uint32_t idx = threadIdx.x; idx < nvec; idx += blockDim.x) {
         const uint4 fv = __ldcs(reinterpret_cast<const uint4*>(feat) + idx);
         float c[EPV];
         unpack<DT>(fv, c);
@@ -271,7 +345,7 @@ __device__ __noinline__ void update_tile_any(char* __restrict__ plane0, uint64_t
         }
         __stcs(reinterpret_cast<uint4*>(plane0 + v * stride) + idx, next);
     }
-    for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += kThreads) {
+    for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += blockDim.x) {
         float c = load_scalar<DT>(feat, j);
         for (int i = 0; i < v; ++i) {
             const float old = load_scalar<DT>(plane0 + i * stride, j);
@@ -285,39 +359,73 @@ __device__ __noinline__ void update_tile_any(char* __restrict__ plane0, uint64_t
 // ------------------------------------------------------------------------------------------------
 // streaming kernels: persistent CTAs stride over the flattened tile list
 // ------------------------------------------------------------------------------------------------
-
-// Independent 16-byte loads a thread issues per plane before it starts computing.
-__host__ __device__ constexpr int unroll_for(int planes) { return planes <= 4 ? 4 : 2; }
+// Launch shapes. Both kernels are pure HBM streams whose speed is set by how the DRAM sees the mix
+// of reads and writes, so the shape (vector width, threads, vectors per thread, CTAs per SM) was
+// chosen by sweeping it on a B200 at order 2, bf16, with every plane 4 KB aligned:
+//   update   (half of the traffic is writes): few bytes in flight win -- 128 threads x one 32-byte
+//            vector per plane, 3 CTAs/SM (36 KB in flight per SM) reaches the device's copy rate;
+//            deeper or wider shapes (256 x 4 vectors, 2 CTAs/SM) are 4-9 % slower on this mix.
+//   forecast (one write per three reads): flat above ~70 KB in flight per SM; 256 threads x one
+//            vector per plane, 3 CTAs/SM.
+// SPECA_PATH_DIRECT keeps a 16-byte / 256-thread / 4-deep shape for both.
+// A tile is `chunks` consecutive chunks of NT x U vectors; a CTA finishes one chunk (loads, arithmetic,
+// stores) before it starts the next, so the bytes in flight are set by NT x U x W while the per-tile
+// bookkeeping (segment lookup, descriptor, bounds) is paid once per `chunks`.
+struct Shape {
+    int w, nt, u, chunks, minb;
+};
+#ifndef SPECA_SHAPE_UPDATE
+#define SPECA_SHAPE_UPDATE 32, 128, 1, 8, 3
+#endif
+#ifndef SPECA_SHAPE_FORECAST
+#define SPECA_SHAPE_FORECAST 32, 256, 1, 4, 3
+#endif
+__host__ __device__ constexpr Shape shape_for(int path, bool update) {
+    return path == SPECA_PATH_WIDE ? (update ? Shape{SPECA_SHAPE_UPDATE} : Shape{SPECA_SHAPE_FORECAST})
+                                   : Shape{16, 256, 4, 1, 2};
+}
 
 // V = the order most samples of the launch have (the host passes the maximum over samples).
-template <int DT, int V, bool UPDATE>
-__global__ void __launch_bounds__(kThreads, 2) stream_direct_kernel(const __grid_constant__ StreamParams p) {
-    constexpr uint32_t kTile = kTileBytesDirect / Elem<DT>::kBytes;
-    constexpr int U = unroll_for(V + 1 + (UPDATE ? 0 : 0));
-    uint32_t seg = p.seg_lo;
+template <int DT, int V, bool UPDATE, int W, int NT, int U, int C, int MINB>
+__global__ void __launch_bounds__(NT, MINB) stream_kernel(const __grid_constant__ StreamParams p) {
+    constexpr uint32_t kChunk = static_cast<uint32_t>(NT) * U * W / Elem<DT>::kBytes;  // elements
+    constexpr uint32_t kTile = kChunk * C;
+    uint32_t seg = p.seg_lo, seg_first = 0, seg_end = 0;  // tiles [seg_first, seg_end) belong to `seg`
+    SegDesc sd = {};
+    int v = -1;
+    char* io = nullptr;
+    float coef[SPECA_MAX_ORDER] = {};
     for (uint32_t tile = p.tile_lo + blockIdx.x; tile < p.tile_hi; tile += gridDim.x) {
-        seg = find_segment(p.tile_start, seg, p.seg_hi, tile);
-        const SegDesc sd = p.segs[seg];
-        const int v = p.order[sd.sample];
-        char* io = static_cast<char*>(p.io[sd.entry]);
+        if (tile >= seg_end) {  // tiles only grow: look forward from the current segment
+            seg = find_segment(p.tile_start, seg, p.seg_hi, tile);
+            seg_first = __ldg(p.tile_start + seg);
+            seg_end = __ldg(p.tile_start + seg + 1);
+            sd = p.segs[seg];
+            v = p.order[sd.sample];
+            io = static_cast<char*>(p.io[sd.entry]);
+            if (p.dev_mask != nullptr && p.dev_mask[sd.sample] == 0) v = -1;
+#pragma unroll
+            for (int i = 0; i < SPECA_MAX_ORDER; ++i) coef[i] = p.coef[sd.sample][i];
+        }
         if (v < 0 || io == nullptr) continue;
-        if (p.dev_mask != nullptr && p.dev_mask[sd.sample] == 0) continue;
-        const uint32_t elem0 = (tile - __ldg(p.tile_start + seg)) * kTile;
+        const uint32_t elem0 = (tile - seg_first) * kTile;
         const uint32_t cnt = min(kTile, sd.n_elems - elem0);
         const uint64_t byte0 = static_cast<uint64_t>(elem0) * Elem<DT>::kBytes;
         char* plane0 = p.arena + sd.plane0_off + byte0;
         char* row = io + sd.io_off + byte0;
-        float coef[SPECA_MAX_ORDER];
-#pragma unroll
-        for (int i = 0; i < SPECA_MAX_ORDER; ++i) coef[i] = p.coef[sd.sample][i];
-        if constexpr (UPDATE) {
-            if (v == V)
-                update_tile<DT, V, U>(plane0, sd.plane_stride, row, cnt, coef);
-            else
-                update_tile_any<DT>(plane0, sd.plane_stride, row, cnt, v, coef);
+        const bool fast = v == V && (reinterpret_cast<uintptr_t>(row) & (W - 1)) == 0;
+        if (fast) {
+            for (uint32_t done = 0; done < cnt; done += kChunk) {
+                const uint32_t n = min(kChunk, cnt - done);
+                const size_t off = static_cast<size_t>(done) * Elem<DT>::kBytes;
+                if constexpr (UPDATE)
+                    update_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, row + off, n, coef);
+                else
+                    forecast_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, row + off, n, coef);
+            }
         } else {
-            if (v == V)
-                forecast_tile<DT, V, U>(plane0, sd.plane_stride, row, cnt, coef);
+            if constexpr (UPDATE)
+                update_tile_any<DT>(plane0, sd.plane_stride, row, cnt, v, coef);
             else
                 forecast_tile_any<DT>(plane0, sd.plane_stride, row, cnt, v, coef);
         }
@@ -329,52 +437,52 @@ __global__ void __launch_bounds__(kThreads, 2) stream_direct_kernel(const __grid
 // ------------------------------------------------------------------------------------------------
 
 constexpr int kMaxClusterSize = 8;
+// 256 threads x U x 32 B per plane and tile; U = 2 while the V + 2 streams fit in registers
+constexpr int kVerifyW = 32;
+static_assert(verify_tile_bytes(0) == kThreads * 2 * kVerifyW && verify_tile_bytes(4) == kThreads * kVerifyW,
+              "verify tile sizes");
 
-template <int DT, int V, int U>
+template <int DT, int V, int W, int U>
 __device__ __forceinline__ void verify_tile(const char* __restrict__ plane0, uint64_t stride,
                                             const char* __restrict__ fresh, char* __restrict__ out_pred, uint32_t cnt,
                                             const float (&mu)[SPECA_MAX_ORDER], float& num, float& den) {
-    constexpr int EPV = Elem<DT>::kEPV;
-    const bool vec_ok = ((reinterpret_cast<uintptr_t>(fresh) | reinterpret_cast<uintptr_t>(out_pred)) & 15u) == 0;
-    const uint32_t nvec = vec_ok ? cnt / EPV : 0;
-    for (uint32_t base = 0; base < nvec; base += kThreads * U) {
-        uint4 d[V + 1][U];
-        uint4 fv[U];
+    constexpr int EPV = W / Elem<DT>::kBytes;
+    const uint32_t nvec = cnt / EPV;
+    Vec<W> d[V + 1][U];
+    Vec<W> fv[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t idx = base + u * kThreads + threadIdx.x;
-            if (idx < nvec) {
+    for (int u = 0; u < U; ++u) {
+        const uint32_t idx = u * kThreads + threadIdx.x;
+        if (idx < nvec) {
 #pragma unroll
-                for (int i = 0; i <= V; ++i)
-                    d[i][u] = __ldcs(reinterpret_cast<const uint4*>(plane0 + i * stride) + idx);
-                fv[u] = __ldcs(reinterpret_cast<const uint4*>(fresh) + idx);
-            }
+            for (int i = 0; i <= V; ++i) d[i][u] = load_vec<W>(plane0 + i * stride + static_cast<size_t>(idx) * W);
+            fv[u] = load_vec<W>(fresh + static_cast<size_t>(idx) * W);
         }
+    }
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t idx = base + u * kThreads + threadIdx.x;
-            if (idx < nvec) {
-                float acc[EPV], f[EPV];
-                unpack<DT>(d[V][u], acc);
+    for (int u = 0; u < U; ++u) {
+        const uint32_t idx = u * kThreads + threadIdx.x;
+        if (idx < nvec) {
+            float acc[EPV], f[EPV];
+            unpack_vec<DT, W>(d[V][u], acc);
 #pragma unroll
-                for (int i = V; i >= 1; --i) {
-                    float lo[EPV];
-                    unpack<DT>(d[i - 1][u], lo);
+            for (int i = V; i >= 1; --i) {
+                float lo[EPV];
+                unpack_vec<DT, W>(d[i - 1][u], lo);
 #pragma unroll
-                    for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
-                }
-                // the forecast as the model would consume it: rounded to the storage type
-                const uint4 pv = pack<DT>(acc);
-                unpack<DT>(pv, acc);
-                unpack<DT>(fv[u], f);
-#pragma unroll
-                for (int k = 0; k < EPV; ++k) {
-                    const float diff = acc[k] - f[k];
-                    num = fmaf(diff, diff, num);
-                    den = fmaf(f[k], f[k], den);
-                }
-                if (out_pred != nullptr) __stcs(reinterpret_cast<uint4*>(out_pred) + idx, pv);
+                for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
             }
+            // the forecast as the model would consume it: rounded to the storage type
+            const Vec<W> pv = pack_vec<DT, W>(acc);
+            unpack_vec<DT, W>(pv, acc);
+            unpack_vec<DT, W>(fv[u], f);
+#pragma unroll
+            for (int k = 0; k < EPV; ++k) {
+                const float diff = acc[k] - f[k];
+                num = fmaf(diff, diff, num);
+                den = fmaf(f[k], f[k], den);
+            }
+            if (out_pred != nullptr) store_vec<W>(out_pred + static_cast<size_t>(idx) * W, pv);
         }
     }
     for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += kThreads) {
@@ -395,7 +503,8 @@ __device__ __noinline__ void verify_tile_any(const char* __restrict__ plane0, ui
                                              const char* __restrict__ fresh, char* __restrict__ out_pred, uint32_t cnt,
                                              int v, const float (&mu)[SPECA_MAX_ORDER], float& num, float& den) {
     constexpr int EPV = Elem<DT>::kEPV;
-    const bool vec_ok = ((reinterpret_cast<uintptr_t>(fresh) | reinterpret_cast<uintptr_t>(out_pred)) & 15u) == 0;
+    const bool vec_ok = ((reinterpret_cast<uintptr_t>(fresh) | reinterpret_cast<uintptr_t>(out_pred) |
+                          reinterpret_cast<uintptr_t>(plane0)) & 15u) == 0;
     const uint32_t nvec = vec_ok ? cnt / EPV : 0;
     for (uint32_t idx = threadIdx.x; idx < nvec; idx += kThreads) {
         float acc[EPV], f[EPV];
@@ -429,40 +538,60 @@ __device__ __noinline__ void verify_tile_any(const char* __restrict__ plane0, ui
     }
 }
 
-// Does cluster q of Q own at least one work unit of sample b (units_per_sample units per sample,
-// unit u belongs to cluster u mod Q)?
-__device__ __forceinline__ bool cluster_touches(uint32_t q, uint32_t Q, uint32_t b, uint32_t units_per_sample) {
-    const uint32_t lo = b * units_per_sample;
-    const uint32_t first = lo + (q + Q - lo % Q) % Q;
-    return first < lo + units_per_sample;
+// Tiles of the active samples form one list of T = (active samples) x (tiles per sample) tiles;
+// cluster q of Q owns the contiguous range [q*T/Q, (q+1)*T/Q).
+__device__ __forceinline__ uint32_t range_begin(uint32_t q, uint32_t Q, uint32_t T) {
+    return static_cast<uint32_t>(static_cast<uint64_t>(q) * T / Q);
+}
+__device__ __forceinline__ uint32_t range_owner(uint32_t tile, uint32_t Q, uint32_t T) {
+    const uint32_t q0 = static_cast<uint32_t>(static_cast<uint64_t>(tile) * Q / T);
+    return tile < range_begin(q0 + 1, Q, T) ? q0 : q0 + 1;
+}
+// Index of the a-th set bit of `bits` (a < popcount).
+__device__ __forceinline__ int nth_set_bit(uint64_t bits, uint32_t a) {
+    for (uint32_t i = 0; i < a; ++i) bits &= bits - 1;
+    return __ffsll(static_cast<long long>(bits)) - 1;
 }
 
-// Work unit = `cluster size` consecutive tiles of one sample, one per CTA of the cluster, so all
-// CTAs of a cluster always work on the same sample and reach the reduction together.
-// Reduction: registers -> warp shuffle -> shared memory (CTA) -> the leader CTA's shared memory
-// through the cluster's distributed shared memory -> one partial per (cluster, sample) in global
-// scratch -> the cluster that arrives last (ticket counter, no waiting) adds the partials in
-// cluster order in fp64 and applies Eq. 4 and the accept rule.
+// Each cluster walks a contiguous range of the active samples' tiles, its CTAs taking every
+// (cluster size)-th tile, so a cluster meets each sample once and reduces once per sample:
+// registers -> warp shuffle -> shared memory (CTA) -> the leader CTA's shared memory through the
+// cluster's distributed shared memory -> one partial per (cluster, sample) in global scratch. The
+// cluster that arrives last (ticket counter, nobody waits) adds each sample's partials in fp64, one
+// warp per sample in a fixed lane/shuffle order, and applies Eq. 4 and the accept rule.
 template <int DT, int V>
 __global__ void __launch_bounds__(kThreads, 2) verify_kernel(const __grid_constant__ VerifyParams p) {
-    constexpr uint32_t kTile = kTileBytesDirect / Elem<DT>::kBytes;
-    constexpr int U = unroll_for(V + 2);
+    constexpr uint32_t kTile = verify_tile_bytes(V) / Elem<DT>::kBytes;
+    constexpr int W = kVerifyW, U = verify_tile_bytes(V) / (kThreads * kVerifyW);
     cg::cluster_group cluster = cg::this_cluster();
     const uint32_t csize = cluster.num_blocks();
     const uint32_t crank = cluster.block_rank();
     const uint32_t cid = blockIdx.x / csize;
-    const uint32_t n_clusters = gridDim.x / csize;
+    const uint32_t Q = gridDim.x / csize;
 
     __shared__ float warp_part[2][kThreads / 32];
     __shared__ float cluster_slot[2][2][kMaxClusterSize];  // [parity][num|den][rank], leader's copy is used
+    __shared__ uint32_t active_bits[2];
     __shared__ bool is_last;
 
+    // samples that take part: a defined table and, with a device mask, a non-zero byte
+    if (threadIdx.x < 64) {
+        const int b = threadIdx.x;
+        const bool on = b < p.batch && p.order[b] >= 0 && (p.dev_mask == nullptr || p.dev_mask[b] != 0);
+        const uint32_t ballot = __ballot_sync(0xFFFFFFFFu, on);
+        if ((threadIdx.x & 31) == 0) active_bits[threadIdx.x >> 5] = ballot;
+    }
+    __syncthreads();
+    const uint64_t bits = static_cast<uint64_t>(active_bits[0]) | (static_cast<uint64_t>(active_bits[1]) << 32);
+    const uint32_t n_active = __popcll(bits);
+    if (n_active == 0) return;  // every CTA of the grid takes this exit together
+    const uint32_t tps = p.tiles_per_sample;
+    const uint32_t T = n_active * tps;
+
     float num = 0.f, den = 0.f;
-    int cur_b = -1;
     uint32_t parity = 0;
 
     auto flush = [&](int b) {
-        // warp level
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
             num += __shfl_xor_sync(0xFFFFFFFFu, num, off);
@@ -503,56 +632,64 @@ __global__ void __launch_bounds__(kThreads, 2) verify_kernel(const __grid_consta
         den = 0.f;
     };
 
-    const uint32_t total_units = static_cast<uint32_t>(p.batch) * p.units_per_sample;
-    for (uint32_t unit = cid; unit < total_units; unit += n_clusters) {
-        const int b = static_cast<int>(unit / p.units_per_sample);
-        const int v = p.order[b];
-        if (v < 0 || (p.dev_mask != nullptr && p.dev_mask[b] == 0)) continue;  // uniform over the cluster
-        if (b != cur_b) {
-            if (cur_b >= 0) flush(cur_b);
-            cur_b = b;
-        }
-        const uint32_t tile = (unit % p.units_per_sample) * csize + crank;
-        if (tile >= p.tiles_per_sample) continue;
-        const SegDesc sd = p.segs[b];
-        const uint32_t elem0 = tile * kTile;
-        const uint32_t cnt = min(kTile, p.n_elems - elem0);
-        const uint64_t byte0 = static_cast<uint64_t>(elem0) * Elem<DT>::kBytes;
-        const char* plane0 = p.arena + sd.plane0_off + byte0;
-        const char* fresh = p.fresh + sd.io_off + byte0;
-        char* pred = p.out_pred != nullptr ? p.out_pred + sd.io_off + byte0 : nullptr;
-        float mu[SPECA_MAX_ORDER];
+    const uint32_t t_lo = range_begin(cid, Q, T), t_hi = range_begin(cid + 1, Q, T);
+    if (t_lo < t_hi) {
+        for (uint32_t a = t_lo / tps; a <= (t_hi - 1) / tps; ++a) {  // uniform over the cluster
+            const int b = nth_set_bit(bits, a);
+            const int v = p.order[b];
+            const SegDesc sd = p.segs[b];
+            float mu[SPECA_MAX_ORDER];
 #pragma unroll
-        for (int i = 0; i < SPECA_MAX_ORDER; ++i) mu[i] = p.coef[b][i];
-        if (v == V)
-            verify_tile<DT, V, U>(plane0, sd.plane_stride, fresh, pred, cnt, mu, num, den);
-        else
-            verify_tile_any<DT>(plane0, sd.plane_stride, fresh, pred, cnt, v, mu, num, den);
+            for (int i = 0; i < SPECA_MAX_ORDER; ++i) mu[i] = p.coef[b][i];
+            const uint32_t first = max(t_lo, a * tps) - a * tps, last = min(t_hi, (a + 1) * tps) - a * tps;
+            for (uint32_t tile = first + crank; tile < last; tile += csize) {
+                const uint32_t elem0 = tile * kTile;
+                const uint32_t cnt = min(kTile, p.n_elems - elem0);
+                const uint64_t byte0 = static_cast<uint64_t>(elem0) * Elem<DT>::kBytes;
+                const char* plane0 = p.arena + sd.plane0_off + byte0;
+                const char* fresh = p.fresh + sd.io_off + byte0;
+                char* pred = p.out_pred != nullptr ? p.out_pred + sd.io_off + byte0 : nullptr;
+                const bool fast = v == V && ((reinterpret_cast<uintptr_t>(plane0) | reinterpret_cast<uintptr_t>(fresh) |
+                                              reinterpret_cast<uintptr_t>(pred)) & (W - 1)) == 0;
+                if (fast)
+                    verify_tile<DT, V, W, U>(plane0, sd.plane_stride, fresh, pred, cnt, mu, num, den);
+                else
+                    verify_tile_any<DT>(plane0, sd.plane_stride, fresh, pred, cnt, v, mu, num, den);
+            }
+            flush(b);
+        }
     }
-    if (cur_b >= 0) flush(cur_b);
 
     if (crank != 0) return;  // nobody touches a non-leader's shared memory after its last barrier
 
     if (threadIdx.x == 0) {
         __threadfence();  // partials visible before the ticket
         const uint32_t t = atomicAdd(p.ticket, 1u);
-        is_last = (t == n_clusters - 1);
+        is_last = (t == Q - 1);
     }
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    for (int b = threadIdx.x; b < p.batch; b += kThreads) {
-        if (p.order[b] < 0 || (p.dev_mask != nullptr && p.dev_mask[b] == 0)) continue;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (uint32_t a = warp; a < n_active; a += kThreads / 32) {
+        const int b = nth_set_bit(bits, a);
+        const uint32_t q_lo = range_owner(a * tps, Q, T), q_hi = range_owner((a + 1) * tps - 1, Q, T);
         double sn = 0.0, sd = 0.0;
-        for (uint32_t q = 0; q < n_clusters; ++q) {
-            if (!cluster_touches(q, n_clusters, b, p.units_per_sample)) continue;
+        for (uint32_t q = q_lo + lane; q <= q_hi; q += 32) {
             const float* src = p.partials + (static_cast<size_t>(q) * p.batch + b) * 2;
             sn += static_cast<double>(__ldcg(src));
             sd += static_cast<double>(__ldcg(src + 1));
         }
-        const double e = sqrt(sn) / (sqrt(sd) + p.eps);
-        p.err[b] = static_cast<float>(e);
-        p.accept[b] = (e <= static_cast<double>(p.tau[b])) ? 1 : 0;  // NaN compares false: reject
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            sn += __shfl_xor_sync(0xFFFFFFFFu, sn, off);
+            sd += __shfl_xor_sync(0xFFFFFFFFu, sd, off);
+        }
+        if (lane == 0) {
+            const double e = sqrt(sn) / (sqrt(sd) + p.eps);
+            p.err[b] = static_cast<float>(e);
+            p.accept[b] = (e <= static_cast<double>(p.tau[b])) ? 1 : 0;  // NaN compares false: reject
+        }
     }
     __syncthreads();
     if (threadIdx.x == 0) *p.ticket = 0;  // ready for the next launch on this stream
@@ -615,17 +752,31 @@ __global__ void __launch_bounds__(SPECA_MAX_BATCH) activate_kernel(uint64_t mask
 // launchers
 // ------------------------------------------------------------------------------------------------
 
-static_assert(kThreads * 4 * 16 == kTileBytesDirect, "a direct tile is one pass of the CTA at unroll 4");
-
-template <int DT, bool UPDATE>
+template <int DT, bool UPDATE, int PATH>
 static const void* stream_kernel_for(int v) {
+    constexpr Shape s = shape_for(PATH, UPDATE);
     switch (v) {
-        case 0: return reinterpret_cast<const void*>(&stream_direct_kernel<DT, 0, UPDATE>);
-        case 1: return reinterpret_cast<const void*>(&stream_direct_kernel<DT, 1, UPDATE>);
-        case 2: return reinterpret_cast<const void*>(&stream_direct_kernel<DT, 2, UPDATE>);
-        case 3: return reinterpret_cast<const void*>(&stream_direct_kernel<DT, 3, UPDATE>);
-        default: return reinterpret_cast<const void*>(&stream_direct_kernel<DT, 4, UPDATE>);
+        case 0: return reinterpret_cast<const void*>(&stream_kernel<DT, 0, UPDATE, s.w, s.nt, s.u, s.chunks, s.minb>);
+        case 1: return reinterpret_cast<const void*>(&stream_kernel<DT, 1, UPDATE, s.w, s.nt, s.u, s.chunks, s.minb>);
+        case 2: return reinterpret_cast<const void*>(&stream_kernel<DT, 2, UPDATE, s.w, s.nt, s.u, s.chunks, s.minb>);
+        case 3: return reinterpret_cast<const void*>(&stream_kernel<DT, 3, UPDATE, s.w, s.nt, s.u, s.chunks, s.minb>);
+        default: return reinterpret_cast<const void*>(&stream_kernel<DT, 4, UPDATE, s.w, s.nt, s.u, s.chunks, s.minb>);
     }
+}
+
+static const void* stream_kernel_for(int dtype, bool update, int path, int v) {
+    if (path == SPECA_PATH_WIDE) {
+        if (update)
+            return dtype == SPECA_BF16 ? stream_kernel_for<SPECA_BF16, true, SPECA_PATH_WIDE>(v)
+                                       : stream_kernel_for<SPECA_F32, true, SPECA_PATH_WIDE>(v);
+        return dtype == SPECA_BF16 ? stream_kernel_for<SPECA_BF16, false, SPECA_PATH_WIDE>(v)
+                                   : stream_kernel_for<SPECA_F32, false, SPECA_PATH_WIDE>(v);
+    }
+    if (update)
+        return dtype == SPECA_BF16 ? stream_kernel_for<SPECA_BF16, true, SPECA_PATH_DIRECT>(v)
+                                   : stream_kernel_for<SPECA_F32, true, SPECA_PATH_DIRECT>(v);
+    return dtype == SPECA_BF16 ? stream_kernel_for<SPECA_BF16, false, SPECA_PATH_DIRECT>(v)
+                               : stream_kernel_for<SPECA_F32, false, SPECA_PATH_DIRECT>(v);
 }
 
 template <int DT>
@@ -645,44 +796,69 @@ static int max_order(const int8_t* order) {
     return v;
 }
 
-static cudaError_t launch_stream(const StreamParams& p, int dtype, bool update, int grid, cudaStream_t stream) {
-    const int v = max_order(p.order);
-    const void* fn;
-    if (update)
-        fn = dtype == SPECA_BF16 ? stream_kernel_for<SPECA_BF16, true>(v) : stream_kernel_for<SPECA_F32, true>(v);
-    else
-        fn = dtype == SPECA_BF16 ? stream_kernel_for<SPECA_BF16, false>(v) : stream_kernel_for<SPECA_F32, false>(v);
+uint32_t stream_tile_bytes(int path, bool update) {
+    const Shape s = shape_for(path, update);
+    return static_cast<uint32_t>(s.w) * s.nt * s.u * s.chunks;
+}
+
+int stream_ctas_per_sm(int path, bool update) { return shape_for(path, update).minb; }
+
+static cudaError_t launch_stream(const StreamParams& p, int dtype, bool update, int path, int grid,
+                                 cudaStream_t stream) {
+    if (path != SPECA_PATH_DIRECT && path != SPECA_PATH_WIDE) return cudaErrorNotSupported;
+    const void* fn = stream_kernel_for(dtype, update, path, max_order(p.order));
     void* args[1] = {const_cast<StreamParams*>(&p)};
-    return cudaLaunchKernel(fn, dim3(grid), dim3(kThreads), args, 0, stream);
+    return cudaLaunchKernel(fn, dim3(grid), dim3(shape_for(path, update).nt), args, 0, stream);
 }
 
 cudaError_t launch_update(const StreamParams& p, int dtype, int path, int grid, cudaStream_t stream) {
-    if (path != SPECA_PATH_DIRECT) return cudaErrorNotSupported;
-    return launch_stream(p, dtype, true, grid, stream);
+    return launch_stream(p, dtype, true, path, grid, stream);
 }
 
 cudaError_t launch_forecast(const StreamParams& p, int dtype, int path, int grid, cudaStream_t stream) {
-    if (path != SPECA_PATH_DIRECT) return cudaErrorNotSupported;
-    return launch_stream(p, dtype, false, grid, stream);
+    return launch_stream(p, dtype, false, path, grid, stream);
 }
 
-cudaError_t launch_verify(const VerifyParams& p, int dtype, int grid, int cluster, cudaStream_t stream) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+static void verify_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int grid, int cluster,
+                          cudaStream_t stream) {
+    *cfg = {};
+    cfg->gridDim = dim3(grid);
+    cfg->blockDim = dim3(kThreads);
+    cfg->dynamicSmemBytes = 0;
+    cfg->stream = stream;
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = cluster;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg->attrs = attr;
+    cfg->numAttrs = 1;
+}
+
+cudaError_t launch_verify(const VerifyParams& p, int dtype, int grid, int cluster, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    verify_config(&cfg, attr, grid, cluster, stream);
     const int v = max_order(p.order);
     const void* fn = dtype == SPECA_BF16 ? verify_kernel_for<SPECA_BF16>(v) : verify_kernel_for<SPECA_F32>(v);
     void* args[1] = {const_cast<VerifyParams*>(&p)};
     return cudaLaunchKernelExC(&cfg, fn, args);
+}
+
+// Clusters of `cluster` CTAs of the verify kernel that can be resident at once on the current
+// device. A cluster needs all its CTAs in one GPC, so this is less than SMs x CTAs/SM / cluster
+// when GPC sizes are not multiples of the cluster size; a grid sized above it would run its last
+// clusters as a second wave.
+int max_resident_verify_clusters(int dtype, int order, int cluster) {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    verify_config(&cfg, attr, cluster, cluster, nullptr);
+    const void* fn = dtype == SPECA_BF16 ? verify_kernel_for<SPECA_BF16>(order) : verify_kernel_for<SPECA_F32>(order);
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, fn, &cfg) != cudaSuccess || n < 1) {
+        (void)cudaGetLastError();
+        n = 1;
+    }
+    return n;
 }
 
 cudaError_t launch_select(const uint8_t* accept, int32_t k_max, int32_t group, int32_t batch, int32_t* spec_count,
@@ -695,24 +871,6 @@ cudaError_t launch_activate(uint64_t mask_bits, int32_t batch, int32_t* spec_cou
                             cudaStream_t stream) {
     activate_kernel<<<1, SPECA_MAX_BATCH, 0, stream>>>(mask_bits, batch, spec_count, active);
     return cudaGetLastError();
-}
-
-static int occupancy(const void* kernel) {
-    int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kThreads, 0) != cudaSuccess || n < 1) n = 1;
-    return n;
-}
-
-int ctas_per_sm_update(int dtype, int order) {
-    return occupancy(dtype == SPECA_BF16 ? stream_kernel_for<SPECA_BF16, true>(order)
-                                         : stream_kernel_for<SPECA_F32, true>(order));
-}
-int ctas_per_sm_forecast(int dtype, int order) {
-    return occupancy(dtype == SPECA_BF16 ? stream_kernel_for<SPECA_BF16, false>(order)
-                                         : stream_kernel_for<SPECA_F32, false>(order));
-}
-int ctas_per_sm_verify(int dtype, int order) {
-    return occupancy(dtype == SPECA_BF16 ? verify_kernel_for<SPECA_BF16>(order) : verify_kernel_for<SPECA_F32>(order));
 }
 
 }  // namespace speca

@@ -128,7 +128,7 @@ extern "C" speca_status_t speca_verify_pred_static(const void* pred, const void*
             p.tau[b] = tau[b];
         }
         const int cluster = 4;
-        const uint32_t te = tile_elems(dtype, SPECA_PATH_DIRECT);
+        const uint32_t te = verify_tile_elems(dtype, 0);
         p.segs = segs;
         p.arena = const_cast<char*>(static_cast<const char*>(pred));
         p.dev_mask = dev_active_mask;
@@ -143,10 +143,9 @@ extern "C" speca_status_t speca_verify_pred_static(const void* pred, const void*
         p.units_per_sample = (p.tiles_per_sample + cluster - 1) / cluster;
         p.batch = batch;
         p.eps = eps > 0.f ? static_cast<double>(eps) : 1e-8;
-        int sm_count = 0;
-        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, device);
-        int grid = sm_count * ctas_per_sm_verify(dtype, 0) / cluster * cluster;
-        if (grid / cluster > kStaticMaxClusters) grid = kStaticMaxClusters * cluster;
+        int n_clusters = max_resident_verify_clusters(dtype, 0, cluster);
+        if (n_clusters > kStaticMaxClusters) n_clusters = kStaticMaxClusters;
+        int grid = n_clusters * cluster;
         const uint64_t units = static_cast<uint64_t>(p.units_per_sample) * batch;
         if (units * cluster < static_cast<uint64_t>(grid)) grid = static_cast<int>(units) * cluster;
         if (launch_verify(p, dtype, grid, cluster, s) != cudaSuccess) st = SPECA_ERR_CUDA;

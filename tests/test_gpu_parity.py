@@ -74,13 +74,14 @@ def test_tiny_config_full_sequence(S, U):
 RAGGED = [(37, 129), (5, 3), (64, 384), (1, 8192 * 2 + 24), (3, 8192), (1, 1)]
 
 
+@pytest.mark.parametrize("path", [1, 3])  # SPECA_PATH_DIRECT, SPECA_PATH_WIDE
 @pytest.mark.parametrize("dtype", [0, 1])
 @pytest.mark.parametrize("basis", [0, 1])
 @pytest.mark.parametrize("m", [0, 1, 2, 3, 4])
-def test_ragged_shapes_all_orders(S, U, dtype, basis, m):
+def test_ragged_shapes_all_orders(S, U, dtype, basis, m, path):
     B = 3
     gen = torch.Generator(device=DEV).manual_seed(1000 + 10 * m + basis)
-    pair = U.Pair(RAGGED, B, m, dtype, basis)
+    pair = U.Pair(RAGGED, B, m, dtype, basis, path=path)
     times = [1.0, 0.93, 0.9, 0.81, 0.8, 0.74]
     for step in range(m + 2):
         t = [times[step], times[step] - 0.003, times[step] + 0.001]  # per-sample times
