@@ -34,9 +34,11 @@ METRIC = "forecast+verify GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes per cached element per launch (dram__bytes_read.sum + dram__bytes_write.sum from the
-# ncu captures summarised under profiles/), keyed by kernel; None until a capture exists.
-NCU_DRAM_BYTES_PER_ELEM = {"update": None, "forecast": None, "verify": None}
+# DRAM bytes per cached element per launch: (dram__bytes_read.sum + dram__bytes_write.sum) / elements
+# from the ncu captures summarised under profiles/ (taken on the DiT-XL/2-shaped cache, order 2,
+# bf16; traffic grows in proportion to the elements a launch covers). Set an entry to None when its
+# kernel changes until the counters have been taken again.
+NCU_DRAM_BYTES_PER_ELEM = {"update": 11.818, "forecast": 7.929, "verify": 8.012}
 
 
 def measured_peak():
@@ -282,6 +284,77 @@ def time_end_to_end(h: Harness, steps: int, warmup: int):
     return ms / steps, h2d, d2h
 
 
+def adaptive_sweep(device: str, peak: float, path: int, orders=(1, 2, 3), horizon: int = 6):
+    """FLUX-shaped batch of 8 samples with different noise levels: after max_order + 1 reference
+    steps, k = 1..horizon speculative steps run from the same table; samples whose verification
+    fails drop out of later forecasts (sequential validation). Per (order, k): samples forecast,
+    their accept flags, device times and GB/s over the bytes of the samples still active."""
+    from paper_2509_11628_b200 import binding as S
+    out = {}
+    dev = torch.device(device)
+    for m in orders:
+        w = W.flux_adaptive(max_order=m, batch=8)
+        B, ne = w.batch, len(w.entries)
+        src = W.FeatureSource(w, device)
+        cache = S.SpecaCache(w.entries, B, m, w.dtype, device, path=path)
+        for step in range(m + 1):
+            t = [w.times[step]] * B
+            for e in range(ne):
+                one = [None] * ne
+                one[e] = src.feature(e, step, t)
+                cache.update(one, t)
+            cache.commit_step()
+        outs = [torch.empty(B, n, d, dtype=w.torch_dtype, device=dev) for n, d in w.entries]
+        err = torch.zeros(B, dtype=torch.float32, device=dev)
+        acc = torch.zeros(B, dtype=torch.uint8, device=dev)
+        active = torch.ones(B, dtype=torch.uint8, device=dev)
+        spec = torch.zeros(B, dtype=torch.int32, device=dev)
+        rows = []
+        for k in range(1, horizon + 1):
+            step = m + k
+            t = [w.times[step]] * B
+            tau = [S.speca_tau(w.tau0, w.beta, w.total_steps - step, w.total_steps)] * B
+            fresh = src.feature(w.vidx, step, t)
+            act_in = active.cpu().tolist()
+            n_act = sum(act_in)
+            if n_act == 0:
+                rows.append({"k": k, "active": 0})
+                continue
+
+            def timed(fn, reps=5):
+                ts = []
+                for _ in range(reps):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    fn()
+                    e1.record()
+                    torch.cuda.synchronize(dev)
+                    ts.append(e0.elapsed_time(e1))
+                return sorted(ts)[len(ts) // 2]
+
+            f_ms = timed(lambda: cache.forecast(t, outs, active))
+            v_ms = timed(lambda: cache.verify(fresh, t, tau, err, acc, active))
+            cache.select_adaptive(acc, horizon, 1, spec, active)
+            torch.cuda.synchronize(dev)
+            per_sample = sum(n * d for n, d in w.entries)
+            f_bytes = (m + 2) * w.elem_bytes * per_sample * n_act
+            v_bytes = (m + 2) * w.elem_bytes * w.entry_elems(w.vidx) * n_act
+            gbs = (f_bytes + v_bytes) / ((f_ms + v_ms) * 1e-3) / 1e9
+            rows.append({"k": k, "active": n_act, "active_mask": act_in,
+                         "accept": [int(a) if act_in[i] else None for i, a in enumerate(acc.cpu().tolist())],
+                         "err": [round(float(x), 5) if act_in[i] else None for i, x in enumerate(err.cpu().tolist())],
+                         "tau": round(tau[0], 5), "forecast_ms": f_ms, "verify_ms": v_ms,
+                         "forecast_verify_gbs": gbs, "frac_of_measured_peak": gbs / peak,
+                         "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS})
+            del fresh
+        out["order_%d" % m] = {"sigma": w.sigma, "cache_bytes": w.elems_per_order * (m + 1) * w.elem_bytes,
+                               "steps": rows}
+        cache.close()
+        del cache, outs, src
+        torch.cuda.empty_cache()
+    return out
+
+
 def oracle_sample_run(w: W.Workload, sample_elems: int, repeats: int, seed: int = 0):
     """The CPU oracle, as it stands, on a bounded sample of the workload: `sample_elems` elements
     per sample of the verification entry go through one full step (update at order m, forecast,
@@ -383,6 +456,8 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "direct", "wide"],
                     help="kernel variant (speca_path_t); results are identical, only speed differs")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-adaptive", action="store_true",
+                    help="skip the B=8 sample-adaptive sweep (orders 1-3, horizon 1-6) reported under 'adaptive'")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
@@ -441,6 +516,13 @@ def main():
             except Exception as exc:  # report, do not hide
                 per_config[name] = {"error": repr(exc)}
 
+    adaptive = None
+    if info.world == 1 and not args.no_adaptive:
+        try:
+            adaptive = adaptive_sweep(device, peak, path)
+        except Exception as exc:  # report, do not hide
+            adaptive = {"error": repr(exc)}
+
     if not info.is_main:
         D.shutdown()
         return
@@ -473,7 +555,7 @@ def main():
         "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches,
         "clocks": clocks, "kernels": kernels, **extra,
         "frac_of_measured_peak": value / info.world / peak, "frac_of_nominal_8TBs": value / info.world / NOMINAL_HBM_GBS,
-        "per_config": per_config,
+        "per_config": per_config, "adaptive": adaptive,
         "paper_context": {"end_to_end_speedups": {"flux_h800": 6.34, "dit_xl2_a800": 7.3, "hunyuan_video_h800": 6.1},
                           "verification_overhead": "1.67%-3.5% of a full forward pass",
                           "note": "other hardware, whole-model numbers; context only"},
