@@ -453,7 +453,7 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--also", default="dit_xl2,hunyuan_video",
                     help="comma list of further configs measured device-resident and reported under per_config")
-    ap.add_argument("--path", default="auto", choices=["auto", "direct", "wide"],
+    ap.add_argument("--path", default="auto", choices=["auto", "direct", "bulk", "wide"],
                     help="kernel variant (speca_path_t); results are identical, only speed differs")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-adaptive", action="store_true",
@@ -479,7 +479,7 @@ def main():
     peak, peak_src = measured_peak()
 
     w = make_workload(args.config)
-    path = {"auto": 0, "direct": 1, "wide": 3}[args.path]
+    path = {"auto": 0, "direct": 1, "bulk": 2, "wide": 3}[args.path]
     h = Harness(w, device, seed_offset=17 * info.rank, path=path)
     total_ms, per_ms, launches, clocks = time_device_resident(h, args.steps, args.warmup, info, True)
     total_ms = D.max_over_ranks(total_ms, device)

@@ -118,7 +118,8 @@ speca_status_t speca_cache_arena_bytes(const speca_cache_config_t* cfg, size_t* 
 speca_status_t speca_cache_create(const speca_cache_config_t* cfg, speca_cache_t** out);
 
 /* Waits for the device to finish work that uses the handle, then frees host state. The arena
- * stays with the caller. NULL is accepted. */
+ * stays with the caller. NULL is accepted. Returns SPECA_ERR_CUDA if the device reported an error
+ * or a SPECA_PATH_BULK kernel gave up waiting for a copy (its results are then incomplete). */
 speca_status_t speca_cache_destroy(speca_cache_t* cache);
 
 /* Forget the reference history of the samples with host_sample_mask[b] != 0 (NULL = all):

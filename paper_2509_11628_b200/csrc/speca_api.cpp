@@ -229,10 +229,6 @@ speca_status_t speca_cache_create(const speca_cache_config_t* cfg, speca_cache_t
         c->n_refs[b] = 0;
         for (int i = 0; i <= SPECA_MAX_ORDER; ++i) c->t_hist[b][i] = std::numeric_limits<double>::quiet_NaN();
     }
-    if (c->path == SPECA_PATH_BULK) {  // not built in this version of the library
-        delete c;
-        return SPECA_ERR_UNSUPPORTED;
-    }
 
     DeviceGuard guard(c->device);
     if (!guard.ok) {
@@ -256,8 +252,8 @@ speca_status_t speca_cache_create(const speca_cache_config_t* cfg, speca_cache_t
         delete c;
         return SPECA_ERR_UNSUPPORTED;
     }
-    c->grid_update = c->sm_count * stream_ctas_per_sm(c->path, true);
-    c->grid_forecast = c->sm_count * stream_ctas_per_sm(c->path, false);
+    c->grid_update = c->sm_count * stream_ctas_per_sm(c->path, true, c->dtype, c->m);
+    c->grid_forecast = c->sm_count * stream_ctas_per_sm(c->path, false, c->dtype, c->m);
     c->cluster = 4;
     int n_clusters = max_resident_verify_clusters(c->dtype, c->m, c->cluster);
     if (n_clusters > kMaxClusters) n_clusters = kMaxClusters;
@@ -270,8 +266,12 @@ speca_status_t speca_cache_destroy(speca_cache_t* c) {
     if (c == nullptr) return SPECA_OK;
     DeviceGuard guard(c->device);
     cudaError_t ce = cudaDeviceSynchronize();
+    // the bulk path's kernels set this word when a bounded wait for a copy gave up
+    uint32_t gave_up = 0;
+    if (ce == cudaSuccess)
+        ce = cudaMemcpy(&gave_up, c->arena + c->L.ticket_off + sizeof(uint32_t), sizeof gave_up, cudaMemcpyDeviceToHost);
     delete c;
-    return ce == cudaSuccess ? SPECA_OK : SPECA_ERR_CUDA;
+    return (ce == cudaSuccess && gave_up == 0) ? SPECA_OK : SPECA_ERR_CUDA;
 }
 
 speca_status_t speca_cache_reset(speca_cache_t* c, const uint8_t* host_sample_mask) {

@@ -84,7 +84,7 @@ cudaError_t launch_activate(uint64_t mask_bits, int32_t batch, int32_t* spec_cou
 
 // Tile size and designed CTAs per SM of the stream kernel a path uses for update / forecast.
 uint32_t stream_tile_bytes(int path, bool update);
-int stream_ctas_per_sm(int path, bool update);
+int stream_ctas_per_sm(int path, bool update, int dtype, int order);
 // Clusters of the verify kernel that fit on the current device at once.
 int max_resident_verify_clusters(int dtype, int order, int cluster);
 

@@ -433,6 +433,224 @@ __global__ void __launch_bounds__(NT, MINB) stream_kernel(const __grid_constant_
 }
 
 // ------------------------------------------------------------------------------------------------
+// bulk path: the same streams staged through shared memory by the TMA engine
+// ------------------------------------------------------------------------------------------------
+// One elected thread issues `cp.async.bulk` copies (untiled TMA, 8 KB per plane and tile, no
+// multicast) into a ring of shared-memory stages and arms the stage's mbarrier with the byte count;
+// the CTA waits on the barrier's phase, computes from shared memory and stores from registers.
+// Measured on B200 this does not beat the register-direct 32-byte path for these reuse-free streams;
+// it is kept as a selectable variant. Tiles the copy engine cannot take (ragged last tile of a row,
+// rows that are not 16-byte aligned, samples at a lower order) go through the generic per-tile
+// routines in the same loop. Every wait is bounded: a copy that never lands sets the cache's error
+// word, and the CTA stops issuing, waits once more (bounded) for what it issued and returns.
+
+constexpr uint32_t kBulkTileBytes = 8192;
+constexpr int kBulkThreads = 256;
+constexpr uint32_t kBulkSpinLimit = 1u << 18;  // polls; a healthy copy completes within a few
+
+__host__ __device__ constexpr int bulk_stages(int v) {
+    const int per_stage = (v + 1) * static_cast<int>(kBulkTileBytes);
+    const int s = 98304 / per_stage;
+    return s > 4 ? 4 : (s < 2 ? 2 : s);
+}
+__host__ __device__ constexpr size_t bulk_smem_bytes(int v) {
+    return 256 + static_cast<size_t>(bulk_stages(v)) * (v + 1) * kBulkTileBytes;
+}
+
+struct BulkSlot {      // what the producer decided for the tile that occupies a stage
+    char* plane0;      // plane 0 of the tile
+    char* row;         // feature (update) / output (forecast) row of the tile
+    uint64_t stride;
+    uint32_t cnt;      // elements; 0 = nothing to do (masked sample, entry not in this call)
+    int32_t v;
+    uint32_t staged;   // 1: copies were issued into the stage; 0: use the generic routine
+    uint32_t sample;
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait; false if the phase did not complete within the limit.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+    for (uint32_t spins = 0; spins < kBulkSpinLimit; ++spins)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// global -> shared bulk copy; dst, src 16-byte aligned, bytes a multiple of 16
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_addr(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+
+template <int DT, int V, bool UPDATE>
+__global__ void __launch_bounds__(kBulkThreads) stream_bulk_kernel(const __grid_constant__ StreamParams p) {
+    constexpr int S = bulk_stages(V);
+    constexpr int NIN = V + 1;  // update: feature + planes 0..V-1; forecast: planes 0..V
+    constexpr uint32_t kTile = kBulkTileBytes / Elem<DT>::kBytes;
+    constexpr int EPV = Elem<DT>::kEPV;
+    constexpr int VPT = kBulkTileBytes / 16 / kBulkThreads;  // 16-byte vectors per thread per plane
+    constexpr int PV = kBulkTileBytes / 16;                  // vectors per plane and tile
+    extern __shared__ __align__(128) unsigned char smem[];
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem);
+    BulkSlot* slots = reinterpret_cast<BulkSlot*>(smem + 64);
+    static_assert(64 + 4 * sizeof(BulkSlot) <= 256, "slot ring fits the header");
+    unsigned char* buf = smem + 256;
+
+    const uint32_t first = p.tile_lo + blockIdx.x;
+    const uint32_t my = first < p.tile_hi ? (p.tile_hi - first + gridDim.x - 1) / gridDim.x : 0;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) mbar_init(&full[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    // producer state (meaningful in thread 0 only)
+    uint32_t pseg = p.seg_lo, pseg_first = 0, pseg_end = 0;
+    uint32_t outstanding = 0;  // stages with copies issued and not yet consumed
+    bool stop = false;
+    auto prepare = [&](uint32_t j, int s) {
+        const uint32_t tile = first + j * gridDim.x;
+        if (tile >= pseg_end) {
+            pseg = find_segment(p.tile_start, pseg, p.seg_hi, tile);
+            pseg_first = __ldg(p.tile_start + pseg);
+            pseg_end = __ldg(p.tile_start + pseg + 1);
+        }
+        const SegDesc sd = p.segs[pseg];
+        int v = p.order[sd.sample];
+        char* io = static_cast<char*>(p.io[sd.entry]);
+        if (p.dev_mask != nullptr && p.dev_mask[sd.sample] == 0) v = -1;
+        BulkSlot d;
+        d.cnt = 0;
+        d.v = v;
+        d.staged = 0;
+        d.sample = sd.sample;
+        d.stride = sd.plane_stride;
+        d.plane0 = nullptr;
+        d.row = nullptr;
+        if (v >= 0 && io != nullptr) {
+            const uint32_t elem0 = (tile - pseg_first) * kTile;
+            const uint64_t byte0 = static_cast<uint64_t>(elem0) * Elem<DT>::kBytes;
+            d.cnt = min(kTile, sd.n_elems - elem0);
+            d.plane0 = p.arena + sd.plane0_off + byte0;
+            d.row = io + sd.io_off + byte0;
+            const bool ok = !stop && v == V && d.cnt == kTile && (reinterpret_cast<uintptr_t>(d.row) & 15u) == 0;
+            if (ok) {
+                unsigned char* b = buf + static_cast<size_t>(s) * NIN * kBulkTileBytes;
+                mbar_expect_tx(&full[s], NIN * kBulkTileBytes);
+                if constexpr (UPDATE) {
+                    bulk_load(b, d.row, kBulkTileBytes, &full[s]);
+#pragma unroll
+                    for (int i = 0; i < V; ++i)
+                        bulk_load(b + (i + 1) * kBulkTileBytes, d.plane0 + i * sd.plane_stride, kBulkTileBytes, &full[s]);
+                } else {
+#pragma unroll
+                    for (int i = 0; i <= V; ++i)
+                        bulk_load(b + i * kBulkTileBytes, d.plane0 + i * sd.plane_stride, kBulkTileBytes, &full[s]);
+                }
+                d.staged = 1;
+                outstanding |= 1u << s;
+            }
+        }
+        slots[s] = d;
+    };
+
+    if (threadIdx.x == 0)
+        for (int s = 0; s < S && static_cast<uint32_t>(s) < my; ++s) prepare(s, s);
+    __syncthreads();
+
+    uint32_t phase_bits = 0;  // per stage: parity of the next phase to wait for (same in every thread)
+    bool dead = false;
+    for (uint32_t j = 0; j < my; ++j) {
+        const int s = j % S;
+        const BulkSlot d = slots[s];
+        if (d.cnt != 0) {
+            float coef[SPECA_MAX_ORDER];
+#pragma unroll
+            for (int i = 0; i < SPECA_MAX_ORDER; ++i) coef[i] = p.coef[d.sample][i];
+            if (d.staged) {
+                const uint32_t parity = (phase_bits >> s) & 1u;
+                bool landed = false;
+                if (!dead) {
+                    if (mbar_wait_bounded(&full[s], parity)) {
+                        landed = true;
+                        phase_bits ^= 1u << s;
+                        outstanding &= ~(1u << s);
+                    } else {
+                        dead = true;  // the phase stays pending: the last loop below waits for it once more
+                        *p.err_flag = 1;
+                    }
+                }
+                if (landed) {
+                    const uint4* in = reinterpret_cast<const uint4*>(buf + static_cast<size_t>(s) * NIN * kBulkTileBytes);
+#pragma unroll
+                    for (int u = 0; u < VPT; ++u) {
+                        const int idx = u * kBulkThreads + threadIdx.x;
+                        if constexpr (UPDATE) {
+                            const uint4 fv = in[idx];
+                            float c[EPV];
+                            unpack<DT>(fv, c);
+                            __stcs(reinterpret_cast<uint4*>(d.plane0) + idx, fv);
+#pragma unroll
+                            for (int i = 0; i < V; ++i) {
+                                float old[EPV];
+                                unpack<DT>(in[(i + 1) * PV + idx], old);
+#pragma unroll
+                                for (int k = 0; k < EPV; ++k) c[k] = (c[k] - old[k]) * coef[i];
+                                __stcs(reinterpret_cast<uint4*>(d.plane0 + (i + 1) * d.stride) + idx, pack<DT>(c));
+                            }
+                        } else {
+                            float acc[EPV];
+                            unpack<DT>(in[V * PV + idx], acc);
+#pragma unroll
+                            for (int i = V; i >= 1; --i) {
+                                float lo[EPV];
+                                unpack<DT>(in[(i - 1) * PV + idx], lo);
+#pragma unroll
+                                for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], coef[i - 1], lo[k]);
+                            }
+                            __stcs(reinterpret_cast<uint4*>(d.row) + idx, pack<DT>(acc));
+                        }
+                    }
+                }
+            } else {
+                if constexpr (UPDATE)
+                    update_tile_any<DT>(d.plane0, d.stride, d.row, d.cnt, d.v, coef);
+                else
+                    forecast_tile_any<DT>(d.plane0, d.stride, d.row, d.cnt, d.v, coef);
+            }
+        }
+        __syncthreads();  // stage s and its slot are free again
+        if (threadIdx.x == 0 && j + S < my) {
+            stop = dead;
+            prepare(j + S, s);
+        }
+    }
+    // After a timeout copies may still be outstanding: give each such stage one more bounded wait so
+    // that nothing lands in the shared memory of a CTA that has already left.
+    if (dead && threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s)
+            if (outstanding & (1u << s)) (void)mbar_wait_bounded(&full[s], (phase_bits >> s) & 1u);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // verify: forecast of one entry fused with the two sums of squares of Eq. 4
 // ------------------------------------------------------------------------------------------------
 
@@ -796,15 +1014,56 @@ static int max_order(const int8_t* order) {
     return v;
 }
 
+template <int DT, bool UPDATE>
+static const void* bulk_kernel_for(int v) {
+    switch (v) {
+        case 0: return reinterpret_cast<const void*>(&stream_bulk_kernel<DT, 0, UPDATE>);
+        case 1: return reinterpret_cast<const void*>(&stream_bulk_kernel<DT, 1, UPDATE>);
+        case 2: return reinterpret_cast<const void*>(&stream_bulk_kernel<DT, 2, UPDATE>);
+        case 3: return reinterpret_cast<const void*>(&stream_bulk_kernel<DT, 3, UPDATE>);
+        default: return reinterpret_cast<const void*>(&stream_bulk_kernel<DT, 4, UPDATE>);
+    }
+}
+
+static const void* bulk_kernel_for(int dtype, bool update, int v) {
+    if (update) return dtype == SPECA_BF16 ? bulk_kernel_for<SPECA_BF16, true>(v) : bulk_kernel_for<SPECA_F32, true>(v);
+    return dtype == SPECA_BF16 ? bulk_kernel_for<SPECA_BF16, false>(v) : bulk_kernel_for<SPECA_F32, false>(v);
+}
+
+static int clamp_order(int v) { return v < 0 ? 0 : (v > SPECA_MAX_ORDER ? SPECA_MAX_ORDER : v); }
+
 uint32_t stream_tile_bytes(int path, bool update) {
+    if (path == SPECA_PATH_BULK) return kBulkTileBytes;
     const Shape s = shape_for(path, update);
     return static_cast<uint32_t>(s.w) * s.nt * s.u * s.chunks;
 }
 
-int stream_ctas_per_sm(int path, bool update) { return shape_for(path, update).minb; }
+int stream_ctas_per_sm(int path, bool update, int dtype, int order) {
+    if (path == SPECA_PATH_BULK) {
+        const void* fn = bulk_kernel_for(dtype, update, clamp_order(order));
+        const int smem = static_cast<int>(bulk_smem_bytes(clamp_order(order)));
+        int n = 0;
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fn, kBulkThreads, smem) != cudaSuccess || n < 1) {
+            (void)cudaGetLastError();
+            n = 1;
+        }
+        return n;
+    }
+    return shape_for(path, update).minb;
+}
 
 static cudaError_t launch_stream(const StreamParams& p, int dtype, bool update, int path, int grid,
                                  cudaStream_t stream) {
+    if (path == SPECA_PATH_BULK) {
+        const int v = max_order(p.order);
+        const void* fn = bulk_kernel_for(dtype, update, v);
+        const size_t smem = bulk_smem_bytes(v);
+        cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+        void* args[1] = {const_cast<StreamParams*>(&p)};
+        return cudaLaunchKernel(fn, dim3(grid), dim3(kBulkThreads), args, smem, stream);
+    }
     if (path != SPECA_PATH_DIRECT && path != SPECA_PATH_WIDE) return cudaErrorNotSupported;
     const void* fn = stream_kernel_for(dtype, update, path, max_order(p.order));
     void* args[1] = {const_cast<StreamParams*>(&p)};

@@ -74,7 +74,7 @@ def test_tiny_config_full_sequence(S, U):
 RAGGED = [(37, 129), (5, 3), (64, 384), (1, 8192 * 2 + 24), (3, 8192), (1, 1)]
 
 
-@pytest.mark.parametrize("path", [1, 3])  # SPECA_PATH_DIRECT, SPECA_PATH_WIDE
+@pytest.mark.parametrize("path", [1, 2, 3])  # SPECA_PATH_DIRECT, SPECA_PATH_BULK, SPECA_PATH_WIDE
 @pytest.mark.parametrize("dtype", [0, 1])
 @pytest.mark.parametrize("basis", [0, 1])
 @pytest.mark.parametrize("m", [0, 1, 2, 3, 4])
@@ -273,16 +273,17 @@ def test_argument_errors_return_status(S):
 # cut-down copies of the model-shaped configs (same dim, dtype, time grid, value structure)
 # ---------------------------------------------------------------------------------------------
 
+@pytest.mark.parametrize("path", [0, 2])  # library default, and the TMA-staged variant
 @pytest.mark.parametrize("name,kw", [
     ("dit_xl2", dict(max_entries=6, max_tokens=0)),
     ("flux", dict(max_entries=5, max_tokens=300)),
     ("hunyuan_video", dict(max_entries=4, max_tokens=1700)),
 ])
-def test_model_shaped_configs_cut_down(S, U, name, kw):
+def test_model_shaped_configs_cut_down(S, U, name, kw, path):
     w = W.scaled(W.BY_NAME[name](), **kw)
     src = W.FeatureSource(w, DEV)
     B = w.batch
-    pair = U.Pair(w.entries, B, w.max_order, w.dtype)
+    pair = U.Pair(w.entries, B, w.max_order, w.dtype, path=path)
     pattern = W.reference_pattern(w)
     spec = torch.zeros(B, dtype=torch.int32, device=DEV)
     active = torch.ones(B, dtype=torch.uint8, device=DEV)
