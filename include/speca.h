@@ -41,6 +41,7 @@ extern "C" {
 #define SPECA_MAX_ORDER   4     /* highest Taylor order m */
 #define SPECA_MAX_BATCH   64    /* most samples B in one cache */
 #define SPECA_MAX_ENTRIES 512   /* most cached tensors (block outputs) in one cache */
+#define SPECA_MAX_HORIZON 8     /* most speculative steps one speca_forecast_multi call evaluates */
 
 typedef struct speca_cache speca_cache_t; /* opaque, owned by the library */
 
@@ -168,6 +169,21 @@ speca_status_t speca_cache_commit_step(speca_cache_t* cache);
  */
 speca_status_t speca_forecast(speca_cache_t* cache, const double* t_target, const uint8_t* dev_active_mask,
                               void* const* outs, void* stream);
+
+/*
+ * Several speculative steps at once: Eq. 2 evaluated for K targets t-1 .. t-K from one read of the
+ * tables (Fig. 1: the draft model predicts the next N timesteps from the latest reference; workflow
+ * step 2 of Section 3.2). Same arithmetic as K calls of speca_forecast, bit for bit, but the planes
+ * are read once: (v + 1 + K) words of traffic per element instead of K (v + 2).
+ *   n_targets       K, 1..SPECA_MAX_HORIZON.
+ *   t_targets       host, K * B doubles, target k of sample b at [k * B + b].
+ *   dev_active_mask device, B bytes, NULL = all: inactive samples are skipped for every target.
+ *   outs            host array of n_entries device pointers, outs[e] = [K, B, N_e, D] (target-major),
+ *                   NULL = skip e.
+ * Errors: INVALID_ARG (null, K out of range, non-finite time), ALIGNMENT, STATE, CUDA.
+ */
+speca_status_t speca_forecast_multi(speca_cache_t* cache, int32_t n_targets, const double* t_targets,
+                                    const uint8_t* dev_active_mask, void* const* outs, void* stream);
 
 /*
  * Verification, Eq. 4 and the accept rule of Section 3.4.2, fused with the forecast of the

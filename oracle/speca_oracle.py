@@ -213,6 +213,17 @@ class OracleCache:
                                  self.planes[e][b], out[b])
         return out
 
+    def forecast_multi(self, e: int, t_targets: Sequence[Sequence[float]], active: Optional[Sequence[int]] = None,
+                       out: Optional[np.ndarray] = None) -> np.ndarray:
+        """Eq. 2 for K speculative steps from the same table (Fig. 1: the draft predicts the next
+        steps t-1 .. t-K): simply K forecasts. Returns [K, B, n_e]."""
+        K = len(t_targets)
+        if out is None:
+            out = np.zeros((K, self.B, self.entry_elems[e]), dtype=np_dtype(self.dtype))
+        for k in range(K):
+            self.forecast_entry(e, t_targets[k], active, out=out[k])
+        return out
+
     def verify(self, fresh: np.ndarray, t_target: Sequence[float], tau: Sequence[float],
                active: Optional[Sequence[int]] = None):
         """Returns (err[B] float64 with NaN for skipped samples, accept[B] int with -1 for skipped,

@@ -22,14 +22,14 @@ SPECA_ERR_ZERO_GAP, SPECA_ERR_NOMEM, SPECA_ERR_CUDA, SPECA_ERR_UNSUPPORTED = 5, 
 SPECA_F32, SPECA_BF16 = 0, 1
 SPECA_BASIS_TAYLOR, SPECA_BASIS_NEWTON = 0, 1
 SPECA_PATH_AUTO, SPECA_PATH_DIRECT, SPECA_PATH_BULK, SPECA_PATH_WIDE = 0, 1, 2, 3
-SPECA_MAX_ORDER, SPECA_MAX_BATCH, SPECA_MAX_ENTRIES = 4, 64, 512
+SPECA_MAX_ORDER, SPECA_MAX_BATCH, SPECA_MAX_ENTRIES, SPECA_MAX_HORIZON = 4, 64, 512, 8
 
 EXPORTS = [
     "speca_cache_arena_bytes", "speca_cache_create", "speca_cache_destroy", "speca_cache_reset",
     "speca_cache_update", "speca_cache_commit_step", "speca_forecast", "speca_verify",
     "speca_select_adaptive", "speca_activate", "speca_tau", "speca_cache_state", "speca_cache_plane",
     "speca_cache_launch_count", "speca_status_string", "speca_last_error", "speca_version",
-    "speca_verify_pred_static",
+    "speca_verify_pred_static", "speca_forecast_multi",
 ]
 
 
@@ -74,6 +74,7 @@ def _lib() -> ctypes.CDLL:
     L.speca_cache_update.argtypes = [vp, vp, vp, vp, vp]
     L.speca_cache_commit_step.argtypes = [vp]
     L.speca_forecast.argtypes = [vp, vp, vp, vp, vp]
+    L.speca_forecast_multi.argtypes = [vp, i32, vp, vp, vp, vp]
     L.speca_verify.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.speca_select_adaptive.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, vp]
     L.speca_activate.argtypes = [vp, vp, vp, vp, vp]
@@ -198,6 +199,13 @@ def speca_forecast(cache, t_target, dev_active_mask, outs, stream=None) -> None:
                                  _stream_ptr(stream)), cache)
 
 
+def speca_forecast_multi(cache, t_targets, dev_active_mask, outs, stream=None) -> None:
+    """``t_targets``: K lists of B times; ``outs[e]``: device tensor [K, B, N_e, D] (None = skip)."""
+    flat = [float(t) for row in t_targets for t in row]
+    _check(_lib().speca_forecast_multi(cache, len(t_targets), _doubles(flat), _dev_ptr(dev_active_mask),
+                                       _ptr_array(outs), _stream_ptr(stream)), cache)
+
+
 def speca_verify(cache, fresh, t_target, tau, dev_active_mask, out_pred, dev_err, dev_accept, stream=None) -> None:
     _check(_lib().speca_verify(cache, _dev_ptr(fresh), _doubles(t_target), _floats(tau), _dev_ptr(dev_active_mask),
                                _dev_ptr(out_pred), _dev_ptr(dev_err), _dev_ptr(dev_accept), _stream_ptr(stream)),
@@ -296,6 +304,9 @@ class SpecaCache:
 
     def forecast(self, t_target, outs, active=None, stream=None):
         speca_forecast(self.handle, t_target, active, outs, stream)
+
+    def forecast_multi(self, t_targets, outs, active=None, stream=None):
+        speca_forecast_multi(self.handle, t_targets, active, outs, stream)
 
     def verify(self, fresh, t_target, tau, err, accept, active=None, out_pred=None, stream=None):
         speca_verify(self.handle, fresh, t_target, tau, active, out_pred, err, accept, stream)

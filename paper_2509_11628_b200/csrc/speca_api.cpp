@@ -428,6 +428,65 @@ speca_status_t speca_forecast(speca_cache_t* c, const double* t_target, const ui
     return SPECA_OK;
 }
 
+speca_status_t speca_forecast_multi(speca_cache_t* c, int32_t n_targets, const double* t_targets,
+                                    const uint8_t* dev_active_mask, void* const* outs, void* stream) {
+    if (c == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (t_targets == nullptr || outs == nullptr) return fail(c, SPECA_ERR_INVALID_ARG, "forecast_multi: null argument");
+    if (n_targets < 1 || n_targets > SPECA_MAX_HORIZON)
+        return fail(c, SPECA_ERR_INVALID_ARG, "forecast_multi: n_targets must be 1..%d", SPECA_MAX_HORIZON);
+    if (c->pending) return fail(c, SPECA_ERR_STATE, "forecast_multi: a reference step is open (commit it first)");
+    static thread_local MultiParams p;  // 13 KB: kept off the stack
+    std::memset(&p, 0, sizeof p);
+    bool any_sample = false;
+    for (int b = 0; b < c->B; ++b) {
+        int order = -1;
+        for (int k = 0; k < n_targets; ++k) {
+            const double t = t_targets[static_cast<size_t>(k) * c->B + b];
+            if (!std::isfinite(t)) return fail(c, SPECA_ERR_INVALID_ARG, "forecast_multi: t_targets[%d][%d] not finite", k, b);
+            forecast_scalars(c, b, t, &order, p.coef[k][b]);
+        }
+        if (order < 0 && dev_active_mask == nullptr)
+            return fail(c, SPECA_ERR_STATE, "forecast_multi: sample %d has no committed reference", b);
+        p.order[b] = static_cast<int8_t>(order);
+        any_sample |= order >= 0;
+    }
+    int e_lo = -1, e_hi = -1;
+    const size_t esz = elem_size(c);
+    for (int e = 0; e < c->n_entries; ++e) {
+        if (outs[e] == nullptr) continue;
+        if (reinterpret_cast<uintptr_t>(outs[e]) % esz != 0)
+            return fail(c, SPECA_ERR_ALIGNMENT, "forecast_multi: outs[%d] not aligned to the element size", e);
+        if (e_lo < 0) e_lo = e;
+        e_hi = e;
+        p.io[e] = outs[e];
+    }
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return fail(c, SPECA_ERR_CUDA, "cudaSetDevice failed");
+    speca_status_t st = check_sticky(c);
+    if (st != SPECA_OK) return st;
+    if (e_lo < 0 || !any_sample) return SPECA_OK;
+    const Layout& L = c->L;
+    const int ti = tile_size_index(multi_tile_bytes());
+    if (ti < 0) return fail(c, SPECA_ERR_UNSUPPORTED, "forecast_multi: no tile table for its tile size");
+    const std::vector<uint32_t>& tiles = L.tiles[ti];
+    p.segs = reinterpret_cast<const SegDesc*>(c->arena + L.segs_off);
+    p.tile_start = reinterpret_cast<const uint32_t*>(c->arena + L.tiles_off[ti]);
+    p.arena = c->arena;
+    p.dev_mask = dev_active_mask;
+    p.n_targets = n_targets;
+    p.seg_lo = static_cast<uint32_t>(e_lo) * c->B;
+    p.seg_hi = static_cast<uint32_t>(e_hi + 1) * c->B;
+    p.tile_lo = tiles[p.seg_lo];
+    p.tile_hi = tiles[p.seg_hi];
+    const uint32_t n_tiles = p.tile_hi - p.tile_lo;
+    const uint32_t full = static_cast<uint32_t>(c->sm_count * multi_ctas_per_sm());
+    const int grid = static_cast<int>(n_tiles < full ? n_tiles : full);
+    cudaError_t ce = launch_forecast_multi(p, c->dtype, c->B, grid, static_cast<cudaStream_t>(stream));
+    if (ce != cudaSuccess) return cuda_fail(c, ce, "forecast_multi launch");
+    c->launches += 1;
+    return SPECA_OK;
+}
+
 speca_status_t speca_verify(speca_cache_t* c, const void* fresh, const double* t_target, const float* tau,
                             const uint8_t* dev_active_mask, void* out_pred, float* dev_err, uint8_t* dev_accept,
                             void* stream) {

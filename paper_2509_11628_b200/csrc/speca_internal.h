@@ -52,6 +52,20 @@ struct StreamParams {
     void* io[SPECA_MAX_ENTRIES];  // per entry: feature (update) or output (forecast); null = skip
 };
 
+// Arguments of the multi-horizon forecast: K targets evaluated from one read of the table.
+struct MultiParams {
+    const SegDesc* segs;
+    const uint32_t* tile_start;  // prefix table for multi_tile_bytes()
+    char* arena;
+    const uint8_t* dev_mask;
+    uint32_t seg_lo, seg_hi;
+    uint32_t tile_lo, tile_hi;
+    int32_t n_targets;                // K
+    int8_t order[SPECA_MAX_BATCH];
+    float coef[SPECA_MAX_HORIZON][SPECA_MAX_BATCH][SPECA_MAX_ORDER];  // Horner multipliers per target
+    void* io[SPECA_MAX_ENTRIES];      // per entry: [K, B, N_e, D] output; null = skip
+};
+
 // Arguments of the fused forecast + relative-L2 kernel over the verification entry.
 struct VerifyParams {
     const SegDesc* segs;  // segments of the verify entry only (B of them)
@@ -85,6 +99,10 @@ cudaError_t launch_activate(uint64_t mask_bits, int32_t batch, int32_t* spec_cou
 // Tile size and designed CTAs per SM of the stream kernel a path uses for update / forecast.
 uint32_t stream_tile_bytes(int path, bool update);
 int stream_ctas_per_sm(int path, bool update, int dtype, int order);
+// Multi-horizon forecast kernel: tile size, designed CTAs per SM, launcher.
+uint32_t multi_tile_bytes();
+int multi_ctas_per_sm();
+cudaError_t launch_forecast_multi(const MultiParams& p, int dtype, int batch, int grid, cudaStream_t stream);
 // Clusters of the verify kernel that fit on the current device at once.
 int max_resident_verify_clusters(int dtype, int order, int cluster);
 

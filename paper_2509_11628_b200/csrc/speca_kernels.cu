@@ -433,6 +433,106 @@ __global__ void __launch_bounds__(NT, MINB) stream_kernel(const __grid_constant_
 }
 
 // ------------------------------------------------------------------------------------------------
+// multi-horizon forecast: Eq. 2 for K speculative steps from one read of the table
+// ------------------------------------------------------------------------------------------------
+// The draft model predicts several future steps from the same reference (Fig. 1, workflow step 2).
+// Evaluating them in one pass reads the v + 1 planes once and writes K outputs: (v + 1 + K) words per
+// element instead of K (v + 2). Output k of entry e is row k of a [K, B, N_e, D] tensor. The mix is
+// write-heavy like the update, so the kernel uses the update's launch shape.
+constexpr Shape kMultiShape = Shape{SPECA_SHAPE_UPDATE};
+
+template <int DT, int V, int W, int NT, int U>
+__device__ __forceinline__ void forecast_multi_tile(const char* __restrict__ plane0, uint64_t stride,
+                                                    char* __restrict__ out, uint64_t target_stride, int n_targets,
+                                                    uint32_t cnt, const float (*__restrict__ mu)[SPECA_MAX_BATCH][SPECA_MAX_ORDER],
+                                                    uint32_t sample) {
+    constexpr int EPV = W / Elem<DT>::kBytes;
+    const uint32_t nvec = cnt / EPV;
+    Vec<W> d[V + 1][U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint32_t idx = u * NT + threadIdx.x;
+        if (idx < nvec) {
+#pragma unroll
+            for (int i = 0; i <= V; ++i) d[i][u] = load_vec<W>(plane0 + i * stride + static_cast<size_t>(idx) * W);
+        }
+    }
+#pragma unroll 1
+    for (int k = 0; k < n_targets; ++k) {
+        float m[SPECA_MAX_ORDER];
+#pragma unroll
+        for (int i = 0; i < SPECA_MAX_ORDER; ++i) m[i] = mu[k][sample][i];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t idx = u * NT + threadIdx.x;
+            if (idx < nvec) {
+                float acc[EPV];
+                unpack_vec<DT, W>(d[V][u], acc);
+#pragma unroll
+                for (int i = V; i >= 1; --i) {
+                    float lo[EPV];
+                    unpack_vec<DT, W>(d[i - 1][u], lo);
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) acc[e] = fmaf(acc[e], m[i - 1], lo[e]);
+                }
+                store_vec<W>(out + k * target_stride + static_cast<size_t>(idx) * W, pack_vec<DT, W>(acc));
+            }
+        }
+        for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += NT) {
+            float acc = load_scalar<DT>(plane0 + V * stride, j);
+#pragma unroll
+            for (int i = V; i >= 1; --i) acc = fmaf(acc, m[i - 1], load_scalar<DT>(plane0 + (i - 1) * stride, j));
+            store_scalar<DT>(out + k * target_stride, j, acc);
+        }
+    }
+}
+
+template <int DT, int V, int W, int NT, int U, int C, int MINB>
+__global__ void __launch_bounds__(NT, MINB) forecast_multi_kernel(const __grid_constant__ MultiParams p, int batch) {
+    constexpr uint32_t kChunk = static_cast<uint32_t>(NT) * U * W / Elem<DT>::kBytes;
+    constexpr uint32_t kTile = kChunk * C;
+    uint32_t seg = p.seg_lo, seg_first = 0, seg_end = 0;
+    SegDesc sd = {};
+    int v = -1;
+    char* io = nullptr;
+    uint64_t target_stride = 0;  // bytes between consecutive targets of this entry's output
+    for (uint32_t tile = p.tile_lo + blockIdx.x; tile < p.tile_hi; tile += gridDim.x) {
+        if (tile >= seg_end) {
+            seg = find_segment(p.tile_start, seg, p.seg_hi, tile);
+            seg_first = __ldg(p.tile_start + seg);
+            seg_end = __ldg(p.tile_start + seg + 1);
+            sd = p.segs[seg];
+            v = p.order[sd.sample];
+            io = static_cast<char*>(p.io[sd.entry]);
+            if (p.dev_mask != nullptr && p.dev_mask[sd.sample] == 0) v = -1;
+            target_stride = static_cast<uint64_t>(batch) * sd.n_elems * Elem<DT>::kBytes;
+        }
+        if (v < 0 || io == nullptr) continue;
+        const uint32_t elem0 = (tile - seg_first) * kTile;
+        const uint32_t cnt = min(kTile, sd.n_elems - elem0);
+        const uint64_t byte0 = static_cast<uint64_t>(elem0) * Elem<DT>::kBytes;
+        char* plane0 = p.arena + sd.plane0_off + byte0;
+        char* row = io + sd.io_off + byte0;
+        const bool fast = v == V && ((reinterpret_cast<uintptr_t>(row) | target_stride) & (W - 1)) == 0;
+        if (fast) {
+            for (uint32_t done = 0; done < cnt; done += kChunk) {
+                const uint32_t n = min(kChunk, cnt - done);
+                const size_t off = static_cast<size_t>(done) * Elem<DT>::kBytes;
+                forecast_multi_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, row + off, target_stride,
+                                                     p.n_targets, n, p.coef, sd.sample);
+            }
+        } else {
+            for (int k = 0; k < p.n_targets; ++k) {
+                float m[SPECA_MAX_ORDER];
+#pragma unroll
+                for (int i = 0; i < SPECA_MAX_ORDER; ++i) m[i] = p.coef[k][sd.sample][i];
+                forecast_tile_any<DT>(plane0, sd.plane_stride, row + k * target_stride, cnt, v, m);
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // bulk path: the same streams staged through shared memory by the TMA engine
 // ------------------------------------------------------------------------------------------------
 // One elected thread issues `cp.async.bulk` copies (untiled TMA, 8 KB per plane and tile, no
@@ -1076,6 +1176,28 @@ cudaError_t launch_update(const StreamParams& p, int dtype, int path, int grid, 
 
 cudaError_t launch_forecast(const StreamParams& p, int dtype, int path, int grid, cudaStream_t stream) {
     return launch_stream(p, dtype, false, path, grid, stream);
+}
+
+template <int DT>
+static const void* multi_kernel_for(int v) {
+    constexpr Shape s = kMultiShape;
+    switch (v) {
+        case 0: return reinterpret_cast<const void*>(&forecast_multi_kernel<DT, 0, s.w, s.nt, s.u, s.chunks, s.minb>);
+        case 1: return reinterpret_cast<const void*>(&forecast_multi_kernel<DT, 1, s.w, s.nt, s.u, s.chunks, s.minb>);
+        case 2: return reinterpret_cast<const void*>(&forecast_multi_kernel<DT, 2, s.w, s.nt, s.u, s.chunks, s.minb>);
+        case 3: return reinterpret_cast<const void*>(&forecast_multi_kernel<DT, 3, s.w, s.nt, s.u, s.chunks, s.minb>);
+        default: return reinterpret_cast<const void*>(&forecast_multi_kernel<DT, 4, s.w, s.nt, s.u, s.chunks, s.minb>);
+    }
+}
+
+uint32_t multi_tile_bytes() { return static_cast<uint32_t>(kMultiShape.w) * kMultiShape.nt * kMultiShape.u * kMultiShape.chunks; }
+int multi_ctas_per_sm() { return kMultiShape.minb; }
+
+cudaError_t launch_forecast_multi(const MultiParams& p, int dtype, int batch, int grid, cudaStream_t stream) {
+    const int v = max_order(p.order);
+    const void* fn = dtype == SPECA_BF16 ? multi_kernel_for<SPECA_BF16>(v) : multi_kernel_for<SPECA_F32>(v);
+    void* args[2] = {const_cast<MultiParams*>(&p), &batch};
+    return cudaLaunchKernel(fn, dim3(grid), dim3(kMultiShape.nt), args, 0, stream);
 }
 
 static void verify_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int grid, int cluster,
