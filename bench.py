@@ -267,6 +267,30 @@ def time_multi_horizon(h: Harness, peak: float, forecast_ms: float, K: int = 4, 
             "speedup_vs_single_forecasts": K * forecast_ms / ms}
 
 
+def time_metrics(h: Harness, reps: int = 20):
+    """Device time of the fused verification with each error metric (same traffic: order + 2 words per
+    element of the verification entry)."""
+    w, dev = h.w, h.device
+    names = {0: "l2", 1: "l1", 2: "linf", 3: "cosine"}
+    t = [h.t_base - 0.02 * (h.j + 1) - 0.01] * h.B
+    tau = [0.1] * h.B
+    nbytes = (w.max_order + 2) * w.elem_bytes * w.batch * w.entry_elems(w.vidx)
+    out = {}
+    for metric, name in names.items():
+        for _ in range(3):
+            h.cache.verify(h.fresh[0], t, tau, h.err, h.accept, h.active, metric=metric)
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            h.cache.verify(h.fresh[0], t, tau, h.err, h.accept, h.active, metric=metric)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        ms = e0.elapsed_time(e1) / reps
+        out[name] = {"ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9, "err": [round(float(x), 6) for x in h.err.cpu().tolist()]}
+    return out
+
+
 def time_end_to_end(h: Harness, steps: int, warmup: int):
     """Same step, but its inputs start in pinned host memory and its results end there."""
     w, dev = h.w, h.device
@@ -512,6 +536,7 @@ def main():
     value, ms_step, kernels, extra = summarize(w, per_ms, total_ms, args.steps, info.world, peak)
 
     multi = time_multi_horizon(h, peak, per_ms["forecast"]) if info.world == 1 else None
+    metrics = time_metrics(h) if info.world == 1 else None
 
     e2e = None
     if not args.no_e2e:
@@ -584,7 +609,7 @@ def main():
         "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches,
         "clocks": clocks, "kernels": kernels, **extra,
         "frac_of_measured_peak": value / info.world / peak, "frac_of_nominal_8TBs": value / info.world / NOMINAL_HBM_GBS,
-        "multi_horizon": multi, "per_config": per_config, "adaptive": adaptive,
+        "multi_horizon": multi, "verify_metrics": metrics, "per_config": per_config, "adaptive": adaptive,
         "paper_context": {"end_to_end_speedups": {"flux_h800": 6.34, "dit_xl2_a800": 7.3, "hunyuan_video_h800": 6.1},
                           "verification_overhead": "1.67%-3.5% of a full forward pass",
                           "note": "other hardware, whole-model numbers; context only"},

@@ -80,6 +80,23 @@ typedef enum {
     SPECA_PATH_WIDE = 3    /* 32-byte vector loads / stores, per-kernel launch shapes */
 } speca_path_t;
 
+/*
+ * Error metric of the verification. Eq. 4 is the relative l2 error (the paper's default); the
+ * appendix on error metrics also evaluates l1, l-infinity and cosine similarity, named there
+ * without formulas. The forms used here (p = forecast, f = computed feature, all over one sample):
+ *   L2      ||p - f||_2   / (||f||_2   + eps)
+ *   L1      ||p - f||_1   / (||f||_1   + eps)
+ *   LINF    ||p - f||_inf / (||f||_inf + eps)
+ *   COSINE  1 - <p, f> / (||p||_2 ||f||_2 + eps)     (a distance: 0 = same direction)
+ * In every case the sample is accepted iff the value is <= tau, and a NaN rejects.
+ */
+typedef enum {
+    SPECA_METRIC_L2 = 0,
+    SPECA_METRIC_L1 = 1,
+    SPECA_METRIC_LINF = 2,
+    SPECA_METRIC_COSINE = 3
+} speca_metric_t;
+
 typedef struct {
     int64_t tokens; /* N_e  >= 1 */
     int32_t dim;    /* D    >= 1 */
@@ -204,6 +221,13 @@ speca_status_t speca_forecast_multi(speca_cache_t* cache, int32_t n_targets, con
 speca_status_t speca_verify(speca_cache_t* cache, const void* fresh, const double* t_target, const float* tau,
                             const uint8_t* dev_active_mask, void* out_pred, float* dev_err,
                             uint8_t* dev_accept, void* stream);
+
+/* speca_verify with another error metric (speca_metric_t); everything else as speca_verify.
+ * speca_verify(...) is speca_verify_metric(..., SPECA_METRIC_L2, ...). Errors: as speca_verify,
+ * and INVALID_ARG for an unknown metric. */
+speca_status_t speca_verify_metric(speca_cache_t* cache, int32_t metric, const void* fresh, const double* t_target,
+                                   const float* tau, const uint8_t* dev_active_mask, void* out_pred, float* dev_err,
+                                   uint8_t* dev_accept, void* stream);
 
 /*
  * Per-sample continuation of the speculative run (sequential validation of Section 3.4.2, the

@@ -11,6 +11,8 @@
  *                            quotients so that reference steps may be unevenly spaced
  *   oracle_forecast_segment  Eq. 2 (TaylorSeer prediction), written as the printed sum
  *   oracle_rel_l2            Eq. 4 (relative error, epsilon = 1e-8)
+ *   oracle_rel_l1/_linf, oracle_cos_dist   the other metrics of the appendix on error metrics
+ *                            (named there without formulas: readings, parity unpinned by the paper)
  *   oracle_accept            Section 3.4.2, rule 1/2 (e <= tau accepts)
  *   oracle_tau               Section 3.4.2, tau_t = tau0 * beta^((T-t)/T)
  *   oracle_speedup           Eq. 8, S = 1 / (1 - alpha + alpha*gamma)
@@ -167,6 +169,58 @@ double oracle_rel_l2(int dtype, int64_t n, const void* pred, const void* fresh, 
         den += f * f;
     }
     return sqrt(num) / (sqrt(den) + eps);
+}
+
+/* ---- other error metrics (appendix "Choice of Error Metrics for Verification") ----------------- */
+/*
+ * The appendix names l1, l-infinity and cosine similarity as alternatives to the l2 norm of Eq. 4
+ * and says a relative formulation is used, but prints no formulas: these are readings, pinned in
+ * the tests by what the mathematics fixes (zero at p = f, |delta| at p = (1+delta) f, scale
+ * invariance, brute force in rationals, the angle between two plane vectors), "parity unpinned" by
+ * the paper itself.
+ *   l1:     sum |p - f| / (sum |f| + eps)
+ *   l-inf:  max |p - f| / (max |f| + eps)
+ *   cosine: 1 - <p, f> / (||p||_2 ||f||_2 + eps), a distance so that "accept iff value <= tau" holds
+ * A NaN element makes every one of them NaN (rejected).
+ */
+double oracle_rel_l1(int dtype, int64_t n, const void* pred, const void* fresh, double eps) {
+    double num = 0.0, den = 0.0;
+#pragma omp parallel for schedule(static) reduction(+ : num, den)
+    for (int64_t j = 0; j < n; ++j) {
+        double p = load_elem(pred, dtype, j);
+        double f = load_elem(fresh, dtype, j);
+        num += fabs(p - f);
+        den += fabs(f);
+    }
+    return num / (den + eps);
+}
+
+double oracle_rel_linf(int dtype, int64_t n, const void* pred, const void* fresh, double eps) {
+    double num = 0.0, den = 0.0;
+    int bad = 0;
+    for (int64_t j = 0; j < n; ++j) {
+        double p = load_elem(pred, dtype, j);
+        double f = load_elem(fresh, dtype, j);
+        double d = fabs(p - f), a = fabs(f);
+        if (isnan(d) || isnan(a)) bad = 1;
+        if (d > num) num = d;
+        if (a > den) den = a;
+    }
+    if (bad) return NAN;
+    return num / (den + eps);
+}
+
+double oracle_cos_dist(int dtype, int64_t n, const void* pred, const void* fresh, double eps) {
+    double dot = 0.0, pp = 0.0, ff = 0.0;
+#pragma omp parallel for schedule(static) reduction(+ : dot, pp, ff)
+    for (int64_t j = 0; j < n; ++j) {
+        double p = load_elem(pred, dtype, j);
+        double f = load_elem(fresh, dtype, j);
+        dot += p * f;
+        pp += p * p;
+        ff += f * f;
+    }
+    return 1.0 - dot / (sqrt(pp) * sqrt(ff) + eps);
 }
 
 /* Section 3.4.2: accepted iff e <= tau. A NaN error compares false and is rejected. */

@@ -25,6 +25,7 @@ _LIB = os.path.join(_HERE, "libspeca_oracle.so")
 
 F32, BF16 = 0, 1
 TAYLOR, NEWTON = 0, 1
+METRIC_L2, METRIC_L1, METRIC_LINF, METRIC_COSINE = 0, 1, 2, 3
 EPS_PAPER = 1e-8  # Eq. 4
 
 
@@ -54,6 +55,9 @@ def lib() -> ctypes.CDLL:
         L.oracle_forecast_segment.restype = i32
         L.oracle_rel_l2.argtypes = [i32, i64, vp, vp, dbl]
         L.oracle_rel_l2.restype = dbl
+        for fn in (L.oracle_rel_l1, L.oracle_rel_linf, L.oracle_cos_dist):
+            fn.argtypes = [i32, i64, vp, vp, dbl]
+            fn.restype = dbl
         L.oracle_accept.argtypes = [dbl, dbl]
         L.oracle_accept.restype = i32
         L.oracle_tau.argtypes = [dbl, dbl, dbl, dbl]
@@ -112,6 +116,15 @@ def rel_l2(dtype, pred: np.ndarray, fresh: np.ndarray, eps: float = EPS_PAPER) -
     assert pred.flags.c_contiguous and fresh.flags.c_contiguous and pred.size == fresh.size
     assert pred.dtype == fresh.dtype == np_dtype(dtype)
     return float(lib().oracle_rel_l2(dtype, pred.size, _ptr(pred), _ptr(fresh), float(eps)))
+
+
+def rel_err(metric: int, dtype, pred: np.ndarray, fresh: np.ndarray, eps: float = EPS_PAPER) -> float:
+    """Eq. 4 (metric 0) or one of the appendix's other metrics over one sample."""
+    assert pred.flags.c_contiguous and fresh.flags.c_contiguous and pred.size == fresh.size
+    assert pred.dtype == fresh.dtype == np_dtype(dtype)
+    fn = {METRIC_L2: lib().oracle_rel_l2, METRIC_L1: lib().oracle_rel_l1, METRIC_LINF: lib().oracle_rel_linf,
+          METRIC_COSINE: lib().oracle_cos_dist}[metric]
+    return float(fn(dtype, pred.size, _ptr(pred), _ptr(fresh), float(eps)))
 
 
 def accept(err: float, tau: float) -> bool:
@@ -225,7 +238,7 @@ class OracleCache:
         return out
 
     def verify(self, fresh: np.ndarray, t_target: Sequence[float], tau: Sequence[float],
-               active: Optional[Sequence[int]] = None):
+               active: Optional[Sequence[int]] = None, metric: int = METRIC_L2):
         """Returns (err[B] float64 with NaN for skipped samples, accept[B] int with -1 for skipped,
         pred [B, n_v])."""
         e = self.verify_entry
@@ -235,6 +248,6 @@ class OracleCache:
         acc = np.full(self.B, -1, dtype=np.int64)
         for b in range(self.B):
             if (active is None or active[b]) and self.n_refs[b] >= 1:
-                err[b] = rel_l2(self.dtype, pred[b], fresh[b], self.eps)
+                err[b] = rel_err(metric, self.dtype, pred[b], fresh[b], self.eps)
                 acc[b] = 1 if accept(err[b], float(np.float32(tau[b]))) else 0
         return err, acc, pred

@@ -21,6 +21,7 @@ SPECA_ERR_INVALID_ARG, SPECA_ERR_SHAPE, SPECA_ERR_ALIGNMENT, SPECA_ERR_STATE = 1
 SPECA_ERR_ZERO_GAP, SPECA_ERR_NOMEM, SPECA_ERR_CUDA, SPECA_ERR_UNSUPPORTED = 5, 6, 7, 8
 SPECA_F32, SPECA_BF16 = 0, 1
 SPECA_BASIS_TAYLOR, SPECA_BASIS_NEWTON = 0, 1
+SPECA_METRIC_L2, SPECA_METRIC_L1, SPECA_METRIC_LINF, SPECA_METRIC_COSINE = 0, 1, 2, 3
 SPECA_PATH_AUTO, SPECA_PATH_DIRECT, SPECA_PATH_BULK, SPECA_PATH_WIDE = 0, 1, 2, 3
 SPECA_MAX_ORDER, SPECA_MAX_BATCH, SPECA_MAX_ENTRIES, SPECA_MAX_HORIZON = 4, 64, 512, 8
 
@@ -29,7 +30,7 @@ EXPORTS = [
     "speca_cache_update", "speca_cache_commit_step", "speca_forecast", "speca_verify",
     "speca_select_adaptive", "speca_activate", "speca_tau", "speca_cache_state", "speca_cache_plane",
     "speca_cache_launch_count", "speca_status_string", "speca_last_error", "speca_version",
-    "speca_verify_pred_static", "speca_forecast_multi",
+    "speca_verify_pred_static", "speca_forecast_multi", "speca_verify_metric",
 ]
 
 
@@ -76,6 +77,7 @@ def _lib() -> ctypes.CDLL:
     L.speca_forecast.argtypes = [vp, vp, vp, vp, vp]
     L.speca_forecast_multi.argtypes = [vp, i32, vp, vp, vp, vp]
     L.speca_verify.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.speca_verify_metric.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     L.speca_select_adaptive.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, vp]
     L.speca_activate.argtypes = [vp, vp, vp, vp, vp]
     L.speca_verify_pred_static.argtypes = [vp, vp, ctypes.c_int64, i32, i32, vp, ctypes.c_float, vp, vp, vp, i32, vp]
@@ -212,6 +214,13 @@ def speca_verify(cache, fresh, t_target, tau, dev_active_mask, out_pred, dev_err
            cache)
 
 
+def speca_verify_metric(cache, metric, fresh, t_target, tau, dev_active_mask, out_pred, dev_err, dev_accept,
+                        stream=None) -> None:
+    _check(_lib().speca_verify_metric(cache, int(metric), _dev_ptr(fresh), _doubles(t_target), _floats(tau),
+                                      _dev_ptr(dev_active_mask), _dev_ptr(out_pred), _dev_ptr(dev_err),
+                                      _dev_ptr(dev_accept), _stream_ptr(stream)), cache)
+
+
 def speca_select_adaptive(cache, dev_accept, k_max, group, dev_spec_count, dev_active_mask, dev_active_idx=None,
                           dev_n_active=None, stream=None) -> None:
     _check(_lib().speca_select_adaptive(cache, _dev_ptr(dev_accept), int(k_max), int(group), _dev_ptr(dev_spec_count),
@@ -308,8 +317,11 @@ class SpecaCache:
     def forecast_multi(self, t_targets, outs, active=None, stream=None):
         speca_forecast_multi(self.handle, t_targets, active, outs, stream)
 
-    def verify(self, fresh, t_target, tau, err, accept, active=None, out_pred=None, stream=None):
-        speca_verify(self.handle, fresh, t_target, tau, active, out_pred, err, accept, stream)
+    def verify(self, fresh, t_target, tau, err, accept, active=None, out_pred=None, stream=None, metric=None):
+        if metric is None:
+            speca_verify(self.handle, fresh, t_target, tau, active, out_pred, err, accept, stream)
+        else:
+            speca_verify_metric(self.handle, metric, fresh, t_target, tau, active, out_pred, err, accept, stream)
 
     def select_adaptive(self, accept, k_max, group, spec_count, active, idx=None, n_active=None, stream=None):
         speca_select_adaptive(self.handle, accept, k_max, group, spec_count, active, idx, n_active, stream)

@@ -53,7 +53,7 @@ speca_status_t make_layout(const speca_cache_config_t* cfg, Layout* L) {
         off = align_up(off + (n_segs + 1) * sizeof(uint32_t), kAlign);
     }
     L->partials_off = off;
-    off = align_up(off + static_cast<size_t>(kMaxClusters) * B * 2 * sizeof(float), kAlign);
+    off = align_up(off + static_cast<size_t>(kMaxClusters) * B * 3 * sizeof(float), kAlign);  // up to 3 values per metric
     L->ticket_off = off;
     off = align_up(off + 2 * sizeof(uint32_t), kPlaneAlign);
     L->tables_off = off;
@@ -490,7 +490,16 @@ speca_status_t speca_forecast_multi(speca_cache_t* c, int32_t n_targets, const d
 speca_status_t speca_verify(speca_cache_t* c, const void* fresh, const double* t_target, const float* tau,
                             const uint8_t* dev_active_mask, void* out_pred, float* dev_err, uint8_t* dev_accept,
                             void* stream) {
+    return speca_verify_metric(c, SPECA_METRIC_L2, fresh, t_target, tau, dev_active_mask, out_pred, dev_err, dev_accept,
+                               stream);
+}
+
+speca_status_t speca_verify_metric(speca_cache_t* c, int32_t metric, const void* fresh, const double* t_target,
+                                   const float* tau, const uint8_t* dev_active_mask, void* out_pred, float* dev_err,
+                                   uint8_t* dev_accept, void* stream) {
     if (c == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (metric < SPECA_METRIC_L2 || metric > SPECA_METRIC_COSINE)
+        return fail(c, SPECA_ERR_INVALID_ARG, "verify: unknown metric %d", metric);
     if (fresh == nullptr || t_target == nullptr || tau == nullptr || dev_err == nullptr || dev_accept == nullptr)
         return fail(c, SPECA_ERR_INVALID_ARG, "verify: null argument");
     if (c->pending) return fail(c, SPECA_ERR_STATE, "verify: a reference step is open (commit it first)");
@@ -536,6 +545,7 @@ speca_status_t speca_verify(speca_cache_t* c, const void* fresh, const double* t
     p.tiles_per_sample = (s0.n_elems + te - 1) / te;
     p.units_per_sample = (p.tiles_per_sample + c->cluster - 1) / c->cluster;
     p.batch = c->B;
+    p.metric = metric;
     p.eps = c->eps;
     const uint64_t units = static_cast<uint64_t>(p.units_per_sample) * c->B;
     int grid = c->grid_verify;

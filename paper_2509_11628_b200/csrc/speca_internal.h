@@ -75,12 +75,13 @@ struct VerifyParams {
     char* out_pred;     // may be null
     float* err;
     uint8_t* accept;
-    float* partials;     // [n_clusters][B][2]
+    float* partials;     // [n_clusters][B][values of the metric: 2, or 3 for cosine]
     uint32_t* ticket;    // arrival counter, zero between launches
     uint32_t n_elems;    // per sample
     uint32_t tiles_per_sample;
     uint32_t units_per_sample;  // ceil(tiles_per_sample / cluster size)
     int32_t batch;
+    int32_t metric;  // speca_metric_t
     double eps;
     int8_t order[SPECA_MAX_BATCH];
     float coef[SPECA_MAX_BATCH][SPECA_MAX_ORDER];

@@ -751,7 +751,7 @@ __global__ void __launch_bounds__(kBulkThreads) stream_bulk_kernel(const __grid_
 }
 
 // ------------------------------------------------------------------------------------------------
-// verify: forecast of one entry fused with the two sums of squares of Eq. 4
+// verify: forecast of one entry fused with the reduction of Eq. 4 (or of another error metric)
 // ------------------------------------------------------------------------------------------------
 
 constexpr int kMaxClusterSize = 8;
@@ -760,10 +760,59 @@ constexpr int kVerifyW = 32;
 static_assert(verify_tile_bytes(0) == kThreads * 2 * kVerifyW && verify_tile_bytes(4) == kThreads * kVerifyW,
               "verify tile sizes");
 
-template <int DT, int V, int W, int U>
+// Error metrics of the verification. Eq. 4 is the relative l2 error; the appendix on error metrics
+// also evaluates l1, l-infinity and cosine similarity, all in relative form. Each metric keeps NA
+// running values per sample, folds one (forecast, feature) pair into them, merges two partial
+// results, and turns the totals into the error e that is compared with tau.
+//   L2    a0 = sum (p-f)^2, a1 = sum f^2            e = sqrt(a0) / (sqrt(a1) + eps)
+//   L1    a0 = sum |p-f|,   a1 = sum |f|            e = a0 / (a1 + eps)
+//   LINF  a0 = max |p-f|,   a1 = max |f|            e = a0 / (a1 + eps)
+//   COS   a0 = sum p f, a1 = sum p^2, a2 = sum f^2  e = 1 - a0 / (sqrt(a1) sqrt(a2) + eps)
+// A NaN in any element must reach e (and reject the sample), so the maxima propagate NaN.
+__device__ __forceinline__ float nan_max(float a, float b) { return (a > b || a != a) ? a : b; }
+__device__ __forceinline__ double nan_max(double a, double b) { return (a > b || a != a) ? a : b; }
+
+template <int M>
+struct Metric {
+    static constexpr int NA = (M == SPECA_METRIC_COSINE) ? 3 : 2;
+    __device__ static __forceinline__ void fold(float p, float f, float (&a)[3]) {
+        if constexpr (M == SPECA_METRIC_L2) {
+            const float d = p - f;
+            a[0] = fmaf(d, d, a[0]);
+            a[1] = fmaf(f, f, a[1]);
+        } else if constexpr (M == SPECA_METRIC_L1) {
+            a[0] += fabsf(p - f);
+            a[1] += fabsf(f);
+        } else if constexpr (M == SPECA_METRIC_LINF) {
+            a[0] = nan_max(a[0], fabsf(p - f));
+            a[1] = nan_max(a[1], fabsf(f));
+        } else {
+            a[0] = fmaf(p, f, a[0]);
+            a[1] = fmaf(p, p, a[1]);
+            a[2] = fmaf(f, f, a[2]);
+        }
+    }
+    template <typename T>
+    __device__ static __forceinline__ T merge(T x, T y) {
+        if constexpr (M == SPECA_METRIC_LINF)
+            return nan_max(x, y);
+        else
+            return x + y;
+    }
+    __device__ static __forceinline__ double error(const double (&s)[3], double eps) {
+        if constexpr (M == SPECA_METRIC_L2)
+            return sqrt(s[0]) / (sqrt(s[1]) + eps);
+        else if constexpr (M == SPECA_METRIC_COSINE)
+            return 1.0 - s[0] / (sqrt(s[1]) * sqrt(s[2]) + eps);
+        else
+            return s[0] / (s[1] + eps);
+    }
+};
+
+template <int DT, int V, int W, int U, int M>
 __device__ __forceinline__ void verify_tile(const char* __restrict__ plane0, uint64_t stride,
                                             const char* __restrict__ fresh, char* __restrict__ out_pred, uint32_t cnt,
-                                            const float (&mu)[SPECA_MAX_ORDER], float& num, float& den) {
+                                            const float (&mu)[SPECA_MAX_ORDER], float (&a)[3]) {
     constexpr int EPV = W / Elem<DT>::kBytes;
     const uint32_t nvec = cnt / EPV;
     Vec<W> d[V + 1][U];
@@ -796,9 +845,7 @@ __device__ __forceinline__ void verify_tile(const char* __restrict__ plane0, uin
             unpack_vec<DT, W>(fv[u], f);
 #pragma unroll
             for (int k = 0; k < EPV; ++k) {
-                const float diff = acc[k] - f[k];
-                num = fmaf(diff, diff, num);
-                den = fmaf(f[k], f[k], den);
+                Metric<M>::fold(acc[k], f[k], a);
             }
             if (out_pred != nullptr) store_vec<W>(out_pred + static_cast<size_t>(idx) * W, pv);
         }
@@ -809,17 +856,15 @@ __device__ __forceinline__ void verify_tile(const char* __restrict__ plane0, uin
         for (int i = V; i >= 1; --i) acc = fmaf(acc, mu[i - 1], load_scalar<DT>(plane0 + (i - 1) * stride, j));
         acc = round_storage<DT>(acc);
         const float f = load_scalar<DT>(fresh, j);
-        const float diff = acc - f;
-        num = fmaf(diff, diff, num);
-        den = fmaf(f, f, den);
+        Metric<M>::fold(acc, f, a);
         if (out_pred != nullptr) store_scalar<DT>(out_pred, j, acc);
     }
 }
 
-template <int DT>
+template <int DT, int M>
 __device__ __noinline__ void verify_tile_any(const char* __restrict__ plane0, uint64_t stride,
                                              const char* __restrict__ fresh, char* __restrict__ out_pred, uint32_t cnt,
-                                             int v, const float (&mu)[SPECA_MAX_ORDER], float& num, float& den) {
+                                             int v, const float (&mu)[SPECA_MAX_ORDER], float (&a)[3]) {
     constexpr int EPV = Elem<DT>::kEPV;
     const bool vec_ok = ((reinterpret_cast<uintptr_t>(fresh) | reinterpret_cast<uintptr_t>(out_pred) |
                           reinterpret_cast<uintptr_t>(plane0)) & 15u) == 0;
@@ -838,9 +883,7 @@ __device__ __noinline__ void verify_tile_any(const char* __restrict__ plane0, ui
         unpack<DT>(__ldcs(reinterpret_cast<const uint4*>(fresh) + idx), f);
 #pragma unroll
         for (int k = 0; k < EPV; ++k) {
-            const float diff = acc[k] - f[k];
-            num = fmaf(diff, diff, num);
-            den = fmaf(f[k], f[k], den);
+            Metric<M>::fold(acc[k], f[k], a);
         }
         if (out_pred != nullptr) __stcs(reinterpret_cast<uint4*>(out_pred) + idx, pv);
     }
@@ -849,9 +892,7 @@ __device__ __noinline__ void verify_tile_any(const char* __restrict__ plane0, ui
         for (int i = v; i >= 1; --i) acc = fmaf(acc, mu[i - 1], load_scalar<DT>(plane0 + (i - 1) * stride, j));
         acc = round_storage<DT>(acc);
         const float f = load_scalar<DT>(fresh, j);
-        const float diff = acc - f;
-        num = fmaf(diff, diff, num);
-        den = fmaf(f, f, den);
+        Metric<M>::fold(acc, f, a);
         if (out_pred != nullptr) store_scalar<DT>(out_pred, j, acc);
     }
 }
@@ -877,7 +918,7 @@ __device__ __forceinline__ int nth_set_bit(uint64_t bits, uint32_t a) {
 // cluster's distributed shared memory -> one partial per (cluster, sample) in global scratch. The
 // cluster that arrives last (ticket counter, nobody waits) adds each sample's partials in fp64, one
 // warp per sample in a fixed lane/shuffle order, and applies Eq. 4 and the accept rule.
-template <int DT, int V>
+template <int DT, int V, int M>
 __global__ void __launch_bounds__(kThreads, 2) verify_kernel(const __grid_constant__ VerifyParams p) {
     constexpr uint32_t kTile = verify_tile_bytes(V) / Elem<DT>::kBytes;
     constexpr int W = kVerifyW, U = verify_tile_bytes(V) / (kThreads * kVerifyW);
@@ -887,8 +928,9 @@ __global__ void __launch_bounds__(kThreads, 2) verify_kernel(const __grid_consta
     const uint32_t cid = blockIdx.x / csize;
     const uint32_t Q = gridDim.x / csize;
 
-    __shared__ float warp_part[2][kThreads / 32];
-    __shared__ float cluster_slot[2][2][kMaxClusterSize];  // [parity][num|den][rank], leader's copy is used
+    constexpr int NA = Metric<M>::NA;
+    __shared__ float warp_part[NA][kThreads / 32];
+    __shared__ float cluster_slot[2][NA][kMaxClusterSize];  // [parity][value][rank], leader's copy is used
     __shared__ uint32_t active_bits[2];
     __shared__ bool is_last;
 
@@ -906,48 +948,43 @@ __global__ void __launch_bounds__(kThreads, 2) verify_kernel(const __grid_consta
     const uint32_t tps = p.tiles_per_sample;
     const uint32_t T = n_active * tps;
 
-    float num = 0.f, den = 0.f;
+    float acc[3] = {0.f, 0.f, 0.f};
     uint32_t parity = 0;
 
     auto flush = [&](int b) {
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            num += __shfl_xor_sync(0xFFFFFFFFu, num, off);
-            den += __shfl_xor_sync(0xFFFFFFFFu, den, off);
-        }
-        if ((threadIdx.x & 31) == 0) {
-            warp_part[0][threadIdx.x >> 5] = num;
-            warp_part[1][threadIdx.x >> 5] = den;
+        for (int i = 0; i < NA; ++i) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1)
+                acc[i] = Metric<M>::merge(acc[i], __shfl_xor_sync(0xFFFFFFFFu, acc[i], off));
+            if ((threadIdx.x & 31) == 0) warp_part[i][threadIdx.x >> 5] = acc[i];
         }
         __syncthreads();
         if (threadIdx.x == 0) {
-            float n = 0.f, d = 0.f;
-#pragma unroll
-            for (int w = 0; w < kThreads / 32; ++w) {
-                n += warp_part[0][w];
-                d += warp_part[1][w];
-            }
-            // hand the CTA's sums to the cluster leader through distributed shared memory
+            // hand the CTA's values to the cluster leader through distributed shared memory
             float* leader = cluster.map_shared_rank(&cluster_slot[parity][0][0], 0);
-            leader[crank] = n;
-            leader[kMaxClusterSize + crank] = d;
+#pragma unroll
+            for (int i = 0; i < NA; ++i) {
+                float s = warp_part[i][0];
+#pragma unroll
+                for (int w = 1; w < kThreads / 32; ++w) s = Metric<M>::merge(s, warp_part[i][w]);
+                leader[i * kMaxClusterSize + crank] = s;
+            }
         }
         cluster.sync();
         if (crank == 0 && threadIdx.x == 0) {
-            float n = 0.f, d = 0.f;
-            for (uint32_t r = 0; r < csize; ++r) {
-                n += cluster_slot[parity][0][r];
-                d += cluster_slot[parity][1][r];
+            float* dst = p.partials + (static_cast<size_t>(cid) * p.batch + b) * NA;
+#pragma unroll
+            for (int i = 0; i < NA; ++i) {
+                float s = cluster_slot[parity][i][0];
+                for (uint32_t r = 1; r < csize; ++r) s = Metric<M>::merge(s, cluster_slot[parity][i][r]);
+                __stcg(dst + i, s);
             }
-            float* dst = p.partials + (static_cast<size_t>(cid) * p.batch + b) * 2;
-            __stcg(dst, n);
-            __stcg(dst + 1, d);
         }
         // Slots alternate between two buffers: a CTA can write the buffer of flush k+2 only after
         // the barrier of flush k+1, which the leader enters after it has read the buffer of flush k.
         parity ^= 1;
-        num = 0.f;
-        den = 0.f;
+        acc[0] = acc[1] = acc[2] = 0.f;
     };
 
     const uint32_t t_lo = range_begin(cid, Q, T), t_hi = range_begin(cid + 1, Q, T);
@@ -970,9 +1007,9 @@ __global__ void __launch_bounds__(kThreads, 2) verify_kernel(const __grid_consta
                 const bool fast = v == V && ((reinterpret_cast<uintptr_t>(plane0) | reinterpret_cast<uintptr_t>(fresh) |
                                               reinterpret_cast<uintptr_t>(pred)) & (W - 1)) == 0;
                 if (fast)
-                    verify_tile<DT, V, W, U>(plane0, sd.plane_stride, fresh, pred, cnt, mu, num, den);
+                    verify_tile<DT, V, W, U, M>(plane0, sd.plane_stride, fresh, pred, cnt, mu, acc);
                 else
-                    verify_tile_any<DT>(plane0, sd.plane_stride, fresh, pred, cnt, v, mu, num, den);
+                    verify_tile_any<DT, M>(plane0, sd.plane_stride, fresh, pred, cnt, v, mu, acc);
             }
             flush(b);
         }
@@ -992,19 +1029,19 @@ __global__ void __launch_bounds__(kThreads, 2) verify_kernel(const __grid_consta
     for (uint32_t a = warp; a < n_active; a += kThreads / 32) {
         const int b = nth_set_bit(bits, a);
         const uint32_t q_lo = range_owner(a * tps, Q, T), q_hi = range_owner((a + 1) * tps - 1, Q, T);
-        double sn = 0.0, sd = 0.0;
+        double s[3] = {0.0, 0.0, 0.0};
         for (uint32_t q = q_lo + lane; q <= q_hi; q += 32) {
-            const float* src = p.partials + (static_cast<size_t>(q) * p.batch + b) * 2;
-            sn += static_cast<double>(__ldcg(src));
-            sd += static_cast<double>(__ldcg(src + 1));
+            const float* src = p.partials + (static_cast<size_t>(q) * p.batch + b) * NA;
+#pragma unroll
+            for (int i = 0; i < NA; ++i) s[i] = Metric<M>::merge(s[i], static_cast<double>(__ldcg(src + i)));
         }
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            sn += __shfl_xor_sync(0xFFFFFFFFu, sn, off);
-            sd += __shfl_xor_sync(0xFFFFFFFFu, sd, off);
+        for (int i = 0; i < NA; ++i) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) s[i] = Metric<M>::merge(s[i], __shfl_xor_sync(0xFFFFFFFFu, s[i], off));
         }
         if (lane == 0) {
-            const double e = sqrt(sn) / (sqrt(sd) + p.eps);
+            const double e = Metric<M>::error(s, p.eps);
             p.err[b] = static_cast<float>(e);
             p.accept[b] = (e <= static_cast<double>(p.tau[b])) ? 1 : 0;  // NaN compares false: reject
         }
@@ -1097,14 +1134,24 @@ static const void* stream_kernel_for(int dtype, bool update, int path, int v) {
                                : stream_kernel_for<SPECA_F32, false, SPECA_PATH_DIRECT>(v);
 }
 
-template <int DT>
+template <int DT, int M>
 static const void* verify_kernel_for(int v) {
     switch (v) {
-        case 0: return reinterpret_cast<const void*>(&verify_kernel<DT, 0>);
-        case 1: return reinterpret_cast<const void*>(&verify_kernel<DT, 1>);
-        case 2: return reinterpret_cast<const void*>(&verify_kernel<DT, 2>);
-        case 3: return reinterpret_cast<const void*>(&verify_kernel<DT, 3>);
-        default: return reinterpret_cast<const void*>(&verify_kernel<DT, 4>);
+        case 0: return reinterpret_cast<const void*>(&verify_kernel<DT, 0, M>);
+        case 1: return reinterpret_cast<const void*>(&verify_kernel<DT, 1, M>);
+        case 2: return reinterpret_cast<const void*>(&verify_kernel<DT, 2, M>);
+        case 3: return reinterpret_cast<const void*>(&verify_kernel<DT, 3, M>);
+        default: return reinterpret_cast<const void*>(&verify_kernel<DT, 4, M>);
+    }
+}
+
+template <int DT>
+static const void* verify_kernel_for(int metric, int v) {
+    switch (metric) {
+        case SPECA_METRIC_L1: return verify_kernel_for<DT, SPECA_METRIC_L1>(v);
+        case SPECA_METRIC_LINF: return verify_kernel_for<DT, SPECA_METRIC_LINF>(v);
+        case SPECA_METRIC_COSINE: return verify_kernel_for<DT, SPECA_METRIC_COSINE>(v);
+        default: return verify_kernel_for<DT, SPECA_METRIC_L2>(v);
     }
 }
 
@@ -1220,7 +1267,8 @@ cudaError_t launch_verify(const VerifyParams& p, int dtype, int grid, int cluste
     cudaLaunchAttribute attr[1];
     verify_config(&cfg, attr, grid, cluster, stream);
     const int v = max_order(p.order);
-    const void* fn = dtype == SPECA_BF16 ? verify_kernel_for<SPECA_BF16>(v) : verify_kernel_for<SPECA_F32>(v);
+    const void* fn = dtype == SPECA_BF16 ? verify_kernel_for<SPECA_BF16>(p.metric, v)
+                                         : verify_kernel_for<SPECA_F32>(p.metric, v);
     void* args[1] = {const_cast<VerifyParams*>(&p)};
     return cudaLaunchKernelExC(&cfg, fn, args);
 }
@@ -1233,7 +1281,8 @@ int max_resident_verify_clusters(int dtype, int order, int cluster) {
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
     verify_config(&cfg, attr, cluster, cluster, nullptr);
-    const void* fn = dtype == SPECA_BF16 ? verify_kernel_for<SPECA_BF16>(order) : verify_kernel_for<SPECA_F32>(order);
+    const void* fn = dtype == SPECA_BF16 ? verify_kernel_for<SPECA_BF16>(SPECA_METRIC_L2, order)
+                                         : verify_kernel_for<SPECA_F32>(SPECA_METRIC_L2, order);
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, fn, &cfg) != cudaSuccess || n < 1) {
         (void)cudaGetLastError();

@@ -363,6 +363,100 @@ def test_relative_error_brute_force_in_rationals(dtype):
         assert O.rel_l2(dtype, p, f) == pytest.approx(want, rel=1e-13)
 
 
+# ---------------------------------------------------------------------------------------------
+# the appendix's other error metrics (named there without formulas: pinned by the mathematics)
+# ---------------------------------------------------------------------------------------------
+
+OTHER_METRICS = [O.METRIC_L1, O.METRIC_LINF, O.METRIC_COSINE]
+
+
+def test_other_metrics_hand_examples():
+    f = np.array([3.0, -4.0, 1.0], dtype=np.float32)
+    p = np.array([2.0, -6.0, 1.5], dtype=np.float32)      # differences -1, -2, 0.5
+    assert O.rel_err(O.METRIC_L1, O.F32, p, f) == pytest.approx(3.5 / (8.0 + 1e-8), rel=1e-15)
+    assert O.rel_err(O.METRIC_LINF, O.F32, p, f) == pytest.approx(2.0 / (4.0 + 1e-8), rel=1e-15)
+    dot, pp, ff = 6.0 + 24.0 + 1.5, 4.0 + 36.0 + 2.25, 26.0
+    assert O.rel_err(O.METRIC_COSINE, O.F32, p, f) == pytest.approx(
+        1.0 - dot / (math.sqrt(pp) * math.sqrt(ff) + 1e-8), rel=1e-14)
+    assert O.rel_err(O.METRIC_L2, O.F32, p, f) == O.rel_l2(O.F32, p, f)
+    # two unit vectors in the plane at angle theta: cosine distance 1 - cos(theta)
+    for theta in (0.0, 0.3, math.pi / 2, 2.5, math.pi):
+        a = np.array([1.0, 0.0], dtype=np.float32)
+        b = np.array([math.cos(theta), math.sin(theta)], dtype=np.float32)
+        assert O.rel_err(O.METRIC_COSINE, O.F32, a, b) == pytest.approx(1.0 - math.cos(theta), abs=2e-7)
+    # orthogonal -> 1, opposite -> 2
+    assert O.rel_err(O.METRIC_COSINE, O.F32, np.array([1, 0], np.float32), np.array([0, 5], np.float32)) == pytest.approx(1.0, abs=1e-12)
+    assert O.rel_err(O.METRIC_COSINE, O.F32, f, -f) == pytest.approx(2.0, abs=1e-7)
+
+
+@pytest.mark.parametrize("metric", OTHER_METRICS)
+def test_other_metrics_properties(metric):
+    g = torch.Generator().manual_seed(31 + metric)
+    f = torch.randn(4000, generator=g).to(torch.bfloat16).to(torch.float32).numpy()   # 8 significant bits
+    p = (f + 0.1 * torch.randn(4000, generator=g).numpy()).astype(np.float32)
+    e = O.rel_err(metric, O.F32, p, f)
+    assert e > 0
+    # forecast equal to the feature: zero error
+    assert O.rel_err(metric, O.F32, f, f) == pytest.approx(0.0, abs=1e-7)
+    # common scale factor (a power of two: exact) leaves the value unchanged
+    assert O.rel_err(metric, O.F32, (4 * p).astype(np.float32), (4 * f).astype(np.float32)) == pytest.approx(e, rel=1e-7)
+    delta = 2.0 ** -3
+    pf = (f * np.float32(1 + delta)).astype(np.float32)   # exact in binary32
+    if metric == O.METRIC_COSINE:
+        assert O.rel_err(metric, O.F32, pf, f) == pytest.approx(0.0, abs=1e-7)      # same direction
+        assert O.rel_err(metric, O.F32, f, p) == pytest.approx(e, rel=1e-9)         # symmetric
+        assert O.rel_err(metric, O.F32, (3 * p).astype(np.float32), f) == pytest.approx(e, abs=1e-6)
+    else:
+        assert O.rel_err(metric, O.F32, pf, f) == pytest.approx(delta, rel=1e-7)    # p = (1+d) f -> |d|
+        z = np.zeros_like(f)
+        assert O.rel_err(metric, O.F32, z, f) == pytest.approx(1.0, rel=1e-7)       # p = 0 -> ||f||/(||f||+eps)
+    # NaN anywhere -> NaN -> rejected
+    q = p.copy()
+    q[17] = np.nan
+    assert math.isnan(O.rel_err(metric, O.F32, q, f))
+    assert not O.accept(O.rel_err(metric, O.F32, q, f), 1e30)
+    q = f.copy()
+    q[5] = np.nan
+    assert math.isnan(O.rel_err(metric, O.F32, p, q))
+
+
+def test_norm_ordering_between_metrics():
+    # for any vector ||x||_inf <= ||x||_2 <= ||x||_1 <= sqrt(n) ||x||_2 <= n ||x||_inf : checked on the
+    # numerators by choosing the feature so that every denominator is 1 (a single unit entry)
+    g = torch.Generator().manual_seed(5)
+    n = 64
+    f = np.zeros(n, dtype=np.float32)
+    f[0] = 1.0
+    d = torch.randn(n, generator=g).numpy().astype(np.float32)
+    d[0] = 0.0
+    p = (f + d).astype(np.float32)
+    l1, l2, li = (O.rel_err(m, O.F32, p, f, eps=0.0) for m in (O.METRIC_L1, O.METRIC_L2, O.METRIC_LINF))
+    assert li <= l2 <= l1 <= math.sqrt(n) * l2 <= n * li
+    assert l1 == pytest.approx(float(np.abs(d.astype(np.float64)).sum()), rel=1e-12)
+    assert li == pytest.approx(float(np.abs(d).max()), rel=1e-12)
+
+
+@pytest.mark.parametrize("dtype", [O.F32, O.BF16])
+def test_other_metrics_brute_force_in_rationals(dtype):
+    g = torch.Generator().manual_seed(41)
+    for n in [1, 2, 7, 16]:
+        a, b = torch.randn(n, generator=g), torch.randn(n, generator=g)
+        if dtype == O.BF16:
+            p, f = bf16_bits(a), bf16_bits(b)
+            pv, fv = bits_to_f64(p), bits_to_f64(f)
+        else:
+            p, f = a.numpy().copy(), b.numpy().copy()
+            pv, fv = p.astype(np.float64), f.astype(np.float64)
+        P, F = [Fraction(float(x)) for x in pv], [Fraction(float(y)) for y in fv]
+        l1 = float(sum(abs(x - y) for x, y in zip(P, F))) / (float(sum(abs(y) for y in F)) + 1e-8)
+        li = float(max(abs(x - y) for x, y in zip(P, F))) / (float(max(abs(y) for y in F)) + 1e-8)
+        cs = 1.0 - float(sum(x * y for x, y in zip(P, F))) / (
+            math.sqrt(sum(x * x for x in P)) * math.sqrt(sum(y * y for y in F)) + 1e-8)
+        assert O.rel_err(O.METRIC_L1, dtype, p, f) == pytest.approx(l1, rel=1e-13)
+        assert O.rel_err(O.METRIC_LINF, dtype, p, f) == pytest.approx(li, rel=1e-13)
+        assert O.rel_err(O.METRIC_COSINE, dtype, p, f) == pytest.approx(cs, abs=1e-13)
+
+
 def test_accept_rule():
     assert O.accept(0.5, 0.5)            # equality accepts
     assert O.accept(0.0, 0.0)
