@@ -69,8 +69,15 @@ typedef enum { SPECA_F32 = 0, SPECA_BF16 = 1 } speca_dtype_t;
  *  SPECA_BASIS_NEWTON  Newton divided differences over the true reference times, evaluated in
  *                      Newton form. Exact for polynomials of degree <= m at any gaps. Same
  *                      kernels, different host-computed scalars.
+ *  SPECA_BASIS_ADAMS_BASHFORTH  The alternative draft model of the appendix's draft-model ablation
+ *                      (named there without a formula). Tables as in the Taylor basis; the forecast
+ *                      is F + x * sum_j b_j g_j with g_j the difference-quotient slope j references
+ *                      back and b the textbook Adams-Bashforth coefficients of as many steps as
+ *                      slopes are known (at most 4), which in Horner form over the planes is
+ *                      F + x (D_1 + h/2 (D_2 + 5h/6 (D_3 + 9h/10 D_4))), h = the latest reference gap.
+ *                      Same kernels again.
  */
-typedef enum { SPECA_BASIS_TAYLOR = 0, SPECA_BASIS_NEWTON = 1 } speca_basis_t;
+typedef enum { SPECA_BASIS_TAYLOR = 0, SPECA_BASIS_NEWTON = 1, SPECA_BASIS_ADAMS_BASHFORTH = 2 } speca_basis_t;
 
 /* Which kernel variant moves the data. Results are identical; only speed differs. */
 typedef enum {

@@ -43,7 +43,7 @@
 #define ORACLE_MAX_ORDER 8
 
 enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
-enum { ORACLE_TAYLOR = 0, ORACLE_NEWTON = 1 };
+enum { ORACLE_TAYLOR = 0, ORACLE_NEWTON = 1, ORACLE_ADAMS_BASHFORTH = 2 };
 
 /* ---- storage <-> double ------------------------------------------------------------------ */
 
@@ -134,6 +134,42 @@ int oracle_forecast_segment(int dtype, int64_t n, int m, int basis, int n_refs, 
                             double t_target, const void* planes, int64_t plane_stride, void* out) {
     if (n_refs < 1) return 1;
     int v = n_refs - 1 < m ? n_refs - 1 : m;
+    size_t esz0 = dtype == ORACLE_F32 ? 4 : 2;
+    if (basis == ORACLE_ADAMS_BASHFORTH && v >= 1) {
+        /*
+         * Adams-Bashforth draft model (appendix, ablation of draft models; named there without a
+         * formula -- this reading is "parity unpinned" by the paper). The table is kept as in the
+         * Taylor basis. With h = t_last - (previous reference time), plane 1 is the latest slope
+         * g_0 = (F_0 - F_1)/h and the slope j references back follows from the higher planes by
+         * backward differencing, g_j = sum_i C(j,i) (-h)^i plane_{1+i}. The v-step Adams-Bashforth
+         * formula with its textbook coefficients b extrapolates over x = t_target - t_last:
+         *     out = F_0 + x * sum_{j<v} b_j g_j   (b = row v-1 of the table below).
+         */
+        static const double b[4][4] = {{1.0, 0, 0, 0},
+                                       {3.0 / 2, -1.0 / 2, 0, 0},
+                                       {23.0 / 12, -16.0 / 12, 5.0 / 12, 0},
+                                       {55.0 / 24, -59.0 / 24, 37.0 / 24, -9.0 / 24}};
+        if (v > 4) return 1;
+        double x = t_target - t_hist[0];
+        double h = v >= 2 ? t_hist[0] - t_hist[1] : 0.0;
+#pragma omp parallel for schedule(static)
+        for (int64_t j = 0; j < n; ++j) {
+            double d[ORACLE_MAX_ORDER + 1];
+            for (int i = 0; i <= v; ++i) d[i] = load_elem((const char*)planes + (size_t)i * plane_stride * esz0, dtype, j);
+            double sum = 0.0;
+            for (int s = 0; s < v; ++s) { /* slope s references back */
+                double g = 0.0, binom = 1.0, hp = 1.0;
+                for (int i = 0; i <= s; ++i) {
+                    g += binom * hp * d[1 + i];
+                    binom = binom * (double)(s - i) / (double)(i + 1);
+                    hp *= -h;
+                }
+                sum += b[v - 1][s] * g;
+            }
+            store_elem(out, dtype, j, d[0] + x * sum);
+        }
+        return 0;
+    }
     double w[ORACLE_MAX_ORDER + 1]; /* weight of plane i */
     w[0] = 1.0;
     if (basis == ORACLE_NEWTON) {

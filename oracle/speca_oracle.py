@@ -24,7 +24,7 @@ _SRC = os.path.join(_HERE, "speca_oracle.c")
 _LIB = os.path.join(_HERE, "libspeca_oracle.so")
 
 F32, BF16 = 0, 1
-TAYLOR, NEWTON = 0, 1
+TAYLOR, NEWTON, ADAMS_BASHFORTH = 0, 1, 2
 METRIC_L2, METRIC_L1, METRIC_LINF, METRIC_COSINE = 0, 1, 2, 3
 EPS_PAPER = 1e-8  # Eq. 4
 

@@ -20,7 +20,7 @@ SPECA_OK = 0
 SPECA_ERR_INVALID_ARG, SPECA_ERR_SHAPE, SPECA_ERR_ALIGNMENT, SPECA_ERR_STATE = 1, 2, 3, 4
 SPECA_ERR_ZERO_GAP, SPECA_ERR_NOMEM, SPECA_ERR_CUDA, SPECA_ERR_UNSUPPORTED = 5, 6, 7, 8
 SPECA_F32, SPECA_BF16 = 0, 1
-SPECA_BASIS_TAYLOR, SPECA_BASIS_NEWTON = 0, 1
+SPECA_BASIS_TAYLOR, SPECA_BASIS_NEWTON, SPECA_BASIS_ADAMS_BASHFORTH = 0, 1, 2
 SPECA_METRIC_L2, SPECA_METRIC_L1, SPECA_METRIC_LINF, SPECA_METRIC_COSINE = 0, 1, 2, 3
 SPECA_PATH_AUTO, SPECA_PATH_DIRECT, SPECA_PATH_BULK, SPECA_PATH_WIDE = 0, 1, 2, 3
 SPECA_MAX_ORDER, SPECA_MAX_BATCH, SPECA_MAX_ENTRIES, SPECA_MAX_HORIZON = 4, 64, 512, 8

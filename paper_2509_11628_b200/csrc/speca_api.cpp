@@ -36,7 +36,9 @@ speca_status_t make_layout(const speca_cache_config_t* cfg, Layout* L) {
     if (cfg->batch < 1 || cfg->batch > SPECA_MAX_BATCH) return SPECA_ERR_SHAPE;
     if (cfg->max_order < 0 || cfg->max_order > SPECA_MAX_ORDER) return SPECA_ERR_SHAPE;
     if (cfg->dtype != SPECA_F32 && cfg->dtype != SPECA_BF16) return SPECA_ERR_INVALID_ARG;
-    if (cfg->basis != SPECA_BASIS_TAYLOR && cfg->basis != SPECA_BASIS_NEWTON) return SPECA_ERR_INVALID_ARG;
+    if (cfg->basis != SPECA_BASIS_TAYLOR && cfg->basis != SPECA_BASIS_NEWTON &&
+        cfg->basis != SPECA_BASIS_ADAMS_BASHFORTH)
+        return SPECA_ERR_INVALID_ARG;
     if (cfg->path != SPECA_PATH_AUTO && cfg->path != SPECA_PATH_DIRECT && cfg->path != SPECA_PATH_BULK &&
         cfg->path != SPECA_PATH_WIDE)
         return SPECA_ERR_INVALID_ARG;
@@ -158,6 +160,14 @@ void forecast_scalars(const speca_cache* c, int b, double t, int* order, float* 
     const int v = c->n_refs[b] < 1 ? -1 : (c->n_refs[b] - 1 < c->m ? c->n_refs[b] - 1 : c->m);
     *order = v;
     for (int i = 0; i < SPECA_MAX_ORDER; ++i) mu[i] = 0.f;
+    if (c->basis == SPECA_BASIS_ADAMS_BASHFORTH) {
+        // F + x (D_1 + h/2 (D_2 + 5h/6 (D_3 + 9h/10 D_4))): the v-step Adams-Bashforth sum over the
+        // slopes g_j = sum_i C(j,i) (-h)^i D_{1+i}, collected by plane (coefficients 1, 1/2, 5/12, 3/8)
+        static const double ratio[SPECA_MAX_ORDER] = {1.0, 1.0 / 2, 5.0 / 6, 9.0 / 10};
+        const double h = v >= 2 ? c->t_hist[b][0] - c->t_hist[b][1] : 0.0;
+        for (int i = 1; i <= v; ++i) mu[i - 1] = static_cast<float>(i == 1 ? t - c->t_hist[b][0] : ratio[i - 1] * h);
+        return;
+    }
     for (int i = 1; i <= v; ++i) {
         const double x = (c->basis == SPECA_BASIS_NEWTON) ? (t - c->t_hist[b][i - 1]) : (t - c->t_hist[b][0]) / i;
         mu[i - 1] = static_cast<float>(x);

@@ -131,6 +131,9 @@ class Pair:
         h = self.cpu.t_hist[b]
         v = min(self.m, self.cpu.n_refs[b] - 1)
         w = [1.0]
+        if self.basis == S.SPECA_BASIS_ADAMS_BASHFORTH:
+            x, hh = t - h[0], (h[0] - h[1]) if len(h) > 1 else 0.0
+            return w + [x * c * hh ** i for i, c in enumerate([1.0, 1 / 2, 5 / 12, 3 / 8][:v])]
         for i in range(1, v + 1):
             if self.basis == S.SPECA_BASIS_NEWTON:
                 w.append(w[-1] * (t - h[i - 1]))

@@ -76,7 +76,7 @@ RAGGED = [(37, 129), (5, 3), (64, 384), (1, 8192 * 2 + 24), (3, 8192), (1, 1)]
 
 @pytest.mark.parametrize("path", [1, 2, 3])  # SPECA_PATH_DIRECT, SPECA_PATH_BULK, SPECA_PATH_WIDE
 @pytest.mark.parametrize("dtype", [0, 1])
-@pytest.mark.parametrize("basis", [0, 1])
+@pytest.mark.parametrize("basis", [0, 1, 2])  # Taylor (Eq. 2-3), Newton, Adams-Bashforth
 @pytest.mark.parametrize("m", [0, 1, 2, 3, 4])
 def test_ragged_shapes_all_orders(S, U, dtype, basis, m, path):
     B = 3

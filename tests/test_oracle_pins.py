@@ -316,6 +316,86 @@ def test_bf16_tables_round_once_per_stored_plane():
 
 
 # ---------------------------------------------------------------------------------------------
+# Adams-Bashforth draft model (appendix: named without a formula; pinned by the textbook method)
+# ---------------------------------------------------------------------------------------------
+
+AB_COEF = {1: [Fraction(1)], 2: [Fraction(3, 2), Fraction(-1, 2)],
+           3: [Fraction(23, 12), Fraction(-16, 12), Fraction(5, 12)],
+           4: [Fraction(55, 24), Fraction(-59, 24), Fraction(37, 24), Fraction(-9, 24)]}
+
+
+@pytest.mark.parametrize("m", [1, 2, 3, 4])
+@pytest.mark.parametrize("h", [-2, -1, 4])
+def test_adams_bashforth_equals_textbook_formula_on_raw_history(m, h):
+    """From the raw feature history on a uniform grid: slopes g_j = (F_j - F_{j+1}) / h, then the
+    m-step Adams-Bashforth sum F_0 + x * sum b_j g_j, in exact rationals."""
+    rng = np.random.default_rng(100 + m)
+    n = 6
+    times = [Fraction(16 + h * k) for k in range(m + 1)]            # oldest first: 16, 16+h, ...
+    feats = [rng.integers(-40, 40, n).astype(np.float32) for _ in range(m + 1)]
+    planes, hist = run_history(O.F32, m, O.ADAMS_BASHFORTH, [float(t) for t in times], feats)
+    newest_first = feats[::-1]
+    for x in (Fraction(h), Fraction(h, 2), Fraction(3 * h)):
+        out = np.zeros(n, dtype=np.float32)
+        O.forecast_segment(O.F32, m, O.ADAMS_BASHFORTH, m + 1, hist, float(times[-1] + x), planes, out)
+        for e in range(n):
+            g = [(Fraction(float(newest_first[j][e])) - Fraction(float(newest_first[j + 1][e]))) / h for j in range(m)]
+            want = Fraction(float(newest_first[0][e])) + x * sum(b * gj for b, gj in zip(AB_COEF[m], g))
+            assert float(out[e]) == pytest.approx(float(want), rel=1e-6, abs=1e-5)
+
+
+def test_adams_bashforth_special_cases():
+    rng = np.random.default_rng(7)
+    n = 50
+    times = [1.0, 0.9, 0.8, 0.7]
+    feats = [rng.standard_normal(n).astype(np.float32) for _ in times]
+    # one step: Euler with the latest slope = the Taylor basis at order 1, bit for bit
+    pa, ha = run_history(O.F32, 1, O.ADAMS_BASHFORTH, times, feats)
+    pt, ht = run_history(O.F32, 1, O.TAYLOR, times, feats)
+    oa, ot = np.zeros(n, np.float32), np.zeros(n, np.float32)
+    O.forecast_segment(O.F32, 1, O.ADAMS_BASHFORTH, 4, ha, 0.63, pa, oa)
+    O.forecast_segment(O.F32, 1, O.TAYLOR, 4, ht, 0.63, pt, ot)
+    assert np.array_equal(oa, ot)
+    # the tables themselves are the Taylor-basis tables
+    p3a, _ = run_history(O.F32, 3, O.ADAMS_BASHFORTH, times, feats)
+    p3t, h3 = run_history(O.F32, 3, O.TAYLOR, times, feats)
+    assert np.array_equal(p3a, p3t)
+    # forecast at the reference time returns the feature; order 0 is plain reuse
+    o = np.zeros(n, np.float32)
+    O.forecast_segment(O.F32, 3, O.ADAMS_BASHFORTH, 4, h3, times[-1], p3a, o)
+    assert np.array_equal(o, feats[-1])
+    p0, h0 = run_history(O.F32, 0, O.ADAMS_BASHFORTH, times, feats)
+    O.forecast_segment(O.F32, 0, O.ADAMS_BASHFORTH, 4, h0, 0.5, p0, o)
+    assert np.array_equal(o, feats[-1])
+    # a feature that is linear in t is extrapolated exactly at every step count
+    lin = [(3.0 - 2.0 * t) * np.ones(n, dtype=np.float64) for t in times]
+    for m in (1, 2, 3):
+        pl, hl = run_history(O.F32, m, O.ADAMS_BASHFORTH, times, [v.astype(np.float32) for v in lin])
+        O.forecast_segment(O.F32, m, O.ADAMS_BASHFORTH, 4, hl, 0.55, pl, o)
+        assert np.allclose(o, 3.0 - 2.0 * 0.55, rtol=1e-5)
+
+
+def test_adams_bashforth_on_a_quadratic_closed_form():
+    """For F quadratic in t a secant slope is F' at the interval's midpoint, so the slopes are exact
+    samples of the (linear) derivative at t_0 - h/2 and t_0 - 3h/2. The 2-step combination
+    3/2 g_0 - 1/2 g_1 extrapolates a linear function half a step forward: it equals F'(t_0) exactly.
+    Hence forecast = F(t_0) + x F'(t_0), and the distance to the truth is the closed form c x^2."""
+    h = -0.125
+    times = [1.0, 1.0 + h, 1.0 + 2 * h]
+    a, bq, cq = 0.5, -1.25, 2.0
+    F = lambda s: a + bq * s + cq * s * s
+    dF = lambda s: bq + 2 * cq * s
+    feats = [np.full(4, F(s), dtype=np.float32) for s in times]
+    planes, hist = run_history(O.F32, 2, O.ADAMS_BASHFORTH, times, feats)
+    out = np.zeros(4, np.float32)
+    t0 = times[-1]
+    for x in (h, 0.5 * h, 3 * h):
+        O.forecast_segment(O.F32, 2, O.ADAMS_BASHFORTH, 3, hist, t0 + x, planes, out)
+        assert np.allclose(out, F(t0) + x * dF(t0), rtol=1e-6)
+        assert np.allclose(F(t0 + x) - out.astype(np.float64), cq * x * x, rtol=1e-4, atol=1e-7)
+
+
+# ---------------------------------------------------------------------------------------------
 # Eq. 4 and the accept rule
 # ---------------------------------------------------------------------------------------------
 
