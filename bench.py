@@ -405,6 +405,69 @@ def adaptive_sweep(device: str, peak: float, path: int, orders=(1, 2, 3), horizo
     return out
 
 
+def sampler_run(device: str, path: int, name: str):
+    """The whole forecast-then-verify loop (50 sampler steps) over the library with the seeded feature
+    generator standing in for the transformer: which steps each sample took in full, acceptance rate,
+    speed-up by the paper's cost model next to Eq. 8, and the device time the cache path itself took."""
+    from paper_2509_11628_b200 import binding as S
+    from paper_2509_11628_b200 import scheduler as SCH
+    w = W.flux_adaptive(max_order=2, batch=8) if name == "flux_adaptive" else W.BY_NAME[name]()
+    gamma = 1.0 / {"dit_xl2": 28, "flux": 57, "flux_adaptive": 57, "hunyuan_video": 60}[name]
+    cache = S.SpecaCache(w.entries, w.batch, w.max_order, w.dtype, device, path=path)
+    src = W.FeatureSource(w, device)
+
+    class Model:
+        def full(self, step, times, mask):
+            return [src.feature(e, step, times) for e in range(len(w.entries))]
+
+        def verify_feature(self, step, times):
+            return src.feature(w.vidx, step, times)
+
+    class Timed(SCH.SpecaCacheBackend):
+        def __init__(self, cache):
+            super().__init__(cache)
+            self.spans = {"forecast": [], "verify+select": [], "update": []}
+
+        def _timed(self, key, fn):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            out = fn()
+            e1.record()
+            self.spans[key].append((e0, e1))
+            return out
+
+        def forecast(self, t):
+            return self._timed("forecast", lambda: SCH.SpecaCacheBackend.forecast(self, t))
+
+        def verify_and_select(self, fresh, t, tau, period):
+            return self._timed("verify+select", lambda: SCH.SpecaCacheBackend.verify_and_select(self, fresh, t, tau, period))
+
+        def reference_step(self, feats, t, mask):
+            return self._timed("update", lambda: SCH.SpecaCacheBackend.reference_step(self, feats, t, mask))
+
+    be = Timed(cache)
+    wall0 = time.perf_counter()
+    tr = SCH.run_sampler(be, Model(), w.times, w.tau0, w.beta, w.period, w.warm_refs, gamma, total_steps=w.total_steps)
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - wall0
+    ms = {k: [a.elapsed_time(b_) for a, b_ in v] for k, v in be.spans.items()}
+    lib_ms = sum(sum(v) for v in ms.values())
+    res = {
+        "workload": w.name, "sampler_steps": len(w.times), "period": w.period, "warm_refs": w.warm_refs, "gamma": gamma,
+        "sigma": w.sigma, "acceptance_rate": tr.acceptance_rate(), "speedup_cost_model": tr.speedup(),
+        "speedup_eq8": tr.predicted_speedup(), "full_steps_histogram": tr.full_steps_histogram(),
+        "per_sample": ["".join(row[b] for row in tr.steps) for b in range(w.batch)],
+        "library_ms_total": lib_ms, "calls": {k: len(v) for k, v in ms.items()},
+        "ms_mean": {k: (sum(v) / len(v) if v else None) for k, v in ms.items()},
+        "sampler_steps_per_s_library_only": len(w.times) / (lib_ms * 1e-3) if lib_ms > 0 else None,
+        "wall_s_with_standin_model": wall,
+    }
+    cache.close()
+    del be, cache
+    torch.cuda.empty_cache()
+    return res
+
+
 def oracle_sample_run(w: W.Workload, sample_elems: int, repeats: int, seed: int = 0):
     """The CPU oracle, as it stands, on a bounded sample of the workload: `sample_elems` elements
     per sample of the verification entry go through one full step (update at order m, forecast,
@@ -577,6 +640,15 @@ def main():
         except Exception as exc:  # report, do not hide
             adaptive = {"error": repr(exc)}
 
+    sampler = None
+    if info.world == 1 and not args.no_adaptive:
+        sampler = {}
+        for name in ("dit_xl2", "flux_adaptive"):
+            try:
+                sampler[name] = sampler_run(device, path, name)
+            except Exception as exc:  # report, do not hide
+                sampler[name] = {"error": repr(exc)}
+
     if not info.is_main:
         D.shutdown()
         return
@@ -609,7 +681,7 @@ def main():
         "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches,
         "clocks": clocks, "kernels": kernels, **extra,
         "frac_of_measured_peak": value / info.world / peak, "frac_of_nominal_8TBs": value / info.world / NOMINAL_HBM_GBS,
-        "multi_horizon": multi, "verify_metrics": metrics, "per_config": per_config, "adaptive": adaptive,
+        "multi_horizon": multi, "verify_metrics": metrics, "per_config": per_config, "adaptive": adaptive, "sampler": sampler,
         "paper_context": {"end_to_end_speedups": {"flux_h800": 6.34, "dit_xl2_a800": 7.3, "hunyuan_video_h800": 6.1},
                           "verification_overhead": "1.67%-3.5% of a full forward pass",
                           "note": "other hardware, whole-model numbers; context only"},

@@ -1,0 +1,153 @@
+"""Forecast-then-verify control flow over the cache library (Section 3.2 workflow, Section 3.4.2
+sequential validation, the forced activation period of the appendix's hyper-parameters).
+
+This module holds control flow and bookkeeping only: every number it branches on (accept flags,
+active masks, thresholds) comes from the backend it drives -- the CUDA library through
+``SpecaCacheBackend`` below, or any object with the same methods. The model is a stand-in supplied by
+the caller: ``full(step, times, mask)`` returns the block outputs of a complete forward pass,
+``verify_feature(step, times)`` the freshly computed verification-layer feature of a speculative step.
+
+Per sampler step, per sample:
+  * a sample that is *active* attempts the step speculatively: its block outputs are forecast
+    (Eq. 2), the verification layer is computed for real, Eq. 4 is compared with tau_t;
+  * accepted (e <= tau_t): the step costs gamma (verification only) and the sample stays active
+    until it has taken ``period`` speculative steps in a row;
+  * rejected: the step is recomputed in full (Eq. 6 puts the rejected step in the rejection set), the
+    tables are updated from it, and the sample becomes active again;
+  * a sample that is not active takes a full step, updates its tables and becomes active.
+Samples of one batch therefore drift apart: each gets as many full steps as its own errors demand
+(sample-adaptive computation allocation).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import List, Sequence
+
+FULL, ACCEPTED, REJECTED = "F", "A", "R"
+
+
+@dataclass
+class Trace:
+    """What happened: ``steps[i][b]`` is FULL, ACCEPTED or REJECTED (rejected = verified, failed,
+    then recomputed in full). ``err[i][b]`` is the verification error where one was computed."""
+    batch: int
+    gamma: float
+    steps: List[List[str]] = field(default_factory=list)
+    err: List[List[float]] = field(default_factory=list)
+    tau: List[float] = field(default_factory=list)
+
+    def counts(self, b: int):
+        col = [row[b] for row in self.steps]
+        return col.count(FULL), col.count(ACCEPTED), col.count(REJECTED)
+
+    def acceptance_rate(self, b: int = None) -> float:
+        """alpha = speculative steps that were accepted / all steps (Section 3.5)."""
+        cols = range(self.batch) if b is None else [b]
+        acc = sum(self.counts(c)[1] for c in cols)
+        return acc / float(len(self.steps) * len(list(cols)))
+
+    def cost(self, b: int) -> float:
+        """In units of one full forward pass: full = 1, accepted = gamma, rejected = gamma + 1."""
+        f, a, r = self.counts(b)
+        return f + a * self.gamma + r * (1.0 + self.gamma)
+
+    def speedup(self, b: int = None) -> float:
+        cols = list(range(self.batch)) if b is None else [b]
+        return len(self.steps) * len(cols) / sum(self.cost(c) for c in cols)
+
+    def predicted_speedup(self, b: int = None) -> float:
+        """Eq. 8 with the measured acceptance rate: S = 1 / (1 - alpha + alpha * gamma)."""
+        a = self.acceptance_rate(b)
+        return 1.0 / (1.0 - a + a * self.gamma)
+
+    def full_steps_histogram(self):
+        """{number of full forward passes: how many samples needed that many}."""
+        hist = {}
+        for b in range(self.batch):
+            f, _, r = self.counts(b)
+            hist[f + r] = hist.get(f + r, 0) + 1
+        return dict(sorted(hist.items()))
+
+
+def run_sampler(backend, model, times: Sequence[float], tau0: float, beta: float, period: int, warm_refs: int,
+                gamma: float, total_steps: int = None) -> Trace:
+    """Drive ``backend`` through the whole timeline. ``times[i]`` is the sampler time of step i;
+    the first ``warm_refs`` steps are always full. ``period`` is the largest number of consecutive
+    speculative steps a sample may take."""
+    B = backend.batch
+    T = total_steps if total_steps is not None else len(times)
+    trace = Trace(batch=B, gamma=gamma)
+    active = [0] * B                      # host mirror of the device mask, refreshed once per step
+    backend.reset_run()
+    for i, t in enumerate(times):
+        tt = [t] * B
+        row = [FULL] * B
+        errs = [float("nan")] * B
+        tau_i = backend.tau(tau0, beta, T - i, T)
+        trace.tau.append(tau_i)
+        attempted = [b for b in range(B) if active[b]] if i >= warm_refs else []
+        if attempted:
+            backend.forecast(tt)                                   # forecasts for the active samples
+            fresh = model.verify_feature(i, tt)                    # the model computes the verify layer
+            e, acc = backend.verify_and_select(fresh, tt, [tau_i] * B, period)
+            for b in attempted:
+                errs[b] = e[b]
+                row[b] = ACCEPTED if acc[b] else REJECTED
+            active = backend.active_mask()
+        # everyone who did not get through speculatively takes the step in full and refreshes the tables
+        need_full = [0 if row[b] == ACCEPTED else 1 for b in range(B)]
+        if any(need_full):
+            feats = model.full(i, tt, need_full)
+            backend.reference_step(feats, tt, need_full)
+            active = backend.active_mask()
+        trace.steps.append(row)
+        trace.err.append(errs)
+    return trace
+
+
+class SpecaCacheBackend:
+    """The CUDA library as a scheduler backend. Device buffers are allocated once; one small
+    device-to-host copy of the decisions per speculative step is the only synchronisation."""
+
+    def __init__(self, cache, metric=None):
+        import torch
+        from . import binding as S
+        self.S, self.torch, self.cache = S, torch, cache
+        self.batch = cache.batch
+        dev = cache.device
+        self.metric = metric
+        self.outs = [torch.empty(cache.batch, n, d, dtype=torch.bfloat16 if cache.dtype == S.SPECA_BF16 else torch.float32,
+                                 device=dev) for n, d in cache.entries]
+        self.err = torch.zeros(self.batch, dtype=torch.float32, device=dev)
+        self.accept = torch.zeros(self.batch, dtype=torch.uint8, device=dev)
+        self.active = torch.zeros(self.batch, dtype=torch.uint8, device=dev)
+        self.spec = torch.zeros(self.batch, dtype=torch.int32, device=dev)
+        self.idx = torch.zeros(self.batch, dtype=torch.int32, device=dev)
+        self.n_active = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def reset_run(self):
+        self.cache.reset()
+        self.active.zero_()
+        self.spec.zero_()
+
+    def tau(self, tau0, beta, t, T):
+        return self.S.speca_tau(tau0, beta, t, T)
+
+    def forecast(self, t_target):
+        self.cache.forecast(t_target, self.outs, self.active)
+
+    def verify_and_select(self, fresh, t_target, tau, period):
+        self.accept.zero_()
+        self.cache.verify(fresh, t_target, tau, self.err, self.accept, self.active, metric=self.metric)
+        e = self.err.cpu().tolist()
+        acc = self.accept.cpu().tolist()
+        self.cache.select_adaptive(self.accept, period, 1, self.spec, self.active, self.idx, self.n_active)
+        return e, acc
+
+    def active_mask(self):
+        return self.active.cpu().tolist()
+
+    def reference_step(self, feats, t_ref, mask):
+        self.cache.update(feats, t_ref, mask)
+        self.cache.commit_step()
+        self.cache.activate(mask, self.spec, self.active)
