@@ -292,46 +292,69 @@ def time_metrics(h: Harness, reps: int = 20):
 
 
 def time_end_to_end(h: Harness, steps: int, warmup: int):
-    """Same step, but its inputs start in pinned host memory and its results end there."""
+    """Same step, but every step's inputs start in pinned host memory and its results end there.
+    The three legs of a step -- host-to-device copy of the features, the library calls, device-to-host
+    copy of forecasts and decisions -- run on three streams with two sets of device buffers, so the
+    copy-in of step k+1 and the copy-out of step k-1 overlap step k (PCIe is full duplex). Time is the
+    host's wall clock from the first enqueue to the moment every result is in host memory."""
     w, dev = h.w, h.device
     host_feats = [[f.cpu().pin_memory() for f in fs] for fs in h.feats]
     host_fresh = [f.cpu().pin_memory() for f in h.fresh]
     host_outs = [torch.empty(o.shape, dtype=o.dtype).pin_memory() for o in h.outs]
-    host_err = torch.empty(h.B, dtype=torch.float32).pin_memory()
-    host_acc = torch.empty(h.B, dtype=torch.uint8).pin_memory()
-    host_act = torch.empty(h.B, dtype=torch.uint8).pin_memory()
-    dev_feats = [torch.empty_like(f) for f in h.feats[0]]
-    dev_fresh = torch.empty_like(h.fresh[0])
+    host_small = [torch.empty(h.B * 6, dtype=torch.uint8).pin_memory() for _ in range(2)]
+    dev_feats = [[torch.empty_like(f) for f in h.feats[0]] for _ in range(2)]
+    dev_fresh = [torch.empty_like(h.fresh[0]) for _ in range(2)]
+    dev_outs = [h.outs, [torch.empty_like(o) for o in h.outs]]
+    dev_small = [torch.empty(h.B * 6, dtype=torch.uint8, device=dev) for _ in range(2)]
     h2d = sum(f.numel() * f.element_size() for f in host_feats[0]) + host_fresh[0].numel() * host_fresh[0].element_size()
     d2h = sum(o.numel() * o.element_size() for o in host_outs) + h.B * (4 + 1 + 1)
+    main = torch.cuda.current_stream(dev)
+    s_in, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    ev_in, ev_done, ev_out = {}, {}, {}
 
     def one(k):
-        for dst, src in zip(dev_feats, host_feats[k & 1]):
-            dst.copy_(src, non_blocking=True)
-        dev_fresh.copy_(host_fresh[k & 1], non_blocking=True)
-        h.step(feats=dev_feats, fresh=dev_fresh)
-        for dst, src in zip(host_outs, h.outs):
-            dst.copy_(src, non_blocking=True)
-        host_err.copy_(h.err, non_blocking=True)
-        host_acc.copy_(h.accept, non_blocking=True)
-        host_act.copy_(h.active, non_blocking=True)
+        p = k & 1
+        with torch.cuda.stream(s_in):
+            if k - 2 in ev_done:
+                s_in.wait_event(ev_done[k - 2])      # the step that last read this buffer set has run
+            for dst, src in zip(dev_feats[p], host_feats[p]):
+                dst.copy_(src, non_blocking=True)
+            dev_fresh[p].copy_(host_fresh[p], non_blocking=True)
+            ev_in[k] = torch.cuda.Event()
+            ev_in[k].record(s_in)
+        main.wait_event(ev_in[k])
+        if k - 2 in ev_out:
+            main.wait_event(ev_out[k - 2])           # the previous results in this output set are on the host
+        saved, h.outs = h.outs, dev_outs[p]
+        h.step(feats=dev_feats[p], fresh=dev_fresh[p])
+        h.outs = saved
+        dev_small[p][: 4 * h.B].copy_(h.err.view(torch.uint8))
+        dev_small[p][4 * h.B: 5 * h.B].copy_(h.accept)
+        dev_small[p][5 * h.B:].copy_(h.active)
+        ev_done[k] = torch.cuda.Event()
+        ev_done[k].record(main)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev_done[k])
+            for dst, src in zip(host_outs, dev_outs[p]):
+                dst.copy_(src, non_blocking=True)
+            host_small[p].copy_(dev_small[p], non_blocking=True)
+            ev_out[k] = torch.cuda.Event()
+            ev_out[k].record(s_out)
+        for old in (k - 3,):
+            ev_in.pop(old, None), ev_done.pop(old, None), ev_out.pop(old, None)
 
     for k in range(warmup):
         one(k)
     torch.cuda.synchronize(dev)
+    ev_in.clear(), ev_done.clear(), ev_out.clear()
     D.barrier()
-    t0 = torch.cuda.Event(enable_timing=True)
-    t1 = torch.cuda.Event(enable_timing=True)
     wall0 = time.perf_counter()
-    t0.record()
     for k in range(steps):
         one(k)
-    t1.record()
     torch.cuda.synchronize(dev)
     wall = (time.perf_counter() - wall0) * 1e3
     D.barrier()
-    ms = max(t0.elapsed_time(t1), wall)  # the host sees the results only after the sync
-    return ms / steps, h2d, d2h
+    return wall / steps, h2d, d2h
 
 
 def adaptive_sweep(device: str, peak: float, path: int, orders=(1, 2, 3), horizon: int = 6):
@@ -603,14 +626,15 @@ def main():
 
     e2e = None
     if not args.no_e2e:
-        e2e_steps = max(3, min(args.steps, 12))
+        e2e_steps = max(3, min(args.steps, 24))
         e2e_ms, h2d, d2h = time_end_to_end(h, e2e_steps, 3)
         e2e_ms = D.max_over_ranks(e2e_ms, device)
         ab = algorithmic_bytes(w, w.max_order)
         e2e = {"value": info.world * (ab["update"] + ab["forecast"] + ab["verify"]) / (e2e_ms * 1e-3) / 1e9,
                "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                "steps": e2e_steps,
-               "note": "features and verification feature copied from pinned host memory, forecasts and decisions copied back, every step"}
+               "note": "features and verification feature copied from pinned host memory, forecasts and decisions copied back, "
+                       "every step; copy-in, library calls and copy-out pipelined on three streams; host wall clock"}
     h.close()
     del h
     torch.cuda.empty_cache()
