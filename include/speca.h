@@ -237,6 +237,26 @@ speca_status_t speca_verify_metric(speca_cache_t* cache, int32_t metric, const v
                                    uint8_t* dev_accept, void* stream);
 
 /*
+ * Verification of a cache that holds only a token range of every entry (sequence-parallel layout:
+ * each GPU caches N_e / R tokens of every block output). Eq. 4 needs sums over the whole sample, so
+ * the step is split: every rank reduces its shard to the metric's running values, the ranks combine
+ * them (one all-reduce of 4*B doubles: sum, or max for SPECA_METRIC_LINF), every rank decides.
+ *
+ * speca_verify_partial: as speca_verify_metric, but instead of err / accept it writes
+ *   dev_sums   device, B x 4 doubles: sample b at [4b .. 4b+2] (unused slots 0), untouched for
+ *              inactive samples. L2: sum (p-f)^2, sum f^2. L1: sum |p-f|, sum |f|.
+ *              LINF: max |p-f|, max |f|. COSINE: sum p f, sum p^2, sum f^2.
+ * speca_verify_decide: e_b from combined values by the metric's formula (eps <= 0 selects 1e-8),
+ *   accept_b = (e_b <= tau_b); needs no handle. dev_active_mask NULL = all.
+ * With one rank, partial followed by decide gives exactly what speca_verify_metric gives.
+ * Errors: as speca_verify_metric; speca_verify_decide: INVALID_ARG, SHAPE (batch), ALIGNMENT, CUDA.
+ */
+speca_status_t speca_verify_partial(speca_cache_t* cache, int32_t metric, const void* fresh, const double* t_target,
+                                    const uint8_t* dev_active_mask, void* out_pred, double* dev_sums, void* stream);
+speca_status_t speca_verify_decide(int32_t metric, const double* dev_sums, int32_t batch, const float* tau, float eps,
+                                   const uint8_t* dev_active_mask, float* dev_err, uint8_t* dev_accept, void* stream);
+
+/*
  * Per-sample continuation of the speculative run (sequential validation of Section 3.4.2, the
  * forced activation period N of Appendix A, sample-adaptive allocation):
  *   for every active sample b: if accept_b then spec_count_b += 1

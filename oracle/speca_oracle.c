@@ -259,6 +259,46 @@ double oracle_cos_dist(int dtype, int64_t n, const void* pred, const void* fresh
     return 1.0 - dot / (sqrt(pp) * sqrt(ff) + eps);
 }
 
+/*
+ * The same metrics split in two stages, for a verification entry whose tokens are spread over
+ * several caches: the running values of one part (sums, or maxima for l-infinity), and the error
+ * from combined values. metric: 0 = l2 (Eq. 4), 1 = l1, 2 = l-infinity, 3 = cosine distance.
+ */
+void oracle_metric_sums(int metric, int dtype, int64_t n, const void* pred, const void* fresh, double* out3) {
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0;
+    int bad = 0;
+    for (int64_t j = 0; j < n; ++j) {
+        double p = load_elem(pred, dtype, j);
+        double f = load_elem(fresh, dtype, j);
+        if (metric == 0) {
+            a0 += (p - f) * (p - f);
+            a1 += f * f;
+        } else if (metric == 1) {
+            a0 += fabs(p - f);
+            a1 += fabs(f);
+        } else if (metric == 2) {
+            double d = fabs(p - f), a = fabs(f);
+            if (isnan(d) || isnan(a)) bad = 1;
+            if (d > a0) a0 = d;
+            if (a > a1) a1 = a;
+        } else {
+            a0 += p * f;
+            a1 += p * p;
+            a2 += f * f;
+        }
+    }
+    if (bad) a0 = a1 = NAN;
+    out3[0] = a0;
+    out3[1] = a1;
+    out3[2] = a2;
+}
+
+double oracle_metric_from_sums(int metric, const double* s, double eps) {
+    if (metric == 0) return sqrt(s[0]) / (sqrt(s[1]) + eps);
+    if (metric == 3) return 1.0 - s[0] / (sqrt(s[1]) * sqrt(s[2]) + eps);
+    return s[0] / (s[1] + eps);
+}
+
 /* Section 3.4.2: accepted iff e <= tau. A NaN error compares false and is rejected. */
 int oracle_accept(double err, double tau) { return err <= tau ? 1 : 0; }
 

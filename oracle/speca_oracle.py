@@ -58,6 +58,10 @@ def lib() -> ctypes.CDLL:
         for fn in (L.oracle_rel_l1, L.oracle_rel_linf, L.oracle_cos_dist):
             fn.argtypes = [i32, i64, vp, vp, dbl]
             fn.restype = dbl
+        L.oracle_metric_sums.argtypes = [i32, i32, i64, vp, vp, dp]
+        L.oracle_metric_sums.restype = None
+        L.oracle_metric_from_sums.argtypes = [i32, dp, dbl]
+        L.oracle_metric_from_sums.restype = dbl
         L.oracle_accept.argtypes = [dbl, dbl]
         L.oracle_accept.restype = i32
         L.oracle_tau.argtypes = [dbl, dbl, dbl, dbl]
@@ -125,6 +129,19 @@ def rel_err(metric: int, dtype, pred: np.ndarray, fresh: np.ndarray, eps: float 
     fn = {METRIC_L2: lib().oracle_rel_l2, METRIC_L1: lib().oracle_rel_l1, METRIC_LINF: lib().oracle_rel_linf,
           METRIC_COSINE: lib().oracle_cos_dist}[metric]
     return float(fn(dtype, pred.size, _ptr(pred), _ptr(fresh), float(eps)))
+
+
+def metric_sums(metric: int, dtype, pred: np.ndarray, fresh: np.ndarray):
+    """Running values of one part of a sample (sums; maxima for l-infinity): [a0, a1, a2]."""
+    assert pred.flags.c_contiguous and fresh.flags.c_contiguous and pred.size == fresh.size
+    out = (ctypes.c_double * 3)()
+    lib().oracle_metric_sums(metric, dtype, pred.size, _ptr(pred), _ptr(fresh), out)
+    return [out[0], out[1], out[2]]
+
+
+def metric_from_sums(metric: int, sums: Sequence[float], eps: float = EPS_PAPER) -> float:
+    buf = (ctypes.c_double * 3)(*[float(x) for x in sums])
+    return float(lib().oracle_metric_from_sums(metric, buf, float(eps)))
 
 
 def accept(err: float, tau: float) -> bool:

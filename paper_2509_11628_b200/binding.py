@@ -31,6 +31,7 @@ EXPORTS = [
     "speca_select_adaptive", "speca_activate", "speca_tau", "speca_cache_state", "speca_cache_plane",
     "speca_cache_launch_count", "speca_status_string", "speca_last_error", "speca_version",
     "speca_verify_pred_static", "speca_forecast_multi", "speca_verify_metric",
+    "speca_verify_partial", "speca_verify_decide",
 ]
 
 
@@ -78,6 +79,8 @@ def _lib() -> ctypes.CDLL:
     L.speca_forecast_multi.argtypes = [vp, i32, vp, vp, vp, vp]
     L.speca_verify.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.speca_verify_metric.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.speca_verify_partial.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
+    L.speca_verify_decide.argtypes = [i32, vp, i32, vp, ctypes.c_float, vp, vp, vp, vp]
     L.speca_select_adaptive.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, vp]
     L.speca_activate.argtypes = [vp, vp, vp, vp, vp]
     L.speca_verify_pred_static.argtypes = [vp, vp, ctypes.c_int64, i32, i32, vp, ctypes.c_float, vp, vp, vp, i32, vp]
@@ -219,6 +222,18 @@ def speca_verify_metric(cache, metric, fresh, t_target, tau, dev_active_mask, ou
     _check(_lib().speca_verify_metric(cache, int(metric), _dev_ptr(fresh), _doubles(t_target), _floats(tau),
                                       _dev_ptr(dev_active_mask), _dev_ptr(out_pred), _dev_ptr(dev_err),
                                       _dev_ptr(dev_accept), _stream_ptr(stream)), cache)
+
+
+def speca_verify_partial(cache, metric, fresh, t_target, dev_active_mask, out_pred, dev_sums, stream=None) -> None:
+    """``dev_sums``: CUDA float64 tensor [B, 4] that receives the metric's running values of this shard."""
+    _check(_lib().speca_verify_partial(cache, int(metric), _dev_ptr(fresh), _doubles(t_target), _dev_ptr(dev_active_mask),
+                                       _dev_ptr(out_pred), _dev_ptr(dev_sums), _stream_ptr(stream)), cache)
+
+
+def speca_verify_decide(metric, dev_sums, batch, tau, eps, dev_active_mask, dev_err, dev_accept, stream=None) -> None:
+    _check(_lib().speca_verify_decide(int(metric), _dev_ptr(dev_sums), int(batch), _floats(tau), float(eps),
+                                      _dev_ptr(dev_active_mask), _dev_ptr(dev_err), _dev_ptr(dev_accept),
+                                      _stream_ptr(stream)))
 
 
 def speca_select_adaptive(cache, dev_accept, k_max, group, dev_spec_count, dev_active_mask, dev_active_idx=None,

@@ -504,14 +504,18 @@ speca_status_t speca_verify(speca_cache_t* c, const void* fresh, const double* t
                                stream);
 }
 
-speca_status_t speca_verify_metric(speca_cache_t* c, int32_t metric, const void* fresh, const double* t_target,
-                                   const float* tau, const uint8_t* dev_active_mask, void* out_pred, float* dev_err,
-                                   uint8_t* dev_accept, void* stream) {
+// speca_verify_metric (dev_sums == nullptr) and speca_verify_partial (dev_sums given, no tau / err / accept).
+static speca_status_t verify_impl(speca_cache_t* c, int32_t metric, const void* fresh, const double* t_target,
+                                  const float* tau, const uint8_t* dev_active_mask, void* out_pred, float* dev_err,
+                                  uint8_t* dev_accept, double* dev_sums, void* stream) {
     if (c == nullptr) return SPECA_ERR_INVALID_ARG;
     if (metric < SPECA_METRIC_L2 || metric > SPECA_METRIC_COSINE)
         return fail(c, SPECA_ERR_INVALID_ARG, "verify: unknown metric %d", metric);
-    if (fresh == nullptr || t_target == nullptr || tau == nullptr || dev_err == nullptr || dev_accept == nullptr)
+    const bool partial = dev_sums != nullptr;
+    if (fresh == nullptr || t_target == nullptr || (!partial && (tau == nullptr || dev_err == nullptr || dev_accept == nullptr)))
         return fail(c, SPECA_ERR_INVALID_ARG, "verify: null argument");
+    if (reinterpret_cast<uintptr_t>(dev_sums) % sizeof(double) != 0)
+        return fail(c, SPECA_ERR_ALIGNMENT, "verify: dev_sums not aligned");
     if (c->pending) return fail(c, SPECA_ERR_STATE, "verify: a reference step is open (commit it first)");
     const size_t esz = elem_size(c);
     if (reinterpret_cast<uintptr_t>(fresh) % esz != 0 || reinterpret_cast<uintptr_t>(out_pred) % esz != 0)
@@ -524,13 +528,13 @@ speca_status_t speca_verify_metric(speca_cache_t* c, int32_t metric, const void*
     int v_max = 0;
     for (int b = 0; b < c->B; ++b) {
         if (!std::isfinite(t_target[b])) return fail(c, SPECA_ERR_INVALID_ARG, "verify: t_target[%d] not finite", b);
-        if (std::isnan(tau[b])) return fail(c, SPECA_ERR_INVALID_ARG, "verify: tau[%d] is NaN", b);
+        if (!partial && std::isnan(tau[b])) return fail(c, SPECA_ERR_INVALID_ARG, "verify: tau[%d] is NaN", b);
         int order;
         forecast_scalars(c, b, t_target[b], &order, p.coef[b]);
         if (order < 0 && dev_active_mask == nullptr)
             return fail(c, SPECA_ERR_STATE, "verify: sample %d has no committed reference", b);
         p.order[b] = static_cast<int8_t>(order);
-        p.tau[b] = tau[b];
+        p.tau[b] = partial ? 0.f : tau[b];
         any_sample |= order >= 0;
         v_max = order > v_max ? order : v_max;
     }
@@ -551,6 +555,7 @@ speca_status_t speca_verify_metric(speca_cache_t* c, int32_t metric, const void*
     p.accept = dev_accept;
     p.partials = reinterpret_cast<float*>(c->arena + L.partials_off);
     p.ticket = reinterpret_cast<uint32_t*>(c->arena + L.ticket_off);
+    p.raw_sums = dev_sums;
     p.n_elems = s0.n_elems;
     p.tiles_per_sample = (s0.n_elems + te - 1) / te;
     p.units_per_sample = (p.tiles_per_sample + c->cluster - 1) / c->cluster;
@@ -564,6 +569,38 @@ speca_status_t speca_verify_metric(speca_cache_t* c, int32_t metric, const void*
     if (ce != cudaSuccess) return cuda_fail(c, ce, "verify launch");
     c->launches += 1;
     return SPECA_OK;
+}
+
+speca_status_t speca_verify_metric(speca_cache_t* c, int32_t metric, const void* fresh, const double* t_target,
+                                   const float* tau, const uint8_t* dev_active_mask, void* out_pred, float* dev_err,
+                                   uint8_t* dev_accept, void* stream) {
+    return verify_impl(c, metric, fresh, t_target, tau, dev_active_mask, out_pred, dev_err, dev_accept, nullptr, stream);
+}
+
+speca_status_t speca_verify_partial(speca_cache_t* c, int32_t metric, const void* fresh, const double* t_target,
+                                    const uint8_t* dev_active_mask, void* out_pred, double* dev_sums, void* stream) {
+    if (c != nullptr && dev_sums == nullptr) return fail(c, SPECA_ERR_INVALID_ARG, "verify_partial: null dev_sums");
+    return verify_impl(c, metric, fresh, t_target, nullptr, dev_active_mask, out_pred, nullptr, nullptr, dev_sums, stream);
+}
+
+speca_status_t speca_verify_decide(int32_t metric, const double* dev_sums, int32_t batch, const float* tau, float eps,
+                                   const uint8_t* dev_active_mask, float* dev_err, uint8_t* dev_accept, void* stream) {
+    if (dev_sums == nullptr || tau == nullptr || dev_err == nullptr || dev_accept == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (metric < SPECA_METRIC_L2 || metric > SPECA_METRIC_COSINE) return SPECA_ERR_INVALID_ARG;
+    if (batch < 1 || batch > SPECA_MAX_BATCH) return SPECA_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(dev_sums) % sizeof(double) != 0 || reinterpret_cast<uintptr_t>(dev_err) % sizeof(float) != 0)
+        return SPECA_ERR_ALIGNMENT;
+    DecideParams q;
+    std::memset(&q, 0, sizeof q);
+    q.eps = eps > 0.f ? static_cast<double>(eps) : 1e-8;
+    for (int b = 0; b < batch; ++b) {
+        if (std::isnan(tau[b])) return SPECA_ERR_INVALID_ARG;
+        q.tau[b] = tau[b];
+    }
+    if (cudaPeekAtLastError() != cudaSuccess) return SPECA_ERR_CUDA;
+    cudaError_t ce = launch_decide(metric, dev_sums, batch, q, dev_active_mask, dev_err, dev_accept,
+                                   static_cast<cudaStream_t>(stream));
+    return ce == cudaSuccess ? SPECA_OK : SPECA_ERR_CUDA;
 }
 
 speca_status_t speca_select_adaptive(speca_cache_t* c, const uint8_t* dev_accept, int32_t k_max, int32_t group,

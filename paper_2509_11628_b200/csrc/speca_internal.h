@@ -77,6 +77,7 @@ struct VerifyParams {
     uint8_t* accept;
     float* partials;     // [n_clusters][B][values of the metric: 2, or 3 for cosine]
     uint32_t* ticket;    // arrival counter, zero between launches
+    double* raw_sums;    // [B][4] or null: write the combined running values instead of err / accept
     uint32_t n_elems;    // per sample
     uint32_t tiles_per_sample;
     uint32_t units_per_sample;  // ceil(tiles_per_sample / cluster size)
@@ -85,6 +86,11 @@ struct VerifyParams {
     double eps;
     int8_t order[SPECA_MAX_BATCH];
     float coef[SPECA_MAX_BATCH][SPECA_MAX_ORDER];
+    float tau[SPECA_MAX_BATCH];
+};
+
+struct DecideParams {
+    double eps;
     float tau[SPECA_MAX_BATCH];
 };
 
@@ -104,6 +110,8 @@ int stream_ctas_per_sm(int path, bool update, int dtype, int order);
 uint32_t multi_tile_bytes();
 int multi_ctas_per_sm();
 cudaError_t launch_forecast_multi(const MultiParams& p, int dtype, int batch, int grid, cudaStream_t stream);
+cudaError_t launch_decide(int metric, const double* sums, int batch, const DecideParams& q, const uint8_t* mask, float* err,
+                          uint8_t* accept, cudaStream_t stream);
 // Clusters of the verify kernel that fit on the current device at once.
 int max_resident_verify_clusters(int dtype, int order, int cluster);
 

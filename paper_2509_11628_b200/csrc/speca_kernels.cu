@@ -1041,13 +1041,51 @@ __global__ void __launch_bounds__(kThreads, 2) verify_kernel(const __grid_consta
             for (int off = 16; off > 0; off >>= 1) s[i] = Metric<M>::merge(s[i], __shfl_xor_sync(0xFFFFFFFFu, s[i], off));
         }
         if (lane == 0) {
-            const double e = Metric<M>::error(s, p.eps);
-            p.err[b] = static_cast<float>(e);
-            p.accept[b] = (e <= static_cast<double>(p.tau[b])) ? 1 : 0;  // NaN compares false: reject
+            if (p.raw_sums != nullptr) {
+                // token-sharded verification: hand out the running values; the caller combines the
+                // shards' values and calls the decision kernel
+#pragma unroll
+                for (int i = 0; i < 3; ++i) p.raw_sums[b * 4 + i] = i < NA ? s[i] : 0.0;
+            } else {
+                const double e = Metric<M>::error(s, p.eps);
+                p.err[b] = static_cast<float>(e);
+                p.accept[b] = (e <= static_cast<double>(p.tau[b])) ? 1 : 0;  // NaN compares false: reject
+            }
         }
     }
     __syncthreads();
     if (threadIdx.x == 0) *p.ticket = 0;  // ready for the next launch on this stream
+}
+
+// Decision from combined running values (token-sharded verification): sums[b][0..2] as the verify
+// kernel hands them out, added (l-infinity: maximised) over the shards by the caller.
+template <int M>
+__device__ __forceinline__ double error_from(const double* s, double eps) {
+    const double v[3] = {s[0], s[1], s[2]};
+    return Metric<M>::error(v, eps);
+}
+
+__global__ void __launch_bounds__(SPECA_MAX_BATCH) decide_kernel(int metric, const double* __restrict__ sums, int batch,
+                                                                  DecideParams q, const uint8_t* __restrict__ mask,
+                                                                  float* __restrict__ err, uint8_t* __restrict__ accept) {
+    const int b = threadIdx.x;
+    if (b >= batch || (mask != nullptr && mask[b] == 0)) return;
+    const double* s = sums + b * 4;
+    double e;
+    switch (metric) {
+        case SPECA_METRIC_L1: e = error_from<SPECA_METRIC_L1>(s, q.eps); break;
+        case SPECA_METRIC_LINF: e = error_from<SPECA_METRIC_LINF>(s, q.eps); break;
+        case SPECA_METRIC_COSINE: e = error_from<SPECA_METRIC_COSINE>(s, q.eps); break;
+        default: e = error_from<SPECA_METRIC_L2>(s, q.eps); break;
+    }
+    err[b] = static_cast<float>(e);
+    accept[b] = (e <= static_cast<double>(q.tau[b])) ? 1 : 0;
+}
+
+cudaError_t launch_decide(int metric, const double* sums, int batch, const DecideParams& q, const uint8_t* mask,
+                          float* err, uint8_t* accept, cudaStream_t stream) {
+    decide_kernel<<<1, SPECA_MAX_BATCH, 0, stream>>>(metric, sums, batch, q, mask, err, accept);
+    return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------------------------------------

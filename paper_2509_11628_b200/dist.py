@@ -67,6 +67,31 @@ def sum_over_ranks(value: float, device: str = "cpu") -> float:
     return float(t.item())
 
 
+def combine_verify_sums(sums: torch.Tensor, linf: bool = False) -> torch.Tensor:
+    """Token-sharded verification: combine every rank's per-sample running values ([B, 4] float64, as
+    speca_verify_partial writes them) in place -- a sum, or a maximum for the l-infinity metric. This
+    is the path's only exchange step in that layout: 32 bytes per sample per speculative step. A NaN
+    in any shard must survive the maximum, so NaNs are counted separately and put back."""
+    if not dist.is_initialized():
+        return sums
+    if linf:
+        nan = torch.isnan(sums).to(sums.dtype)
+        clean = torch.nan_to_num(sums, nan=0.0)
+        dist.all_reduce(clean, op=dist.ReduceOp.MAX)
+        dist.all_reduce(nan, op=dist.ReduceOp.MAX)
+        sums.copy_(torch.where(nan > 0, torch.full_like(clean, float("nan")), clean))
+    else:
+        dist.all_reduce(sums, op=dist.ReduceOp.SUM)
+    return sums
+
+
+def shard_tokens(n_tokens: int, world: int, rank: int):
+    """(first token, count) of this rank's contiguous token range; sizes differ by at most one."""
+    base, extra = divmod(n_tokens, world)
+    start = rank * base + min(rank, extra)
+    return start, base + (1 if rank < extra else 0)
+
+
 def shard_samples(n_samples: int, world: int, rank: int) -> List[int]:
     """Contiguous, balanced split of global sample indices over ranks (sizes differ by at most 1)."""
     base, extra = divmod(n_samples, world)

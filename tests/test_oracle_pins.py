@@ -537,6 +537,20 @@ def test_other_metrics_brute_force_in_rationals(dtype):
         assert O.rel_err(O.METRIC_COSINE, dtype, p, f) == pytest.approx(cs, abs=1e-13)
 
 
+@pytest.mark.parametrize("metric", [O.METRIC_L2] + OTHER_METRICS)
+def test_two_stage_metrics_agree_with_the_one_stage_ones_and_split_over_parts(metric):
+    g = torch.Generator().manual_seed(77 + metric)
+    f = torch.randn(3001, generator=g).numpy()
+    p = (f + 0.05 * torch.randn(3001, generator=g).numpy()).astype(np.float32)
+    whole = O.metric_sums(metric, O.F32, p, f)
+    assert O.metric_from_sums(metric, whole) == pytest.approx(O.rel_err(metric, O.F32, p, f), rel=1e-12, abs=1e-15)
+    cut = 1234
+    a = O.metric_sums(metric, O.F32, p[:cut].copy(), f[:cut].copy())
+    b = O.metric_sums(metric, O.F32, p[cut:].copy(), f[cut:].copy())
+    both = [max(x, y) for x, y in zip(a, b)] if metric == O.METRIC_LINF else [x + y for x, y in zip(a, b)]
+    assert O.metric_from_sums(metric, both) == pytest.approx(O.rel_err(metric, O.F32, p, f), rel=1e-12, abs=1e-15)
+
+
 def test_accept_rule():
     assert O.accept(0.5, 0.5)            # equality accepts
     assert O.accept(0.0, 0.0)
