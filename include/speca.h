@@ -325,6 +325,18 @@ double speca_tau(double tau0, double beta, double t, double T);
  * Either output may be NULL. */
 speca_status_t speca_cache_state(const speca_cache_t* cache, int32_t* host_n_refs, double* host_t_last);
 
+/*
+ * Checkpoint / resume. The tables live in the caller's arena; the only other state of a cache is
+ * the reference history of each sample. speca_cache_get_history copies it out (host_n_refs: B
+ * int32; host_t_hist: B x (SPECA_MAX_ORDER + 1) doubles, most recent first, NaN where undefined);
+ * speca_cache_set_history installs it in a cache of the same configuration -- built over a copy of
+ * the saved arena bytes, it continues exactly where the saved one stopped. Host only.
+ * Errors: INVALID_ARG (null, negative count, a defined time that is not finite), STATE (set while a
+ * reference step is open).
+ */
+speca_status_t speca_cache_get_history(const speca_cache_t* cache, int32_t* host_n_refs, double* host_t_hist);
+speca_status_t speca_cache_set_history(speca_cache_t* cache, const int32_t* host_n_refs, const double* host_t_hist);
+
 /* Device address and byte stride of the table of (entry, sample): plane i starts at
  * *plane0 + i * *plane_stride_bytes. For checkpointing and tests. */
 speca_status_t speca_cache_plane(const speca_cache_t* cache, int32_t entry, int32_t sample, void** plane0,

@@ -31,7 +31,7 @@ EXPORTS = [
     "speca_select_adaptive", "speca_activate", "speca_tau", "speca_cache_state", "speca_cache_plane",
     "speca_cache_launch_count", "speca_status_string", "speca_last_error", "speca_version",
     "speca_verify_pred_static", "speca_forecast_multi", "speca_verify_metric",
-    "speca_verify_partial", "speca_verify_decide",
+    "speca_verify_partial", "speca_verify_decide", "speca_cache_get_history", "speca_cache_set_history",
 ]
 
 
@@ -87,6 +87,8 @@ def _lib() -> ctypes.CDLL:
     L.speca_tau.argtypes = [dbl, dbl, dbl, dbl]
     L.speca_tau.restype = dbl
     L.speca_cache_state.argtypes = [vp, vp, vp]
+    L.speca_cache_get_history.argtypes = [vp, vp, vp]
+    L.speca_cache_set_history.argtypes = [vp, vp, vp]
     L.speca_cache_plane.argtypes = [vp, i32, i32, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_size_t)]
     L.speca_cache_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64)]
     L.speca_status_string.argtypes = [i32]
@@ -267,6 +269,22 @@ def speca_cache_state(cache, batch: int):
     t = (ctypes.c_double * batch)()
     _check(_lib().speca_cache_state(cache, n, t), cache)
     return list(n), list(t)
+
+
+def speca_cache_get_history(cache, batch: int):
+    """(n_refs[B], t_hist[B][SPECA_MAX_ORDER + 1]) -- with the arena bytes, everything a checkpoint needs."""
+    n = (ctypes.c_int32 * batch)()
+    t = (ctypes.c_double * (batch * (SPECA_MAX_ORDER + 1)))()
+    _check(_lib().speca_cache_get_history(cache, n, t), cache)
+    w = SPECA_MAX_ORDER + 1
+    return list(n), [list(t[b * w:(b + 1) * w]) for b in range(batch)]
+
+
+def speca_cache_set_history(cache, n_refs, t_hist) -> None:
+    n = (ctypes.c_int32 * len(n_refs))(*[int(x) for x in n_refs])
+    flat = [float(x) for row in t_hist for x in row]
+    t = (ctypes.c_double * len(flat))(*flat)
+    _check(_lib().speca_cache_set_history(cache, n, t), cache)
 
 
 def speca_cache_plane(cache, entry: int, sample: int):

@@ -659,6 +659,33 @@ speca_status_t speca_cache_state(const speca_cache_t* c, int32_t* host_n_refs, d
     return SPECA_OK;
 }
 
+speca_status_t speca_cache_get_history(const speca_cache_t* c, int32_t* host_n_refs, double* host_t_hist) {
+    if (c == nullptr || host_n_refs == nullptr || host_t_hist == nullptr) return SPECA_ERR_INVALID_ARG;
+    for (int b = 0; b < c->B; ++b) {
+        host_n_refs[b] = c->n_refs[b];
+        for (int i = 0; i <= SPECA_MAX_ORDER; ++i) host_t_hist[b * (SPECA_MAX_ORDER + 1) + i] = c->t_hist[b][i];
+    }
+    return SPECA_OK;
+}
+
+speca_status_t speca_cache_set_history(speca_cache_t* c, const int32_t* host_n_refs, const double* host_t_hist) {
+    if (c == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (host_n_refs == nullptr || host_t_hist == nullptr) return fail(c, SPECA_ERR_INVALID_ARG, "set_history: null argument");
+    if (c->pending) return fail(c, SPECA_ERR_STATE, "set_history while a reference step is open");
+    for (int b = 0; b < c->B; ++b) {
+        if (host_n_refs[b] < 0) return fail(c, SPECA_ERR_INVALID_ARG, "set_history: n_refs[%d] negative", b);
+        const int defined = host_n_refs[b] < SPECA_MAX_ORDER + 1 ? host_n_refs[b] : SPECA_MAX_ORDER + 1;
+        for (int i = 0; i < defined; ++i)
+            if (!std::isfinite(host_t_hist[b * (SPECA_MAX_ORDER + 1) + i]))
+                return fail(c, SPECA_ERR_INVALID_ARG, "set_history: time %d of sample %d not finite", i, b);
+    }
+    for (int b = 0; b < c->B; ++b) {
+        c->n_refs[b] = host_n_refs[b];
+        for (int i = 0; i <= SPECA_MAX_ORDER; ++i) c->t_hist[b][i] = host_t_hist[b * (SPECA_MAX_ORDER + 1) + i];
+    }
+    return SPECA_OK;
+}
+
 speca_status_t speca_cache_plane(const speca_cache_t* c, int32_t entry, int32_t sample, void** plane0,
                                  size_t* plane_stride_bytes) {
     if (c == nullptr || plane0 == nullptr || plane_stride_bytes == nullptr) return SPECA_ERR_INVALID_ARG;

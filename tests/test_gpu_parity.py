@@ -341,3 +341,43 @@ def test_adaptive_batch_rejected_samples_stop_forecasting(S, U):
                 break
         assert seen_reject
         pair.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# checkpoint / resume: arena bytes + reference history are the whole state
+# ---------------------------------------------------------------------------------------------
+
+def test_checkpoint_and_resume_continue_bit_for_bit(S, U):
+    entries = [(16, 520), (33, 1031)]
+    B, m = 3, 2
+    gen = torch.Generator(device=DEV).manual_seed(12)
+    a = S.SpecaCache(entries, B, m, 1, DEV)
+    feats = [rand_feats(entries, B, torch.bfloat16, gen) for _ in range(4)]
+    a.update(feats[0], [1.0, 1.0, 1.0]); a.commit_step()
+    a.update(feats[1], [0.9, 0.91, 0.9], [1, 1, 0]); a.commit_step()
+    torch.cuda.synchronize()
+    saved_arena = a.arena.clone()
+    n_refs, t_hist = S.speca_cache_get_history(a.handle, B)
+    assert n_refs == [2, 2, 1] and t_hist[1][:2] == [0.91, 1.0] and np.isnan(t_hist[2][1])
+    # a second cache over a copy of the bytes, history installed
+    b = S.SpecaCache(entries, B, m, 1, DEV)
+    b.arena.copy_(saved_arena)
+    S.speca_cache_set_history(b.handle, n_refs, t_hist)
+    assert b.state() == a.state()
+    for c in (a, b):
+        c.update(feats[2], [0.8, 0.8, 0.8]); c.commit_step()
+    outs_a = [torch.zeros(B, n, d, dtype=torch.bfloat16, device=DEV) for n, d in entries]
+    outs_b = [torch.zeros(B, n, d, dtype=torch.bfloat16, device=DEV) for n, d in entries]
+    a.forecast([0.77] * B, outs_a)
+    b.forecast([0.77] * B, outs_b)
+    torch.cuda.synchronize()
+    for x, y in zip(outs_a, outs_b):
+        assert torch.equal(x.view(torch.int16), y.view(torch.int16))
+    with pytest.raises(S.SpecaError) as ei:
+        S.speca_cache_set_history(b.handle, [1, -1, 0], t_hist)
+    assert ei.value.status == S.SPECA_ERR_INVALID_ARG
+    b.update(feats[3], [0.7] * B)
+    with pytest.raises(S.SpecaError) as ei:
+        S.speca_cache_set_history(b.handle, n_refs, t_hist)
+    assert ei.value.status == S.SPECA_ERR_STATE
+    a.close(); b.close()
