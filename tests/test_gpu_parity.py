@@ -381,3 +381,35 @@ def test_checkpoint_and_resume_continue_bit_for_bit(S, U):
         S.speca_cache_set_history(b.handle, n_refs, t_hist)
     assert ei.value.status == S.SPECA_ERR_STATE
     a.close(); b.close()
+
+
+def test_arena_that_is_only_256_byte_aligned(S, U):
+    """4 KB alignment of the arena is a speed matter only: at base + 256 the planes start 256 bytes
+    off their 4 KB boundaries and every result must be the same."""
+    entries = [(37, 129), (64, 384), (3, 8192)]
+    B, m = 2, 2
+    gen = torch.Generator(device=DEV).manual_seed(31)
+    nbytes = S.speca_cache_arena_bytes(entries, B, m, 1)
+    raw = torch.empty(nbytes + 4096, dtype=torch.uint8, device=DEV)
+    aligned = S.SpecaCache(entries, B, m, 1, DEV)
+    handle = S.speca_cache_create(entries, B, m, 1, raw.data_ptr() + 256, arena_bytes=nbytes, device=0)
+    feats = [rand_feats(entries, B, torch.bfloat16, gen) for _ in range(3)]
+    for k, f in enumerate(feats):
+        t = [1.0 - 0.1 * k] * B
+        aligned.update(f, t); aligned.commit_step()
+        S.speca_cache_update(handle, f, t); S.speca_cache_commit_step(handle)
+    oa = [torch.zeros(B, n, d, dtype=torch.bfloat16, device=DEV) for n, d in entries]
+    ob = [torch.zeros(B, n, d, dtype=torch.bfloat16, device=DEV) for n, d in entries]
+    aligned.forecast([0.72] * B, oa)
+    S.speca_forecast(handle, [0.72] * B, None, ob)
+    ea, eb = torch.zeros(B, device=DEV), torch.zeros(B, device=DEV)
+    aa, ab = torch.zeros(B, dtype=torch.uint8, device=DEV), torch.zeros(B, dtype=torch.uint8, device=DEV)
+    fresh = rand_feats([entries[-1]], B, torch.bfloat16, gen)[0]
+    aligned.verify(fresh, [0.72] * B, [1.5] * B, ea, aa)
+    S.speca_verify(handle, fresh, [0.72] * B, [1.5] * B, None, None, eb, ab)
+    torch.cuda.synchronize()
+    for x, y in zip(oa, ob):
+        assert torch.equal(x.view(torch.int16), y.view(torch.int16))
+    assert torch.equal(ea, eb) and torch.equal(aa, ab)
+    S.speca_cache_destroy(handle)
+    aligned.close()
