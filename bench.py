@@ -267,6 +267,31 @@ def time_multi_horizon(h: Harness, peak: float, forecast_ms: float, K: int = 4, 
             "speedup_vs_single_forecasts": K * forecast_ms / ms}
 
 
+def time_update_per_entry(h: Harness, reps: int = 5):
+    """A model hands over one block output at a time: the same reference step as one launch per entry."""
+    w, dev = h.w, h.device
+    ne = len(w.entries)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    total = 0.0
+    for r in range(reps + 1):
+        j = h.j
+        h.j += 1
+        t_ref, _ = h.times_for(j)
+        e0.record()
+        for e in range(ne):
+            one = [None] * ne
+            one[e] = h.feats[j & 1][e]
+            h.cache.update(one, t_ref)
+        h.cache.commit_step()
+        e1.record()
+        torch.cuda.synchronize(dev)
+        if r > 0:
+            total += e0.elapsed_time(e1)
+    ms = total / reps
+    nbytes = algorithmic_bytes(w, w.max_order)["update"]
+    return {"launches": ne, "ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9}
+
+
 def time_metrics(h: Harness, reps: int = 20):
     """Device time of the fused verification with each error metric (same traffic: order + 2 words per
     element of the verification entry)."""
@@ -623,6 +648,7 @@ def main():
 
     multi = time_multi_horizon(h, peak, per_ms["forecast"]) if info.world == 1 else None
     metrics = time_metrics(h) if info.world == 1 else None
+    per_entry = time_update_per_entry(h) if info.world == 1 else None
 
     e2e = None
     if not args.no_e2e:
@@ -650,7 +676,8 @@ def main():
                 v2, ms2, kern2, ex2 = summarize(w2, p2, t2, k2, 1, peak)
                 per_config[name] = {"value": v2, "unit": "GB/s", "ms_per_step": ms2, "steps": k2,
                                     "config": workload_config(w2), "kernels": kern2, **ex2,
-                                    "multi_horizon": time_multi_horizon(h2, peak, p2["forecast"])}
+                                    "multi_horizon": time_multi_horizon(h2, peak, p2["forecast"]),
+                                    "update_one_launch_per_entry": time_update_per_entry(h2)}
                 h2.close()
                 del h2
                 torch.cuda.empty_cache()
@@ -705,7 +732,7 @@ def main():
         "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches,
         "clocks": clocks, "kernels": kernels, **extra,
         "frac_of_measured_peak": value / info.world / peak, "frac_of_nominal_8TBs": value / info.world / NOMINAL_HBM_GBS,
-        "multi_horizon": multi, "verify_metrics": metrics, "per_config": per_config, "adaptive": adaptive, "sampler": sampler,
+        "multi_horizon": multi, "verify_metrics": metrics, "update_one_launch_per_entry": per_entry, "per_config": per_config, "adaptive": adaptive, "sampler": sampler,
         "paper_context": {"end_to_end_speedups": {"flux_h800": 6.34, "dit_xl2_a800": 7.3, "hunyuan_video_h800": 6.1},
                           "verification_overhead": "1.67%-3.5% of a full forward pass",
                           "note": "other hardware, whole-model numbers; context only"},
