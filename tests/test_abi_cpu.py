@@ -92,3 +92,16 @@ def test_product_package_does_not_touch_the_oracle():
                 assert "oracle" not in text.lower() or fn == "workloads.py", fn
     text = open(os.path.join(pkg, "workloads.py")).read()
     assert "import oracle" not in text and "from oracle" not in text
+
+
+def test_header_is_valid_c99_and_usable_from_a_c_program(S, tmp_path):
+    """gcc -std=c99 -pedantic -Werror on a C program that includes only speca.h, linked against the
+    library and run on the host (it touches host-only entry points)."""
+    import subprocess
+    src = os.path.join(ROOT, "tests", "c_abi", "abi_check.c")
+    exe = os.path.join(str(tmp_path), "abi_check")
+    libdir = os.path.dirname(S.LIB_PATH)
+    subprocess.check_call(["gcc", "-std=c99", "-pedantic", "-Wall", "-Wextra", "-Werror", "-I", os.path.join(ROOT, "include"),
+                           src, "-o", exe, "-L", libdir, "-l:libspeca.so", "-Wl,-rpath," + libdir, "-lm"])
+    out = subprocess.run([exe], stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
+    assert out.returncode == 0 and "abi ok" in out.stdout, out.stdout

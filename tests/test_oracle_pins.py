@@ -316,6 +316,39 @@ def test_bf16_tables_round_once_per_stored_plane():
 
 
 # ---------------------------------------------------------------------------------------------
+# the appendix's prediction-error bound, as a soft check (it equates differences with derivatives)
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("m", [1, 2, 3])
+def test_error_follows_the_taylor_remainder_and_the_appendix_bound(m):
+    """Features c * exp(lambda * t): every derivative is lambda^i F, so the theorem's constant L is
+    lambda. The forecast error must (i) stay below the theorem's leading term times (1 + L|x|) plus
+    the O(h) finite-difference bias, (ii) approach the exact Taylor remainder
+    |exp(lx) - sum (lx)^i / i!| linearly as the reference spacing h shrinks."""
+    lam, x = 0.8, -0.5
+    g = torch.Generator().manual_seed(3)
+    c = (torch.rand(4000, generator=g) + 0.5).numpy().astype(np.float64)
+    remainder = abs(math.exp(lam * x) - sum((lam * x) ** i / math.factorial(i) for i in range(m + 1)))
+    gaps = []
+    for h in (0.08, 0.04, 0.02):
+        times = [1.0 - h * k for k in range(m + 1)]                     # oldest first, decreasing t
+        feats = [(c * math.exp(lam * t)).astype(np.float32) for t in times]
+        planes, hist = run_history(O.F32, m, O.TAYLOR, times, feats)
+        out = np.zeros(c.size, np.float32)
+        t0 = times[-1]
+        O.forecast_segment(O.F32, m, O.TAYLOR, m + 1, hist, t0 + x, planes, out)
+        truth = (c * math.exp(lam * (t0 + x))).astype(np.float32)
+        now = (c * math.exp(lam * t0)).astype(np.float32)
+        e_rel_to_now = float(np.linalg.norm(out.astype(np.float64) - truth) / np.linalg.norm(now))
+        bound = (lam * abs(x)) ** (m + 1) / math.factorial(m + 1) * (1 + lam * abs(x)) + m * lam ** 2 * h * abs(x)
+        assert e_rel_to_now <= bound, (m, h, e_rel_to_now, bound)
+        gaps.append(abs(e_rel_to_now - remainder))
+    # the distance to the exact Taylor remainder is the O(h) difference-quotient bias: it halves with h
+    assert 1.5 < gaps[0] / gaps[1] < 2.6 and 1.5 < gaps[1] / gaps[2] < 2.6, gaps
+    assert gaps[2] < 0.6 * m * lam ** 2 * 0.02 * abs(x) * 2
+
+
+# ---------------------------------------------------------------------------------------------
 # Adams-Bashforth draft model (appendix: named without a formula; pinned by the textbook method)
 # ---------------------------------------------------------------------------------------------
 
