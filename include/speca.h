@@ -23,8 +23,8 @@
  *     error has enqueued nothing and has not changed the cache's state.
  *   - Tensors are dense, row-major [B, N_e, D] in the cache's storage dtype; sample b of an entry
  *     starts at element b*N_e*D. Device tensor pointers must be aligned to the element size;
- *     16-byte aligned pointers (with N_e*D*sizeof(element) a multiple of 16) take the fast
- *     vectorised / bulk-copy path, anything else a slower element-wise path with equal results.
+ *     32-byte aligned rows (pointer and N_e*D*sizeof(element) multiples of 32) take the fast
+ *     vector path, anything else a slower 16-byte or element-wise path with equal results.
  *   - A handle is not thread safe: use one handle from one host thread at a time.
  *   - There is no CPU fallback: without a usable CUDA device speca_cache_create fails.
  */

@@ -80,7 +80,7 @@ struct VerifyParams {
     double* raw_sums;    // [B][4] or null: write the combined running values instead of err / accept
     uint32_t n_elems;    // per sample
     uint32_t tiles_per_sample;
-    uint32_t units_per_sample;  // ceil(tiles_per_sample / cluster size)
+    uint32_t units_per_sample;  // ceil(tiles_per_sample / cluster size): host-side grid sizing only
     int32_t batch;
     int32_t metric;  // speca_metric_t
     double eps;

@@ -1,15 +1,17 @@
 // CUDA kernels of the SpeCa feature-cache hot path for sm_100a (B200).
 //
-//   update   : Eq. 3 -- fold a freshly computed feature into the derivative table, in place
-//   forecast : Eq. 2 -- Horner evaluation of the table at a speculative time
-//   verify   : Eq. 4 -- forecast of the verification entry fused with ||p - f||, ||f|| and the
-//              accept rule of Section 3.4.2
-//   select   : per-sample continuation of the speculative run (Section 3.4.2, Appendix A)
+//   update         : Eq. 3 -- fold a freshly computed feature into the derivative table, in place
+//   forecast       : Eq. 2 -- Horner evaluation of the table at a speculative time
+//   forecast_multi : Eq. 2 for several speculative times from one read of the table (Fig. 1)
+//   verify         : Eq. 4 -- forecast of the verification entry fused with the error reduction and
+//                    the accept rule of Section 3.4.2 (l2, or the appendix's other metrics)
+//   select         : per-sample continuation of the speculative run (Section 3.4.2, Appendix A)
 //
-// Every kernel is a pure HBM stream (about half a flop per byte), so the design goal is bytes in
-// flight, coalescing and no re-reads: 16-byte vectors, several independent loads per thread before
-// the first use, persistent grids sized from the SM count, streaming cache hints (nothing is
-// reused before it leaves L2). No tensor cores are involved.
+// Every kernel is a pure HBM stream (about half a flop per byte, no reuse), so the design is about
+// how the DRAM sees it: 32-byte vector loads and stores (sm_100), all of a chunk's loads issued
+// before the first use, persistent grids of a few CTAs per SM whose bytes in flight are matched to
+// the read / write mix, planes on 4 KB boundaries, no re-reads. No tensor cores are involved. The
+// TMA-staged variant (cp.async.bulk + mbarrier) is kept for comparison.
 #include <cooperative_groups.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
