@@ -30,7 +30,7 @@ struct Layout {
 };
 
 // Shape checks and arena layout shared by speca_cache_arena_bytes and speca_cache_create.
-speca_status_t make_layout(const speca_cache_config_t* cfg, Layout* L) {
+speca_status_t make_layout_impl(const speca_cache_config_t* cfg, Layout* L) {
     if (cfg == nullptr || cfg->entries == nullptr) return SPECA_ERR_INVALID_ARG;
     if (cfg->n_entries < 1 || cfg->n_entries > SPECA_MAX_ENTRIES) return SPECA_ERR_SHAPE;
     if (cfg->batch < 1 || cfg->batch > SPECA_MAX_BATCH) return SPECA_ERR_SHAPE;
@@ -93,6 +93,17 @@ speca_status_t make_layout(const speca_cache_config_t* cfg, Layout* L) {
     for (int k = 0; k < kNumTileSizes; ++k) L->tiles[k][n_segs] = static_cast<uint32_t>(n_tiles[k]);
     L->total = off;
     return SPECA_OK;
+}
+
+// The C ABI never lets an exception out: a failed host allocation becomes SPECA_ERR_NOMEM.
+speca_status_t make_layout(const speca_cache_config_t* cfg, Layout* L) noexcept {
+    try {
+        return make_layout_impl(cfg, L);
+    } catch (const std::bad_alloc&) {
+        return SPECA_ERR_NOMEM;
+    } catch (...) {
+        return SPECA_ERR_INVALID_ARG;
+    }
 }
 
 struct DeviceGuard {
@@ -234,7 +245,12 @@ speca_status_t speca_cache_create(const speca_cache_config_t* cfg, speca_cache_t
     c->pending = false;
     c->launches = 0;
     c->last_error[0] = 0;
-    c->entry_updated.assign(c->n_entries, 0);
+    try {
+        c->entry_updated.assign(c->n_entries, 0);
+    } catch (const std::bad_alloc&) {
+        delete c;
+        return SPECA_ERR_NOMEM;
+    }
     for (int b = 0; b < SPECA_MAX_BATCH; ++b) {
         c->n_refs[b] = 0;
         for (int i = 0; i <= SPECA_MAX_ORDER; ++i) c->t_hist[b][i] = std::numeric_limits<double>::quiet_NaN();
