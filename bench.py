@@ -292,6 +292,43 @@ def time_update_per_entry(h: Harness, reps: int = 5):
     return {"launches": ne, "ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9}
 
 
+def time_forecast_sum(h: Harness, peak: float, reps: int = 20):
+    """base + sum of the forecasts of the largest group of equally shaped entries (all 56 block outputs
+    of the DiT shape, the 38 single blocks of the FLUX shape, ...) in one pass, in place on a residual
+    buffer: E (order + 1) + 2 words per element."""
+    w, dev = h.w, h.device
+    groups = {}
+    for e, shape in enumerate(w.entries):
+        groups.setdefault(shape, []).append(e)
+    shape, ids = max(groups.items(), key=lambda kv: len(kv[1]) * kv[0][0] * kv[0][1])
+    resid = torch.zeros(h.B, shape[0], shape[1], dtype=w.torch_dtype, device=dev)
+    t = [h.t_base - 0.02 * (h.j + 1) - 0.01] * h.B
+    for _ in range(3):
+        h.cache.forecast_sum(ids, t, resid, resid, h.active)
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        resid.zero_()
+        h.cache.forecast_sum(ids, t, resid, resid, h.active)
+    e1.record()
+    torch.cuda.synchronize(dev)
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record()
+    for _ in range(reps):
+        resid.zero_()
+    e3.record()
+    torch.cuda.synchronize(dev)
+    ms = (e0.elapsed_time(e1) - e2.elapsed_time(e3)) / reps
+    n = h.B * shape[0] * shape[1]
+    nbytes = (len(ids) * (w.max_order + 1) + 2) * w.elem_bytes * n
+    separate = len(ids) * (w.max_order + 2) * w.elem_bytes * n
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"entries": len(ids), "shape": list(shape), "ms": ms, "algorithmic_bytes": nbytes, "gbs": gbs,
+            "frac_of_measured_peak": gbs / peak, "bytes_of_separate_forecasts": separate,
+            "traffic_saved_vs_separate": 1.0 - nbytes / separate}
+
+
 def time_metrics(h: Harness, reps: int = 20):
     """Device time of the fused verification with each error metric (same traffic: order + 2 words per
     element of the verification entry)."""
@@ -649,6 +686,7 @@ def main():
     multi = time_multi_horizon(h, peak, per_ms["forecast"]) if info.world == 1 else None
     metrics = time_metrics(h) if info.world == 1 else None
     per_entry = time_update_per_entry(h) if info.world == 1 else None
+    fsum = time_forecast_sum(h, peak) if info.world == 1 else None
 
     e2e = None
     if not args.no_e2e:
@@ -677,7 +715,8 @@ def main():
                 per_config[name] = {"value": v2, "unit": "GB/s", "ms_per_step": ms2, "steps": k2,
                                     "config": workload_config(w2), "kernels": kern2, **ex2,
                                     "multi_horizon": time_multi_horizon(h2, peak, p2["forecast"]),
-                                    "update_one_launch_per_entry": time_update_per_entry(h2)}
+                                    "update_one_launch_per_entry": time_update_per_entry(h2),
+                                    "forecast_sum": time_forecast_sum(h2, peak)}
                 h2.close()
                 del h2
                 torch.cuda.empty_cache()
@@ -732,7 +771,7 @@ def main():
         "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches,
         "clocks": clocks, "kernels": kernels, **extra,
         "frac_of_measured_peak": value / info.world / peak, "frac_of_nominal_8TBs": value / info.world / NOMINAL_HBM_GBS,
-        "multi_horizon": multi, "verify_metrics": metrics, "update_one_launch_per_entry": per_entry, "per_config": per_config, "adaptive": adaptive, "sampler": sampler,
+        "multi_horizon": multi, "verify_metrics": metrics, "update_one_launch_per_entry": per_entry, "forecast_sum": fsum, "per_config": per_config, "adaptive": adaptive, "sampler": sampler,
         "paper_context": {"end_to_end_speedups": {"flux_h800": 6.34, "dit_xl2_a800": 7.3, "hunyuan_video_h800": 6.1},
                           "verification_overhead": "1.67%-3.5% of a full forward pass",
                           "note": "other hardware, whole-model numbers; context only"},

@@ -210,6 +210,25 @@ speca_status_t speca_forecast_multi(speca_cache_t* cache, int32_t n_targets, con
                                     const uint8_t* dev_active_mask, void* const* outs, void* stream);
 
 /*
+ * Forecasts consumed as a sum. A transformer adds its block outputs to a residual stream, so on a
+ * speculative step the forecasts (Eq. 2) of equally shaped blocks are only needed as
+ *     out = base + sum over the listed entries of forecast_e(t_target),
+ * which this call computes without writing the individual forecasts: each entry's Horner result
+ * stays in fp32, is added unrounded in list order, and the total is rounded once to the storage
+ * dtype. (An extension of workflow step 2 that assumes the model's residual structure; the paper
+ * itself only forecasts per block.)
+ *   entry_ids       host, n_ids entry indices (1..SPECA_MAX_ENTRIES of them), all with the same
+ *                   tokens * dim; an entry may be listed more than once.
+ *   t_target        host, B doubles.  dev_active_mask: device, B bytes, NULL = all (inactive samples'
+ *                   rows of out are not written).
+ *   base            device [B, N, D] or NULL (= 0).  out: device [B, N, D]; may alias base.
+ * Errors: INVALID_ARG (null, empty list, index out of range, non-finite time), SHAPE (entries of
+ * different sizes), ALIGNMENT, STATE, CUDA.
+ */
+speca_status_t speca_forecast_sum(speca_cache_t* cache, const int32_t* entry_ids, int32_t n_ids, const double* t_target,
+                                  const uint8_t* dev_active_mask, const void* base, void* out, void* stream);
+
+/*
  * Verification, Eq. 4 and the accept rule of Section 3.4.2, fused with the forecast of the
  * verification entry:  e_b = ||p_b - f_b||_2 / (||f_b||_2 + eps),  accept_b = (e_b <= tau_b),
  * with p the forecast rounded to the storage dtype and the norms taken over all N_v*D elements

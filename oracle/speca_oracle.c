@@ -193,6 +193,60 @@ int oracle_forecast_segment(int dtype, int64_t n, int m, int basis, int n_refs, 
     return 0;
 }
 
+/* ---- Eq. 2 summed over several entries ---------------------------------------------------------- */
+/*
+ * A transformer adds its block outputs to a residual stream, so on a speculative step the forecasts
+ * of blocks with equal shapes are only ever consumed as a sum: out = base + sum_e forecast_e. The two
+ * functions below state that in the plainest form: each entry's forecast (Eq. 2, any basis) is added
+ * UNROUNDED, in double, to an accumulator; the total is rounded once (double -> binary32 -> storage).
+ * oracle_forecast_accumulate_segment returns 0, or 1 if the table is empty / the basis unknown.
+ */
+int oracle_forecast_accumulate_segment(int dtype, int64_t n, int m, int basis, int n_refs, const double* t_hist,
+                                       double t_target, const void* planes, int64_t plane_stride, double* acc) {
+    if (n_refs < 1) return 1;
+    int v = n_refs - 1 < m ? n_refs - 1 : m;
+    size_t esz = dtype == ORACLE_F32 ? 4 : 2;
+    double w[ORACLE_MAX_ORDER + 1];
+    w[0] = 1.0;
+    if (basis == ORACLE_NEWTON) {
+        for (int i = 1; i <= v; ++i) w[i] = w[i - 1] * (t_target - t_hist[i - 1]);
+    } else if (basis == ORACLE_TAYLOR) {
+        double x = t_target - t_hist[0], fact = 1.0;
+        for (int i = 1; i <= v; ++i) {
+            fact *= (double)i;
+            w[i] = pow(x, (double)i) / fact;
+        }
+    } else if (basis == ORACLE_ADAMS_BASHFORTH) {
+        /* collected by plane: F + x (D1 + h/2 D2 + 5h^2/12 D3 + 3h^3/8 D4) -- the same polynomial the
+         * slope form in oracle_forecast_segment evaluates (tests check the two against each other) */
+        static const double gam[4] = {1.0, 1.0 / 2, 5.0 / 12, 3.0 / 8};
+        double x = t_target - t_hist[0], h = v >= 2 ? t_hist[0] - t_hist[1] : 0.0, hp = 1.0;
+        if (v > 4) return 1;
+        for (int i = 1; i <= v; ++i) {
+            w[i] = x * gam[i - 1] * hp;
+            hp *= h;
+        }
+    } else {
+        return 1;
+    }
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < n; ++j) {
+        double s = load_elem(planes, dtype, j);
+        for (int i = 1; i <= v; ++i)
+            s += load_elem((const char*)planes + (size_t)i * plane_stride * esz, dtype, j) * w[i];
+        acc[j] += s;
+    }
+    return 0;
+}
+
+void oracle_accumulate_elems(int dtype, int64_t n, const void* src, double* acc) {
+    for (int64_t j = 0; j < n; ++j) acc[j] += load_elem(src, dtype, j);
+}
+
+void oracle_round_store(int dtype, int64_t n, const double* acc, void* out) {
+    for (int64_t j = 0; j < n; ++j) store_elem(out, dtype, j, acc[j]);
+}
+
 /* ---- Eq. 4: relative error ------------------------------------------------------------------- */
 /* e = ||pred - fresh||_2 / (||fresh||_2 + eps), Euclidean norms over the n elements of a sample. */
 double oracle_rel_l2(int dtype, int64_t n, const void* pred, const void* fresh, double eps) {

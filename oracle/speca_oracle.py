@@ -53,6 +53,12 @@ def lib() -> ctypes.CDLL:
         L.oracle_update_segment.restype = i32
         L.oracle_forecast_segment.argtypes = [i32, i64, i32, i32, i32, dp, dbl, vp, i64, vp]
         L.oracle_forecast_segment.restype = i32
+        L.oracle_forecast_accumulate_segment.argtypes = [i32, i64, i32, i32, i32, dp, dbl, vp, i64, vp]
+        L.oracle_forecast_accumulate_segment.restype = i32
+        L.oracle_accumulate_elems.argtypes = [i32, i64, vp, vp]
+        L.oracle_accumulate_elems.restype = None
+        L.oracle_round_store.argtypes = [i32, i64, vp, vp]
+        L.oracle_round_store.restype = None
         L.oracle_rel_l2.argtypes = [i32, i64, vp, vp, dbl]
         L.oracle_rel_l2.restype = dbl
         for fn in (L.oracle_rel_l1, L.oracle_rel_linf, L.oracle_cos_dist):
@@ -252,6 +258,30 @@ class OracleCache:
             out = np.zeros((K, self.B, self.entry_elems[e]), dtype=np_dtype(self.dtype))
         for k in range(K):
             self.forecast_entry(e, t_targets[k], active, out=out[k])
+        return out
+
+    def forecast_sum(self, entry_ids: Sequence[int], t_target: Sequence[float], base: Optional[np.ndarray] = None,
+                     active: Optional[Sequence[int]] = None, out: Optional[np.ndarray] = None) -> np.ndarray:
+        """out[b] = round(base[b] + sum over the listed entries of their unrounded forecasts), the form
+        in which a residual stream consumes the forecasts of equally shaped blocks. Inactive samples
+        keep what `out` held."""
+        n = self.entry_elems[entry_ids[0]]
+        assert all(self.entry_elems[e] == n for e in entry_ids)
+        if out is None:
+            out = np.zeros((self.B, n), dtype=np_dtype(self.dtype))
+        for b in range(self.B):
+            if (active is not None and not active[b]) or self.n_refs[b] < 1:
+                continue
+            acc = np.zeros(n, dtype=np.float64)
+            if base is not None:
+                lib().oracle_accumulate_elems(self.dtype, n, _ptr(np.ascontiguousarray(base[b])), _ptr(acc))
+            for e in entry_ids:
+                p = self.planes[e][b]
+                rc = lib().oracle_forecast_accumulate_segment(self.dtype, n, self.m, self.basis, self.n_refs[b],
+                                                              _hist(self.t_hist[b], self.m), float(t_target[b]),
+                                                              _ptr(p), p.strides[0] // p.itemsize, _ptr(acc))
+                assert rc == 0
+            lib().oracle_round_store(self.dtype, n, _ptr(acc), _ptr(out[b]))
         return out
 
     def verify(self, fresh: np.ndarray, t_target: Sequence[float], tau: Sequence[float],

@@ -32,6 +32,7 @@ EXPORTS = [
     "speca_cache_launch_count", "speca_status_string", "speca_last_error", "speca_version",
     "speca_verify_pred_static", "speca_forecast_multi", "speca_verify_metric",
     "speca_verify_partial", "speca_verify_decide", "speca_cache_get_history", "speca_cache_set_history",
+    "speca_forecast_sum",
 ]
 
 
@@ -76,6 +77,7 @@ def _lib() -> ctypes.CDLL:
     L.speca_cache_update.argtypes = [vp, vp, vp, vp, vp]
     L.speca_cache_commit_step.argtypes = [vp]
     L.speca_forecast.argtypes = [vp, vp, vp, vp, vp]
+    L.speca_forecast_sum.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]
     L.speca_forecast_multi.argtypes = [vp, i32, vp, vp, vp, vp]
     L.speca_verify.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.speca_verify_metric.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -204,6 +206,13 @@ def speca_cache_commit_step(cache) -> None:
 def speca_forecast(cache, t_target, dev_active_mask, outs, stream=None) -> None:
     _check(_lib().speca_forecast(cache, _doubles(t_target), _dev_ptr(dev_active_mask), _ptr_array(outs),
                                  _stream_ptr(stream)), cache)
+
+
+def speca_forecast_sum(cache, entry_ids, t_target, dev_active_mask, base, out, stream=None) -> None:
+    """out = base + sum of the forecasts of the listed (equally shaped) entries; base may be None."""
+    ids = (ctypes.c_int32 * len(entry_ids))(*[int(e) for e in entry_ids])
+    _check(_lib().speca_forecast_sum(cache, ids, len(entry_ids), _doubles(t_target), _dev_ptr(dev_active_mask),
+                                     _dev_ptr(base), _dev_ptr(out), _stream_ptr(stream)), cache)
 
 
 def speca_forecast_multi(cache, t_targets, dev_active_mask, outs, stream=None) -> None:
@@ -346,6 +355,9 @@ class SpecaCache:
 
     def forecast(self, t_target, outs, active=None, stream=None):
         speca_forecast(self.handle, t_target, active, outs, stream)
+
+    def forecast_sum(self, entry_ids, t_target, out, base=None, active=None, stream=None):
+        speca_forecast_sum(self.handle, entry_ids, t_target, active, base, out, stream)
 
     def forecast_multi(self, t_targets, outs, active=None, stream=None):
         speca_forecast_multi(self.handle, t_targets, active, outs, stream)

@@ -513,6 +513,60 @@ speca_status_t speca_forecast_multi(speca_cache_t* c, int32_t n_targets, const d
     return SPECA_OK;
 }
 
+speca_status_t speca_forecast_sum(speca_cache_t* c, const int32_t* entry_ids, int32_t n_ids, const double* t_target,
+                                  const uint8_t* dev_active_mask, const void* base, void* out, void* stream) {
+    if (c == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (entry_ids == nullptr || t_target == nullptr || out == nullptr)
+        return fail(c, SPECA_ERR_INVALID_ARG, "forecast_sum: null argument");
+    if (n_ids < 1 || n_ids > SPECA_MAX_ENTRIES) return fail(c, SPECA_ERR_INVALID_ARG, "forecast_sum: n_ids out of range");
+    if (c->pending) return fail(c, SPECA_ERR_STATE, "forecast_sum: a reference step is open (commit it first)");
+    static thread_local SumParams p;
+    std::memset(&p, 0, sizeof p);
+    const Layout& L = c->L;
+    for (int j = 0; j < n_ids; ++j) {
+        if (entry_ids[j] < 0 || entry_ids[j] >= c->n_entries)
+            return fail(c, SPECA_ERR_INVALID_ARG, "forecast_sum: entry_ids[%d] out of range", j);
+        const uint32_t n = L.segs[static_cast<size_t>(entry_ids[j]) * c->B].n_elems;
+        if (j == 0) p.n_elems = n;
+        if (n != p.n_elems) return fail(c, SPECA_ERR_SHAPE, "forecast_sum: entries %d and %d differ in size", entry_ids[0], entry_ids[j]);
+        p.ids[j] = static_cast<uint16_t>(entry_ids[j]);
+    }
+    const size_t esz = elem_size(c);
+    if (reinterpret_cast<uintptr_t>(out) % esz != 0 || reinterpret_cast<uintptr_t>(base) % esz != 0)
+        return fail(c, SPECA_ERR_ALIGNMENT, "forecast_sum: base / out not aligned to the element size");
+    bool any_sample = false;
+    for (int b = 0; b < c->B; ++b) {
+        if (!std::isfinite(t_target[b])) return fail(c, SPECA_ERR_INVALID_ARG, "forecast_sum: t_target[%d] not finite", b);
+        int order;
+        forecast_scalars(c, b, t_target[b], &order, p.coef[b]);
+        if (order < 0 && dev_active_mask == nullptr)
+            return fail(c, SPECA_ERR_STATE, "forecast_sum: sample %d has no committed reference", b);
+        p.order[b] = static_cast<int8_t>(order);
+        any_sample |= order >= 0;
+    }
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return fail(c, SPECA_ERR_CUDA, "cudaSetDevice failed");
+    speca_status_t st = check_sticky(c);
+    if (st != SPECA_OK) return st;
+    if (!any_sample) return SPECA_OK;
+    const uint32_t te = sum_tile_bytes() / static_cast<uint32_t>(esz);
+    p.segs = reinterpret_cast<const SegDesc*>(c->arena + L.segs_off);
+    p.arena = c->arena;
+    p.dev_mask = dev_active_mask;
+    p.base = static_cast<const char*>(base);
+    p.out = static_cast<char*>(out);
+    p.tiles_per_sample = (p.n_elems + te - 1) / te;
+    p.batch = c->B;
+    p.n_ids = n_ids;
+    const uint64_t tiles = static_cast<uint64_t>(p.tiles_per_sample) * c->B;
+    const uint64_t full = static_cast<uint64_t>(c->sm_count) * sum_ctas_per_sm();
+    const int grid = static_cast<int>(tiles < full ? tiles : full);
+    cudaError_t ce = launch_forecast_sum(p, c->dtype, grid, static_cast<cudaStream_t>(stream));
+    if (ce != cudaSuccess) return cuda_fail(c, ce, "forecast_sum launch");
+    c->launches += 1;
+    return SPECA_OK;
+}
+
 speca_status_t speca_verify(speca_cache_t* c, const void* fresh, const double* t_target, const float* tau,
                             const uint8_t* dev_active_mask, void* out_pred, float* dev_err, uint8_t* dev_accept,
                             void* stream) {

@@ -66,6 +66,22 @@ struct MultiParams {
     void* io[SPECA_MAX_ENTRIES];      // per entry: [K, B, N_e, D] output; null = skip
 };
 
+// Arguments of the summed forecast: out = base + sum over a list of equally shaped entries.
+struct SumParams {
+    const SegDesc* segs;  // all segments of the cache
+    char* arena;
+    const uint8_t* dev_mask;
+    const char* base;     // [B, n_elems] or null
+    char* out;            // [B, n_elems]
+    uint32_t n_elems;     // per sample (common to the listed entries)
+    uint32_t tiles_per_sample;
+    int32_t batch;
+    int32_t n_ids;
+    int8_t order[SPECA_MAX_BATCH];
+    float coef[SPECA_MAX_BATCH][SPECA_MAX_ORDER];
+    uint16_t ids[SPECA_MAX_ENTRIES];  // entries to add, in this order
+};
+
 // Arguments of the fused forecast + relative-L2 kernel over the verification entry.
 struct VerifyParams {
     const SegDesc* segs;  // segments of the verify entry only (B of them)
@@ -112,6 +128,9 @@ int multi_ctas_per_sm();
 cudaError_t launch_forecast_multi(const MultiParams& p, int dtype, int batch, int grid, cudaStream_t stream);
 cudaError_t launch_decide(int metric, const double* sums, int batch, const DecideParams& q, const uint8_t* mask, float* err,
                           uint8_t* accept, cudaStream_t stream);
+uint32_t sum_tile_bytes();
+int sum_ctas_per_sm();
+cudaError_t launch_forecast_sum(const SumParams& p, int dtype, int grid, cudaStream_t stream);
 // Clusters of the verify kernel that fit on the current device at once.
 int max_resident_verify_clusters(int dtype, int order, int cluster);
 

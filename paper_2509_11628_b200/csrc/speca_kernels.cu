@@ -535,6 +535,94 @@ __global__ void __launch_bounds__(NT, MINB) forecast_multi_kernel(const __grid_c
 }
 
 // ------------------------------------------------------------------------------------------------
+// summed forecast: the forecasts of equally shaped entries added into one output
+// ------------------------------------------------------------------------------------------------
+// A transformer adds its block outputs to a residual stream, so on a speculative step the forecasts
+// of equally shaped blocks are only consumed as base + sum_e forecast_e. Computing that sum directly
+// reads the v + 1 planes of every listed entry and writes one tensor: E (v + 1) + 1 (+ 1 with a base)
+// words per element instead of E (v + 2) for separate forecasts (and the adds the model would then
+// do). Each entry's Horner result stays in fp32 and is added unrounded, in list order; the total is
+// rounded once. Read-dominated, so it uses the forecast's launch shape: 256 threads, one 32-byte
+// vector per plane, 3 CTAs/SM; a tile is 8 KB of the output row.
+constexpr int kSumW = 32, kSumThreads = 256, kSumMinBlocks = 3;
+constexpr uint32_t kSumTileBytes = kSumW * kSumThreads;
+
+template <int DT, int V>
+__global__ void __launch_bounds__(kSumThreads, kSumMinBlocks) forecast_sum_kernel(const __grid_constant__ SumParams p) {
+    constexpr int W = kSumW;
+    constexpr int EPV = W / Elem<DT>::kBytes;
+    constexpr uint32_t kTile = kSumTileBytes / Elem<DT>::kBytes;
+    const uint32_t total = static_cast<uint32_t>(p.batch) * p.tiles_per_sample;
+    const uint64_t row_bytes = static_cast<uint64_t>(p.n_elems) * Elem<DT>::kBytes;
+    for (uint32_t t = blockIdx.x; t < total; t += gridDim.x) {
+        const uint32_t b = t / p.tiles_per_sample;
+        const int v = p.order[b];
+        if (v < 0 || (p.dev_mask != nullptr && p.dev_mask[b] == 0)) continue;
+        const uint32_t elem0 = (t - b * p.tiles_per_sample) * kTile;
+        const uint32_t cnt = min(kTile, p.n_elems - elem0);
+        const uint64_t byte0 = static_cast<uint64_t>(elem0) * Elem<DT>::kBytes;
+        const char* base = p.base != nullptr ? p.base + b * row_bytes + byte0 : nullptr;
+        char* out = p.out + b * row_bytes + byte0;
+        float mu[SPECA_MAX_ORDER];
+#pragma unroll
+        for (int i = 0; i < SPECA_MAX_ORDER; ++i) mu[i] = p.coef[b][i];
+        const uint32_t idx = threadIdx.x;
+        const bool vec_ok = ((reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(base)) & (W - 1)) == 0;
+        const uint32_t nvec = vec_ok ? cnt / EPV : 0;
+        if (idx < nvec) {
+            float sum[EPV];
+            if (base != nullptr) {
+                unpack_vec<DT, W>(load_vec<W>(base + static_cast<size_t>(idx) * W), sum);
+            } else {
+#pragma unroll
+                for (int k = 0; k < EPV; ++k) sum[k] = 0.f;
+            }
+            for (int j = 0; j < p.n_ids; ++j) {
+                const SegDesc sd = p.segs[static_cast<uint32_t>(p.ids[j]) * p.batch + b];
+                const char* plane0 = p.arena + sd.plane0_off + byte0 + static_cast<size_t>(idx) * W;
+                float acc[EPV];
+                if (v == V) {
+                    Vec<W> d[V + 1];
+#pragma unroll
+                    for (int i = 0; i <= V; ++i) d[i] = load_vec<W>(plane0 + i * sd.plane_stride);
+                    unpack_vec<DT, W>(d[V], acc);
+#pragma unroll
+                    for (int i = V; i >= 1; --i) {
+                        float lo[EPV];
+                        unpack_vec<DT, W>(d[i - 1], lo);
+#pragma unroll
+                        for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+                    }
+                } else {  // a sample with fewer references than the launch's common order
+                    unpack_vec<DT, W>(load_vec<W>(plane0 + v * sd.plane_stride), acc);
+                    for (int i = v; i >= 1; --i) {
+                        float lo[EPV];
+                        unpack_vec<DT, W>(load_vec<W>(plane0 + (i - 1) * sd.plane_stride), lo);
+#pragma unroll
+                        for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < EPV; ++k) sum[k] += acc[k];
+            }
+            store_vec<W>(out + static_cast<size_t>(idx) * W, pack_vec<DT, W>(sum));
+        }
+        // ragged tail of the row, or the whole tile when a row is not 32-byte aligned
+        for (uint32_t e = nvec * EPV + threadIdx.x; e < cnt; e += kSumThreads) {
+            float sum = base != nullptr ? load_scalar<DT>(base, e) : 0.f;
+            for (int j = 0; j < p.n_ids; ++j) {
+                const SegDesc sd = p.segs[static_cast<uint32_t>(p.ids[j]) * p.batch + b];
+                const char* plane0 = p.arena + sd.plane0_off + byte0;
+                float acc = load_scalar<DT>(plane0 + v * sd.plane_stride, e);
+                for (int i = v; i >= 1; --i) acc = fmaf(acc, mu[i - 1], load_scalar<DT>(plane0 + (i - 1) * sd.plane_stride, e));
+                sum += acc;
+            }
+            store_scalar<DT>(out, e, sum);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // bulk path: the same streams staged through shared memory by the TMA engine
 // ------------------------------------------------------------------------------------------------
 // One elected thread issues `cp.async.bulk` copies (untiled TMA, 8 KB per plane and tile, no
@@ -1285,6 +1373,27 @@ cudaError_t launch_forecast_multi(const MultiParams& p, int dtype, int batch, in
     const void* fn = dtype == SPECA_BF16 ? multi_kernel_for<SPECA_BF16>(v) : multi_kernel_for<SPECA_F32>(v);
     void* args[2] = {const_cast<MultiParams*>(&p), &batch};
     return cudaLaunchKernel(fn, dim3(grid), dim3(kMultiShape.nt), args, 0, stream);
+}
+
+template <int DT>
+static const void* sum_kernel_for(int v) {
+    switch (v) {
+        case 0: return reinterpret_cast<const void*>(&forecast_sum_kernel<DT, 0>);
+        case 1: return reinterpret_cast<const void*>(&forecast_sum_kernel<DT, 1>);
+        case 2: return reinterpret_cast<const void*>(&forecast_sum_kernel<DT, 2>);
+        case 3: return reinterpret_cast<const void*>(&forecast_sum_kernel<DT, 3>);
+        default: return reinterpret_cast<const void*>(&forecast_sum_kernel<DT, 4>);
+    }
+}
+
+uint32_t sum_tile_bytes() { return kSumTileBytes; }
+int sum_ctas_per_sm() { return kSumMinBlocks; }
+
+cudaError_t launch_forecast_sum(const SumParams& p, int dtype, int grid, cudaStream_t stream) {
+    const int v = max_order(p.order);
+    const void* fn = dtype == SPECA_BF16 ? sum_kernel_for<SPECA_BF16>(v) : sum_kernel_for<SPECA_F32>(v);
+    void* args[1] = {const_cast<SumParams*>(&p)};
+    return cudaLaunchKernel(fn, dim3(grid), dim3(kSumThreads), args, 0, stream);
 }
 
 static void verify_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int grid, int cluster,

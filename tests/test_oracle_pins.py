@@ -316,6 +316,51 @@ def test_bf16_tables_round_once_per_stored_plane():
 
 
 # ---------------------------------------------------------------------------------------------
+# forecasts consumed as a sum (residual stream)
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("basis", [O.TAYLOR, O.NEWTON, O.ADAMS_BASHFORTH])
+@pytest.mark.parametrize("dtype", [O.F32, O.BF16])
+def test_summed_forecast_of_one_entry_is_the_plain_forecast_bit_for_bit(basis, dtype):
+    g = torch.Generator().manual_seed(90 + basis)
+    B, n, m = 2, 300, 3
+    cache = O.OracleCache([n, n], B, m, dtype, basis)
+    for k, t in enumerate([1.0, 0.93, 0.9, 0.81]):
+        fs = [torch.randn(B, n, generator=g) for _ in range(2)]
+        fs = [bf16_bits(f) if dtype == O.BF16 else f.numpy().copy() for f in fs]
+        cache.update(fs, [t, t - 0.004])
+        cache.commit_step()
+    tt = [0.77, 0.75]
+    for e in (0, 1):
+        assert np.array_equal(cache.forecast_sum([e], tt), cache.forecast_entry(e, tt))
+
+
+def test_summed_forecast_is_the_sum_of_the_forecasts_in_exact_arithmetic():
+    # integer features, integer times, fp32 storage: every product and sum below is exact, so the sum
+    # of the separately stored forecasts must equal the summed forecast, and adding a base adds it
+    rng = np.random.default_rng(9)
+    B, n, m, E = 2, 64, 2, 5
+    cache = O.OracleCache([n] * E, B, m, O.F32)
+    for t in (8.0, 6.0, 4.0):
+        cache.update([rng.integers(-20, 20, (B, n)).astype(np.float32) * 8 for _ in range(E)], [t] * B)
+        cache.commit_step()
+    tt = [2.0, 0.0]
+    parts = [as64(cache.forecast_entry(e, tt)) for e in range(E)]
+    base = rng.integers(-100, 100, (B, n)).astype(np.float32)
+    total = cache.forecast_sum(list(range(E)), tt)
+    assert np.array_equal(as64(total), sum(parts))
+    assert np.array_equal(as64(cache.forecast_sum([1, 3], tt, base=base)), parts[1] + parts[3] + base)
+    # inactive samples keep what the output held
+    out = np.full((B, n), 7.0, dtype=np.float32)
+    cache.forecast_sum([0, 1], tt, active=[0, 1], out=out)
+    assert np.all(out[0] == 7.0) and np.array_equal(as64(out[1]), (parts[0] + parts[1])[1])
+
+
+def as64(a):
+    return a.astype(np.float64)
+
+
+# ---------------------------------------------------------------------------------------------
 # the appendix's prediction-error bound, as a soft check (it equates differences with derivatives)
 # ---------------------------------------------------------------------------------------------
 
