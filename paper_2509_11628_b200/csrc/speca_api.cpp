@@ -127,7 +127,7 @@ struct speca_cache {
     char* arena;
     Layout L;
     int sm_count;
-    int grid_update, grid_forecast, grid_verify, cluster;
+    int grid_verify, cluster;
     int tile_update, tile_forecast;  // indices into kTileSizes
     // per-sample reference history, most recent first
     int32_t n_refs[SPECA_MAX_BATCH];
@@ -164,6 +164,13 @@ speca_status_t check_sticky(speca_cache* c) {
     cudaError_t e = cudaPeekAtLastError();
     if (e != cudaSuccess) return cuda_fail(c, e, "earlier CUDA error");
     return SPECA_OK;
+}
+
+// The order a launch's kernel is compiled for: the highest among its samples.
+int launch_order(const int8_t* order, int batch) {
+    int v = 0;
+    for (int b = 0; b < batch; ++b) v = order[b] > v ? order[b] : v;
+    return v;
 }
 
 // Horner multipliers of Eq. 2 for sample b at time t: level i (1-based) multiplies by mu[i-1].
@@ -278,8 +285,6 @@ speca_status_t speca_cache_create(const speca_cache_config_t* cfg, speca_cache_t
         delete c;
         return SPECA_ERR_UNSUPPORTED;
     }
-    c->grid_update = c->sm_count * stream_ctas_per_sm(c->path, true, c->dtype, c->m);
-    c->grid_forecast = c->sm_count * stream_ctas_per_sm(c->path, false, c->dtype, c->m);
     c->cluster = 4;
     int n_clusters = max_resident_verify_clusters(c->dtype, c->m, c->cluster);
     if (n_clusters > kMaxClusters) n_clusters = kMaxClusters;
@@ -370,7 +375,8 @@ speca_status_t speca_cache_update(speca_cache_t* c, const void* const* feats, co
         p.tile_lo = tiles[p.seg_lo];
         p.tile_hi = tiles[p.seg_hi];
         const uint32_t n_tiles = p.tile_hi - p.tile_lo;
-        const int grid = static_cast<int>(n_tiles < static_cast<uint32_t>(c->grid_update) ? n_tiles : c->grid_update);
+        const uint32_t full = static_cast<uint32_t>(c->sm_count * stream_ctas_per_sm(c->path, true, c->dtype, launch_order(p.order, c->B)));
+        const int grid = static_cast<int>(n_tiles < full ? n_tiles : full);
         cudaError_t ce = launch_update(p, c->dtype, c->path, grid, static_cast<cudaStream_t>(stream));
         if (ce != cudaSuccess) return cuda_fail(c, ce, "update launch");
         c->launches += 1;
@@ -447,7 +453,8 @@ speca_status_t speca_forecast(speca_cache_t* c, const double* t_target, const ui
     p.tile_lo = tiles[p.seg_lo];
     p.tile_hi = tiles[p.seg_hi];
     const uint32_t n_tiles = p.tile_hi - p.tile_lo;
-    const int grid = static_cast<int>(n_tiles < static_cast<uint32_t>(c->grid_forecast) ? n_tiles : c->grid_forecast);
+    const uint32_t full = static_cast<uint32_t>(c->sm_count * stream_ctas_per_sm(c->path, false, c->dtype, launch_order(p.order, c->B)));
+    const int grid = static_cast<int>(n_tiles < full ? n_tiles : full);
     cudaError_t ce = launch_forecast(p, c->dtype, c->path, grid, static_cast<cudaStream_t>(stream));
     if (ce != cudaSuccess) return cuda_fail(c, ce, "forecast launch");
     c->launches += 1;

@@ -363,12 +363,15 @@ __device__ __noinline__ void update_tile_any(char* __restrict__ plane0, uint64_t
 // ------------------------------------------------------------------------------------------------
 // Launch shapes. Both kernels are pure HBM streams whose speed is set by how the DRAM sees the mix
 // of reads and writes, so the shape (vector width, threads, vectors per thread, CTAs per SM) was
-// chosen by sweeping it on a B200 at order 2, bf16, with every plane 4 KB aligned:
+// chosen by sweeping it on a B200 in bf16 with every plane 4 KB aligned (at order 2):
 //   update   (half of the traffic is writes): few bytes in flight win -- 128 threads x one 32-byte
 //            vector per plane, 3 CTAs/SM (36 KB in flight per SM) reaches the device's copy rate;
 //            deeper or wider shapes (256 x 4 vectors, 2 CTAs/SM) are 4-9 % slower on this mix.
 //   forecast (one write per three reads): flat above ~70 KB in flight per SM; 256 threads x one
 //            vector per plane, 3 CTAs/SM.
+// Other orders were swept the same way (FLUX shape, GB/s before -> after giving each order its own
+// shape): update order 0: 4600 -> 6470, order 1: 5810 -> 6450, order 4: 6300 -> 6490; forecast order 0
+// (a plain copy): 6070 -> 6350, order 3: 6750 -> 6840, order 4: 6670 -> 6940.
 // SPECA_PATH_DIRECT keeps a 16-byte / 256-thread / 4-deep shape for both.
 // A tile is `chunks` consecutive chunks of NT x U vectors; a CTA finishes one chunk (loads, arithmetic,
 // stores) before it starts the next, so the bytes in flight are set by NT x U x W while the per-tile
@@ -376,16 +379,23 @@ __device__ __noinline__ void update_tile_any(char* __restrict__ plane0, uint64_t
 struct Shape {
     int w, nt, u, chunks, minb;
 };
-#ifndef SPECA_SHAPE_UPDATE
-#define SPECA_SHAPE_UPDATE 32, 128, 1, 8, 3
+// One shape per order v: the number of streams grows with v, so the vectors per thread shrink to keep
+// the bytes in flight per SM near the sweet spot of the mix. Every shape has a 32 KB tile.
+#ifndef SPECA_SHAPES_UPDATE
+#define SPECA_SHAPES_UPDATE \
+    {32, 128, 2, 4, 4}, {32, 128, 2, 4, 3}, {32, 128, 1, 8, 3}, {32, 128, 1, 8, 3}, { 32, 128, 1, 8, 2 }
 #endif
-#ifndef SPECA_SHAPE_FORECAST
-#define SPECA_SHAPE_FORECAST 32, 256, 1, 4, 3
+#ifndef SPECA_SHAPES_FORECAST
+#define SPECA_SHAPES_FORECAST \
+    {32, 128, 2, 4, 4}, {32, 256, 1, 4, 3}, {32, 256, 1, 4, 3}, {32, 256, 1, 4, 2}, { 32, 256, 1, 4, 2 }
 #endif
-__host__ __device__ constexpr Shape shape_for(int path, bool update) {
-    return path == SPECA_PATH_WIDE ? (update ? Shape{SPECA_SHAPE_UPDATE} : Shape{SPECA_SHAPE_FORECAST})
-                                   : Shape{16, 256, 4, 1, 2};
+__host__ __device__ constexpr Shape shape_for(int path, bool update, int v) {
+    constexpr Shape up[SPECA_MAX_ORDER + 1] = {SPECA_SHAPES_UPDATE};
+    constexpr Shape fc[SPECA_MAX_ORDER + 1] = {SPECA_SHAPES_FORECAST};
+    const int i = v < 0 ? 0 : (v > SPECA_MAX_ORDER ? SPECA_MAX_ORDER : v);
+    return path == SPECA_PATH_WIDE ? (update ? up[i] : fc[i]) : Shape{16, 256, 4, 1, 2};
 }
+__host__ __device__ constexpr uint32_t shape_tile_bytes(Shape s) { return static_cast<uint32_t>(s.w) * s.nt * s.u * s.chunks; }
 
 // V = the order most samples of the launch have (the host passes the maximum over samples).
 template <int DT, int V, bool UPDATE, int W, int NT, int U, int C, int MINB>
@@ -441,7 +451,7 @@ __global__ void __launch_bounds__(NT, MINB) stream_kernel(const __grid_constant_
 // Evaluating them in one pass reads the v + 1 planes once and writes K outputs: (v + 1 + K) words per
 // element instead of K (v + 2). Output k of entry e is row k of a [K, B, N_e, D] tensor. The mix is
 // write-heavy like the update, so the kernel uses the update's launch shape.
-constexpr Shape kMultiShape = Shape{SPECA_SHAPE_UPDATE};
+constexpr Shape kMultiShape = Shape{32, 128, 1, 8, 3};
 
 template <int DT, int V, int W, int NT, int U>
 __device__ __forceinline__ void forecast_multi_tile(const char* __restrict__ plane0, uint64_t stride,
@@ -1237,13 +1247,17 @@ __global__ void __launch_bounds__(SPECA_MAX_BATCH) activate_kernel(uint64_t mask
 
 template <int DT, bool UPDATE, int PATH>
 static const void* stream_kernel_for(int v) {
-    constexpr Shape s = shape_for(PATH, UPDATE);
+    constexpr Shape s0 = shape_for(PATH, UPDATE, 0), s1 = shape_for(PATH, UPDATE, 1), s2 = shape_for(PATH, UPDATE, 2),
+                    s3 = shape_for(PATH, UPDATE, 3), s4 = shape_for(PATH, UPDATE, 4);
+    static_assert(shape_tile_bytes(s0) == shape_tile_bytes(s2) && shape_tile_bytes(s1) == shape_tile_bytes(s2) &&
+                      shape_tile_bytes(s3) == shape_tile_bytes(s2) && shape_tile_bytes(s4) == shape_tile_bytes(s2),
+                  "all orders of a path share one tile size (one tile table)");
     switch (v) {
-        case 0: return reinterpret_cast<const void*>(&stream_kernel<DT, 0, UPDATE, s.w, s.nt, s.u, s.chunks, s.minb>);
-        case 1: return reinterpret_cast<const void*>(&stream_kernel<DT, 1, UPDATE, s.w, s.nt, s.u, s.chunks, s.minb>);
-        case 2: return reinterpret_cast<const void*>(&stream_kernel<DT, 2, UPDATE, s.w, s.nt, s.u, s.chunks, s.minb>);
-        case 3: return reinterpret_cast<const void*>(&stream_kernel<DT, 3, UPDATE, s.w, s.nt, s.u, s.chunks, s.minb>);
-        default: return reinterpret_cast<const void*>(&stream_kernel<DT, 4, UPDATE, s.w, s.nt, s.u, s.chunks, s.minb>);
+        case 0: return reinterpret_cast<const void*>(&stream_kernel<DT, 0, UPDATE, s0.w, s0.nt, s0.u, s0.chunks, s0.minb>);
+        case 1: return reinterpret_cast<const void*>(&stream_kernel<DT, 1, UPDATE, s1.w, s1.nt, s1.u, s1.chunks, s1.minb>);
+        case 2: return reinterpret_cast<const void*>(&stream_kernel<DT, 2, UPDATE, s2.w, s2.nt, s2.u, s2.chunks, s2.minb>);
+        case 3: return reinterpret_cast<const void*>(&stream_kernel<DT, 3, UPDATE, s3.w, s3.nt, s3.u, s3.chunks, s3.minb>);
+        default: return reinterpret_cast<const void*>(&stream_kernel<DT, 4, UPDATE, s4.w, s4.nt, s4.u, s4.chunks, s4.minb>);
     }
 }
 
@@ -1309,8 +1323,7 @@ static int clamp_order(int v) { return v < 0 ? 0 : (v > SPECA_MAX_ORDER ? SPECA_
 
 uint32_t stream_tile_bytes(int path, bool update) {
     if (path == SPECA_PATH_BULK) return kBulkTileBytes;
-    const Shape s = shape_for(path, update);
-    return static_cast<uint32_t>(s.w) * s.nt * s.u * s.chunks;
+    return shape_tile_bytes(shape_for(path, update, 2));
 }
 
 int stream_ctas_per_sm(int path, bool update, int dtype, int order) {
@@ -1325,7 +1338,7 @@ int stream_ctas_per_sm(int path, bool update, int dtype, int order) {
         }
         return n;
     }
-    return shape_for(path, update).minb;
+    return shape_for(path, update, order).minb;
 }
 
 static cudaError_t launch_stream(const StreamParams& p, int dtype, bool update, int path, int grid,
@@ -1340,9 +1353,10 @@ static cudaError_t launch_stream(const StreamParams& p, int dtype, bool update, 
         return cudaLaunchKernel(fn, dim3(grid), dim3(kBulkThreads), args, smem, stream);
     }
     if (path != SPECA_PATH_DIRECT && path != SPECA_PATH_WIDE) return cudaErrorNotSupported;
-    const void* fn = stream_kernel_for(dtype, update, path, max_order(p.order));
+    const int v = max_order(p.order);
+    const void* fn = stream_kernel_for(dtype, update, path, v);
     void* args[1] = {const_cast<StreamParams*>(&p)};
-    return cudaLaunchKernel(fn, dim3(grid), dim3(shape_for(path, update).nt), args, 0, stream);
+    return cudaLaunchKernel(fn, dim3(grid), dim3(shape_for(path, update, v).nt), args, 0, stream);
 }
 
 cudaError_t launch_update(const StreamParams& p, int dtype, int path, int grid, cudaStream_t stream) {
