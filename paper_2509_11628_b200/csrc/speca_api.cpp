@@ -512,7 +512,7 @@ speca_status_t speca_forecast_multi(speca_cache_t* c, int32_t n_targets, const d
     p.tile_lo = tiles[p.seg_lo];
     p.tile_hi = tiles[p.seg_hi];
     const uint32_t n_tiles = p.tile_hi - p.tile_lo;
-    const uint32_t full = static_cast<uint32_t>(c->sm_count * multi_ctas_per_sm());
+    const uint32_t full = static_cast<uint32_t>(c->sm_count * multi_ctas_per_sm(n_targets));
     const int grid = static_cast<int>(n_tiles < full ? n_tiles : full);
     cudaError_t ce = launch_forecast_multi(p, c->dtype, c->B, grid, static_cast<cudaStream_t>(stream));
     if (ce != cudaSuccess) return cuda_fail(c, ce, "forecast_multi launch");

@@ -124,7 +124,7 @@ uint32_t stream_tile_bytes(int path, bool update);
 int stream_ctas_per_sm(int path, bool update, int dtype, int order);
 // Multi-horizon forecast kernel: tile size, designed CTAs per SM, launcher.
 uint32_t multi_tile_bytes();
-int multi_ctas_per_sm();
+int multi_ctas_per_sm(int n_targets);
 cudaError_t launch_forecast_multi(const MultiParams& p, int dtype, int batch, int grid, cudaStream_t stream);
 cudaError_t launch_decide(int metric, const double* sums, int batch, const DecideParams& q, const uint8_t* mask, float* err,
                           uint8_t* accept, cudaStream_t stream);

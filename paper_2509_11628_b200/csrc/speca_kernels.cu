@@ -449,9 +449,14 @@ __global__ void __launch_bounds__(NT, MINB) stream_kernel(const __grid_constant_
 // ------------------------------------------------------------------------------------------------
 // The draft model predicts several future steps from the same reference (Fig. 1, workflow step 2).
 // Evaluating them in one pass reads the v + 1 planes once and writes K outputs: (v + 1 + K) words per
-// element instead of K (v + 2). Output k of entry e is row k of a [K, B, N_e, D] tensor. The mix is
-// write-heavy like the update, so the kernel uses the update's launch shape.
-constexpr Shape kMultiShape = Shape{32, 128, 1, 8, 3};
+// element instead of K (v + 2). Output k of entry e is row k of a [K, B, N_e, D] tensor.
+// Swept like the others: up to 5 targets the mix is close to the update's and 256 threads x 2 CTAs/SM
+// win (6700 / 6480 GB/s at K = 2 / 4 on the FLUX shape against 6090 / 6350); with more targets writes
+// dominate and the narrower 128 x 3 shape is better (6320 against 5930 at K = 8).
+__host__ __device__ constexpr Shape multi_shape(int n_targets) {
+    return n_targets <= 5 ? Shape{32, 256, 1, 4, 2} : Shape{32, 128, 1, 8, 3};
+}
+static_assert(shape_tile_bytes(multi_shape(1)) == shape_tile_bytes(multi_shape(8)), "one tile table for both");
 
 template <int DT, int V, int W, int NT, int U>
 __device__ __forceinline__ void forecast_multi_tile(const char* __restrict__ plane0, uint64_t stride,
@@ -1367,9 +1372,9 @@ cudaError_t launch_forecast(const StreamParams& p, int dtype, int path, int grid
     return launch_stream(p, dtype, false, path, grid, stream);
 }
 
-template <int DT>
+template <int DT, int KCLASS>
 static const void* multi_kernel_for(int v) {
-    constexpr Shape s = kMultiShape;
+    constexpr Shape s = multi_shape(KCLASS);
     switch (v) {
         case 0: return reinterpret_cast<const void*>(&forecast_multi_kernel<DT, 0, s.w, s.nt, s.u, s.chunks, s.minb>);
         case 1: return reinterpret_cast<const void*>(&forecast_multi_kernel<DT, 1, s.w, s.nt, s.u, s.chunks, s.minb>);
@@ -1379,14 +1384,18 @@ static const void* multi_kernel_for(int v) {
     }
 }
 
-uint32_t multi_tile_bytes() { return static_cast<uint32_t>(kMultiShape.w) * kMultiShape.nt * kMultiShape.u * kMultiShape.chunks; }
-int multi_ctas_per_sm() { return kMultiShape.minb; }
+uint32_t multi_tile_bytes() { return shape_tile_bytes(multi_shape(1)); }
+int multi_ctas_per_sm(int n_targets) { return multi_shape(n_targets).minb; }
 
 cudaError_t launch_forecast_multi(const MultiParams& p, int dtype, int batch, int grid, cudaStream_t stream) {
     const int v = max_order(p.order);
-    const void* fn = dtype == SPECA_BF16 ? multi_kernel_for<SPECA_BF16>(v) : multi_kernel_for<SPECA_F32>(v);
+    const void* fn;
+    if (p.n_targets <= 5)
+        fn = dtype == SPECA_BF16 ? multi_kernel_for<SPECA_BF16, 1>(v) : multi_kernel_for<SPECA_F32, 1>(v);
+    else
+        fn = dtype == SPECA_BF16 ? multi_kernel_for<SPECA_BF16, 8>(v) : multi_kernel_for<SPECA_F32, 8>(v);
     void* args[2] = {const_cast<MultiParams*>(&p), &batch};
-    return cudaLaunchKernel(fn, dim3(grid), dim3(kMultiShape.nt), args, 0, stream);
+    return cudaLaunchKernel(fn, dim3(grid), dim3(multi_shape(p.n_targets).nt), args, 0, stream);
 }
 
 template <int DT>
