@@ -588,6 +588,60 @@ def oracle_sample_run(w: W.Workload, sample_elems: int, repeats: int, seed: int 
     return dt, bytes_step, O.threads(), n
 
 
+def parity_on_verify_entry(w: W.Workload, device: str, path: int):
+    """The same seeded features through the library and through the oracle, on the workload's
+    verification entry alone (full size): norm-wise forecast difference, verification errors,
+    decisions. Part of the CPU-baseline leg: the one place the benchmark runs the oracle."""
+    import numpy as np
+    from oracle import speca_oracle as O
+    from paper_2509_11628_b200 import binding as S
+    B, m = w.batch, w.max_order
+    n_tok, dim = w.entries[w.vidx]
+    one = W.Workload(name=w.name + "_verify_entry", index=w.index, entries=[(n_tok, dim)], batch=B, max_order=m,
+                     dtype=w.dtype, times=w.times, poly_degree=w.poly_degree, sigma=w.sigma, outlier_frac=w.outlier_frac,
+                     frame_tokens=w.frame_tokens, n_frames=w.n_frames, video_tokens=min(w.video_tokens, n_tok))
+    src = W.FeatureSource(one, device)
+    gpu = S.SpecaCache(one.entries, B, m, w.dtype, device, path=path)
+    cpu = O.OracleCache([n_tok * dim], B, m, w.dtype)
+
+    def host(x):
+        x = x.detach().contiguous().cpu()
+        if x.dtype == torch.bfloat16:
+            return x.view(torch.int16).numpy().view(np.uint16).reshape(B, -1).copy()
+        return x.numpy().reshape(B, -1).copy()
+
+    def f64(a):
+        return (a.astype(np.uint32) << 16).view(np.float32).astype(np.float64) if a.dtype == np.uint16 else a.astype(np.float64)
+
+    for step in range(m + 1):
+        t = [w.times[step]] * B
+        f = src.feature(0, step, t)
+        gpu.update([f], t)
+        gpu.commit_step()
+        cpu.update([host(f)], t)
+        cpu.commit_step()
+    step = m + 1
+    t = [w.times[step]] * B
+    tau = [0.1] * B
+    fresh = src.feature(0, step, t)
+    pred = torch.empty_like(fresh)
+    err = torch.zeros(B, dtype=torch.float32, device=device)
+    acc = torch.zeros(B, dtype=torch.uint8, device=device)
+    gpu.verify(fresh, t, tau, err, acc, out_pred=pred)
+    torch.cuda.synchronize()
+    e_want, a_want, p_want = cpu.verify(host(fresh), t, tau)
+    g, o = f64(host(pred)), f64(p_want)
+    rel = [float(np.linalg.norm(g[b] - o[b]) / max(np.linalg.norm(o[b]), 1e-30)) for b in range(B)]
+    e_got = [float(x) for x in err.cpu().tolist()]
+    out = {"entry_elems": n_tok * dim, "samples": B,
+           "forecast_norm_rel_diff_max": max(rel), "forecast_tolerance": 2e-3,
+           "err_library": e_got, "err_oracle": [float(x) for x in e_want],
+           "err_abs_diff_max": max(abs(a - b_) for a, b_ in zip(e_got, e_want)), "err_tolerance": 1e-4,
+           "decisions_equal": [int(x) for x in acc.cpu().tolist()] == [int(x) for x in a_want]}
+    gpu.close()
+    return out
+
+
 def run_reference(args, info: D.RankInfo):
     """The oracle timed on the host cores for the same metric (bounded sample per step)."""
     if not info.is_main:
@@ -763,6 +817,16 @@ def main():
                         "sample": "%d steps of update+forecast+verify+select over the verification entry only "
                                   "(%d elements x %d samples), not all %d entries" % (reps, n, w.batch, len(w.entries)),
                         "s_per_step": dt}
+        from oracle import speca_oracle as _O
+        n_threads = _O.threads()
+        _O.set_threads(1)
+        dt_one, _, _, _ = oracle_sample_run(w, n_s, 1)
+        _O.set_threads(n_threads)
+        cpu_baseline["value_1_thread"] = bytes_step / dt_one / 1e9
+        try:
+            cpu_baseline["parity"] = parity_on_verify_entry(w, device, path)
+        except Exception as exc:  # report, do not hide
+            cpu_baseline["parity"] = {"error": repr(exc)}
 
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": info.world, "steps": args.steps,
