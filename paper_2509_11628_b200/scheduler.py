@@ -124,11 +124,23 @@ class SpecaCacheBackend:
         self.spec = torch.zeros(self.batch, dtype=torch.int32, device=dev)
         self.idx = torch.zeros(self.batch, dtype=torch.int32, device=dev)
         self.n_active = torch.zeros(1, dtype=torch.int32, device=dev)
+        # pinned host mirrors: one stream synchronisation per step brings back errors, decisions and mask
+        self.h_err = torch.zeros(self.batch, dtype=torch.float32).pin_memory()
+        self.h_accept = torch.zeros(self.batch, dtype=torch.uint8).pin_memory()
+        self.h_active = torch.zeros(self.batch, dtype=torch.uint8).pin_memory()
 
     def reset_run(self):
         self.cache.reset()
         self.active.zero_()
         self.spec.zero_()
+        self.h_active.zero_()
+
+    def _fetch(self, with_decisions):
+        if with_decisions:
+            self.h_err.copy_(self.err, non_blocking=True)
+            self.h_accept.copy_(self.accept, non_blocking=True)
+        self.h_active.copy_(self.active, non_blocking=True)
+        self.torch.cuda.current_stream(self.cache.device).synchronize()
 
     def tau(self, tau0, beta, t, T):
         return self.S.speca_tau(tau0, beta, t, T)
@@ -139,15 +151,15 @@ class SpecaCacheBackend:
     def verify_and_select(self, fresh, t_target, tau, period):
         self.accept.zero_()
         self.cache.verify(fresh, t_target, tau, self.err, self.accept, self.active, metric=self.metric)
-        e = self.err.cpu().tolist()
-        acc = self.accept.cpu().tolist()
         self.cache.select_adaptive(self.accept, period, 1, self.spec, self.active, self.idx, self.n_active)
-        return e, acc
+        self._fetch(with_decisions=True)
+        return self.h_err.tolist(), self.h_accept.tolist()
 
     def active_mask(self):
-        return self.active.cpu().tolist()
+        return self.h_active.tolist()
 
     def reference_step(self, feats, t_ref, mask):
         self.cache.update(feats, t_ref, mask)
         self.cache.commit_step()
         self.cache.activate(mask, self.spec, self.active)
+        self._fetch(with_decisions=False)
