@@ -34,11 +34,11 @@ METRIC = "forecast+verify GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes per cached element per launch: (dram__bytes_read.sum + dram__bytes_write.sum) / elements
-# from the ncu captures summarised under profiles/ (taken on the DiT-XL/2-shaped cache, order 2,
-# bf16; traffic grows in proportion to the elements a launch covers). Set an entry to None when its
-# kernel changes until the counters have been taken again.
-NCU_DRAM_BYTES_PER_ELEM = {"update": 11.818, "forecast": 7.929, "verify": 8.012}
+# DRAM bytes per cached element per launch: (dram__bytes_read.sum + dram__bytes_write.sum) / elements,
+# from the one-pass ncu capture of this benchmark's default workload at full size (FLUX-shaped cache,
+# order 2, bf16; profiles/dram_traffic_flux_full_size.md). Other workloads scale by the elements a
+# launch covers. Set an entry to None when its kernel changes until the counters have been taken again.
+NCU_DRAM_BYTES_PER_ELEM = {"update": 11.987, "forecast": 8.036, "verify": 8.110}
 
 
 def measured_peak():
