@@ -69,21 +69,23 @@ def bits_to_tensor(a, tdt):
 
 
 FULL = [
-    ("dit_xl2", {}),
-    ("flux", {}),
-    ("hunyuan_video", {}),
-    ("flux_adaptive", {"max_order": 3}),
+    ("dit_xl2", {}, 0),
+    ("flux", {}, 0),
+    ("hunyuan_video", {}, 0),
+    ("flux_adaptive", {"max_order": 3}, 0),
+    ("flux", {}, 2),          # the TMA-staged kernels at full size
+    ("dit_xl2", {}, 1),       # the 16-byte register path at full size
 ]
 
 
-@pytest.mark.parametrize("name,kw", FULL)
-def test_full_size_config_on_sampled_blocks(S, U, name, kw):
+@pytest.mark.parametrize("name,kw,path", FULL)
+def test_full_size_config_on_sampled_blocks(S, U, name, kw, path):
     w = W.BY_NAME[name](**kw)
     B, m, ne = w.batch, w.max_order, len(w.entries)
     rng = np.random.default_rng(1234 + w.index)
     blocks = choose_blocks(w, rng)
     src = W.FeatureSource(w, DEV)
-    cache = S.SpecaCache(w.entries, B, m, w.dtype, DEV)
+    cache = S.SpecaCache(w.entries, B, m, w.dtype, DEV, path=path)
     tdt = w.torch_dtype
     orc = {(e, blk): np.zeros((m + 1, blk[2]), dtype=O.np_dtype(w.dtype)) for e, lst in blocks.items() for blk in lst}
     hist = []
