@@ -94,6 +94,12 @@ struct VerifyParams {
     float* partials;     // [n_clusters][B][values of the metric: 2, or 3 for cosine]
     uint32_t* ticket;    // arrival counter, zero between launches
     double* raw_sums;    // [B][4] or null: write the combined running values instead of err / accept
+    // fused per-sample continuation (speca_verify_select); sel_active == null: not fused
+    uint8_t* sel_active;  // receives the next active mask once every decision is final; must not alias dev_mask
+    int32_t* sel_spec;
+    int32_t* sel_idx;
+    int32_t* sel_n;
+    int32_t sel_kmax, sel_group;
     uint32_t n_elems;    // per sample
     uint32_t tiles_per_sample;
     uint32_t units_per_sample;  // ceil(tiles_per_sample / cluster size): host-side grid sizing only

@@ -1002,14 +1002,52 @@ __device__ __noinline__ void verify_tile_any(const char* __restrict__ plane0, ui
     }
 }
 
+// Per-sample continuation of the speculative run, for the first `batch` threads of a block (every
+// thread of the block must call it: it synchronises). keep / next: shared scratch of SPECA_MAX_BATCH bytes.
+// No __restrict__ here: the fused caller wrote `accept` earlier in the same kernel.
+__device__ __forceinline__ void select_in_block(const uint8_t* accept, int32_t k_max, int32_t group, int32_t batch,
+                                                int32_t* spec_count, const uint8_t* active_in, uint8_t* active_out,
+                                                int32_t* idx_out, int32_t* n_out, uint8_t* keep, uint8_t* next) {
+    const int b = threadIdx.x;
+    if (b < batch) {
+        const bool a = active_in[b] != 0;
+        const bool ok = a && accept[b] != 0;
+        int32_t c = spec_count[b];
+        if (ok) {
+            c += 1;
+            spec_count[b] = c;
+        }
+        keep[b] = (ok && c < k_max) ? 1 : 0;
+    }
+    __syncthreads();
+    if (b < batch) {
+        const int g0 = (b / group) * group;
+        uint8_t all = 1;
+        for (int i = 0; i < group; ++i) all &= keep[g0 + i];
+        next[b] = all;
+        active_out[b] = all;
+    }
+    __syncthreads();
+    if (b == 0) {
+        int32_t n = 0;
+        for (int i = 0; i < batch; ++i)
+            if (next[i]) {
+                if (idx_out != nullptr) idx_out[n] = i;
+                ++n;
+            }
+        if (n_out != nullptr) *n_out = n;
+    }
+}
+
 // Tiles of the active samples form one list of T = (active samples) x (tiles per sample) tiles;
 // cluster q of Q owns the contiguous range [q*T/Q, (q+1)*T/Q).
 __device__ __forceinline__ uint32_t range_begin(uint32_t q, uint32_t Q, uint32_t T) {
     return static_cast<uint32_t>(static_cast<uint64_t>(q) * T / Q);
 }
+// The cluster whose range holds `tile`: the smallest q with range_begin(q + 1) > tile, that is
+// ceil((tile + 1) * Q / T) - 1. Holds for Q > T too, where some clusters own nothing.
 __device__ __forceinline__ uint32_t range_owner(uint32_t tile, uint32_t Q, uint32_t T) {
-    const uint32_t q0 = static_cast<uint32_t>(static_cast<uint64_t>(tile) * Q / T);
-    return tile < range_begin(q0 + 1, Q, T) ? q0 : q0 + 1;
+    return static_cast<uint32_t>(((static_cast<uint64_t>(tile) + 1) * Q - 1) / T);
 }
 // Index of the a-th set bit of `bits` (a < popcount).
 __device__ __forceinline__ int nth_set_bit(uint64_t bits, uint32_t a) {
@@ -1038,6 +1076,7 @@ __global__ void __launch_bounds__(kThreads, 2) verify_kernel(const __grid_consta
     __shared__ float cluster_slot[2][NA][kMaxClusterSize];  // [parity][value][rank], leader's copy is used
     __shared__ uint32_t active_bits[2];
     __shared__ bool is_last;
+    __shared__ uint8_t sel_keep[SPECA_MAX_BATCH], sel_next[SPECA_MAX_BATCH];
 
     // samples that take part: a defined table and, with a device mask, a non-zero byte
     if (threadIdx.x < 64) {
@@ -1049,7 +1088,12 @@ __global__ void __launch_bounds__(kThreads, 2) verify_kernel(const __grid_consta
     __syncthreads();
     const uint64_t bits = static_cast<uint64_t>(active_bits[0]) | (static_cast<uint64_t>(active_bits[1]) << 32);
     const uint32_t n_active = __popcll(bits);
-    if (n_active == 0) return;  // every CTA of the grid takes this exit together
+    if (n_active == 0) {  // every CTA of the grid takes this exit together
+        if (p.sel_active != nullptr && blockIdx.x == 0)
+            select_in_block(p.accept, p.sel_kmax, p.sel_group, p.batch, p.sel_spec, p.dev_mask, p.sel_active, p.sel_idx,
+                            p.sel_n, sel_keep, sel_next);
+        return;
+    }
     const uint32_t tps = p.tiles_per_sample;
     const uint32_t T = n_active * tps;
 
@@ -1136,6 +1180,7 @@ __global__ void __launch_bounds__(kThreads, 2) verify_kernel(const __grid_consta
         const uint32_t q_lo = range_owner(a * tps, Q, T), q_hi = range_owner((a + 1) * tps - 1, Q, T);
         double s[3] = {0.0, 0.0, 0.0};
         for (uint32_t q = q_lo + lane; q <= q_hi; q += 32) {
+            if (range_begin(q, Q, T) == range_begin(q + 1, Q, T)) continue;  // owns no tile (Q > T): wrote nothing
             const float* src = p.partials + (static_cast<size_t>(q) * p.batch + b) * NA;
 #pragma unroll
             for (int i = 0; i < NA; ++i) s[i] = Metric<M>::merge(s[i], static_cast<double>(__ldcg(src + i)));
@@ -1159,6 +1204,11 @@ __global__ void __launch_bounds__(kThreads, 2) verify_kernel(const __grid_consta
         }
     }
     __syncthreads();
+    // Fused continuation: every decision of this step is final by now. The new mask goes to a buffer
+    // of its own: CTAs of this grid may still be reading the step's mask.
+    if (p.sel_active != nullptr)
+        select_in_block(p.accept, p.sel_kmax, p.sel_group, p.batch, p.sel_spec, p.dev_mask, p.sel_active, p.sel_idx, p.sel_n,
+                        sel_keep, sel_next);
     if (threadIdx.x == 0) *p.ticket = 0;  // ready for the next launch on this stream
 }
 
@@ -1205,35 +1255,7 @@ __global__ void __launch_bounds__(SPECA_MAX_BATCH) select_kernel(const uint8_t* 
                                                                   int32_t* __restrict__ n_out) {
     __shared__ uint8_t keep[SPECA_MAX_BATCH];
     __shared__ uint8_t next[SPECA_MAX_BATCH];
-    const int b = threadIdx.x;
-    if (b < batch) {
-        const bool a = active[b] != 0;
-        const bool ok = a && accept[b] != 0;
-        int32_t c = spec_count[b];
-        if (ok) {
-            c += 1;
-            spec_count[b] = c;
-        }
-        keep[b] = (ok && c < k_max) ? 1 : 0;
-    }
-    __syncthreads();
-    if (b < batch) {
-        const int g0 = (b / group) * group;
-        uint8_t all = 1;
-        for (int i = 0; i < group; ++i) all &= keep[g0 + i];
-        next[b] = all;
-        active[b] = all;
-    }
-    __syncthreads();
-    if (b == 0) {
-        int32_t n = 0;
-        for (int i = 0; i < batch; ++i)
-            if (next[i]) {
-                if (idx_out != nullptr) idx_out[n] = i;
-                ++n;
-            }
-        if (n_out != nullptr) *n_out = n;
-    }
+    select_in_block(accept, k_max, group, batch, spec_count, active, active, idx_out, n_out, keep, next);
 }
 
 __global__ void __launch_bounds__(SPECA_MAX_BATCH) activate_kernel(uint64_t mask_bits, int32_t batch,

@@ -166,6 +166,30 @@ def test_masks_leave_other_samples_untouched(S, U, dtype):
     pair.close()
 
 
+@pytest.mark.parametrize("entry", [(17, 130), (40, 1030), (301, 1160)])   # 1, 3 and 22 tiles per sample
+def test_verify_with_any_number_of_active_samples(S, U, entry):
+    """The grid is sized for the whole batch, so with few active samples there are more clusters than
+    tiles and some clusters own nothing; every ratio of clusters to tiles must find its partials."""
+    entries = [(2, 8), entry]
+    B, m = 64, 1
+    gen = torch.Generator(device=DEV).manual_seed(911)
+    rng = np.random.default_rng(12)
+    pair = U.Pair(entries, B, m, 1)
+    for t in (1.0, 0.9):
+        pair.update(rand_feats(entries, B, pair.tdt, gen), [t] * B)
+        pair.commit()
+    pair.sync_tables()
+    fresh = rand_feats([entry], B, pair.tdt, gen)[0]
+    for n_on in (1, 2, 3, 5, 7, 11, 15, 23, 30, 31, 33, 47, 63, 64):
+        act = [0] * B
+        for b in rng.choice(B, n_on, replace=False):
+            act[int(b)] = 1
+        e, a, ew, aw = pair.check_verify(fresh, [0.85] * B, [1.0] * B, active=act, with_pred=(n_on % 2 == 0),
+                                         what="%d of %d active" % (n_on, B))
+        assert all(e[b] > 0.1 for b in range(B) if act[b])
+    pair.close()
+
+
 # ---------------------------------------------------------------------------------------------
 # degenerate inputs
 # ---------------------------------------------------------------------------------------------
