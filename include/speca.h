@@ -291,6 +291,22 @@ speca_status_t speca_select_adaptive(speca_cache_t* cache, const uint8_t* dev_ac
                                      int32_t group, int32_t* dev_spec_count, uint8_t* dev_active_mask,
                                      int32_t* dev_active_idx, int32_t* dev_n_active, void* stream);
 
+/*
+ * speca_verify_metric followed by speca_select_adaptive in one launch: the cluster that finishes the
+ * reduction also applies the continuation rule, once every sample's decision is final. Same results
+ * as the two calls; saves a kernel launch per speculative step.
+ *   dev_active_mask       device, B bytes, required: this step's mask (read only).
+ *   dev_next_active_mask  device, B bytes, must not overlap dev_active_mask: receives the mask of the
+ *                         next step (other thread blocks may still be reading this step's mask when
+ *                         it is written, hence two buffers; a caller alternates between them).
+ * The other arguments are those of the two calls. If no sample is active, the next mask is all zero
+ * and *dev_n_active = 0. Errors: those of the two calls, INVALID_ARG for overlapping masks.
+ */
+speca_status_t speca_verify_select(speca_cache_t* cache, int32_t metric, const void* fresh, const double* t_target,
+                                   const float* tau, const uint8_t* dev_active_mask, uint8_t* dev_next_active_mask,
+                                   void* out_pred, float* dev_err, uint8_t* dev_accept, int32_t k_max, int32_t group,
+                                   int32_t* dev_spec_count, int32_t* dev_active_idx, int32_t* dev_n_active, void* stream);
+
 /* After a reference step: mark the samples with host_sample_mask[b] != 0 (NULL = all) active again
  * and clear their speculative-step counters, on the stream. Errors: INVALID_ARG, CUDA. */
 speca_status_t speca_activate(speca_cache_t* cache, const uint8_t* host_sample_mask, int32_t* dev_spec_count,

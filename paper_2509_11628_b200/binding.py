@@ -32,7 +32,7 @@ EXPORTS = [
     "speca_cache_launch_count", "speca_status_string", "speca_last_error", "speca_version",
     "speca_verify_pred_static", "speca_forecast_multi", "speca_verify_metric",
     "speca_verify_partial", "speca_verify_decide", "speca_cache_get_history", "speca_cache_set_history",
-    "speca_forecast_sum",
+    "speca_forecast_sum", "speca_verify_select",
 ]
 
 
@@ -81,6 +81,7 @@ def _lib() -> ctypes.CDLL:
     L.speca_forecast_multi.argtypes = [vp, i32, vp, vp, vp, vp]
     L.speca_verify.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.speca_verify_metric.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.speca_verify_select.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
     L.speca_verify_partial.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
     L.speca_verify_decide.argtypes = [i32, vp, i32, vp, ctypes.c_float, vp, vp, vp, vp]
     L.speca_select_adaptive.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, vp]
@@ -235,6 +236,16 @@ def speca_verify_metric(cache, metric, fresh, t_target, tau, dev_active_mask, ou
                                       _dev_ptr(dev_accept), _stream_ptr(stream)), cache)
 
 
+def speca_verify_select(cache, metric, fresh, t_target, tau, dev_active_mask, dev_next_active_mask, out_pred, dev_err,
+                        dev_accept, k_max, group, dev_spec_count, dev_active_idx=None, dev_n_active=None, stream=None) -> None:
+    """speca_verify_metric + speca_select_adaptive in one launch; the next mask goes to its own buffer."""
+    _check(_lib().speca_verify_select(cache, int(metric), _dev_ptr(fresh), _doubles(t_target), _floats(tau),
+                                      _dev_ptr(dev_active_mask), _dev_ptr(dev_next_active_mask), _dev_ptr(out_pred),
+                                      _dev_ptr(dev_err), _dev_ptr(dev_accept), int(k_max), int(group),
+                                      _dev_ptr(dev_spec_count), _dev_ptr(dev_active_idx), _dev_ptr(dev_n_active),
+                                      _stream_ptr(stream)), cache)
+
+
 def speca_verify_partial(cache, metric, fresh, t_target, dev_active_mask, out_pred, dev_sums, stream=None) -> None:
     """``dev_sums``: CUDA float64 tensor [B, 4] that receives the metric's running values of this shard."""
     _check(_lib().speca_verify_partial(cache, int(metric), _dev_ptr(fresh), _doubles(t_target), _dev_ptr(dev_active_mask),
@@ -367,6 +378,11 @@ class SpecaCache:
             speca_verify(self.handle, fresh, t_target, tau, active, out_pred, err, accept, stream)
         else:
             speca_verify_metric(self.handle, metric, fresh, t_target, tau, active, out_pred, err, accept, stream)
+
+    def verify_select(self, fresh, t_target, tau, err, accept, active, next_active, k_max, group, spec_count, idx=None,
+                      n_active=None, out_pred=None, stream=None, metric=0):
+        speca_verify_select(self.handle, metric, fresh, t_target, tau, active, next_active, out_pred, err, accept, k_max,
+                            group, spec_count, idx, n_active, stream)
 
     def select_adaptive(self, accept, k_max, group, spec_count, active, idx=None, n_active=None, stream=None):
         speca_select_adaptive(self.handle, accept, k_max, group, spec_count, active, idx, n_active, stream)

@@ -582,9 +582,17 @@ speca_status_t speca_verify(speca_cache_t* c, const void* fresh, const double* t
 }
 
 // speca_verify_metric (dev_sums == nullptr) and speca_verify_partial (dev_sums given, no tau / err / accept).
+struct SelectArgs {
+    int32_t k_max, group;
+    int32_t* spec_count;
+    uint8_t* active;
+    int32_t* idx;
+    int32_t* n_active;
+};
+
 static speca_status_t verify_impl(speca_cache_t* c, int32_t metric, const void* fresh, const double* t_target,
                                   const float* tau, const uint8_t* dev_active_mask, void* out_pred, float* dev_err,
-                                  uint8_t* dev_accept, double* dev_sums, void* stream) {
+                                  uint8_t* dev_accept, double* dev_sums, void* stream, const SelectArgs* sel = nullptr) {
     if (c == nullptr) return SPECA_ERR_INVALID_ARG;
     if (metric < SPECA_METRIC_L2 || metric > SPECA_METRIC_COSINE)
         return fail(c, SPECA_ERR_INVALID_ARG, "verify: unknown metric %d", metric);
@@ -619,7 +627,9 @@ static speca_status_t verify_impl(speca_cache_t* c, int32_t metric, const void* 
     if (!guard.ok) return fail(c, SPECA_ERR_CUDA, "cudaSetDevice failed");
     speca_status_t st = check_sticky(c);
     if (st != SPECA_OK) return st;
-    if (!any_sample) return SPECA_OK;
+    // No sample has a table: nothing to verify. The fused form still launches, so that the kernel's
+    // early exit writes the next mask.
+    if (!any_sample && sel == nullptr) return SPECA_OK;
     const Layout& L = c->L;
     const SegDesc& s0 = L.segs[static_cast<size_t>(c->verify_entry) * c->B];
     const uint32_t te = verify_tile_elems(c->dtype, v_max);
@@ -633,6 +643,14 @@ static speca_status_t verify_impl(speca_cache_t* c, int32_t metric, const void* 
     p.partials = reinterpret_cast<float*>(c->arena + L.partials_off);
     p.ticket = reinterpret_cast<uint32_t*>(c->arena + L.ticket_off);
     p.raw_sums = dev_sums;
+    if (sel != nullptr) {
+        p.sel_active = sel->active;
+        p.sel_spec = sel->spec_count;
+        p.sel_idx = sel->idx;
+        p.sel_n = sel->n_active;
+        p.sel_kmax = sel->k_max;
+        p.sel_group = sel->group;
+    }
     p.n_elems = s0.n_elems;
     p.tiles_per_sample = (s0.n_elems + te - 1) / te;
     p.units_per_sample = (p.tiles_per_sample + c->cluster - 1) / c->cluster;
@@ -652,6 +670,25 @@ speca_status_t speca_verify_metric(speca_cache_t* c, int32_t metric, const void*
                                    const float* tau, const uint8_t* dev_active_mask, void* out_pred, float* dev_err,
                                    uint8_t* dev_accept, void* stream) {
     return verify_impl(c, metric, fresh, t_target, tau, dev_active_mask, out_pred, dev_err, dev_accept, nullptr, stream);
+}
+
+speca_status_t speca_verify_select(speca_cache_t* c, int32_t metric, const void* fresh, const double* t_target,
+                                   const float* tau, const uint8_t* dev_active_mask, uint8_t* dev_next_active_mask,
+                                   void* out_pred, float* dev_err, uint8_t* dev_accept, int32_t k_max, int32_t group,
+                                   int32_t* dev_spec_count, int32_t* dev_active_idx, int32_t* dev_n_active, void* stream) {
+    if (c == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (dev_active_mask == nullptr || dev_next_active_mask == nullptr || dev_spec_count == nullptr)
+        return fail(c, SPECA_ERR_INVALID_ARG, "verify_select: null argument");
+    const uintptr_t a = reinterpret_cast<uintptr_t>(dev_active_mask), b = reinterpret_cast<uintptr_t>(dev_next_active_mask);
+    if (a < b + static_cast<uintptr_t>(c->B) && b < a + static_cast<uintptr_t>(c->B))
+        return fail(c, SPECA_ERR_INVALID_ARG, "verify_select: the next mask must not overlap this step's mask");
+    if (k_max < 1 || group < 1 || c->B % group != 0)
+        return fail(c, SPECA_ERR_INVALID_ARG, "verify_select: k_max >= 1 and group must divide the batch");
+    if (reinterpret_cast<uintptr_t>(dev_spec_count) % 4 != 0 || reinterpret_cast<uintptr_t>(dev_active_idx) % 4 != 0 ||
+        reinterpret_cast<uintptr_t>(dev_n_active) % 4 != 0)
+        return fail(c, SPECA_ERR_ALIGNMENT, "verify_select: int32 buffers must be 4-byte aligned");
+    const SelectArgs sel = {k_max, group, dev_spec_count, dev_next_active_mask, dev_active_idx, dev_n_active};
+    return verify_impl(c, metric, fresh, t_target, tau, dev_active_mask, out_pred, dev_err, dev_accept, nullptr, stream, &sel);
 }
 
 speca_status_t speca_verify_partial(speca_cache_t* c, int32_t metric, const void* fresh, const double* t_target,

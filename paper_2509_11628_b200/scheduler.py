@@ -121,6 +121,7 @@ class SpecaCacheBackend:
         self.err = torch.zeros(self.batch, dtype=torch.float32, device=dev)
         self.accept = torch.zeros(self.batch, dtype=torch.uint8, device=dev)
         self.active = torch.zeros(self.batch, dtype=torch.uint8, device=dev)
+        self.active_next = torch.zeros(self.batch, dtype=torch.uint8, device=dev)   # the fused call's output mask
         self.spec = torch.zeros(self.batch, dtype=torch.int32, device=dev)
         self.idx = torch.zeros(self.batch, dtype=torch.int32, device=dev)
         self.n_active = torch.zeros(1, dtype=torch.int32, device=dev)
@@ -150,8 +151,10 @@ class SpecaCacheBackend:
 
     def verify_and_select(self, fresh, t_target, tau, period):
         self.accept.zero_()
-        self.cache.verify(fresh, t_target, tau, self.err, self.accept, self.active, metric=self.metric)
-        self.cache.select_adaptive(self.accept, period, 1, self.spec, self.active, self.idx, self.n_active)
+        # Eq. 4 and the continuation rule in one launch; the next mask arrives in the other buffer
+        self.cache.verify_select(fresh, t_target, tau, self.err, self.accept, self.active, self.active_next, period, 1,
+                                 self.spec, self.idx, self.n_active, metric=self.metric or 0)
+        self.active, self.active_next = self.active_next, self.active
         self._fetch(with_decisions=True)
         return self.h_err.tolist(), self.h_accept.tolist()
 

@@ -1,0 +1,152 @@
+"""speca_verify_select (verification and the per-sample continuation rule in one launch) against the
+two separate calls on the same inputs -- bit for bit -- and against the oracle's decisions."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import speca_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def S():
+    from paper_2509_11628_b200 import binding
+    binding._lib()
+    return binding
+
+
+@pytest.fixture(scope="module")
+def U():
+    from tests import gpu_util
+    return gpu_util
+
+
+def rand_feats(entries, B, tdt, gen):
+    return [torch.randn(B, n, d, generator=gen, device=DEV, dtype=torch.float32).to(tdt) for n, d in entries]
+
+
+def both_ways(pair, fresh, t, tau, act, cnt, k_max, group, metric=0):
+    """Runs verify + select, then the fused call, from the same state. Returns both result sets."""
+    B = pair.B
+    n, d = pair.entries[pair.vidx]
+    dev = lambda x, dt: torch.tensor(x, dtype=dt, device=DEV)
+    # two calls
+    err_a = torch.full((B,), -7.0, device=DEV)
+    acc_a = torch.zeros(B, dtype=torch.uint8, device=DEV)
+    act_a, cnt_a = dev(act, torch.uint8), dev(cnt, torch.int32)
+    idx_a, n_a = torch.full((B,), -1, dtype=torch.int32, device=DEV), torch.full((1,), -1, dtype=torch.int32, device=DEV)
+    pred_a = torch.zeros(B, n, d, dtype=pair.tdt, device=DEV)
+    pair.gpu.verify(fresh, t, tau, err_a, acc_a, act_a, pred_a, metric=metric)
+    pair.gpu.select_adaptive(acc_a, k_max, group, cnt_a, act_a, idx_a, n_a)
+    # one call
+    err_b = torch.full((B,), -7.0, device=DEV)
+    acc_b = torch.zeros(B, dtype=torch.uint8, device=DEV)
+    act_b, cnt_b = dev(act, torch.uint8), dev(cnt, torch.int32)
+    nxt_b = torch.full((B,), 5, dtype=torch.uint8, device=DEV)
+    idx_b, n_b = torch.full((B,), -1, dtype=torch.int32, device=DEV), torch.full((1,), -1, dtype=torch.int32, device=DEV)
+    pred_b = torch.zeros(B, n, d, dtype=pair.tdt, device=DEV)
+    launches = pair.gpu.launches
+    pair.gpu.verify_select(fresh, t, tau, err_b, acc_b, act_b, nxt_b, k_max, group, cnt_b, idx_b, n_b, pred_b, metric=metric)
+    assert pair.gpu.launches == launches + 1
+    torch.cuda.synchronize()
+    assert act_b.cpu().tolist() == act, "the step's own mask must stay as it was"
+    two = dict(err=err_a.cpu().numpy(), acc=acc_a.cpu().tolist(), act=act_a.cpu().tolist(), cnt=cnt_a.cpu().tolist(),
+               n=n_a.item(), idx=idx_a.cpu().tolist(), pred=pred_a)
+    one = dict(err=err_b.cpu().numpy(), acc=acc_b.cpu().tolist(), act=nxt_b.cpu().tolist(), cnt=cnt_b.cpu().tolist(),
+               n=n_b.item(), idx=idx_b.cpu().tolist(), pred=pred_b)
+    return two, one
+
+
+def assert_same(two, one):
+    assert np.array_equal(two["err"].view(np.uint32), one["err"].view(np.uint32))
+    assert two["acc"] == one["acc"] and two["act"] == one["act"] and two["cnt"] == one["cnt"]
+    assert two["n"] == one["n"] and two["idx"][: two["n"]] == one["idx"][: one["n"]]
+    assert torch.equal(two["pred"].view(torch.uint8), one["pred"].view(torch.uint8))
+
+
+@pytest.mark.parametrize("metric", [O.METRIC_L2, O.METRIC_LINF])
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("B,group,entry", [(8, 1, (301, 1160)), (8, 2, (301, 1160)), (6, 3, (5, 24)), (64, 8, (17, 130)),
+                                           (1, 1, (2050, 1152))])
+def test_fused_call_equals_the_two_calls_and_the_oracle(S, U, metric, dtype, B, group, entry):
+    entries = [(3, 16), entry]
+    m = 2
+    gen = torch.Generator(device=DEV).manual_seed(4100 + B + group + metric)
+    rng = np.random.default_rng(B * 7 + group)
+    pair = U.Pair(entries, B, m, dtype)
+    for t in (1.0, 0.93, 0.9):
+        pair.update(rand_feats(entries, B, pair.tdt, gen), [t] * B)
+        pair.commit()
+        pair.sync_tables()
+    t = [0.86] * B
+    outs = pair.check_forecast(t)
+    level = torch.tensor(rng.choice([0.0, 0.01, 0.05, 0.3], B), device=DEV, dtype=torch.float32).view(B, 1, 1)
+    fresh = (outs[1].float() + level * torch.randn(B, *entry, generator=gen, device=DEV)).to(pair.tdt)
+    tau = [0.03] * B
+    for trial in range(3):
+        act = rng.integers(0, 2, B).tolist() if trial else [1] * B
+        cnt = rng.integers(0, 4, B).tolist()
+        k_max = int(rng.integers(1, 6))
+        two, one = both_ways(pair, fresh, t, tau, act, cnt, k_max, group, metric)
+        assert_same(two, one)
+        # and the decisions the oracle takes (skipping samples within tolerance of the threshold)
+        e_want, a_want, _ = pair.cpu.verify(U.to_oracle(fresh).reshape(B, -1), t, tau, act, metric=metric)
+        near = [a_want[b] >= 0 and abs(e_want[b] - float(np.float32(tau[b]))) < 1e-3 for b in range(B)]
+        if not any(near):
+            want_act, want_cnt, want_idx = O.select_adaptive([max(int(a), 0) for a in a_want], k_max, group, cnt, act)
+            assert one["act"] == want_act and one["cnt"] == want_cnt
+            assert one["n"] == len(want_idx) and one["idx"][: one["n"]] == want_idx
+    pair.close()
+
+
+def test_nobody_active_and_nobody_with_a_table(S, U):
+    entries = [(4, 32), (40, 256)]
+    B = 4
+    gen = torch.Generator(device=DEV).manual_seed(5)
+    pair = U.Pair(entries, B, 1, 1)
+    fresh = rand_feats(entries, B, pair.tdt, gen)[1]
+    # no reference step yet: nothing is verified, the continuation rule still runs on what it is given
+    two, one = both_ways(pair, fresh, [0.9] * B, [0.5] * B, [1, 0, 1, 0], [0, 1, 2, 3], 4, 1)
+    assert_same(two, one)
+    assert one["act"] == [0, 0, 0, 0] and one["n"] == 0 and (one["err"] == -7.0).all()
+    pair.update(rand_feats(entries, B, pair.tdt, gen), [1.0] * B)
+    pair.commit()
+    # tables exist, nobody active
+    two, one = both_ways(pair, fresh, [0.9] * B, [0.5] * B, [0] * B, [1] * B, 4, 2)
+    assert_same(two, one)
+    assert one["act"] == [0] * B and one["n"] == 0 and one["cnt"] == [1] * B and (one["err"] == -7.0).all()
+    pair.close()
+
+
+def test_argument_errors(S):
+    B = 4
+    c = S.SpecaCache([(8, 64)], B, 1, 1, DEV)
+    f = torch.zeros(B, 8, 64, dtype=torch.bfloat16, device=DEV)
+    c.update([f], [1.0] * B)
+    c.commit_step()
+    err, acc = torch.zeros(B, device=DEV), torch.zeros(B, dtype=torch.uint8, device=DEV)
+    masks = torch.ones(2 * B, dtype=torch.uint8, device=DEV)
+    cnt = torch.zeros(B, dtype=torch.int32, device=DEV)
+    launches = c.launches
+
+    def status_of(fn):
+        with pytest.raises(S.SpecaError) as ei:
+            fn()
+        return ei.value.status
+
+    t, tau = [0.9] * B, [0.1] * B
+    assert status_of(lambda: c.verify_select(f, t, tau, err, acc, masks[:B], masks[:B], 2, 1, cnt)) == S.SPECA_ERR_INVALID_ARG
+    assert status_of(lambda: c.verify_select(f, t, tau, err, acc, masks[:B], masks[2:2 + B], 2, 1, cnt)) == S.SPECA_ERR_INVALID_ARG
+    assert "overlap" in S.speca_last_error(c.handle)
+    assert status_of(lambda: c.verify_select(f, t, tau, err, acc, None, masks[B:], 2, 1, cnt)) == S.SPECA_ERR_INVALID_ARG
+    assert status_of(lambda: c.verify_select(f, t, tau, err, acc, masks[:B], masks[B:], 0, 1, cnt)) == S.SPECA_ERR_INVALID_ARG
+    assert status_of(lambda: c.verify_select(f, t, tau, err, acc, masks[:B], masks[B:], 2, 3, cnt)) == S.SPECA_ERR_INVALID_ARG
+    assert status_of(lambda: c.verify_select(f, t, tau, err, acc, masks[:B], masks[B:], 2, 1, None)) == S.SPECA_ERR_INVALID_ARG
+    assert c.launches == launches
+    c.verify_select(f, t, tau, err, acc, masks[:B], masks[B:], 2, 1, cnt)   # adjacent buffers are fine
+    torch.cuda.synchronize()
+    assert acc.cpu().tolist() == [1] * B and masks[B:].cpu().tolist() == [1] * B and cnt.cpu().tolist() == [1] * B
+    c.close()
