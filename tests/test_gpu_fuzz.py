@@ -1,0 +1,117 @@
+"""Seeded random scenarios: random shapes, batch sizes, orders, bases, storage types and kernel paths,
+and a random sequence of masked reference steps, speculative steps (forecast, verify under a random
+metric, the fused verify + continuation call) and resets -- every result compared with the oracle.
+The hand-written cases elsewhere pick the shapes someone thought of; this file picks the others."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import speca_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+MAX_ELEMS = 3_000_000   # per scenario, over all entries and samples: keeps the oracle in the seconds
+
+
+@pytest.fixture(scope="module")
+def S():
+    from paper_2509_11628_b200 import binding
+    binding._lib()
+    return binding
+
+
+@pytest.fixture(scope="module")
+def U():
+    from tests import gpu_util
+    return gpu_util
+
+
+def draw_shape(rng):
+    B = int(rng.choice([1, 2, 3, 5, 8, 16, 33, 64]))
+    n_entries = int(rng.integers(1, 6))
+    budget = MAX_ELEMS // B
+    entries = []
+    for _ in range(n_entries):
+        kind = rng.integers(0, 4)
+        if kind == 0:      # a handful of elements
+            n, d = int(rng.integers(1, 6)), int(rng.integers(1, 40))
+        elif kind == 1:    # odd row length, around one tile
+            n, d = int(rng.integers(1, 40)), int(rng.integers(100, 1400))
+        elif kind == 2:    # model-like width, several tiles
+            n, d = int(rng.integers(20, 400)), int(rng.choice([1152, 3072, 768]))
+        else:              # one long row
+            n, d = 1, int(rng.integers(8000, 70000))
+        while n * d > budget // n_entries and n > 1:
+            n = max(1, n // 2)
+        if n * d > budget // n_entries:
+            d = max(1, budget // n_entries)
+        entries.append((n, d))
+    return B, entries
+
+
+@pytest.mark.parametrize("seed", list(range(64)))
+def test_random_scenario(S, U, seed):
+    rng = np.random.default_rng(90_000 + seed)
+    gen = torch.Generator(device=DEV).manual_seed(90_000 + seed)
+    B, entries = draw_shape(rng)
+    m = int(rng.integers(0, 5))
+    dtype = int(rng.integers(0, 2))
+    basis = int(rng.integers(0, 3))
+    path = int(rng.integers(0, 4))
+    vidx = int(rng.integers(-1, len(entries)))
+    pair = U.Pair(entries, B, m, dtype, basis, verify_entry=vidx, path=path)
+    nv, dv = entries[pair.vidx]
+    what = "seed %d (B=%d m=%d dtype=%d basis=%d path=%d entries=%s)" % (seed, B, m, dtype, basis, path, entries)
+
+    def feats():
+        return [torch.randn(B, n, d, generator=gen, device=DEV, dtype=torch.float32).to(pair.tdt) for n, d in entries]
+
+    clock = 1.0
+    cnt = [0] * B
+    for step in range(int(rng.integers(m + 2, m + 7))):
+        have = [int(r >= 1) for r in pair.cpu.n_refs]
+        kind = "ref" if step == 0 or not any(have) else rng.choice(["ref", "spec", "spec", "reset"], p=[0.4, 0.3, 0.2, 0.1])
+        clock -= float(rng.uniform(0.012, 0.06))
+        jitter = rng.uniform(-0.004, 0.004, B)
+        t = [clock + float(j) for j in jitter]
+        if kind == "ref":
+            mask = None if rng.random() < 0.4 else rng.integers(0, 2, B).tolist()
+            if mask is not None and not any(mask):
+                mask[int(rng.integers(0, B))] = 1
+            pair.update(feats(), t, mask, per_entry_calls=bool(rng.integers(0, 2)))
+            pair.commit()
+            pair.check_tables(what + " step %d tables" % step)
+            pair.sync_tables()
+        elif kind == "reset":
+            mask = rng.integers(0, 2, B).tolist()
+            pair.gpu.reset(mask)
+            pair.cpu.reset(mask)
+        else:
+            act = [h & int(a) for h, a in zip(have, rng.integers(0, 2, B).tolist())]
+            if rng.random() < 0.3:
+                act = list(have)
+            outs = pair.check_forecast(t, active=act, sentinel=2.5, what=what + " step %d forecast" % step)
+            level = torch.tensor(rng.choice([0.0, 0.02, 0.3], B), device=DEV, dtype=torch.float32).view(B, 1, 1)
+            fresh = (outs[pair.vidx].float() + level * torch.randn(B, nv, dv, generator=gen, device=DEV)).to(pair.tdt)
+            metric = int(rng.integers(0, 4))
+            tau = [1e-3 if metric == O.METRIC_COSINE else 0.05] * B
+            pair.check_verify(fresh, t, tau, active=act, with_pred=bool(rng.integers(0, 2)), metric=metric,
+                              ulp_slack=(metric == O.METRIC_LINF), what=what + " step %d verify metric %d" % (step, metric))
+            # the fused call against the two calls, from the same state
+            k_max, group = int(rng.integers(1, 5)), int(rng.choice([g for g in (1, 2, 4) if B % g == 0]))
+            err2, acc2 = torch.zeros(B, device=DEV), torch.zeros(B, dtype=torch.uint8, device=DEV)
+            err1, acc1 = torch.zeros(B, device=DEV), torch.zeros(B, dtype=torch.uint8, device=DEV)
+            m2, m1 = torch.tensor(act, dtype=torch.uint8, device=DEV), torch.tensor(act, dtype=torch.uint8, device=DEV)
+            c2, c1 = torch.tensor(cnt, dtype=torch.int32, device=DEV), torch.tensor(cnt, dtype=torch.int32, device=DEV)
+            nxt = torch.zeros(B, dtype=torch.uint8, device=DEV)
+            pair.gpu.verify(fresh, t, tau, err2, acc2, m2, metric=metric)
+            pair.gpu.select_adaptive(acc2, k_max, group, c2, m2)
+            pair.gpu.verify_select(fresh, t, tau, err1, acc1, m1, nxt, k_max, group, c1, metric=metric)
+            torch.cuda.synchronize()
+            assert torch.equal(err1.view(torch.int32), err2.view(torch.int32)) and torch.equal(acc1, acc2), what
+            assert torch.equal(nxt, m2) and torch.equal(c1, c2), what
+            want_act, want_cnt, _ = O.select_adaptive(acc2.cpu().tolist(), k_max, group, cnt, act)
+            assert nxt.cpu().tolist() == want_act and c1.cpu().tolist() == want_cnt, what
+            cnt = want_cnt
+    pair.close()
