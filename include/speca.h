@@ -377,6 +377,23 @@ speca_status_t speca_cache_set_history(speca_cache_t* cache, const int32_t* host
 speca_status_t speca_cache_plane(const speca_cache_t* cache, int32_t entry, int32_t sample, void** plane0,
                                  size_t* plane_stride_bytes);
 
+/*
+ * Host-side counters of a handle since it was created (nothing here is read back from the device, so
+ * the call neither launches nor synchronises). Launch counts are per kernel kind; the fused
+ * verify + continuation call counts as one verify launch. reference_steps[b] counts committed
+ * reference steps of sample b (it does not go back to zero on a reset, unlike the history length
+ * that speca_cache_state reports); resets[b] counts how often sample b's history was cleared.
+ * Entries at and beyond the batch size are zero. reference_steps is the number of full passes each
+ * sample of a batch needed: the quantity that sample-adaptive computation allocation varies.
+ */
+typedef struct {
+    uint64_t update_launches, forecast_launches, forecast_multi_launches, forecast_sum_launches;
+    uint64_t verify_launches, select_launches, activate_launches;
+    uint64_t reference_steps[SPECA_MAX_BATCH];
+    uint64_t resets[SPECA_MAX_BATCH];
+} speca_cache_stats_t;
+speca_status_t speca_cache_stats(const speca_cache_t* cache, speca_cache_stats_t* out);
+
 /* How many kernels the handle has launched since it was created. */
 speca_status_t speca_cache_launch_count(const speca_cache_t* cache, uint64_t* out);
 

@@ -29,7 +29,7 @@ EXPORTS = [
     "speca_cache_arena_bytes", "speca_cache_create", "speca_cache_destroy", "speca_cache_reset",
     "speca_cache_update", "speca_cache_commit_step", "speca_forecast", "speca_verify",
     "speca_select_adaptive", "speca_activate", "speca_tau", "speca_cache_state", "speca_cache_plane",
-    "speca_cache_launch_count", "speca_status_string", "speca_last_error", "speca_version",
+    "speca_cache_launch_count", "speca_cache_stats", "speca_status_string", "speca_last_error", "speca_version",
     "speca_verify_pred_static", "speca_forecast_multi", "speca_verify_metric",
     "speca_verify_partial", "speca_verify_decide", "speca_cache_get_history", "speca_cache_set_history",
     "speca_forecast_sum", "speca_verify_select",
@@ -45,6 +45,13 @@ class SpecaError(RuntimeError):
 
 class EntryDesc(ctypes.Structure):
     _fields_ = [("tokens", ctypes.c_int64), ("dim", ctypes.c_int32)]
+
+
+class CacheStats(ctypes.Structure):
+    _fields_ = [(name, ctypes.c_uint64) for name in (
+        "update_launches", "forecast_launches", "forecast_multi_launches", "forecast_sum_launches",
+        "verify_launches", "select_launches", "activate_launches")] + [
+        ("reference_steps", ctypes.c_uint64 * 64), ("resets", ctypes.c_uint64 * 64)]
 
 
 class CacheConfig(ctypes.Structure):
@@ -94,6 +101,7 @@ def _lib() -> ctypes.CDLL:
     L.speca_cache_set_history.argtypes = [vp, vp, vp]
     L.speca_cache_plane.argtypes = [vp, i32, i32, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_size_t)]
     L.speca_cache_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64)]
+    L.speca_cache_stats.argtypes = [vp, ctypes.POINTER(CacheStats)]
     L.speca_status_string.argtypes = [i32]
     L.speca_status_string.restype = ctypes.c_char_p
     L.speca_last_error.argtypes = [vp]
@@ -314,6 +322,16 @@ def speca_cache_plane(cache, entry: int, sample: int):
     return p.value, s.value
 
 
+def speca_cache_stats(cache, batch: int) -> dict:
+    """Host-side counters of the handle: launches per kernel kind, reference steps and resets per sample."""
+    st = CacheStats()
+    _check(_lib().speca_cache_stats(cache, ctypes.byref(st)), cache)
+    out = {name: int(getattr(st, name)) for name, _ in CacheStats._fields_[:7]}
+    out["reference_steps"] = [int(x) for x in st.reference_steps[:batch]]
+    out["resets"] = [int(x) for x in st.resets[:batch]]
+    return out
+
+
 def speca_cache_launch_count(cache) -> int:
     n = ctypes.c_uint64(0)
     _check(_lib().speca_cache_launch_count(cache, ctypes.byref(n)), cache)
@@ -409,3 +427,6 @@ class SpecaCache:
     @property
     def launches(self) -> int:
         return speca_cache_launch_count(self.handle)
+
+    def stats(self):
+        return speca_cache_stats(self.handle, self.batch)

@@ -138,6 +138,7 @@ struct speca_cache {
     uint8_t pend_mask[SPECA_MAX_BATCH];
     std::vector<uint8_t> entry_updated;
     uint64_t launches;
+    speca_cache_stats_t stats;
     char last_error[256];
 };
 
@@ -251,6 +252,7 @@ speca_status_t speca_cache_create(const speca_cache_config_t* cfg, speca_cache_t
     c->arena = static_cast<char*>(cfg->arena);
     c->pending = false;
     c->launches = 0;
+    std::memset(&c->stats, 0, sizeof c->stats);
     c->last_error[0] = 0;
     try {
         c->entry_updated.assign(c->n_entries, 0);
@@ -311,6 +313,7 @@ speca_status_t speca_cache_reset(speca_cache_t* c, const uint8_t* host_sample_ma
     for (int b = 0; b < c->B; ++b) {
         if (host_sample_mask != nullptr && host_sample_mask[b] == 0) continue;
         c->n_refs[b] = 0;
+        c->stats.resets[b] += 1;
         for (int i = 0; i <= SPECA_MAX_ORDER; ++i) c->t_hist[b][i] = std::numeric_limits<double>::quiet_NaN();
     }
     return SPECA_OK;
@@ -380,6 +383,7 @@ speca_status_t speca_cache_update(speca_cache_t* c, const void* const* feats, co
         cudaError_t ce = launch_update(p, c->dtype, c->path, grid, static_cast<cudaStream_t>(stream));
         if (ce != cudaSuccess) return cuda_fail(c, ce, "update launch");
         c->launches += 1;
+        c->stats.update_launches += 1;
     }
     if (!c->pending) {
         c->pending = true;
@@ -403,6 +407,7 @@ speca_status_t speca_cache_commit_step(speca_cache_t* c) {
         for (int i = SPECA_MAX_ORDER; i >= 1; --i) c->t_hist[b][i] = c->t_hist[b][i - 1];
         c->t_hist[b][0] = c->pend_t[b];
         c->n_refs[b] += 1;
+        c->stats.reference_steps[b] += 1;
     }
     c->pending = false;
     std::fill(c->entry_updated.begin(), c->entry_updated.end(), 0);
@@ -458,6 +463,7 @@ speca_status_t speca_forecast(speca_cache_t* c, const double* t_target, const ui
     cudaError_t ce = launch_forecast(p, c->dtype, c->path, grid, static_cast<cudaStream_t>(stream));
     if (ce != cudaSuccess) return cuda_fail(c, ce, "forecast launch");
     c->launches += 1;
+    c->stats.forecast_launches += 1;
     return SPECA_OK;
 }
 
@@ -517,6 +523,7 @@ speca_status_t speca_forecast_multi(speca_cache_t* c, int32_t n_targets, const d
     cudaError_t ce = launch_forecast_multi(p, c->dtype, c->B, grid, static_cast<cudaStream_t>(stream));
     if (ce != cudaSuccess) return cuda_fail(c, ce, "forecast_multi launch");
     c->launches += 1;
+    c->stats.forecast_multi_launches += 1;
     return SPECA_OK;
 }
 
@@ -571,6 +578,7 @@ speca_status_t speca_forecast_sum(speca_cache_t* c, const int32_t* entry_ids, in
     cudaError_t ce = launch_forecast_sum(p, c->dtype, grid, static_cast<cudaStream_t>(stream));
     if (ce != cudaSuccess) return cuda_fail(c, ce, "forecast_sum launch");
     c->launches += 1;
+    c->stats.forecast_sum_launches += 1;
     return SPECA_OK;
 }
 
@@ -663,6 +671,7 @@ static speca_status_t verify_impl(speca_cache_t* c, int32_t metric, const void* 
     cudaError_t ce = launch_verify(p, c->dtype, grid, c->cluster, static_cast<cudaStream_t>(stream));
     if (ce != cudaSuccess) return cuda_fail(c, ce, "verify launch");
     c->launches += 1;
+    c->stats.verify_launches += 1;
     return SPECA_OK;
 }
 
@@ -736,6 +745,7 @@ speca_status_t speca_select_adaptive(speca_cache_t* c, const uint8_t* dev_accept
                                    dev_n_active, static_cast<cudaStream_t>(stream));
     if (ce != cudaSuccess) return cuda_fail(c, ce, "select launch");
     c->launches += 1;
+    c->stats.select_launches += 1;
     return SPECA_OK;
 }
 
@@ -756,6 +766,7 @@ speca_status_t speca_activate(speca_cache_t* c, const uint8_t* host_sample_mask,
     cudaError_t ce = launch_activate(bits, c->B, dev_spec_count, dev_active_mask, static_cast<cudaStream_t>(stream));
     if (ce != cudaSuccess) return cuda_fail(c, ce, "activate launch");
     c->launches += 1;
+    c->stats.activate_launches += 1;
     return SPECA_OK;
 }
 
@@ -807,6 +818,12 @@ speca_status_t speca_cache_plane(const speca_cache_t* c, int32_t entry, int32_t 
     const SegDesc& s = c->L.segs[static_cast<size_t>(entry) * c->B + sample];
     *plane0 = c->arena + s.plane0_off;
     *plane_stride_bytes = s.plane_stride;
+    return SPECA_OK;
+}
+
+speca_status_t speca_cache_stats(const speca_cache_t* c, speca_cache_stats_t* out) {
+    if (c == nullptr || out == nullptr) return SPECA_ERR_INVALID_ARG;
+    *out = c->stats;
     return SPECA_OK;
 }
 

@@ -55,4 +55,12 @@ def test_sampler_trace_matches_oracle(S, name, metric):
     if not parted:
         assert tr_gpu.acceptance_rate() == tr_cpu.acceptance_rate()
     assert cache.launches > 30
+    # the handle's own tallies agree with the trace: full passes per sample, one verify launch per
+    # speculative step (the fused call), no separate continuation launches
+    st = cache.stats()
+    assert st["reference_steps"] == [f + r for f, _, r in (tr_gpu.counts(b) for b in range(w.batch))]
+    n_spec_steps = sum(1 for row in tr_gpu.steps if any(x != SCH.FULL for x in row))
+    assert st["verify_launches"] == n_spec_steps and st["forecast_launches"] == n_spec_steps
+    assert st["select_launches"] == 0 and st["resets"] == [1] * w.batch
+    assert sum(st[k] for k in st if k.endswith("_launches")) == cache.launches
     cache.close()
