@@ -134,9 +134,10 @@ def physical_gpu_index(local_index: int) -> int:
 class Harness:
     """Device-resident state for one workload: cache, two alternating feature sets, outputs."""
 
-    def __init__(self, w: W.Workload, device: str, seed_offset: int = 0, path: int = 0):
+    def __init__(self, w: W.Workload, device: str, seed_offset: int = 0, path: int = 0, fused_select: bool = True):
         from paper_2509_11628_b200 import binding as S
         self.S, self.w, self.device = S, w, torch.device(device)
+        self.fused_select = fused_select
         self.B, self.m = w.batch, w.max_order
         self.cache = S.SpecaCache(w.entries, w.batch, w.max_order, w.dtype, device, path=path)
         self.src = W.FeatureSource(w, device, seed_offset)
@@ -162,6 +163,7 @@ class Harness:
         self.err = torch.zeros(self.B, dtype=torch.float32, device=self.device)
         self.accept = torch.zeros(self.B, dtype=torch.uint8, device=self.device)
         self.active = torch.ones(self.B, dtype=torch.uint8, device=self.device)
+        self.active_next = torch.ones(self.B, dtype=torch.uint8, device=self.device)
         self.spec = torch.zeros(self.B, dtype=torch.int32, device=self.device)
         self.idx = torch.zeros(self.B, dtype=torch.int32, device=self.device)
         self.n_active = torch.zeros(1, dtype=torch.int32, device=self.device)
@@ -176,7 +178,8 @@ class Harness:
         return [t_ref] * self.B, [t_ref - 0.5 * gap] * self.B
 
     def step(self, events=None, feats=None, fresh=None):
-        """update -> commit -> forecast -> verify -> select on the current stream."""
+        """update -> commit -> forecast -> verify -> select on the current stream; verify and select are
+        one launch (speca_verify_select) unless the harness was made with fused_select=False."""
         S, c, w = self.S, self.cache, self.w
         j = self.j
         self.j += 1
@@ -196,10 +199,17 @@ class Harness:
         c.forecast(t_tgt, self.outs, self.active)
         if events is not None:
             events[3].record()
-        c.verify(fresh, t_tgt, tau, self.err, self.accept, self.active)
-        if events is not None:
-            events[4].record()
-        c.select_adaptive(self.accept, 1 << 30, 1, self.spec, self.active, self.idx, self.n_active)
+        if self.fused_select:
+            c.verify_select(fresh, t_tgt, tau, self.err, self.accept, self.active, self.active_next, 1 << 30, 1, self.spec,
+                            self.idx, self.n_active)
+            self.active, self.active_next = self.active_next, self.active
+            if events is not None:
+                events[4].record()
+        else:
+            c.verify(fresh, t_tgt, tau, self.err, self.accept, self.active)
+            if events is not None:
+                events[4].record()
+            c.select_adaptive(self.accept, 1 << 30, 1, self.spec, self.active, self.idx, self.n_active)
         if events is not None:
             events[5].record()
 
@@ -707,6 +717,8 @@ def main():
                     help="comma list of further configs measured device-resident and reported under per_config")
     ap.add_argument("--path", default="auto", choices=["auto", "direct", "bulk", "wide"],
                     help="kernel variant (speca_path_t); results are identical, only speed differs")
+    ap.add_argument("--separate-select", action="store_true",
+                    help="speca_verify then speca_select_adaptive as two launches instead of speca_verify_select")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-adaptive", action="store_true",
                     help="skip the B=8 sample-adaptive sweep (orders 1-3, horizon 1-6) reported under 'adaptive'")
@@ -732,7 +744,7 @@ def main():
 
     w = make_workload(args.config)
     path = {"auto": 0, "direct": 1, "bulk": 2, "wide": 3}[args.path]
-    h = Harness(w, device, seed_offset=17 * info.rank, path=path)
+    h = Harness(w, device, seed_offset=17 * info.rank, path=path, fused_select=not args.separate_select)
     total_ms, per_ms, launches, clocks = time_device_resident(h, args.steps, args.warmup, info, True)
     total_ms = D.max_over_ranks(total_ms, device)
     value, ms_step, kernels, extra = summarize(w, per_ms, total_ms, args.steps, info.world, peak)
@@ -762,7 +774,7 @@ def main():
         for name in [n for n in args.also.split(",") if n and n != args.config]:
             try:
                 w2 = make_workload(name)
-                h2 = Harness(w2, device, path=path)
+                h2 = Harness(w2, device, path=path, fused_select=not args.separate_select)
                 k2 = max(5, min(args.steps, 2000 // max(1, len(w2.entries)) * 4))
                 t2, p2, _, _ = time_device_resident(h2, k2, 3, info, False)
                 v2, ms2, kern2, ex2 = summarize(w2, p2, t2, k2, 1, peak)
@@ -831,7 +843,9 @@ def main():
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": info.world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(w),
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": dict(workload_config(w), select="its own launch (speca_select_adaptive)" if args.separate_select
+                       else "inside the verify launch (speca_verify_select)"),
         "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches,
         "clocks": clocks, "kernels": kernels, **extra,
         "frac_of_measured_peak": value / info.world / peak, "frac_of_nominal_8TBs": value / info.world / NOMINAL_HBM_GBS,
