@@ -38,7 +38,7 @@ FALLBACK_HBM_GBS = 6650.0
 # from the one-pass ncu capture of this benchmark's default workload at full size (FLUX-shaped cache,
 # order 2, bf16; profiles/dram_traffic_flux_full_size.md). Other workloads scale by the elements a
 # launch covers. Set an entry to None when its kernel changes until the counters have been taken again.
-NCU_DRAM_BYTES_PER_ELEM = {"update": 11.987, "forecast": 8.036, "verify": 8.110}
+NCU_DRAM_BYTES_PER_ELEM = {"update": 11.987, "forecast": 8.042, "verify": 8.107}
 
 
 def measured_peak():
