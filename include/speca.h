@@ -25,6 +25,11 @@
  *     starts at element b*N_e*D. Device tensor pointers must be aligned to the element size;
  *     32-byte aligned rows (pointer and N_e*D*sizeof(element) multiples of 32) take the fast
  *     vector path, anything else a slower 16-byte or element-wise path with equal results.
+ *   - The calls that enqueue work (update, forecast*, verify*, select, activate) neither allocate
+ *     nor synchronise, so they may be issued while `stream` is being captured into a CUDA graph.
+ *     Times, thresholds and host masks are folded into the kernel arguments at capture; a replay
+ *     reads the device buffers (features, masks, counters) as they are then. The host-side history
+ *     (update / commit_step / reset) advances at capture time only, not on replay.
  *   - A handle is not thread safe: use one handle from one host thread at a time.
  *   - There is no CPU fallback: without a usable CUDA device speca_cache_create fails.
  */

@@ -150,3 +150,66 @@ def test_argument_errors(S):
     torch.cuda.synchronize()
     assert acc.cpu().tolist() == [1] * B and masks[B:].cpu().tolist() == [1] * B and cnt.cpu().tolist() == [1] * B
     c.close()
+
+
+def test_speculative_steps_replay_from_a_cuda_graph(S, U):
+    """The calls neither synchronise nor allocate, so a run of speculative steps (forecast, then
+    verification + continuation, at two successive times) can be captured once into a CUDA graph and
+    replayed on new verification features: same bits as the eager calls."""
+    entries = [(40, 1030), (301, 1160)]
+    B, m = 4, 2
+    gen = torch.Generator(device=DEV).manual_seed(31)
+    pair = U.Pair(entries, B, m, 1)
+    for t in (1.0, 0.93, 0.9):
+        pair.update(rand_feats(entries, B, pair.tdt, gen), [t] * B)
+        pair.commit()
+    t1, t2, tau = [0.87] * B, [0.84] * B, [0.05] * B
+    c = pair.gpu
+
+    def buffers():
+        return dict(outs=[[torch.zeros(B, n, d, dtype=pair.tdt, device=DEV) for n, d in entries] for _ in range(2)],
+                    err=torch.zeros(2, B, device=DEV), acc=torch.zeros(2, B, dtype=torch.uint8, device=DEV),
+                    masks=torch.ones(3, B, dtype=torch.uint8, device=DEV), cnt=torch.zeros(B, dtype=torch.int32, device=DEV))
+
+    fresh = [torch.zeros(B, *entries[1], dtype=pair.tdt, device=DEV) for _ in range(2)]
+
+    def steps(x):
+        c.forecast(t1, x["outs"][0], x["masks"][0])
+        c.verify_select(fresh[0], t1, tau, x["err"][0], x["acc"][0], x["masks"][0], x["masks"][1], 4, 1, x["cnt"])
+        c.forecast(t2, x["outs"][1], x["masks"][1])
+        c.verify_select(fresh[1], t2, tau, x["err"][1], x["acc"][1], x["masks"][1], x["masks"][2], 4, 1, x["cnt"])
+
+    def new_fresh(seed):
+        g = torch.Generator(device=DEV).manual_seed(seed)
+        ref = buffers()
+        c.forecast(t1, ref["outs"][0]); c.forecast(t2, ref["outs"][1])
+        level = torch.tensor([0.0, 0.01, 0.4, 0.02], device=DEV).view(B, 1, 1).roll(seed, 0)
+        for k in range(2):
+            fresh[k].copy_((ref["outs"][k][1].float() + level * torch.randn(B, *entries[1], generator=g, device=DEV)).to(pair.tdt))
+
+    graphed = buffers()
+    new_fresh(1)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    launches = c.launches
+    with torch.cuda.graph(graph):
+        steps(graphed)
+    assert c.launches == launches + 4
+    for seed in (1, 2, 3):
+        new_fresh(seed)
+        eager = buffers()
+        steps(eager)
+        graphed["masks"].fill_(1); graphed["cnt"].zero_(); graphed["acc"].zero_(); graphed["err"].zero_()
+        for o in graphed["outs"][0] + graphed["outs"][1]:
+            o.zero_()          # rows of samples that this replay leaves out must compare equal to the eager zeros
+        graph.replay()
+        torch.cuda.synchronize()
+        for k in ("err", "acc", "masks", "cnt"):
+            assert torch.equal(eager[k].view(torch.uint8), graphed[k].view(torch.uint8)), (seed, k)
+        for a, b_ in zip(eager["outs"], graphed["outs"]):
+            for x, y in zip(a, b_):
+                assert torch.equal(x.view(torch.uint8), y.view(torch.uint8))
+        want = [0 if lv == 0.4 else 1 for lv in np.roll([0.0, 0.01, 0.4, 0.02], seed)]
+        assert eager["acc"][0].cpu().tolist() == want and eager["masks"][1].cpu().tolist() == want
+        assert eager["outs"][1][1][want.index(0)].abs().sum().item() == 0     # dropped after step 1: not forecast at step 2
+    pair.close()
