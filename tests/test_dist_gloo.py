@@ -79,7 +79,9 @@ def test_two_ranks_shard_samples_without_a_data_path_collective(tmp_path):
     err_all, acc_all = _decisions(list(range(B)), feats, fresh_noise, n)
     assert got["acc"] == acc_all            # per-sample decisions do not depend on the sharding
     assert got["shard0"] == [0, 1, 2]
-    assert got["err_rank0"] == err_all[:3]  # bit-identical: a sample's error depends on that sample alone
+    # a sample's error depends on that sample alone; the oracle adds up in a thread-count-dependent
+    # order, so two processes may differ in the last place of a double
+    assert got["err_rank0"] == pytest.approx(err_all[:3], rel=1e-12, abs=0.0)
     assert acc_all[0] == 1 and acc_all[3] == 0
 
 
