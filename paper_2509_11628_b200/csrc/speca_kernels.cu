@@ -389,11 +389,19 @@ struct Shape {
 #define SPECA_SHAPES_FORECAST \
     {32, 128, 2, 4, 4}, {32, 256, 1, 4, 3}, {32, 256, 1, 4, 3}, {32, 256, 1, 4, 2}, { 32, 256, 1, 4, 2 }
 #endif
-__host__ __device__ constexpr Shape shape_for(int path, bool update, int v) {
+// fp32 storage takes the same shapes with one exception, measured on the FLUX-shaped entries: the
+// order-4 update (five reads, five writes) ran at 5.2 TB/s with one vector per thread against 6.3-6.4
+// with four vectors per thread and one CTA per SM; bf16 prefers the table's shape (6.49 against 6.38).
+#ifndef SPECA_SHAPE_UPDATE4_F32
+#define SPECA_SHAPE_UPDATE4_F32 { 32, 128, 4, 2, 1 }
+#endif
+__host__ __device__ constexpr Shape shape_for(int path, bool update, int v, int dtype) {
     constexpr Shape up[SPECA_MAX_ORDER + 1] = {SPECA_SHAPES_UPDATE};
     constexpr Shape fc[SPECA_MAX_ORDER + 1] = {SPECA_SHAPES_FORECAST};
     const int i = v < 0 ? 0 : (v > SPECA_MAX_ORDER ? SPECA_MAX_ORDER : v);
-    return path == SPECA_PATH_WIDE ? (update ? up[i] : fc[i]) : Shape{16, 256, 4, 1, 2};
+    if (path != SPECA_PATH_WIDE) return Shape{16, 256, 4, 1, 2};
+    if (update && i == 4 && dtype == SPECA_F32) return Shape SPECA_SHAPE_UPDATE4_F32;
+    return update ? up[i] : fc[i];
 }
 __host__ __device__ constexpr uint32_t shape_tile_bytes(Shape s) { return static_cast<uint32_t>(s.w) * s.nt * s.u * s.chunks; }
 
@@ -1274,8 +1282,9 @@ __global__ void __launch_bounds__(SPECA_MAX_BATCH) activate_kernel(uint64_t mask
 
 template <int DT, bool UPDATE, int PATH>
 static const void* stream_kernel_for(int v) {
-    constexpr Shape s0 = shape_for(PATH, UPDATE, 0), s1 = shape_for(PATH, UPDATE, 1), s2 = shape_for(PATH, UPDATE, 2),
-                    s3 = shape_for(PATH, UPDATE, 3), s4 = shape_for(PATH, UPDATE, 4);
+    constexpr Shape s0 = shape_for(PATH, UPDATE, 0, DT), s1 = shape_for(PATH, UPDATE, 1, DT),
+                    s2 = shape_for(PATH, UPDATE, 2, DT), s3 = shape_for(PATH, UPDATE, 3, DT),
+                    s4 = shape_for(PATH, UPDATE, 4, DT);
     static_assert(shape_tile_bytes(s0) == shape_tile_bytes(s2) && shape_tile_bytes(s1) == shape_tile_bytes(s2) &&
                       shape_tile_bytes(s3) == shape_tile_bytes(s2) && shape_tile_bytes(s4) == shape_tile_bytes(s2),
                   "all orders of a path share one tile size (one tile table)");
@@ -1350,7 +1359,7 @@ static int clamp_order(int v) { return v < 0 ? 0 : (v > SPECA_MAX_ORDER ? SPECA_
 
 uint32_t stream_tile_bytes(int path, bool update) {
     if (path == SPECA_PATH_BULK) return kBulkTileBytes;
-    return shape_tile_bytes(shape_for(path, update, 2));
+    return shape_tile_bytes(shape_for(path, update, 2, SPECA_BF16));  // the same for every order and dtype
 }
 
 int stream_ctas_per_sm(int path, bool update, int dtype, int order) {
@@ -1365,7 +1374,7 @@ int stream_ctas_per_sm(int path, bool update, int dtype, int order) {
         }
         return n;
     }
-    return shape_for(path, update, order).minb;
+    return shape_for(path, update, order, dtype).minb;
 }
 
 static cudaError_t launch_stream(const StreamParams& p, int dtype, bool update, int path, int grid,
@@ -1383,7 +1392,7 @@ static cudaError_t launch_stream(const StreamParams& p, int dtype, bool update, 
     const int v = max_order(p.order);
     const void* fn = stream_kernel_for(dtype, update, path, v);
     void* args[1] = {const_cast<StreamParams*>(&p)};
-    return cudaLaunchKernel(fn, dim3(grid), dim3(shape_for(path, update, v).nt), args, 0, stream);
+    return cudaLaunchKernel(fn, dim3(grid), dim3(shape_for(path, update, v, dtype).nt), args, 0, stream);
 }
 
 cudaError_t launch_update(const StreamParams& p, int dtype, int path, int grid, cudaStream_t stream) {
