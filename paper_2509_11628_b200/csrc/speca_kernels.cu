@@ -600,7 +600,39 @@ __global__ void __launch_bounds__(kSumThreads, kSumMinBlocks) forecast_sum_kerne
 #pragma unroll
                 for (int k = 0; k < EPV; ++k) sum[k] = 0.f;
             }
-            for (int j = 0; j < p.n_ids; ++j) {
+            int j = 0;
+            if (v == V) {
+                // Low orders read one or two planes per entry: take the entries in groups so that every
+                // thread keeps four loads in flight. The forecasts are still added one by one, in list order.
+                constexpr int G = V == 0 ? 4 : (V == 1 ? 2 : 1);
+                if constexpr (G > 1) {
+                    for (; j + G <= p.n_ids; j += G) {
+                        Vec<W> d[G][V + 1];
+#pragma unroll
+                        for (int g = 0; g < G; ++g) {
+                            const SegDesc sd = p.segs[static_cast<uint32_t>(p.ids[j + g]) * p.batch + b];
+                            const char* plane0 = p.arena + sd.plane0_off + byte0 + static_cast<size_t>(idx) * W;
+#pragma unroll
+                            for (int i = 0; i <= V; ++i) d[g][i] = load_vec<W>(plane0 + i * sd.plane_stride);
+                        }
+#pragma unroll
+                        for (int g = 0; g < G; ++g) {
+                            float acc[EPV];
+                            unpack_vec<DT, W>(d[g][V], acc);
+#pragma unroll
+                            for (int i = V; i >= 1; --i) {
+                                float lo[EPV];
+                                unpack_vec<DT, W>(d[g][i - 1], lo);
+#pragma unroll
+                                for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+                            }
+#pragma unroll
+                            for (int k = 0; k < EPV; ++k) sum[k] += acc[k];
+                        }
+                    }
+                }
+            }
+            for (; j < p.n_ids; ++j) {
                 const SegDesc sd = p.segs[static_cast<uint32_t>(p.ids[j]) * p.batch + b];
                 const char* plane0 = p.arena + sd.plane0_off + byte0 + static_cast<size_t>(idx) * W;
                 float acc[EPV];

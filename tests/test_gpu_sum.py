@@ -44,19 +44,22 @@ def U_as64(a):
 @pytest.mark.parametrize("dtype", [0, 1])
 @pytest.mark.parametrize("basis", [0, 1, 2])
 @pytest.mark.parametrize("shape", [(37, 129), (3, 8192 + 8), (1, 5)])
-def test_summed_forecast_matches_oracle(S, U, dtype, basis, shape):
-    E, B, m = 5, 3, 2
+@pytest.mark.parametrize("m", [0, 1, 2, 4])   # orders 0 and 1 take the entries in groups of 4 and 2
+def test_summed_forecast_matches_oracle(S, U, dtype, basis, shape, m):
+    E, B = 7, 3
     entries = [shape] * E + [(2, 7)]                      # a differently shaped entry that is never listed
     gen = torch.Generator(device=DEV).manual_seed(300 + 10 * basis + dtype)
     pair = U.Pair(entries, B, m, dtype, basis)
-    for k, t in enumerate([1.0, 0.93, 0.9]):
+    for k, t in enumerate([1.0, 0.93, 0.9, 0.84, 0.8][: m + 1]):
         pair.update(rand_feats(entries, B, pair.tdt, gen), [t, t - 0.003, t + 0.001])
         pair.commit()
         pair.sync_tables()
-    tt = [0.86, 0.85, 0.87]
+    t_last = [1.0, 0.93, 0.9, 0.84, 0.8][m]
+    tt = [t_last - 0.04, t_last - 0.05, t_last - 0.03]
     n = shape[0] * shape[1]
     base = torch.randn(B, shape[0], shape[1], generator=gen, device=DEV).to(pair.tdt)
-    for ids, use_base, active in [([0, 1, 2, 3, 4], True, None), ([3], False, None), ([4, 0, 4], True, [1, 0, 1])]:
+    for ids, use_base, active in [([0, 1, 2, 3, 4, 5, 6], True, None), ([3], False, None), ([4, 0, 4], True, [1, 0, 1]),
+                                  ([6, 5, 4, 3, 2, 1], False, [0, 1, 1])]:
         out = torch.full((B, shape[0], shape[1]), 3.0, dtype=pair.tdt, device=DEV)
         mask = torch.tensor(active, dtype=torch.uint8, device=DEV) if active else None
         pair.gpu.forecast_sum(ids, tt, out, base if use_base else None, mask)
