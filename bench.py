@@ -846,6 +846,8 @@ def main():
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": dict(workload_config(w), select="its own launch (speca_select_adaptive)" if args.separate_select
                        else "inside the verify launch (speca_verify_select)"),
+        "metric_note": "value = algorithmic bytes of the whole step (update + forecast + verify/select) / step time; "
+                       "forecast + verify alone (one speculative step) is forecast_verify_gbs, the update alone kernels.update.gbs",
         "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches,
         "clocks": clocks, "kernels": kernels, **extra,
         "frac_of_measured_peak": value / info.world / peak, "frac_of_nominal_8TBs": value / info.world / NOMINAL_HBM_GBS,
