@@ -46,7 +46,9 @@ _lib = None
 def lib() -> ctypes.CDLL:
     global _lib
     if _lib is None:
-        L = ctypes.CDLL(build())
+        # SPECA_ORACLE_LIB: a library built elsewhere from (a variant of) speca_oracle.c; the mutation
+        # tests use it to check that the pins notice mistakes planted in the C source
+        L = ctypes.CDLL(os.environ.get("SPECA_ORACLE_LIB") or build())
         i64, i32, dbl, vp = ctypes.c_int64, ctypes.c_int, ctypes.c_double, ctypes.c_void_p
         dp = ctypes.POINTER(ctypes.c_double)
         L.oracle_update_segment.argtypes = [i32, i64, i32, i32, i32, dp, dbl, vp, vp, i64]

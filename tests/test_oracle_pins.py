@@ -321,11 +321,12 @@ def test_bf16_tables_round_once_per_stored_plane():
 
 @pytest.mark.parametrize("basis", [O.TAYLOR, O.NEWTON, O.ADAMS_BASHFORTH])
 @pytest.mark.parametrize("dtype", [O.F32, O.BF16])
-def test_summed_forecast_of_one_entry_is_the_plain_forecast_bit_for_bit(basis, dtype):
+@pytest.mark.parametrize("m", [1, 2, 3, 4])   # every order: each has its own Adams-Bashforth coefficient
+def test_summed_forecast_of_one_entry_is_the_plain_forecast_bit_for_bit(basis, dtype, m):
     g = torch.Generator().manual_seed(90 + basis)
-    B, n, m = 2, 300, 3
+    B, n = 2, 300
     cache = O.OracleCache([n, n], B, m, dtype, basis)
-    for k, t in enumerate([1.0, 0.93, 0.9, 0.81]):
+    for k, t in enumerate([1.0, 0.93, 0.9, 0.81, 0.79][: m + 1]):
         fs = [torch.randn(B, n, generator=g) for _ in range(2)]
         fs = [bf16_bits(f) if dtype == O.BF16 else f.numpy().copy() for f in fs]
         cache.update(fs, [t, t - 0.004])
@@ -621,12 +622,32 @@ def test_two_stage_metrics_agree_with_the_one_stage_ones_and_split_over_parts(me
     f = torch.randn(3001, generator=g).numpy()
     p = (f + 0.05 * torch.randn(3001, generator=g).numpy()).astype(np.float32)
     whole = O.metric_sums(metric, O.F32, p, f)
-    assert O.metric_from_sums(metric, whole) == pytest.approx(O.rel_err(metric, O.F32, p, f), rel=1e-12, abs=1e-15)
+    # the cosine distance is a difference of two numbers near 1: its absolute error is what the order
+    # of summation (which depends on the thread count) moves
+    tol = dict(rel=1e-12, abs=1e-13 if metric == O.METRIC_COSINE else 1e-15)
+    assert O.metric_from_sums(metric, whole) == pytest.approx(O.rel_err(metric, O.F32, p, f), **tol)
     cut = 1234
     a = O.metric_sums(metric, O.F32, p[:cut].copy(), f[:cut].copy())
     b = O.metric_sums(metric, O.F32, p[cut:].copy(), f[cut:].copy())
     both = [max(x, y) for x, y in zip(a, b)] if metric == O.METRIC_LINF else [x + y for x, y in zip(a, b)]
-    assert O.metric_from_sums(metric, both) == pytest.approx(O.rel_err(metric, O.F32, p, f), rel=1e-12, abs=1e-15)
+    assert O.metric_from_sums(metric, both) == pytest.approx(O.rel_err(metric, O.F32, p, f), **tol)
+
+
+@pytest.mark.parametrize("metric", [O.METRIC_L2] + OTHER_METRICS)
+@pytest.mark.parametrize("where", ["forecast", "feature"])
+def test_a_nan_element_makes_every_metric_nan_in_one_stage_and_in_two(metric, where):
+    f = np.arange(1, 41, dtype=np.float32)
+    p = f + 0.5
+    (p if where == "forecast" else f)[17] = np.nan
+    assert math.isnan(O.rel_err(metric, O.F32, p, f))
+    assert math.isnan(O.metric_from_sums(metric, O.metric_sums(metric, O.F32, p, f)))
+    # the part without the NaN is finite; combined with the other part the result is NaN again
+    a, b = O.metric_sums(metric, O.F32, p[:10].copy(), f[:10].copy()), O.metric_sums(metric, O.F32, p[10:].copy(), f[10:].copy())
+    assert all(math.isfinite(x) for x in a)
+    both = [max(x, y) if not (math.isnan(x) or math.isnan(y)) else math.nan for x, y in zip(a, b)] \
+        if metric == O.METRIC_LINF else [x + y for x, y in zip(a, b)]
+    assert math.isnan(O.metric_from_sums(metric, both))
+    assert not O.accept(math.nan, 1e30)
 
 
 def test_accept_rule():
@@ -727,3 +748,31 @@ def test_cache_masks_and_per_sample_history():
     assert err[0] == 0.0 and acc[0] == 1 and np.isnan(err[1]) and acc[1] == -1 and acc[2] == 1
     c.reset([0, 1, 0])
     assert c.n_refs == [2, 0, 1]
+
+
+def test_cache_verify_scores_the_forecast_against_the_fresh_feature():
+    # features linear in t with small-integer values: the forecast is exact in fp32 (degree 1), so a
+    # fresh feature that is (1 + d) times the truth must score e = |d| / (1 + d), sample by sample
+    B, m, n = 3, 2, 40
+    rng = np.random.default_rng(15)
+    a = rng.integers(-8, 9, (B, n)).astype(np.float64) * 4
+    s = rng.integers(-8, 9, (B, n)).astype(np.float64) * 4
+    s[:, 0] = 4.0                               # no sample is all zero
+    feat = lambda t: (a + s * t).astype(np.float32)
+    c = O.OracleCache([7, n], B, m, O.F32)      # verification entry = the last one
+    for t in (8.0, 6.0, 4.0):
+        c.update([np.zeros((B, 7), dtype=np.float32), feat(t)], [t] * B)
+        c.commit_step()
+    truth = feat(2.0)
+    d = [0.0, 0.25, -0.5]
+    fresh = np.stack([truth[b] * np.float32(1.0 + d[b]) for b in range(B)])
+    err, acc, pred = c.verify(fresh, [2.0] * B, [0.3] * B)
+    assert np.array_equal(pred, truth) and np.array_equal(pred, c.forecast_entry(1, [2.0] * B))
+    for b in range(B):
+        norm = math.sqrt(sum(float(x) ** 2 for x in truth[b]))           # ||truth||, exact integers
+        assert err[b] == pytest.approx(abs(d[b]) * norm / ((1.0 + d[b]) * norm + 1e-8), rel=1e-12, abs=1e-15)
+        assert err[b] == pytest.approx(abs(d[b]) / (1.0 + d[b]), rel=1e-9, abs=1e-15)   # epsilon is negligible here
+    assert acc.tolist() == [1, 1, 0]            # 0 <= 0.3, 0.2 <= 0.3, 1.0 > 0.3
+    # per-sample thresholds, and the l1 reading through the same call
+    err1, acc1, _ = c.verify(fresh, [2.0] * B, [0.0, 0.1, 2.0], metric=O.METRIC_L1)
+    assert err1 == pytest.approx(err, rel=1e-9, abs=1e-15) and acc1.tolist() == [1, 0, 1]   # up to epsilon's share
