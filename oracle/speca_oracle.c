@@ -10,6 +10,8 @@
  *   oracle_update_segment    Eq. 3 (finite differences of the cached feature), kept as difference
  *                            quotients so that reference steps may be unevenly spaced
  *   oracle_forecast_segment  Eq. 2 (TaylorSeer prediction), written as the printed sum
+ *   oracle_forecast_history_segment  Eq. 2-3 evaluated from the stored raw features of the last
+ *                            references (no rounded intermediate planes)
  *   oracle_rel_l2            Eq. 4 (relative error, epsilon = 1e-8)
  *   oracle_rel_l1/_linf, oracle_cos_dist   the other metrics of the appendix on error metrics
  *                            (named there without formulas: readings, parity unpinned by the paper)
@@ -188,6 +190,65 @@ int oracle_forecast_segment(int dtype, int64_t n, int m, int basis, int n_refs, 
         double s = load_elem(planes, dtype, j);
         for (int i = 1; i <= v; ++i)
             s += load_elem((const char*)planes + (size_t)i * plane_stride * esz, dtype, j) * w[i];
+        store_elem(out, dtype, j, s);
+    }
+    return 0;
+}
+
+/* ---- Eq. 2-3 straight from the raw feature history ------------------------------------------------ */
+/*
+ * The same forecast when the cache keeps the last references' FEATURES instead of their difference
+ * quotients: hist[0] is the feature at t_hist[0] (the latest reference), hist[1] the one before, ...;
+ * n_hist = min(m + 1, references seen) of them exist. Eq. 3's differences are formed here, in double,
+ * by folding the features in one by one from the oldest to the newest exactly as
+ * oracle_update_segment would have (same divisors), but without rounding any intermediate plane to
+ * the storage type; Eq. 2 (or the Newton / Adams-Bashforth reading) is then applied as in
+ * oracle_forecast_segment and the result is rounded once. On a uniform grid this is Eq. 2-3 as
+ * printed, evaluated from the raw features.
+ * Returns 0, or 1 if there is no reference or a divisor is zero.
+ */
+int oracle_forecast_history_segment(int dtype, int64_t n, int m, int basis, int n_hist, const double* t_hist,
+                                    double t_target, const void* const* hist, void* out) {
+    if (n_hist < 1 || n_hist > m + 1 || m > ORACLE_MAX_ORDER) return 1;
+    int v = n_hist - 1;
+    if (basis == ORACLE_ADAMS_BASHFORTH && v > 4) return 1;
+    for (int k = v - 1; k >= 0; --k)
+        for (int i = 0; i < v - k; ++i)
+            if (t_hist[k] - (basis == ORACLE_NEWTON ? t_hist[k + 1 + i] : t_hist[k + 1]) == 0.0) return 1;
+    static const double gam[4] = {1.0, 1.0 / 2, 5.0 / 12, 3.0 / 8}; /* Adams-Bashforth, collected by plane */
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < n; ++j) {
+        double d[ORACLE_MAX_ORDER + 1]; /* the planes a table would hold, unrounded */
+        d[0] = load_elem(hist[v], dtype, j);
+        for (int k = v - 1; k >= 0; --k) { /* fold in the feature at t_hist[k]; v - k references came before */
+            double c[ORACLE_MAX_ORDER + 1];
+            c[0] = load_elem(hist[k], dtype, j);
+            for (int i = 0; i < v - k; ++i) {
+                double gap = t_hist[k] - (basis == ORACLE_NEWTON ? t_hist[k + 1 + i] : t_hist[k + 1]);
+                c[i + 1] = (c[i] - d[i]) / gap;
+            }
+            for (int i = 0; i <= v - k; ++i) d[i] = c[i];
+        }
+        double s = d[0];
+        if (basis == ORACLE_NEWTON) {
+            double w = 1.0;
+            for (int i = 1; i <= v; ++i) {
+                w *= t_target - t_hist[i - 1];
+                s += d[i] * w;
+            }
+        } else if (basis == ORACLE_TAYLOR) {
+            double x = t_target - t_hist[0], fact = 1.0;
+            for (int i = 1; i <= v; ++i) {
+                fact *= (double)i;
+                s += d[i] * pow(x, (double)i) / fact;
+            }
+        } else {
+            double x = t_target - t_hist[0], h = v >= 2 ? t_hist[0] - t_hist[1] : 0.0, hp = 1.0;
+            for (int i = 1; i <= v; ++i) {
+                s += d[i] * x * gam[i - 1] * hp;
+                hp *= h;
+            }
+        }
         store_elem(out, dtype, j, s);
     }
     return 0;

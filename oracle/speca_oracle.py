@@ -26,6 +26,7 @@ _LIB = os.path.join(_HERE, "libspeca_oracle.so")
 F32, BF16 = 0, 1
 TAYLOR, NEWTON, ADAMS_BASHFORTH = 0, 1, 2
 METRIC_L2, METRIC_L1, METRIC_LINF, METRIC_COSINE = 0, 1, 2, 3
+LAYOUT_TABLES, LAYOUT_HISTORY = 0, 1   # what the cache keeps: difference quotients, or the raw features
 EPS_PAPER = 1e-8  # Eq. 4
 
 
@@ -55,6 +56,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_update_segment.restype = i32
         L.oracle_forecast_segment.argtypes = [i32, i64, i32, i32, i32, dp, dbl, vp, i64, vp]
         L.oracle_forecast_segment.restype = i32
+        L.oracle_forecast_history_segment.argtypes = [i32, i64, i32, i32, i32, dp, dbl, ctypes.POINTER(vp), vp]
+        L.oracle_forecast_history_segment.restype = i32
         L.oracle_forecast_accumulate_segment.argtypes = [i32, i64, i32, i32, i32, dp, dbl, vp, i64, vp]
         L.oracle_forecast_accumulate_segment.restype = i32
         L.oracle_accumulate_elems.argtypes = [i32, i64, vp, vp]
@@ -121,6 +124,19 @@ def forecast_segment(dtype, m, basis, n_refs, t_hist, t_target, planes: np.ndarr
                                        _ptr(planes), planes.strides[0] // planes.itemsize, _ptr(out))
     if rc != 0:
         raise RuntimeError("forecast from an empty table")
+
+
+def forecast_history_segment(dtype, m, basis, t_hist, t_target, hist: Sequence[np.ndarray], out: np.ndarray) -> None:
+    """Eq. 2-3 from the raw features of the last references: ``hist[0]`` at ``t_hist[0]`` (the latest),
+    ``hist[1]`` the one before, ...; at most ``m + 1`` of them."""
+    k = len(hist)
+    assert 1 <= k <= m + 1 and len(t_hist) >= k
+    assert all(h.flags.c_contiguous and h.dtype == np_dtype(dtype) and h.size == out.size for h in hist)
+    assert out.flags.c_contiguous and out.dtype == np_dtype(dtype)
+    ptrs = (ctypes.c_void_p * k)(*[h.ctypes.data for h in hist])
+    rc = lib().oracle_forecast_history_segment(dtype, out.size, m, basis, k, _hist(t_hist, m), float(t_target), ptrs, _ptr(out))
+    if rc != 0:
+        raise RuntimeError("forecast from an empty history, or a repeated reference time")
 
 
 def rel_l2(dtype, pred: np.ndarray, fresh: np.ndarray, eps: float = EPS_PAPER) -> float:
@@ -203,9 +219,12 @@ class OracleCache:
     """Derivative tables for a list of entries, with per-sample reference history."""
 
     def __init__(self, entry_elems: Sequence[int], batch: int, max_order: int, dtype: int,
-                 basis: int = TAYLOR, verify_entry: int = -1, eps: float = EPS_PAPER):
+                 basis: int = TAYLOR, verify_entry: int = -1, eps: float = EPS_PAPER, layout: int = LAYOUT_TABLES):
         self.entry_elems = [int(n) for n in entry_elems]
         self.B, self.m, self.dtype, self.basis = batch, max_order, dtype, basis
+        self.layout = layout
+        # LAYOUT_HISTORY: hist[e][b] = stored features of the last <= m + 1 references, latest first
+        self.hist: List[List[List[np.ndarray]]] = [[[] for _ in range(batch)] for _ in self.entry_elems]
         self.verify_entry = verify_entry if verify_entry >= 0 else len(self.entry_elems) - 1
         self.eps = eps
         self.planes: List[np.ndarray] = [np.zeros((batch, max_order + 1, n), dtype=np_dtype(dtype))
@@ -223,7 +242,12 @@ class OracleCache:
                 continue
             f = np.ascontiguousarray(f).reshape(self.B, self.entry_elems[e])
             for b in range(self.B):
-                if mask[b]:
+                if mask[b] and self.layout == LAYOUT_HISTORY:
+                    if self.n_refs[b] >= 1 and float(t_ref[b]) == self.t_hist[b][0]:
+                        raise ZeroDivisionError("reference time repeats: zero gap")
+                    kept = self.hist[e][b] if self.n_refs[b] >= 1 else []   # a reset sample starts over
+                    self.hist[e][b] = ([f[b].copy()] + kept)[: self.m + 1]
+                elif mask[b]:
                     update_segment(self.dtype, self.m, self.basis, self.n_refs[b], self.t_hist[b], t_ref[b],
                                    f[b], self.planes[e][b])
 
@@ -247,8 +271,12 @@ class OracleCache:
             out = np.zeros((self.B, self.entry_elems[e]), dtype=np_dtype(self.dtype))
         for b in range(self.B):
             if (active is None or active[b]) and self.n_refs[b] >= 1:
-                forecast_segment(self.dtype, self.m, self.basis, self.n_refs[b], self.t_hist[b], t_target[b],
-                                 self.planes[e][b], out[b])
+                if self.layout == LAYOUT_HISTORY:
+                    forecast_history_segment(self.dtype, self.m, self.basis, self.t_hist[b], t_target[b],
+                                             self.hist[e][b][: min(self.n_refs[b], self.m + 1)], out[b])
+                else:
+                    forecast_segment(self.dtype, self.m, self.basis, self.n_refs[b], self.t_hist[b], t_target[b],
+                                     self.planes[e][b], out[b])
         return out
 
     def forecast_multi(self, e: int, t_targets: Sequence[Sequence[float]], active: Optional[Sequence[int]] = None,
@@ -269,6 +297,7 @@ class OracleCache:
         keep what `out` held."""
         n = self.entry_elems[entry_ids[0]]
         assert all(self.entry_elems[e] == n for e in entry_ids)
+        assert self.layout == LAYOUT_TABLES, "the summed forecast is defined on difference tables"
         if out is None:
             out = np.zeros((self.B, n), dtype=np_dtype(self.dtype))
         for b in range(self.B):

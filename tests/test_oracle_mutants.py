@@ -32,7 +32,7 @@ MUTANTS = [
     ("adams_bashforth_backward_difference_sign", "hp *= -h;", "hp *= h;", 0, 1),
     ("summed_forecast_keeps_only_the_last_entry", "acc[j] += s;", "acc[j] = s;", 0, 1),
     ("summed_forecast_drops_the_factorial", "w[i] = pow(x, (double)i) / fact;", "w[i] = pow(x, (double)i);", 1, 2),
-    ("summed_adams_bashforth_wrong_coefficient", "{1.0, 1.0 / 2, 5.0 / 12, 3.0 / 8}", "{1.0, 1.0 / 2, 5.0 / 12, 1.0 / 3}", 0, 1),
+    ("summed_adams_bashforth_wrong_coefficient", "static const double gam[4] = {1.0, 1.0 / 2, 5.0 / 12, 3.0 / 8};\n", "static const double gam[4] = {1.0, 1.0 / 2, 5.0 / 12, 1.0 / 3};\n", 0, 1),
     ("bf16_store_truncates", "nearbyint(ldexp(v, 7 - lead))", "trunc(ldexp(v, 7 - lead))", 0, 1),
     ("store_rounds_the_double_directly", "float r = (float)v; /* the binary32 register that holds the result */",
      "double r = v;", 0, 1),
@@ -53,6 +53,18 @@ MUTANTS = [
     ("two_stage_linf_hides_a_nan", "if (bad) a0 = a1 = NAN;", "", 0, 1),
     ("summed_forecast_base_added_twice", "for (int64_t j = 0; j < n; ++j) acc[j] += load_elem(src, dtype, j);",
      "for (int64_t j = 0; j < n; ++j) acc[j] += 2.0 * load_elem(src, dtype, j);", 0, 1),
+    ("history_wrong_sign", "c[i + 1] = (c[i] - d[i]) / gap;", "c[i + 1] = (d[i] - c[i]) / gap;", 0, 1),
+    ("history_taylor_divides_by_span", "double gap = t_hist[k] - (basis == ORACLE_NEWTON ? t_hist[k + 1 + i] : t_hist[k + 1]);",
+     "double gap = t_hist[k] - t_hist[k + 1 + i];", 0, 1),
+    ("history_newton_divides_by_last_gap", "double gap = t_hist[k] - (basis == ORACLE_NEWTON ? t_hist[k + 1 + i] : t_hist[k + 1]);",
+     "double gap = t_hist[k] - t_hist[k + 1];", 0, 1),
+    ("history_starts_from_the_newest", "d[0] = load_elem(hist[v], dtype, j);\n        for (int k = v - 1; k >= 0; --k) {",
+     "d[0] = load_elem(hist[0], dtype, j);\n        for (int k = v - 1; k >= 0; --k) {", 0, 1),
+    ("history_drops_the_factorial", "s += d[i] * pow(x, (double)i) / fact;", "s += d[i] * pow(x, (double)i);", 0, 1),
+    ("history_newton_nodes_shifted", "w *= t_target - t_hist[i - 1];", "w *= t_target - t_hist[i];", 0, 1),
+    ("history_adams_bashforth_wrong_coefficient", "static const double gam[4] = {1.0, 1.0 / 2, 5.0 / 12, 3.0 / 8}; /* Adams-Bashforth, collected by plane */",
+     "static const double gam[4] = {1.0, 1.0 / 2, 5.0 / 12, 1.0 / 3};", 0, 1),
+    ("history_keeps_only_low_orders", "for (int i = 0; i <= v - k; ++i) d[i] = c[i];", "for (int i = 0; i < v - k; ++i) d[i] = c[i];", 0, 1),
     ("accept_is_strict", "return err <= tau ? 1 : 0;", "return err < tau ? 1 : 0;", 0, 1),
     ("threshold_decays_the_wrong_way", "pow(beta, (T - t) / T)", "pow(beta, t / T)", 0, 1),
     ("speedup_forgets_the_verification_cost", "1.0 / (1.0 - alpha + alpha * gamma)", "1.0 / (1.0 - alpha)", 0, 1),
@@ -65,16 +77,20 @@ PY_MUTANTS = [
     ("continuation_counts_inactive_samples", "        if active[b]:\n            if accept_flags[b]:", "        if True:\n            if accept_flags[b]:", 0, 1),
     ("continuation_keeps_rejected_samples", "keep[b] = 1 if (accept_flags[b] and count[b] < k_max) else 0", "keep[b] = 1 if count[b] < k_max else 0", 0, 1),
     ("group_survives_if_any_member_does", "ok = all(keep[g + i] for i in range(group))", "ok = any(keep[g + i] for i in range(group))", 0, 1),
-    ("update_ignores_the_sample_mask", "                if mask[b]:\n                    update_segment(", "                if True:\n                    update_segment(", 0, 1),
+    ("update_ignores_the_sample_mask", "                elif mask[b]:\n                    update_segment(", "                else:\n                    update_segment(", 0, 1),
+    ("history_update_ignores_the_sample_mask", "if mask[b] and self.layout == LAYOUT_HISTORY:", "if self.layout == LAYOUT_HISTORY:", 0, 1),
     ("commit_advances_every_sample", "            if mask[b]:\n                self.t_hist[b] =", "            if True:\n                self.t_hist[b] =", 0, 1),
     ("commit_appends_instead_of_prepending", "([float(t_ref[b])] + self.t_hist[b])[: self.m + 1]", "(self.t_hist[b] + [float(t_ref[b])])[: self.m + 1]", 0, 1),
     ("reset_keeps_the_count", "                self.n_refs[b] = 0\n", "                pass\n", 0, 1),
-    ("forecast_ignores_the_active_mask", "if (active is None or active[b]) and self.n_refs[b] >= 1:\n                forecast_segment(",
-     "if self.n_refs[b] >= 1:\n                forecast_segment(", 0, 1),
+    ("forecast_ignores_the_active_mask", "if (active is None or active[b]) and self.n_refs[b] >= 1:\n                if self.layout == LAYOUT_HISTORY:",
+     "if self.n_refs[b] >= 1:\n                if self.layout == LAYOUT_HISTORY:", 0, 1),
     ("verify_scores_inactive_samples", "if (active is None or active[b]) and self.n_refs[b] >= 1:\n                err[b] =",
      "if self.n_refs[b] >= 1:\n                err[b] =", 0, 1),
     ("verify_compares_fresh_with_itself", "err[b] = rel_err(metric, self.dtype, pred[b], fresh[b], self.eps)",
      "err[b] = rel_err(metric, self.dtype, fresh[b], fresh[b], self.eps)", 0, 1),
+    ("history_appends_instead_of_prepending", "self.hist[e][b] = ([f[b].copy()] + kept)[: self.m + 1]", "self.hist[e][b] = (kept + [f[b].copy()])[: self.m + 1]", 0, 1),
+    ("history_survives_a_reset", "kept = self.hist[e][b] if self.n_refs[b] >= 1 else []   # a reset sample starts over", "kept = self.hist[e][b]", 0, 1),
+    ("history_keeps_one_feature_too_few", "self.hist[e][b] = ([f[b].copy()] + kept)[: self.m + 1]", "self.hist[e][b] = ([f[b].copy()] + kept)[: self.m]", 0, 1),
     ("summed_forecast_skips_the_base", "            if base is not None:\n", "            if False:\n", 0, 1),
 ]
 

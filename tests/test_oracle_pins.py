@@ -776,3 +776,130 @@ def test_cache_verify_scores_the_forecast_against_the_fresh_feature():
     # per-sample thresholds, and the l1 reading through the same call
     err1, acc1, _ = c.verify(fresh, [2.0] * B, [0.0, 0.1, 2.0], metric=O.METRIC_L1)
     assert err1 == pytest.approx(err, rel=1e-9, abs=1e-15) and acc1.tolist() == [1, 0, 1]   # up to epsilon's share
+
+
+# ---------------------------------------------------------------------------------------------
+# the cache that keeps raw features (history layout): Eq. 2-3 evaluated from them at forecast time
+# ---------------------------------------------------------------------------------------------
+
+def history_forecast(dtype, m, basis, times, feats, t_target):
+    """times/feats oldest first; keeps the last m + 1 like the cache does."""
+    hist_t = [float(t) for t in times][::-1][: m + 1]
+    hist_f = [np.ascontiguousarray(f) for f in feats][::-1][: m + 1]
+    out = np.zeros(hist_f[0].size, dtype=O.np_dtype(dtype))
+    O.forecast_history_segment(dtype, m, basis, hist_t, float(t_target), hist_f, out)
+    return out
+
+
+@pytest.mark.parametrize("m", [1, 2, 3, 4])
+@pytest.mark.parametrize("N", [1, 2, 3])
+def test_history_layout_equals_printed_equations_in_rationals(m, N):
+    # any N: nothing is stored between Eq. 3 and Eq. 2, so N = 3 (inexact quotients) works too
+    rng = np.random.default_rng(500 + 10 * m + N)
+    n, t = 23, 40
+    raw = {j: rng.integers(-50, 51, size=n) for j in range(m + 1)}      # F(x_{t+jN})
+    times = [float(t + j * N) for j in range(m, -1, -1)]
+    feats = [raw[j].astype(np.float32) for j in range(m, -1, -1)]
+    for k in [1, 2, 3, 5]:
+        out = history_forecast(O.F32, m, O.TAYLOR, times, feats, t - k)
+        for e in range(n):
+            want = float(eq2_pred(m, N, k, lambda j: Fraction(int(raw[j][e]))))
+            assert float(out[e]) == pytest.approx(want, rel=1.2e-7, abs=1.2e-7)
+
+
+@pytest.mark.parametrize("m", [0, 1, 2, 3, 4])
+def test_history_layout_equals_the_tables_when_nothing_rounds(m):
+    # integer features and power-of-two gaps: every difference quotient is exact in binary32, so keeping
+    # the quotients (tables) or the features (history) must give the same bits; more references than m + 1
+    rng = np.random.default_rng(40 + m)
+    a = O.OracleCache([16], 2, m, O.F32, O.TAYLOR)
+    b = O.OracleCache([16], 2, m, O.F32, O.TAYLOR, layout=O.LAYOUT_HISTORY)
+    t = 64.0
+    for k in range(m + 4):
+        f = [(rng.integers(-8, 8, (2, 16)) * 64).astype(np.float32)]
+        t -= [1.0, 2.0, 4.0][k % 3]
+        for c in (a, b):
+            c.update(f, [t, t - 0.5])
+            c.commit_step()
+        tt = [t - 2.0, t - 1.0]
+        assert np.array_equal(a.forecast_entry(0, tt), b.forecast_entry(0, tt)), k
+        ea, aa, _ = a.verify(f[0], tt, [0.5, 0.5])
+        eb, ab, _ = b.verify(f[0], tt, [0.5, 0.5])
+        assert ea == pytest.approx(eb, rel=1e-12) and np.array_equal(aa, ab)   # same forecasts; the sum's order may vary
+
+
+@pytest.mark.parametrize("basis", [O.TAYLOR, O.NEWTON, O.ADAMS_BASHFORTH])
+@pytest.mark.parametrize("dtype", [O.F32, O.BF16])
+def test_history_layout_tracks_the_tables_within_their_rounding(basis, dtype):
+    # general inputs: the two layouts differ only by the tables' rounding of the stored quotients
+    g = torch.Generator().manual_seed(60 + basis)
+    m, B, n = 3, 2, 400
+    a = O.OracleCache([n], B, m, dtype, basis)
+    b = O.OracleCache([n], B, m, dtype, basis, layout=O.LAYOUT_HISTORY)
+    for t in [1.0, 0.93, 0.9, 0.81, 0.78, 0.7]:
+        f = torch.randn(B, n, generator=g)
+        f = [bf16_bits(f) if dtype == O.BF16 else f.numpy().copy()]
+        for c in (a, b):
+            c.update(f, [t, t - 0.004])
+            c.commit_step()
+    x = a.forecast_entry(0, [0.66, 0.65])
+    y = b.forecast_entry(0, [0.66, 0.65])
+    xf, yf = (bits_to_f64(x), bits_to_f64(y)) if dtype == O.BF16 else (x.astype(np.float64), y.astype(np.float64))
+    rel = np.linalg.norm(xf - yf) / np.linalg.norm(yf)
+    assert 0 < rel < (3e-2 if dtype == O.BF16 else 1e-4)   # bf16 quotients amplified by (x / gap)^i
+
+
+@pytest.mark.parametrize("m", [1, 2, 3, 4])
+def test_history_layout_polynomial_exactness(m):
+    rng = np.random.default_rng(70 + m)
+    coef = rng.integers(-4, 5, size=(m + 1, 9)).astype(np.float64)
+    times = [3.0, 2.5, 2.25, 1.5, 1.0, 0.875][: m + 2]
+    poly = lambda t, deg: sum(coef[i] * t ** i for i in range(deg + 1))
+    for tt in [0.5, 0.25, 0.0, 2.0]:
+        # Newton reading: exact up to degree m at any gaps
+        out = history_forecast(O.F32, m, O.NEWTON, times, [poly(t, m).astype(np.float32) for t in times], tt)
+        np.testing.assert_allclose(out.astype(np.float64), poly(tt, m), rtol=2e-6, atol=2e-5)
+        # Eq. 2-3 as printed: exact up to degree 1 at any gaps
+        out = history_forecast(O.F32, m, O.TAYLOR, times, [poly(t, 1).astype(np.float32) for t in times], tt)
+        np.testing.assert_allclose(out.astype(np.float64), poly(tt, 1), rtol=2e-6, atol=2e-5)
+    # order 0 / one reference: plain reuse, bit for bit
+    f = rng.standard_normal(9).astype(np.float32)
+    assert np.array_equal(history_forecast(O.F32, m, O.TAYLOR, [1.0], [f], 0.3), f)
+    assert np.array_equal(history_forecast(O.F32, 0, O.NEWTON, [1.0, 0.9], [f + 1, f], 0.3), f)
+
+
+@pytest.mark.parametrize("m", [1, 2, 3, 4])
+def test_history_layout_adams_bashforth_equals_textbook_formula(m):
+    # uniform spacing h: F + x * sum_j b_j g_j with the slopes g_j = (F_j - F_{j+1}) / h taken from the raw features
+    b = {1: [1.0], 2: [3 / 2, -1 / 2], 3: [23 / 12, -16 / 12, 5 / 12], 4: [55 / 24, -59 / 24, 37 / 24, -9 / 24]}[m]
+    rng = np.random.default_rng(80 + m)
+    h = -0.25
+    times = [2.0 + h * k for k in range(m + 1)]                 # oldest first, time decreasing
+    feats = [rng.integers(-20, 21, 11).astype(np.float32) for _ in times]
+    x = -0.125
+    out = history_forecast(O.F32, m, O.ADAMS_BASHFORTH, times, feats, times[-1] + x)
+    newest_first = [f.astype(np.float64) for f in feats[::-1]]
+    slopes = [(newest_first[j] - newest_first[j + 1]) / h for j in range(m)]
+    want = newest_first[0] + x * sum(bj * gj for bj, gj in zip(b, slopes))
+    np.testing.assert_allclose(out.astype(np.float64), want, rtol=1e-6, atol=1e-5)
+
+
+def test_history_layout_cache_masks_resets_and_zero_gap():
+    rng = np.random.default_rng(90)
+    B, m, n = 3, 2, 12
+    c = O.OracleCache([n], B, m, O.F32, O.TAYLOR, layout=O.LAYOUT_HISTORY)
+    fs = [rng.integers(-9, 10, (B, n)).astype(np.float32) for _ in range(4)]
+    c.update([fs[0]], [4.0] * B); c.commit_step()
+    c.update([fs[1]], [3.0] * B, mask=[1, 0, 1]); c.commit_step()
+    assert c.n_refs == [2, 1, 2] and len(c.hist[0][1]) == 1
+    out = c.forecast_entry(0, [2.0] * B)
+    assert np.array_equal(out[1], fs[0][1])                                   # one reference: reuse
+    assert np.array_equal(out[0], 2 * fs[1][0] - fs[0][0])                     # two: linear extrapolation
+    with pytest.raises(ZeroDivisionError):
+        c.update([fs[2]], [3.0] * B)
+    c.reset([1, 0, 0])
+    c.update([fs[2]], [2.0] * B); c.commit_step()
+    assert c.n_refs == [1, 2, 3] and len(c.hist[0][0]) == 1 and len(c.hist[0][2]) == 3
+    out = c.forecast_entry(0, [1.0] * B, active=[1, 1, 0], out=np.full((B, n), 7.0, dtype=np.float32))
+    assert np.array_equal(out[0], fs[2][0]) and np.all(out[2] == 7.0)
+    assert np.array_equal(out[1], fs[2][1] + (fs[2][1] - fs[0][1]) / (2.0 - 4.0) * (1.0 - 2.0))   # its references: t = 4 and t = 2
