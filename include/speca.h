@@ -102,6 +102,23 @@ typedef enum {
  *   COSINE  1 - <p, f> / (||p||_2 ||f||_2 + eps)     (a distance: 0 = same direction)
  * In every case the sample is accepted iff the value is <= tau, and a NaN rejects.
  */
+/*
+ * What the cache keeps per (entry, sample) in its max_order + 1 planes.
+ * TABLES   the difference quotients of Eq. 3, rewritten at every reference step (the paper's derivative
+ *          tables): an update reads the feature and the old planes and writes all planes.
+ * HISTORY  the raw features of the last max_order + 1 references, in a ring: an update only copies the
+ *          feature into the next plane (2 words per element instead of 2 * order + 2), and Eq. 3's
+ *          differences are folded into per-plane weights on the host when a forecast is asked for:
+ *          out = sum_i w_i * plane_i. Same Eq. 2-3 (and the same Newton / Adams-Bashforth readings), any
+ *          gaps; the results differ from TABLES only in that no intermediate quotient is rounded to the
+ *          storage type. Not available for speca_forecast_multi / speca_forecast_sum and only on the
+ *          default kernel path.
+ */
+typedef enum {
+    SPECA_LAYOUT_TABLES = 0,
+    SPECA_LAYOUT_HISTORY = 1
+} speca_layout_t;
+
 typedef enum {
     SPECA_METRIC_L2 = 0,
     SPECA_METRIC_L1 = 1,
@@ -128,6 +145,7 @@ typedef struct {
     size_t arena_bytes;                /* >= speca_cache_arena_bytes() */
     int32_t device;                    /* CUDA device ordinal that owns the arena */
     int32_t path;                      /* speca_path_t */
+    int32_t layout;                    /* speca_layout_t; 0 = the paper's derivative tables */
 } speca_cache_config_t;
 
 /*

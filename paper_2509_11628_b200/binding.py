@@ -23,6 +23,7 @@ SPECA_F32, SPECA_BF16 = 0, 1
 SPECA_BASIS_TAYLOR, SPECA_BASIS_NEWTON, SPECA_BASIS_ADAMS_BASHFORTH = 0, 1, 2
 SPECA_METRIC_L2, SPECA_METRIC_L1, SPECA_METRIC_LINF, SPECA_METRIC_COSINE = 0, 1, 2, 3
 SPECA_PATH_AUTO, SPECA_PATH_DIRECT, SPECA_PATH_BULK, SPECA_PATH_WIDE = 0, 1, 2, 3
+SPECA_LAYOUT_TABLES, SPECA_LAYOUT_HISTORY = 0, 1
 SPECA_MAX_ORDER, SPECA_MAX_BATCH, SPECA_MAX_ENTRIES, SPECA_MAX_HORIZON = 4, 64, 512, 8
 
 EXPORTS = [
@@ -60,6 +61,7 @@ class CacheConfig(ctypes.Structure):
         ("max_order", ctypes.c_int32), ("dtype", ctypes.c_int32), ("basis", ctypes.c_int32),
         ("verify_entry", ctypes.c_int32), ("eps", ctypes.c_float), ("arena", ctypes.c_void_p),
         ("arena_bytes", ctypes.c_size_t), ("device", ctypes.c_int32), ("path", ctypes.c_int32),
+        ("layout", ctypes.c_int32),
     ]
 
 
@@ -161,10 +163,11 @@ def _check(status: int, handle=None):
         raise SpecaError(status, detail)
 
 
-def _config(entries, batch, max_order, dtype, basis, verify_entry, eps, arena, arena_bytes, device, path):
+def _config(entries, batch, max_order, dtype, basis, verify_entry, eps, arena, arena_bytes, device, path,
+            layout=SPECA_LAYOUT_TABLES):
     arr = (EntryDesc * len(entries))(*[EntryDesc(int(n), int(d)) for n, d in entries])
     cfg = CacheConfig(len(entries), arr, batch, max_order, dtype, basis, verify_entry, eps,
-                      _dev_ptr(arena), arena_bytes, device, path)
+                      _dev_ptr(arena), arena_bytes, device, path, layout)
     cfg._keep = arr
     return cfg
 
@@ -172,15 +175,15 @@ def _config(entries, batch, max_order, dtype, basis, verify_entry, eps, arena, a
 # ---- the entry points, same names as the header ----------------------------------------------------
 
 def speca_cache_arena_bytes(entries, batch, max_order, dtype, basis=SPECA_BASIS_TAYLOR, verify_entry=-1,
-                            path=SPECA_PATH_AUTO) -> int:
-    cfg = _config(entries, batch, max_order, dtype, basis, verify_entry, 0.0, None, 0, 0, path)
+                            path=SPECA_PATH_AUTO, layout=SPECA_LAYOUT_TABLES) -> int:
+    cfg = _config(entries, batch, max_order, dtype, basis, verify_entry, 0.0, None, 0, 0, path, layout)
     out = ctypes.c_size_t(0)
     _check(_lib().speca_cache_arena_bytes(ctypes.byref(cfg), ctypes.byref(out)))
     return out.value
 
 
 def speca_cache_create(entries, batch, max_order, dtype, arena, basis=SPECA_BASIS_TAYLOR, verify_entry=-1,
-                       eps=0.0, device=None, path=SPECA_PATH_AUTO, arena_bytes=None) -> int:
+                       eps=0.0, device=None, path=SPECA_PATH_AUTO, arena_bytes=None, layout=SPECA_LAYOUT_TABLES) -> int:
     """Returns the opaque handle (an integer address). ``arena`` is a CUDA uint8 tensor the caller
     keeps alive, or a raw device address together with ``arena_bytes``."""
     if isinstance(arena, torch.Tensor):
@@ -189,7 +192,7 @@ def speca_cache_create(entries, batch, max_order, dtype, arena, basis=SPECA_BASI
         if arena_bytes is None:
             arena_bytes = arena.numel() * arena.element_size()
     cfg = _config(entries, batch, max_order, dtype, basis, verify_entry, eps, arena, arena_bytes or 0,
-                  device or 0, path)
+                  device or 0, path, layout)
     out = ctypes.c_void_p(None)
     _check(_lib().speca_cache_create(ctypes.byref(cfg), ctypes.byref(out)))
     return out.value
@@ -354,16 +357,17 @@ class SpecaCache:
     """Owns an arena tensor and a handle; forwards to the entry points above."""
 
     def __init__(self, entries, batch, max_order, dtype, device="cuda:0", basis=SPECA_BASIS_TAYLOR,
-                 verify_entry=-1, eps=0.0, path=SPECA_PATH_AUTO):
+                 verify_entry=-1, eps=0.0, path=SPECA_PATH_AUTO, layout=SPECA_LAYOUT_TABLES):
         self.entries = [(int(n), int(d)) for n, d in entries]
         self.batch, self.max_order, self.dtype, self.basis = batch, max_order, dtype, basis
+        self.layout = layout
         self.device = torch.device(device)
         self.verify_entry = verify_entry if verify_entry >= 0 else len(self.entries) - 1
-        nbytes = speca_cache_arena_bytes(self.entries, batch, max_order, dtype, basis, verify_entry, path)
+        nbytes = speca_cache_arena_bytes(self.entries, batch, max_order, dtype, basis, verify_entry, path, layout)
         self.arena = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
         assert self.arena.data_ptr() % 256 == 0
         self.handle = speca_cache_create(self.entries, batch, max_order, dtype, self.arena, basis, verify_entry,
-                                         eps, self.device.index or 0, path)
+                                         eps, self.device.index or 0, path, layout=layout)
 
     def close(self):
         if self.handle:

@@ -43,6 +43,10 @@ speca_status_t make_layout_impl(const speca_cache_config_t* cfg, Layout* L) {
         cfg->path != SPECA_PATH_WIDE)
         return SPECA_ERR_INVALID_ARG;
     if (cfg->verify_entry < -1 || cfg->verify_entry >= cfg->n_entries) return SPECA_ERR_INVALID_ARG;
+    if (cfg->layout != SPECA_LAYOUT_TABLES && cfg->layout != SPECA_LAYOUT_HISTORY) return SPECA_ERR_INVALID_ARG;
+    // the raw-feature cache runs on the default kernels only
+    if (cfg->layout == SPECA_LAYOUT_HISTORY && cfg->path != SPECA_PATH_AUTO && cfg->path != SPECA_PATH_WIDE)
+        return SPECA_ERR_UNSUPPORTED;
     const size_t esz = cfg->dtype == SPECA_BF16 ? 2 : 4;
     const size_t n_segs = static_cast<size_t>(cfg->n_entries) * cfg->batch;
     const int B = cfg->batch, m = cfg->max_order;
@@ -122,7 +126,7 @@ struct DeviceGuard {
 }  // namespace
 
 struct speca_cache {
-    int n_entries, B, m, dtype, basis, verify_entry, device, path;
+    int n_entries, B, m, dtype, basis, verify_entry, device, path, layout;
     double eps;
     char* arena;
     Layout L;
@@ -193,6 +197,62 @@ void forecast_scalars(const speca_cache* c, int b, double t, int* order, float* 
     }
 }
 
+// SPECA_LAYOUT_HISTORY: the planes hold the features of the last references, the one of age j (0 =
+// latest) in physical plane (references - 1 - j) mod (m + 1). The table a SPECA_LAYOUT_TABLES cache
+// would hold is a linear map of those features: run Eq. 3's recursion on unit vectors, oldest feature
+// first, to get the map; weigh its rows as the basis weighs the planes (Eq. 2); the result is one weight
+// per stored feature, scattered to physical plane order. The forecast is sum_i w[i] * plane_i, i <= order.
+void history_weights(const speca_cache* c, int b, double t, int* order, float* w) {
+    const int refs = c->n_refs[b];
+    const int v = refs < 1 ? -1 : (refs - 1 < c->m ? refs - 1 : c->m);
+    *order = v;
+    for (int i = 0; i < kCoef; ++i) w[i] = 0.f;
+    if (v < 0) return;
+    const double* th = c->t_hist[b];
+    double rows[kCoef][kCoef] = {};  // rows[i][j]: share of the feature of age j in plane i
+    rows[0][v] = 1.0;
+    for (int k = v - 1; k >= 0; --k) {  // fold in the feature of age k; v - k references came before it
+        double next[kCoef][kCoef] = {};
+        next[0][k] = 1.0;
+        for (int i = 0; i < v - k; ++i) {
+            const double gap = th[k] - (c->basis == SPECA_BASIS_NEWTON ? th[k + 1 + i] : th[k + 1]);
+            for (int j = 0; j <= v; ++j) next[i + 1][j] = (next[i][j] - rows[i][j]) / gap;
+        }
+        for (int i = 0; i <= v - k; ++i)
+            for (int j = 0; j <= v; ++j) rows[i][j] = next[i][j];
+    }
+    double plane_w[kCoef];
+    plane_w[0] = 1.0;
+    if (c->basis == SPECA_BASIS_NEWTON) {
+        for (int i = 1; i <= v; ++i) plane_w[i] = plane_w[i - 1] * (t - th[i - 1]);
+    } else if (c->basis == SPECA_BASIS_ADAMS_BASHFORTH) {
+        static const double collected[SPECA_MAX_ORDER] = {1.0, 1.0 / 2, 5.0 / 12, 3.0 / 8};
+        const double x = t - th[0], h = v >= 2 ? th[0] - th[1] : 0.0;
+        double hp = 1.0;
+        for (int i = 1; i <= v; ++i) {
+            plane_w[i] = x * collected[i - 1] * hp;
+            hp *= h;
+        }
+    } else {
+        const double x = t - th[0];
+        for (int i = 1; i <= v; ++i) plane_w[i] = plane_w[i - 1] * x / i;
+    }
+    const int ring = c->m + 1;
+    for (int j = 0; j <= v; ++j) {
+        double a = 0.0;
+        for (int i = 0; i <= v; ++i) a += plane_w[i] * rows[i][j];
+        w[((refs - 1 - j) % ring + ring) % ring] = static_cast<float>(a);
+    }
+}
+
+// Scalars of a forecast for sample b, whichever layout the cache has.
+void forecast_coefficients(const speca_cache* c, int b, double t, int* order, float* coef) {
+    if (c->layout == SPECA_LAYOUT_HISTORY)
+        history_weights(c, b, t, order, coef);
+    else
+        forecast_scalars(c, b, t, order, coef);
+}
+
 }  // namespace
 
 extern "C" {
@@ -245,6 +305,7 @@ speca_status_t speca_cache_create(const speca_cache_config_t* cfg, speca_cache_t
     c->m = cfg->max_order;
     c->dtype = cfg->dtype;
     c->basis = cfg->basis;
+    c->layout = cfg->layout;
     c->verify_entry = cfg->verify_entry < 0 ? cfg->n_entries - 1 : cfg->verify_entry;
     c->device = cfg->device;
     c->path = cfg->path == SPECA_PATH_AUTO ? SPECA_PATH_WIDE : cfg->path;
@@ -349,6 +410,12 @@ speca_status_t speca_cache_update(speca_cache_t* c, const void* const* feats, co
             p.coef[b][i] = static_cast<float>(1.0 / gap);
         }
         p.order[b] = static_cast<int8_t>(v_new);
+        if (c->layout == SPECA_LAYOUT_HISTORY) {
+            // nothing is differenced now: the feature is copied into the plane after the latest one
+            // (the gaps above were only checked, so that no later forecast divides by zero)
+            p.order[b] = 0;
+            p.slot[b] = static_cast<uint8_t>(c->n_refs[b] % (c->m + 1));
+        }
     }
     int e_lo = -1, e_hi = -1;
     const size_t esz = elem_size(c);
@@ -425,7 +492,7 @@ speca_status_t speca_forecast(speca_cache_t* c, const double* t_target, const ui
     for (int b = 0; b < c->B; ++b) {
         if (!std::isfinite(t_target[b])) return fail(c, SPECA_ERR_INVALID_ARG, "forecast: t_target[%d] not finite", b);
         int order;
-        forecast_scalars(c, b, t_target[b], &order, p.coef[b]);
+        forecast_coefficients(c, b, t_target[b], &order, p.coef[b]);
         if (order < 0 && dev_active_mask == nullptr)
             return fail(c, SPECA_ERR_STATE, "forecast: sample %d has no committed reference", b);
         p.order[b] = static_cast<int8_t>(order);
@@ -452,6 +519,7 @@ speca_status_t speca_forecast(speca_cache_t* c, const double* t_target, const ui
     p.tile_start = reinterpret_cast<const uint32_t*>(c->arena + L.tiles_off[c->tile_forecast]);
     p.arena = c->arena;
     p.dev_mask = dev_active_mask;
+    p.weighted = c->layout == SPECA_LAYOUT_HISTORY ? 1 : 0;
     p.err_flag = reinterpret_cast<uint32_t*>(c->arena + L.ticket_off) + 1;
     p.seg_lo = static_cast<uint32_t>(e_lo) * c->B;
     p.seg_hi = static_cast<uint32_t>(e_hi + 1) * c->B;
@@ -473,6 +541,8 @@ speca_status_t speca_forecast_multi(speca_cache_t* c, int32_t n_targets, const d
     if (t_targets == nullptr || outs == nullptr) return fail(c, SPECA_ERR_INVALID_ARG, "forecast_multi: null argument");
     if (n_targets < 1 || n_targets > SPECA_MAX_HORIZON)
         return fail(c, SPECA_ERR_INVALID_ARG, "forecast_multi: n_targets must be 1..%d", SPECA_MAX_HORIZON);
+    if (c->layout != SPECA_LAYOUT_TABLES)
+        return fail(c, SPECA_ERR_UNSUPPORTED, "forecast_multi: only for caches that keep difference tables");
     if (c->pending) return fail(c, SPECA_ERR_STATE, "forecast_multi: a reference step is open (commit it first)");
     static thread_local MultiParams p;  // 13 KB: kept off the stack
     std::memset(&p, 0, sizeof p);
@@ -533,6 +603,8 @@ speca_status_t speca_forecast_sum(speca_cache_t* c, const int32_t* entry_ids, in
     if (entry_ids == nullptr || t_target == nullptr || out == nullptr)
         return fail(c, SPECA_ERR_INVALID_ARG, "forecast_sum: null argument");
     if (n_ids < 1 || n_ids > SPECA_MAX_ENTRIES) return fail(c, SPECA_ERR_INVALID_ARG, "forecast_sum: n_ids out of range");
+    if (c->layout != SPECA_LAYOUT_TABLES)
+        return fail(c, SPECA_ERR_UNSUPPORTED, "forecast_sum: only for caches that keep difference tables");
     if (c->pending) return fail(c, SPECA_ERR_STATE, "forecast_sum: a reference step is open (commit it first)");
     static thread_local SumParams p;
     std::memset(&p, 0, sizeof p);
@@ -623,7 +695,7 @@ static speca_status_t verify_impl(speca_cache_t* c, int32_t metric, const void* 
         if (!std::isfinite(t_target[b])) return fail(c, SPECA_ERR_INVALID_ARG, "verify: t_target[%d] not finite", b);
         if (!partial && std::isnan(tau[b])) return fail(c, SPECA_ERR_INVALID_ARG, "verify: tau[%d] is NaN", b);
         int order;
-        forecast_scalars(c, b, t_target[b], &order, p.coef[b]);
+        forecast_coefficients(c, b, t_target[b], &order, p.coef[b]);
         if (order < 0 && dev_active_mask == nullptr)
             return fail(c, SPECA_ERR_STATE, "verify: sample %d has no committed reference", b);
         p.order[b] = static_cast<int8_t>(order);
@@ -644,6 +716,7 @@ static speca_status_t verify_impl(speca_cache_t* c, int32_t metric, const void* 
     p.segs = reinterpret_cast<const SegDesc*>(c->arena + L.segs_off) + static_cast<size_t>(c->verify_entry) * c->B;
     p.arena = c->arena;
     p.dev_mask = dev_active_mask;
+    p.weighted = c->layout == SPECA_LAYOUT_HISTORY ? 1 : 0;
     p.fresh = static_cast<const char*>(fresh);
     p.out_pred = static_cast<char*>(out_pred);
     p.err = dev_err;

@@ -35,6 +35,10 @@ struct SegDesc {
 };
 static_assert(sizeof(SegDesc) == 32, "SegDesc layout");
 
+// Per-sample scalars of a launch: Horner multipliers or reciprocal gaps (SPECA_MAX_ORDER of them), or the
+// weights of a raw-feature cache (one per plane).
+constexpr int kCoef = SPECA_MAX_ORDER + 1;
+
 // Arguments of the streaming kernels (update, forecast), passed by value as one kernel parameter.
 struct StreamParams {
     const SegDesc* segs;         // all segments of the cache
@@ -47,8 +51,13 @@ struct StreamParams {
     // update:   order = highest plane written (v_new), coef[b][i] = 1 / gap_i
     // forecast: order = highest plane read (v),        coef[b][i] = Horner multiplier of level i+1
     // order < 0: sample is skipped
+    // A cache that keeps raw features (SPECA_LAYOUT_HISTORY):
+    // update:   order = 0, slot[b] = plane that receives the feature
+    // forecast: weighted = 1, coef[b][i] = weight of physical plane i (i <= order): out = sum_i coef_i * plane_i
     int8_t order[SPECA_MAX_BATCH];
-    float coef[SPECA_MAX_BATCH][SPECA_MAX_ORDER];
+    uint8_t slot[SPECA_MAX_BATCH];
+    int32_t weighted;
+    float coef[SPECA_MAX_BATCH][kCoef];
     void* io[SPECA_MAX_ENTRIES];  // per entry: feature (update) or output (forecast); null = skip
 };
 
@@ -106,8 +115,9 @@ struct VerifyParams {
     int32_t batch;
     int32_t metric;  // speca_metric_t
     double eps;
+    int32_t weighted;  // raw-feature cache: coef[b][i] = weight of physical plane i instead of Horner multipliers
     int8_t order[SPECA_MAX_BATCH];
-    float coef[SPECA_MAX_BATCH][SPECA_MAX_ORDER];
+    float coef[SPECA_MAX_BATCH][kCoef];
     float tau[SPECA_MAX_BATCH];
 };
 

@@ -206,9 +206,12 @@ __device__ __forceinline__ uint32_t find_segment(const uint32_t* __restrict__ ti
 // scalar loop. `row` must be W-byte aligned (the planes always are).
 
 // Eq. 2 in Horner form: acc = D_v; acc = D_{i-1} + acc * mu_i for i = v..1.
+// With `weighted` (a cache that keeps raw features) the same planes are combined as a plain weighted
+// sum instead: acc = sum_i w_i * plane_i, w = mu[0..V].
 template <int DT, int V, int W, int NT, int U>
 __device__ __forceinline__ void forecast_tile(const char* __restrict__ plane0, uint64_t stride,
-                                              char* __restrict__ out, uint32_t cnt, const float (&mu)[SPECA_MAX_ORDER]) {
+                                              char* __restrict__ out, uint32_t cnt, const float (&mu)[kCoef],
+                                              bool weighted) {
     constexpr int EPV = W / Elem<DT>::kBytes;
     const uint32_t nvec = cnt / EPV;
     Vec<W> d[V + 1][U];
@@ -226,20 +229,33 @@ __device__ __forceinline__ void forecast_tile(const char* __restrict__ plane0, u
         if (idx < nvec) {
             float acc[EPV];
             unpack_vec<DT, W>(d[V][u], acc);
+            if (weighted) {
+#pragma unroll
+                for (int k = 0; k < EPV; ++k) acc[k] *= mu[V];
+            }
 #pragma unroll
             for (int i = V; i >= 1; --i) {
                 float lo[EPV];
                 unpack_vec<DT, W>(d[i - 1][u], lo);
+                if (weighted) {
 #pragma unroll
-                for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+                    for (int k = 0; k < EPV; ++k) acc[k] = fmaf(lo[k], mu[i - 1], acc[k]);
+                } else {
+#pragma unroll
+                    for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+                }
             }
             store_vec<W>(out + static_cast<size_t>(idx) * W, pack_vec<DT, W>(acc));
         }
     }
     for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += NT) {
         float acc = load_scalar<DT>(plane0 + V * stride, j);
+        if (weighted) acc *= mu[V];
 #pragma unroll
-        for (int i = V; i >= 1; --i) acc = fmaf(acc, mu[i - 1], load_scalar<DT>(plane0 + (i - 1) * stride, j));
+        for (int i = V; i >= 1; --i) {
+            const float lo = load_scalar<DT>(plane0 + (i - 1) * stride, j);
+            acc = weighted ? fmaf(lo, mu[i - 1], acc) : fmaf(acc, mu[i - 1], lo);
+        }
         store_scalar<DT>(out, j, acc);
     }
 }
@@ -248,7 +264,7 @@ __device__ __forceinline__ void forecast_tile(const char* __restrict__ plane0, u
 // V = highest plane written. Reads f and planes 0..V-1, writes planes 0..V, each element once.
 template <int DT, int V, int W, int NT, int U>
 __device__ __forceinline__ void update_tile(char* __restrict__ plane0, uint64_t stride, const char* __restrict__ feat,
-                                            uint32_t cnt, const float (&r)[SPECA_MAX_ORDER]) {
+                                            uint32_t cnt, const float (&r)[kCoef]) {
     constexpr int EPV = W / Elem<DT>::kBytes;
     const uint32_t nvec = cnt / EPV;
     Vec<W> fv[U];
@@ -304,31 +320,39 @@ __device__ __forceinline__ void update_tile(char* __restrict__ plane0, uint64_t 
 // vectors when the row allows it, else one element at a time; planes visited in a loop.
 template <int DT>
 __device__ __noinline__ void forecast_tile_any(const char* __restrict__ plane0, uint64_t stride, char* __restrict__ out,
-                                               uint32_t cnt, int v, const float (&mu)[SPECA_MAX_ORDER]) {
+                                               uint32_t cnt, int v, const float (&mu)[kCoef], bool weighted = false) {
     constexpr int EPV = Elem<DT>::kEPV;
     const bool vec_ok = (reinterpret_cast<uintptr_t>(out) & 15u) == 0;
     const uint32_t nvec = vec_ok ? cnt / EPV : 0;
     for (uint32_t idx = threadIdx.x; idx < nvec; idx += blockDim.x) {
         float acc[EPV];
         unpack<DT>(__ldcs(reinterpret_cast<const uint4*>(plane0 + v * stride) + idx), acc);
+        if (weighted) {
+#pragma unroll
+            for (int k = 0; k < EPV; ++k) acc[k] *= mu[v];
+        }
         for (int i = v; i >= 1; --i) {
             float lo[EPV];
             unpack<DT>(__ldcs(reinterpret_cast<const uint4*>(plane0 + (i - 1) * stride) + idx), lo);
 #pragma unroll
-            for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+            for (int k = 0; k < EPV; ++k) acc[k] = weighted ? fmaf(lo[k], mu[i - 1], acc[k]) : fmaf(acc[k], mu[i - 1], lo[k]);
         }
         __stcs(reinterpret_cast<uint4*>(out) + idx, pack<DT>(acc));
     }
     for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += blockDim.x) {
         float acc = load_scalar<DT>(plane0 + v * stride, j);
-        for (int i = v; i >= 1; --i) acc = fmaf(acc, mu[i - 1], load_scalar<DT>(plane0 + (i - 1) * stride, j));
+        if (weighted) acc *= mu[v];
+        for (int i = v; i >= 1; --i) {
+            const float lo = load_scalar<DT>(plane0 + (i - 1) * stride, j);
+            acc = weighted ? fmaf(lo, mu[i - 1], acc) : fmaf(acc, mu[i - 1], lo);
+        }
         store_scalar<DT>(out, j, acc);
     }
 }
 
 template <int DT>
 __device__ __noinline__ void update_tile_any(char* __restrict__ plane0, uint64_t stride, const char* __restrict__ feat,
-                                             uint32_t cnt, int v, const float (&r)[SPECA_MAX_ORDER]) {
+                                             uint32_t cnt, int v, const float (&r)[kCoef]) {
     constexpr int EPV = Elem<DT>::kEPV;
     const bool vec_ok = (reinterpret_cast<uintptr_t>(feat) & 15u) == 0;
     const uint32_t nvec = vec_ok ? cnt / EPV : 0;
@@ -414,7 +438,8 @@ __global__ void __launch_bounds__(NT, MINB) stream_kernel(const __grid_constant_
     SegDesc sd = {};
     int v = -1;
     char* io = nullptr;
-    float coef[SPECA_MAX_ORDER] = {};
+    float coef[kCoef] = {};
+    uint32_t slot = 0;  // history layout, update only: the plane that receives the feature
     for (uint32_t tile = p.tile_lo + blockIdx.x; tile < p.tile_hi; tile += gridDim.x) {
         if (tile >= seg_end) {  // tiles only grow: look forward from the current segment
             seg = find_segment(p.tile_start, seg, p.seg_hi, tile);
@@ -425,13 +450,14 @@ __global__ void __launch_bounds__(NT, MINB) stream_kernel(const __grid_constant_
             io = static_cast<char*>(p.io[sd.entry]);
             if (p.dev_mask != nullptr && p.dev_mask[sd.sample] == 0) v = -1;
 #pragma unroll
-            for (int i = 0; i < SPECA_MAX_ORDER; ++i) coef[i] = p.coef[sd.sample][i];
+            for (int i = 0; i < kCoef; ++i) coef[i] = p.coef[sd.sample][i];
+            slot = p.slot[sd.sample];
         }
         if (v < 0 || io == nullptr) continue;
         const uint32_t elem0 = (tile - seg_first) * kTile;
         const uint32_t cnt = min(kTile, sd.n_elems - elem0);
         const uint64_t byte0 = static_cast<uint64_t>(elem0) * Elem<DT>::kBytes;
-        char* plane0 = p.arena + sd.plane0_off + byte0;
+        char* plane0 = p.arena + sd.plane0_off + slot * sd.plane_stride + byte0;
         char* row = io + sd.io_off + byte0;
         const bool fast = v == V && (reinterpret_cast<uintptr_t>(row) & (W - 1)) == 0;
         if (fast) {
@@ -441,13 +467,13 @@ __global__ void __launch_bounds__(NT, MINB) stream_kernel(const __grid_constant_
                 if constexpr (UPDATE)
                     update_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, row + off, n, coef);
                 else
-                    forecast_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, row + off, n, coef);
+                    forecast_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, row + off, n, coef, p.weighted != 0);
             }
         } else {
             if constexpr (UPDATE)
                 update_tile_any<DT>(plane0, sd.plane_stride, row, cnt, v, coef);
             else
-                forecast_tile_any<DT>(plane0, sd.plane_stride, row, cnt, v, coef);
+                forecast_tile_any<DT>(plane0, sd.plane_stride, row, cnt, v, coef, p.weighted != 0);
         }
     }
 }
@@ -548,7 +574,7 @@ __global__ void __launch_bounds__(NT, MINB) forecast_multi_kernel(const __grid_c
             }
         } else {
             for (int k = 0; k < p.n_targets; ++k) {
-                float m[SPECA_MAX_ORDER];
+                float m[kCoef] = {};
 #pragma unroll
                 for (int i = 0; i < SPECA_MAX_ORDER; ++i) m[i] = p.coef[k][sd.sample][i];
                 forecast_tile_any<DT>(plane0, sd.plane_stride, row + k * target_stride, cnt, v, m);
@@ -826,9 +852,9 @@ __global__ void __launch_bounds__(kBulkThreads) stream_bulk_kernel(const __grid_
         const int s = j % S;
         const BulkSlot d = slots[s];
         if (d.cnt != 0) {
-            float coef[SPECA_MAX_ORDER];
+            float coef[kCoef];
 #pragma unroll
-            for (int i = 0; i < SPECA_MAX_ORDER; ++i) coef[i] = p.coef[d.sample][i];
+            for (int i = 0; i < kCoef; ++i) coef[i] = p.coef[d.sample][i];
             if (d.staged) {
                 const uint32_t parity = (phase_bits >> s) & 1u;
                 bool landed = false;
@@ -957,7 +983,7 @@ struct Metric {
 template <int DT, int V, int W, int U, int M>
 __device__ __forceinline__ void verify_tile(const char* __restrict__ plane0, uint64_t stride,
                                             const char* __restrict__ fresh, char* __restrict__ out_pred, uint32_t cnt,
-                                            const float (&mu)[SPECA_MAX_ORDER], float (&a)[3]) {
+                                            const float (&mu)[kCoef], bool weighted, float (&a)[3]) {
     constexpr int EPV = W / Elem<DT>::kBytes;
     const uint32_t nvec = cnt / EPV;
     Vec<W> d[V + 1][U];
@@ -977,12 +1003,21 @@ __device__ __forceinline__ void verify_tile(const char* __restrict__ plane0, uin
         if (idx < nvec) {
             float acc[EPV], f[EPV];
             unpack_vec<DT, W>(d[V][u], acc);
+            if (weighted) {
+#pragma unroll
+                for (int k = 0; k < EPV; ++k) acc[k] *= mu[V];
+            }
 #pragma unroll
             for (int i = V; i >= 1; --i) {
                 float lo[EPV];
                 unpack_vec<DT, W>(d[i - 1][u], lo);
+                if (weighted) {
 #pragma unroll
-                for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+                    for (int k = 0; k < EPV; ++k) acc[k] = fmaf(lo[k], mu[i - 1], acc[k]);
+                } else {
+#pragma unroll
+                    for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+                }
             }
             // the forecast as the model would consume it: rounded to the storage type
             const Vec<W> pv = pack_vec<DT, W>(acc);
@@ -997,8 +1032,12 @@ __device__ __forceinline__ void verify_tile(const char* __restrict__ plane0, uin
     }
     for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += kThreads) {
         float acc = load_scalar<DT>(plane0 + V * stride, j);
+        if (weighted) acc *= mu[V];
 #pragma unroll
-        for (int i = V; i >= 1; --i) acc = fmaf(acc, mu[i - 1], load_scalar<DT>(plane0 + (i - 1) * stride, j));
+        for (int i = V; i >= 1; --i) {
+            const float lo = load_scalar<DT>(plane0 + (i - 1) * stride, j);
+            acc = weighted ? fmaf(lo, mu[i - 1], acc) : fmaf(acc, mu[i - 1], lo);
+        }
         acc = round_storage<DT>(acc);
         const float f = load_scalar<DT>(fresh, j);
         Metric<M>::fold(acc, f, a);
@@ -1009,7 +1048,7 @@ __device__ __forceinline__ void verify_tile(const char* __restrict__ plane0, uin
 template <int DT, int M>
 __device__ __noinline__ void verify_tile_any(const char* __restrict__ plane0, uint64_t stride,
                                              const char* __restrict__ fresh, char* __restrict__ out_pred, uint32_t cnt,
-                                             int v, const float (&mu)[SPECA_MAX_ORDER], float (&a)[3]) {
+                                             int v, const float (&mu)[kCoef], bool weighted, float (&a)[3]) {
     constexpr int EPV = Elem<DT>::kEPV;
     const bool vec_ok = ((reinterpret_cast<uintptr_t>(fresh) | reinterpret_cast<uintptr_t>(out_pred) |
                           reinterpret_cast<uintptr_t>(plane0)) & 15u) == 0;
@@ -1017,11 +1056,15 @@ __device__ __noinline__ void verify_tile_any(const char* __restrict__ plane0, ui
     for (uint32_t idx = threadIdx.x; idx < nvec; idx += kThreads) {
         float acc[EPV], f[EPV];
         unpack<DT>(__ldcs(reinterpret_cast<const uint4*>(plane0 + v * stride) + idx), acc);
+        if (weighted) {
+#pragma unroll
+            for (int k = 0; k < EPV; ++k) acc[k] *= mu[v];
+        }
         for (int i = v; i >= 1; --i) {
             float lo[EPV];
             unpack<DT>(__ldcs(reinterpret_cast<const uint4*>(plane0 + (i - 1) * stride) + idx), lo);
 #pragma unroll
-            for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+            for (int k = 0; k < EPV; ++k) acc[k] = weighted ? fmaf(lo[k], mu[i - 1], acc[k]) : fmaf(acc[k], mu[i - 1], lo[k]);
         }
         const uint4 pv = pack<DT>(acc);
         unpack<DT>(pv, acc);
@@ -1034,7 +1077,11 @@ __device__ __noinline__ void verify_tile_any(const char* __restrict__ plane0, ui
     }
     for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += kThreads) {
         float acc = load_scalar<DT>(plane0 + v * stride, j);
-        for (int i = v; i >= 1; --i) acc = fmaf(acc, mu[i - 1], load_scalar<DT>(plane0 + (i - 1) * stride, j));
+        if (weighted) acc *= mu[v];
+        for (int i = v; i >= 1; --i) {
+            const float lo = load_scalar<DT>(plane0 + (i - 1) * stride, j);
+            acc = weighted ? fmaf(lo, mu[i - 1], acc) : fmaf(acc, mu[i - 1], lo);
+        }
         acc = round_storage<DT>(acc);
         const float f = load_scalar<DT>(fresh, j);
         Metric<M>::fold(acc, f, a);
@@ -1182,9 +1229,9 @@ __global__ void __launch_bounds__(kThreads, 2) verify_kernel(const __grid_consta
             const int b = nth_set_bit(bits, a);
             const int v = p.order[b];
             const SegDesc sd = p.segs[b];
-            float mu[SPECA_MAX_ORDER];
+            float mu[kCoef];
 #pragma unroll
-            for (int i = 0; i < SPECA_MAX_ORDER; ++i) mu[i] = p.coef[b][i];
+            for (int i = 0; i < kCoef; ++i) mu[i] = p.coef[b][i];
             const uint32_t first = max(t_lo, a * tps) - a * tps, last = min(t_hi, (a + 1) * tps) - a * tps;
             for (uint32_t tile = first + crank; tile < last; tile += csize) {
                 const uint32_t elem0 = tile * kTile;
@@ -1196,9 +1243,9 @@ __global__ void __launch_bounds__(kThreads, 2) verify_kernel(const __grid_consta
                 const bool fast = v == V && ((reinterpret_cast<uintptr_t>(plane0) | reinterpret_cast<uintptr_t>(fresh) |
                                               reinterpret_cast<uintptr_t>(pred)) & (W - 1)) == 0;
                 if (fast)
-                    verify_tile<DT, V, W, U, M>(plane0, sd.plane_stride, fresh, pred, cnt, mu, acc);
+                    verify_tile<DT, V, W, U, M>(plane0, sd.plane_stride, fresh, pred, cnt, mu, p.weighted != 0, acc);
                 else
-                    verify_tile_any<DT, M>(plane0, sd.plane_stride, fresh, pred, cnt, v, mu, acc);
+                    verify_tile_any<DT, M>(plane0, sd.plane_stride, fresh, pred, cnt, v, mu, p.weighted != 0, acc);
             }
             flush(b);
         }

@@ -61,13 +61,14 @@ class Pair:
     """A CUDA cache and an oracle cache driven with identical inputs."""
 
     def __init__(self, entries, batch, max_order, dtype, basis=S.SPECA_BASIS_TAYLOR, verify_entry=-1,
-                 device="cuda:0", path=S.SPECA_PATH_AUTO):
+                 device="cuda:0", path=S.SPECA_PATH_AUTO, layout=S.SPECA_LAYOUT_TABLES):
         self.entries = list(entries)
         self.B, self.m, self.dtype, self.basis = batch, max_order, dtype, basis
         self.device = torch.device(device)
         self.tdt = torch.bfloat16 if dtype == S.SPECA_BF16 else torch.float32
-        self.gpu = S.SpecaCache(entries, batch, max_order, dtype, device, basis, verify_entry, path=path)
-        self.cpu = O.OracleCache([n * d for n, d in entries], batch, max_order, dtype, basis, verify_entry)
+        self.layout = layout
+        self.gpu = S.SpecaCache(entries, batch, max_order, dtype, device, basis, verify_entry, path=path, layout=layout)
+        self.cpu = O.OracleCache([n * d for n, d in entries], batch, max_order, dtype, basis, verify_entry, layout=layout)
         self.vidx = self.gpu.verify_entry
 
     def close(self):
@@ -92,6 +93,15 @@ class Pair:
 
     def check_tables(self, what="tables"):
         torch.cuda.synchronize()
+        if self.layout == S.SPECA_LAYOUT_HISTORY:
+            # the planes hold copies of the last features: age j sits in plane (references - 1 - j) mod (m + 1)
+            for e in range(len(self.entries)):
+                for b in range(self.B):
+                    got = to_oracle(self.gpu.plane_tensor(e, b))
+                    for j, want in enumerate(self.cpu.hist[e][b][: min(self.cpu.n_refs[b], self.m + 1)]):
+                        phys = (self.cpu.n_refs[b] - 1 - j) % (self.m + 1)
+                        assert np.array_equal(got[phys], want), "%s entry %d sample %d age %d" % (what, e, b, j)
+            return
         for e in range(len(self.entries)):
             for b in range(self.B):
                 v = min(self.m, self.cpu.n_refs[b] - 1)
@@ -111,6 +121,8 @@ class Pair:
         """Overwrite the GPU tables with the oracle's bits so that both sides continue from the same
         state (a one-ulp rounding flip in a stored plane would otherwise be amplified by 1/gap at
         the next reference step and hide real errors behind a loose tolerance)."""
+        if self.layout == S.SPECA_LAYOUT_HISTORY:
+            return  # the planes are bit-exact copies of the features: nothing can drift
         for e in range(len(self.entries)):
             for b in range(self.B):
                 src = torch.from_numpy(self.cpu.planes[e][b].view(np.int16) if self.dtype == O.BF16
@@ -126,6 +138,15 @@ class Pair:
             return 0.0
         gaps = [abs(h[0] - h[j]) for j in range(1, len(h))]
         return 1.0 / min(gaps)
+
+    def history_scale(self, e, b, t):
+        """sum_j |a_j * F_j| per element for the raw-feature cache: the weight a_j of the feature of age j
+        is read off by forecasting one-hot features."""
+        k = min(self.cpu.n_refs[b], self.m + 1)
+        unit = [np.eye(k, dtype=np.float32)[j].copy() for j in range(k)]
+        a = np.zeros(k, dtype=np.float32)
+        O.forecast_history_segment(O.F32, self.m, self.basis, self.cpu.t_hist[b], t, unit, a)
+        return sum(np.abs(as_f64(self.cpu.hist[e][b][j])) * abs(float(a[j])) for j in range(k))
 
     def forecast_weights(self, b, t):
         h = self.cpu.t_hist[b]
@@ -162,7 +183,10 @@ class Pair:
                 if (active is not None and not active[b]) or self.cpu.n_refs[b] < 1:
                     assert np.array_equal(got[b], want[b]), "%s: inactive sample %d of entry %d was written" % (what, b, e)
                     continue
-                scale = term_scale(self.cpu.planes[e][b], self.forecast_weights(b, t_target[b]))
+                if self.layout == S.SPECA_LAYOUT_HISTORY:
+                    scale = self.history_scale(e, b, t_target[b])
+                else:
+                    scale = term_scale(self.cpu.planes[e][b], self.forecast_weights(b, t_target[b]))
                 assert_close_storage(got[b], want[b], self.dtype, scale, "%s entry %d sample %d" % (what, e, b))
         return outs
 
@@ -199,7 +223,10 @@ class Pair:
             else:
                 assert int(a_got[b]) in (0, 1)
             if with_pred:
-                scale = term_scale(self.cpu.planes[self.vidx][b], self.forecast_weights(b, t_target[b]))
+                if self.layout == S.SPECA_LAYOUT_HISTORY:
+                    scale = self.history_scale(self.vidx, b, t_target[b])
+                else:
+                    scale = term_scale(self.cpu.planes[self.vidx][b], self.forecast_weights(b, t_target[b]))
                 assert_close_storage(to_oracle(pred[b]).reshape(-1), p_want[b], self.dtype, scale,
                                      "%s pred sample %d" % (what, b))
         return e_got, a_got, e_want, a_want

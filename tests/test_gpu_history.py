@@ -1,0 +1,145 @@
+"""The cache that keeps raw features (SPECA_LAYOUT_HISTORY): a reference step only copies the feature
+into the next plane of a ring; Eq. 2-3 are evaluated from the stored features at forecast time. Parity
+against the oracle's history layout (which folds the features in double, in the order Eq. 3 does)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import speca_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+RAGGED = [(37, 129), (5, 3), (64, 384), (1, 8192 * 2 + 24), (3, 8192), (1, 1)]
+HIST = 1
+
+
+@pytest.fixture(scope="module")
+def S():
+    from paper_2509_11628_b200 import binding
+    binding._lib()
+    return binding
+
+
+@pytest.fixture(scope="module")
+def U():
+    from tests import gpu_util
+    return gpu_util
+
+
+def rand_feats(entries, B, tdt, gen):
+    return [torch.randn(B, n, d, generator=gen, device=DEV, dtype=torch.float32).to(tdt) for n, d in entries]
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("basis", [0, 1, 2])
+@pytest.mark.parametrize("m", [0, 1, 2, 3, 4])
+def test_ragged_shapes_all_orders(S, U, dtype, basis, m):
+    B = 3
+    gen = torch.Generator(device=DEV).manual_seed(7000 + 10 * m + basis)
+    pair = U.Pair(RAGGED, B, m, dtype, basis, layout=HIST)
+    times = [1.0, 0.93, 0.9, 0.81, 0.8, 0.74, 0.7, 0.66]
+    for step in range(m + 4):                       # past the point where the ring wraps
+        t = [times[step], times[step] - 0.003, times[step] + 0.001]
+        pair.update(rand_feats(RAGGED, B, pair.tdt, gen), t, per_entry_calls=(step % 2 == 1))
+        pair.commit()
+        pair.check_tables("step %d" % step)
+        tt = [times[step] - 0.02, times[step] - 0.035, times[step] - 0.011]
+        pair.check_forecast(tt, what="m=%d basis=%d step %d" % (m, basis, step))
+    outs = pair.check_forecast(tt)
+    n, d = RAGGED[-1] if pair.vidx == len(RAGGED) - 1 else RAGGED[pair.vidx]
+    fresh = (outs[pair.vidx].float() * 1.02).to(pair.tdt)
+    pair.check_verify(fresh, tt, [0.5, 0.01, 0.03])
+    pair.close()
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_masks_resets_and_verification_on_many_tiles(S, U, dtype):
+    entries = [(16, 520), (301, 1160)]
+    B, m = 5, 2
+    gen = torch.Generator(device=DEV).manual_seed(11)
+    pair = U.Pair(entries, B, m, dtype, layout=HIST)
+    clock = 1.0
+    masks = [None, None, [1, 0, 1, 1, 0], None, [0, 1, 1, 0, 1], [1, 1, 0, 0, 0]]
+    for step, mask in enumerate(masks):
+        clock -= 0.04
+        pair.update(rand_feats(entries, B, pair.tdt, gen), [clock - 0.001 * b for b in range(B)], mask)
+        pair.commit()
+        pair.check_tables("masked step %d" % step)
+        if step == 3:
+            pair.gpu.reset([0, 0, 0, 1, 0])
+            pair.cpu.reset([0, 0, 0, 1, 0])
+    n_refs, _ = pair.gpu.state()
+    assert n_refs == pair.cpu.n_refs == [5, 5, 5, 0, 4]
+    act = [1, 1, 1, 0, 1]
+    tt = [clock - 0.03] * B
+    outs = pair.check_forecast(tt, active=act, sentinel=2.5)
+    noise = torch.randn(B, 301, 1160, generator=gen, device=DEV) * torch.tensor([0.0, 0.01, 0.05, 0.2, 1.0], device=DEV).view(B, 1, 1)
+    fresh = (outs[1].float() + noise).to(pair.tdt)
+    for metric in (None, O.METRIC_L1, O.METRIC_LINF, O.METRIC_COSINE):
+        tau = [1e-3] * B if metric == O.METRIC_COSINE else [0.03] * B
+        e, a, _, _ = pair.check_verify(fresh, tt, tau, active=act, metric=metric, ulp_slack=(metric == O.METRIC_LINF))
+    # the fused continuation works on this layout too
+    err = torch.zeros(B, device=DEV); acc = torch.zeros(B, dtype=torch.uint8, device=DEV)
+    cur = torch.tensor(act, dtype=torch.uint8, device=DEV); nxt = torch.zeros(B, dtype=torch.uint8, device=DEV)
+    cnt = torch.zeros(B, dtype=torch.int32, device=DEV)
+    pair.gpu.verify_select(fresh, tt, [0.03] * B, err, acc, cur, nxt, 3, 1, cnt)
+    torch.cuda.synchronize()
+    _, a_want, _ = pair.cpu.verify(U.to_oracle(fresh).reshape(B, -1), tt, [0.03] * B, act)
+    want_act, want_cnt, _ = O.select_adaptive([max(int(a), 0) for a in a_want], 3, 1, [0] * B, act)
+    assert nxt.cpu().tolist() == want_act and cnt.cpu().tolist() == want_cnt
+    assert want_act[0] == 1 and want_act[3] == 0 and want_act[4] == 0     # exact match kept; inactive and noisy dropped
+    pair.close()
+
+
+def test_an_update_moves_two_words_per_element_and_other_calls_are_refused(S):
+    entries = [(8, 64), (4, 32)]
+    B = 2
+    c = S.SpecaCache(entries, B, 2, 1, DEV, layout=HIST)
+    f = [torch.ones(B, n, d, dtype=torch.bfloat16, device=DEV) for n, d in entries]
+    for t in (1.0, 0.9, 0.8, 0.7):
+        c.update([x * t for x in f], [t] * B)
+        c.commit_step()
+    torch.cuda.synchronize()
+    # four references in a ring of three planes: 0.7 overwrote 1.0 in plane 0
+    planes = c.plane_tensor(0, 1).float().cpu()
+    assert torch.allclose(planes[:, 0], torch.tensor([0.7, 0.9, 0.8]), atol=4e-3)
+    outs = [torch.zeros_like(x) for x in f]
+    c.forecast([0.6] * B, outs)
+    torch.cuda.synchronize()
+    assert torch.allclose(outs[0].float().cpu(), torch.full((B, 8, 64), 0.6), atol=8e-3)   # linear in t: exact
+
+    def status_of(fn):
+        with pytest.raises(S.SpecaError) as ei:
+            fn()
+        return ei.value.status
+
+    multi = [torch.zeros(2, B, n, d, dtype=torch.bfloat16, device=DEV) for n, d in entries]
+    assert status_of(lambda: c.forecast_multi([[0.6] * B, [0.5] * B], multi)) == S.SPECA_ERR_UNSUPPORTED
+    assert status_of(lambda: c.forecast_sum([0], [0.6] * B, outs[0])) == S.SPECA_ERR_UNSUPPORTED
+    assert status_of(lambda: c.update(f, [0.7] * B)) == S.SPECA_ERR_ZERO_GAP
+    assert status_of(lambda: S.SpecaCache(entries, B, 2, 1, DEV, path=S.SPECA_PATH_BULK, layout=HIST)) == S.SPECA_ERR_UNSUPPORTED
+    c.close()
+
+
+def test_history_and_tables_agree_on_exactly_representable_inputs(S):
+    # integer features, power-of-two gaps, fp32, order 2 (x^2 / 2 is dyadic; order 3 would bring in thirds):
+    # both layouts compute the same numbers without any rounding, so they must agree bit for bit
+    entries = [(33, 130)]
+    B, m = 2, 2
+    gen = torch.Generator(device=DEV).manual_seed(3)
+    a = S.SpecaCache(entries, B, m, 0, DEV)
+    b = S.SpecaCache(entries, B, m, 0, DEV, layout=HIST)
+    t = 64.0
+    for k in range(7):
+        f = [(torch.randint(-8, 8, (B, 33, 130), generator=gen, device=DEV) * 64).float()]
+        t -= [1.0, 2.0, 4.0][k % 3]
+        for c in (a, b):
+            c.update(f, [t, t - 0.5])
+            c.commit_step()
+        oa, ob = [torch.zeros_like(f[0])], [torch.zeros_like(f[0])]
+        a.forecast([t - 2.0, t - 1.0], oa)
+        b.forecast([t - 2.0, t - 1.0], ob)
+        torch.cuda.synchronize()
+        assert torch.equal(oa[0], ob[0]), k
+    a.close(); b.close()
