@@ -56,15 +56,16 @@ def make_workload(name: str) -> W.Workload:
     return W.BY_NAME[name]()
 
 
-def algorithmic_bytes(w: W.Workload, order: int):
+def algorithmic_bytes(w: W.Workload, order: int, layout: int = 0):
     """Bytes a step must move per kernel, from the per-element figures: update reads the feature
-    and `order` old planes and writes order+1 planes; forecast reads order+1 planes and writes one;
-    verify reads order+1 planes and the fresh feature."""
+    and `order` old planes and writes order+1 planes (a cache that keeps raw features, layout 1, reads
+    the feature and writes one plane); forecast reads order+1 planes and writes one; verify reads
+    order+1 planes and the fresh feature."""
     eb = w.elem_bytes
     n_all = w.elems_per_order
     n_ver = w.batch * w.entry_elems(w.vidx)
     return {
-        "update": (2 * order + 2) * eb * n_all,
+        "update": (2 if layout == 1 else 2 * order + 2) * eb * n_all,
         "forecast": (order + 2) * eb * n_all,
         "verify": (order + 2) * eb * n_ver,
         "select": 0,
@@ -134,12 +135,13 @@ def physical_gpu_index(local_index: int) -> int:
 class Harness:
     """Device-resident state for one workload: cache, two alternating feature sets, outputs."""
 
-    def __init__(self, w: W.Workload, device: str, seed_offset: int = 0, path: int = 0, fused_select: bool = True):
+    def __init__(self, w: W.Workload, device: str, seed_offset: int = 0, path: int = 0, fused_select: bool = True,
+                 layout: int = 0):
         from paper_2509_11628_b200 import binding as S
         self.S, self.w, self.device = S, w, torch.device(device)
         self.fused_select = fused_select
         self.B, self.m = w.batch, w.max_order
-        self.cache = S.SpecaCache(w.entries, w.batch, w.max_order, w.dtype, device, path=path)
+        self.cache = S.SpecaCache(w.entries, w.batch, w.max_order, w.dtype, device, path=path, layout=layout)
         self.src = W.FeatureSource(w, device, seed_offset)
         ne = len(w.entries)
         # warm the tables with max_order + 1 fully computed steps of the generator
@@ -689,8 +691,8 @@ def workload_config(w: W.Workload):
     }
 
 
-def summarize(w, per_ms, total_ms, steps, n_gpus, peak):
-    ab = algorithmic_bytes(w, w.max_order)
+def summarize(w, per_ms, total_ms, steps, n_gpus, peak, layout=0):
+    ab = algorithmic_bytes(w, w.max_order, layout)
     step_bytes = ab["update"] + ab["forecast"] + ab["verify"]
     ms_step = total_ms / steps
     kernels = {}
@@ -704,6 +706,23 @@ def summarize(w, per_ms, total_ms, steps, n_gpus, peak):
     return value, ms_step, kernels, {"speculative_steps_per_s": 1e3 / spec_ms, "forecast_verify_gbs": fv_gbs,
                                      "forecast_verify_frac_of_nominal_8TBs": fv_gbs / NOMINAL_HBM_GBS,
                                      "forecast_verify_frac_of_measured_peak": fv_gbs / peak}
+
+
+def time_history_layout(w, device, path, steps, info, peak, tables_ms_step, tables_kernels):
+    """The same step on a cache that keeps the raw features of the last references instead of the
+    difference tables (SPECA_LAYOUT_HISTORY): the reference step becomes one copy."""
+    h = Harness(w, device, path=path, layout=1)
+    total_ms, per_ms, _, _ = time_device_resident(h, steps, 3, info, False)
+    value, ms_step, kernels, extra = summarize(w, per_ms, total_ms, steps, 1, peak, layout=1)
+    h.close()
+    del h
+    torch.cuda.empty_cache()
+    return {"ms_per_step": ms_step, "value": value, "unit": "GB/s", "kernels": kernels,
+            "speculative_steps_per_s": extra["speculative_steps_per_s"],
+            "update_ms_tables_layout": tables_kernels["update"]["ms"],
+            "update_speedup_vs_tables_layout": tables_kernels["update"]["ms"] / kernels["update"]["ms"],
+            "step_speedup_vs_tables_layout": tables_ms_step / ms_step,
+            "note": "update moves 2 words per element instead of 2 * order + 2; forecast and verify move the same bytes"}
 
 
 def main():
@@ -769,6 +788,13 @@ def main():
     del h
     torch.cuda.empty_cache()
 
+    history = None
+    if info.world == 1 and path in (0, 3):
+        try:
+            history = time_history_layout(w, device, path, min(args.steps, 100), info, peak, ms_step, kernels)
+        except Exception as exc:  # report, do not hide
+            history = {"error": repr(exc)}
+
     per_config = {}
     if info.world == 1:
         for name in [n for n in args.also.split(",") if n and n != args.config]:
@@ -786,6 +812,8 @@ def main():
                 h2.close()
                 del h2
                 torch.cuda.empty_cache()
+                if path in (0, 3):
+                    per_config[name]["history_layout"] = time_history_layout(w2, device, path, k2, info, peak, ms2, kern2)
             except Exception as exc:  # report, do not hide
                 per_config[name] = {"error": repr(exc)}
 
@@ -851,7 +879,7 @@ def main():
         "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches,
         "clocks": clocks, "kernels": kernels, **extra,
         "frac_of_measured_peak": value / info.world / peak, "frac_of_nominal_8TBs": value / info.world / NOMINAL_HBM_GBS,
-        "multi_horizon": multi, "verify_metrics": metrics, "update_one_launch_per_entry": per_entry, "forecast_sum": fsum, "per_config": per_config, "adaptive": adaptive, "sampler": sampler,
+        "multi_horizon": multi, "verify_metrics": metrics, "update_one_launch_per_entry": per_entry, "forecast_sum": fsum, "history_layout": history, "per_config": per_config, "adaptive": adaptive, "sampler": sampler,
         "paper_context": {"end_to_end_speedups": {"flux_h800": 6.34, "dit_xl2_a800": 7.3, "hunyuan_video_h800": 6.1},
                           "verification_overhead": "1.67%-3.5% of a full forward pass",
                           "note": "other hardware, whole-model numbers; context only"},

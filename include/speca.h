@@ -401,6 +401,17 @@ speca_status_t speca_cache_plane(const speca_cache_t* cache, int32_t entry, int3
                                  size_t* plane_stride_bytes);
 
 /*
+ * SPECA_LAYOUT_HISTORY only: device address of the plane that the next reference step of `sample` will
+ * fill for `entry` (N_e * D elements of the storage type, 4 KB aligned). A model that writes its block
+ * output there directly, and then passes that same address (minus sample * N_e * D elements, i.e. the
+ * address a [B, N_e, D] tensor would need for the row to land there; for B = 1 simply the address
+ * itself) as feats[entry] to speca_cache_update, pays nothing for the reference step: the entry is
+ * recognised as already in place and not copied. The address changes after every committed step of
+ * that sample. Errors: INVALID_ARG, UNSUPPORTED (a cache that keeps difference tables).
+ */
+speca_status_t speca_cache_next_slot(const speca_cache_t* cache, int32_t entry, int32_t sample, void** out);
+
+/*
  * Host-side counters of a handle since it was created (nothing here is read back from the device, so
  * the call neither launches nor synchronises). Launch counts are per kernel kind; the fused
  * verify + continuation call counts as one verify launch. reference_steps[b] counts committed

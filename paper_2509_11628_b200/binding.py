@@ -30,7 +30,7 @@ EXPORTS = [
     "speca_cache_arena_bytes", "speca_cache_create", "speca_cache_destroy", "speca_cache_reset",
     "speca_cache_update", "speca_cache_commit_step", "speca_forecast", "speca_verify",
     "speca_select_adaptive", "speca_activate", "speca_tau", "speca_cache_state", "speca_cache_plane",
-    "speca_cache_launch_count", "speca_cache_stats", "speca_status_string", "speca_last_error", "speca_version",
+    "speca_cache_launch_count", "speca_cache_stats", "speca_cache_next_slot", "speca_status_string", "speca_last_error", "speca_version",
     "speca_verify_pred_static", "speca_forecast_multi", "speca_verify_metric",
     "speca_verify_partial", "speca_verify_decide", "speca_cache_get_history", "speca_cache_set_history",
     "speca_forecast_sum", "speca_verify_select",
@@ -104,6 +104,7 @@ def _lib() -> ctypes.CDLL:
     L.speca_cache_plane.argtypes = [vp, i32, i32, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_size_t)]
     L.speca_cache_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64)]
     L.speca_cache_stats.argtypes = [vp, ctypes.POINTER(CacheStats)]
+    L.speca_cache_next_slot.argtypes = [vp, i32, i32, ctypes.POINTER(vp)]
     L.speca_status_string.argtypes = [i32]
     L.speca_status_string.restype = ctypes.c_char_p
     L.speca_last_error.argtypes = [vp]
@@ -325,6 +326,13 @@ def speca_cache_plane(cache, entry: int, sample: int):
     return p.value, s.value
 
 
+def speca_cache_next_slot(cache, entry: int, sample: int) -> int:
+    """Device address of the plane the next reference step of ``sample`` fills for ``entry`` (raw-feature cache)."""
+    out = ctypes.c_void_p(None)
+    _check(_lib().speca_cache_next_slot(cache, int(entry), int(sample), ctypes.byref(out)), cache)
+    return out.value
+
+
 def speca_cache_stats(cache, batch: int) -> dict:
     """Host-side counters of the handle: launches per kernel kind, reference steps and resets per sample."""
     st = CacheStats()
@@ -434,3 +442,12 @@ class SpecaCache:
 
     def stats(self):
         return speca_cache_stats(self.handle, self.batch)
+
+    def next_slot_tensor(self, entry: int, sample: int = 0) -> torch.Tensor:
+        """The plane that the next reference step of ``sample`` fills, as an ``[N_e, D]`` view of the arena
+        (raw-feature cache): write the block output here and pass it to ``update`` to skip the copy."""
+        ptr = speca_cache_next_slot(self.handle, entry, sample)
+        n, d = self.entries[entry]
+        tdt = torch.bfloat16 if self.dtype == SPECA_BF16 else torch.float32
+        off = ptr - self.arena.data_ptr()
+        return self.arena[off: off + n * d * (2 if self.dtype == SPECA_BF16 else 4)].view(tdt).view(n, d)

@@ -424,6 +424,18 @@ speca_status_t speca_cache_update(speca_cache_t* c, const void* const* feats, co
         if (c->entry_updated[e]) return fail(c, SPECA_ERR_STATE, "update: entry %d already updated in this step", e);
         if (reinterpret_cast<uintptr_t>(feats[e]) % esz != 0)
             return fail(c, SPECA_ERR_ALIGNMENT, "update: feats[%d] not aligned to the element size", e);
+        if (c->layout == SPECA_LAYOUT_HISTORY) {
+            // The model may have written the feature straight into the plane that is next in the ring
+            // (speca_cache_next_slot): then there is nothing to copy for this entry.
+            bool in_place = any_sample;
+            for (int b = 0; b < c->B && in_place; ++b) {
+                if (!mask[b]) continue;
+                const SegDesc& s = c->L.segs[static_cast<size_t>(e) * c->B + b];
+                const char* slot_ptr = c->arena + s.plane0_off + static_cast<size_t>(p.slot[b]) * s.plane_stride;
+                in_place = static_cast<const char*>(feats[e]) + s.io_off == slot_ptr;
+            }
+            if (in_place) continue;  // p.io[e] stays null: the launch skips the entry
+        }
         if (e_lo < 0) e_lo = e;
         e_hi = e;
         p.io[e] = const_cast<void*>(feats[e]);
@@ -891,6 +903,15 @@ speca_status_t speca_cache_plane(const speca_cache_t* c, int32_t entry, int32_t 
     const SegDesc& s = c->L.segs[static_cast<size_t>(entry) * c->B + sample];
     *plane0 = c->arena + s.plane0_off;
     *plane_stride_bytes = s.plane_stride;
+    return SPECA_OK;
+}
+
+speca_status_t speca_cache_next_slot(const speca_cache_t* c, int32_t entry, int32_t sample, void** out) {
+    if (c == nullptr || out == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (c->layout != SPECA_LAYOUT_HISTORY) return SPECA_ERR_UNSUPPORTED;
+    if (entry < 0 || entry >= c->n_entries || sample < 0 || sample >= c->B) return SPECA_ERR_INVALID_ARG;
+    const SegDesc& s = c->L.segs[static_cast<size_t>(entry) * c->B + sample];
+    *out = c->arena + s.plane0_off + static_cast<size_t>(c->n_refs[sample] % (c->m + 1)) * s.plane_stride;
     return SPECA_OK;
 }
 

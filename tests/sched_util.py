@@ -10,9 +10,9 @@ from paper_2509_11628_b200 import workloads as W
 
 
 class OracleBackend:
-    def __init__(self, w: W.Workload, metric: int = O.METRIC_L2):
+    def __init__(self, w: W.Workload, metric: int = O.METRIC_L2, layout: int = O.LAYOUT_TABLES):
         self.w, self.batch, self.metric = w, w.batch, metric
-        self.cache = O.OracleCache([n * d for n, d in w.entries], w.batch, w.max_order, w.dtype)
+        self.cache = O.OracleCache([n * d for n, d in w.entries], w.batch, w.max_order, w.dtype, layout=layout)
         self.reset_run()
 
     def reset_run(self):

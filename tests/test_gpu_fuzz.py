@@ -60,9 +60,12 @@ def test_random_scenario(S, U, seed):
     basis = int(rng.integers(0, 3))
     path = int(rng.integers(0, 4))
     vidx = int(rng.integers(-1, len(entries)))
-    pair = U.Pair(entries, B, m, dtype, basis, verify_entry=vidx, path=path)
+    layout = int(seed % 3 == 2)               # every third scenario runs on the raw-feature cache
+    if layout == 1:
+        path = int(rng.choice([0, 3]))        # which only the default kernels serve
+    pair = U.Pair(entries, B, m, dtype, basis, verify_entry=vidx, path=path, layout=layout)
     nv, dv = entries[pair.vidx]
-    what = "seed %d (B=%d m=%d dtype=%d basis=%d path=%d entries=%s)" % (seed, B, m, dtype, basis, path, entries)
+    what = "seed %d (B=%d m=%d dtype=%d basis=%d path=%d layout=%d entries=%s)" % (seed, B, m, dtype, basis, path, layout, entries)
 
     def feats():
         return [torch.randn(B, n, d, generator=gen, device=DEV, dtype=torch.float32).to(pair.tdt) for n, d in entries]

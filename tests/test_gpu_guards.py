@@ -77,3 +77,39 @@ def test_nothing_is_written_outside_the_buffers(S, path, dtype, tdt, m):
         assert not bool((outs[2].t.view(torch.uint8) == PATTERN).all())       # and the outputs were written
     S.speca_cache_destroy(handle)
     assert arena.intact()
+
+
+@pytest.mark.parametrize("dtype,tdt", [(0, torch.float32), (1, torch.bfloat16)])
+@pytest.mark.parametrize("m", [0, 2, 4])
+def test_nothing_is_written_outside_the_buffers_raw_feature_cache(S, dtype, tdt, m):
+    """The same for a cache that keeps raw features: copies into the ring (past the wrap), weighted
+    forecasts, verification with the continuation rule inside."""
+    B = 3
+    gen = torch.Generator(device=DEV).manual_seed(78)
+    nbytes = S.speca_cache_arena_bytes(RAGGED, B, m, dtype, layout=S.SPECA_LAYOUT_HISTORY)
+    arena = Guarded((nbytes,), torch.uint8, offset=(256 - GUARD % 256) % 256)
+    handle = S.speca_cache_create(RAGGED, B, m, dtype, arena.t, device=0, layout=S.SPECA_LAYOUT_HISTORY)
+    esz = 4 if dtype == 0 else 2
+    for shift in (0, esz):
+        for k in range(m + 3):
+            feats = [Guarded((B, n, d), tdt, offset=shift) for n, d in RAGGED]
+            for f in feats:
+                f.t.copy_(torch.randn(f.t.shape, generator=gen, device=DEV).to(tdt))
+            S.speca_cache_update(handle, [f.t for f in feats], [1.0 - 0.1 * k - shift] * B, [1, k % 2, 1])
+            S.speca_cache_commit_step(handle)
+        outs = [Guarded((B, n, d), tdt, offset=shift) for n, d in RAGGED]
+        t = [0.1 - shift] * B
+        S.speca_forecast(handle, t, None, [o.t for o in outs])
+        n_v, d_v = RAGGED[-1]
+        pred = Guarded((B, n_v, d_v), tdt, offset=shift)
+        err, acc = Guarded((B,), torch.float32), Guarded((B,), torch.uint8)
+        fresh = torch.randn(B, n_v, d_v, generator=gen, device=DEV).to(tdt)
+        cur, nxt = Guarded((B,), torch.uint8, fill=1), Guarded((B,), torch.uint8)
+        spec, idx, n_act = Guarded((B,), torch.int32, fill=0), Guarded((B,), torch.int32), Guarded((1,), torch.int32)
+        S.speca_verify_select(handle, 0, fresh, t, [0.1] * B, cur.t, nxt.t, pred.t, err.t, acc.t, 3, 1, spec.t, idx.t, n_act.t)
+        torch.cuda.synchronize()
+        for g in outs + [pred, err, acc, cur, nxt, spec, idx, n_act, arena]:
+            assert g.intact(), "a guard zone was overwritten (dtype %d, order %d, shift %d)" % (dtype, m, shift)
+        assert not bool((outs[2].t.view(torch.uint8) == PATTERN).all())
+    S.speca_cache_destroy(handle)
+    assert arena.intact()

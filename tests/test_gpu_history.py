@@ -143,3 +143,37 @@ def test_history_and_tables_agree_on_exactly_representable_inputs(S):
         torch.cuda.synchronize()
         assert torch.equal(oa[0], ob[0]), k
     a.close(); b.close()
+
+
+def test_features_written_in_place_cost_no_launch(S, U):
+    """B = 1: the model writes each block output straight into the plane that is next in the ring and
+    hands that address to update: nothing is copied, the reference step launches nothing."""
+    entries = [(37, 129), (64, 384), (3, 8192)]
+    m = 2
+    gen = torch.Generator(device=DEV).manual_seed(23)
+    pair = U.Pair(entries, 1, m, 1, layout=HIST)
+    clock = 1.0
+    for step in range(6):
+        clock -= 0.03 + 0.01 * (step % 2)
+        slots = [pair.gpu.next_slot_tensor(e, 0) for e in range(len(entries))]
+        for s, f in zip(slots, rand_feats(entries, 1, pair.tdt, gen)):
+            s.copy_(f[0])
+        launches = pair.gpu.launches
+        if step == 3:   # one entry handed over from elsewhere: only that one is copied
+            other = slots[1].clone().view(1, *entries[1])
+            pair.update([slots[0].view(1, *entries[0]), other, slots[2].view(1, *entries[2])], [clock])
+            assert pair.gpu.launches == launches + 1
+        else:
+            pair.update([s.view(1, n, d) for s, (n, d) in zip(slots, entries)], [clock])
+            assert pair.gpu.launches == launches
+        pair.commit()
+        pair.check_tables("in place, step %d" % step)
+        pair.check_forecast([clock - 0.02], what="in place, step %d" % step)
+    assert pair.gpu.stats()["update_launches"] == 1 and pair.gpu.stats()["reference_steps"] == [6]
+    # a cache that keeps tables has no such slot
+    c = S.SpecaCache(entries, 1, m, 1, DEV)
+    with pytest.raises(S.SpecaError) as ei:
+        S.speca_cache_next_slot(c.handle, 0, 0)
+    assert ei.value.status == S.SPECA_ERR_UNSUPPORTED
+    c.close()
+    pair.close()

@@ -21,8 +21,9 @@ def S():
     return binding
 
 
-@pytest.mark.parametrize("name,metric", [("dit_xl2", None), ("flux", None), ("dit_xl2", 3)])
-def test_sampler_trace_matches_oracle(S, name, metric):
+@pytest.mark.parametrize("name,metric,layout", [("dit_xl2", None, 0), ("flux", None, 0), ("dit_xl2", 3, 0),
+                                                ("dit_xl2", None, 1), ("flux", None, 1)])   # 1: the raw-feature cache
+def test_sampler_trace_matches_oracle(S, name, metric, layout):
     w = W.scaled(W.BY_NAME[name](), max_entries=3, max_tokens=40)
     if name == "dit_xl2":
         w.batch = 6
@@ -30,10 +31,10 @@ def test_sampler_trace_matches_oracle(S, name, metric):
     w.times = w.times[:30]
     tau0 = {None: w.tau0, 3: 0.02}[metric]
     gamma = 1.0 / 28
-    cache = S.SpecaCache(w.entries, w.batch, w.max_order, w.dtype, DEV)
+    cache = S.SpecaCache(w.entries, w.batch, w.max_order, w.dtype, DEV, layout=layout)
     gpu = SCH.SpecaCacheBackend(cache, metric=metric)
     tr_gpu = SCH.run_sampler(gpu, SU.GeneratorModel(w, DEV), w.times, tau0, w.beta, 4, 3, gamma, total_steps=50)
-    cpu = SU.OracleBackend(w, metric=metric or 0)
+    cpu = SU.OracleBackend(w, metric=metric or 0, layout=layout)
     tr_cpu = SCH.run_sampler(cpu, SU.GeneratorModel(w, DEV, SU.to_oracle_array), w.times, tau0, w.beta, 4, 3, gamma,
                              total_steps=50)
     n_spec, parted = 0, False
@@ -42,9 +43,15 @@ def test_sampler_trace_matches_oracle(S, name, metric):
             eg, ec = tr_gpu.err[i][b], tr_cpu.err[i][b]
             if rc[b] != SCH.FULL:
                 # unlike the single-call tests the tables are not re-synchronised between steps, so a
-                # one-ulp rounding flip in a stored plane may move a later error by a little more than 1e-4
-                assert abs(eg - ec) <= ERR_TOL * max(1.0, ec) + 1e-3 * ec, (i, b, eg, ec)
-                if abs(ec - tr_cpu.tau[i]) < ERR_TOL + 1e-3 * ec:
+                # one-ulp rounding flip in a stored plane may move a later error by a little more than 1e-4.
+                # The raw-feature cache has no stored quotients to drift, but on this exactly uniform time
+                # grid its weights are ratios of small integers (25/18, -10/18, 3/18, ...), a few per cent
+                # of the bf16 forecasts are exact ties, and fp32 weights break them by the sign of their
+                # 1e-8 error where the oracle (double, then binary32) rounds them to even: every element
+                # still agrees within one storage ulp, the error moves by up to a few 1e-3 of itself.
+                slack = (1e-3 if layout == 0 else 6e-3) * ec
+                assert abs(eg - ec) <= ERR_TOL * max(1.0, ec) + slack, (i, b, eg, ec)
+                if abs(ec - tr_cpu.tau[i]) < ERR_TOL + slack:
                     parted = True      # a decision within the tolerance of its threshold: the runs may part ways
                     break
                 n_spec += 1
