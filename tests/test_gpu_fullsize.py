@@ -197,3 +197,84 @@ def test_full_size_config_on_sampled_blocks(S, U, name, kw, path):
             else:
                 assert bool((row == five).all()), "%s: inactive sample %d of entry %d was written" % (name, b, e)
     cache.close()
+
+
+@pytest.mark.parametrize("name", ["dit_xl2", "flux"])
+def test_full_size_raw_feature_cache_on_sampled_blocks(S, U, name):
+    """The same at full size for the cache that keeps raw features: reference steps past the point where
+    the ring wraps (every element: the newest plane is the feature, bit for bit), forecast of every entry
+    in one launch against the oracle on the sampled blocks, Eq. 4 on the whole verification entry, and
+    the k = 0 property on every element."""
+    w = W.BY_NAME[name]()
+    B, m, ne = w.batch, w.max_order, len(w.entries)
+    rng = np.random.default_rng(4321 + w.index)
+    blocks = choose_blocks(w, rng)
+    src = W.FeatureSource(w, DEV)
+    cache = S.SpecaCache(w.entries, B, m, w.dtype, DEV, layout=S.SPECA_LAYOUT_HISTORY)
+    tdt = w.torch_dtype
+    it = torch.int16 if w.dtype == W.BF16 else torch.int32
+    kept = {(e, blk): [] for e, lst in blocks.items() for blk in lst}      # raw feature blocks, latest first
+    hist = []
+    n_steps = m + 2
+    for step in range(n_steps):
+        t = [w.times[step]] * B
+        feats = [src.feature(e, step, t) for e in range(ne)]
+        cache.update(feats, t)
+        cache.commit_step()
+        torch.cuda.synchronize()
+        slot = step % (m + 1)
+        for e in range(ne):
+            for b in range(B):
+                assert torch.equal(cache.plane_tensor(e, b)[slot].view(it), feats[e][b].reshape(-1).view(it)), \
+                    "%s step %d entry %d sample %d: the newest plane differs from the feature" % (name, step, e, b)
+        for e, lst in blocks.items():
+            for blk in lst:
+                b, s, ln = blk
+                kept[(e, blk)] = ([U.to_oracle(feats[e][b].reshape(-1)[s:s + ln])] + kept[(e, blk)])[: m + 1]
+        hist = ([t[0]] + hist)[: m + 1]
+        del feats
+    step = n_steps
+    t_tgt = [w.times[step]] * B
+    outs = [torch.full((B, n, d), 7.0, dtype=tdt, device=DEV) for n, d in w.entries]
+    cache.forecast(t_tgt, outs)
+    torch.cuda.synchronize()
+    unit = [np.eye(m + 1, dtype=np.float32)[j].copy() for j in range(m + 1)]
+    a = np.zeros(m + 1, dtype=np.float32)
+    O.forecast_history_segment(O.F32, m, O.TAYLOR, hist, t_tgt[0], unit, a)            # weights, for the tolerance only
+
+    def oracle_forecast(e, blk):
+        want = np.zeros(blk[2], dtype=O.np_dtype(w.dtype))
+        O.forecast_history_segment(w.dtype, m, O.TAYLOR, hist, t_tgt[blk[0]], kept[(e, blk)], want)
+        scale = sum(np.abs(U.as_f64(f)) * abs(float(a[j])) for j, f in enumerate(kept[(e, blk)]))
+        return want, scale
+
+    for e, lst in blocks.items():
+        for blk in lst:
+            b, s, ln = blk
+            want, scale = oracle_forecast(e, blk)
+            got = U.to_oracle(outs[e][b].reshape(-1)[s:s + ln])
+            U.assert_close_storage(got, want, w.dtype, scale, "%s forecast entry %d block %r" % (name, e, blk))
+    fresh = src.feature(w.vidx, step, t_tgt)
+    tau = [S.speca_tau(w.tau0, w.beta, w.total_steps - step, w.total_steps)] * B
+    err = torch.full((B,), -7.0, dtype=torch.float32, device=DEV)
+    acc = torch.full((B,), 9, dtype=torch.uint8, device=DEV)
+    cache.verify(fresh, t_tgt, tau, err, acc)
+    torch.cuda.synchronize()
+    fresh_np = U.to_oracle(fresh).reshape(B, -1)
+    for b in range(B):
+        pred, _ = oracle_forecast(w.vidx, (b, 0, w.entry_elems(w.vidx)))
+        e_want = O.rel_l2(w.dtype, pred, fresh_np[b])
+        # on this uniform time grid the weights are ratios of small integers and a few per cent of the bf16
+        # forecasts are exact ties, which fp32 weights cannot break the way double arithmetic does
+        assert abs(float(err[b]) - e_want) <= U.ERR_TOL * max(1.0, e_want) + 6e-3 * e_want, (name, b, float(err[b]), e_want)
+        if abs(e_want - float(np.float32(tau[b]))) >= U.ERR_TOL + 6e-3 * e_want:
+            assert int(acc[b]) == (1 if O.accept(e_want, float(np.float32(tau[b]))) else 0)
+    for o in outs:
+        o.fill_(5.0)
+    cache.forecast([hist[0]] * B, outs)          # k = 0: the newest feature itself
+    torch.cuda.synchronize()
+    newest = (n_steps - 1) % (m + 1)
+    for e in range(ne):
+        for b in range(B):
+            assert torch.equal(outs[e][b].reshape(-1).view(it), cache.plane_tensor(e, b)[newest].view(it)), (name, e, b)
+    cache.close()
