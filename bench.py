@@ -38,6 +38,7 @@ FALLBACK_HBM_GBS = 6650.0
 # from the one-pass ncu capture of this benchmark's default workload at full size (FLUX-shaped cache,
 # order 2, bf16; profiles/dram_traffic_flux_full_size.md). Other workloads scale by the elements a
 # launch covers. Set an entry to None when its kernel changes until the counters have been taken again.
+NCU_DRAM_BYTES_PER_ELEM_HISTORY_UPDATE = 3.955   # profiles/history_layout_flux_full_size.md
 NCU_DRAM_BYTES_PER_ELEM = {"update": 11.987, "forecast": 8.042, "verify": 8.107}
 
 
@@ -736,6 +737,9 @@ def main():
                     help="comma list of further configs measured device-resident and reported under per_config")
     ap.add_argument("--path", default="auto", choices=["auto", "direct", "bulk", "wide"],
                     help="kernel variant (speca_path_t); results are identical, only speed differs")
+    ap.add_argument("--layout", default="tables", choices=["tables", "history"],
+                    help="what the cache keeps: the paper's difference tables (default) or the raw features of "
+                         "the last references (speca_layout_t)")
     ap.add_argument("--separate-select", action="store_true",
                     help="speca_verify then speca_select_adaptive as two launches instead of speca_verify_select")
     ap.add_argument("--no-e2e", action="store_true")
@@ -763,22 +767,24 @@ def main():
 
     w = make_workload(args.config)
     path = {"auto": 0, "direct": 1, "bulk": 2, "wide": 3}[args.path]
-    h = Harness(w, device, seed_offset=17 * info.rank, path=path, fused_select=not args.separate_select)
+    layout = 1 if args.layout == "history" else 0
+    h = Harness(w, device, seed_offset=17 * info.rank, path=path, fused_select=not args.separate_select, layout=layout)
     total_ms, per_ms, launches, clocks = time_device_resident(h, args.steps, args.warmup, info, True)
     total_ms = D.max_over_ranks(total_ms, device)
-    value, ms_step, kernels, extra = summarize(w, per_ms, total_ms, args.steps, info.world, peak)
+    value, ms_step, kernels, extra = summarize(w, per_ms, total_ms, args.steps, info.world, peak, layout=layout)
 
-    multi = time_multi_horizon(h, peak, per_ms["forecast"]) if info.world == 1 else None
+    tables = info.world == 1 and layout == 0      # these calls exist for the table layout only
+    multi = time_multi_horizon(h, peak, per_ms["forecast"]) if tables else None
     metrics = time_metrics(h) if info.world == 1 else None
-    per_entry = time_update_per_entry(h) if info.world == 1 else None
-    fsum = time_forecast_sum(h, peak) if info.world == 1 else None
+    per_entry = time_update_per_entry(h) if tables else None
+    fsum = time_forecast_sum(h, peak) if tables else None
 
     e2e = None
     if not args.no_e2e:
         e2e_steps = max(3, min(args.steps, 24))
         e2e_ms, h2d, d2h = time_end_to_end(h, e2e_steps, 3)
         e2e_ms = D.max_over_ranks(e2e_ms, device)
-        ab = algorithmic_bytes(w, w.max_order)
+        ab = algorithmic_bytes(w, w.max_order, layout)
         e2e = {"value": info.world * (ab["update"] + ab["forecast"] + ab["verify"]) / (e2e_ms * 1e-3) / 1e9,
                "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                "steps": e2e_steps,
@@ -789,14 +795,14 @@ def main():
     torch.cuda.empty_cache()
 
     history = None
-    if info.world == 1 and path in (0, 3):
+    if info.world == 1 and path in (0, 3) and layout == 0:
         try:
             history = time_history_layout(w, device, path, min(args.steps, 100), info, peak, ms_step, kernels)
         except Exception as exc:  # report, do not hide
             history = {"error": repr(exc)}
 
     per_config = {}
-    if info.world == 1:
+    if info.world == 1 and layout == 0:
         for name in [n for n in args.also.split(",") if n and n != args.config]:
             try:
                 w2 = make_workload(name)
@@ -840,6 +846,8 @@ def main():
     dominant = max(("update", "forecast", "verify"), key=lambda k: per_ms[k])
     dom = kernels[dominant]
     per_elem = NCU_DRAM_BYTES_PER_ELEM.get(dominant)
+    if layout == 1 and dominant == "update":
+        per_elem = NCU_DRAM_BYTES_PER_ELEM_HISTORY_UPDATE
     n_dom = w.batch * w.entry_elems(w.vidx) if dominant == "verify" else w.elems_per_order
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": dom["gbs"], "peak": peak, "unit": "GB/s",
                 "frac": dom["gbs"] / peak, "peak_source": peak_src,
@@ -872,7 +880,7 @@ def main():
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": info.world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": dict(workload_config(w), select="its own launch (speca_select_adaptive)" if args.separate_select
+        "config": dict(workload_config(w), layout=args.layout, select="its own launch (speca_select_adaptive)" if args.separate_select
                        else "inside the verify launch (speca_verify_select)"),
         "metric_note": "value = algorithmic bytes of the whole step (update + forecast + verify/select) / step time; "
                        "forecast + verify alone (one speculative step) is forecast_verify_gbs, the update alone kernels.update.gbs",
