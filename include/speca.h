@@ -111,8 +111,7 @@ typedef enum {
  *          differences are folded into per-plane weights on the host when a forecast is asked for:
  *          out = sum_i w_i * plane_i. Same Eq. 2-3 (and the same Newton / Adams-Bashforth readings), any
  *          gaps; the results differ from TABLES only in that no intermediate quotient is rounded to the
- *          storage type. Not available for speca_forecast_multi / speca_forecast_sum and only on the
- *          default kernel path.
+ *          storage type. Served by the default kernel path only (SPECA_PATH_AUTO / SPECA_PATH_WIDE).
  */
 typedef enum {
     SPECA_LAYOUT_TABLES = 0,

@@ -207,50 +207,69 @@ int oracle_forecast_segment(int dtype, int64_t n, int m, int basis, int n_refs, 
  * printed, evaluated from the raw features.
  * Returns 0, or 1 if there is no reference or a divisor is zero.
  */
-int oracle_forecast_history_segment(int dtype, int64_t n, int m, int basis, int n_hist, const double* t_hist,
-                                    double t_target, const void* const* hist, void* out) {
-    if (n_hist < 1 || n_hist > m + 1 || m > ORACLE_MAX_ORDER) return 1;
+static int history_times_ok(int m, int basis, int n_hist, const double* t_hist) {
+    if (n_hist < 1 || n_hist > m + 1 || m > ORACLE_MAX_ORDER) return 0;
     int v = n_hist - 1;
-    if (basis == ORACLE_ADAMS_BASHFORTH && v > 4) return 1;
+    if (basis == ORACLE_ADAMS_BASHFORTH && v > 4) return 0;
     for (int k = v - 1; k >= 0; --k)
         for (int i = 0; i < v - k; ++i)
-            if (t_hist[k] - (basis == ORACLE_NEWTON ? t_hist[k + 1 + i] : t_hist[k + 1]) == 0.0) return 1;
+            if (t_hist[k] - (basis == ORACLE_NEWTON ? t_hist[k + 1 + i] : t_hist[k + 1]) == 0.0) return 0;
+    return 1;
+}
+
+/* The unrounded forecast of element j from the v + 1 stored features. */
+static double history_forecast_elem(int dtype, int basis, int v, const double* t_hist, double t_target,
+                                    const void* const* hist, int64_t j) {
     static const double gam[4] = {1.0, 1.0 / 2, 5.0 / 12, 3.0 / 8}; /* Adams-Bashforth, collected by plane */
-#pragma omp parallel for schedule(static)
-    for (int64_t j = 0; j < n; ++j) {
-        double d[ORACLE_MAX_ORDER + 1]; /* the planes a table would hold, unrounded */
-        d[0] = load_elem(hist[v], dtype, j);
-        for (int k = v - 1; k >= 0; --k) { /* fold in the feature at t_hist[k]; v - k references came before */
-            double c[ORACLE_MAX_ORDER + 1];
-            c[0] = load_elem(hist[k], dtype, j);
-            for (int i = 0; i < v - k; ++i) {
-                double gap = t_hist[k] - (basis == ORACLE_NEWTON ? t_hist[k + 1 + i] : t_hist[k + 1]);
-                c[i + 1] = (c[i] - d[i]) / gap;
-            }
-            for (int i = 0; i <= v - k; ++i) d[i] = c[i];
+    double d[ORACLE_MAX_ORDER + 1]; /* the planes a table would hold, unrounded */
+    d[0] = load_elem(hist[v], dtype, j);
+    for (int k = v - 1; k >= 0; --k) { /* fold in the feature at t_hist[k]; v - k references came before */
+        double c[ORACLE_MAX_ORDER + 1];
+        c[0] = load_elem(hist[k], dtype, j);
+        for (int i = 0; i < v - k; ++i) {
+            double gap = t_hist[k] - (basis == ORACLE_NEWTON ? t_hist[k + 1 + i] : t_hist[k + 1]);
+            c[i + 1] = (c[i] - d[i]) / gap;
         }
-        double s = d[0];
-        if (basis == ORACLE_NEWTON) {
-            double w = 1.0;
-            for (int i = 1; i <= v; ++i) {
-                w *= t_target - t_hist[i - 1];
-                s += d[i] * w;
-            }
-        } else if (basis == ORACLE_TAYLOR) {
-            double x = t_target - t_hist[0], fact = 1.0;
-            for (int i = 1; i <= v; ++i) {
-                fact *= (double)i;
-                s += d[i] * pow(x, (double)i) / fact;
-            }
-        } else {
-            double x = t_target - t_hist[0], h = v >= 2 ? t_hist[0] - t_hist[1] : 0.0, hp = 1.0;
-            for (int i = 1; i <= v; ++i) {
-                s += d[i] * x * gam[i - 1] * hp;
-                hp *= h;
-            }
-        }
-        store_elem(out, dtype, j, s);
+        for (int i = 0; i <= v - k; ++i) d[i] = c[i];
     }
+    double s = d[0];
+    if (basis == ORACLE_NEWTON) {
+        double w = 1.0;
+        for (int i = 1; i <= v; ++i) {
+            w *= t_target - t_hist[i - 1];
+            s += d[i] * w;
+        }
+    } else if (basis == ORACLE_TAYLOR) {
+        double x = t_target - t_hist[0], fact = 1.0;
+        for (int i = 1; i <= v; ++i) {
+            fact *= (double)i;
+            s += d[i] * pow(x, (double)i) / fact;
+        }
+    } else {
+        double x = t_target - t_hist[0], h = v >= 2 ? t_hist[0] - t_hist[1] : 0.0, hp = 1.0;
+        for (int i = 1; i <= v; ++i) {
+            s += d[i] * x * gam[i - 1] * hp;
+            hp *= h;
+        }
+    }
+    return s;
+}
+
+int oracle_forecast_history_segment(int dtype, int64_t n, int m, int basis, int n_hist, const double* t_hist,
+                                    double t_target, const void* const* hist, void* out) {
+    if (!history_times_ok(m, basis, n_hist, t_hist)) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < n; ++j)
+        store_elem(out, dtype, j, history_forecast_elem(dtype, basis, n_hist - 1, t_hist, t_target, hist, j));
+    return 0;
+}
+
+/* The same forecast added, unrounded, to an accumulator (for the summed forecast below). */
+int oracle_forecast_history_accumulate_segment(int dtype, int64_t n, int m, int basis, int n_hist, const double* t_hist,
+                                               double t_target, const void* const* hist, double* acc) {
+    if (!history_times_ok(m, basis, n_hist, t_hist)) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < n; ++j) acc[j] += history_forecast_elem(dtype, basis, n_hist - 1, t_hist, t_target, hist, j);
     return 0;
 }
 

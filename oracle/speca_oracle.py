@@ -58,6 +58,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_forecast_segment.restype = i32
         L.oracle_forecast_history_segment.argtypes = [i32, i64, i32, i32, i32, dp, dbl, ctypes.POINTER(vp), vp]
         L.oracle_forecast_history_segment.restype = i32
+        L.oracle_forecast_history_accumulate_segment.argtypes = [i32, i64, i32, i32, i32, dp, dbl, ctypes.POINTER(vp), vp]
+        L.oracle_forecast_history_accumulate_segment.restype = i32
         L.oracle_forecast_accumulate_segment.argtypes = [i32, i64, i32, i32, i32, dp, dbl, vp, i64, vp]
         L.oracle_forecast_accumulate_segment.restype = i32
         L.oracle_accumulate_elems.argtypes = [i32, i64, vp, vp]
@@ -297,7 +299,6 @@ class OracleCache:
         keep what `out` held."""
         n = self.entry_elems[entry_ids[0]]
         assert all(self.entry_elems[e] == n for e in entry_ids)
-        assert self.layout == LAYOUT_TABLES, "the summed forecast is defined on difference tables"
         if out is None:
             out = np.zeros((self.B, n), dtype=np_dtype(self.dtype))
         for b in range(self.B):
@@ -307,6 +308,14 @@ class OracleCache:
             if base is not None:
                 lib().oracle_accumulate_elems(self.dtype, n, _ptr(np.ascontiguousarray(base[b])), _ptr(acc))
             for e in entry_ids:
+                if self.layout == LAYOUT_HISTORY:
+                    hist = self.hist[e][b][: min(self.n_refs[b], self.m + 1)]
+                    ptrs = (ctypes.c_void_p * len(hist))(*[h.ctypes.data for h in hist])
+                    rc = lib().oracle_forecast_history_accumulate_segment(self.dtype, n, self.m, self.basis, len(hist),
+                                                                          _hist(self.t_hist[b], self.m), float(t_target[b]),
+                                                                          ptrs, _ptr(acc))
+                    assert rc == 0
+                    continue
                 p = self.planes[e][b]
                 rc = lib().oracle_forecast_accumulate_segment(self.dtype, n, self.m, self.basis, self.n_refs[b],
                                                               _hist(self.t_hist[b], self.m), float(t_target[b]),

@@ -553,8 +553,6 @@ speca_status_t speca_forecast_multi(speca_cache_t* c, int32_t n_targets, const d
     if (t_targets == nullptr || outs == nullptr) return fail(c, SPECA_ERR_INVALID_ARG, "forecast_multi: null argument");
     if (n_targets < 1 || n_targets > SPECA_MAX_HORIZON)
         return fail(c, SPECA_ERR_INVALID_ARG, "forecast_multi: n_targets must be 1..%d", SPECA_MAX_HORIZON);
-    if (c->layout != SPECA_LAYOUT_TABLES)
-        return fail(c, SPECA_ERR_UNSUPPORTED, "forecast_multi: only for caches that keep difference tables");
     if (c->pending) return fail(c, SPECA_ERR_STATE, "forecast_multi: a reference step is open (commit it first)");
     static thread_local MultiParams p;  // 13 KB: kept off the stack
     std::memset(&p, 0, sizeof p);
@@ -564,7 +562,7 @@ speca_status_t speca_forecast_multi(speca_cache_t* c, int32_t n_targets, const d
         for (int k = 0; k < n_targets; ++k) {
             const double t = t_targets[static_cast<size_t>(k) * c->B + b];
             if (!std::isfinite(t)) return fail(c, SPECA_ERR_INVALID_ARG, "forecast_multi: t_targets[%d][%d] not finite", k, b);
-            forecast_scalars(c, b, t, &order, p.coef[k][b]);
+            forecast_coefficients(c, b, t, &order, p.coef[k][b]);
         }
         if (order < 0 && dev_active_mask == nullptr)
             return fail(c, SPECA_ERR_STATE, "forecast_multi: sample %d has no committed reference", b);
@@ -594,6 +592,7 @@ speca_status_t speca_forecast_multi(speca_cache_t* c, int32_t n_targets, const d
     p.tile_start = reinterpret_cast<const uint32_t*>(c->arena + L.tiles_off[ti]);
     p.arena = c->arena;
     p.dev_mask = dev_active_mask;
+    p.weighted = c->layout == SPECA_LAYOUT_HISTORY ? 1 : 0;
     p.n_targets = n_targets;
     p.seg_lo = static_cast<uint32_t>(e_lo) * c->B;
     p.seg_hi = static_cast<uint32_t>(e_hi + 1) * c->B;
@@ -615,8 +614,6 @@ speca_status_t speca_forecast_sum(speca_cache_t* c, const int32_t* entry_ids, in
     if (entry_ids == nullptr || t_target == nullptr || out == nullptr)
         return fail(c, SPECA_ERR_INVALID_ARG, "forecast_sum: null argument");
     if (n_ids < 1 || n_ids > SPECA_MAX_ENTRIES) return fail(c, SPECA_ERR_INVALID_ARG, "forecast_sum: n_ids out of range");
-    if (c->layout != SPECA_LAYOUT_TABLES)
-        return fail(c, SPECA_ERR_UNSUPPORTED, "forecast_sum: only for caches that keep difference tables");
     if (c->pending) return fail(c, SPECA_ERR_STATE, "forecast_sum: a reference step is open (commit it first)");
     static thread_local SumParams p;
     std::memset(&p, 0, sizeof p);
@@ -636,7 +633,7 @@ speca_status_t speca_forecast_sum(speca_cache_t* c, const int32_t* entry_ids, in
     for (int b = 0; b < c->B; ++b) {
         if (!std::isfinite(t_target[b])) return fail(c, SPECA_ERR_INVALID_ARG, "forecast_sum: t_target[%d] not finite", b);
         int order;
-        forecast_scalars(c, b, t_target[b], &order, p.coef[b]);
+        forecast_coefficients(c, b, t_target[b], &order, p.coef[b]);
         if (order < 0 && dev_active_mask == nullptr)
             return fail(c, SPECA_ERR_STATE, "forecast_sum: sample %d has no committed reference", b);
         p.order[b] = static_cast<int8_t>(order);
@@ -651,6 +648,7 @@ speca_status_t speca_forecast_sum(speca_cache_t* c, const int32_t* entry_ids, in
     p.segs = reinterpret_cast<const SegDesc*>(c->arena + L.segs_off);
     p.arena = c->arena;
     p.dev_mask = dev_active_mask;
+    p.weighted = c->layout == SPECA_LAYOUT_HISTORY ? 1 : 0;
     p.base = static_cast<const char*>(base);
     p.out = static_cast<char*>(out);
     p.tiles_per_sample = (p.n_elems + te - 1) / te;

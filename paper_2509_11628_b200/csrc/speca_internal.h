@@ -70,8 +70,9 @@ struct MultiParams {
     uint32_t seg_lo, seg_hi;
     uint32_t tile_lo, tile_hi;
     int32_t n_targets;                // K
+    int32_t weighted;                 // raw-feature cache: coef = weights of the physical planes
     int8_t order[SPECA_MAX_BATCH];
-    float coef[SPECA_MAX_HORIZON][SPECA_MAX_BATCH][SPECA_MAX_ORDER];  // Horner multipliers per target
+    float coef[SPECA_MAX_HORIZON][SPECA_MAX_BATCH][kCoef];  // Horner multipliers (or plane weights) per target
     void* io[SPECA_MAX_ENTRIES];      // per entry: [K, B, N_e, D] output; null = skip
 };
 
@@ -86,8 +87,9 @@ struct SumParams {
     uint32_t tiles_per_sample;
     int32_t batch;
     int32_t n_ids;
+    int32_t weighted;  // raw-feature cache: coef = weights of the physical planes
     int8_t order[SPECA_MAX_BATCH];
-    float coef[SPECA_MAX_BATCH][SPECA_MAX_ORDER];
+    float coef[SPECA_MAX_BATCH][kCoef];
     uint16_t ids[SPECA_MAX_ENTRIES];  // entries to add, in this order
 };
 

@@ -205,6 +205,12 @@ __device__ __forceinline__ uint32_t find_segment(const uint32_t* __restrict__ ti
 // of a segment is ragged): whole vectors go through the vector loop, the remainder through the
 // scalar loop. `row` must be W-byte aligned (the planes always are).
 
+// One level of a forecast: Horner (acc * mu + lo), or for a cache that keeps raw features one more term
+// of the weighted sum (acc + lo * mu).
+__device__ __forceinline__ float forecast_level(float acc, float lo, float mu, bool weighted) {
+    return weighted ? fmaf(lo, mu, acc) : fmaf(acc, mu, lo);
+}
+
 // Eq. 2 in Horner form: acc = D_v; acc = D_{i-1} + acc * mu_i for i = v..1.
 // With `weighted` (a cache that keeps raw features) the same planes are combined as a plain weighted
 // sum instead: acc = sum_i w_i * plane_i, w = mu[0..V].
@@ -495,8 +501,8 @@ static_assert(shape_tile_bytes(multi_shape(1)) == shape_tile_bytes(multi_shape(8
 template <int DT, int V, int W, int NT, int U>
 __device__ __forceinline__ void forecast_multi_tile(const char* __restrict__ plane0, uint64_t stride,
                                                     char* __restrict__ out, uint64_t target_stride, int n_targets,
-                                                    uint32_t cnt, const float (*__restrict__ mu)[SPECA_MAX_BATCH][SPECA_MAX_ORDER],
-                                                    uint32_t sample) {
+                                                    uint32_t cnt, const float (*__restrict__ mu)[SPECA_MAX_BATCH][kCoef],
+                                                    uint32_t sample, bool weighted) {
     constexpr int EPV = W / Elem<DT>::kBytes;
     const uint32_t nvec = cnt / EPV;
     Vec<W> d[V + 1][U];
@@ -510,29 +516,42 @@ __device__ __forceinline__ void forecast_multi_tile(const char* __restrict__ pla
     }
 #pragma unroll 1
     for (int k = 0; k < n_targets; ++k) {
-        float m[SPECA_MAX_ORDER];
+        float m[kCoef];
 #pragma unroll
-        for (int i = 0; i < SPECA_MAX_ORDER; ++i) m[i] = mu[k][sample][i];
+        for (int i = 0; i < kCoef; ++i) m[i] = mu[k][sample][i];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const uint32_t idx = u * NT + threadIdx.x;
             if (idx < nvec) {
                 float acc[EPV];
                 unpack_vec<DT, W>(d[V][u], acc);
+                if (weighted) {
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) acc[e] *= m[V];
+                }
 #pragma unroll
                 for (int i = V; i >= 1; --i) {
                     float lo[EPV];
                     unpack_vec<DT, W>(d[i - 1][u], lo);
+                    if (weighted) {
 #pragma unroll
-                    for (int e = 0; e < EPV; ++e) acc[e] = fmaf(acc[e], m[i - 1], lo[e]);
+                        for (int e = 0; e < EPV; ++e) acc[e] = fmaf(lo[e], m[i - 1], acc[e]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < EPV; ++e) acc[e] = fmaf(acc[e], m[i - 1], lo[e]);
+                    }
                 }
                 store_vec<W>(out + k * target_stride + static_cast<size_t>(idx) * W, pack_vec<DT, W>(acc));
             }
         }
         for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += NT) {
             float acc = load_scalar<DT>(plane0 + V * stride, j);
+            if (weighted) acc *= m[V];
 #pragma unroll
-            for (int i = V; i >= 1; --i) acc = fmaf(acc, m[i - 1], load_scalar<DT>(plane0 + (i - 1) * stride, j));
+            for (int i = V; i >= 1; --i) {
+                const float lo = load_scalar<DT>(plane0 + (i - 1) * stride, j);
+                acc = weighted ? fmaf(lo, m[i - 1], acc) : fmaf(acc, m[i - 1], lo);
+            }
             store_scalar<DT>(out + k * target_stride, j, acc);
         }
     }
@@ -570,14 +589,14 @@ __global__ void __launch_bounds__(NT, MINB) forecast_multi_kernel(const __grid_c
                 const uint32_t n = min(kChunk, cnt - done);
                 const size_t off = static_cast<size_t>(done) * Elem<DT>::kBytes;
                 forecast_multi_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, row + off, target_stride,
-                                                     p.n_targets, n, p.coef, sd.sample);
+                                                     p.n_targets, n, p.coef, sd.sample, p.weighted != 0);
             }
         } else {
             for (int k = 0; k < p.n_targets; ++k) {
-                float m[kCoef] = {};
+                float m[kCoef];
 #pragma unroll
-                for (int i = 0; i < SPECA_MAX_ORDER; ++i) m[i] = p.coef[k][sd.sample][i];
-                forecast_tile_any<DT>(plane0, sd.plane_stride, row + k * target_stride, cnt, v, m);
+                for (int i = 0; i < kCoef; ++i) m[i] = p.coef[k][sd.sample][i];
+                forecast_tile_any<DT>(plane0, sd.plane_stride, row + k * target_stride, cnt, v, m, p.weighted != 0);
             }
         }
     }
@@ -612,9 +631,10 @@ __global__ void __launch_bounds__(kSumThreads, kSumMinBlocks) forecast_sum_kerne
         const uint64_t byte0 = static_cast<uint64_t>(elem0) * Elem<DT>::kBytes;
         const char* base = p.base != nullptr ? p.base + b * row_bytes + byte0 : nullptr;
         char* out = p.out + b * row_bytes + byte0;
-        float mu[SPECA_MAX_ORDER];
+        float mu[kCoef];
 #pragma unroll
-        for (int i = 0; i < SPECA_MAX_ORDER; ++i) mu[i] = p.coef[b][i];
+        for (int i = 0; i < kCoef; ++i) mu[i] = p.coef[b][i];
+        const bool weighted = p.weighted != 0;  // raw-feature cache: sum_i mu[i] * plane_i instead of Horner
         const uint32_t idx = threadIdx.x;
         const bool vec_ok = ((reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(base)) & (W - 1)) == 0;
         const uint32_t nvec = vec_ok ? cnt / EPV : 0;
@@ -645,12 +665,16 @@ __global__ void __launch_bounds__(kSumThreads, kSumMinBlocks) forecast_sum_kerne
                         for (int g = 0; g < G; ++g) {
                             float acc[EPV];
                             unpack_vec<DT, W>(d[g][V], acc);
+                            if (weighted) {
+#pragma unroll
+                                for (int k = 0; k < EPV; ++k) acc[k] *= mu[V];
+                            }
 #pragma unroll
                             for (int i = V; i >= 1; --i) {
                                 float lo[EPV];
                                 unpack_vec<DT, W>(d[g][i - 1], lo);
 #pragma unroll
-                                for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+                                for (int k = 0; k < EPV; ++k) acc[k] = forecast_level(acc[k], lo[k], mu[i - 1], weighted);
                             }
 #pragma unroll
                             for (int k = 0; k < EPV; ++k) sum[k] += acc[k];
@@ -667,20 +691,28 @@ __global__ void __launch_bounds__(kSumThreads, kSumMinBlocks) forecast_sum_kerne
 #pragma unroll
                     for (int i = 0; i <= V; ++i) d[i] = load_vec<W>(plane0 + i * sd.plane_stride);
                     unpack_vec<DT, W>(d[V], acc);
+                    if (weighted) {
+#pragma unroll
+                        for (int k = 0; k < EPV; ++k) acc[k] *= mu[V];
+                    }
 #pragma unroll
                     for (int i = V; i >= 1; --i) {
                         float lo[EPV];
                         unpack_vec<DT, W>(d[i - 1], lo);
 #pragma unroll
-                        for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+                        for (int k = 0; k < EPV; ++k) acc[k] = forecast_level(acc[k], lo[k], mu[i - 1], weighted);
                     }
                 } else {  // a sample with fewer references than the launch's common order
                     unpack_vec<DT, W>(load_vec<W>(plane0 + v * sd.plane_stride), acc);
+                    if (weighted) {
+#pragma unroll
+                        for (int k = 0; k < EPV; ++k) acc[k] *= mu[v];
+                    }
                     for (int i = v; i >= 1; --i) {
                         float lo[EPV];
                         unpack_vec<DT, W>(load_vec<W>(plane0 + (i - 1) * sd.plane_stride), lo);
 #pragma unroll
-                        for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+                        for (int k = 0; k < EPV; ++k) acc[k] = forecast_level(acc[k], lo[k], mu[i - 1], weighted);
                     }
                 }
 #pragma unroll
@@ -695,7 +727,9 @@ __global__ void __launch_bounds__(kSumThreads, kSumMinBlocks) forecast_sum_kerne
                 const SegDesc sd = p.segs[static_cast<uint32_t>(p.ids[j]) * p.batch + b];
                 const char* plane0 = p.arena + sd.plane0_off + byte0;
                 float acc = load_scalar<DT>(plane0 + v * sd.plane_stride, e);
-                for (int i = v; i >= 1; --i) acc = fmaf(acc, mu[i - 1], load_scalar<DT>(plane0 + (i - 1) * sd.plane_stride, e));
+                if (weighted) acc *= mu[v];
+                for (int i = v; i >= 1; --i)
+                    acc = forecast_level(acc, load_scalar<DT>(plane0 + (i - 1) * sd.plane_stride, e), mu[i - 1], weighted);
                 sum += acc;
             }
             store_scalar<DT>(out, e, sum);

@@ -92,7 +92,7 @@ def test_masks_resets_and_verification_on_many_tiles(S, U, dtype):
     pair.close()
 
 
-def test_an_update_moves_two_words_per_element_and_other_calls_are_refused(S):
+def test_the_ring_wraps_and_other_kernel_paths_are_refused(S):
     entries = [(8, 64), (4, 32)]
     B = 2
     c = S.SpecaCache(entries, B, 2, 1, DEV, layout=HIST)
@@ -114,9 +114,6 @@ def test_an_update_moves_two_words_per_element_and_other_calls_are_refused(S):
             fn()
         return ei.value.status
 
-    multi = [torch.zeros(2, B, n, d, dtype=torch.bfloat16, device=DEV) for n, d in entries]
-    assert status_of(lambda: c.forecast_multi([[0.6] * B, [0.5] * B], multi)) == S.SPECA_ERR_UNSUPPORTED
-    assert status_of(lambda: c.forecast_sum([0], [0.6] * B, outs[0])) == S.SPECA_ERR_UNSUPPORTED
     assert status_of(lambda: c.update(f, [0.7] * B)) == S.SPECA_ERR_ZERO_GAP
     assert status_of(lambda: S.SpecaCache(entries, B, 2, 1, DEV, path=S.SPECA_PATH_BULK, layout=HIST)) == S.SPECA_ERR_UNSUPPORTED
     c.close()
@@ -176,4 +173,57 @@ def test_features_written_in_place_cost_no_launch(S, U):
         S.speca_cache_next_slot(c.handle, 0, 0)
     assert ei.value.status == S.SPECA_ERR_UNSUPPORTED
     c.close()
+    pair.close()
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("basis", [0, 1, 2])
+@pytest.mark.parametrize("m", [0, 1, 2, 4])
+def test_multi_horizon_and_summed_forecasts(S, U, dtype, basis, m):
+    """speca_forecast_multi and speca_forecast_sum on the raw-feature cache: K targets bit-identical to K
+    single forecasts and equal to the oracle; the sum of several entries equal to the oracle's sum."""
+    shape = (37, 129)
+    E, B, K = 7, 3, 3
+    entries = [shape] * E + [(3, 8192 + 8)]
+    gen = torch.Generator(device=DEV).manual_seed(9100 + 10 * m + basis)
+    pair = U.Pair(entries, B, m, dtype, basis, layout=HIST)
+    times = [1.0, 0.93, 0.9, 0.84, 0.8, 0.77, 0.71]
+    for step in range(m + 3):
+        pair.update(rand_feats(entries, B, pair.tdt, gen), [times[step], times[step] - 0.003, times[step] + 0.001])
+        pair.commit()
+    t_last = times[m + 2]
+    targets = [[t_last - 0.011 * (k + 1) - 0.001 * b for b in range(B)] for k in range(K)]
+    active = [1, 0, 1]
+    mask = torch.tensor(active, dtype=torch.uint8, device=DEV)
+    outs = [torch.full((K, B, n, d), 3.0, dtype=pair.tdt, device=DEV) for n, d in entries]
+    pair.gpu.forecast_multi(targets, outs, mask)
+    it = torch.int16 if dtype == 1 else torch.int32
+    three = U.to_oracle(torch.full((1,), 3.0, dtype=pair.tdt))[0]
+    for k in range(K):
+        single = [torch.full((B, n, d), 3.0, dtype=pair.tdt, device=DEV) for n, d in entries]
+        pair.gpu.forecast(targets[k], single, mask)
+        torch.cuda.synchronize()
+        for e, (n, d) in enumerate(entries):
+            assert torch.equal(outs[e][k].view(it), single[e].view(it)), (k, e)
+            init = np.full((B, n * d), three, dtype=O.np_dtype(dtype))
+            want = pair.cpu.forecast_entry(e, targets[k], active, out=init)
+            got = U.to_oracle(outs[e][k]).reshape(B, -1)
+            for b in range(B):
+                if not active[b]:
+                    assert np.array_equal(got[b], want[b])
+                else:
+                    U.assert_close_storage(got[b], want[b], dtype, pair.history_scale(e, b, targets[k][b]), "multi %d %d %d" % (k, e, b))
+    tt = targets[0]
+    base = torch.randn(B, *shape, generator=gen, device=DEV).to(pair.tdt)
+    for ids, use_base in [(list(range(E)), True), ([3], False), ([4, 0, 4, 6, 5, 1], True)]:
+        out = torch.full((B, *shape), 3.0, dtype=pair.tdt, device=DEV)
+        pair.gpu.forecast_sum(ids, tt, out, base if use_base else None)
+        torch.cuda.synchronize()
+        want = pair.cpu.forecast_sum(ids, tt, U.to_oracle(base).reshape(B, -1) if use_base else None)
+        got = U.to_oracle(out).reshape(B, -1)
+        for b in range(B):
+            scale = sum(pair.history_scale(e, b, tt[b]) for e in ids)
+            if use_base:
+                scale = scale + np.abs(U.as_f64(U.to_oracle(base).reshape(B, -1)[b]))
+            U.assert_close_storage(got[b], want[b], dtype, scale, "sum %r sample %d" % (ids, b))
     pair.close()

@@ -58,8 +58,9 @@ MUTANTS = [
      "double gap = t_hist[k] - t_hist[k + 1 + i];", 0, 1),
     ("history_newton_divides_by_last_gap", "double gap = t_hist[k] - (basis == ORACLE_NEWTON ? t_hist[k + 1 + i] : t_hist[k + 1]);",
      "double gap = t_hist[k] - t_hist[k + 1];", 0, 1),
-    ("history_starts_from_the_newest", "d[0] = load_elem(hist[v], dtype, j);\n        for (int k = v - 1; k >= 0; --k) {",
-     "d[0] = load_elem(hist[0], dtype, j);\n        for (int k = v - 1; k >= 0; --k) {", 0, 1),
+    ("history_starts_from_the_newest", "d[0] = load_elem(hist[v], dtype, j);\n    for (int k = v - 1; k >= 0; --k) {",
+     "d[0] = load_elem(hist[0], dtype, j);\n    for (int k = v - 1; k >= 0; --k) {", 0, 1),
+    ("history_sum_keeps_only_the_last_entry", "acc[j] += history_forecast_elem(", "acc[j] = history_forecast_elem(", 0, 1),
     ("history_drops_the_factorial", "s += d[i] * pow(x, (double)i) / fact;", "s += d[i] * pow(x, (double)i);", 0, 1),
     ("history_newton_nodes_shifted", "w *= t_target - t_hist[i - 1];", "w *= t_target - t_hist[i];", 0, 1),
     ("history_adams_bashforth_wrong_coefficient", "static const double gam[4] = {1.0, 1.0 / 2, 5.0 / 12, 3.0 / 8}; /* Adams-Bashforth, collected by plane */",

@@ -322,10 +322,11 @@ def test_bf16_tables_round_once_per_stored_plane():
 @pytest.mark.parametrize("basis", [O.TAYLOR, O.NEWTON, O.ADAMS_BASHFORTH])
 @pytest.mark.parametrize("dtype", [O.F32, O.BF16])
 @pytest.mark.parametrize("m", [1, 2, 3, 4])   # every order: each has its own Adams-Bashforth coefficient
-def test_summed_forecast_of_one_entry_is_the_plain_forecast_bit_for_bit(basis, dtype, m):
+@pytest.mark.parametrize("layout", [O.LAYOUT_TABLES, O.LAYOUT_HISTORY])
+def test_summed_forecast_of_one_entry_is_the_plain_forecast_bit_for_bit(basis, dtype, m, layout):
     g = torch.Generator().manual_seed(90 + basis)
     B, n = 2, 300
-    cache = O.OracleCache([n, n], B, m, dtype, basis)
+    cache = O.OracleCache([n, n], B, m, dtype, basis, layout=layout)
     for k, t in enumerate([1.0, 0.93, 0.9, 0.81, 0.79][: m + 1]):
         fs = [torch.randn(B, n, generator=g) for _ in range(2)]
         fs = [bf16_bits(f) if dtype == O.BF16 else f.numpy().copy() for f in fs]
@@ -336,12 +337,13 @@ def test_summed_forecast_of_one_entry_is_the_plain_forecast_bit_for_bit(basis, d
         assert np.array_equal(cache.forecast_sum([e], tt), cache.forecast_entry(e, tt))
 
 
-def test_summed_forecast_is_the_sum_of_the_forecasts_in_exact_arithmetic():
+@pytest.mark.parametrize("layout", [O.LAYOUT_TABLES, O.LAYOUT_HISTORY])
+def test_summed_forecast_is_the_sum_of_the_forecasts_in_exact_arithmetic(layout):
     # integer features, integer times, fp32 storage: every product and sum below is exact, so the sum
     # of the separately stored forecasts must equal the summed forecast, and adding a base adds it
     rng = np.random.default_rng(9)
     B, n, m, E = 2, 64, 2, 5
-    cache = O.OracleCache([n] * E, B, m, O.F32)
+    cache = O.OracleCache([n] * E, B, m, O.F32, layout=layout)
     for t in (8.0, 6.0, 4.0):
         cache.update([rng.integers(-20, 20, (B, n)).astype(np.float32) * 8 for _ in range(E)], [t] * B)
         cache.commit_step()
