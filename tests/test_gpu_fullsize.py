@@ -199,7 +199,7 @@ def test_full_size_config_on_sampled_blocks(S, U, name, kw, path):
     cache.close()
 
 
-@pytest.mark.parametrize("name", ["dit_xl2", "flux"])
+@pytest.mark.parametrize("name", ["dit_xl2", "flux", "hunyuan_video"])
 def test_full_size_raw_feature_cache_on_sampled_blocks(S, U, name):
     """The same at full size for the cache that keeps raw features: reference steps past the point where
     the ring wraps (every element: the newest plane is the feature, bit for bit), forecast of every entry

@@ -29,14 +29,15 @@ def U():
 
 @pytest.mark.parametrize("metric", [0, 1, 2, 3])
 @pytest.mark.parametrize("dtype", [0, 1])
-def test_two_token_shards_match_unsharded_and_oracle(S, U, metric, dtype):
+@pytest.mark.parametrize("layout", [0, 1])    # difference tables, raw features
+def test_two_token_shards_match_unsharded_and_oracle(S, U, metric, dtype, layout):
     from paper_2509_11628_b200 import dist as D
     B, tokens, dim, m = 4, 301, 1160, 2
     tdt = torch.bfloat16 if dtype == 1 else torch.float32
     gen = torch.Generator(device=DEV).manual_seed(900 + metric)
     ranges = [D.shard_tokens(tokens, 2, r) for r in range(2)]
-    whole = U.Pair([(tokens, dim)], B, m, dtype)
-    shards = [S.SpecaCache([(n, dim)], B, m, dtype, DEV) for _, n in ranges]
+    whole = U.Pair([(tokens, dim)], B, m, dtype, layout=layout)
+    shards = [S.SpecaCache([(n, dim)], B, m, dtype, DEV, layout=layout) for _, n in ranges]
     for t in (1.0, 0.9, 0.85):
         f = torch.randn(B, tokens, dim, generator=gen, device=DEV).to(tdt)
         whole.update([f], [t] * B)
