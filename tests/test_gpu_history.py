@@ -227,3 +227,37 @@ def test_multi_horizon_and_summed_forecasts(S, U, dtype, basis, m):
                 scale = scale + np.abs(U.as_f64(U.to_oracle(base).reshape(B, -1)[b]))
             U.assert_close_storage(got[b], want[b], dtype, scale, "sum %r sample %d" % (ids, b))
     pair.close()
+
+
+def test_checkpoint_and_resume_continue_bit_for_bit(S):
+    """Arena bytes + reference history are the whole state of a raw-feature cache too: the ring position
+    follows from the number of references, so a restored cache continues exactly where the saved one was."""
+    entries = [(16, 520), (33, 1031)]
+    B, m = 3, 2
+    gen = torch.Generator(device=DEV).manual_seed(13)
+    a = S.SpecaCache(entries, B, m, 1, DEV, layout=HIST)
+    steps = [([1.0, 1.0, 1.0], None), ([0.95, 0.96, 0.95], [1, 1, 0]), ([0.9, 0.91, 0.9], None), ([0.85, 0.85, 0.85], [1, 0, 1]),
+             ([0.8, 0.8, 0.8], None)]
+    for t, mask in steps:
+        a.update(rand_feats(entries, B, torch.bfloat16, gen), t, mask)
+        a.commit_step()
+    torch.cuda.synchronize()
+    saved = a.arena.clone()
+    n_refs, t_hist = S.speca_cache_get_history(a.handle, B)
+    assert n_refs == [5, 4, 4]                     # past the wrap of the three-plane ring, at different positions
+    b = S.SpecaCache(entries, B, m, 1, DEV, layout=HIST)
+    b.arena.copy_(saved)
+    S.speca_cache_set_history(b.handle, n_refs, t_hist)
+    nxt = rand_feats(entries, B, torch.bfloat16, gen)
+    for c in (a, b):
+        c.update(nxt, [0.75, 0.74, 0.76], [0, 1, 1])
+        c.commit_step()
+    oa = [torch.zeros(B, n, d, dtype=torch.bfloat16, device=DEV) for n, d in entries]
+    ob = [torch.zeros(B, n, d, dtype=torch.bfloat16, device=DEV) for n, d in entries]
+    a.forecast([0.7] * B, oa)
+    b.forecast([0.7] * B, ob)
+    torch.cuda.synchronize()
+    for x, y in zip(oa, ob):
+        assert torch.equal(x.view(torch.int16), y.view(torch.int16))
+    assert torch.equal(a.arena, b.arena)
+    a.close(); b.close()
