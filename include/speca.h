@@ -187,6 +187,10 @@ speca_status_t speca_cache_reset(speca_cache_t* cache, const uint8_t* host_sampl
  * plane i+1 <- (new plane i - old plane i) / gap_i, the chain carried in fp32 and each plane
  * rounded once to the storage dtype. gap_i is t_ref - t_last (TAYLOR) or t_ref - (i-th previous
  * reference time) (NEWTON).
+ * A SPECA_LAYOUT_HISTORY cache does none of this arithmetic here: it copies f into the plane after the
+ * latest one, plane (references mod (m + 1)), and leaves the differencing to the forecast's weights
+ * (nothing at all is copied for an entry whose feats pointer is the address speca_cache_next_slot
+ * gave); the checks, states and errors are the same.
  * All entries of one reference step must be updated (each exactly once per masked sample)
  * before speca_cache_commit_step; t_ref and the mask must be the same in all of those calls.
  * Errors: INVALID_ARG, ALIGNMENT, ZERO_GAP, STATE (entry updated twice in one step, or
@@ -395,7 +399,9 @@ speca_status_t speca_cache_get_history(const speca_cache_t* cache, int32_t* host
 speca_status_t speca_cache_set_history(speca_cache_t* cache, const int32_t* host_n_refs, const double* host_t_hist);
 
 /* Device address and byte stride of the table of (entry, sample): plane i starts at
- * *plane0 + i * *plane_stride_bytes. For checkpointing and tests. */
+ * *plane0 + i * *plane_stride_bytes. For checkpointing and tests. In a SPECA_LAYOUT_HISTORY cache
+ * plane i is a ring slot: the feature of the j-th latest reference sits in plane
+ * (references - 1 - j) mod (max_order + 1). */
 speca_status_t speca_cache_plane(const speca_cache_t* cache, int32_t entry, int32_t sample, void** plane0,
                                  size_t* plane_stride_bytes);
 
