@@ -503,7 +503,7 @@ def adaptive_sweep(device: str, peak: float, path: int, orders=(1, 2, 3), horizo
     return out
 
 
-def sampler_run(device: str, path: int, name: str):
+def sampler_run(device: str, path: int, name: str, layout: int = 0):
     """The whole forecast-then-verify loop (50 sampler steps) over the library with the seeded feature
     generator standing in for the transformer: which steps each sample took in full, acceptance rate,
     speed-up by the paper's cost model next to Eq. 8, and the device time the cache path itself took."""
@@ -511,7 +511,7 @@ def sampler_run(device: str, path: int, name: str):
     from paper_2509_11628_b200 import scheduler as SCH
     w = W.flux_adaptive(max_order=2, batch=8) if name == "flux_adaptive" else W.BY_NAME[name]()
     gamma = 1.0 / {"dit_xl2": 28, "flux": 57, "flux_adaptive": 57, "hunyuan_video": 60}[name]
-    cache = S.SpecaCache(w.entries, w.batch, w.max_order, w.dtype, device, path=path)
+    cache = S.SpecaCache(w.entries, w.batch, w.max_order, w.dtype, device, path=path, layout=layout)
     src = W.FeatureSource(w, device)
 
     class Model:
@@ -836,6 +836,10 @@ def main():
         for name in ("dit_xl2", "flux_adaptive"):
             try:
                 sampler[name] = sampler_run(device, path, name)
+                if path in (0, 3):   # the same run on a cache that keeps raw features: cache-path time only
+                    hist = sampler_run(device, path, name, layout=1)
+                    sampler[name]["history_layout"] = {k: hist[k] for k in (
+                        "acceptance_rate", "library_ms_total", "ms_mean", "sampler_steps_per_s_library_only")}
             except Exception as exc:  # report, do not hide
                 sampler[name] = {"error": repr(exc)}
 
