@@ -417,6 +417,15 @@ speca_status_t speca_cache_plane(const speca_cache_t* cache, int32_t entry, int3
 speca_status_t speca_cache_next_slot(const speca_cache_t* cache, int32_t entry, int32_t sample, void** out);
 
 /*
+ * SPECA_LAYOUT_HISTORY only: pass this as feats[entry] to speca_cache_update to say that the feature of
+ * every masked sample of that entry already sits in the plane speca_cache_next_slot names for it (a
+ * batch whose samples are at the same ring position forms a strided [B, N_e, D] tensor there: sample
+ * stride = (max_order + 1) * plane stride). The entry then takes part in the reference step like any
+ * other, and nothing is copied.
+ */
+#define SPECA_FEATURE_IN_PLACE ((const void*)(uintptr_t)1)
+
+/*
  * Host-side counters of a handle since it was created (nothing here is read back from the device, so
  * the call neither launches nor synchronises). Launch counts are per kernel kind; the fused
  * verify + continuation call counts as one verify launch. reference_steps[b] counts committed

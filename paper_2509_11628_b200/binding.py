@@ -24,6 +24,7 @@ SPECA_BASIS_TAYLOR, SPECA_BASIS_NEWTON, SPECA_BASIS_ADAMS_BASHFORTH = 0, 1, 2
 SPECA_METRIC_L2, SPECA_METRIC_L1, SPECA_METRIC_LINF, SPECA_METRIC_COSINE = 0, 1, 2, 3
 SPECA_PATH_AUTO, SPECA_PATH_DIRECT, SPECA_PATH_BULK, SPECA_PATH_WIDE = 0, 1, 2, 3
 SPECA_LAYOUT_TABLES, SPECA_LAYOUT_HISTORY = 0, 1
+SPECA_FEATURE_IN_PLACE = 1   # as feats[entry]: the features already sit in the planes speca_cache_next_slot names
 SPECA_MAX_ORDER, SPECA_MAX_BATCH, SPECA_MAX_ENTRIES, SPECA_MAX_HORIZON = 4, 64, 512, 8
 
 EXPORTS = [
@@ -442,6 +443,21 @@ class SpecaCache:
 
     def stats(self):
         return speca_cache_stats(self.handle, self.batch)
+
+    def next_slot_batch(self, entry: int) -> torch.Tensor:
+        """All samples' next planes of ``entry`` as one strided ``[B, N_e, D]`` view of the arena (raw-feature
+        cache whose samples are at the same ring position): write the block output here and pass
+        ``SPECA_FEATURE_IN_PLACE`` for the entry to ``update``."""
+        ptrs = [speca_cache_next_slot(self.handle, entry, b) for b in range(self.batch)]
+        n, d = self.entries[entry]
+        esz = 2 if self.dtype == SPECA_BF16 else 4
+        tdt = torch.bfloat16 if self.dtype == SPECA_BF16 else torch.float32
+        step = (ptrs[1] - ptrs[0]) if self.batch > 1 else n * d * esz
+        if any(ptrs[b] - ptrs[0] != b * step for b in range(self.batch)):
+            raise ValueError("the samples are at different ring positions: use next_slot_tensor per sample")
+        off = ptrs[0] - self.arena.data_ptr()
+        flat = self.arena[off:].view(tdt)
+        return torch.as_strided(flat, (self.batch, n, d), (step // esz, d, 1))
 
     def next_slot_tensor(self, entry: int, sample: int = 0) -> torch.Tensor:
         """The plane that the next reference step of ``sample`` fills, as an ``[N_e, D]`` view of the arena

@@ -422,6 +422,11 @@ speca_status_t speca_cache_update(speca_cache_t* c, const void* const* feats, co
     for (int e = 0; e < c->n_entries; ++e) {
         if (feats[e] == nullptr) continue;
         if (c->entry_updated[e]) return fail(c, SPECA_ERR_STATE, "update: entry %d already updated in this step", e);
+        if (feats[e] == SPECA_FEATURE_IN_PLACE) {
+            if (c->layout != SPECA_LAYOUT_HISTORY)
+                return fail(c, SPECA_ERR_INVALID_ARG, "update: SPECA_FEATURE_IN_PLACE needs a cache that keeps raw features");
+            continue;  // the caller wrote every masked sample's feature into its next plane: nothing to copy
+        }
         if (reinterpret_cast<uintptr_t>(feats[e]) % esz != 0)
             return fail(c, SPECA_ERR_ALIGNMENT, "update: feats[%d] not aligned to the element size", e);
         if (c->layout == SPECA_LAYOUT_HISTORY) {

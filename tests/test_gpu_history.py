@@ -261,3 +261,51 @@ def test_checkpoint_and_resume_continue_bit_for_bit(S):
         assert torch.equal(x.view(torch.int16), y.view(torch.int16))
     assert torch.equal(a.arena, b.arena)
     a.close(); b.close()
+
+
+def test_a_batch_written_in_place_through_a_strided_view(S, U):
+    """B = 3 in lockstep: the next planes of all samples form one strided [B, N, D] tensor; the model
+    writes there and the reference step copies nothing. When a masked step has moved the samples to
+    different ring positions the per-sample views still work."""
+    entries = [(37, 129), (64, 384)]
+    B, m = 3, 2
+    gen = torch.Generator(device=DEV).manual_seed(29)
+    pair = U.Pair(entries, B, m, 1, layout=HIST)
+    clock = 1.0
+    for step in range(5):
+        clock -= 0.03
+        feats = rand_feats(entries, B, pair.tdt, gen)
+        for e in range(len(entries)):
+            pair.gpu.next_slot_batch(e).copy_(feats[e])
+        launches = pair.gpu.launches
+        pair.gpu.update([S.SPECA_FEATURE_IN_PLACE] * len(entries), [clock] * B)
+        pair.cpu.update([U.to_oracle(f).reshape(B, -1) for f in feats], [clock] * B)
+        assert pair.gpu.launches == launches
+        pair.commit()
+        pair.check_tables("strided in place, step %d" % step)
+        pair.check_forecast([clock - 0.02] * B)
+    # a masked step: samples 0 and 2 advance, sample 1 stays; per-sample planes from now on
+    for step in range(3):
+        clock -= 0.03
+        mask = [1, 0, 1] if step == 0 else None
+        feats = rand_feats(entries, B, pair.tdt, gen)
+        for e in range(len(entries)):
+            for b in range(B):
+                if mask is None or mask[b]:
+                    pair.gpu.next_slot_tensor(e, b).copy_(feats[e][b])
+        if step == 1:
+            with pytest.raises(ValueError):
+                pair.gpu.next_slot_batch(0)
+        pair.gpu.update([S.SPECA_FEATURE_IN_PLACE] * len(entries), [clock] * B, mask)
+        pair.cpu.update([U.to_oracle(f).reshape(B, -1) for f in feats], [clock] * B, mask)
+        pair.commit()
+        pair.check_tables("per-sample in place, step %d" % step)
+        pair.check_forecast([clock - 0.02] * B)
+    assert pair.gpu.stats()["update_launches"] == 0
+    # the marker means nothing to a cache that keeps tables
+    c = S.SpecaCache(entries, B, m, 1, DEV)
+    with pytest.raises(S.SpecaError) as ei:
+        c.update([S.SPECA_FEATURE_IN_PLACE, None], [1.0] * B)
+    assert ei.value.status == S.SPECA_ERR_INVALID_ARG
+    c.close()
+    pair.close()
