@@ -53,6 +53,13 @@ int main(void) {
     CHECK(strstr(speca_version(), "sm_100a") != NULL);
     CHECK(speca_cache_destroy(NULL) == SPECA_OK);
     {
+        const void* marker = SPECA_FEATURE_IN_PLACE;
+        speca_cache_config_t zero;
+        memset(&zero, 0, sizeof zero);
+        CHECK(marker != NULL && zero.layout == SPECA_LAYOUT_TABLES);   /* a zeroed config asks for the paper's tables */
+        CHECK(speca_cache_next_slot(NULL, 0, 0, NULL) == SPECA_ERR_INVALID_ARG);
+    }
+    {
         speca_cache_stats_t st;
         CHECK(sizeof st == (7 + 2 * SPECA_MAX_BATCH) * sizeof(uint64_t));   /* the binding mirrors this layout */
         CHECK(speca_cache_stats(NULL, &st) == SPECA_ERR_INVALID_ARG);
