@@ -342,6 +342,48 @@ def time_forecast_sum(h: Harness, peak: float, reps: int = 20):
             "traffic_saved_vs_separate": 1.0 - nbytes / separate}
 
 
+def time_draft_models(w: W.Workload, device: str, path: int, reps: int = 10):
+    """The other draft models of the ablation on the same tables (Newton-form divided differences, the
+    Adams-Bashforth predictor): they differ from Eq. 2-3 in host-computed scalars only, so the kernels and
+    their times must be the same. Device time of a reference step and of a forecast per basis."""
+    from paper_2509_11628_b200 import binding as S
+    dev = torch.device(device)
+    ne = len(w.entries)
+    src = W.FeatureSource(w, device)
+    feats = [[src.feature(e, k, [w.times[k]] * w.batch) for e in range(ne)] for k in range(2)]
+    outs = [torch.empty(w.batch, n, d, dtype=w.torch_dtype, device=dev) for n, d in w.entries]
+    ab = algorithmic_bytes(w, w.max_order)
+    res = {}
+    for basis, name in ((S.SPECA_BASIS_TAYLOR, "taylor_eq2_3"), (S.SPECA_BASIS_NEWTON, "newton"),
+                        (S.SPECA_BASIS_ADAMS_BASHFORTH, "adams_bashforth")):
+        cache = S.SpecaCache(w.entries, w.batch, w.max_order, w.dtype, device, basis=basis, path=path)
+        t = 1.0
+        for k in range(w.max_order + 2):
+            t -= 0.02
+            cache.update(feats[k & 1], [t] * w.batch)
+            cache.commit_step()
+        torch.cuda.synchronize(dev)
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        upd = fc = 0.0
+        for r in range(reps):
+            t -= 0.02
+            e0.record()
+            cache.update(feats[r & 1], [t] * w.batch)
+            cache.commit_step()
+            e1.record()
+            cache.forecast([t - 0.01] * w.batch, outs)
+            e2.record()
+            torch.cuda.synchronize(dev)
+            upd += e0.elapsed_time(e1)
+            fc += e1.elapsed_time(e2)
+        res[name] = {"update_ms": upd / reps, "update_gbs": ab["update"] / (upd / reps * 1e-3) / 1e9,
+                     "forecast_ms": fc / reps, "forecast_gbs": ab["forecast"] / (fc / reps * 1e-3) / 1e9}
+        cache.close()
+        del cache
+        torch.cuda.empty_cache()
+    return res
+
+
 def time_metrics(h: Harness, reps: int = 20):
     """Device time of the fused verification with each error metric (same traffic: order + 2 words per
     element of the verification entry)."""
@@ -794,6 +836,13 @@ def main():
     del h
     torch.cuda.empty_cache()
 
+    drafts = None
+    if info.world == 1 and layout == 0:
+        try:
+            drafts = time_draft_models(w, device, path)
+        except Exception as exc:  # report, do not hide
+            drafts = {"error": repr(exc)}
+
     history = None
     if info.world == 1 and path in (0, 3) and layout == 0:
         try:
@@ -891,7 +940,7 @@ def main():
         "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches,
         "clocks": clocks, "kernels": kernels, **extra,
         "frac_of_measured_peak": value / info.world / peak, "frac_of_nominal_8TBs": value / info.world / NOMINAL_HBM_GBS,
-        "multi_horizon": multi, "verify_metrics": metrics, "update_one_launch_per_entry": per_entry, "forecast_sum": fsum, "history_layout": history, "per_config": per_config, "adaptive": adaptive, "sampler": sampler,
+        "multi_horizon": multi, "verify_metrics": metrics, "update_one_launch_per_entry": per_entry, "forecast_sum": fsum, "draft_models": drafts, "history_layout": history, "per_config": per_config, "adaptive": adaptive, "sampler": sampler,
         "paper_context": {"end_to_end_speedups": {"flux_h800": 6.34, "dit_xl2_a800": 7.3, "hunyuan_video_h800": 6.1},
                           "verification_overhead": "1.67%-3.5% of a full forward pass",
                           "note": "other hardware, whole-model numbers; context only"},
