@@ -406,6 +406,20 @@ speca_status_t speca_cache_plane(const speca_cache_t* cache, int32_t entry, int3
                                  size_t* plane_stride_bytes);
 
 /*
+ * The per-sample scalars a forecast (or verification) at t_target hands to the kernels, for a sample
+ * with n_refs committed references at times t_hist[0] (latest), t_hist[1], ... (min(n_refs,
+ * max_order + 1) of them are read). Host only; touches no GPU and needs no cache.
+ *   *out_order  v = min(max_order, n_refs - 1), -1 without references: planes 0..v are read.
+ *   out_coef    SPECA_MAX_ORDER + 1 floats. TABLES: the Horner multipliers of Eq. 2, out =
+ *               plane_0 + c_0 (plane_1 + c_1 (plane_2 + ...)); TAYLOR c_i = (t_target - t_last)/(i + 1).
+ *               HISTORY: one weight per physical plane, out = sum_i c_i * plane_i, with Eq. 3's
+ *               differencing over the actual gaps folded in.
+ * Errors: INVALID_ARG.
+ */
+speca_status_t speca_forecast_weights(int32_t layout, int32_t basis, int32_t max_order, int32_t n_refs,
+                                      const double* t_hist, double t_target, int32_t* out_order, float* out_coef);
+
+/*
  * SPECA_LAYOUT_HISTORY only: device address of the plane that the next reference step of `sample` will
  * fill for `entry` (N_e * D elements of the storage type, 4 KB aligned). A model that writes its block
  * output there directly, and then passes that same address (minus sample * N_e * D elements, i.e. the

@@ -31,7 +31,7 @@ EXPORTS = [
     "speca_cache_arena_bytes", "speca_cache_create", "speca_cache_destroy", "speca_cache_reset",
     "speca_cache_update", "speca_cache_commit_step", "speca_forecast", "speca_verify",
     "speca_select_adaptive", "speca_activate", "speca_tau", "speca_cache_state", "speca_cache_plane",
-    "speca_cache_launch_count", "speca_cache_stats", "speca_cache_next_slot", "speca_status_string", "speca_last_error", "speca_version",
+    "speca_cache_launch_count", "speca_cache_stats", "speca_cache_next_slot", "speca_forecast_weights", "speca_status_string", "speca_last_error", "speca_version",
     "speca_verify_pred_static", "speca_forecast_multi", "speca_verify_metric",
     "speca_verify_partial", "speca_verify_decide", "speca_cache_get_history", "speca_cache_set_history",
     "speca_forecast_sum", "speca_verify_select",
@@ -106,6 +106,7 @@ def _lib() -> ctypes.CDLL:
     L.speca_cache_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64)]
     L.speca_cache_stats.argtypes = [vp, ctypes.POINTER(CacheStats)]
     L.speca_cache_next_slot.argtypes = [vp, i32, i32, ctypes.POINTER(vp)]
+    L.speca_forecast_weights.argtypes = [i32, i32, i32, i32, vp, dbl, ctypes.POINTER(i32), vp]
     L.speca_status_string.argtypes = [i32]
     L.speca_status_string.restype = ctypes.c_char_p
     L.speca_last_error.argtypes = [vp]
@@ -325,6 +326,15 @@ def speca_cache_plane(cache, entry: int, sample: int):
     s = ctypes.c_size_t(0)
     _check(_lib().speca_cache_plane(cache, entry, sample, ctypes.byref(p), ctypes.byref(s)), cache)
     return p.value, s.value
+
+
+def speca_forecast_weights(layout: int, basis: int, max_order: int, n_refs: int, t_hist: Sequence[float], t_target: float):
+    """(order, coefficients) a forecast at ``t_target`` hands to the kernels; host only, no GPU needed."""
+    order = ctypes.c_int32(0)
+    coef = (ctypes.c_float * (SPECA_MAX_ORDER + 1))()
+    _check(_lib().speca_forecast_weights(layout, basis, max_order, n_refs, _doubles(t_hist), float(t_target),
+                                         ctypes.byref(order), coef))
+    return order.value, [float(x) for x in coef]
 
 
 def speca_cache_next_slot(cache, entry: int, sample: int) -> int:

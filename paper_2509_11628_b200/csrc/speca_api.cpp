@@ -909,6 +909,31 @@ speca_status_t speca_cache_plane(const speca_cache_t* c, int32_t entry, int32_t 
     return SPECA_OK;
 }
 
+speca_status_t speca_forecast_weights(int32_t layout, int32_t basis, int32_t max_order, int32_t n_refs,
+                                      const double* t_hist, double t_target, int32_t* out_order, float* out_coef) {
+    if (t_hist == nullptr || out_order == nullptr || out_coef == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (layout != SPECA_LAYOUT_TABLES && layout != SPECA_LAYOUT_HISTORY) return SPECA_ERR_INVALID_ARG;
+    if (basis != SPECA_BASIS_TAYLOR && basis != SPECA_BASIS_NEWTON && basis != SPECA_BASIS_ADAMS_BASHFORTH)
+        return SPECA_ERR_INVALID_ARG;
+    if (max_order < 0 || max_order > SPECA_MAX_ORDER || n_refs < 0 || !std::isfinite(t_target)) return SPECA_ERR_INVALID_ARG;
+    speca_cache tmp;
+    tmp.m = max_order;
+    tmp.basis = basis;
+    tmp.layout = layout;
+    tmp.n_refs[0] = n_refs;
+    const int known = n_refs < max_order + 1 ? n_refs : max_order + 1;
+    for (int i = 0; i <= SPECA_MAX_ORDER; ++i)
+        tmp.t_hist[0][i] = i < known ? t_hist[i] : std::numeric_limits<double>::quiet_NaN();
+    for (int i = 0; i < known; ++i)
+        if (!std::isfinite(t_hist[i])) return SPECA_ERR_INVALID_ARG;
+    int order = -1;
+    float coef[kCoef] = {};
+    forecast_coefficients(&tmp, 0, t_target, &order, coef);
+    *out_order = order;
+    for (int i = 0; i < kCoef; ++i) out_coef[i] = coef[i];
+    return SPECA_OK;
+}
+
 speca_status_t speca_cache_next_slot(const speca_cache_t* c, int32_t entry, int32_t sample, void** out) {
     if (c == nullptr || out == nullptr) return SPECA_ERR_INVALID_ARG;
     if (c->layout != SPECA_LAYOUT_HISTORY) return SPECA_ERR_UNSUPPORTED;
