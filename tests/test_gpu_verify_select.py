@@ -213,3 +213,49 @@ def test_speculative_steps_replay_from_a_cuda_graph(S, U):
         assert eager["acc"][0].cpu().tolist() == want and eager["masks"][1].cpu().tolist() == want
         assert eager["outs"][1][1][want.index(0)].abs().sum().item() == 0     # dropped after step 1: not forecast at step 2
     pair.close()
+
+
+def test_two_handles_on_two_streams_do_not_disturb_each_other(S, U):
+    """Each handle carries its own reduction scratch and ticket, so two caches can work on two streams at
+    once: results equal those of running them one after the other."""
+    entries = [(40, 1030), (301, 1160)]
+    B, m = 4, 2
+    gen = torch.Generator(device=DEV).manual_seed(57)
+    caches = [S.SpecaCache(entries, B, m, 1, DEV) for _ in range(2)]
+    feats = [[rand_feats(entries, B, torch.bfloat16, gen) for _ in range(3)] for _ in range(2)]
+    fresh = [rand_feats(entries, B, torch.bfloat16, gen)[1] for _ in range(2)]
+
+    def run(streams, rounds=6):
+        res = []
+        for c in caches:
+            c.reset()
+        bufs = [dict(outs=[torch.zeros(B, n, d, dtype=torch.bfloat16, device=DEV) for n, d in entries],
+                     err=torch.zeros(rounds, B, device=DEV), acc=torch.zeros(rounds, B, dtype=torch.uint8, device=DEV),
+                     cur=torch.ones(B, dtype=torch.uint8, device=DEV), nxt=torch.zeros(rounds, B, dtype=torch.uint8, device=DEV),
+                     cnt=torch.zeros(B, dtype=torch.int32, device=DEV)) for _ in caches]
+        torch.cuda.synchronize()
+        for k, t in enumerate((1.0, 0.93, 0.9)):
+            for i, c in enumerate(caches):
+                c.update(feats[i][k], [t] * B, stream=streams[i])
+                c.commit_step()
+        for r in range(rounds):
+            tt = [0.88 - 0.01 * r] * B
+            for i, c in enumerate(caches):      # interleaved enqueue: the two streams overlap on the device
+                c.forecast(tt, bufs[i]["outs"], stream=streams[i])
+                c.verify_select(fresh[i], tt, [1e30] * B, bufs[i]["err"][r], bufs[i]["acc"][r], bufs[i]["cur"],
+                                bufs[i]["nxt"][r], 1 << 20, 1, bufs[i]["cnt"], stream=streams[i])
+        torch.cuda.synchronize()
+        return [(b["err"].clone(), b["acc"].clone(), b["nxt"].clone(), b["cnt"].clone(), [o.clone() for o in b["outs"]]) for b in bufs]
+
+    main = torch.cuda.current_stream()
+    serial = run([main, main])
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    overlapped = run([s1, s2])
+    for a, b_ in zip(serial, overlapped):
+        for x, y in zip(a[:4], b_[:4]):
+            assert torch.equal(x.view(torch.uint8), y.view(torch.uint8))
+        for x, y in zip(a[4], b_[4]):
+            assert torch.equal(x.view(torch.uint8), y.view(torch.uint8))
+    assert bool((serial[0][1] == 1).all()) and serial[0][3].tolist() == [6] * B
+    for c in caches:
+        c.close()
