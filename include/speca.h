@@ -93,16 +93,6 @@ typedef enum {
 } speca_path_t;
 
 /*
- * Error metric of the verification. Eq. 4 is the relative l2 error (the paper's default); the
- * appendix on error metrics also evaluates l1, l-infinity and cosine similarity, named there
- * without formulas. The forms used here (p = forecast, f = computed feature, all over one sample):
- *   L2      ||p - f||_2   / (||f||_2   + eps)
- *   L1      ||p - f||_1   / (||f||_1   + eps)
- *   LINF    ||p - f||_inf / (||f||_inf + eps)
- *   COSINE  1 - <p, f> / (||p||_2 ||f||_2 + eps)     (a distance: 0 = same direction)
- * In every case the sample is accepted iff the value is <= tau, and a NaN rejects.
- */
-/*
  * What the cache keeps per (entry, sample) in its max_order + 1 planes.
  * TABLES   the difference quotients of Eq. 3, rewritten at every reference step (the paper's derivative
  *          tables): an update reads the feature and the old planes and writes all planes.
@@ -118,6 +108,16 @@ typedef enum {
     SPECA_LAYOUT_HISTORY = 1
 } speca_layout_t;
 
+/*
+ * Error metric of the verification. Eq. 4 is the relative l2 error (the paper's default); the
+ * appendix on error metrics also evaluates l1, l-infinity and cosine similarity, named there
+ * without formulas. The forms used here (p = forecast, f = computed feature, all over one sample):
+ *   L2      ||p - f||_2   / (||f||_2   + eps)
+ *   L1      ||p - f||_1   / (||f||_1   + eps)
+ *   LINF    ||p - f||_inf / (||f||_inf + eps)
+ *   COSINE  1 - <p, f> / (||p||_2 ||f||_2 + eps)     (a distance: 0 = same direction)
+ * In every case the sample is accepted iff the value is <= tau, and a NaN rejects.
+ */
 typedef enum {
     SPECA_METRIC_L2 = 0,
     SPECA_METRIC_L1 = 1,
