@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # order 2, bf16; profiles/dram_traffic_flux_full_size.md). Other workloads scale by the elements a
 # launch covers. Set an entry to None when its kernel changes until the counters have been taken again.
 NCU_DRAM_BYTES_PER_ELEM_HISTORY_UPDATE = 3.955   # profiles/history_layout_flux_full_size.md
-NCU_DRAM_BYTES_PER_ELEM = {"update": 11.987, "forecast": 8.042, "verify": 8.107}
+NCU_DRAM_BYTES_PER_ELEM = {"update": 12.000, "forecast": 8.060, "verify": 8.147}
 
 
 def measured_peak():
@@ -181,8 +181,9 @@ class Harness:
         return [t_ref] * self.B, [t_ref - 0.5 * gap] * self.B
 
     def step(self, events=None, feats=None, fresh=None):
-        """update -> commit -> forecast -> verify -> select on the current stream; verify and select are
-        one launch (speca_verify_select) unless the harness was made with fused_select=False."""
+        """update -> commit -> forecast -> verify -> select on the current stream: three launches
+        (speca_cache_update_activate, speca_forecast, speca_verify_select), or five with
+        fused_select=False (update, activate, forecast, verify, select)."""
         S, c, w = self.S, self.cache, self.w
         j = self.j
         self.j += 1
@@ -192,11 +193,17 @@ class Harness:
         tau = [S.speca_tau(w.tau0, w.beta, w.total_steps - (j % w.total_steps), w.total_steps)] * self.B
         if events is not None:
             events[0].record()
-        c.update(feats, t_ref)
-        c.commit_step()
-        if events is not None:
-            events[1].record()
-        c.activate(None, self.spec, self.active)
+        if self.fused_select:
+            c.update_activate(feats, t_ref, None, self.spec, self.active)   # the re-arming rides in the update launch
+            c.commit_step()
+            if events is not None:
+                events[1].record()
+        else:
+            c.update(feats, t_ref)
+            c.commit_step()
+            if events is not None:
+                events[1].record()
+            c.activate(None, self.spec, self.active)
         if events is not None:
             events[2].record()
         c.forecast(t_tgt, self.outs, self.active)
@@ -783,7 +790,7 @@ def main():
                     help="what the cache keeps: the paper's difference tables (default) or the raw features of "
                          "the last references (speca_layout_t)")
     ap.add_argument("--separate-select", action="store_true",
-                    help="speca_verify then speca_select_adaptive as two launches instead of speca_verify_select")
+                    help="five launches per step (update, activate, forecast, verify, select) instead of the three fused ones")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-adaptive", action="store_true",
                     help="skip the B=8 sample-adaptive sweep (orders 1-3, horizon 1-6) reported under 'adaptive'")
@@ -933,8 +940,10 @@ def main():
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": info.world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": dict(workload_config(w), layout=args.layout, select="its own launch (speca_select_adaptive)" if args.separate_select
-                       else "inside the verify launch (speca_verify_select)"),
+        "config": dict(workload_config(w), layout=args.layout, select="its own launch (speca_select_adaptive); re-arming its own launch (speca_activate)"
+                       if args.separate_select else
+                       "inside the verify launch (speca_verify_select); re-arming inside the update launch "
+                       "(speca_cache_update_activate)"),
         "metric_note": "value = algorithmic bytes of the whole step (update + forecast + verify/select) / step time; "
                        "forecast + verify alone (one speculative step) is forecast_verify_gbs, the update alone kernels.update.gbs",
         "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches,

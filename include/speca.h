@@ -200,6 +200,17 @@ speca_status_t speca_cache_update(speca_cache_t* cache, const void* const* feats
                                   const uint8_t* host_sample_mask, void* stream);
 
 /*
+ * speca_cache_update that also re-arms the masked samples for speculation, as speca_activate would
+ * (dev_active_mask[b] = 1, dev_spec_count[b] = 0 for every masked sample), in the same launch: after a
+ * reference step the samples that took it may speculate again. When the call copies nothing (features
+ * already in place, or an empty mask) the re-arming runs as a launch of its own. Both device buffers are
+ * required. Errors: those of speca_cache_update and speca_activate.
+ */
+speca_status_t speca_cache_update_activate(speca_cache_t* cache, const void* const* feats, const double* t_ref,
+                                           const uint8_t* host_sample_mask, int32_t* dev_spec_count,
+                                           uint8_t* dev_active_mask, void* stream);
+
+/*
  * Close a reference step: push t_ref into each masked sample's reference history and raise its
  * reference count. Host state only. Errors: STATE if some entry has not been updated for
  * exactly the masked samples since the last commit, or no update is pending.

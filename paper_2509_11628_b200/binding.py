@@ -29,7 +29,7 @@ SPECA_MAX_ORDER, SPECA_MAX_BATCH, SPECA_MAX_ENTRIES, SPECA_MAX_HORIZON = 4, 64, 
 
 EXPORTS = [
     "speca_cache_arena_bytes", "speca_cache_create", "speca_cache_destroy", "speca_cache_reset",
-    "speca_cache_update", "speca_cache_commit_step", "speca_forecast", "speca_verify",
+    "speca_cache_update", "speca_cache_update_activate", "speca_cache_commit_step", "speca_forecast", "speca_verify",
     "speca_select_adaptive", "speca_activate", "speca_tau", "speca_cache_state", "speca_cache_plane",
     "speca_cache_launch_count", "speca_cache_stats", "speca_cache_next_slot", "speca_forecast_weights", "speca_status_string", "speca_last_error", "speca_version",
     "speca_verify_pred_static", "speca_forecast_multi", "speca_verify_metric",
@@ -85,6 +85,7 @@ def _lib() -> ctypes.CDLL:
     L.speca_cache_destroy.argtypes = [vp]
     L.speca_cache_reset.argtypes = [vp, vp]
     L.speca_cache_update.argtypes = [vp, vp, vp, vp, vp]
+    L.speca_cache_update_activate.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.speca_cache_commit_step.argtypes = [vp]
     L.speca_forecast.argtypes = [vp, vp, vp, vp, vp]
     L.speca_forecast_sum.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]
@@ -212,6 +213,12 @@ def speca_cache_reset(cache, host_sample_mask=None) -> None:
 def speca_cache_update(cache, feats, t_ref, host_sample_mask=None, stream=None) -> None:
     _check(_lib().speca_cache_update(cache, _ptr_array(feats), _doubles(t_ref), _bytes(host_sample_mask),
                                      _stream_ptr(stream)), cache)
+
+
+def speca_cache_update_activate(cache, feats, t_ref, host_sample_mask, dev_spec_count, dev_active_mask, stream=None) -> None:
+    """speca_cache_update + speca_activate for the masked samples in one launch."""
+    _check(_lib().speca_cache_update_activate(cache, _ptr_array(feats), _doubles(t_ref), _bytes(host_sample_mask),
+                                              _dev_ptr(dev_spec_count), _dev_ptr(dev_active_mask), _stream_ptr(stream)), cache)
 
 
 def speca_cache_commit_step(cache) -> None:
@@ -401,6 +408,9 @@ class SpecaCache:
 
     def update(self, feats, t_ref, mask=None, stream=None):
         speca_cache_update(self.handle, feats, t_ref, mask, stream)
+
+    def update_activate(self, feats, t_ref, mask, spec_count, active, stream=None):
+        speca_cache_update_activate(self.handle, feats, t_ref, mask, spec_count, active, stream)
 
     def commit_step(self):
         speca_cache_commit_step(self.handle)

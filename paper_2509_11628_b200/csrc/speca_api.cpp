@@ -380,8 +380,14 @@ speca_status_t speca_cache_reset(speca_cache_t* c, const uint8_t* host_sample_ma
     return SPECA_OK;
 }
 
-speca_status_t speca_cache_update(speca_cache_t* c, const void* const* feats, const double* t_ref,
-                                  const uint8_t* host_sample_mask, void* stream) {
+}  // extern "C"
+
+namespace {
+
+// speca_cache_update, optionally re-arming the masked samples (act_spec / act_active non-null) in the
+// same launch.
+speca_status_t update_impl(speca_cache_t* c, const void* const* feats, const double* t_ref,
+                           const uint8_t* host_sample_mask, void* stream, int32_t* act_spec, uint8_t* act_active) {
     if (c == nullptr) return SPECA_ERR_INVALID_ARG;
     if (feats == nullptr || t_ref == nullptr) return fail(c, SPECA_ERR_INVALID_ARG, "update: null argument");
     uint8_t mask[SPECA_MAX_BATCH];
@@ -464,10 +470,28 @@ speca_status_t speca_cache_update(speca_cache_t* c, const void* const* feats, co
         const uint32_t n_tiles = p.tile_hi - p.tile_lo;
         const uint32_t full = static_cast<uint32_t>(c->sm_count * stream_ctas_per_sm(c->path, true, c->dtype, launch_order(p.order, c->B)));
         const int grid = static_cast<int>(n_tiles < full ? n_tiles : full);
+        uint64_t bits = 0;
+        for (int b = 0; b < c->B; ++b)
+            if (mask[b]) bits |= uint64_t(1) << b;
+        if (act_active != nullptr && c->path != SPECA_PATH_BULK) {  // the kernel's first CTA re-arms the samples
+            p.act_spec = act_spec;
+            p.act_active = act_active;
+            p.act_bits = bits;
+            act_active = nullptr;
+        }
         cudaError_t ce = launch_update(p, c->dtype, c->path, grid, static_cast<cudaStream_t>(stream));
         if (ce != cudaSuccess) return cuda_fail(c, ce, "update launch");
         c->launches += 1;
         c->stats.update_launches += 1;
+    }
+    if (act_active != nullptr && any_sample) {  // nothing was copied (or the staged kernels ran): a launch of its own
+        uint64_t bits = 0;
+        for (int b = 0; b < c->B; ++b)
+            if (mask[b]) bits |= uint64_t(1) << b;
+        cudaError_t ce = launch_activate(bits, c->B, act_spec, act_active, static_cast<cudaStream_t>(stream));
+        if (ce != cudaSuccess) return cuda_fail(c, ce, "activate launch");
+        c->launches += 1;
+        c->stats.activate_launches += 1;
     }
     if (!c->pending) {
         c->pending = true;
@@ -479,6 +503,26 @@ speca_status_t speca_cache_update(speca_cache_t* c, const void* const* feats, co
     for (int e = 0; e < c->n_entries; ++e)
         if (feats[e] != nullptr) c->entry_updated[e] = 1;
     return SPECA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+speca_status_t speca_cache_update(speca_cache_t* c, const void* const* feats, const double* t_ref,
+                                  const uint8_t* host_sample_mask, void* stream) {
+    return update_impl(c, feats, t_ref, host_sample_mask, stream, nullptr, nullptr);
+}
+
+speca_status_t speca_cache_update_activate(speca_cache_t* c, const void* const* feats, const double* t_ref,
+                                           const uint8_t* host_sample_mask, int32_t* dev_spec_count,
+                                           uint8_t* dev_active_mask, void* stream) {
+    if (c == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (dev_spec_count == nullptr || dev_active_mask == nullptr)
+        return fail(c, SPECA_ERR_INVALID_ARG, "update_activate: null argument");
+    if (reinterpret_cast<uintptr_t>(dev_spec_count) % 4 != 0)
+        return fail(c, SPECA_ERR_ALIGNMENT, "update_activate: dev_spec_count must be 4-byte aligned");
+    return update_impl(c, feats, t_ref, host_sample_mask, stream, dev_spec_count, dev_active_mask);
 }
 
 speca_status_t speca_cache_commit_step(speca_cache_t* c) {

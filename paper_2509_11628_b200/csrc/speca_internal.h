@@ -54,6 +54,10 @@ struct StreamParams {
     // A cache that keeps raw features (SPECA_LAYOUT_HISTORY):
     // update:   order = 0, slot[b] = plane that receives the feature
     // forecast: weighted = 1, coef[b][i] = weight of physical plane i (i <= order): out = sum_i coef_i * plane_i
+    // update only, optional: samples (bits of act_bits) to re-arm for speculation in the same launch
+    int32_t* act_spec;
+    uint8_t* act_active;
+    uint64_t act_bits;
     int8_t order[SPECA_MAX_BATCH];
     uint8_t slot[SPECA_MAX_BATCH];
     int32_t weighted;

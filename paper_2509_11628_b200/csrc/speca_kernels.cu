@@ -440,6 +440,13 @@ template <int DT, int V, bool UPDATE, int W, int NT, int U, int C, int MINB>
 __global__ void __launch_bounds__(NT, MINB) stream_kernel(const __grid_constant__ StreamParams p) {
     constexpr uint32_t kChunk = static_cast<uint32_t>(NT) * U * W / Elem<DT>::kBytes;  // elements
     constexpr uint32_t kTile = kChunk * C;
+    if constexpr (UPDATE) {
+        // a reference step re-arms its samples for speculation: folded into this launch on request
+        if (p.act_active != nullptr && blockIdx.x == 0 && threadIdx.x < SPECA_MAX_BATCH && ((p.act_bits >> threadIdx.x) & 1ull)) {
+            p.act_active[threadIdx.x] = 1;
+            p.act_spec[threadIdx.x] = 0;
+        }
+    }
     uint32_t seg = p.seg_lo, seg_first = 0, seg_end = 0;  // tiles [seg_first, seg_end) belong to `seg`
     SegDesc sd = {};
     int v = -1;

@@ -162,7 +162,6 @@ class SpecaCacheBackend:
         return self.h_active.tolist()
 
     def reference_step(self, feats, t_ref, mask):
-        self.cache.update(feats, t_ref, mask)
+        self.cache.update_activate(feats, t_ref, mask, self.spec, self.active)   # Eq. 3 and the re-arming, one launch
         self.cache.commit_step()
-        self.cache.activate(mask, self.spec, self.active)
         self._fetch(with_decisions=False)

@@ -259,3 +259,55 @@ def test_two_handles_on_two_streams_do_not_disturb_each_other(S, U):
     assert bool((serial[0][1] == 1).all()) and serial[0][3].tolist() == [6] * B
     for c in caches:
         c.close()
+
+
+@pytest.mark.parametrize("path,layout", [(0, 0), (1, 0), (2, 0), (0, 1)])
+def test_update_that_also_rearms_the_samples(S, U, path, layout):
+    """speca_cache_update_activate = speca_cache_update + speca_activate for the masked samples: same
+    tables, same mask and counters, one launch fewer (the staged kernels keep a launch of their own)."""
+    entries = [(37, 129), (64, 384)]
+    B, m = 5, 2
+    gen = torch.Generator(device=DEV).manual_seed(61)
+    a = S.SpecaCache(entries, B, m, 1, DEV, path=path, layout=layout)
+    b = S.SpecaCache(entries, B, m, 1, DEV, path=path, layout=layout)
+    act = [torch.tensor([0, 1, 0, 1, 0], dtype=torch.uint8, device=DEV) for _ in range(2)]
+    cnt = [torch.tensor([3, 1, 4, 1, 5], dtype=torch.int32, device=DEV) for _ in range(2)]
+    clock = 1.0
+    for step, mask in enumerate([None, [1, 0, 1, 0, 0], [0, 0, 0, 0, 1], None]):
+        clock -= 0.04
+        feats = rand_feats(entries, B, torch.bfloat16, gen)
+        la, lb = a.launches, b.launches
+        a.update(feats, [clock] * B, mask)
+        a.commit_step()
+        a.activate(mask, cnt[0], act[0])
+        b.update_activate(feats, [clock] * B, mask, cnt[1], act[1])
+        b.commit_step()
+        torch.cuda.synchronize()
+        assert a.launches - la == 2 and b.launches - lb == (2 if path == 2 else 1)
+        la, lb = a.launches, b.launches
+        assert torch.equal(act[0], act[1]) and torch.equal(cnt[0], cnt[1])
+        if step >= 1:     # every sample has a reference by now: the two caches must forecast the same bits
+            oa = [torch.zeros(B, n, d, dtype=torch.bfloat16, device=DEV) for n, d in entries]
+            ob = [torch.zeros(B, n, d, dtype=torch.bfloat16, device=DEV) for n, d in entries]
+            a.forecast([clock - 0.02] * B, oa)
+            b.forecast([clock - 0.02] * B, ob)
+            torch.cuda.synchronize()
+            assert all(torch.equal(x.view(torch.int16), y.view(torch.int16)) for x, y in zip(oa, ob))
+        act[0][2] = act[1][2] = 0                      # something for the next step to re-arm
+        cnt[0][2] = cnt[1][2] = 7
+    if layout == 1:   # features already in place: nothing is copied, the re-arming runs on its own
+        nxt = rand_feats(entries, B, torch.bfloat16, gen)
+        for e in range(len(entries)):
+            for smp in range(B):      # the masked steps above left the samples at different ring positions
+                b.next_slot_tensor(e, smp).copy_(nxt[e][smp])
+        lb = b.launches
+        b.update_activate([S.SPECA_FEATURE_IN_PLACE] * len(entries), [clock - 0.04] * B, None, cnt[1], act[1])
+        b.commit_step()
+        torch.cuda.synchronize()
+        st = b.stats()
+        assert b.launches - lb == 1 and st["activate_launches"] == 1 and act[1].tolist() == [1] * B and cnt[1].tolist() == [0] * B
+    err = S.SpecaError
+    with pytest.raises(err) as ei:
+        b.update_activate(rand_feats(entries, B, torch.bfloat16, gen), [0.1] * B, None, None, act[1])
+    assert ei.value.status == S.SPECA_ERR_INVALID_ARG
+    a.close(); b.close()
