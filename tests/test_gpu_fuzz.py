@@ -1,7 +1,7 @@
 """Seeded random scenarios: random shapes, batch sizes, orders, bases, storage types and kernel paths,
-and a random sequence of masked reference steps, speculative steps (forecast, verify under a random
-metric, the fused verify + continuation call) and resets -- every result compared with the oracle.
-The hand-written cases elsewhere pick the shapes someone thought of; this file picks the others."""
+and a random sequence of masked reference steps, speculative steps (forecast, multi-horizon and summed
+forecasts, verify under a random metric, the fused verify + continuation call) and resets -- every result
+compared with the oracle. The hand-written cases elsewhere pick the shapes someone thought of; this file picks the others."""
 import numpy as np
 import pytest
 import torch
@@ -95,6 +95,28 @@ def test_random_scenario(S, U, seed):
             if rng.random() < 0.3:
                 act = list(have)
             outs = pair.check_forecast(t, active=act, sentinel=2.5, what=what + " step %d forecast" % step)
+            # several targets at once: row 0 is this very forecast, bit for bit
+            t2 = [x - 0.007 for x in t]
+            mask_dev = torch.tensor(act, dtype=torch.uint8, device=DEV)
+            multi = [torch.full((2, B, n, d), 2.5, dtype=pair.tdt, device=DEV) for n, d in entries]
+            pair.gpu.forecast_multi([t, t2], multi, mask_dev)
+            # and an entry consumed twice as a sum, against the oracle's sum
+            e0 = int(rng.integers(0, len(entries)))
+            total = torch.full((B, *entries[e0]), 2.5, dtype=pair.tdt, device=DEV)
+            pair.gpu.forecast_sum([e0, e0], t, total, None, mask_dev)
+            torch.cuda.synchronize()
+            for e in range(len(entries)):
+                assert torch.equal(multi[e][0].view(torch.uint8), outs[e].view(torch.uint8)), what + " multi row 0 entry %d" % e
+            init = U.to_oracle(torch.full((B, entries[e0][0] * entries[e0][1]), 2.5, dtype=pair.tdt))
+            want_sum = pair.cpu.forecast_sum([e0, e0], t, None, act, out=init)
+            got_sum = U.to_oracle(total).reshape(B, -1)
+            for b in range(B):
+                if not act[b]:
+                    assert np.array_equal(got_sum[b], want_sum[b]), what
+                    continue
+                scale = 2 * (pair.history_scale(e0, b, t[b]) if layout == 1 else
+                             U.term_scale(pair.cpu.planes[e0][b], pair.forecast_weights(b, t[b])))
+                U.assert_close_storage(got_sum[b], want_sum[b], dtype, scale, what + " sum of entry %d twice, sample %d" % (e0, b))
             level = torch.tensor(rng.choice([0.0, 0.02, 0.3], B), device=DEV, dtype=torch.float32).view(B, 1, 1)
             fresh = (outs[pair.vidx].float() + level * torch.randn(B, nv, dv, generator=gen, device=DEV)).to(pair.tdt)
             metric = int(rng.integers(0, 4))
