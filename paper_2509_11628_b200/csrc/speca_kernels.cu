@@ -197,6 +197,29 @@ __device__ __forceinline__ uint32_t find_segment(const uint32_t* __restrict__ ti
     return lo;
 }
 
+// The same, starting from a guess: caches of one model hold runs of equally sized segments, so the
+// segment of a tile further on is usually (tiles ahead) / (tiles per segment) segments ahead. The
+// guess costs two independent loads; the search runs only when it is wrong. Returns the segment and
+// its tile range.
+__device__ __forceinline__ uint32_t next_segment(const uint32_t* __restrict__ tile_start, uint32_t seg, uint32_t seg_hi,
+                                                 uint32_t tile, uint32_t& seg_first, uint32_t& seg_end) {
+    if (seg_end > seg_first) {
+        const uint32_t guess = seg + (tile - seg_first) / (seg_end - seg_first);
+        if (guess < seg_hi) {
+            const uint32_t a = __ldg(tile_start + guess), b = __ldg(tile_start + guess + 1);
+            if (a <= tile && tile < b) {
+                seg_first = a;
+                seg_end = b;
+                return guess;
+            }
+        }
+    }
+    seg = find_segment(tile_start, seg, seg_hi, tile);
+    seg_first = __ldg(tile_start + seg);
+    seg_end = __ldg(tile_start + seg + 1);
+    return seg;
+}
+
 // ------------------------------------------------------------------------------------------------
 // per-tile bodies
 // ------------------------------------------------------------------------------------------------
@@ -455,9 +478,7 @@ __global__ void __launch_bounds__(NT, MINB) stream_kernel(const __grid_constant_
     uint32_t slot = 0;  // history layout, update only: the plane that receives the feature
     for (uint32_t tile = p.tile_lo + blockIdx.x; tile < p.tile_hi; tile += gridDim.x) {
         if (tile >= seg_end) {  // tiles only grow: look forward from the current segment
-            seg = find_segment(p.tile_start, seg, p.seg_hi, tile);
-            seg_first = __ldg(p.tile_start + seg);
-            seg_end = __ldg(p.tile_start + seg + 1);
+            seg = next_segment(p.tile_start, seg, p.seg_hi, tile, seg_first, seg_end);
             sd = p.segs[seg];
             v = p.order[sd.sample];
             io = static_cast<char*>(p.io[sd.entry]);
@@ -575,9 +596,7 @@ __global__ void __launch_bounds__(NT, MINB) forecast_multi_kernel(const __grid_c
     uint64_t target_stride = 0;  // bytes between consecutive targets of this entry's output
     for (uint32_t tile = p.tile_lo + blockIdx.x; tile < p.tile_hi; tile += gridDim.x) {
         if (tile >= seg_end) {
-            seg = find_segment(p.tile_start, seg, p.seg_hi, tile);
-            seg_first = __ldg(p.tile_start + seg);
-            seg_end = __ldg(p.tile_start + seg + 1);
+            seg = next_segment(p.tile_start, seg, p.seg_hi, tile, seg_first, seg_end);
             sd = p.segs[seg];
             v = p.order[sd.sample];
             io = static_cast<char*>(p.io[sd.entry]);
