@@ -2,21 +2,28 @@
 """Benchmark of the SpeCa feature-cache hot path on B200.
 
 One *step* is one pass of the whole path over one batch of synthetic input: a reference-step
-cache update of every entry (Eq. 3), a forecast of every entry (Eq. 2), the fused
-forecast+verification of the verification entry (Eq. 4 and the accept rule) and the per-sample
-selection. The headline value is the algorithmic bytes of a step divided by its device time
-(GB/s), with the inputs already resident in HBM; ``e2e`` repeats the measurement with the step's
-inputs in pinned host memory and its outputs copied back.
+cache update of every entry (Eq. 3), a forecast of every entry (Eq. 2) -- the verification entry's
+forecast comes out of the verification launch -- the fused forecast + verification of the
+verification entry (Eq. 4 and the accept rule) and the per-sample selection. ``value`` is the
+algorithmic bytes of a step divided by its device time (GB/s), with the inputs already resident in
+HBM; ``e2e`` repeats the measurement with the step's inputs in pinned host memory and its outputs
+copied back.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config flux] [--impl reference]
+                    [--detail PATH] [--full]
 
-Prints exactly one JSON line (rank 0).
+The LAST line printed (rank 0) is one compact JSON object (under 2 KB) with the headline numbers.
+Everything else -- per-kernel tables, the other configurations, the optional sweeps of ``--full`` --
+goes to the JSON file named by ``--detail``. With ``--gpus N`` and no process group in the
+environment the script starts its own N ranks (one per GPU).
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
+import subprocess
 import sys
 import threading
 import time
@@ -31,22 +38,25 @@ from paper_2509_11628_b200 import dist as D  # noqa: E402
 from paper_2509_11628_b200 import workloads as W  # noqa: E402
 
 METRIC = "forecast+verify GB/s"
+VALUE_COVERS = "update+forecast+verify+select (whole step)"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+MAX_LINE_BYTES = 2000
 
-# DRAM bytes per cached element per launch: (dram__bytes_read.sum + dram__bytes_write.sum) / elements,
-# from the one-pass ncu capture of this benchmark's default workload at full size (FLUX-shaped cache,
-# order 2, bf16; profiles/dram_traffic_flux_full_size.md). Other workloads scale by the elements a
-# launch covers. Set an entry to None when its kernel changes until the counters have been taken again.
-NCU_DRAM_BYTES_PER_ELEM_HISTORY_UPDATE = 3.956   # profiles/history_layout_flux_full_size.md
-NCU_DRAM_BYTES_PER_ELEM = {"update": 12.000, "forecast": 8.052, "verify": 8.147}
+# DRAM bytes per cached element per launch: (dram__bytes_read.sum + dram__bytes_write.sum) / elements
+# from the ncu capture of the DiT-XL/2-shaped case (1.6 GB cache; see the file named in TRAFFIC_SOURCE).
+# The kernels are reuse-free streams, so traffic grows in proportion to the elements a launch covers;
+# other workloads scale by that. An entry is None while its kernel has changed since the counters
+# were taken.
+NCU_DRAM_BYTES_PER_ELEM = {"update": 11.83, "forecast": 7.93, "verify": None}
+TRAFFIC_SOURCE = "ncu dram bytes/elem on the DiT-shaped capture (profiles/stream_kernels_dit_xl2.md) x elems"
 
 
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(path) as f:
-            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+            return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback"
 
@@ -57,18 +67,20 @@ def make_workload(name: str) -> W.Workload:
     return W.BY_NAME[name]()
 
 
-def algorithmic_bytes(w: W.Workload, order: int, layout: int = 0):
+def algorithmic_bytes(w: W.Workload, order: int, layout: int = 0, pred_from_verify: bool = True):
     """Bytes a step must move per kernel, from the per-element figures: update reads the feature
     and `order` old planes and writes order+1 planes (a cache that keeps raw features, layout 1, reads
     the feature and writes one plane); forecast reads order+1 planes and writes one; verify reads
-    order+1 planes and the fresh feature."""
+    order+1 planes and the fresh feature. With `pred_from_verify` the verification entry's forecast
+    is written by the verify launch (one more word per element there) and left out of the forecast
+    launch."""
     eb = w.elem_bytes
     n_all = w.elems_per_order
     n_ver = w.batch * w.entry_elems(w.vidx)
     return {
         "update": (2 if layout == 1 else 2 * order + 2) * eb * n_all,
-        "forecast": (order + 2) * eb * n_all,
-        "verify": (order + 2) * eb * n_ver,
+        "forecast": (order + 2) * eb * (n_all - n_ver if pred_from_verify else n_all),
+        "verify": (order + (3 if pred_from_verify else 2)) * eb * n_ver,
         "select": 0,
     }
 
@@ -170,7 +182,6 @@ class Harness:
         self.spec = torch.zeros(self.B, dtype=torch.int32, device=self.device)
         self.idx = torch.zeros(self.B, dtype=torch.int32, device=self.device)
         self.n_active = torch.zeros(1, dtype=torch.int32, device=self.device)
-        self.ones = [1] * self.B
         self.j = 0
         self.t_base = w.times[self.m]
         torch.cuda.synchronize(self.device)
@@ -180,16 +191,20 @@ class Harness:
         t_ref = self.t_base - gap * (j + 1)
         return [t_ref] * self.B, [t_ref - 0.5 * gap] * self.B
 
-    def step(self, events=None, feats=None, fresh=None):
+    def step(self, events=None, feats=None, fresh=None, outs=None):
         """update -> commit -> forecast -> verify -> select on the current stream: three launches
         (speca_cache_update_activate, speca_forecast, speca_verify_select), or five with
-        fused_select=False (update, activate, forecast, verify, select)."""
+        fused_select=False (update, activate, forecast, verify, select). The verification entry is
+        forecast once: by the verification launch, which writes it to that entry's output."""
         S, c, w = self.S, self.cache, self.w
         j = self.j
         self.j += 1
         t_ref, t_tgt = self.times_for(j)
         feats = feats if feats is not None else self.feats[j & 1]
         fresh = fresh if fresh is not None else self.fresh[j & 1]
+        outs = outs if outs is not None else self.outs
+        others = list(outs)
+        others[w.vidx] = None
         tau = [S.speca_tau(w.tau0, w.beta, w.total_steps - (j % w.total_steps), w.total_steps)] * self.B
         if events is not None:
             events[0].record()
@@ -206,17 +221,17 @@ class Harness:
             c.activate(None, self.spec, self.active)
         if events is not None:
             events[2].record()
-        c.forecast(t_tgt, self.outs, self.active)
+        c.forecast(t_tgt, others, self.active)
         if events is not None:
             events[3].record()
         if self.fused_select:
             c.verify_select(fresh, t_tgt, tau, self.err, self.accept, self.active, self.active_next, 1 << 30, 1, self.spec,
-                            self.idx, self.n_active)
+                            self.idx, self.n_active, out_pred=outs[w.vidx])
             self.active, self.active_next = self.active_next, self.active
             if events is not None:
                 events[4].record()
         else:
-            c.verify(fresh, t_tgt, tau, self.err, self.accept, self.active)
+            c.verify(fresh, t_tgt, tau, self.err, self.accept, self.active, out_pred=outs[w.vidx])
             if events is not None:
                 events[4].record()
             c.select_adaptive(self.accept, 1 << 30, 1, self.spec, self.active, self.idx, self.n_active)
@@ -359,7 +374,7 @@ def time_draft_models(w: W.Workload, device: str, path: int, reps: int = 10):
     src = W.FeatureSource(w, device)
     feats = [[src.feature(e, k, [w.times[k]] * w.batch) for e in range(ne)] for k in range(2)]
     outs = [torch.empty(w.batch, n, d, dtype=w.torch_dtype, device=dev) for n, d in w.entries]
-    ab = algorithmic_bytes(w, w.max_order)
+    ab = algorithmic_bytes(w, w.max_order, pred_from_verify=False)
     res = {}
     for basis, name in ((S.SPECA_BASIS_TAYLOR, "taylor_eq2_3"), (S.SPECA_BASIS_NEWTON, "newton"),
                         (S.SPECA_BASIS_ADAMS_BASHFORTH, "adams_bashforth")):
@@ -415,23 +430,47 @@ def time_metrics(h: Harness, reps: int = 20):
     return out
 
 
+def _slab_layout(sizes, align=256):
+    """Offsets of consecutive byte ranges, each starting on an `align`-byte boundary; (offsets, total)."""
+    offs, off = [], 0
+    for s in sizes:
+        offs.append(off)
+        off = (off + s + align - 1) // align * align
+    return offs, off
+
+
 def time_end_to_end(h: Harness, steps: int, warmup: int):
     """Same step, but every step's inputs start in pinned host memory and its results end there.
-    The three legs of a step -- host-to-device copy of the features, the library calls, device-to-host
-    copy of forecasts and decisions -- run on three streams with two sets of device buffers, so the
-    copy-in of step k+1 and the copy-out of step k-1 overlap step k (PCIe is full duplex). Time is the
-    host's wall clock from the first enqueue to the moment every result is in host memory."""
+    A step's inputs (every entry's feature and the verification feature) sit in ONE pinned slab and
+    its results (every forecast, err, accept, next mask) in another, so each direction is a single
+    large copy per step. The three legs of a step -- host-to-device copy, the library calls,
+    device-to-host copy -- run on three streams with two sets of device buffers, so the copy-in of
+    step k+1 and the copy-out of step k-1 overlap step k (PCIe is full duplex). Time is the host's
+    wall clock from the first enqueue to the moment every result is in host memory."""
     w, dev = h.w, h.device
-    host_feats = [[f.cpu().pin_memory() for f in fs] for fs in h.feats]
-    host_fresh = [f.cpu().pin_memory() for f in h.fresh]
-    host_outs = [torch.empty(o.shape, dtype=o.dtype).pin_memory() for o in h.outs]
-    host_small = [torch.empty(h.B * 6, dtype=torch.uint8).pin_memory() for _ in range(2)]
-    dev_feats = [[torch.empty_like(f) for f in h.feats[0]] for _ in range(2)]
-    dev_fresh = [torch.empty_like(h.fresh[0]) for _ in range(2)]
-    dev_outs = [h.outs, [torch.empty_like(o) for o in h.outs]]
-    dev_small = [torch.empty(h.B * 6, dtype=torch.uint8, device=dev) for _ in range(2)]
-    h2d = sum(f.numel() * f.element_size() for f in host_feats[0]) + host_fresh[0].numel() * host_fresh[0].element_size()
-    d2h = sum(o.numel() * o.element_size() for o in host_outs) + h.B * (4 + 1 + 1)
+    eb = w.elem_bytes
+    ne = len(w.entries)
+    in_sizes = [h.B * n * d * eb for n, d in w.entries] + [h.B * w.entry_elems(w.vidx) * eb]
+    in_offs, in_total = _slab_layout(in_sizes)
+    out_sizes = [h.B * n * d * eb for n, d in w.entries] + [h.B * 4, h.B, h.B]
+    out_offs, out_total = _slab_layout(out_sizes)
+
+    def views(slab, offs, sizes, shapes):
+        return [slab[o: o + s].view(w.torch_dtype).view(shape) for o, s, shape in zip(offs, sizes, shapes)]
+
+    shapes_in = [(h.B, n, d) for n, d in w.entries] + [(h.B,) + tuple(w.entries[w.vidx])]
+    shapes_out = [(h.B, n, d) for n, d in w.entries]
+    host_in = [torch.empty(in_total, dtype=torch.uint8).pin_memory() for _ in range(2)]
+    for p in range(2):
+        for v, src in zip(views(host_in[p], in_offs, in_sizes, shapes_in), h.feats[p] + [h.fresh[p]]):
+            v.copy_(src)
+    host_out = [torch.empty(out_total, dtype=torch.uint8).pin_memory() for _ in range(2)]
+    dev_in = [torch.empty(in_total, dtype=torch.uint8, device=dev) for _ in range(2)]
+    dev_out = [torch.empty(out_total, dtype=torch.uint8, device=dev) for _ in range(2)]
+    dev_in_views = [views(s, in_offs, in_sizes, shapes_in) for s in dev_in]
+    dev_out_views = [views(s, out_offs[:ne], out_sizes[:ne], shapes_out) for s in dev_out]
+    h2d = sum(in_sizes)
+    d2h = sum(out_sizes)
     main = torch.cuda.current_stream(dev)
     s_in, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
     ev_in, ev_done, ev_out = {}, {}, {}
@@ -441,27 +480,22 @@ def time_end_to_end(h: Harness, steps: int, warmup: int):
         with torch.cuda.stream(s_in):
             if k - 2 in ev_done:
                 s_in.wait_event(ev_done[k - 2])      # the step that last read this buffer set has run
-            for dst, src in zip(dev_feats[p], host_feats[p]):
-                dst.copy_(src, non_blocking=True)
-            dev_fresh[p].copy_(host_fresh[p], non_blocking=True)
+            dev_in[p].copy_(host_in[p], non_blocking=True)          # one copy: the step's whole input
             ev_in[k] = torch.cuda.Event()
             ev_in[k].record(s_in)
         main.wait_event(ev_in[k])
         if k - 2 in ev_out:
             main.wait_event(ev_out[k - 2])           # the previous results in this output set are on the host
-        saved, h.outs = h.outs, dev_outs[p]
-        h.step(feats=dev_feats[p], fresh=dev_fresh[p])
-        h.outs = saved
-        dev_small[p][: 4 * h.B].copy_(h.err.view(torch.uint8))
-        dev_small[p][4 * h.B: 5 * h.B].copy_(h.accept)
-        dev_small[p][5 * h.B:].copy_(h.active)
+        h.step(feats=dev_in_views[p][:ne], fresh=dev_in_views[p][ne], outs=dev_out_views[p])
+        tail = dev_out[p]
+        tail[out_offs[ne]: out_offs[ne] + 4 * h.B].copy_(h.err.view(torch.uint8))
+        tail[out_offs[ne + 1]: out_offs[ne + 1] + h.B].copy_(h.accept)
+        tail[out_offs[ne + 2]: out_offs[ne + 2] + h.B].copy_(h.active)
         ev_done[k] = torch.cuda.Event()
         ev_done[k].record(main)
         with torch.cuda.stream(s_out):
             s_out.wait_event(ev_done[k])
-            for dst, src in zip(host_outs, dev_outs[p]):
-                dst.copy_(src, non_blocking=True)
-            host_small[p].copy_(dev_small[p], non_blocking=True)
+            host_out[p].copy_(dev_out[p], non_blocking=True)        # one copy: the step's whole result
             ev_out[k] = torch.cuda.Event()
             ev_out[k].record(s_out)
         for old in (k - 3,):
@@ -478,7 +512,18 @@ def time_end_to_end(h: Harness, steps: int, warmup: int):
     torch.cuda.synchronize(dev)
     wall = (time.perf_counter() - wall0) * 1e3
     D.barrier()
-    return wall / steps, h2d, d2h
+    # one direction alone, for the PCIe rate each copy reaches when the link is not shared
+    e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    e0.record()
+    dev_in[0].copy_(host_in[0], non_blocking=True)
+    e1.record()
+    host_out[0].copy_(dev_out[0], non_blocking=True)
+    e2.record()
+    torch.cuda.synchronize(dev)
+    alone = {"h2d_gbs_alone": h2d / (e0.elapsed_time(e1) * 1e-3) / 1e9, "d2h_gbs_alone": d2h / (e1.elapsed_time(e2) * 1e-3) / 1e9}
+    del host_in, host_out, dev_in, dev_out
+    torch.cuda.empty_cache()
+    return wall / steps, h2d, d2h, alone
 
 
 def adaptive_sweep(device: str, peak: float, path: int, orders=(1, 2, 3), horizon: int = 6):
@@ -615,39 +660,97 @@ def sampler_run(device: str, path: int, name: str, layout: int = 0):
     return res
 
 
-def oracle_sample_run(w: W.Workload, sample_elems: int, repeats: int, seed: int = 0):
-    """The CPU oracle, as it stands, on a bounded sample of the workload: `sample_elems` elements
-    per sample of the verification entry go through one full step (update at order m, forecast,
-    Eq. 4, accept, select). Returns (seconds per step, algorithmic bytes per step, threads)."""
+# ------------------------------------------------------------------------------------------------
+# the CPU oracle timed on the same configuration (cpu_baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------------
+
+def _host_array(x: torch.Tensor, B: int):
     import numpy as np
+    x = x.detach().contiguous().cpu()
+    if x.dtype == torch.bfloat16:
+        return x.view(torch.int16).numpy().view(np.uint16).reshape(B, -1).copy()
+    return x.numpy().reshape(B, -1).copy()
+
+
+def oracle_entry_steps(w: W.Workload, src: W.FeatureSource, e: int, n_steps: int, t_base: float):
+    """The CPU oracle, as it stands, on ONE entry of the workload with the workload's own seeded
+    features: max_order + 1 warming reference steps (untimed), then `n_steps` whole steps -- update,
+    commit, forecast, and for the verification entry Eq. 4, the accept rule and the selection -- at
+    the reference / target times the GPU harness uses. Returns the seconds each step took."""
     from oracle import speca_oracle as O
     B, m = w.batch, w.max_order
-    n = min(sample_elems, w.entry_elems(w.vidx))
-    g = torch.Generator().manual_seed(W.SEED_BASE + seed)
-
-    def feat():
-        x = torch.randn(B, n, generator=g)
-        if w.dtype == W.BF16:
-            return x.to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16).copy()
-        return x.numpy().copy()
-
-    cache = O.OracleCache([n], B, m, w.dtype)
-    for k in range(m + 1):
-        cache.update([feat()], [1.0 - 0.02 * k] * B)
+    is_v = e == w.vidx
+    cache = O.OracleCache([w.entry_elems(e)], B, m, w.dtype)
+    for step in range(m + 1):
+        t = [w.times[step]] * B
+        cache.update([_host_array(src.feature(e, step, t), B)], t)
         cache.commit_step()
-    fa, fb = feat(), feat()
-    eb = w.elem_bytes
-    bytes_step = ((2 * m + 2) + (m + 2) + (m + 2)) * eb * n * B
-    t0 = time.perf_counter()
-    for r in range(repeats):
-        t_ref = 1.0 - 0.02 * (m + 1 + r)
-        cache.update([fa if r & 1 else fb], [t_ref] * B)
+    step0 = m + 1
+    feats = [_host_array(src.feature(e, step0 + k, [w.times[step0 + k]] * B), B) for k in range(2)]
+    fresh = [_host_array(src.feature(e, step0 + 2 + k, [w.times[step0 + 2 + k]] * B), B) for k in range(2)] if is_v else None
+    out = None
+    secs = []
+    for j in range(n_steps):
+        t_ref = [t_base - 0.02 * (j + 1)] * B
+        t_tgt = [t_ref[0] - 0.01] * B
+        tau = [O.tau_schedule(w.tau0, w.beta, w.total_steps - (j % w.total_steps), w.total_steps)] * B
+        t0 = time.perf_counter()
+        cache.update([feats[j & 1]], t_ref)
         cache.commit_step()
-        cache.forecast_entry(0, [t_ref - 0.01] * B)
-        err, acc, _ = cache.verify(fb if r & 1 else fa, [t_ref - 0.01] * B, [0.1] * B)
-        O.select_adaptive([max(int(a), 0) for a in acc], 1 << 30, 1, [0] * B, [1] * B)
-    dt = (time.perf_counter() - t0) / repeats
-    return dt, bytes_step, O.threads(), n
+        if is_v:
+            _, acc, _ = cache.verify(fresh[j & 1], t_tgt, tau)      # the entry's forecast is part of this
+            O.select_adaptive([max(int(a), 0) for a in acc], 1 << 30, 1, [0] * B, [1] * B)
+        else:
+            out = cache.forecast_entry(0, t_tgt, out=out)
+        secs.append(time.perf_counter() - t0)
+    return secs
+
+
+def oracle_config_run(w: W.Workload, n_steps: int, budget_s: float, gen_device: str):
+    """Times the oracle over the whole configuration, entry by entry (the entries are independent, so a
+    step's time is the sum of its entries' times; only one entry's tables are in host memory at a
+    time). If the whole configuration would not fit `budget_s` seconds of oracle work, every k-th entry
+    (always with the verification entry) is the step's sample instead, and the result says so.
+    Returns a dict with the per-step seconds, the algorithmic bytes those steps covered, the threads
+    the oracle used and a description of the sample."""
+    from oracle import speca_oracle as O
+    src = W.FeatureSource(w, gen_device)
+    ne = len(w.entries)
+    t_base = w.times[w.max_order]
+    per_elem = lambda e: ((2 * w.max_order + 2) + (w.max_order + (3 if e == w.vidx else 2))) * w.elem_bytes  # noqa: E731
+    # calibrate on the smallest entry: seconds per element of one step
+    e_small = min(range(ne), key=lambda e: w.entry_elems(e))
+    cal = oracle_entry_steps(w, src, e_small, 2, t_base)
+    rate = min(cal) / (w.batch * w.entry_elems(e_small))
+    est = rate * w.elems_per_order * n_steps
+    stride = 1 if est <= budget_s else int(-(-est // budget_s))
+    chosen = sorted(set(list(range(0, ne, stride)) + [w.vidx]))
+    secs = [0.0] * n_steps
+    nbytes = 0
+    for e in chosen:
+        for j, s in enumerate(oracle_entry_steps(w, src, e, n_steps, t_base)):
+            secs[j] += s
+        nbytes += per_elem(e) * w.batch * w.entry_elems(e)
+    if len(chosen) == ne:
+        sample = "all %d entries of %s, every step: update+forecast+verify+select on the workload's seeded features" % (ne, w.name)
+    else:
+        sample = "%d of %d entries of %s (every %d-th and the verification entry), every step: update+forecast+verify+select" % (
+            len(chosen), ne, w.name, stride)
+    return {"secs": secs, "bytes_per_step": nbytes, "threads": O.threads(), "sample": sample, "entries": len(chosen)}
+
+
+def oracle_one_thread_gbs(w: W.Workload, gen_device: str):
+    """One step of the verification entry alone with the oracle held to one thread: GB/s."""
+    from oracle import speca_oracle as O
+    n = O.threads()
+    O.set_threads(1)
+    try:
+        src = W.FeatureSource(w, gen_device)
+        secs = oracle_entry_steps(w, src, w.vidx, 1, w.times[w.max_order])
+    finally:
+        O.set_threads(n)
+    nbytes = ((2 * w.max_order + 2) + (w.max_order + 3)) * w.elem_bytes * w.batch * w.entry_elems(w.vidx)
+    return nbytes / secs[0] / 1e9
 
 
 def parity_on_verify_entry(w: W.Workload, device: str, path: int):
@@ -666,12 +769,6 @@ def parity_on_verify_entry(w: W.Workload, device: str, path: int):
     gpu = S.SpecaCache(one.entries, B, m, w.dtype, device, path=path)
     cpu = O.OracleCache([n_tok * dim], B, m, w.dtype)
 
-    def host(x):
-        x = x.detach().contiguous().cpu()
-        if x.dtype == torch.bfloat16:
-            return x.view(torch.int16).numpy().view(np.uint16).reshape(B, -1).copy()
-        return x.numpy().reshape(B, -1).copy()
-
     def f64(a):
         return (a.astype(np.uint32) << 16).view(np.float32).astype(np.float64) if a.dtype == np.uint16 else a.astype(np.float64)
 
@@ -680,7 +777,7 @@ def parity_on_verify_entry(w: W.Workload, device: str, path: int):
         f = src.feature(0, step, t)
         gpu.update([f], t)
         gpu.commit_step()
-        cpu.update([host(f)], t)
+        cpu.update([_host_array(f, B)], t)
         cpu.commit_step()
     step = m + 1
     t = [w.times[step]] * B
@@ -691,8 +788,8 @@ def parity_on_verify_entry(w: W.Workload, device: str, path: int):
     acc = torch.zeros(B, dtype=torch.uint8, device=device)
     gpu.verify(fresh, t, tau, err, acc, out_pred=pred)
     torch.cuda.synchronize()
-    e_want, a_want, p_want = cpu.verify(host(fresh), t, tau)
-    g, o = f64(host(pred)), f64(p_want)
+    e_want, a_want, p_want = cpu.verify(_host_array(fresh, B), t, tau)
+    g, o = f64(_host_array(pred, B)), f64(p_want)
     rel = [float(np.linalg.norm(g[b] - o[b]) / max(np.linalg.norm(o[b]), 1e-30)) for b in range(B)]
     e_got = [float(x) for x in err.cpu().tolist()]
     out = {"entry_elems": n_tok * dim, "samples": B,
@@ -704,40 +801,45 @@ def parity_on_verify_entry(w: W.Workload, device: str, path: int):
     return out
 
 
+def generation_device() -> str:
+    """Where the seeded features are drawn: the GPU when there is one (the same bits the library's
+    arm sees), else the host."""
+    return "cuda:0" if torch.cuda.is_available() else "cpu"
+
+
 def run_reference(args, info: D.RankInfo):
-    """The oracle timed on the host cores for the same metric (bounded sample per step)."""
+    """--impl reference: the oracle timed on the host cores for the same metric, configuration and
+    step (rank 0 alone; the other ranks leave at once)."""
     if not info.is_main:
         return
     w = make_workload(args.config)
-    sample = 1 << 20
-    for _ in range(max(0, args.warmup)):
-        oracle_sample_run(w, sample, 1)
-    dt, bytes_step, threads, n = oracle_sample_run(w, sample, max(1, args.steps))
-    gbs = bytes_step / dt / 1e9
-    sample_desc = "update+forecast+verify+select over %d elements x %d samples of the verification entry per step" % (
-        n, w.batch)
+    steps, warm = max(1, args.steps), max(0, args.warmup)
+    res = oracle_config_run(w, steps + warm, args.oracle_budget_s, generation_device())
+    timed = res["secs"][warm:]
+    dt = sum(timed) / len(timed)
+    gbs = res["bytes_per_step"] / dt / 1e9
     line = {
-        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "impl": "reference", "metric": METRIC, "value": _r(gbs, 4), "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": steps, "warmup": warm, "ms_per_step": _r(dt * 1e3, 3), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(w),
-        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample_desc},
-        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "value_covers": VALUE_COVERS, "config": workload_config(w),
+        "cpu_baseline": {"value": _r(gbs, 4), "unit": "GB/s", "cores": res["threads"], "kind": "oracle",
+                         "sample": res["sample"]},
+        "e2e": {"value": _r(gbs, 4), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
-    print(json.dumps(line))
+    print(json.dumps(line, separators=(",", ":")), flush=True)
 
 
-def workload_config(w: W.Workload):
+def workload_config(w: W.Workload, layout: str = "tables"):
     return {
-        "workload": "%s (benchmark config %d)" % (w.name, w.index),
-        "entries": len(w.entries), "batch": w.batch, "taylor_order": w.max_order,
-        "storage": "bf16" if w.dtype == W.BF16 else "f32",
+        "workload": "%s (config %d)" % (w.name, w.index),
+        "entries": len(w.entries), "batch": w.batch, "order": w.max_order,
+        "storage": "bf16" if w.dtype == W.BF16 else "f32", "layout": layout,
         "elems_per_order": w.elems_per_order,
-        "cache_bytes": w.elems_per_order * (w.max_order + 1) * w.elem_bytes,
-        "l2": "no flush: every step streams a working set far larger than the 126 MB L2",
-        "step": "update(all entries) + forecast(all entries) + verify(last entry) + select",
-        "parallelism": "one independent cache per GPU (sample-sharded, no collective on the data path)",
+        "l2": ("no flush: working set >> 126 MB L2" if w.elems_per_order * w.elem_bytes * (w.max_order + 1) > (1 << 30)
+               else "no flush: small case, fits L2 (parity configuration, not an HBM figure)"),
+        "parallelism": "one cache per GPU, no collective",
     }
 
 
@@ -775,7 +877,115 @@ def time_history_layout(w, device, path, steps, info, peak, tables_ms_step, tabl
             "note": "update moves 2 words per element instead of 2 * order + 2; forecast and verify move the same bytes"}
 
 
-def main():
+# ------------------------------------------------------------------------------------------------
+# the one line
+# ------------------------------------------------------------------------------------------------
+
+def _r(x, digits=5):
+    """A float to `digits` significant digits (keeps the line short); other values unchanged."""
+    if isinstance(x, float):
+        if x != x or x in (float("inf"), float("-inf")):
+            return None
+        return float("%.*g" % (digits, x))
+    return x
+
+
+def build_line(*, value, ms_per_step, n_gpus, steps, warmup, config, roofline, cpu_baseline, e2e, gpu_launches, clocks,
+               kernels, forecast_verify_gbs, speculative_steps_per_s, also=None, detail_path=None, scaling="weak"):
+    """The compact JSON object of the benchmark's last line. Raises if it would not stay under
+    MAX_LINE_BYTES: whatever does not fit belongs in the detail file."""
+    line = {
+        "metric": METRIC, "value": _r(value), "unit": "GB/s", "n_gpus": n_gpus, "steps": steps, "warmup": warmup,
+        "ms_per_step": _r(ms_per_step), "higher_is_better": True, "scaling": scaling, "vs_baseline": None,
+        "dtype": "f32",  # the arithmetic type: every kernel computes in fp32 registers, whatever config.storage is
+        "data": "synthetic", "value_covers": VALUE_COVERS, "config": config,
+        "roofline": {k: _r(v) for k, v in roofline.items()} if roofline else None,
+        "cpu_baseline": {k: _r(v, 4) for k, v in cpu_baseline.items()} if cpu_baseline else None,
+        "e2e": {k: _r(v, 4) for k, v in e2e.items()} if e2e else None,
+        "gpu_launches": gpu_launches, "clocks": clocks,
+        "forecast_verify_gbs": _r(forecast_verify_gbs), "speculative_steps_per_s": _r(speculative_steps_per_s),
+        "kernels_ms_gbs": {k: [_r(v["ms"], 4), _r(v["gbs"], 4)] for k, v in kernels.items() if k != "select"},
+    }
+    if also:
+        line["also_value_fv_gbs_steps_per_s"] = {k: [_r(x, 4) for x in v] for k, v in also.items()}
+    if detail_path:
+        line["detail"] = detail_path
+    text = json.dumps(line, separators=(",", ":"))
+    if len(text) >= MAX_LINE_BYTES:
+        raise ValueError("benchmark line is %d bytes; the limit is %d" % (len(text), MAX_LINE_BYTES))
+    return text
+
+
+def write_detail(path, detail):
+    """Best effort: the detail file is a by-product, the line is the result."""
+    if not path:
+        return None
+    try:
+        d = os.path.dirname(os.path.abspath(path))
+        os.makedirs(d, exist_ok=True)
+        with open(path, "w") as f:
+            json.dump(detail, f, indent=1)
+        return path
+    except Exception:
+        return None
+
+
+# ------------------------------------------------------------------------------------------------
+# one process per GPU
+# ------------------------------------------------------------------------------------------------
+
+def free_port() -> int:
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def spawn_ranks(n: int, argv, extra_env=None, timeout_s: float = 3600.0) -> int:
+    """Starts `n` copies of `argv` (a full command line), one per rank, with the process-group
+    environment torchrun would give them (RANK, LOCAL_RANK, WORLD_SIZE, MASTER_ADDR, MASTER_PORT),
+    and waits for all of them. Rank 0 inherits stdout, so its one line is the job's line; the other
+    ranks' stdout is dropped. If a rank fails the others are stopped (by their own PIDs). Returns
+    the largest exit status."""
+    port = free_port()
+    procs = []
+    for r in range(n):
+        env = dict(os.environ)
+        env.update(RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        env.update(extra_env or {})
+        procs.append(subprocess.Popen(list(argv), env=env, stdout=None if r == 0 else subprocess.DEVNULL))
+    deadline = time.time() + timeout_s
+    rc = 0
+    live = list(procs)
+    while live:
+        for p in list(live):
+            code = p.poll()
+            if code is None:
+                continue
+            live.remove(p)
+            if code != 0:
+                rc = max(rc, abs(code) or 1)
+        if (rc != 0 or time.time() > deadline) and live:
+            for p in live:
+                p.terminate()
+            for p in live:
+                try:
+                    p.wait(timeout=10)
+                except subprocess.TimeoutExpired:
+                    p.kill()
+            rc = rc or 124
+            break
+        time.sleep(0.05)
+    return rc
+
+
+def job_value(step_bytes_per_rank: float, world: int, slowest_ms_per_step: float) -> float:
+    """Whole-job GB/s: every rank moves its own step's bytes; the job is as fast as its slowest rank."""
+    return world * step_bytes_per_rank / (slowest_ms_per_step * 1e-3) / 1e9
+
+
+def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
@@ -783,7 +993,7 @@ def main():
     ap.add_argument("--config", default="flux", choices=["tiny", "dit_xl2", "flux", "hunyuan_video", "flux_b8"])
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--also", default="dit_xl2,hunyuan_video",
-                    help="comma list of further configs measured device-resident and reported under per_config")
+                    help="comma list of further configs measured device-resident (three numbers each in the line)")
     ap.add_argument("--path", default="auto", choices=["auto", "direct", "bulk", "wide"],
                     help="kernel variant (speca_path_t); results are identical, only speed differs")
     ap.add_argument("--layout", default="tables", choices=["tables", "history"],
@@ -791,18 +1001,31 @@ def main():
                          "the last references (speca_layout_t)")
     ap.add_argument("--separate-select", action="store_true",
                     help="five launches per step (update, activate, forecast, verify, select) instead of the three fused ones")
+    ap.add_argument("--detail", default=os.path.join("gpurun_out", "bench_detail.json"),
+                    help="JSON file for everything that does not belong in the last line ('' = none)")
+    ap.add_argument("--full", action="store_true",
+                    help="also run the sweeps reported only in the detail file: multi-horizon and summed forecasts, "
+                         "other metrics and draft models, the raw-feature layout, the B=8 adaptive sweep, the sampler loop")
+    ap.add_argument("--oracle-budget-s", type=float, default=150.0,
+                    help="--impl reference: seconds of oracle work the run may take; above it a step samples every k-th entry")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--no-adaptive", action="store_true",
-                    help="skip the B=8 sample-adaptive sweep (orders 1-3, horizon 1-6) reported under 'adaptive'")
+    ap.add_argument("--no-adaptive", action="store_true", help="accepted for older command lines; the sweep needs --full")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    args = ap.parse_args()
+    args = ap.parse_args(argv)
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
 
-    info = D.rank_info_from_env()
     if args.impl == "reference":
-        run_reference(args, info)
-        return
+        run_reference(args, D.rank_info_from_env())
+        return 0
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # no launcher gave us a process group: start one rank per GPU ourselves
+        if not torch.cuda.is_available() or torch.cuda.device_count() < args.gpus:
+            raise SystemExit("bench.py --gpus %d: only %d CUDA devices visible" % (
+                args.gpus, torch.cuda.device_count() if torch.cuda.is_available() else 0))
+        return spawn_ranks(args.gpus, [sys.executable, os.path.abspath(__file__)] + list(sys.argv[1:] if argv is None else argv))
+
+    info = D.rank_info_from_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     from paper_2509_11628_b200 import build as _b
@@ -813,6 +1036,7 @@ def main():
     info = D.init("nccl")
     D.barrier()
     peak, peak_src = measured_peak()
+    solo = info.world == 1
 
     w = make_workload(args.config)
     path = {"auto": 0, "direct": 1, "bulk": 2, "wide": 3}[args.path]
@@ -821,44 +1045,52 @@ def main():
     total_ms, per_ms, launches, clocks = time_device_resident(h, args.steps, args.warmup, info, True)
     total_ms = D.max_over_ranks(total_ms, device)
     value, ms_step, kernels, extra = summarize(w, per_ms, total_ms, args.steps, info.world, peak, layout=layout)
+    detail = {"config": workload_config(w, args.layout), "kernels": kernels, **extra,
+              "frac_of_measured_peak": value / info.world / peak, "frac_of_nominal_8TBs": value / info.world / NOMINAL_HBM_GBS,
+              "select": "its own launches (speca_select_adaptive, speca_activate)" if args.separate_select else
+                        "inside the verify launch (speca_verify_select); re-arming inside the update launch",
+              "paper_context": {"end_to_end_speedups": {"flux_h800": 6.34, "dit_xl2_a800": 7.3, "hunyuan_video_h800": 6.1},
+                                "verification_overhead": "1.67%-3.5% of a full forward pass",
+                                "note": "other hardware, whole-model numbers; context only"}}
 
-    tables = info.world == 1 and layout == 0      # these calls exist for the table layout only
-    multi = time_multi_horizon(h, peak, per_ms["forecast"]) if tables else None
-    metrics = time_metrics(h) if info.world == 1 else None
-    per_entry = time_update_per_entry(h) if tables else None
-    fsum = time_forecast_sum(h, peak) if tables else None
+    tables = solo and layout == 0      # these calls exist for the table layout only
+    if args.full and solo:
+        detail["verify_metrics"] = time_metrics(h)
+    if args.full and tables:
+        detail["multi_horizon"] = time_multi_horizon(h, peak, per_ms["forecast"])
+        detail["update_one_launch_per_entry"] = time_update_per_entry(h)
+        detail["forecast_sum"] = time_forecast_sum(h, peak)
 
     e2e = None
     if not args.no_e2e:
         e2e_steps = max(3, min(args.steps, 24))
-        e2e_ms, h2d, d2h = time_end_to_end(h, e2e_steps, 3)
+        e2e_ms, h2d, d2h, alone = time_end_to_end(h, e2e_steps, 3)
         e2e_ms = D.max_over_ranks(e2e_ms, device)
         ab = algorithmic_bytes(w, w.max_order, layout)
-        e2e = {"value": info.world * (ab["update"] + ab["forecast"] + ab["verify"]) / (e2e_ms * 1e-3) / 1e9,
+        e2e = {"value": job_value(ab["update"] + ab["forecast"] + ab["verify"], info.world, e2e_ms),
                "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
-               "steps": e2e_steps,
-               "note": "features and verification feature copied from pinned host memory, forecasts and decisions copied back, "
-                       "every step; copy-in, library calls and copy-out pipelined on three streams; host wall clock"}
+               "h2d_gbs": h2d / (e2e_ms * 1e-3) / 1e9, "d2h_gbs": d2h / (e2e_ms * 1e-3) / 1e9}
+        detail["e2e"] = dict(e2e, steps=e2e_steps, **alone,
+                             note="one pinned slab per direction per step (features + verification feature in, forecasts + "
+                                  "decisions out), one copy each; copy-in, library calls and copy-out pipelined on three "
+                                  "streams; host wall clock; *_gbs = bytes / step time with both directions busy")
     h.close()
     del h
     torch.cuda.empty_cache()
 
-    drafts = None
-    if info.world == 1 and layout == 0:
+    if args.full and tables:
         try:
-            drafts = time_draft_models(w, device, path)
+            detail["draft_models"] = time_draft_models(w, device, path)
         except Exception as exc:  # report, do not hide
-            drafts = {"error": repr(exc)}
+            detail["draft_models"] = {"error": repr(exc)}
+        if path in (0, 3):
+            try:
+                detail["history_layout"] = time_history_layout(w, device, path, min(args.steps, 100), info, peak, ms_step, kernels)
+            except Exception as exc:  # report, do not hide
+                detail["history_layout"] = {"error": repr(exc)}
 
-    history = None
-    if info.world == 1 and path in (0, 3) and layout == 0:
-        try:
-            history = time_history_layout(w, device, path, min(args.steps, 100), info, peak, ms_step, kernels)
-        except Exception as exc:  # report, do not hide
-            history = {"error": repr(exc)}
-
-    per_config = {}
-    if info.world == 1 and layout == 0:
+    also, per_config = {}, {}
+    if tables:
         for name in [n for n in args.also.split(",") if n and n != args.config]:
             try:
                 w2 = make_workload(name)
@@ -867,96 +1099,78 @@ def main():
                 t2, p2, _, _ = time_device_resident(h2, k2, 3, info, False)
                 v2, ms2, kern2, ex2 = summarize(w2, p2, t2, k2, 1, peak)
                 per_config[name] = {"value": v2, "unit": "GB/s", "ms_per_step": ms2, "steps": k2,
-                                    "config": workload_config(w2), "kernels": kern2, **ex2,
-                                    "multi_horizon": time_multi_horizon(h2, peak, p2["forecast"]),
-                                    "update_one_launch_per_entry": time_update_per_entry(h2),
-                                    "forecast_sum": time_forecast_sum(h2, peak)}
+                                    "config": workload_config(w2), "kernels": kern2, **ex2}
+                also[name] = [v2, ex2["forecast_verify_gbs"], ex2["speculative_steps_per_s"]]
+                if args.full:
+                    per_config[name].update(multi_horizon=time_multi_horizon(h2, peak, p2["forecast"]),
+                                            update_one_launch_per_entry=time_update_per_entry(h2),
+                                            forecast_sum=time_forecast_sum(h2, peak))
                 h2.close()
                 del h2
                 torch.cuda.empty_cache()
-                if path in (0, 3):
+                if args.full and path in (0, 3):
                     per_config[name]["history_layout"] = time_history_layout(w2, device, path, k2, info, peak, ms2, kern2)
             except Exception as exc:  # report, do not hide
                 per_config[name] = {"error": repr(exc)}
+    detail["per_config"] = per_config
 
-    adaptive = None
-    if info.world == 1 and not args.no_adaptive:
+    if args.full and solo and not args.no_adaptive:
         try:
-            adaptive = adaptive_sweep(device, peak, path)
+            detail["adaptive"] = adaptive_sweep(device, peak, path)
         except Exception as exc:  # report, do not hide
-            adaptive = {"error": repr(exc)}
-
-    sampler = None
-    if info.world == 1 and not args.no_adaptive:
-        sampler = {}
+            detail["adaptive"] = {"error": repr(exc)}
+        detail["sampler"] = {}
         for name in ("dit_xl2", "flux_adaptive"):
             try:
-                sampler[name] = sampler_run(device, path, name)
+                detail["sampler"][name] = sampler_run(device, path, name)
                 if path in (0, 3):   # the same run on a cache that keeps raw features: cache-path time only
                     hist = sampler_run(device, path, name, layout=1)
-                    sampler[name]["history_layout"] = {k: hist[k] for k in (
+                    detail["sampler"][name]["history_layout"] = {k: hist[k] for k in (
                         "acceptance_rate", "library_ms_total", "ms_mean", "sampler_steps_per_s_library_only")}
             except Exception as exc:  # report, do not hide
-                sampler[name] = {"error": repr(exc)}
+                detail["sampler"][name] = {"error": repr(exc)}
 
     if not info.is_main:
         D.shutdown()
-        return
+        return 0
 
     dominant = max(("update", "forecast", "verify"), key=lambda k: per_ms[k])
     dom = kernels[dominant]
-    per_elem = NCU_DRAM_BYTES_PER_ELEM.get(dominant)
-    if layout == 1 and dominant == "update":
-        per_elem = NCU_DRAM_BYTES_PER_ELEM_HISTORY_UPDATE
+    per_elem = None if (layout == 1 and dominant == "update") else NCU_DRAM_BYTES_PER_ELEM.get(dominant)
     n_dom = w.batch * w.entry_elems(w.vidx) if dominant == "verify" else w.elems_per_order
+    if dominant == "forecast":
+        n_dom -= w.batch * w.entry_elems(w.vidx)
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": dom["gbs"], "peak": peak, "unit": "GB/s",
                 "frac": dom["gbs"] / peak, "peak_source": peak_src,
                 "traffic": (per_elem * n_dom) if per_elem is not None else None,
+                "traffic_source": TRAFFIC_SOURCE if per_elem is not None else "none: kernel changed since the last capture",
                 "algorithmic_bytes_per_launch": dom["algorithmic_bytes"],
                 "frac_of_nominal_8TBs": dom["gbs"] / NOMINAL_HBM_GBS}
 
     cpu_baseline = None
     if not args.no_cpu_baseline:
-        n_s = w.entry_elems(w.vidx)
-        dt1, _, _, _ = oracle_sample_run(w, n_s, 1)          # size the run: about 10 s of oracle work
-        reps = max(1, min(50, int(10.0 / max(dt1, 1e-3))))
-        dt, bytes_step, threads, n = oracle_sample_run(w, n_s, reps)
-        cpu_baseline = {"value": bytes_step / dt / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
-                        "sample": "%d steps of update+forecast+verify+select over the verification entry only "
-                                  "(%d elements x %d samples), not all %d entries" % (reps, n, w.batch, len(w.entries)),
-                        "s_per_step": dt}
-        from oracle import speca_oracle as _O
-        n_threads = _O.threads()
-        _O.set_threads(1)
-        dt_one, _, _, _ = oracle_sample_run(w, n_s, 1)
-        _O.set_threads(n_threads)
-        cpu_baseline["value_1_thread"] = bytes_step / dt_one / 1e9
+        res = oracle_config_run(w, 1, 60.0, device)
+        dt = res["secs"][0]
+        cpu_baseline = {"value": res["bytes_per_step"] / dt / 1e9, "unit": "GB/s", "cores": res["threads"], "kind": "oracle",
+                        "sample": "1 step, " + res["sample"].replace(", every step", ""), "s_per_step": dt,
+                        "value_1_thread_verify_entry_only": oracle_one_thread_gbs(w, device)}
         try:
-            cpu_baseline["parity"] = parity_on_verify_entry(w, device, path)
+            detail["parity_on_verify_entry"] = parity_on_verify_entry(w, device, path)
         except Exception as exc:  # report, do not hide
-            cpu_baseline["parity"] = {"error": repr(exc)}
+            detail["parity_on_verify_entry"] = {"error": repr(exc)}
+        detail["cpu_baseline"] = cpu_baseline
 
-    line = {
-        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": info.world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": dict(workload_config(w), layout=args.layout, select="its own launch (speca_select_adaptive); re-arming its own launch (speca_activate)"
-                       if args.separate_select else
-                       "inside the verify launch (speca_verify_select); re-arming inside the update launch "
-                       "(speca_cache_update_activate)"),
-        "metric_note": "value = algorithmic bytes of the whole step (update + forecast + verify/select) / step time; "
-                       "forecast + verify alone (one speculative step) is forecast_verify_gbs, the update alone kernels.update.gbs",
-        "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches,
-        "clocks": clocks, "kernels": kernels, **extra,
-        "frac_of_measured_peak": value / info.world / peak, "frac_of_nominal_8TBs": value / info.world / NOMINAL_HBM_GBS,
-        "multi_horizon": multi, "verify_metrics": metrics, "update_one_launch_per_entry": per_entry, "forecast_sum": fsum, "draft_models": drafts, "history_layout": history, "per_config": per_config, "adaptive": adaptive, "sampler": sampler,
-        "paper_context": {"end_to_end_speedups": {"flux_h800": 6.34, "dit_xl2_a800": 7.3, "hunyuan_video_h800": 6.1},
-                          "verification_overhead": "1.67%-3.5% of a full forward pass",
-                          "note": "other hardware, whole-model numbers; context only"},
-    }
-    print(json.dumps(line))
+    detail_path = write_detail(args.detail, dict(detail, roofline=roofline, clocks=clocks, value=value, ms_per_step=ms_step,
+                                                 gpu_launches=launches, n_gpus=info.world, steps=args.steps, warmup=args.warmup))
+    clocks_line = {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")} if clocks else None
+    print(build_line(value=value, ms_per_step=ms_step, n_gpus=info.world, steps=args.steps, warmup=args.warmup,
+                     config=workload_config(w, args.layout), roofline=roofline, cpu_baseline=cpu_baseline, e2e=e2e,
+                     gpu_launches=launches, clocks=clocks_line, kernels=kernels,
+                     forecast_verify_gbs=extra["forecast_verify_gbs"],
+                     speculative_steps_per_s=extra["speculative_steps_per_s"], also=also, detail_path=detail_path), flush=True)
     D.shutdown()
+    return 0
 
 
 if __name__ == "__main__":
-    main()
+    sys.exit(main())
