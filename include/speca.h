@@ -30,6 +30,10 @@
  *     Times, thresholds and host masks are folded into the kernel arguments at capture; a replay
  *     reads the device buffers (features, masks, counters) as they are then. The host-side history
  *     (update / commit_step / reset) advances at capture time only, not on replay.
+ *   - A CUDA error that an earlier call on the thread left behind is reported once (SPECA_ERR_CUDA,
+ *     "earlier CUDA error") by the next call that enqueues work, and cleared: a recoverable error
+ *     (a rejected launch configuration, say) does not poison later calls, while an error that broke
+ *     the context keeps coming back from the runtime itself.
  *   - A handle is not thread safe: use one handle from one host thread at a time.
  *   - There is no CPU fallback: without a usable CUDA device speca_cache_create fails.
  */
@@ -102,6 +106,14 @@ typedef enum {
  *          out = sum_i w_i * plane_i. Same Eq. 2-3 (and the same Newton / Adams-Bashforth readings), any
  *          gaps; the results differ from TABLES only in that no intermediate quotient is rounded to the
  *          storage type. Served by the default kernel path only (SPECA_PATH_AUTO / SPECA_PATH_WIDE).
+ *          Accuracy: every forecast element is a correct rounding to the storage type of Eq. 2-3 evaluated
+ *          in fp32 (within 4e-6 of the summed magnitudes of its terms). Because the forecast is rounded
+ *          once from a combination of stored values, on a UNIFORM time grid with bf16 storage (weights are
+ *          then ratios of small integers) a few per cent of the elements land exactly on a rounding tie,
+ *          where an fp64 evaluation may pick the other neighbour; both are correct. The verification error
+ *          computed on the library's forecast meets the 1e-4 bound; against an fp64 evaluation of the
+ *          whole chain it can differ by up to 6e-3 of itself on such grids (measured: 1e-3 to 4e-3), and
+ *          by no more than the TABLES layout does on uneven grids.
  */
 typedef enum {
     SPECA_LAYOUT_TABLES = 0,
@@ -358,7 +370,7 @@ speca_status_t speca_activate(speca_cache_t* cache, const uint8_t* host_sample_m
  * whose framework pool took all of HBM at start-up, a plug-in that is only handed input and output
  * tensors, a host thread that must not call cudaMalloc because that call synchronises the whole
  * device. speca_verify keeps its reduction scratch in the caller's arena; this variant keeps it in
- * a fixed array inside the library image instead, SPECA_STATIC_SCRATCH_BYTES (about 66 KB) that
+ * a fixed array inside the library image instead, SPECA_STATIC_SCRATCH_BYTES (about 65 KB) that
  * every GPU which loads the library holds until the process exits. The call path contains no
  * cudaMalloc, cudaFree or other allocating routine.
  *
@@ -373,19 +385,21 @@ speca_status_t speca_activate(speca_cache_t* cache, const uint8_t* host_sample_m
  *   dev_err         device, batch floats.  dev_accept: device, batch bytes (1 = accept).
  *   device          CUDA device ordinal that owns all the buffers; stream as everywhere else.
  *
- * The first call on a device looks up the scratch array's device address
- * (cudaGetSymbolAddress, with that device current) and remembers it; make that first call before
- * any stream capture begins. Every call on a device shares the one array, which keeps whatever the
+ * The first call on a device (and per storage type) looks up the scratch array's device address
+ * (cudaGetSymbolAddress, with that device current) and the number of thread-block clusters the
+ * device can hold, and remembers both; make that first call before any stream capture begins.
+ * Later calls do no driver queries. Every call on a device shares the one array, which keeps whatever the
  * previous call left: each call re-initialises what it needs on the stream before the reduction
  * runs, so calls in stream order are independent, but two calls whose kernels overlap on the GPU
  * (different streams, no dependency between them) race on the scratch and give wrong results.
  * Errors: INVALID_ARG (null, dtype, NaN tau, bad device), SHAPE (batch or n_elems beyond the
- * maxima above), ALIGNMENT, UNSUPPORTED (not an sm_100 device), CUDA. On error nothing is enqueued.
+ * maxima above), ALIGNMENT, UNSUPPORTED (not an sm_100 device), CUDA. On error nothing that writes
+ * dev_err or dev_accept is enqueued (the scratch's counters may already have been cleared on the stream).
  */
 #define SPECA_STATIC_MAX_BATCH 64
 #define SPECA_STATIC_MAX_ELEMS 2147483647LL
 #define SPECA_STATIC_MAX_CLUSTERS 128
-#define SPECA_STATIC_SCRATCH_BYTES (32 * 64 + 8 * 64 * SPECA_STATIC_MAX_CLUSTERS + 256)
+#define SPECA_STATIC_SCRATCH_BYTES (8 * 64 * SPECA_STATIC_MAX_CLUSTERS + 512)
 speca_status_t speca_verify_pred_static(const void* pred, const void* fresh, int64_t n_elems, int32_t batch,
                                         int32_t dtype, const float* tau, float eps, const uint8_t* dev_active_mask,
                                         float* dev_err, uint8_t* dev_accept, int32_t device, void* stream);
@@ -466,6 +480,16 @@ typedef struct {
     uint64_t resets[SPECA_MAX_BATCH];
 } speca_cache_stats_t;
 speca_status_t speca_cache_stats(const speca_cache_t* cache, speca_cache_stats_t* out);
+
+/*
+ * Health check of the work a handle has enqueued on `stream`: waits for that stream (the one call
+ * besides destroy that synchronises), then reads the cache's gave-up word. The SPECA_PATH_BULK kernels
+ * wait for their staged copies with a bounded wait; if one ever gives up, the kernel sets that word
+ * and finishes without the tile, so results since the previous check are incomplete. Returns
+ * SPECA_ERR_CUDA in that case (and clears the word), or if the stream reports an error; SPECA_OK
+ * otherwise. The other kernel paths never set the word. Errors: INVALID_ARG (null handle), CUDA.
+ */
+speca_status_t speca_cache_check(speca_cache_t* cache, void* stream);
 
 /* How many kernels the handle has launched since it was created. */
 speca_status_t speca_cache_launch_count(const speca_cache_t* cache, uint64_t* out);

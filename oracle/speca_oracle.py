@@ -141,6 +141,21 @@ def forecast_history_segment(dtype, m, basis, t_hist, t_target, hist: Sequence[n
         raise RuntimeError("forecast from an empty history, or a repeated reference time")
 
 
+def forecast_history_unrounded(dtype, m, basis, t_hist, t_target, hist: Sequence[np.ndarray]) -> np.ndarray:
+    """The same forecast before it is rounded to the storage type, as float64 (tests use it to tell which
+    elements sit so close to a rounding tie of the storage type that either neighbour is a correct result)."""
+    k = len(hist)
+    assert 1 <= k <= m + 1 and len(t_hist) >= k
+    n = hist[0].size
+    assert all(h.flags.c_contiguous and h.dtype == np_dtype(dtype) and h.size == n for h in hist)
+    acc = np.zeros(n, dtype=np.float64)
+    ptrs = (ctypes.c_void_p * k)(*[h.ctypes.data for h in hist])
+    rc = lib().oracle_forecast_history_accumulate_segment(dtype, n, m, basis, k, _hist(t_hist, m), float(t_target), ptrs, _ptr(acc))
+    if rc != 0:
+        raise RuntimeError("forecast from an empty history, or a repeated reference time")
+    return acc
+
+
 def rel_l2(dtype, pred: np.ndarray, fresh: np.ndarray, eps: float = EPS_PAPER) -> float:
     """Eq. 4 over one sample."""
     assert pred.flags.c_contiguous and fresh.flags.c_contiguous and pred.size == fresh.size

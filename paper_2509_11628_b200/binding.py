@@ -31,7 +31,7 @@ EXPORTS = [
     "speca_cache_arena_bytes", "speca_cache_create", "speca_cache_destroy", "speca_cache_reset",
     "speca_cache_update", "speca_cache_update_activate", "speca_cache_commit_step", "speca_forecast", "speca_verify",
     "speca_select_adaptive", "speca_activate", "speca_tau", "speca_cache_state", "speca_cache_plane",
-    "speca_cache_launch_count", "speca_cache_stats", "speca_cache_next_slot", "speca_forecast_weights", "speca_status_string", "speca_last_error", "speca_version",
+    "speca_cache_launch_count", "speca_cache_stats", "speca_cache_check", "speca_cache_next_slot", "speca_forecast_weights", "speca_status_string", "speca_last_error", "speca_version",
     "speca_verify_pred_static", "speca_forecast_multi", "speca_verify_metric",
     "speca_verify_partial", "speca_verify_decide", "speca_cache_get_history", "speca_cache_set_history",
     "speca_forecast_sum", "speca_verify_select",
@@ -106,6 +106,7 @@ def _lib() -> ctypes.CDLL:
     L.speca_cache_plane.argtypes = [vp, i32, i32, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_size_t)]
     L.speca_cache_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64)]
     L.speca_cache_stats.argtypes = [vp, ctypes.POINTER(CacheStats)]
+    L.speca_cache_check.argtypes = [vp, vp]
     L.speca_cache_next_slot.argtypes = [vp, i32, i32, ctypes.POINTER(vp)]
     L.speca_forecast_weights.argtypes = [i32, i32, i32, i32, vp, dbl, ctypes.POINTER(i32), vp]
     L.speca_status_string.argtypes = [i32]
@@ -361,6 +362,10 @@ def speca_cache_stats(cache, batch: int) -> dict:
     return out
 
 
+def speca_cache_check(cache, stream=None) -> None:
+    _check(_lib().speca_cache_check(cache, _stream_ptr(stream)), cache)
+
+
 def speca_cache_launch_count(cache) -> int:
     n = ctypes.c_uint64(0)
     _check(_lib().speca_cache_launch_count(cache, ctypes.byref(n)), cache)
@@ -463,6 +468,10 @@ class SpecaCache:
 
     def stats(self):
         return speca_cache_stats(self.handle, self.batch)
+
+    def check(self, stream=None):
+        """Waits for `stream` and raises if a staged copy of the bulk path gave up."""
+        speca_cache_check(self.handle, stream)
 
     def next_slot_batch(self, entry: int) -> torch.Tensor:
         """All samples' next planes of ``entry`` as one strided ``[B, N_e, D]`` view of the arena (raw-feature

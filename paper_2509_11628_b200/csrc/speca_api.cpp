@@ -22,6 +22,8 @@ constexpr size_t kAlign = 256;
 // interleave boundaries and measured 3-5 % slower on B200.
 constexpr size_t kPlaneAlign = 4096;
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+constexpr size_t kGaveUpWord = kVerifyTickets;  // index of the bulk path's flag among the counter words
+constexpr size_t kCounterBytes = (kVerifyTickets + 1) * sizeof(uint32_t);
 
 struct Layout {
     size_t segs_off, tiles_off[kNumTileSizes], partials_off, ticket_off, tables_off, total;
@@ -60,8 +62,8 @@ speca_status_t make_layout_impl(const speca_cache_config_t* cfg, Layout* L) {
     }
     L->partials_off = off;
     off = align_up(off + static_cast<size_t>(kMaxClusters) * B * 3 * sizeof(float), kAlign);  // up to 3 values per metric
-    L->ticket_off = off;
-    off = align_up(off + 2 * sizeof(uint32_t), kPlaneAlign);
+    L->ticket_off = off;  // the verify kernel's arrival counters, then the bulk path's gave-up flag
+    off = align_up(off + kCounterBytes, kPlaneAlign);
     L->tables_off = off;
 
     L->segs.resize(n_segs);
@@ -158,15 +160,19 @@ speca_status_t fail(speca_cache* c, speca_status_t st, const char* fmt, ...) {
     return st;
 }
 
+// Reports a failed runtime call and takes its error out of the thread's last-error slot, so that a
+// recoverable failure is not reported a second time by the next call (an error that broke the
+// context is returned again by the runtime itself).
 speca_status_t cuda_fail(speca_cache* c, cudaError_t err, const char* what) {
+    (void)cudaGetLastError();
     return fail(c, SPECA_ERR_CUDA, "%s: %s", what, cudaGetErrorString(err));
 }
 
 inline size_t elem_size(const speca_cache* c) { return c->dtype == SPECA_BF16 ? 2 : 4; }
 
-// An asynchronous error left by earlier work on this device surfaces here, before new work is queued.
+// An error left by earlier work on this thread surfaces here, once, before new work is queued.
 speca_status_t check_sticky(speca_cache* c) {
-    cudaError_t e = cudaPeekAtLastError();
+    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(c, e, "earlier CUDA error");
     return SPECA_OK;
 }
@@ -336,7 +342,7 @@ speca_status_t speca_cache_create(const speca_cache_config_t* cfg, speca_cache_t
     for (int k = 0; k < kNumTileSizes && ce == cudaSuccess; ++k)
         ce = cudaMemcpy(c->arena + L.tiles_off[k], L.tiles[k].data(), L.tiles[k].size() * sizeof(uint32_t),
                         cudaMemcpyHostToDevice);
-    if (ce == cudaSuccess) ce = cudaMemset(c->arena + L.ticket_off, 0, kAlign);
+    if (ce == cudaSuccess) ce = cudaMemset(c->arena + L.ticket_off, 0, kCounterBytes);
     if (ce != cudaSuccess) {
         delete c;
         return SPECA_ERR_CUDA;
@@ -348,8 +354,13 @@ speca_status_t speca_cache_create(const speca_cache_config_t* cfg, speca_cache_t
         delete c;
         return SPECA_ERR_UNSUPPORTED;
     }
-    c->cluster = 4;
-    int n_clusters = max_resident_verify_clusters(c->dtype, c->m, c->cluster);
+    c->cluster = SPECA_VERIFY_CLUSTER;
+    // the fewest over the orders a launch may have: samples below max_order run lower-order kernels
+    int n_clusters = kMaxClusters;
+    for (int v = 0; v <= c->m; ++v) {
+        const int n = max_resident_verify_clusters(c->dtype, v, c->cluster);
+        n_clusters = n < n_clusters ? n : n_clusters;
+    }
     if (n_clusters > kMaxClusters) n_clusters = kMaxClusters;
     c->grid_verify = n_clusters * c->cluster;
     *out = c;
@@ -363,7 +374,8 @@ speca_status_t speca_cache_destroy(speca_cache_t* c) {
     // the bulk path's kernels set this word when a bounded wait for a copy gave up
     uint32_t gave_up = 0;
     if (ce == cudaSuccess)
-        ce = cudaMemcpy(&gave_up, c->arena + c->L.ticket_off + sizeof(uint32_t), sizeof gave_up, cudaMemcpyDeviceToHost);
+        ce = cudaMemcpy(&gave_up, c->arena + c->L.ticket_off + kGaveUpWord * sizeof(uint32_t), sizeof gave_up,
+                        cudaMemcpyDeviceToHost);
     delete c;
     return (ce == cudaSuccess && gave_up == 0) ? SPECA_OK : SPECA_ERR_CUDA;
 }
@@ -462,7 +474,7 @@ speca_status_t update_impl(speca_cache_t* c, const void* const* feats, const dou
         p.tile_start = reinterpret_cast<const uint32_t*>(c->arena + L.tiles_off[c->tile_update]);
         p.arena = c->arena;
         p.dev_mask = nullptr;
-        p.err_flag = reinterpret_cast<uint32_t*>(c->arena + L.ticket_off) + 1;
+        p.err_flag = reinterpret_cast<uint32_t*>(c->arena + L.ticket_off) + kGaveUpWord;
         p.seg_lo = static_cast<uint32_t>(e_lo) * c->B;
         p.seg_hi = static_cast<uint32_t>(e_hi + 1) * c->B;
         p.tile_lo = tiles[p.seg_lo];
@@ -581,7 +593,7 @@ speca_status_t speca_forecast(speca_cache_t* c, const double* t_target, const ui
     p.arena = c->arena;
     p.dev_mask = dev_active_mask;
     p.weighted = c->layout == SPECA_LAYOUT_HISTORY ? 1 : 0;
-    p.err_flag = reinterpret_cast<uint32_t*>(c->arena + L.ticket_off) + 1;
+    p.err_flag = reinterpret_cast<uint32_t*>(c->arena + L.ticket_off) + kGaveUpWord;
     p.seg_lo = static_cast<uint32_t>(e_lo) * c->B;
     p.seg_hi = static_cast<uint32_t>(e_hi + 1) * c->B;
     p.tile_lo = tiles[p.seg_lo];
@@ -772,7 +784,11 @@ static speca_status_t verify_impl(speca_cache_t* c, int32_t metric, const void* 
     const Layout& L = c->L;
     const SegDesc& s0 = L.segs[static_cast<size_t>(c->verify_entry) * c->B];
     const uint32_t te = verify_tile_elems(c->dtype, v_max);
-    p.segs = reinterpret_cast<const SegDesc*>(c->arena + L.segs_off) + static_cast<size_t>(c->verify_entry) * c->B;
+    // the entry's B tables follow one another in the arena, one table (max_order + 1 planes) apart
+    p.plane0_off = s0.plane0_off;
+    p.sample_pitch = s0.plane_stride * static_cast<uint64_t>(c->m + 1);
+    p.plane_stride = s0.plane_stride;
+    p.io_pitch = static_cast<uint64_t>(s0.n_elems) * esz;
     p.arena = c->arena;
     p.dev_mask = dev_active_mask;
     p.weighted = c->layout == SPECA_LAYOUT_HISTORY ? 1 : 0;
@@ -852,9 +868,10 @@ speca_status_t speca_verify_decide(int32_t metric, const double* dev_sums, int32
         if (std::isnan(tau[b])) return SPECA_ERR_INVALID_ARG;
         q.tau[b] = tau[b];
     }
-    if (cudaPeekAtLastError() != cudaSuccess) return SPECA_ERR_CUDA;
+    if (cudaGetLastError() != cudaSuccess) return SPECA_ERR_CUDA;  // an earlier error, reported once
     cudaError_t ce = launch_decide(metric, dev_sums, batch, q, dev_active_mask, dev_err, dev_accept,
                                    static_cast<cudaStream_t>(stream));
+    if (ce != cudaSuccess) (void)cudaGetLastError();
     return ce == cudaSuccess ? SPECA_OK : SPECA_ERR_CUDA;
 }
 
@@ -990,6 +1007,26 @@ speca_status_t speca_cache_next_slot(const speca_cache_t* c, int32_t entry, int3
 speca_status_t speca_cache_stats(const speca_cache_t* c, speca_cache_stats_t* out) {
     if (c == nullptr || out == nullptr) return SPECA_ERR_INVALID_ARG;
     *out = c->stats;
+    return SPECA_OK;
+}
+
+speca_status_t speca_cache_check(speca_cache_t* c, void* stream) {
+    if (c == nullptr) return SPECA_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return fail(c, SPECA_ERR_CUDA, "cudaSetDevice failed");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t ce = cudaStreamSynchronize(s);
+    if (ce != cudaSuccess) return cuda_fail(c, ce, "check: stream");
+    uint32_t* word = reinterpret_cast<uint32_t*>(c->arena + c->L.ticket_off) + kGaveUpWord;
+    uint32_t gave_up = 0;
+    ce = cudaMemcpyAsync(&gave_up, word, sizeof gave_up, cudaMemcpyDeviceToHost, s);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(s);
+    if (ce != cudaSuccess) return cuda_fail(c, ce, "check: read-back");
+    if (gave_up != 0) {
+        ce = cudaMemsetAsync(word, 0, sizeof gave_up, s);
+        if (ce != cudaSuccess) return cuda_fail(c, ce, "check: clear");
+        return fail(c, SPECA_ERR_CUDA, "a staged copy never landed: results since the last check are incomplete");
+    }
     return SPECA_OK;
 }
 

@@ -14,9 +14,25 @@ namespace speca {
 constexpr uint32_t kTileSizes[] = {4096, 8192, 16384, 32768};
 constexpr int kNumTileSizes = 4;
 constexpr int kThreads = 256;       // verify kernel CTA size
-// Tile of the verify kernel compiled for order v (the highest order among the launch's samples).
-__host__ __device__ constexpr uint32_t verify_tile_bytes(int v) { return v <= 2 ? 16384u : 8192u; }
+// Launch shape of the verify kernel: 32-byte vectors per thread and plane for orders 0-2 (orders 3-4
+// always hold one), the CTAs per SM the registers are capped for, and the cluster size.
+#ifndef SPECA_VERIFY_U
+#define SPECA_VERIFY_U 2
+#endif
+#ifndef SPECA_VERIFY_MINB
+#define SPECA_VERIFY_MINB 2
+#endif
+#ifndef SPECA_VERIFY_CLUSTER
+#define SPECA_VERIFY_CLUSTER 4
+#endif
+__host__ __device__ constexpr int verify_vectors(int v) { return v <= 2 ? SPECA_VERIFY_U : 1; }
+// Tile of the verify kernel compiled for order v (the highest order among the launch's samples):
+// 256 threads x verify_vectors(v) x 32 bytes per plane.
+__host__ __device__ constexpr uint32_t verify_tile_bytes(int v) { return 8192u * verify_vectors(v); }
 constexpr int kMaxClusters = 1024;  // upper bound on verify clusters (reduction scratch rows)
+// Arrival counter of the verify kernel, zero between launches. (The word after it is the bulk
+// path's gave-up flag in a cache's arena.)
+constexpr int kVerifyTickets = 1;
 
 inline int tile_size_index(uint32_t tile_bytes) {
     for (int i = 0; i < kNumTileSizes; ++i)
@@ -99,14 +115,17 @@ struct SumParams {
 
 // Arguments of the fused forecast + relative-L2 kernel over the verification entry.
 struct VerifyParams {
-    const SegDesc* segs;  // segments of the verify entry only (B of them)
+    // The verification entry's B tables are laid out evenly: sample b's plane 0 starts at
+    // arena + plane0_off + b * sample_pitch, its planes are plane_stride bytes apart, and its row of
+    // the [B, N_v, D] tensors (fresh, out_pred) starts b * io_pitch bytes in.
+    uint64_t plane0_off, sample_pitch, plane_stride, io_pitch;
     char* arena;
     const uint8_t* dev_mask;
     const char* fresh;  // [B, N_v, D]
     char* out_pred;     // may be null
     float* err;
     uint8_t* accept;
-    float* partials;     // [n_clusters][B][values of the metric: 2, or 3 for cosine]
+    float* partials;     // [B][n_clusters][values of the metric: 2, or 3 for cosine]
     uint32_t* ticket;    // arrival counter, zero between launches
     double* raw_sums;    // [B][4] or null: write the combined running values instead of err / accept
     // fused per-sample continuation (speca_verify_select); sel_active == null: not fused

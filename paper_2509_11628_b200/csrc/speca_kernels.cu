@@ -986,10 +986,10 @@ __global__ void __launch_bounds__(kBulkThreads) stream_bulk_kernel(const __grid_
 // ------------------------------------------------------------------------------------------------
 
 constexpr int kMaxClusterSize = 8;
-// 256 threads x U x 32 B per plane and tile; U = 2 while the V + 2 streams fit in registers
+// 256 threads x verify_vectors(order) 32-byte vectors per plane and tile
 constexpr int kVerifyW = 32;
-static_assert(verify_tile_bytes(0) == kThreads * 2 * kVerifyW && verify_tile_bytes(4) == kThreads * kVerifyW,
-              "verify tile sizes");
+static_assert(verify_tile_bytes(0) == kThreads * kVerifyW * verify_vectors(0) && verify_tile_bytes(4) == kThreads * kVerifyW,
+              "verify tile size");
 
 // Error metrics of the verification. Eq. 4 is the relative l2 error; the appendix on error metrics
 // also evaluates l1, l-infinity and cosine similarity, all in relative form. Each metric keeps NA
@@ -1030,7 +1030,22 @@ struct Metric {
         else
             return x + y;
     }
+    // The error from the totals. err is handed out as a binary32, so the square roots and the division
+    // are binary32 too (a few ulp of the stored value; fp64 square roots and divisions are long dependent
+    // instruction sequences on the kernel's critical tail) and the accept flag is exactly err <= tau on
+    // the stored values. Totals outside the binary32 range (or NaN) take the fp64 formulas.
     __device__ static __forceinline__ double error(const double (&s)[3], double eps) {
+        const bool fits = fabs(s[0]) < 1e38 && fabs(s[1]) < 1e38 && (NA < 3 || fabs(s[2]) < 1e38);
+        if (fits) {
+            const float a0 = static_cast<float>(s[0]), a1 = static_cast<float>(s[1]), a2 = static_cast<float>(s[2]);
+            const float e = static_cast<float>(eps);
+            if constexpr (M == SPECA_METRIC_L2)
+                return static_cast<double>(sqrtf(a0) / (sqrtf(a1) + e));
+            else if constexpr (M == SPECA_METRIC_COSINE)
+                return static_cast<double>(1.0f - a0 / (sqrtf(a1) * sqrtf(a2) + e));
+            else
+                return static_cast<double>(a0 / (a1 + e));
+        }
         if constexpr (M == SPECA_METRIC_L2)
             return sqrt(s[0]) / (sqrt(s[1]) + eps);
         else if constexpr (M == SPECA_METRIC_COSINE)
@@ -1040,68 +1055,105 @@ struct Metric {
     }
 };
 
-template <int DT, int V, int W, int U, int M>
-__device__ __forceinline__ void verify_tile(const char* __restrict__ plane0, uint64_t stride,
-                                            const char* __restrict__ fresh, char* __restrict__ out_pred, uint32_t cnt,
-                                            const float (&mu)[kCoef], bool weighted, float (&a)[3]) {
-    constexpr int EPV = W / Elem<DT>::kBytes;
-    const uint32_t nvec = cnt / EPV;
-    Vec<W> d[V + 1][U];
-    Vec<W> fv[U];
+// One tile of the verification entry as a CTA sees it.
+struct VTile {
+    const char* plane0;  // plane 0 of the tile
+    const char* fresh;
+    char* pred;          // null: the forecast is not kept
+    uint32_t cnt;        // elements (the last tile of a sample is ragged)
+    int32_t slot;        // sample's position among the samples this cluster meets
+    int32_t b;           // sample
+    int32_t v;           // the sample's order
+    bool fast;           // compiled order and 32-byte aligned rows: vector registers hold the tile
+};
+
+// The tile's v + 1 planes and the fresh feature, U 32-byte vectors per thread each.
+template <int V, int U>
+struct VRegs {
+    Vec<kVerifyW> d[V + 1][U];
+    Vec<kVerifyW> f[U];
+};
+
+// Issues all of the tile's loads before anything is consumed.
+template <int DT, int V, int U>
+__device__ __forceinline__ void verify_issue(VRegs<V, U>& r, const VTile& t, uint64_t stride) {
+    constexpr int W = kVerifyW, EPV = W / Elem<DT>::kBytes;
+    const uint32_t nvec = t.cnt / EPV;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const uint32_t idx = u * kThreads + threadIdx.x;
         if (idx < nvec) {
+            const size_t o = static_cast<size_t>(idx) * W;
 #pragma unroll
-            for (int i = 0; i <= V; ++i) d[i][u] = load_vec<W>(plane0 + i * stride + static_cast<size_t>(idx) * W);
-            fv[u] = load_vec<W>(fresh + static_cast<size_t>(idx) * W);
+            for (int i = 0; i <= V; ++i) r.d[i][u] = load_vec<W>(t.plane0 + i * stride + o);
+            r.f[u] = load_vec<W>(t.fresh + o);
         }
     }
+}
+
+// Eq. 2 on the tile's registers, the forecast rounded to the storage type as the model would consume it,
+// then one fold of (forecast, feature) per element into the running values. A vector is worked
+// through in 16-byte halves so that few unpacked values are live beside the vectors still to come.
+template <int DT, int V, int U, int M>
+__device__ __forceinline__ void verify_fold(const VRegs<V, U>& r, const VTile& t, uint64_t stride, const float (&mu)[kCoef],
+                                            bool weighted, float (&a)[3]) {
+    constexpr int W = kVerifyW, EPV = W / Elem<DT>::kBytes, H = EPV / 2;
+    const uint32_t nvec = t.cnt / EPV;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const uint32_t idx = u * kThreads + threadIdx.x;
         if (idx < nvec) {
-            float acc[EPV], f[EPV];
-            unpack_vec<DT, W>(d[V][u], acc);
-            if (weighted) {
+            Vec<W> pv;
 #pragma unroll
-                for (int k = 0; k < EPV; ++k) acc[k] *= mu[V];
-            }
+            for (int h = 0; h < 2; ++h) {
+                Vec<16> part;
+                float acc[H], f[H];
 #pragma unroll
-            for (int i = V; i >= 1; --i) {
-                float lo[EPV];
-                unpack_vec<DT, W>(d[i - 1][u], lo);
+                for (int k = 0; k < 4; ++k) part.r[k] = r.d[V][u].r[4 * h + k];
+                unpack_vec<DT, 16>(part, acc);
                 if (weighted) {
 #pragma unroll
-                    for (int k = 0; k < EPV; ++k) acc[k] = fmaf(lo[k], mu[i - 1], acc[k]);
-                } else {
-#pragma unroll
-                    for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+                    for (int k = 0; k < H; ++k) acc[k] *= mu[V];
                 }
-            }
-            // the forecast as the model would consume it: rounded to the storage type
-            const Vec<W> pv = pack_vec<DT, W>(acc);
-            unpack_vec<DT, W>(pv, acc);
-            unpack_vec<DT, W>(fv[u], f);
 #pragma unroll
-            for (int k = 0; k < EPV; ++k) {
-                Metric<M>::fold(acc[k], f[k], a);
+                for (int i = V; i >= 1; --i) {
+                    float lo[H];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) part.r[k] = r.d[i - 1][u].r[4 * h + k];
+                    unpack_vec<DT, 16>(part, lo);
+                    if (weighted) {
+#pragma unroll
+                        for (int k = 0; k < H; ++k) acc[k] = fmaf(lo[k], mu[i - 1], acc[k]);
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < H; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+                    }
+                }
+                part = pack_vec<DT, 16>(acc);
+                unpack_vec<DT, 16>(part, acc);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) pv.r[4 * h + k] = part.r[k];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) part.r[k] = r.f[u].r[4 * h + k];
+                unpack_vec<DT, 16>(part, f);
+#pragma unroll
+                for (int k = 0; k < H; ++k) Metric<M>::fold(acc[k], f[k], a);
             }
-            if (out_pred != nullptr) store_vec<W>(out_pred + static_cast<size_t>(idx) * W, pv);
+            if (t.pred != nullptr) store_vec<W>(t.pred + static_cast<size_t>(idx) * W, pv);
         }
     }
-    for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += kThreads) {
-        float acc = load_scalar<DT>(plane0 + V * stride, j);
+    // ragged end of a sample's last tile
+    for (uint32_t j = nvec * EPV + threadIdx.x; j < t.cnt; j += kThreads) {
+        float acc = load_scalar<DT>(t.plane0 + V * stride, j);
         if (weighted) acc *= mu[V];
 #pragma unroll
         for (int i = V; i >= 1; --i) {
-            const float lo = load_scalar<DT>(plane0 + (i - 1) * stride, j);
+            const float lo = load_scalar<DT>(t.plane0 + (i - 1) * stride, j);
             acc = weighted ? fmaf(lo, mu[i - 1], acc) : fmaf(acc, mu[i - 1], lo);
         }
         acc = round_storage<DT>(acc);
-        const float f = load_scalar<DT>(fresh, j);
-        Metric<M>::fold(acc, f, a);
-        if (out_pred != nullptr) store_scalar<DT>(out_pred, j, acc);
+        Metric<M>::fold(acc, load_scalar<DT>(t.fresh, j), a);
+        if (t.pred != nullptr) store_scalar<DT>(t.pred, j, acc);
     }
 }
 
@@ -1149,51 +1201,63 @@ __device__ __noinline__ void verify_tile_any(const char* __restrict__ plane0, ui
     }
 }
 
-// Per-sample continuation of the speculative run, for the first `batch` threads of a block (every
-// thread of the block must call it: it synchronises). keep / next: shared scratch of SPECA_MAX_BATCH bytes.
-// No __restrict__ here: the fused caller wrote `accept` earlier in the same kernel.
-__device__ __forceinline__ void select_in_block(const uint8_t* accept, int32_t k_max, int32_t group, int32_t batch,
-                                                int32_t* spec_count, const uint8_t* active_in, uint8_t* active_out,
-                                                int32_t* idx_out, int32_t* n_out, uint8_t* keep, uint8_t* next) {
-    const int b = threadIdx.x;
-    if (b < batch) {
-        const bool a = active_in[b] != 0;
-        const bool ok = a && accept[b] != 0;
-        int32_t c = spec_count[b];
-        if (ok) {
-            c += 1;
-            spec_count[b] = c;
-        }
-        keep[b] = (ok && c < k_max) ? 1 : 0;
-    }
-    __syncthreads();
-    if (b < batch) {
-        const int g0 = (b / group) * group;
-        uint8_t all = 1;
-        for (int i = 0; i < group; ++i) all &= keep[g0 + i];
-        next[b] = all;
-        active_out[b] = all;
-    }
-    __syncthreads();
-    if (b == 0) {
-        int32_t n = 0;
-        for (int i = 0; i < batch; ++i)
-            if (next[i]) {
-                if (idx_out != nullptr) idx_out[n] = i;
-                ++n;
+// Per-sample continuation of the speculative run by ONE warp (all 32 lanes call it; B <= 64, lane l
+// looks after samples l and l + 32). `accept` may have been written by other CTAs of the same kernel
+// just before (the caller has fenced): it is read around L1.
+__device__ __forceinline__ void select_in_warp(const uint8_t* accept, int32_t k_max, int32_t group, int32_t batch,
+                                               int32_t* spec_count, const uint8_t* active_in, uint8_t* active_out,
+                                               int32_t* idx_out, int32_t* n_out) {
+    const int lane = threadIdx.x & 31;
+    uint64_t keep = 0;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int b = lane + 32 * h;
+        bool k = false;
+        if (b < batch) {
+            const bool ok = active_in[b] != 0 && __ldcg(accept + b) != 0;
+            int32_t c = spec_count[b];
+            if (ok) {
+                c += 1;
+                spec_count[b] = c;
             }
-        if (n_out != nullptr) *n_out = n;
+            k = ok && c < k_max;
+        }
+        keep |= static_cast<uint64_t>(__ballot_sync(0xFFFFFFFFu, k)) << (32 * h);
     }
+    uint64_t next = 0;  // a group continues only if every member does
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int b = lane + 32 * h;
+        bool all = false;
+        if (b < batch) {
+            const int g0 = (b / group) * group;
+            const uint64_t members = (group >= 64 ? ~0ull : ((1ull << group) - 1ull)) << g0;
+            all = (keep & members) == members;
+            active_out[b] = all ? 1 : 0;
+        }
+        next |= static_cast<uint64_t>(__ballot_sync(0xFFFFFFFFu, all)) << (32 * h);
+    }
+    if (idx_out != nullptr) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int b = lane + 32 * h;
+            if (b < batch && ((next >> b) & 1ull)) idx_out[__popcll(next & ((1ull << b) - 1ull))] = b;
+        }
+    }
+    if (lane == 0 && n_out != nullptr) *n_out = __popcll(next);
 }
 
 // Tiles of the active samples form one list of T = (active samples) x (tiles per sample) tiles;
-// cluster q of Q owns the contiguous range [q*T/Q, (q+1)*T/Q).
+// cluster q of Q owns the contiguous range [q*T/Q, (q+1)*T/Q). Q <= 1024, so the products fit 32 bits
+// whenever T < 2^22 (every benchmark shape: T is a few thousand): the 64-bit division is the rare case.
 __device__ __forceinline__ uint32_t range_begin(uint32_t q, uint32_t Q, uint32_t T) {
+    if (T < (1u << 22)) return q * T / Q;
     return static_cast<uint32_t>(static_cast<uint64_t>(q) * T / Q);
 }
 // The cluster whose range holds `tile`: the smallest q with range_begin(q + 1) > tile, that is
 // ceil((tile + 1) * Q / T) - 1. Holds for Q > T too, where some clusters own nothing.
 __device__ __forceinline__ uint32_t range_owner(uint32_t tile, uint32_t Q, uint32_t T) {
+    if (T < (1u << 22)) return ((tile + 1) * Q - 1) / T;
     return static_cast<uint32_t>(((static_cast<uint64_t>(tile) + 1) * Q - 1) / T);
 }
 // Index of the a-th set bit of `bits` (a < popcount).
@@ -1202,142 +1266,221 @@ __device__ __forceinline__ int nth_set_bit(uint64_t bits, uint32_t a) {
     return __ffsll(static_cast<long long>(bits)) - 1;
 }
 
+// Release / acquire fences at device scope (lighter than the sequentially consistent __threadfence).
+__device__ __forceinline__ void fence_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
+
 // Each cluster walks a contiguous range of the active samples' tiles, its CTAs taking every
-// (cluster size)-th tile, so a cluster meets each sample once and reduces once per sample:
-// registers -> warp shuffle -> shared memory (CTA) -> the leader CTA's shared memory through the
-// cluster's distributed shared memory -> one partial per (cluster, sample) in global scratch. The
-// cluster that arrives last (ticket counter, nobody waits) adds each sample's partials in fp64, one
-// warp per sample in a fixed lane/shuffle order, and applies Eq. 4 and the accept rule.
+// (cluster size)-th tile. The running values go
+//   registers -> warp shuffle -> this CTA's shared memory, one slot per sample the cluster meets
+//   -> once, at the end of the range: the leader CTA's shared memory through the cluster's distributed
+//      shared memory, ONE cluster barrier per launch
+//   -> one partial per (cluster, sample) in global scratch.
+// The cluster that arrives last (ticket counter, nobody waits) adds every sample's partials in fp64 in
+// a fixed lane / shuffle order, applies Eq. 4 and the accept rule, runs the fused continuation rule
+// and re-zeroes the ticket.
 template <int DT, int V, int M>
-__global__ void __launch_bounds__(kThreads, 2) verify_kernel(const __grid_constant__ VerifyParams p) {
+__global__ void __launch_bounds__(kThreads, V <= 2 ? SPECA_VERIFY_MINB : 2) verify_kernel(const __grid_constant__ VerifyParams p) {
     constexpr uint32_t kTile = verify_tile_bytes(V) / Elem<DT>::kBytes;
-    constexpr int W = kVerifyW, U = verify_tile_bytes(V) / (kThreads * kVerifyW);
+    constexpr int W = kVerifyW, U = verify_vectors(V);
+    constexpr int NA = Metric<M>::NA;
+    constexpr int kWarps = kThreads / 32;
     cg::cluster_group cluster = cg::this_cluster();
     const uint32_t csize = cluster.num_blocks();
     const uint32_t crank = cluster.block_rank();
     const uint32_t cid = blockIdx.x / csize;
     const uint32_t Q = gridDim.x / csize;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    constexpr int NA = Metric<M>::NA;
-    __shared__ float warp_part[NA][kThreads / 32];
-    __shared__ float cluster_slot[2][NA][kMaxClusterSize];  // [parity][value][rank], leader's copy is used
+    __shared__ float warp_part[SPECA_MAX_BATCH][NA][kWarps];            // [slot][value][warp], this CTA's
+    __shared__ float cluster_slot[SPECA_MAX_BATCH][NA][kMaxClusterSize];  // [slot][value][rank], the leader's copy is used
     __shared__ uint32_t active_bits[2];
     __shared__ bool is_last;
-    __shared__ uint8_t sel_keep[SPECA_MAX_BATCH], sel_next[SPECA_MAX_BATCH];
 
+    // Every CTA of the cluster is running once this barrier completes; it is only waited for right
+    // before the first access to the leader's shared memory.
+    cluster.barrier_arrive();
+
+    for (int i = threadIdx.x; i < SPECA_MAX_BATCH * NA * kWarps; i += kThreads) (&warp_part[0][0][0])[i] = 0.f;
     // samples that take part: a defined table and, with a device mask, a non-zero byte
     if (threadIdx.x < 64) {
         const int b = threadIdx.x;
         const bool on = b < p.batch && p.order[b] >= 0 && (p.dev_mask == nullptr || p.dev_mask[b] != 0);
         const uint32_t ballot = __ballot_sync(0xFFFFFFFFu, on);
-        if ((threadIdx.x & 31) == 0) active_bits[threadIdx.x >> 5] = ballot;
+        if (lane == 0) active_bits[warp] = ballot;
     }
     __syncthreads();
     const uint64_t bits = static_cast<uint64_t>(active_bits[0]) | (static_cast<uint64_t>(active_bits[1]) << 32);
     const uint32_t n_active = __popcll(bits);
-    if (n_active == 0) {  // every CTA of the grid takes this exit together
-        if (p.sel_active != nullptr && blockIdx.x == 0)
-            select_in_block(p.accept, p.sel_kmax, p.sel_group, p.batch, p.sel_spec, p.dev_mask, p.sel_active, p.sel_idx,
-                            p.sel_n, sel_keep, sel_next);
-        return;
-    }
     const uint32_t tps = p.tiles_per_sample;
     const uint32_t T = n_active * tps;
+    const uint32_t t_lo = n_active ? range_begin(cid, Q, T) : 0, t_hi = n_active ? range_begin(cid + 1, Q, T) : 0;
+    if (t_lo >= t_hi) {  // nobody active, or more clusters than tiles: the whole cluster leaves together
+        cluster.barrier_wait();
+        if (n_active == 0 && p.sel_active != nullptr && blockIdx.x == 0 && warp == 0)
+            select_in_warp(p.accept, p.sel_kmax, p.sel_group, p.batch, p.sel_spec, p.dev_mask, p.sel_active, p.sel_idx, p.sel_n);
+        return;
+    }
+    const uint32_t a_first = t_lo / tps;
+    const uint32_t span = (t_hi - 1) / tps - a_first + 1;  // samples this cluster meets
+    const uint32_t Q_busy = Q < T ? Q : T;                 // clusters that own at least one tile
 
-    float acc[3] = {0.f, 0.f, 0.f};
-    uint32_t parity = 0;
-
-    auto flush = [&](int b) {
-#pragma unroll
-        for (int i = 0; i < NA; ++i) {
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1)
-                acc[i] = Metric<M>::merge(acc[i], __shfl_xor_sync(0xFFFFFFFFu, acc[i], off));
-            if ((threadIdx.x & 31) == 0) warp_part[i][threadIdx.x >> 5] = acc[i];
+    // tile number -> what to load; the sample lookup is redone only when the sample changes
+    uint32_t known_a = 0xFFFFFFFFu;
+    int known_b = 0;
+    auto locate = [&](uint32_t t) {
+        VTile x;
+        const uint32_t a = t / tps;
+        if (a != known_a) {
+            known_a = a;
+            known_b = nth_set_bit(bits, a);
         }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            // hand the CTA's values to the cluster leader through distributed shared memory
-            float* leader = cluster.map_shared_rank(&cluster_slot[parity][0][0], 0);
-#pragma unroll
-            for (int i = 0; i < NA; ++i) {
-                float s = warp_part[i][0];
-#pragma unroll
-                for (int w = 1; w < kThreads / 32; ++w) s = Metric<M>::merge(s, warp_part[i][w]);
-                leader[i * kMaxClusterSize + crank] = s;
-            }
-        }
-        cluster.sync();
-        if (crank == 0 && threadIdx.x == 0) {
-            float* dst = p.partials + (static_cast<size_t>(cid) * p.batch + b) * NA;
-#pragma unroll
-            for (int i = 0; i < NA; ++i) {
-                float s = cluster_slot[parity][i][0];
-                for (uint32_t r = 1; r < csize; ++r) s = Metric<M>::merge(s, cluster_slot[parity][i][r]);
-                __stcg(dst + i, s);
-            }
-        }
-        // Slots alternate between two buffers: a CTA can write the buffer of flush k+2 only after
-        // the barrier of flush k+1, which the leader enters after it has read the buffer of flush k.
-        parity ^= 1;
-        acc[0] = acc[1] = acc[2] = 0.f;
+        const uint32_t elem0 = (t - a * tps) * kTile;
+        const uint64_t byte0 = static_cast<uint64_t>(elem0) * Elem<DT>::kBytes;
+        const uint64_t io = static_cast<uint64_t>(known_b) * p.io_pitch + byte0;
+        x.b = known_b;
+        x.slot = static_cast<int32_t>(a - a_first);
+        x.v = p.order[known_b];
+        x.cnt = min(kTile, p.n_elems - elem0);
+        x.plane0 = p.arena + p.plane0_off + static_cast<uint64_t>(known_b) * p.sample_pitch + byte0;
+        x.fresh = p.fresh + io;
+        x.pred = p.out_pred != nullptr ? p.out_pred + io : nullptr;
+        x.fast = x.v == V && ((reinterpret_cast<uintptr_t>(x.plane0) | reinterpret_cast<uintptr_t>(x.fresh) |
+                               reinterpret_cast<uintptr_t>(x.pred)) & (W - 1)) == 0;
+        return x;
     };
 
-    const uint32_t t_lo = range_begin(cid, Q, T), t_hi = range_begin(cid + 1, Q, T);
-    if (t_lo < t_hi) {
-        for (uint32_t a = t_lo / tps; a <= (t_hi - 1) / tps; ++a) {  // uniform over the cluster
-            const int b = nth_set_bit(bits, a);
-            const int v = p.order[b];
-            const SegDesc sd = p.segs[b];
-            float mu[kCoef];
+    float acc[3] = {0.f, 0.f, 0.f};
+    float mu[kCoef] = {};
+    int32_t acc_slot = -1;
+    // the warp's running values of the sample it has been folding go to the sample's slot
+    auto park = [&]() {
+        if (acc_slot < 0) return;
 #pragma unroll
-            for (int i = 0; i < kCoef; ++i) mu[i] = p.coef[b][i];
-            const uint32_t first = max(t_lo, a * tps) - a * tps, last = min(t_hi, (a + 1) * tps) - a * tps;
-            for (uint32_t tile = first + crank; tile < last; tile += csize) {
-                const uint32_t elem0 = tile * kTile;
-                const uint32_t cnt = min(kTile, p.n_elems - elem0);
-                const uint64_t byte0 = static_cast<uint64_t>(elem0) * Elem<DT>::kBytes;
-                const char* plane0 = p.arena + sd.plane0_off + byte0;
-                const char* fresh = p.fresh + sd.io_off + byte0;
-                char* pred = p.out_pred != nullptr ? p.out_pred + sd.io_off + byte0 : nullptr;
-                const bool fast = v == V && ((reinterpret_cast<uintptr_t>(plane0) | reinterpret_cast<uintptr_t>(fresh) |
-                                              reinterpret_cast<uintptr_t>(pred)) & (W - 1)) == 0;
-                if (fast)
-                    verify_tile<DT, V, W, U, M>(plane0, sd.plane_stride, fresh, pred, cnt, mu, p.weighted != 0, acc);
-                else
-                    verify_tile_any<DT, M>(plane0, sd.plane_stride, fresh, pred, cnt, v, mu, p.weighted != 0, acc);
+        for (int i = 0; i < NA; ++i) {
+            float s = acc[i];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) s = Metric<M>::merge(s, __shfl_xor_sync(0xFFFFFFFFu, s, off));
+            if (lane == 0) warp_part[acc_slot][i][warp] = s;
+        }
+        acc[0] = acc[1] = acc[2] = 0.f;
+    };
+    auto enter = [&](const VTile& t) {  // uniform over the CTA
+        if (t.slot != acc_slot) {
+            park();
+            acc_slot = t.slot;
+#pragma unroll
+            for (int i = 0; i < kCoef; ++i) mu[i] = p.coef[t.b][i];
+        }
+    };
+    // A sample's tiles are all vector tiles or all generic ones (its rows are 32-byte aligned and its
+    // order is the compiled one, or not). First pass: the vector tiles -- all of a tile's loads, then its
+    // arithmetic. Second pass, rarely needed: the generic ones (kept out of the first loop so that no
+    // call sits between a tile's loads and their use).
+    bool any_generic = false;
+    {
+        VRegs<V, U> r;
+        for (uint32_t t = t_lo + crank; t < t_hi; t += csize) {
+            const VTile x = locate(t);
+            if (!x.fast) {
+                any_generic = true;
+                continue;
             }
-            flush(b);
+            verify_issue<DT, V, U>(r, x, p.plane_stride);
+            enter(x);
+            verify_fold<DT, V, U, M>(r, x, p.plane_stride, mu, p.weighted != 0, acc);
+        }
+        park();
+        acc_slot = -1;
+    }
+    if (any_generic) {
+        for (uint32_t t = t_lo + crank; t < t_hi; t += csize) {
+            const VTile x = locate(t);
+            if (x.fast) continue;
+            enter(x);
+            verify_tile_any<DT, M>(x.plane0, p.plane_stride, x.fresh, x.pred, x.cnt, x.v, mu, p.weighted != 0, acc);
+        }
+        park();
+    }
+    __syncthreads();
+
+    // this CTA's value of every sample the cluster met -> the leader's shared memory, one barrier
+    cluster.barrier_wait();
+    if (threadIdx.x < span * NA) {
+        const uint32_t slot = threadIdx.x / NA, i = threadIdx.x % NA;
+        float s = warp_part[slot][i][0];
+#pragma unroll
+        for (int w = 1; w < kWarps; ++w) s = Metric<M>::merge(s, warp_part[slot][i][w]);
+        float* leader = cluster.map_shared_rank(&cluster_slot[0][0][0], 0);
+        leader[(slot * NA + i) * kMaxClusterSize + crank] = s;
+    }
+    cluster.sync();
+    if (crank != 0) return;  // nobody touches a non-leader's shared memory after this barrier
+
+    // the cluster's partial of every sample it met -> global scratch
+    for (uint32_t slot = warp; slot < span; slot += kWarps) {
+        const int b = nth_set_bit(bits, a_first + slot);
+        float part[3] = {0.f, 0.f, 0.f};
+#pragma unroll
+        for (int i = 0; i < NA; ++i) {
+            float s = lane < csize ? cluster_slot[slot][i][lane] : 0.f;  // 0 is neutral for the sums and for maxima of magnitudes
+#pragma unroll
+            for (int off = kMaxClusterSize / 2; off > 0; off >>= 1) s = Metric<M>::merge(s, __shfl_xor_sync(0xFFFFFFFFu, s, off));
+            part[i] = s;
+        }
+        if (lane == 0) {
+            float* dst = p.partials + (static_cast<size_t>(b) * Q + cid) * NA;
+#pragma unroll
+            for (int i = 0; i < NA; ++i) __stcg(dst + i, part[i]);
+            fence_gpu();  // this partial is visible device-wide before the ticket below is taken
         }
     }
-
-    if (crank != 0) return;  // nobody touches a non-leader's shared memory after its last barrier
-
+    __syncthreads();
     if (threadIdx.x == 0) {
-        __threadfence();  // partials visible before the ticket
         const uint32_t t = atomicAdd(p.ticket, 1u);
-        is_last = (t == Q - 1);
+        fence_gpu();
+        is_last = (t == Q_busy - 1);
     }
     __syncthreads();
     if (!is_last) return;
-    __threadfence();
-    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (uint32_t a = warp; a < n_active; a += kThreads / 32) {
-        const int b = nth_set_bit(bits, a);
-        const uint32_t q_lo = range_owner(a * tps, Q, T), q_hi = range_owner((a + 1) * tps - 1, Q, T);
+
+    // Last cluster to arrive. A sample's partials sit side by side in the scratch ([sample][cluster]).
+    // A group of L lanes adds one sample's partials: with few samples each has many partials and a
+    // whole warp takes one sample; with many samples each has few and a warp takes four at a time.
+    // Per sample the order is fixed (lane l adds clusters q_lo + l, q_lo + l + L, ..., then a shuffle
+    // tree over the group), four loads per lane are in flight at once, and the sums are fp64.
+    const uint32_t L = n_active > 8 ? 8 : 32, per_warp = 32 / L;
+    const uint32_t g = lane / L, l = lane % L;
+    const bool holes = Q > T;  // more clusters than tiles: some clusters in a sample's span own nothing
+    for (uint32_t a0 = 0; a0 < n_active; a0 += kWarps * per_warp) {  // uniform over the CTA
+        const uint32_t a = a0 + warp * per_warp + g;
+        const bool live = a < n_active;
+        int b = 0;
         double s[3] = {0.0, 0.0, 0.0};
-        for (uint32_t q = q_lo + lane; q <= q_hi; q += 32) {
-            if (range_begin(q, Q, T) == range_begin(q + 1, Q, T)) continue;  // owns no tile (Q > T): wrote nothing
-            const float* src = p.partials + (static_cast<size_t>(q) * p.batch + b) * NA;
+        if (live) {
+            b = nth_set_bit(bits, a);
+            const uint32_t q_lo = range_owner(a * tps, Q, T), q_hi = range_owner((a + 1) * tps - 1, Q, T);
+            const float* row = p.partials + static_cast<size_t>(b) * Q * NA;
+            for (uint32_t q0 = q_lo + l; q0 <= q_hi; q0 += 4 * L) {
+                float v[4][3];
 #pragma unroll
-            for (int i = 0; i < NA; ++i) s[i] = Metric<M>::merge(s[i], static_cast<double>(__ldcg(src + i)));
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t q = q0 + j * L;
+                    const bool has = q <= q_hi && !(holes && range_begin(q, Q, T) == range_begin(q + 1, Q, T));
+#pragma unroll
+                    for (int i = 0; i < NA; ++i) v[j][i] = has ? __ldcg(row + static_cast<size_t>(q) * NA + i) : 0.f;  // 0: neutral
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+#pragma unroll
+                    for (int i = 0; i < NA; ++i) s[i] = Metric<M>::merge(s[i], static_cast<double>(v[j][i]));
+                }
+            }
         }
 #pragma unroll
         for (int i = 0; i < NA; ++i) {
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) s[i] = Metric<M>::merge(s[i], __shfl_xor_sync(0xFFFFFFFFu, s[i], off));
+            for (uint32_t off = L / 2; off > 0; off >>= 1) s[i] = Metric<M>::merge(s[i], __shfl_xor_sync(0xFFFFFFFFu, s[i], off));
         }
-        if (lane == 0) {
+        if (live && l == 0) {
             if (p.raw_sums != nullptr) {
                 // token-sharded verification: hand out the running values; the caller combines the
                 // shards' values and calls the decision kernel
@@ -1353,9 +1496,8 @@ __global__ void __launch_bounds__(kThreads, 2) verify_kernel(const __grid_consta
     __syncthreads();
     // Fused continuation: every decision of this step is final by now. The new mask goes to a buffer
     // of its own: CTAs of this grid may still be reading the step's mask.
-    if (p.sel_active != nullptr)
-        select_in_block(p.accept, p.sel_kmax, p.sel_group, p.batch, p.sel_spec, p.dev_mask, p.sel_active, p.sel_idx, p.sel_n,
-                        sel_keep, sel_next);
+    if (p.sel_active != nullptr && warp == 0)
+        select_in_warp(p.accept, p.sel_kmax, p.sel_group, p.batch, p.sel_spec, p.dev_mask, p.sel_active, p.sel_idx, p.sel_n);
     if (threadIdx.x == 0) *p.ticket = 0;  // ready for the next launch on this stream
 }
 
@@ -1394,15 +1536,11 @@ cudaError_t launch_decide(int metric, const double* sums, int batch, const Decid
 // select / activate: B <= 64 samples, one small CTA
 // ------------------------------------------------------------------------------------------------
 
-__global__ void __launch_bounds__(SPECA_MAX_BATCH) select_kernel(const uint8_t* __restrict__ accept, int32_t k_max,
-                                                                  int32_t group, int32_t batch,
-                                                                  int32_t* __restrict__ spec_count,
-                                                                  uint8_t* __restrict__ active,
-                                                                  int32_t* __restrict__ idx_out,
-                                                                  int32_t* __restrict__ n_out) {
-    __shared__ uint8_t keep[SPECA_MAX_BATCH];
-    __shared__ uint8_t next[SPECA_MAX_BATCH];
-    select_in_block(accept, k_max, group, batch, spec_count, active, active, idx_out, n_out, keep, next);
+__global__ void __launch_bounds__(32) select_kernel(const uint8_t* accept, int32_t k_max, int32_t group, int32_t batch,
+                                                     int32_t* spec_count, uint8_t* active, int32_t* idx_out,
+                                                     int32_t* n_out) {
+    // in place: a lane reads its own samples' mask bytes before the ballots and writes them after
+    select_in_warp(accept, k_max, group, batch, spec_count, active, active, idx_out, n_out);
 }
 
 __global__ void __launch_bounds__(SPECA_MAX_BATCH) activate_kernel(uint64_t mask_bits, int32_t batch,
@@ -1607,8 +1745,8 @@ static void verify_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, in
 cudaError_t launch_verify(const VerifyParams& p, int dtype, int grid, int cluster, cudaStream_t stream) {
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
-    verify_config(&cfg, attr, grid, cluster, stream);
     const int v = max_order(p.order);
+    verify_config(&cfg, attr, grid, cluster, stream);
     const void* fn = dtype == SPECA_BF16 ? verify_kernel_for<SPECA_BF16>(p.metric, v)
                                          : verify_kernel_for<SPECA_F32>(p.metric, v);
     void* args[1] = {const_cast<VerifyParams*>(&p)};
@@ -1635,7 +1773,7 @@ int max_resident_verify_clusters(int dtype, int order, int cluster) {
 
 cudaError_t launch_select(const uint8_t* accept, int32_t k_max, int32_t group, int32_t batch, int32_t* spec_count,
                           uint8_t* active, int32_t* idx, int32_t* n_active, cudaStream_t stream) {
-    select_kernel<<<1, SPECA_MAX_BATCH, 0, stream>>>(accept, k_max, group, batch, spec_count, active, idx, n_active);
+    select_kernel<<<1, 32, 0, stream>>>(accept, k_max, group, batch, spec_count, active, idx, n_active);
     return cudaGetLastError();
 }
 

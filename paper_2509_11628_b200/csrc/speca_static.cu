@@ -2,10 +2,10 @@
 // callers that have no device memory to give the library and cannot allocate any.
 //
 // The verification kernel needs a little global scratch for its cross-CTA reduction (one pair of
-// partial sums per (cluster, sample), an arrival counter) and a descriptor per sample. A cache
-// handle keeps those in the caller's arena. Here they live in one file-scope __device__ array that
-// is part of the loaded library image on every GPU, so the call path contains no cudaMalloc,
-// cudaFree or other allocating routine.
+// partial sums per (cluster, sample), an arrival counter). A cache handle keeps those in
+// the caller's arena. Here they live in one file-scope __device__ array that is part of the loaded
+// library image on every GPU, so the call path contains no cudaMalloc, cudaFree or other allocating
+// routine.
 #include <cuda_runtime.h>
 
 #include <cmath>
@@ -18,10 +18,10 @@ namespace speca {
 namespace {
 
 constexpr int kStaticMaxClusters = SPECA_STATIC_MAX_CLUSTERS;
-constexpr size_t kSegBytes = sizeof(SegDesc) * SPECA_MAX_BATCH;                                   // 2 KB
 constexpr size_t kPartialBytes = sizeof(float) * 2 * SPECA_MAX_BATCH * size_t(kStaticMaxClusters);  // 64 KB
-constexpr size_t kTicketBytes = 256;
-constexpr size_t kScratchBytes = kSegBytes + kPartialBytes + kTicketBytes;
+constexpr size_t kCounterBytes = 512;  // the arrival counter, padded
+constexpr size_t kScratchBytes = kPartialBytes + kCounterBytes;
+static_assert(kVerifyTickets * sizeof(uint32_t) <= kCounterBytes, "the counters fit their slot");
 static_assert(kScratchBytes == SPECA_STATIC_SCRATCH_BYTES, "header and library disagree on the scratch size");
 
 // The scratch itself. In host code this name is only a handle for the runtime's symbol table; the
@@ -29,11 +29,16 @@ static_assert(kScratchBytes == SPECA_STATIC_SCRATCH_BYTES, "header and library d
 static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
 
 constexpr int kMaxDevices = 64;
+constexpr int kCluster = SPECA_VERIFY_CLUSTER;
 std::mutex g_mu;
-unsigned char* g_scratch_addr[kMaxDevices];  // per device, filled on first use
+// per device, filled on the first call there: the scratch array's device address, and how many
+// clusters of the verification kernel are resident at once (per storage type)
+unsigned char* g_scratch_addr[kMaxDevices];
+int g_resident_clusters[kMaxDevices][2];
 
-// Device address of g_static_scratch on `device`, which must be the current device.
-cudaError_t scratch_on_device(int device, unsigned char** out) {
+// Device address of g_static_scratch on `device` and the resident cluster count for `dtype`; `device`
+// must be the current device. Both are looked up once per device (and storage type) and remembered.
+cudaError_t device_setup(int device, int dtype, unsigned char** scratch, int* n_clusters) {
     std::lock_guard<std::mutex> lock(g_mu);
     if (g_scratch_addr[device] == nullptr) {
         void* p = nullptr;
@@ -41,26 +46,20 @@ cudaError_t scratch_on_device(int device, unsigned char** out) {
         if (e != cudaSuccess) return e;
         g_scratch_addr[device] = static_cast<unsigned char*>(p);
     }
-    *out = g_scratch_addr[device];
+    const int k = dtype == SPECA_BF16 ? 1 : 0;
+    if (g_resident_clusters[device][k] == 0) {
+        int n = max_resident_verify_clusters(dtype, 0, kCluster);
+        g_resident_clusters[device][k] = n > kStaticMaxClusters ? kStaticMaxClusters : n;
+    }
+    *scratch = g_scratch_addr[device];
+    *n_clusters = g_resident_clusters[device][k];
     return cudaSuccess;
 }
 
-// Sample b of a dense [B, n_elems] tensor is one "table" with a single plane: its row.
-// Also clears the arrival counter, which must be zero when the verification kernel starts.
-__global__ void __launch_bounds__(SPECA_MAX_BATCH) dense_rows_kernel(SegDesc* segs, uint32_t* ticket, uint32_t n_elems,
-                                                                      uint32_t elem_bytes, int32_t batch) {
-    const int b = threadIdx.x;
-    if (b < batch) {
-        SegDesc s;
-        s.plane0_off = static_cast<uint64_t>(b) * n_elems * elem_bytes;
-        s.plane_stride = 0;
-        s.io_off = s.plane0_off;
-        s.n_elems = n_elems;
-        s.entry = 0;
-        s.sample = static_cast<uint16_t>(b);
-        segs[b] = s;
-    }
-    if (b == 0) *ticket = 0;
+// The arrival counter must be zero when the verification kernel starts. The kernel leaves it at
+// zero itself; this clears whatever an interrupted earlier call may have left.
+__global__ void __launch_bounds__(32) clear_counters_kernel(uint32_t* counters) {
+    if (threadIdx.x < kVerifyTickets) counters[threadIdx.x] = 0;
 }
 
 }  // namespace
@@ -99,23 +98,23 @@ extern "C" speca_status_t speca_verify_pred_static(const void* pred, const void*
 
     speca_status_t st = SPECA_OK;
     do {
-        if (cudaPeekAtLastError() != cudaSuccess) {
+        if (cudaGetLastError() != cudaSuccess) {  // an earlier error on this thread: reported once, not kept
             st = SPECA_ERR_CUDA;
             break;
         }
         unsigned char* scratch = nullptr;
-        if (scratch_on_device(device, &scratch) != cudaSuccess) {
+        int n_clusters = 0;
+        if (device_setup(device, dtype, &scratch, &n_clusters) != cudaSuccess) {
+            (void)cudaGetLastError();  // a failed lookup is not left behind for later calls to trip over
             st = SPECA_ERR_CUDA;
             break;
         }
-        SegDesc* segs = reinterpret_cast<SegDesc*>(scratch);
-        float* partials = reinterpret_cast<float*>(scratch + kSegBytes);
-        uint32_t* ticket = reinterpret_cast<uint32_t*>(scratch + kSegBytes + kPartialBytes);
+        float* partials = reinterpret_cast<float*>(scratch);
+        uint32_t* counters = reinterpret_cast<uint32_t*>(scratch + kPartialBytes);
         cudaStream_t s = static_cast<cudaStream_t>(stream);
 
-        dense_rows_kernel<<<1, SPECA_MAX_BATCH, 0, s>>>(segs, ticket, static_cast<uint32_t>(n_elems),
-                                                         static_cast<uint32_t>(esz), batch);
-        if (cudaGetLastError() != cudaSuccess) {
+        clear_counters_kernel<<<1, 32, 0, s>>>(counters);
+        if (cudaGetLastError() != cudaSuccess) {  // also clears it
             st = SPECA_ERR_CUDA;
             break;
         }
@@ -127,9 +126,12 @@ extern "C" speca_status_t speca_verify_pred_static(const void* pred, const void*
             p.order[b] = 0;  // the "table" is the forecast itself: nothing to extrapolate
             p.tau[b] = tau[b];
         }
-        const int cluster = 4;
         const uint32_t te = verify_tile_elems(dtype, 0);
-        p.segs = segs;
+        // sample b of the dense [B, n_elems] forecast is a one-plane table: its row
+        p.plane0_off = 0;
+        p.sample_pitch = static_cast<uint64_t>(n_elems) * esz;
+        p.plane_stride = 0;
+        p.io_pitch = p.sample_pitch;
         p.arena = const_cast<char*>(static_cast<const char*>(pred));
         p.dev_mask = dev_active_mask;
         p.fresh = static_cast<const char*>(fresh);
@@ -137,18 +139,19 @@ extern "C" speca_status_t speca_verify_pred_static(const void* pred, const void*
         p.err = dev_err;
         p.accept = dev_accept;
         p.partials = partials;
-        p.ticket = ticket;
+        p.ticket = counters;
         p.n_elems = static_cast<uint32_t>(n_elems);
         p.tiles_per_sample = (p.n_elems + te - 1) / te;
-        p.units_per_sample = (p.tiles_per_sample + cluster - 1) / cluster;
+        p.units_per_sample = (p.tiles_per_sample + kCluster - 1) / kCluster;
         p.batch = batch;
         p.eps = eps > 0.f ? static_cast<double>(eps) : 1e-8;
-        int n_clusters = max_resident_verify_clusters(dtype, 0, cluster);
-        if (n_clusters > kStaticMaxClusters) n_clusters = kStaticMaxClusters;
-        int grid = n_clusters * cluster;
+        int grid = n_clusters * kCluster;
         const uint64_t units = static_cast<uint64_t>(p.units_per_sample) * batch;
-        if (units * cluster < static_cast<uint64_t>(grid)) grid = static_cast<int>(units) * cluster;
-        if (launch_verify(p, dtype, grid, cluster, s) != cudaSuccess) st = SPECA_ERR_CUDA;
+        if (units * kCluster < static_cast<uint64_t>(grid)) grid = static_cast<int>(units) * kCluster;
+        if (launch_verify(p, dtype, grid, kCluster, s) != cudaSuccess) {
+            (void)cudaGetLastError();
+            st = SPECA_ERR_CUDA;
+        }
     } while (false);
 
     if (prev != device) cudaSetDevice(prev);

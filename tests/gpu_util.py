@@ -51,6 +51,27 @@ def assert_close_storage(got: np.ndarray, want: np.ndarray, dtype: int, scale: n
         assert rel <= FORECAST_NORM_TOL, "%s: norm-wise error %g" % (what, rel)
 
 
+def assert_equal_or_tie(got: np.ndarray, want: np.ndarray, unrounded: np.ndarray, dtype: int, scale, what: str) -> float:
+    """Where a result is a rounding of a value that sits (within the fp32 evaluation error of its terms,
+    4e-6 of their magnitude `scale`) on the midpoint of two neighbouring storage values, both neighbours
+    are correct roundings. `got` must equal the oracle's `want` bit for bit everywhere else; where it
+    differs it must be the neighbour on the other side of such a midpoint (`unrounded` is the oracle's
+    float64 value before rounding). Returns the share of elements that took the other neighbour."""
+    g, w = as_f64(got), as_f64(want)
+    diff = (got != want) & ~(np.isnan(g) & np.isnan(w))
+    if not diff.any():
+        return 0.0
+    mid = 0.5 * (g[diff] + w[diff])
+    ulp = storage_ulp(w[diff], dtype)
+    sc = np.broadcast_to(np.asarray(scale, dtype=np.float64), g.shape)[diff]
+    adjacent = np.abs(g[diff] - w[diff]) <= 1.0001 * np.maximum(ulp, storage_ulp(g[diff], dtype))
+    near_tie = np.abs(unrounded[diff] - mid) <= 4e-6 * sc + 1e-30
+    bad = ~(adjacent & near_tie)
+    assert not bad.any(), "%s: %d elements differ from the oracle away from a rounding tie; first: got %g want %g unrounded %.17g" % (
+        what, int(bad.sum()), float(g[diff][bad][0]), float(w[diff][bad][0]), float(unrounded[diff][bad][0]))
+    return float(diff.sum()) / got.size
+
+
 def term_scale(planes: np.ndarray, weights) -> np.ndarray:
     """Sum of |plane_i * w_i| per element: magnitude of the terms the forecast adds up."""
     p = as_f64(planes)

@@ -68,40 +68,25 @@ def bits_to_tensor(a, tdt):
     return torch.from_numpy(a)
 
 
-FULL = [
-    ("dit_xl2", {}, 0),
-    ("flux", {}, 0),
-    ("hunyuan_video", {}, 0),
-    ("flux_adaptive", {"max_order": 3}, 0),
-    ("flux", {}, 2),          # the TMA-staged kernels at full size
-    ("dit_xl2", {}, 1),       # the 16-byte register path at full size
-]
-
-
-@pytest.mark.parametrize("name,kw,path", FULL)
-def test_full_size_config_on_sampled_blocks(S, U, name, kw, path):
-    w = W.BY_NAME[name](**kw)
+def reference_steps(U, w, cache, src, blocks, name):
+    """max_order + 1 reference steps, every entry in one launch as the benchmark does. After each, on
+    every element: plane 0 is the feature bit for bit; on the sampled blocks: the tables against the
+    oracle's, then overwritten with the oracle's bits. Returns the oracle's tables per block and the
+    reference times (latest first)."""
     B, m, ne = w.batch, w.max_order, len(w.entries)
-    rng = np.random.default_rng(1234 + w.index)
-    blocks = choose_blocks(w, rng)
-    src = W.FeatureSource(w, DEV)
-    cache = S.SpecaCache(w.entries, B, m, w.dtype, DEV, path=path)
     tdt = w.torch_dtype
+    it = torch.int16 if w.dtype == W.BF16 else torch.int32
     orc = {(e, blk): np.zeros((m + 1, blk[2]), dtype=O.np_dtype(w.dtype)) for e, lst in blocks.items() for blk in lst}
     hist = []
-
     for step in range(m + 1):
         t = [w.times[step]] * B
         feats = [src.feature(e, step, t) for e in range(ne)]
         cache.update(feats, t)           # all entries, one launch: the benchmark's configuration
         cache.commit_step()
         torch.cuda.synchronize()
-        # every element: plane 0 is the feature, bit for bit
         for e in range(ne):
             for b in range(B):
-                n = w.entry_elems(e)
-                assert torch.equal(cache.plane_tensor(e, b)[0].view(torch.int16 if w.dtype == W.BF16 else torch.int32),
-                                   feats[e][b].reshape(-1).view(torch.int16 if w.dtype == W.BF16 else torch.int32)), \
+                assert torch.equal(cache.plane_tensor(e, b)[0].view(it), feats[e][b].reshape(-1).view(it)), \
                     "%s step %d entry %d sample %d: plane 0 differs from the feature" % (name, step, e, b)
         R = 0.0 if not hist else 1.0 / min(abs(t[0] - h) for h in hist)
         for e, lst in blocks.items():
@@ -119,12 +104,41 @@ def test_full_size_config_on_sampled_blocks(S, U, name, kw, path):
         hist = [t[0]] + hist
         del feats
     torch.cuda.synchronize()
+    return orc, hist
+
+
+def taylor_weights(m, x):
+    ws = [1.0]
+    for i in range(1, m + 1):
+        ws.append(ws[-1] * x / i)
+    return ws
+
+
+FULL = [
+    ("dit_xl2", {}, 0),
+    ("flux", {}, 0),
+    ("hunyuan_video", {}, 0),
+    ("flux_adaptive", {"max_order": 3}, 0),
+    ("flux_adaptive", {"max_order": 2}, 0),
+    ("flux_adaptive", {"max_order": 1}, 0),
+    ("flux", {}, 2),          # the TMA-staged kernels at full size
+    ("dit_xl2", {}, 1),       # the 16-byte register path at full size
+]
+
+
+@pytest.mark.parametrize("name,kw,path", FULL)
+def test_full_size_config_on_sampled_blocks(S, U, name, kw, path):
+    w = W.BY_NAME[name](**kw)
+    B, m, ne = w.batch, w.max_order, len(w.entries)
+    rng = np.random.default_rng(1234 + w.index)
+    blocks = choose_blocks(w, rng)
+    src = W.FeatureSource(w, DEV)
+    cache = S.SpecaCache(w.entries, B, m, w.dtype, DEV, path=path)
+    tdt = w.torch_dtype
+    orc, hist = reference_steps(U, w, cache, src, blocks, name)
 
     def weights(x):
-        ws = [1.0]
-        for i in range(1, m + 1):
-            ws.append(ws[-1] * x / i)
-        return ws
+        return taylor_weights(m, x)
 
     # forecast of every entry in one launch, compared on the blocks
     step = m + 1
@@ -199,6 +213,79 @@ def test_full_size_config_on_sampled_blocks(S, U, name, kw, path):
     cache.close()
 
 
+def test_full_size_adaptive_batch_over_a_speculative_run(S, U):
+    """The sample-adaptive configuration (FLUX shape, 8 samples with three noise levels, order 2) at full
+    size over a run of speculative steps k = 1, 2, 3 from the same tables. At every k the oracle's own
+    accept flags decide who stays active: the forecast launch is checked on the sampled blocks (active
+    samples against the oracle, inactive rows untouched), the fused verification on the whole
+    verification entry per active sample, and the continuation rule against the oracle's."""
+    name = "flux_adaptive_m2"
+    w = W.flux_adaptive(max_order=2, batch=8)
+    B, m, ne = w.batch, w.max_order, len(w.entries)
+    rng = np.random.default_rng(977)
+    blocks = choose_blocks(w, rng)
+    src = W.FeatureSource(w, DEV)
+    cache = S.SpecaCache(w.entries, B, m, w.dtype, DEV)
+    tdt = w.torch_dtype
+    it = torch.int16 if w.dtype == W.BF16 else torch.int32
+    orc, hist = reference_steps(U, w, cache, src, blocks, name)
+    outs = [torch.empty(B, n, d, dtype=tdt, device=DEV) for n, d in w.entries]
+    err = torch.zeros(B, dtype=torch.float32, device=DEV)
+    acc = torch.zeros(B, dtype=torch.uint8, device=DEV)
+    active = torch.ones(B, dtype=torch.uint8, device=DEV)
+    nxt = torch.ones(B, dtype=torch.uint8, device=DEV)
+    spec = torch.zeros(B, dtype=torch.int32, device=DEV)
+    act, cnt = [1] * B, [0] * B
+    seven = torch.full((1,), 7.0, dtype=tdt, device=DEV).view(it)
+    seen_inactive = False
+    for k in range(1, 4):
+        step = m + k
+        t_tgt = [w.times[step]] * B
+        tau = [S.speca_tau(w.tau0, w.beta, w.total_steps - step, w.total_steps)] * B
+        for o in outs:
+            o.fill_(7.0)
+        err.fill_(-7.0)
+        acc.fill_(9)
+        fresh = src.feature(w.vidx, step, t_tgt)
+        others = list(outs)
+        others[w.vidx] = None            # as the benchmark's step: the verification launch writes that entry's forecast
+        cache.forecast(t_tgt, others, active)
+        cache.verify_select(fresh, t_tgt, tau, err, acc, active, nxt, 6, 1, spec, out_pred=outs[w.vidx])
+        torch.cuda.synchronize()
+        fresh_np = U.to_oracle(fresh).reshape(B, -1)
+        e_got, a_got = err.cpu().numpy().astype(np.float64), acc.cpu().numpy()
+        flags = [0] * B
+        for e, lst in blocks.items():
+            for blk in lst:
+                b, s, ln = blk
+                got_t = outs[e][b].reshape(-1)[s:s + ln]
+                if not act[b]:
+                    seen_inactive = True
+                    assert bool((got_t.view(it) == seven).all()), "%s k=%d: inactive sample %d of entry %d was written" % (name, k, b, e)
+                    continue
+                want = np.zeros(ln, dtype=O.np_dtype(w.dtype))
+                O.forecast_segment(w.dtype, m, O.TAYLOR, m + 1, hist, t_tgt[b], orc[(e, blk)], want)
+                scale = U.term_scale(orc[(e, blk)], taylor_weights(m, t_tgt[b] - hist[0]))
+                U.assert_close_storage(U.to_oracle(got_t), want, w.dtype, scale, "%s k=%d forecast entry %d block %r" % (name, k, e, blk))
+                if e == w.vidx:
+                    e_want = O.rel_l2(w.dtype, want, fresh_np[b])
+                    assert abs(e_got[b] - e_want) <= U.ERR_TOL * max(1.0, e_want), (name, k, b, e_got[b], e_want)
+                    flags[b] = 1 if O.accept(e_want, float(np.float32(tau[b]))) else 0
+                    if abs(e_want - float(np.float32(tau[b]))) >= U.ERR_TOL:
+                        assert int(a_got[b]) == flags[b], (name, k, b, e_want, tau[b])
+                    else:
+                        flags[b] = int(a_got[b])     # inside the tolerance band either decision is right: follow the library
+        for b in range(B):
+            if not act[b]:
+                assert e_got[b] == -7.0 and a_got[b] == 9, (name, k, b)
+        act, cnt, _ = O.select_adaptive(flags, 6, 1, cnt, act)
+        assert nxt.cpu().tolist() == act and spec.cpu().tolist() == cnt, (name, k)
+        active, nxt = nxt, active
+        del fresh
+    assert seen_inactive and any(act), "the noise levels were chosen so that some samples drop out and some stay: %r" % (act,)
+    cache.close()
+
+
 @pytest.mark.parametrize("name", ["dit_xl2", "flux", "hunyuan_video"])
 def test_full_size_raw_feature_cache_on_sampled_blocks(S, U, name):
     """The same at full size for the cache that keeps raw features: reference steps past the point where
@@ -258,17 +345,33 @@ def test_full_size_raw_feature_cache_on_sampled_blocks(S, U, name):
     tau = [S.speca_tau(w.tau0, w.beta, w.total_steps - step, w.total_steps)] * B
     err = torch.full((B,), -7.0, dtype=torch.float32, device=DEV)
     acc = torch.full((B,), 9, dtype=torch.uint8, device=DEV)
-    cache.verify(fresh, t_tgt, tau, err, acc)
+    pred_gpu = torch.empty_like(fresh)
+    cache.verify(fresh, t_tgt, tau, err, acc, out_pred=pred_gpu)
     torch.cuda.synchronize()
     fresh_np = U.to_oracle(fresh).reshape(B, -1)
+    pred_np = U.to_oracle(pred_gpu).reshape(B, -1)
     for b in range(B):
-        pred, _ = oracle_forecast(w.vidx, (b, 0, w.entry_elems(w.vidx)))
+        blk = (b, 0, w.entry_elems(w.vidx))
+        pred, scale = oracle_forecast(w.vidx, blk)
+        # The forecast of a raw-feature cache is rounded ONCE, from an exact combination of stored values.
+        # On a uniform time grid the weights are ratios of small integers, so a few per cent of the
+        # results sit exactly on a rounding tie of the storage type, where fp32 and fp64 evaluation may
+        # pick different neighbours and both are correct roundings. So: (1) every element of the
+        # library's forecast equals the oracle's, or is the other neighbour of such a tie; (2) Eq. 4 and
+        # the accept rule, by the oracle, ON THAT FORECAST agree with the library's err / accept within
+        # the usual bound -- no widened tolerance anywhere.
+        raw = O.forecast_history_unrounded(w.dtype, m, O.TAYLOR, hist, t_tgt[b], kept[(w.vidx, blk)])
+        share = U.assert_equal_or_tie(pred_np[b], pred, raw, w.dtype, scale, "%s forecast of the verify entry sample %d" % (name, b))
+        assert share < 0.1, (name, b, share)
+        e_on_it = O.rel_l2(w.dtype, np.ascontiguousarray(pred_np[b]), fresh_np[b])
+        assert abs(float(err[b]) - e_on_it) <= U.ERR_TOL * max(1.0, e_on_it), (name, b, float(err[b]), e_on_it)
+        if abs(e_on_it - float(np.float32(tau[b]))) >= U.ERR_TOL:
+            assert int(acc[b]) == (1 if O.accept(e_on_it, float(np.float32(tau[b]))) else 0)
+        # for the record: how far the ties move the error from the oracle's own end-to-end value
         e_want = O.rel_l2(w.dtype, pred, fresh_np[b])
-        # on this uniform time grid the weights are ratios of small integers and a few per cent of the bf16
-        # forecasts are exact ties, which fp32 weights cannot break the way double arithmetic does
-        assert abs(float(err[b]) - e_want) <= U.ERR_TOL * max(1.0, e_want) + 6e-3 * e_want, (name, b, float(err[b]), e_want)
-        if abs(e_want - float(np.float32(tau[b]))) >= U.ERR_TOL + 6e-3 * e_want:
-            assert int(acc[b]) == (1 if O.accept(e_want, float(np.float32(tau[b]))) else 0)
+        print("%s sample %d: %.3f %% of the forecast on the other side of a tie; err %.6f, oracle end to end %.6f (%.2e relative)" % (
+            name, b, 100 * share, float(err[b]), e_want, abs(float(err[b]) - e_want) / max(e_want, 1e-30)))
+        assert abs(float(err[b]) - e_want) <= 2e-2 * max(e_want, 1e-3)     # sanity only; the bound that binds is the one above
     for o in outs:
         o.fill_(5.0)
     cache.forecast([hist[0]] * B, outs)          # k = 0: the newest feature itself

@@ -126,3 +126,25 @@ def test_row_of_almost_2_to_31_elements(S, U):
         U.assert_close_storage(got, want_gpu, 1, scale, "2^31 row forecast block %r" % (blk,))
     assert out.view(-1)[-1].item() != 3.0 and out.view(-1)[0].item() != 3.0
     cache.close()
+
+
+@pytest.mark.parametrize("path", [0, 2])
+def test_health_check_after_a_step(S, path):
+    """speca_cache_check waits for the stream and reports whether a staged copy of the bulk path ever gave
+    up; after an ordinary step on either path it says OK, and it can be asked repeatedly."""
+    entries = [(64, 1024), (33, 520)]
+    B, m = 3, 2
+    cache = S.SpecaCache(entries, B, m, 1, DEV, path=path)
+    gen = torch.Generator(device=DEV).manual_seed(7)
+    side = torch.cuda.Stream(DEV)
+    with torch.cuda.stream(side):
+        for k in range(3):
+            cache.update([torch.randn(B, n, d, generator=gen, device=DEV).bfloat16() for n, d in entries], [1.0 - 0.1 * k] * B,
+                         stream=side)
+            cache.commit_step()
+        outs = [torch.empty(B, n, d, dtype=torch.bfloat16, device=DEV) for n, d in entries]
+        cache.forecast([0.75] * B, outs, stream=side)
+    cache.check(side)
+    cache.check(side)
+    assert all(bool(torch.isfinite(o.float()).all()) for o in outs)   # the check has waited for the forecast
+    cache.close()

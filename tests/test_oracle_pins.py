@@ -10,6 +10,8 @@ import os
 from fractions import Fraction
 from math import comb, factorial
 
+import ctypes
+
 import numpy as np
 import pytest
 import torch
@@ -905,3 +907,26 @@ def test_history_layout_cache_masks_resets_and_zero_gap():
     out = c.forecast_entry(0, [1.0] * B, active=[1, 1, 0], out=np.full((B, n), 7.0, dtype=np.float32))
     assert np.array_equal(out[0], fs[2][0]) and np.all(out[2] == 7.0)
     assert np.array_equal(out[1], fs[2][1] + (fs[2][1] - fs[0][1]) / (2.0 - 4.0) * (1.0 - 2.0))   # its references: t = 4 and t = 2
+
+
+def test_unrounded_history_forecast_rounds_to_the_stored_one():
+    """forecast_history_unrounded is the value oracle_forecast_history_segment rounds: rounding it (double ->
+    binary32 -> storage, as the oracle's store does) must give that function's output bit for bit, and for
+    order 1 on two hand-picked features it is the straight line through them."""
+    rng = np.random.default_rng(5)
+    for dtype in (O.F32, O.BF16):
+        for m in (1, 2, 3):
+            t_hist = [0.7, 0.8, 0.95, 1.0][: m + 1]
+            if dtype == O.F32:
+                hist = [rng.standard_normal(257).astype(np.float32) for _ in range(m + 1)]
+            else:
+                hist = [(rng.standard_normal(257).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16) for _ in range(m + 1)]
+            raw = O.forecast_history_unrounded(dtype, m, O.TAYLOR, t_hist, 0.64, hist)
+            want = np.zeros(257, dtype=O.np_dtype(dtype))
+            O.forecast_history_segment(dtype, m, O.TAYLOR, t_hist, 0.64, hist, want)
+            got = np.zeros(257, dtype=O.np_dtype(dtype))
+            O.lib().oracle_round_store(dtype, 257, raw.ctypes.data_as(ctypes.c_void_p), got.ctypes.data_as(ctypes.c_void_p))
+            assert np.array_equal(got, want)
+    a, b = np.array([3.0], dtype=np.float32), np.array([1.0], dtype=np.float32)   # f(0.5) = 3, f(1.0) = 1: slope -4
+    raw = O.forecast_history_unrounded(O.F32, 1, O.TAYLOR, [0.5, 1.0], 0.25, [a, b])
+    assert raw[0] == pytest.approx(4.0, abs=1e-12)
