@@ -1030,28 +1030,28 @@ struct Metric {
         else
             return x + y;
     }
-    // The error from the totals. err is handed out as a binary32, so the square roots and the division
-    // are binary32 too (a few ulp of the stored value; fp64 square roots and divisions are long dependent
-    // instruction sequences on the kernel's critical tail) and the accept flag is exactly err <= tau on
-    // the stored values. Totals outside the binary32 range (or NaN) take the fp64 formulas.
+    // The error from the totals. err is handed out as a binary32, so for the ratio metrics the square
+    // roots and the division are binary32 too (a few ulp of the stored value; fp64 square roots and
+    // divisions are long dependent instruction sequences on the kernel's critical tail) and the accept
+    // flag is exactly err <= tau on the stored values. Totals outside the binary32 range (or NaN) take
+    // the fp64 formulas, and so does the cosine distance, whose 1 - ratio cancels.
     __device__ static __forceinline__ double error(const double (&s)[3], double eps) {
-        const bool fits = fabs(s[0]) < 1e38 && fabs(s[1]) < 1e38 && (NA < 3 || fabs(s[2]) < 1e38);
-        if (fits) {
-            const float a0 = static_cast<float>(s[0]), a1 = static_cast<float>(s[1]), a2 = static_cast<float>(s[2]);
-            const float e = static_cast<float>(eps);
-            if constexpr (M == SPECA_METRIC_L2)
-                return static_cast<double>(sqrtf(a0) / (sqrtf(a1) + e));
-            else if constexpr (M == SPECA_METRIC_COSINE)
-                return static_cast<double>(1.0f - a0 / (sqrtf(a1) * sqrtf(a2) + e));
-            else
-                return static_cast<double>(a0 / (a1 + e));
-        }
-        if constexpr (M == SPECA_METRIC_L2)
-            return sqrt(s[0]) / (sqrt(s[1]) + eps);
-        else if constexpr (M == SPECA_METRIC_COSINE)
+        if constexpr (M == SPECA_METRIC_COSINE) {
             return 1.0 - s[0] / (sqrt(s[1]) * sqrt(s[2]) + eps);
-        else
-            return s[0] / (s[1] + eps);
+        } else {
+            const bool fits = fabs(s[0]) < 1e38 && fabs(s[1]) < 1e38;
+            if (fits) {
+                const float a0 = static_cast<float>(s[0]), a1 = static_cast<float>(s[1]), e = static_cast<float>(eps);
+                if constexpr (M == SPECA_METRIC_L2)
+                    return static_cast<double>(sqrtf(a0) / (sqrtf(a1) + e));
+                else
+                    return static_cast<double>(a0 / (a1 + e));
+            }
+            if constexpr (M == SPECA_METRIC_L2)
+                return sqrt(s[0]) / (sqrt(s[1]) + eps);
+            else
+                return s[0] / (s[1] + eps);
+        }
     }
 };
 

@@ -29,7 +29,7 @@ def _canned_line(n_gpus=1):
            "sample": "1 step, all 76 entries of flux_dev_1024: update+forecast+verify+select on the workload's seeded features",
            "s_per_step": 4.123456789, "value_1_thread_verify_entry_only": 0.3123456}
     e2e = {"value": 463.123456, "unit": "GB/s", "h2d_bytes_per_step": 1642070016, "d2h_bytes_per_step": 1613758470,
-           "ms_per_step": 35.0123456, "h2d_gbs": 46.9, "d2h_gbs": 46.1}
+           "ms_per_step": 35.0123456, "h2d_gbs": 46.9, "d2h_gbs": 46.1, "pcie_gbs_one_direction_alone": [55.4, 54.7]}
     clocks = {"sm_mhz": 1905, "sm_max_mhz": 1965, "reasons": ["sw_power_cap"]}
     also = {"dit_xl2": [5630.778151259666, 6338.307730945065, 2945.751117193706],
             "hunyuan_video": [6699.123456789, 6901.123456, 190.123456]}
@@ -64,11 +64,18 @@ def test_line_is_compact_and_carries_the_contract_keys():
     assert set(line["also_value_fv_gbs_steps_per_s"]) == {"dit_xl2", "hunyuan_video"}
 
 
-def test_line_refuses_to_grow_past_the_limit():
-    with pytest.raises(ValueError):
-        bench.build_line(value=1.0, ms_per_step=1.0, n_gpus=1, steps=1, warmup=3, config={"workload": "x" * 2100},
-                         roofline=None, cpu_baseline=None, e2e=None, gpu_launches=1, clocks=None,
-                         kernels={}, forecast_verify_gbs=1.0, speculative_steps_per_s=1.0)
+def test_line_sheds_its_extras_before_it_grows_past_the_limit():
+    k = {"ms": 1.0, "gbs": 1.0, "algorithmic_bytes": 1}
+    common = dict(value=1.0, ms_per_step=1.0, n_gpus=1, steps=1, warmup=3, roofline=None, cpu_baseline=None, e2e=None,
+                  gpu_launches=1, clocks=None, kernels={"update": k, "forecast": k, "verify": k},
+                  forecast_verify_gbs=1.0, speculative_steps_per_s=1.0, detail_path="d.json")
+    long_also = {"config_%d" % i: [1.0, 2.0, 3.0] for i in range(60)}
+    line = json.loads(bench.build_line(config={"workload": "w"}, also=long_also, **common))
+    assert "also_value_fv_gbs_steps_per_s" not in line and "kernels_ms_gbs" in line      # the extras go first
+    for key in REQUIRED:
+        assert key in line
+    with pytest.raises(ValueError):     # the contract keys alone do not fit: nothing sensible can be printed
+        bench.build_line(config={"workload": "x" * 2100}, **common)
 
 
 def test_step_bytes_follow_the_per_element_figures():
