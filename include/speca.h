@@ -112,8 +112,9 @@ typedef enum {
  *          then ratios of small integers) a few per cent of the elements land exactly on a rounding tie,
  *          where an fp64 evaluation may pick the other neighbour; both are correct. The verification error
  *          computed on the library's forecast meets the 1e-4 bound; against an fp64 evaluation of the
- *          whole chain it can differ by up to 6e-3 of itself on such grids (measured: 1e-3 to 4e-3), and
- *          by no more than the TABLES layout does on uneven grids.
+ *          whole chain it can differ by up to 6e-3 of itself on such grids when the forecast offsets make
+ *          the weights inexact in fp32 (with integer weights, and on uneven grids, the difference stays
+ *          far below 1e-4).
  */
 typedef enum {
     SPECA_LAYOUT_TABLES = 0,
