@@ -302,6 +302,52 @@ def time_multi_horizon(h: Harness, peak: float, forecast_ms: float, K: int = 4, 
             "speedup_vs_single_forecasts": K * forecast_ms / ms}
 
 
+def time_graph_replay(h: Harness, K: int = 4, reps: int = 20):
+    """K consecutive speculative steps (forecast of every other entry + verification / continuation) issued
+    call by call, against the same K steps captured once into a CUDA graph and replayed: the calls neither
+    allocate nor synchronise, and the masks chain on the device, so a whole speculative run needs no host
+    round trip. The threshold is set so that every sample stays active (constant work per step)."""
+    w, dev = h.w, h.device
+    others = list(h.outs)
+    others[w.vidx] = None
+    tau = [1e30] * h.B
+    masks = [torch.ones(h.B, dtype=torch.uint8, device=dev) for _ in range(2)]
+    t0 = h.t_base - 0.02 * (h.j + 1)
+    targets = [[t0 - 0.004 * (k + 1)] * h.B for k in range(K)]
+
+    def run():
+        for k in range(K):
+            h.cache.forecast(targets[k], others, masks[k & 1])
+            h.cache.verify_select(h.fresh[k & 1], targets[k], tau, h.err, h.accept, masks[k & 1], masks[(k + 1) & 1], 1 << 30, 1,
+                                  h.spec, h.idx, h.n_active, out_pred=h.outs[w.vidx])
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize(dev)
+        return e0.elapsed_time(e1) / reps / K
+
+    eager_ms = timed(run)
+    side = torch.cuda.Stream(dev)
+    side.wait_stream(torch.cuda.current_stream(dev))
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        run()                                   # the capture must not be the first use of anything
+        torch.cuda.synchronize(dev)
+        with torch.cuda.graph(graph, stream=side):
+            run()
+    torch.cuda.current_stream(dev).wait_stream(side)
+    graph_ms = timed(graph.replay)
+    return {"steps_per_graph": K, "eager_ms_per_step": eager_ms, "graph_ms_per_step": graph_ms,
+            "eager_steps_per_s": 1e3 / eager_ms, "graph_steps_per_s": 1e3 / graph_ms}
+
+
 def time_update_per_entry(h: Harness, reps: int = 5):
     """A model hands over one block output at a time: the same reference step as one launch per entry."""
     w, dev = h.w, h.device
@@ -1062,6 +1108,10 @@ def main(argv=None):
         detail["verify_metrics"] = time_metrics(h)
     if args.full and tables:
         detail["multi_horizon"] = time_multi_horizon(h, peak, per_ms["forecast"])
+        try:
+            detail["speculative_run_as_cuda_graph"] = time_graph_replay(h)
+        except Exception as exc:  # report, do not hide
+            detail["speculative_run_as_cuda_graph"] = {"error": repr(exc)}
         detail["update_one_launch_per_entry"] = time_update_per_entry(h)
         detail["forecast_sum"] = time_forecast_sum(h, peak)
 
@@ -1107,6 +1157,10 @@ def main(argv=None):
                                     "config": workload_config(w2), "kernels": kern2, **ex2}
                 also[name] = [v2, ex2["forecast_verify_gbs"], ex2["speculative_steps_per_s"]]
                 if args.full:
+                    try:
+                        per_config[name]["speculative_run_as_cuda_graph"] = time_graph_replay(h2)
+                    except Exception as exc:  # report, do not hide
+                        per_config[name]["speculative_run_as_cuda_graph"] = {"error": repr(exc)}
                     per_config[name].update(multi_horizon=time_multi_horizon(h2, peak, p2["forecast"]),
                                             update_one_launch_per_entry=time_update_per_entry(h2),
                                             forecast_sum=time_forecast_sum(h2, peak))
@@ -1153,7 +1207,7 @@ def main(argv=None):
                 "frac_of_nominal_8TBs": dom["gbs"] / NOMINAL_HBM_GBS}
 
     cpu_baseline = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and solo:      # timed on rank 0 of a one-GPU run only
         res = oracle_config_run(w, 1, 60.0, device)
         dt = res["secs"][0]
         cpu_baseline = {"value": res["bytes_per_step"] / dt / 1e9, "unit": "GB/s", "cores": res["threads"], "kind": "oracle",
