@@ -224,6 +224,35 @@ speca_status_t speca_cache_update_activate(speca_cache_t* cache, const void* con
                                            uint8_t* dev_active_mask, void* stream);
 
 /*
+ * A whole reference step and the first speculative step after it in ONE pass over the tables
+ * (Section 3.2, workflow steps 1 and 2; Eq. 3 followed by Eq. 2): exactly
+ *     speca_cache_update(_activate)(feats, t_ref, host_sample_mask);  speca_cache_commit_step();
+ *     speca_forecast(t_target, dev_active_mask, outs);
+ * bit for bit, but the forecast of a sample that takes the reference step is evaluated from the planes
+ * the update has just formed (rounded to the storage dtype, as a forecast launch would read them), so
+ * the table is not read again: 2v + 3 words per element instead of (2v + 2) + (v + 2). A reference
+ * step is always followed by a speculative one, so this is the normal way to take it.
+ *   feats            every entry's feature (no NULLs: the call is the whole step and commits it).
+ *   t_ref, host_sample_mask   as in speca_cache_update.
+ *   t_target         host, B doubles: the speculative time to forecast, per sample.
+ *   dev_active_mask  device, B bytes, NULL = all: consulted only for samples that do NOT take this
+ *                    reference step (they are forecast from their unchanged tables if non-zero);
+ *                    samples that take it are always forecast. The kernel does not write it.
+ *   outs             per entry: forecast output, or NULL for an entry that is only updated (the
+ *                    verification entry, whose forecast comes out of speca_verify's out_pred).
+ *   dev_spec_count, dev_rearm_mask   both or neither: as speca_cache_update_activate, the samples
+ *                    of host_sample_mask are marked active in dev_rearm_mask and their counters
+ *                    cleared (dev_rearm_mask may be the buffer dev_active_mask names).
+ * Difference-table caches (SPECA_LAYOUT_TABLES) on the default kernel path only. On error nothing is
+ * enqueued and the history is unchanged. Errors: INVALID_ARG, ALIGNMENT, ZERO_GAP, STATE (a reference
+ * step is open; or a sample has no reference and no device mask is given), UNSUPPORTED, CUDA.
+ */
+speca_status_t speca_cache_update_forecast(speca_cache_t* cache, const void* const* feats, const double* t_ref,
+                                           const uint8_t* host_sample_mask, const double* t_target,
+                                           const uint8_t* dev_active_mask, void* const* outs, int32_t* dev_spec_count,
+                                           uint8_t* dev_rearm_mask, void* stream);
+
+/*
  * Close a reference step: push t_ref into each masked sample's reference history and raise its
  * reference count. Host state only. Errors: STATE if some entry has not been updated for
  * exactly the masked samples since the last commit, or no update is pending.
@@ -468,7 +497,8 @@ speca_status_t speca_cache_next_slot(const speca_cache_t* cache, int32_t entry, 
 /*
  * Host-side counters of a handle since it was created (nothing here is read back from the device, so
  * the call neither launches nor synchronises). Launch counts are per kernel kind; the fused
- * verify + continuation call counts as one verify launch. reference_steps[b] counts committed
+ * verify + continuation call counts as one verify launch, the fused reference step
+ * (speca_cache_update_forecast) has a count of its own. reference_steps[b] counts committed
  * reference steps of sample b (it does not go back to zero on a reset, unlike the history length
  * that speca_cache_state reports); resets[b] counts how often sample b's history was cleared.
  * Entries at and beyond the batch size are zero. reference_steps is the number of full passes each
@@ -476,7 +506,7 @@ speca_status_t speca_cache_next_slot(const speca_cache_t* cache, int32_t entry, 
  */
 typedef struct {
     uint64_t update_launches, forecast_launches, forecast_multi_launches, forecast_sum_launches;
-    uint64_t verify_launches, select_launches, activate_launches;
+    uint64_t verify_launches, select_launches, activate_launches, update_forecast_launches;
     uint64_t reference_steps[SPECA_MAX_BATCH];
     uint64_t resets[SPECA_MAX_BATCH];
 } speca_cache_stats_t;

@@ -29,7 +29,7 @@ SPECA_MAX_ORDER, SPECA_MAX_BATCH, SPECA_MAX_ENTRIES, SPECA_MAX_HORIZON = 4, 64, 
 
 EXPORTS = [
     "speca_cache_arena_bytes", "speca_cache_create", "speca_cache_destroy", "speca_cache_reset",
-    "speca_cache_update", "speca_cache_update_activate", "speca_cache_commit_step", "speca_forecast", "speca_verify",
+    "speca_cache_update", "speca_cache_update_activate", "speca_cache_update_forecast", "speca_cache_commit_step", "speca_forecast", "speca_verify",
     "speca_select_adaptive", "speca_activate", "speca_tau", "speca_cache_state", "speca_cache_plane",
     "speca_cache_launch_count", "speca_cache_stats", "speca_cache_check", "speca_cache_next_slot", "speca_forecast_weights", "speca_status_string", "speca_last_error", "speca_version",
     "speca_verify_pred_static", "speca_forecast_multi", "speca_verify_metric",
@@ -52,7 +52,7 @@ class EntryDesc(ctypes.Structure):
 class CacheStats(ctypes.Structure):
     _fields_ = [(name, ctypes.c_uint64) for name in (
         "update_launches", "forecast_launches", "forecast_multi_launches", "forecast_sum_launches",
-        "verify_launches", "select_launches", "activate_launches")] + [
+        "verify_launches", "select_launches", "activate_launches", "update_forecast_launches")] + [
         ("reference_steps", ctypes.c_uint64 * 64), ("resets", ctypes.c_uint64 * 64)]
 
 
@@ -86,6 +86,7 @@ def _lib() -> ctypes.CDLL:
     L.speca_cache_reset.argtypes = [vp, vp]
     L.speca_cache_update.argtypes = [vp, vp, vp, vp, vp]
     L.speca_cache_update_activate.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    L.speca_cache_update_forecast.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.speca_cache_commit_step.argtypes = [vp]
     L.speca_forecast.argtypes = [vp, vp, vp, vp, vp]
     L.speca_forecast_sum.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]
@@ -222,6 +223,14 @@ def speca_cache_update_activate(cache, feats, t_ref, host_sample_mask, dev_spec_
                                               _dev_ptr(dev_spec_count), _dev_ptr(dev_active_mask), _stream_ptr(stream)), cache)
 
 
+def speca_cache_update_forecast(cache, feats, t_ref, host_sample_mask, t_target, dev_active_mask, outs, dev_spec_count=None,
+                                dev_rearm_mask=None, stream=None) -> None:
+    """A whole reference step (update + commit) and the forecast at t_target in one launch."""
+    _check(_lib().speca_cache_update_forecast(cache, _ptr_array(feats), _doubles(t_ref), _bytes(host_sample_mask),
+                                              _doubles(t_target), _dev_ptr(dev_active_mask), _ptr_array(outs),
+                                              _dev_ptr(dev_spec_count), _dev_ptr(dev_rearm_mask), _stream_ptr(stream)), cache)
+
+
 def speca_cache_commit_step(cache) -> None:
     _check(_lib().speca_cache_commit_step(cache), cache)
 
@@ -356,7 +365,7 @@ def speca_cache_stats(cache, batch: int) -> dict:
     """Host-side counters of the handle: launches per kernel kind, reference steps and resets per sample."""
     st = CacheStats()
     _check(_lib().speca_cache_stats(cache, ctypes.byref(st)), cache)
-    out = {name: int(getattr(st, name)) for name, _ in CacheStats._fields_[:7]}
+    out = {name: int(getattr(st, name)) for name, _ in CacheStats._fields_[:8]}
     out["reference_steps"] = [int(x) for x in st.reference_steps[:batch]]
     out["resets"] = [int(x) for x in st.resets[:batch]]
     return out
@@ -416,6 +425,10 @@ class SpecaCache:
 
     def update_activate(self, feats, t_ref, mask, spec_count, active, stream=None):
         speca_cache_update_activate(self.handle, feats, t_ref, mask, spec_count, active, stream)
+
+    def update_forecast(self, feats, t_ref, t_target, outs, mask=None, active=None, spec_count=None, rearm=None, stream=None):
+        """A whole reference step and the first forecast after it in one launch (commits the step)."""
+        speca_cache_update_forecast(self.handle, feats, t_ref, mask, t_target, active, outs, spec_count, rearm, stream)
 
     def commit_step(self):
         speca_cache_commit_step(self.handle)

@@ -537,6 +537,127 @@ speca_status_t speca_cache_update_activate(speca_cache_t* c, const void* const* 
     return update_impl(c, feats, t_ref, host_sample_mask, stream, dev_spec_count, dev_active_mask);
 }
 
+speca_status_t speca_cache_update_forecast(speca_cache_t* c, const void* const* feats, const double* t_ref,
+                                           const uint8_t* host_sample_mask, const double* t_target,
+                                           const uint8_t* dev_active_mask, void* const* outs, int32_t* dev_spec_count,
+                                           uint8_t* dev_rearm_mask, void* stream) {
+    if (c == nullptr) return SPECA_ERR_INVALID_ARG;
+    if (feats == nullptr || t_ref == nullptr || t_target == nullptr || outs == nullptr)
+        return fail(c, SPECA_ERR_INVALID_ARG, "update_forecast: null argument");
+    if ((dev_spec_count == nullptr) != (dev_rearm_mask == nullptr))
+        return fail(c, SPECA_ERR_INVALID_ARG, "update_forecast: give both re-arming buffers or neither");
+    if (reinterpret_cast<uintptr_t>(dev_spec_count) % 4 != 0)
+        return fail(c, SPECA_ERR_ALIGNMENT, "update_forecast: dev_spec_count must be 4-byte aligned");
+    if (c->layout != SPECA_LAYOUT_TABLES || c->path != SPECA_PATH_WIDE)
+        return fail(c, SPECA_ERR_UNSUPPORTED, "update_forecast: difference-table caches on the default kernel path only");
+    if (c->pending) return fail(c, SPECA_ERR_STATE, "update_forecast: a reference step is open (commit it first)");
+    uint8_t mask[SPECA_MAX_BATCH];
+    bool any_sample = false;
+    for (int b = 0; b < c->B; ++b) {
+        mask[b] = (host_sample_mask == nullptr || host_sample_mask[b] != 0) ? 1 : 0;
+        any_sample |= mask[b] != 0;
+        if (mask[b] && !std::isfinite(t_ref[b])) return fail(c, SPECA_ERR_INVALID_ARG, "update_forecast: t_ref[%d] not finite", b);
+        if (!std::isfinite(t_target[b])) return fail(c, SPECA_ERR_INVALID_ARG, "update_forecast: t_target[%d] not finite", b);
+    }
+    static thread_local FusedParams q;  // 10 KB: kept off the stack
+    std::memset(&q, 0, sizeof q);
+    StreamParams& p = q.up;
+    uint64_t bits = 0;
+    for (int b = 0; b < c->B; ++b) {  // scalars of Eq. 3, as in speca_cache_update
+        p.order[b] = -1;
+        if (!mask[b]) continue;
+        bits |= uint64_t(1) << b;
+        const int v_new = c->n_refs[b] < c->m ? c->n_refs[b] : c->m;
+        for (int i = 0; i < v_new; ++i) {
+            const double gap = t_ref[b] - (c->basis == SPECA_BASIS_NEWTON ? c->t_hist[b][i] : c->t_hist[b][0]);
+            if (gap == 0.0) return fail(c, SPECA_ERR_ZERO_GAP, "update_forecast: sample %d repeats a reference time", b);
+            p.coef[b][i] = static_cast<float>(1.0 / gap);
+        }
+        p.order[b] = static_cast<int8_t>(v_new);
+    }
+    const size_t esz = elem_size(c);
+    bool any_out = false;
+    for (int e = 0; e < c->n_entries; ++e) {
+        if (feats[e] == nullptr) return fail(c, SPECA_ERR_INVALID_ARG, "update_forecast: feats[%d] is null (the call is a whole reference step)", e);
+        if (reinterpret_cast<uintptr_t>(feats[e]) % esz != 0 || reinterpret_cast<uintptr_t>(outs[e]) % esz != 0)
+            return fail(c, SPECA_ERR_ALIGNMENT, "update_forecast: feats[%d] / outs[%d] not aligned to the element size", e, e);
+        p.io[e] = const_cast<void*>(feats[e]);
+        q.out[e] = outs[e];
+        any_out |= outs[e] != nullptr;
+    }
+    // The forecast's scalars are those of the history AFTER this step: commit on a copy of the host
+    // state, keep the copy if anything below fails.
+    int32_t saved_refs[SPECA_MAX_BATCH];
+    double saved_hist[SPECA_MAX_BATCH][SPECA_MAX_ORDER + 1];
+    std::memcpy(saved_refs, c->n_refs, sizeof saved_refs);
+    std::memcpy(saved_hist, c->t_hist, sizeof saved_hist);
+    auto roll_back = [&]() {
+        std::memcpy(c->n_refs, saved_refs, sizeof saved_refs);
+        std::memcpy(c->t_hist, saved_hist, sizeof saved_hist);
+    };
+    for (int b = 0; b < c->B; ++b) {
+        if (!mask[b]) continue;
+        for (int i = SPECA_MAX_ORDER; i >= 1; --i) c->t_hist[b][i] = c->t_hist[b][i - 1];
+        c->t_hist[b][0] = t_ref[b];
+        c->n_refs[b] += 1;
+    }
+    bool any_forecast = false;
+    for (int b = 0; b < c->B; ++b) {
+        int order;
+        forecast_scalars(c, b, t_target[b], &order, q.fc_coef[b]);
+        if (order < 0 && dev_active_mask == nullptr && any_out) {
+            roll_back();
+            return fail(c, SPECA_ERR_STATE, "update_forecast: sample %d has no reference, in this step or before", b);
+        }
+        q.fc_order[b] = static_cast<int8_t>(order);
+        any_forecast |= order >= 0;
+    }
+    q.fc_mask = dev_active_mask;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) {
+        roll_back();
+        return fail(c, SPECA_ERR_CUDA, "cudaSetDevice failed");
+    }
+    speca_status_t st = check_sticky(c);
+    if (st != SPECA_OK) {
+        roll_back();
+        return st;
+    }
+    if (any_sample || (any_forecast && any_out)) {
+        const Layout& L = c->L;
+        const std::vector<uint32_t>& tiles = L.tiles[c->tile_update];
+        p.segs = reinterpret_cast<const SegDesc*>(c->arena + L.segs_off);
+        p.tile_start = reinterpret_cast<const uint32_t*>(c->arena + L.tiles_off[c->tile_update]);
+        p.arena = c->arena;
+        p.err_flag = reinterpret_cast<uint32_t*>(c->arena + L.ticket_off) + kGaveUpWord;
+        p.seg_lo = 0;
+        p.seg_hi = static_cast<uint32_t>(c->n_entries) * c->B;
+        p.tile_lo = tiles[p.seg_lo];
+        p.tile_hi = tiles[p.seg_hi];
+        if (dev_rearm_mask != nullptr && any_sample) {  // the kernel's first CTA re-arms the updated samples
+            p.act_spec = dev_spec_count;
+            p.act_active = dev_rearm_mask;
+            p.act_bits = bits;
+        }
+        int v = launch_order(p.order, c->B);
+        const int vf = launch_order(q.fc_order, c->B);
+        v = vf > v ? vf : v;
+        const uint32_t n_tiles = p.tile_hi - p.tile_lo;
+        const uint32_t full = static_cast<uint32_t>(c->sm_count * fused_ctas_per_sm(v));
+        const int grid = static_cast<int>(n_tiles < full ? n_tiles : full);
+        cudaError_t ce = launch_update_forecast(q, c->dtype, grid, static_cast<cudaStream_t>(stream));
+        if (ce != cudaSuccess) {
+            roll_back();
+            return cuda_fail(c, ce, "update_forecast launch");
+        }
+        c->launches += 1;
+        c->stats.update_forecast_launches += 1;
+    }
+    for (int b = 0; b < c->B; ++b)
+        if (mask[b]) c->stats.reference_steps[b] += 1;
+    return SPECA_OK;
+}
+
 speca_status_t speca_cache_commit_step(speca_cache_t* c) {
     if (c == nullptr) return SPECA_ERR_INVALID_ARG;
     if (!c->pending) return fail(c, SPECA_ERR_STATE, "commit: no reference step is open");

@@ -81,6 +81,17 @@ struct StreamParams {
     void* io[SPECA_MAX_ENTRIES];  // per entry: feature (update) or output (forecast); null = skip
 };
 
+// Arguments of the fused reference step: Eq. 3 for the samples that were fully computed and, in the
+// same pass over the tables, Eq. 2 at the next speculative time for them (from the planes just
+// written) and for the samples that keep speculating (from their unchanged planes).
+struct FusedParams {
+    StreamParams up;                  // the update half: io = features, order / coef as for an update
+    const uint8_t* fc_mask;           // device, per sample, may be null: consulted for samples NOT updated here
+    int8_t fc_order[SPECA_MAX_BATCH]; // order of the forecast after this step (-1: nothing to forecast)
+    float fc_coef[SPECA_MAX_BATCH][kCoef];  // Horner multipliers relative to the history after this step
+    void* out[SPECA_MAX_ENTRIES];     // per entry: forecast output; null = update only
+};
+
 // Arguments of the multi-horizon forecast: K targets evaluated from one read of the table.
 struct MultiParams {
     const SegDesc* segs;
@@ -154,6 +165,8 @@ struct DecideParams {
 // Launchers. `dtype` is a speca_dtype_t. All enqueue on `stream` and return the launch status.
 cudaError_t launch_update(const StreamParams& p, int dtype, int path, int grid, cudaStream_t stream);
 cudaError_t launch_forecast(const StreamParams& p, int dtype, int path, int grid, cudaStream_t stream);
+cudaError_t launch_update_forecast(const FusedParams& p, int dtype, int grid, cudaStream_t stream);
+int fused_ctas_per_sm(int order);
 cudaError_t launch_verify(const VerifyParams& p, int dtype, int grid, int cluster, cudaStream_t stream);
 cudaError_t launch_select(const uint8_t* accept, int32_t k_max, int32_t group, int32_t batch, int32_t* spec_count,
                           uint8_t* active, int32_t* idx, int32_t* n_active, cudaStream_t stream);

@@ -344,6 +344,85 @@ __device__ __forceinline__ void update_tile(char* __restrict__ plane0, uint64_t 
     }
 }
 
+// Eq. 3 and, from the planes it has just formed, Eq. 2 at the next speculative time: the reference step
+// that is followed by a speculative one (it always is) hands over its first forecast without reading the
+// table again. Reads f and planes 0..V-1, writes planes 0..V and the forecast: 2V + 3 words per element
+// instead of (2V + 2) + (V + 2). The forecast is evaluated from the ROUNDED planes, exactly as a
+// forecast launch would find them in memory, so the result is bit for bit that of the two calls.
+template <int DT, int V, int W, int NT, int U>
+__device__ __forceinline__ void update_forecast_tile(char* __restrict__ plane0, uint64_t stride,
+                                                     const char* __restrict__ feat, char* __restrict__ out, uint32_t cnt,
+                                                     const float (&r)[kCoef], const float (&mu)[kCoef]) {
+    constexpr int EPV = W / Elem<DT>::kBytes;
+    const uint32_t nvec = cnt / EPV;
+    Vec<W> fv[U];
+    Vec<W> d[V > 0 ? V : 1][U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint32_t idx = u * NT + threadIdx.x;
+        if (idx < nvec) {
+            fv[u] = load_vec<W>(feat + static_cast<size_t>(idx) * W);
+#pragma unroll
+            for (int i = 0; i < V; ++i) d[i][u] = load_vec<W>(plane0 + i * stride + static_cast<size_t>(idx) * W);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint32_t idx = u * NT + threadIdx.x;
+        if (idx < nvec) {
+            float c[EPV];
+            unpack_vec<DT, W>(fv[u], c);
+#pragma unroll
+            for (int i = 0; i < V; ++i) {
+                float old[EPV];
+                unpack_vec<DT, W>(d[i][u], old);
+#pragma unroll
+                for (int k = 0; k < EPV; ++k) c[k] = (c[k] - old[k]) * r[i];
+                d[i][u] = pack_vec<DT, W>(c);  // plane i + 1, rounded
+            }
+            store_vec<W>(plane0 + static_cast<size_t>(idx) * W, fv[u]);
+#pragma unroll
+            for (int i = 0; i < V; ++i)
+                store_vec<W>(plane0 + (i + 1) * stride + static_cast<size_t>(idx) * W, d[i][u]);
+            // Horner over the stored values: acc = D_V; acc = D_{i-1} + acc * mu_i
+            float acc[EPV];
+            if constexpr (V > 0)
+                unpack_vec<DT, W>(d[V - 1][u], acc);
+            else
+                unpack_vec<DT, W>(fv[u], acc);
+#pragma unroll
+            for (int i = V; i >= 1; --i) {
+                float lo[EPV];
+                if (i == 1)
+                    unpack_vec<DT, W>(fv[u], lo);
+                else
+                    unpack_vec<DT, W>(d[i - 2 >= 0 ? i - 2 : 0][u], lo);
+#pragma unroll
+                for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+            }
+            store_vec<W>(out + static_cast<size_t>(idx) * W, pack_vec<DT, W>(acc));
+        }
+    }
+    for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += NT) {
+        float c = load_scalar<DT>(feat, j);
+        float old[V > 0 ? V : 1], neu[V + 1];
+#pragma unroll
+        for (int i = 0; i < V; ++i) old[i] = load_scalar<DT>(plane0 + i * stride, j);
+        neu[0] = c;  // already a storage value
+        store_scalar<DT>(plane0, j, c);
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            c = (c - old[i]) * r[i];
+            store_scalar<DT>(plane0 + (i + 1) * stride, j, c);
+            neu[i + 1] = round_storage<DT>(c);
+        }
+        float acc = neu[V];
+#pragma unroll
+        for (int i = V; i >= 1; --i) acc = fmaf(acc, mu[i - 1], neu[i - 1]);
+        store_scalar<DT>(out, j, acc);
+    }
+}
+
 // Runtime-order, any-alignment variants for the rare tiles whose sample has fewer references than
 // the launch's common order (warm-up after a reset) or whose row is not vector aligned: 16-byte
 // vectors when the row allows it, else one element at a time; planes visited in a loop.
@@ -508,6 +587,84 @@ __global__ void __launch_bounds__(NT, MINB) stream_kernel(const __grid_constant_
                 update_tile_any<DT>(plane0, sd.plane_stride, row, cnt, v, coef);
             else
                 forecast_tile_any<DT>(plane0, sd.plane_stride, row, cnt, v, coef, p.weighted != 0);
+        }
+    }
+}
+
+// The fused reference step: stream_kernel's walk over the update's tile list with, per tile, one of
+//   sample updated, output given      -> update_forecast_tile
+//   sample updated, no output         -> update_tile
+//   sample not updated but forecast   -> forecast_tile from its unchanged planes
+// Launch shape: the update's for the order (the mix is write-heavy: V + 2 of 2V + 3 streams are stores).
+template <int DT, int V, int W, int NT, int U, int C, int MINB>
+__global__ void __launch_bounds__(NT, MINB) update_forecast_kernel(const __grid_constant__ FusedParams q) {
+    constexpr uint32_t kChunk = static_cast<uint32_t>(NT) * U * W / Elem<DT>::kBytes;  // elements
+    constexpr uint32_t kTile = kChunk * C;
+    const StreamParams& p = q.up;
+    if (p.act_active != nullptr && blockIdx.x == 0 && threadIdx.x < SPECA_MAX_BATCH && ((p.act_bits >> threadIdx.x) & 1ull)) {
+        p.act_active[threadIdx.x] = 1;
+        p.act_spec[threadIdx.x] = 0;
+    }
+    uint32_t seg = p.seg_lo, seg_first = 0, seg_end = 0;
+    SegDesc sd = {};
+    int v_up = -1, v_fc = -1;
+    char* in = nullptr;
+    char* out = nullptr;
+    float r[kCoef] = {}, mu[kCoef] = {};
+    for (uint32_t tile = p.tile_lo + blockIdx.x; tile < p.tile_hi; tile += gridDim.x) {
+        if (tile >= seg_end) {
+            seg = next_segment(p.tile_start, seg, p.seg_hi, tile, seg_first, seg_end);
+            sd = p.segs[seg];
+            v_up = p.order[sd.sample];
+            v_fc = q.fc_order[sd.sample];
+            in = static_cast<char*>(p.io[sd.entry]);
+            out = static_cast<char*>(q.out[sd.entry]);
+            // a sample that is not updated here is forecast only if it is still speculating
+            if (v_up < 0 && q.fc_mask != nullptr && q.fc_mask[sd.sample] == 0) v_fc = -1;
+#pragma unroll
+            for (int i = 0; i < kCoef; ++i) {
+                r[i] = p.coef[sd.sample][i];
+                mu[i] = q.fc_coef[sd.sample][i];
+            }
+        }
+        const bool do_up = v_up >= 0 && in != nullptr, do_fc = v_fc >= 0 && out != nullptr;
+        if (!do_up && !do_fc) continue;
+        const uint32_t elem0 = (tile - seg_first) * kTile;
+        const uint32_t cnt = min(kTile, sd.n_elems - elem0);
+        const uint64_t byte0 = static_cast<uint64_t>(elem0) * Elem<DT>::kBytes;
+        char* plane0 = p.arena + sd.plane0_off + byte0;
+        char* frow = do_up ? in + sd.io_off + byte0 : nullptr;
+        char* orow = do_fc ? out + sd.io_off + byte0 : nullptr;
+        const bool aligned = ((reinterpret_cast<uintptr_t>(frow) | reinterpret_cast<uintptr_t>(orow)) & (W - 1)) == 0;
+        if (do_up && do_fc && v_up == V && v_fc == V && aligned) {
+            for (uint32_t done = 0; done < cnt; done += kChunk) {
+                const size_t off = static_cast<size_t>(done) * Elem<DT>::kBytes;
+                update_forecast_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, frow + off, orow + off,
+                                                      min(kChunk, cnt - done), r, mu);
+            }
+            continue;
+        }
+        // the rare shapes: halves done one after the other by the single-purpose routines
+        if (do_up) {
+            if (v_up == V && (reinterpret_cast<uintptr_t>(frow) & (W - 1)) == 0) {
+                for (uint32_t done = 0; done < cnt; done += kChunk) {
+                    const size_t off = static_cast<size_t>(done) * Elem<DT>::kBytes;
+                    update_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, frow + off, min(kChunk, cnt - done), r);
+                }
+            } else {
+                update_tile_any<DT>(plane0, sd.plane_stride, frow, cnt, v_up, r);
+            }
+        }
+        if (do_fc) {
+            if (do_up) __syncthreads();  // the forecast may read a plane element another thread of the CTA has just written
+            if (v_fc == V && (reinterpret_cast<uintptr_t>(orow) & (W - 1)) == 0) {
+                for (uint32_t done = 0; done < cnt; done += kChunk) {
+                    const size_t off = static_cast<size_t>(done) * Elem<DT>::kBytes;
+                    forecast_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, orow + off, min(kChunk, cnt - done), mu, false);
+                }
+            } else {
+                forecast_tile_any<DT>(plane0, sd.plane_stride, orow, cnt, v_fc, mu);
+            }
         }
     }
 }
@@ -1678,6 +1835,34 @@ cudaError_t launch_update(const StreamParams& p, int dtype, int path, int grid, 
 
 cudaError_t launch_forecast(const StreamParams& p, int dtype, int path, int grid, cudaStream_t stream) {
     return launch_stream(p, dtype, false, path, grid, stream);
+}
+
+// The fused kernel takes the update's shape for the order (the table's, for either storage type: the
+// four-vector shape the fp32 order-4 update prefers does not fit the fused body's registers).
+__host__ __device__ constexpr Shape fused_shape(int v) { return shape_for(SPECA_PATH_WIDE, true, v, SPECA_BF16); }
+
+template <int DT>
+static const void* fused_kernel_for(int v) {
+    constexpr Shape s0 = fused_shape(0), s1 = fused_shape(1), s2 = fused_shape(2), s3 = fused_shape(3), s4 = fused_shape(4);
+    switch (v) {
+        case 0: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 0, s0.w, s0.nt, s0.u, s0.chunks, s0.minb>);
+        case 1: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 1, s1.w, s1.nt, s1.u, s1.chunks, s1.minb>);
+        case 2: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 2, s2.w, s2.nt, s2.u, s2.chunks, s2.minb>);
+        case 3: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 3, s3.w, s3.nt, s3.u, s3.chunks, s3.minb>);
+        default: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 4, s4.w, s4.nt, s4.u, s4.chunks, s4.minb>);
+    }
+}
+
+int fused_ctas_per_sm(int order) { return fused_shape(order).minb; }
+
+// The kernel is compiled for the highest order any sample has in either half of the launch.
+cudaError_t launch_update_forecast(const FusedParams& p, int dtype, int grid, cudaStream_t stream) {
+    int v = max_order(p.up.order);
+    const int vf = max_order(p.fc_order);
+    v = vf > v ? vf : v;
+    const void* fn = dtype == SPECA_BF16 ? fused_kernel_for<SPECA_BF16>(v) : fused_kernel_for<SPECA_F32>(v);
+    void* args[1] = {const_cast<FusedParams*>(&p)};
+    return cudaLaunchKernel(fn, dim3(grid), dim3(fused_shape(v).nt), args, 0, stream);
 }
 
 template <int DT, int KCLASS>

@@ -1,0 +1,182 @@
+"""speca_cache_update_forecast: a whole reference step and the first speculative step after it in one
+pass over the tables. It must be, bit for bit, speca_cache_update_activate + speca_cache_commit_step +
+speca_forecast -- which the other tests hold against the oracle -- and it is held against the oracle
+here as well (tables after every step, forecasts of every step), over ragged shapes, orders 0-4, the
+three draft models, both storage types, warm-up orders, samples that skip a reference step and keep
+speculating, samples that have dropped out, and entries that are only updated."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import speca_oracle as O
+from paper_2509_11628_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def S():
+    from paper_2509_11628_b200 import binding
+    binding._lib()
+    return binding
+
+
+@pytest.fixture(scope="module")
+def U():
+    from tests import gpu_util
+    return gpu_util
+
+
+def bits(x):
+    return x.contiguous().view(torch.uint8)
+
+
+ENTRIES = [(3, 520), (9, 1031), (65, 1024), (40, 1030)]   # rows that are and are not 32-byte aligned, several tiles
+
+
+@pytest.mark.parametrize("dtype", [1, 0])
+@pytest.mark.parametrize("basis", [0, 1, 2])
+@pytest.mark.parametrize("m", [0, 1, 2, 3, 4])
+def test_fused_reference_step_equals_the_three_calls_and_the_oracle(S, U, dtype, basis, m):
+    B = 4
+    pair = U.Pair(ENTRIES, B, m, dtype, basis=basis)          # the three calls + the oracle
+    fused = S.SpecaCache(ENTRIES, B, m, dtype, DEV, basis=basis)
+    gen = torch.Generator(device=DEV).manual_seed(100 * dtype + 10 * basis + m)
+    ne = len(ENTRIES)
+    st = {k: torch.zeros(B, dtype=torch.int32, device=DEV) for k in ("spec_a", "spec_b")}
+    act_a = torch.ones(B, dtype=torch.uint8, device=DEV)
+    act_b = torch.ones(B, dtype=torch.uint8, device=DEV)
+    t = 1.0
+    # who takes which reference step: everybody warms up, then sample 1 skips one (and keeps speculating),
+    # sample 2 skips one after having dropped out (inactive: not forecast), sample 3 always takes part
+    plan = [([1, 1, 1, 1], None)] * (m + 1) + [([1, 0, 1, 1], None), ([1, 1, 0, 1], 2), ([1, 1, 1, 1], None)]
+    for k, (mask, drop) in enumerate(plan):
+        t -= 0.03 + 0.004 * (k % 3)                          # uneven gaps
+        t_ref = [t - 0.001 * b for b in range(B)]            # every sample on its own clock
+        t_tgt = [x - 0.011 for x in t_ref]
+        if drop is not None:                                 # a sample the verification rejected earlier
+            act_a[drop] = 0
+            act_b[drop] = 0
+            st["spec_a"][drop] = 3
+            st["spec_b"][drop] = 3
+        feats = [torch.randn(B, n, d, generator=gen, device=DEV).to(pair.tdt) for n, d in ENTRIES]
+        outs_a = [torch.full((B, n, d), 7.0, dtype=pair.tdt, device=DEV) for n, d in ENTRIES]
+        only_update = ne - 1 if k % 2 == 1 else None        # every other step one entry gets no forecast
+        give = list(outs_a)
+        if only_update is not None:
+            give[only_update] = None
+        launches = fused.launches
+        fused.update_forecast(feats, t_ref, t_tgt, give, mask=mask, active=act_a, spec_count=st["spec_a"], rearm=act_a)
+        assert fused.launches == launches + 1
+        # the same through the three calls (update with the re-arming, commit, forecast) and the oracle
+        pair.gpu.update_activate(feats, t_ref, mask, st["spec_b"], act_b)
+        pair.cpu.update([U.to_oracle(f).reshape(B, -1) for f in feats], t_ref, mask)
+        pair.commit()
+        pair.check_tables("step %d" % k)
+        active_host = [int(x) for x in act_b.cpu().tolist()]
+        outs_b = [torch.full((B, n, d), 7.0, dtype=pair.tdt, device=DEV) for n, d in ENTRIES]
+        pair.gpu.forecast(t_tgt, outs_b, act_b)
+        torch.cuda.synchronize()
+        # Eq. 2 by the oracle on the very planes the library holds (its tables were checked against the
+        # oracle's just above; they are re-synchronised only after the step, as the fused call forecasts
+        # from what it has just written)
+        for e in range(ne):
+            for b in range(B):
+                row = U.to_oracle(outs_b[e][b].reshape(-1))
+                if not active_host[b]:
+                    assert bool((outs_b[e][b].float() == 7.0).all()), ("an inactive sample was forecast", k, e, b)
+                    continue
+                planes = U.to_oracle(pair.gpu.plane_tensor(e, b))
+                planes[min(m, pair.cpu.n_refs[b] - 1) + 1:] = 0      # planes above the sample's order hold nothing yet
+                want = np.zeros(row.size, dtype=O.np_dtype(dtype))
+                O.forecast_segment(dtype, m, basis, pair.cpu.n_refs[b], pair.cpu.t_hist[b], t_tgt[b], planes, want)
+                scale = U.term_scale(planes, pair.forecast_weights(b, t_tgt[b]))
+                U.assert_close_storage(row, want, dtype, scale, "step %d forecast entry %d sample %d" % (k, e, b))
+        refs = fused.state()[0]
+        for e in range(ne):
+            for b in range(B):
+                live = min(m, refs[b] - 1) + 1               # planes above the sample's order are not defined yet
+                assert torch.equal(bits(fused.plane_tensor(e, b)[:live]), bits(pair.gpu.plane_tensor(e, b)[:live])), ("planes", k, e, b)
+            if e == only_update:
+                assert bool((outs_a[e].float() == 7.0).all()), ("an entry without an output was written", k, e)
+            else:
+                assert torch.equal(bits(outs_a[e]), bits(outs_b[e])), ("forecast", k, e)
+        assert torch.equal(act_a, act_b) and torch.equal(st["spec_a"], st["spec_b"])
+        assert fused.state() == pair.gpu.state()
+        # both sides continue from the oracle's bits (see gpu_util.Pair.sync_tables)
+        pair.sync_tables()
+        for e in range(ne):
+            for b in range(B):
+                fused.plane_tensor(e, b).copy_(pair.gpu.plane_tensor(e, b))
+    assert fused.stats()["update_forecast_launches"] == len(plan) and fused.stats()["update_launches"] == 0
+    assert fused.stats()["reference_steps"] == pair.gpu.stats()["reference_steps"]
+    fused.close()
+    pair.close()
+
+
+def test_fused_reference_step_refuses_what_it_cannot_do_and_leaves_the_history_alone(S):
+    entries = [(8, 512), (5, 520)]
+    B = 2
+    feats = [torch.randn(B, n, d, device=DEV).bfloat16() for n, d in entries]
+    outs = [torch.empty_like(f) for f in feats]
+
+    def status(fn):
+        with pytest.raises(S.SpecaError) as ei:
+            fn()
+        return ei.value.status
+
+    hist = S.SpecaCache(entries, B, 2, 1, DEV, layout=S.SPECA_LAYOUT_HISTORY)
+    assert status(lambda: hist.update_forecast(feats, [1.0] * B, [0.9] * B, outs)) == S.SPECA_ERR_UNSUPPORTED
+    hist.close()
+    bulk = S.SpecaCache(entries, B, 2, 1, DEV, path=S.SPECA_PATH_BULK)
+    assert status(lambda: bulk.update_forecast(feats, [1.0] * B, [0.9] * B, outs)) == S.SPECA_ERR_UNSUPPORTED
+    bulk.close()
+    c = S.SpecaCache(entries, B, 2, 1, DEV)
+    assert status(lambda: c.update_forecast([feats[0], None], [1.0] * B, [0.9] * B, outs)) == S.SPECA_ERR_INVALID_ARG
+    assert status(lambda: c.update_forecast(feats, [float("nan")] * B, [0.9] * B, outs)) == S.SPECA_ERR_INVALID_ARG
+    assert status(lambda: c.update_forecast(feats, [1.0] * B, [float("inf")] * B, outs)) == S.SPECA_ERR_INVALID_ARG
+    # a sample that is not part of the step and has never had a reference, with no device mask to excuse it
+    assert status(lambda: c.update_forecast(feats, [1.0] * B, [0.9] * B, outs, mask=[1, 0])) == S.SPECA_ERR_STATE
+    assert c.state()[0] == [0, 0] and c.launches == 0
+    c.update_forecast(feats, [1.0] * B, [0.9] * B, outs)
+    before = c.state()
+    assert before[0] == [1, 1]
+    assert status(lambda: c.update_forecast(feats, [1.0, 0.95], [0.9] * B, outs)) == S.SPECA_ERR_ZERO_GAP   # sample 0 repeats t = 1.0
+    assert c.state() == before
+    c.update([feats[0], None], [0.9] * B)                                 # an open reference step
+    assert status(lambda: c.update_forecast(feats, [0.9] * B, [0.8] * B, outs)) == S.SPECA_ERR_STATE
+    torch.cuda.synchronize()
+    c.close()
+
+
+def test_fused_reference_step_at_full_size(S):
+    """FLUX-shaped cache at full size, every entry in the one launch, the verification entry updated only:
+    every plane and every forecast bit for bit equal to the three calls."""
+    w = W.flux()
+    B, m, ne = w.batch, w.max_order, len(w.entries)
+    src = W.FeatureSource(w, DEV)
+    a = S.SpecaCache(w.entries, B, m, w.dtype, DEV)
+    b = S.SpecaCache(w.entries, B, m, w.dtype, DEV)
+    outs_a = [torch.empty(B, n, d, dtype=w.torch_dtype, device=DEV) for n, d in w.entries]
+    outs_b = [torch.empty(B, n, d, dtype=w.torch_dtype, device=DEV) for n, d in w.entries]
+    give_a, give_b = list(outs_a), list(outs_b)
+    give_a[w.vidx] = None
+    give_b[w.vidx] = None
+    for step in range(m + 2):                                # orders 0, 1, 2 warming up, then steady state
+        t = [w.times[step]] * B
+        t_tgt = [w.times[step + 1]] * B
+        feats = [src.feature(e, step, t) for e in range(ne)]
+        a.update_forecast(feats, t, t_tgt, give_a)
+        b.update(feats, t)
+        b.commit_step()
+        b.forecast(t_tgt, give_b)
+        torch.cuda.synchronize()
+        for e in range(ne):
+            live = min(m, step) + 1
+            assert torch.equal(bits(a.plane_tensor(e, 0)[:live]), bits(b.plane_tensor(e, 0)[:live])), (step, e)
+            if e != w.vidx:
+                assert torch.equal(bits(outs_a[e]), bits(outs_b[e])), (step, e)
+        del feats
+    a.close()
+    b.close()
