@@ -348,6 +348,38 @@ def time_graph_replay(h: Harness, K: int = 4, reps: int = 20):
             "eager_steps_per_s": 1e3 / eager_ms, "graph_steps_per_s": 1e3 / graph_ms}
 
 
+def time_fused_reference_step(h: Harness, peak: float, reps: int = 20):
+    """A reference step and the first forecast after it as ONE launch (speca_cache_update_forecast): the
+    forecast is evaluated from the planes the update has just formed, so the tables are not read again --
+    2 * order + 3 words per element (order + 2 of them writes) instead of (2 * order + 2) + (order + 2).
+    The verification entry is only updated (its forecast comes out of the verification launch)."""
+    w, dev = h.w, h.device
+    others = list(h.outs)
+    others[w.vidx] = None
+    m, eb = w.max_order, w.elem_bytes
+    n_ver = w.batch * w.entry_elems(w.vidx)
+    nbytes = (2 * m + 3) * eb * (w.elems_per_order - n_ver) + (2 * m + 2) * eb * n_ver
+    ab = algorithmic_bytes(w, m)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    total = 0.0
+    for r in range(reps + 3):
+        j = h.j
+        h.j += 1
+        t_ref, t_tgt = h.times_for(j)
+        e0.record()
+        h.cache.update_forecast(h.feats[j & 1], t_ref, t_tgt, others, spec_count=h.spec, rearm=h.active)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        if r >= 3:
+            total += e0.elapsed_time(e1)
+    ms = total / reps
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"ms": ms, "algorithmic_bytes": nbytes, "gbs": gbs, "frac_of_measured_peak": gbs / peak,
+            "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
+            "bytes_of_the_two_launches": ab["update"] + ab["forecast"],
+            "traffic_saved_vs_two_launches": 1.0 - nbytes / float(ab["update"] + ab["forecast"])}
+
+
 def time_update_per_entry(h: Harness, reps: int = 5):
     """A model hands over one block output at a time: the same reference step as one launch per entry."""
     w, dev = h.w, h.device
@@ -680,8 +712,8 @@ def sampler_run(device: str, path: int, name: str, layout: int = 0):
         def verify_and_select(self, fresh, t, tau, period):
             return self._timed("verify+select", lambda: SCH.SpecaCacheBackend.verify_and_select(self, fresh, t, tau, period))
 
-        def reference_step(self, feats, t, mask):
-            return self._timed("update", lambda: SCH.SpecaCacheBackend.reference_step(self, feats, t, mask))
+        def reference_step(self, feats, t, mask, t_next=None):
+            return self._timed("update", lambda: SCH.SpecaCacheBackend.reference_step(self, feats, t, mask, t_next))
 
     be = Timed(cache)
     wall0 = time.perf_counter()
@@ -937,7 +969,7 @@ def _r(x, digits=5):
 
 
 def build_line(*, value, ms_per_step, n_gpus, steps, warmup, config, roofline, cpu_baseline, e2e, gpu_launches, clocks,
-               kernels, forecast_verify_gbs, speculative_steps_per_s, also=None, detail_path=None, scaling="weak"):
+               kernels, forecast_verify_gbs, speculative_steps_per_s, also=None, detail_path=None, scaling="weak", fused=None):
     """The compact JSON object of the benchmark's last line, kept under MAX_LINE_BYTES: whatever does
     not fit belongs in the detail file. Raises only if the contract keys alone are too long."""
     line = {
@@ -952,12 +984,15 @@ def build_line(*, value, ms_per_step, n_gpus, steps, warmup, config, roofline, c
         "forecast_verify_gbs": _r(forecast_verify_gbs), "speculative_steps_per_s": _r(speculative_steps_per_s),
         "kernels_ms_gbs": {k: [_r(v["ms"], 4), _r(v["gbs"], 4)] for k, v in kernels.items() if k != "select"},
     }
+    if fused:   # update + first forecast as one launch: [ms, GB/s over its own 2*order+3 words, ms of the two launches]
+        line["fused_update_forecast_ms_gbs_vs_ms"] = [_r(fused["ms"], 4), _r(fused["gbs"], 4), _r(fused["ms_of_the_two_launches"], 4)]
     if also:
         line["also_value_fv_gbs_steps_per_s"] = {k: [_r(x, 4) for x in v] for k, v in also.items()}
     if detail_path:
         line["detail"] = detail_path
     # the contract keys always go out; the extras are dropped, last first, if the line would grow too long
-    for extra in (None, "also_value_fv_gbs_steps_per_s", "kernels_ms_gbs", "detail", "value_covers"):
+    for extra in (None, "also_value_fv_gbs_steps_per_s", "fused_update_forecast_ms_gbs_vs_ms", "kernels_ms_gbs", "detail",
+                  "value_covers"):
         if extra is not None:
             line.pop(extra, None)
         text = json.dumps(line, separators=(",", ":"))
@@ -1104,6 +1139,12 @@ def main(argv=None):
                                 "note": "other hardware, whole-model numbers; context only"}}
 
     tables = solo and layout == 0      # these calls exist for the table layout only
+    fused = None
+    if layout == 0 and path in (0, 3):
+        fused = time_fused_reference_step(h, peak)
+        fused["ms_of_the_two_launches"] = per_ms["update"] + per_ms["forecast"]
+        fused["speedup_vs_two_launches"] = fused["ms_of_the_two_launches"] / fused["ms"]
+        detail["fused_reference_step"] = fused
     if args.full and solo:
         detail["verify_metrics"] = time_metrics(h)
     if args.full and tables:
@@ -1155,6 +1196,9 @@ def main(argv=None):
                 v2, ms2, kern2, ex2 = summarize(w2, p2, t2, k2, 1, peak)
                 per_config[name] = {"value": v2, "unit": "GB/s", "ms_per_step": ms2, "steps": k2,
                                     "config": workload_config(w2), "kernels": kern2, **ex2}
+                if path in (0, 3):
+                    per_config[name]["fused_reference_step"] = time_fused_reference_step(h2, peak)
+                    per_config[name]["fused_reference_step"]["ms_of_the_two_launches"] = p2["update"] + p2["forecast"]
                 also[name] = [v2, ex2["forecast_verify_gbs"], ex2["speculative_steps_per_s"]]
                 if args.full:
                     try:
@@ -1226,7 +1270,8 @@ def main(argv=None):
                      config=workload_config(w, args.layout), roofline=roofline, cpu_baseline=cpu_baseline, e2e=e2e,
                      gpu_launches=launches, clocks=clocks_line, kernels=kernels,
                      forecast_verify_gbs=extra["forecast_verify_gbs"],
-                     speculative_steps_per_s=extra["speculative_steps_per_s"], also=also, detail_path=detail_path), flush=True)
+                     speculative_steps_per_s=extra["speculative_steps_per_s"], also=also, detail_path=detail_path,
+                     fused=fused), flush=True)
     D.shutdown()
     return 0
 

@@ -400,7 +400,7 @@ class SpecaCache:
                  verify_entry=-1, eps=0.0, path=SPECA_PATH_AUTO, layout=SPECA_LAYOUT_TABLES):
         self.entries = [(int(n), int(d)) for n, d in entries]
         self.batch, self.max_order, self.dtype, self.basis = batch, max_order, dtype, basis
-        self.layout = layout
+        self.layout, self.path = layout, path
         self.device = torch.device(device)
         self.verify_entry = verify_entry if verify_entry >= 0 else len(self.entries) - 1
         nbytes = speca_cache_arena_bytes(self.entries, batch, max_order, dtype, basis, verify_entry, path, layout)

@@ -1837,9 +1837,24 @@ cudaError_t launch_forecast(const StreamParams& p, int dtype, int path, int grid
     return launch_stream(p, dtype, false, path, grid, stream);
 }
 
-// The fused kernel takes the update's shape for the order (the table's, for either storage type: the
-// four-vector shape the fp32 order-4 update prefers does not fit the fused body's registers).
-__host__ __device__ constexpr Shape fused_shape(int v) { return shape_for(SPECA_PATH_WIDE, true, v, SPECA_BF16); }
+// Launch shapes of the fused kernel per order (2v + 3 streams, v + 2 of them stores), 32 KB tiles like
+// the update's so that the two share a tile table. Swept on a B200 on 20 FLUX-sized entries (bf16 / fp32,
+// GB/s over the 2v + 3 words): unlike the plain update this mix wants two vectors per thread and one
+// 256-thread CTA per SM (order 2: 6310 / 6270 against 4680 / 6340 with the update's 128 x 1 x 3 CTAs/SM
+// shape, 5010 / 6010 with 256 x 1 x 2); only order 0 (one load, two stores) prefers one vector
+// (5720 / 5930 against 5440 / 5600).
+#ifndef SPECA_SHAPES_FUSED
+#define SPECA_SHAPES_FUSED \
+    {32, 256, 1, 4, 2}, {32, 256, 2, 2, 1}, {32, 256, 2, 2, 1}, {32, 256, 2, 2, 1}, { 32, 256, 2, 2, 1 }
+#endif
+__host__ __device__ constexpr Shape fused_shape(int v) {
+    constexpr Shape fs[SPECA_MAX_ORDER + 1] = {SPECA_SHAPES_FUSED};
+    return fs[v < 0 ? 0 : (v > SPECA_MAX_ORDER ? SPECA_MAX_ORDER : v)];
+}
+static_assert(shape_tile_bytes(fused_shape(0)) == shape_tile_bytes(shape_for(SPECA_PATH_WIDE, true, 0, SPECA_BF16)) &&
+                  shape_tile_bytes(fused_shape(2)) == shape_tile_bytes(shape_for(SPECA_PATH_WIDE, true, 2, SPECA_BF16)) &&
+                  shape_tile_bytes(fused_shape(4)) == shape_tile_bytes(shape_for(SPECA_PATH_WIDE, true, 4, SPECA_BF16)),
+              "the fused kernel walks the update's tile table");
 
 template <int DT>
 static const void* fused_kernel_for(int v) {

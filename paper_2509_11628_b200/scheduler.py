@@ -98,7 +98,10 @@ def run_sampler(backend, model, times: Sequence[float], tau0: float, beta: float
         need_full = [0 if row[b] == ACCEPTED else 1 for b in range(B)]
         if any(need_full):
             feats = model.full(i, tt, need_full)
-            backend.reference_step(feats, tt, need_full)
+            # the next step is speculative for everyone who is active after this one: a backend that can
+            # may hand over that step's forecasts from the same pass over the tables
+            t_next = [times[i + 1]] * B if i + 1 < len(times) and i + 1 >= warm_refs else None
+            backend.reference_step(feats, tt, need_full, t_next)
             active = backend.active_mask()
         trace.steps.append(row)
         trace.err.append(errs)
@@ -109,10 +112,12 @@ class SpecaCacheBackend:
     """The CUDA library as a scheduler backend. Device buffers are allocated once; one small
     device-to-host copy of the decisions per speculative step is the only synchronisation."""
 
-    def __init__(self, cache, metric=None):
+    def __init__(self, cache, metric=None, use_fused=True):
         import torch
         from . import binding as S
         self.S, self.torch, self.cache = S, torch, cache
+        self.use_fused = use_fused      # reference steps also hand over the next step's forecasts (one launch)
+        self.forecast_for = None        # the times the output buffers already hold forecasts for
         self.batch = cache.batch
         dev = cache.device
         self.metric = metric
@@ -132,6 +137,7 @@ class SpecaCacheBackend:
 
     def reset_run(self):
         self.cache.reset()
+        self.forecast_for = None
         self.active.zero_()
         self.spec.zero_()
         self.h_active.zero_()
@@ -147,6 +153,10 @@ class SpecaCacheBackend:
         return self.S.speca_tau(tau0, beta, t, T)
 
     def forecast(self, t_target):
+        if self.forecast_for is not None and list(t_target) == self.forecast_for:
+            self.forecast_for = None      # the reference step before this one already wrote these forecasts
+            return
+        self.forecast_for = None
         self.cache.forecast(t_target, self.outs, self.active)
 
     def verify_and_select(self, fresh, t_target, tau, period):
@@ -161,7 +171,18 @@ class SpecaCacheBackend:
     def active_mask(self):
         return self.h_active.tolist()
 
-    def reference_step(self, feats, t_ref, mask):
-        self.cache.update_activate(feats, t_ref, mask, self.spec, self.active)   # Eq. 3 and the re-arming, one launch
-        self.cache.commit_step()
+    def reference_step(self, feats, t_ref, mask, t_next=None):
+        S = self.S
+        fused = (self.use_fused and t_next is not None and self.cache.layout == S.SPECA_LAYOUT_TABLES and
+                 self.cache.path in (S.SPECA_PATH_AUTO, S.SPECA_PATH_WIDE))
+        if fused:
+            # Eq. 3, the re-arming and Eq. 2 at the next step's time in one launch: samples that took this
+            # step are forecast from the planes just written, the ones still speculating from theirs
+            self.cache.update_forecast(feats, t_ref, t_next, self.outs, mask=mask, active=self.active,
+                                       spec_count=self.spec, rearm=self.active)
+            self.forecast_for = list(t_next)
+        else:
+            self.cache.update_activate(feats, t_ref, mask, self.spec, self.active)   # Eq. 3 and the re-arming, one launch
+            self.cache.commit_step()
+            self.forecast_for = None
         self._fetch(with_decisions=False)

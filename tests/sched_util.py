@@ -35,7 +35,7 @@ class OracleBackend:
     def active_mask(self):
         return list(self.active)
 
-    def reference_step(self, feats, t_ref, mask):
+    def reference_step(self, feats, t_ref, mask, t_next=None):
         self.cache.update(feats, t_ref, mask)
         self.cache.commit_step()
         for b in range(self.batch):
@@ -69,7 +69,7 @@ class ScriptedBackend:
     def active_mask(self):
         return list(self.active)
 
-    def reference_step(self, feats, t_ref, mask):
+    def reference_step(self, feats, t_ref, mask, t_next=None):
         self.calls.append(("update", self.step, tuple(mask)))
         for b in range(self.batch):
             if mask[b]:
