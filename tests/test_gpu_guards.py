@@ -71,8 +71,18 @@ def test_nothing_is_written_outside_the_buffers(S, path, dtype, tdt, m):
         idx, n_act = Guarded((B,), torch.int32), Guarded((1,), torch.int32)
         S.speca_select_adaptive(handle, acc.t, 3, 1, spec.t, active.t, idx.t, n_act.t)
         S.speca_activate(handle, None, spec.t, active.t)
+        fouts = []
+        if path == 3:                           # the fused reference step exists on the default path only
+            fouts = [Guarded((B, n, d), tdt, offset=shift) for n, d in RAGGED]
+            ffeats = [Guarded((B, n, d), tdt, offset=shift) for n, d in RAGGED]
+            for f in ffeats:
+                f.t.copy_(torch.randn(f.t.shape, generator=gen, device=DEV).to(tdt))
+            t_new = 0.4 - 0.05 * (1 if shift else 0)
+            S.speca_cache_update_forecast(handle, [f.t for f in ffeats], [t_new] * B, [1, 0, 1], [t_new - 0.02] * B, active.t,
+                                          [o.t for o in fouts], spec.t, active.t)
+            fouts += ffeats
         torch.cuda.synchronize()
-        for g in outs + mouts + [pred, err, acc, sums, total, spec, active, idx, n_act, arena]:
+        for g in outs + mouts + fouts + [pred, err, acc, sums, total, spec, active, idx, n_act, arena]:
             assert g.intact(), "a guard zone was overwritten (path %d, dtype %d, order %d, shift %d)" % (path, dtype, m, shift)
         assert not bool((outs[2].t.view(torch.uint8) == PATTERN).all())       # and the outputs were written
     S.speca_cache_destroy(handle)
