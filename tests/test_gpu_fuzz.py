@@ -65,6 +65,10 @@ def test_random_scenario(S, U, seed):
         path = int(rng.choice([0, 3]))        # which only the default kernels serve
     pair = U.Pair(entries, B, m, dtype, basis, verify_entry=vidx, path=path, layout=layout)
     nv, dv = entries[pair.vidx]
+    # a second cache takes every reference step through the fused call (where that call exists): its tables
+    # and its forecast must be, bit for bit, those of update + commit + forecast on the first one
+    shadow = S.SpecaCache(entries, B, m, dtype, DEV, basis, vidx, path=path) if layout == 0 and path in (0, 3) else None
+    ones = torch.ones(B, dtype=torch.uint8, device=DEV)
     what = "seed %d (B=%d m=%d dtype=%d basis=%d path=%d layout=%d entries=%s)" % (seed, B, m, dtype, basis, path, layout, entries)
 
     def feats():
@@ -82,14 +86,41 @@ def test_random_scenario(S, U, seed):
             mask = None if rng.random() < 0.4 else rng.integers(0, 2, B).tolist()
             if mask is not None and not any(mask):
                 mask[int(rng.integers(0, B))] = 1
-            pair.update(feats(), t, mask, per_entry_calls=bool(rng.integers(0, 2)))
+            fs = feats()
+            pair.update(fs, t, mask, per_entry_calls=bool(rng.integers(0, 2)))
             pair.commit()
             pair.check_tables(what + " step %d tables" % step)
+            if shadow is not None:
+                t_next = [x - 0.009 for x in t]
+                give = [torch.full((B, n, d), 2.5, dtype=pair.tdt, device=DEV) for n, d in entries]
+                plain = [torch.full((B, n, d), 2.5, dtype=pair.tdt, device=DEV) for n, d in entries]
+                skip = int(rng.integers(-1, len(entries)))          # one entry may be updated only
+                if skip >= 0:
+                    give[skip] = None
+                shadow.update_forecast(fs, t, t_next, give, mask=mask, active=ones)
+                pair.gpu.forecast(t_next, [None if e == skip else o for e, o in enumerate(plain)], ones)
+                torch.cuda.synchronize()
+                assert shadow.state()[0] == pair.gpu.state()[0], what
+                for e in range(len(entries)):
+                    for b in range(B):
+                        live = min(m, pair.cpu.n_refs[b] - 1) + 1
+                        if live > 0:
+                            assert torch.equal(shadow.plane_tensor(e, b)[:live].contiguous().view(torch.uint8),
+                                               pair.gpu.plane_tensor(e, b)[:live].contiguous().view(torch.uint8)), \
+                                what + " step %d fused tables entry %d sample %d" % (step, e, b)
+                    if e != skip:
+                        assert torch.equal(give[e].view(torch.uint8), plain[e].view(torch.uint8)), what + " step %d fused forecast entry %d" % (step, e)
             pair.sync_tables()
+            if shadow is not None:
+                for e in range(len(entries)):
+                    for b in range(B):
+                        shadow.plane_tensor(e, b).copy_(pair.gpu.plane_tensor(e, b))
         elif kind == "reset":
             mask = rng.integers(0, 2, B).tolist()
             pair.gpu.reset(mask)
             pair.cpu.reset(mask)
+            if shadow is not None:
+                shadow.reset(mask)
         else:
             act = [h & int(a) for h, a in zip(have, rng.integers(0, 2, B).tolist())]
             if rng.random() < 0.3:
@@ -139,4 +170,6 @@ def test_random_scenario(S, U, seed):
             want_act, want_cnt, _ = O.select_adaptive(acc2.cpu().tolist(), k_max, group, cnt, act)
             assert nxt.cpu().tolist() == want_act and c1.cpu().tolist() == want_cnt, what
             cnt = want_cnt
+    if shadow is not None:
+        shadow.close()
     pair.close()
