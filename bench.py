@@ -46,9 +46,10 @@ MAX_LINE_BYTES = 2000
 # DRAM bytes per cached element per launch: (dram__bytes_read.sum + dram__bytes_write.sum) / elements
 # from the ncu capture of the DiT-XL/2-shaped case (1.6 GB cache; see the file named in TRAFFIC_SOURCE).
 # The kernels are reuse-free streams, so traffic grows in proportion to the elements a launch covers;
-# other workloads scale by that. An entry is None while its kernel has changed since the counters
-# were taken.
-NCU_DRAM_BYTES_PER_ELEM = {"update": 11.83, "forecast": 7.93, "verify": None}
+# other workloads scale by that (the verify figure is from profiles/verify_kernel_dit_xl2.md and counts
+# reads only: the forecast it stores is still dirty in L2 when the kernel ends). An entry is None while
+# its kernel has changed since the counters were taken.
+NCU_DRAM_BYTES_PER_ELEM = {"update": 11.80, "forecast": 7.93, "verify": 8.01}
 TRAFFIC_SOURCE = "ncu dram bytes/elem on the DiT-shaped capture (profiles/stream_kernels_dit_xl2.md) x elems"
 
 

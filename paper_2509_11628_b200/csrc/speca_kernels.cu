@@ -496,9 +496,10 @@ __device__ __noinline__ void update_tile_any(char* __restrict__ plane0, uint64_t
 // Launch shapes. Both kernels are pure HBM streams whose speed is set by how the DRAM sees the mix
 // of reads and writes, so the shape (vector width, threads, vectors per thread, CTAs per SM) was
 // chosen by sweeping it on a B200 in bf16 with every plane 4 KB aligned (at order 2):
-//   update   (half of the traffic is writes): few bytes in flight win -- 128 threads x one 32-byte
-//            vector per plane, 3 CTAs/SM (36 KB in flight per SM) reaches the device's copy rate;
-//            deeper or wider shapes (256 x 4 vectors, 2 CTAs/SM) are 4-9 % slower on this mix.
+//   update   (half of the traffic is writes): few bytes in flight win -- 128 threads x two 32-byte
+//            vectors per plane, 2 CTAs/SM (48 KB in flight per SM) reaches the device's copy rate
+//            (one vector x 3 CTAs/SM is 1-3 % behind: 496 / 1489 us against 483 / 1474 on the DiT /
+//            FLUX shapes); deeper or wider shapes (256 x 4 vectors, 2 CTAs/SM) are 4-9 % slower.
 //   forecast (one write per three reads): flat above ~70 KB in flight per SM; 256 threads x one
 //            vector per plane, 3 CTAs/SM.
 // Other orders were swept the same way (FLUX shape, GB/s before -> after giving each order its own
@@ -515,7 +516,7 @@ struct Shape {
 // the bytes in flight per SM near the sweet spot of the mix. Every shape has a 32 KB tile.
 #ifndef SPECA_SHAPES_UPDATE
 #define SPECA_SHAPES_UPDATE \
-    {32, 128, 2, 4, 4}, {32, 128, 2, 4, 3}, {32, 128, 1, 8, 3}, {32, 128, 1, 8, 3}, { 32, 128, 1, 8, 2 }
+    {32, 128, 2, 4, 4}, {32, 128, 2, 4, 3}, {32, 128, 2, 4, 2}, {32, 128, 1, 8, 3}, { 32, 128, 1, 8, 2 }
 #endif
 #ifndef SPECA_SHAPES_FORECAST
 #define SPECA_SHAPES_FORECAST \
