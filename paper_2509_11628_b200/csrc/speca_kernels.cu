@@ -1359,12 +1359,28 @@ __device__ __noinline__ void verify_tile_any(const char* __restrict__ plane0, ui
     }
 }
 
-// Per-sample continuation of the speculative run by ONE warp (all 32 lanes call it; B <= 64, lane l
-// looks after samples l and l + 32). `accept` may have been written by other CTAs of the same kernel
-// just before (the caller has fenced): it is read around L1.
-__device__ __forceinline__ void select_in_warp(const uint8_t* accept, int32_t k_max, int32_t group, int32_t batch,
-                                               int32_t* spec_count, const uint8_t* active_in, uint8_t* active_out,
-                                               int32_t* idx_out, int32_t* n_out) {
+// Per-sample continuation of the speculative run by ONE warp (all 32 lanes take part; B <= 64, lane l
+// looks after samples l and l + 32). In two halves, so that the fused caller can have the loads of the
+// first in flight while it is still summing: what the rule reads from memory ...
+struct SelectIn {
+    bool act[2];
+    int32_t cnt[2];
+};
+__device__ __forceinline__ SelectIn select_load(int32_t batch, const int32_t* spec_count, const uint8_t* active_in) {
+    const int lane = threadIdx.x & 31;
+    SelectIn in;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int b = lane + 32 * h;
+        in.act[h] = b < batch && active_in[b] != 0;
+        in.cnt[h] = b < batch ? spec_count[b] : 0;
+    }
+    return in;
+}
+// ... and the rule itself, given each sample's accept flag (acc[h] for sample lane + 32 h).
+__device__ __forceinline__ void select_apply(const SelectIn& in, const bool (&acc)[2], int32_t k_max, int32_t group,
+                                             int32_t batch, int32_t* spec_count, uint8_t* active_out, int32_t* idx_out,
+                                             int32_t* n_out) {
     const int lane = threadIdx.x & 31;
     uint64_t keep = 0;
 #pragma unroll
@@ -1372,8 +1388,8 @@ __device__ __forceinline__ void select_in_warp(const uint8_t* accept, int32_t k_
         const int b = lane + 32 * h;
         bool k = false;
         if (b < batch) {
-            const bool ok = active_in[b] != 0 && __ldcg(accept + b) != 0;
-            int32_t c = spec_count[b];
+            const bool ok = in.act[h] && acc[h];
+            int32_t c = in.cnt[h];
             if (ok) {
                 c += 1;
                 spec_count[b] = c;
@@ -1403,6 +1419,18 @@ __device__ __forceinline__ void select_in_warp(const uint8_t* accept, int32_t k_
         }
     }
     if (lane == 0 && n_out != nullptr) *n_out = __popcll(next);
+}
+// Both halves, with the accept flags read from memory (in place is fine: a lane reads its own samples'
+// mask bytes before it writes them).
+__device__ __forceinline__ void select_in_warp(const uint8_t* accept, int32_t k_max, int32_t group, int32_t batch,
+                                               int32_t* spec_count, const uint8_t* active_in, uint8_t* active_out,
+                                               int32_t* idx_out, int32_t* n_out) {
+    const int lane = threadIdx.x & 31;
+    const SelectIn in = select_load(batch, spec_count, active_in);
+    bool acc[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) acc[h] = lane + 32 * h < batch && in.act[h] && accept[lane + 32 * h] != 0;
+    select_apply(in, acc, k_max, group, batch, spec_count, active_out, idx_out, n_out);
 }
 
 // Tiles of the active samples form one list of T = (active samples) x (tiles per sample) tiles;
@@ -1453,12 +1481,14 @@ __global__ void __launch_bounds__(kThreads, V <= 2 ? SPECA_VERIFY_MINB : 2) veri
     __shared__ float cluster_slot[SPECA_MAX_BATCH][NA][kMaxClusterSize];  // [slot][value][rank], the leader's copy is used
     __shared__ uint32_t active_bits[2];
     __shared__ bool is_last;
+    __shared__ uint8_t sel_accept[SPECA_MAX_BATCH];  // this launch's accept flags, for the fused continuation
 
     // Every CTA of the cluster is running once this barrier completes; it is only waited for right
     // before the first access to the leader's shared memory.
     cluster.barrier_arrive();
 
     for (int i = threadIdx.x; i < SPECA_MAX_BATCH * NA * kWarps; i += kThreads) (&warp_part[0][0][0])[i] = 0.f;
+    if (threadIdx.x < SPECA_MAX_BATCH) sel_accept[threadIdx.x] = 0;  // a sample that is not verified does not continue
     // samples that take part: a defined table and, with a device mask, a non-zero byte
     if (threadIdx.x < 64) {
         const int b = threadIdx.x;
@@ -1606,6 +1636,9 @@ __global__ void __launch_bounds__(kThreads, V <= 2 ? SPECA_VERIFY_MINB : 2) veri
     // whole warp takes one sample; with many samples each has few and a warp takes four at a time.
     // Per sample the order is fixed (lane l adds clusters q_lo + l, q_lo + l + L, ..., then a shuffle
     // tree over the group), four loads per lane are in flight at once, and the sums are fp64.
+    // the continuation rule's own inputs are asked for now and used after the sums
+    SelectIn sel_in = {};
+    if (p.sel_active != nullptr && warp == 0) sel_in = select_load(p.batch, p.sel_spec, p.dev_mask);
     const uint32_t L = n_active > 8 ? 8 : 32, per_warp = 32 / L;
     const uint32_t g = lane / L, l = lane % L;
     const bool holes = Q > T;  // more clusters than tiles: some clusters in a sample's span own nothing
@@ -1646,16 +1679,20 @@ __global__ void __launch_bounds__(kThreads, V <= 2 ? SPECA_VERIFY_MINB : 2) veri
                 for (int i = 0; i < 3; ++i) p.raw_sums[b * 4 + i] = i < NA ? s[i] : 0.0;
             } else {
                 const double e = Metric<M>::error(s, p.eps);
+                const uint8_t ok = (e <= static_cast<double>(p.tau[b])) ? 1 : 0;  // NaN compares false: reject
                 p.err[b] = static_cast<float>(e);
-                p.accept[b] = (e <= static_cast<double>(p.tau[b])) ? 1 : 0;  // NaN compares false: reject
+                p.accept[b] = ok;
+                sel_accept[b] = ok;
             }
         }
     }
     __syncthreads();
     // Fused continuation: every decision of this step is final by now. The new mask goes to a buffer
     // of its own: CTAs of this grid may still be reading the step's mask.
-    if (p.sel_active != nullptr && warp == 0)
-        select_in_warp(p.accept, p.sel_kmax, p.sel_group, p.batch, p.sel_spec, p.dev_mask, p.sel_active, p.sel_idx, p.sel_n);
+    if (p.sel_active != nullptr && warp == 0) {
+        const bool acc[2] = {sel_accept[lane] != 0, sel_accept[lane + 32] != 0};
+        select_apply(sel_in, acc, p.sel_kmax, p.sel_group, p.batch, p.sel_spec, p.sel_active, p.sel_idx, p.sel_n);
+    }
     if (threadIdx.x == 0) *p.ticket = 0;  // ready for the next launch on this stream
 }
 
