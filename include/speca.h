@@ -253,6 +253,20 @@ speca_status_t speca_cache_update_forecast(speca_cache_t* cache, const void* con
                                            uint8_t* dev_rearm_mask, void* stream);
 
 /*
+ * The same with K = n_targets speculative times at once (Fig. 1: the draft predicts the next steps
+ * from one reference): exactly speca_cache_update(_activate) + speca_cache_commit_step +
+ * speca_forecast_multi, bit for bit, in one pass: 2v + 2 + K words per element instead of
+ * (2v + 2) + (v + 1 + K). t_target is K x B doubles (target-major) and outs[e] a [K, B, N_e, D] tensor,
+ * as in speca_forecast_multi; everything else as above. n_targets = 1 is speca_cache_update_forecast.
+ * Errors: as above, and INVALID_ARG for n_targets outside 1..SPECA_MAX_HORIZON.
+ */
+speca_status_t speca_cache_update_forecast_multi(speca_cache_t* cache, const void* const* feats, const double* t_ref,
+                                                 const uint8_t* host_sample_mask, int32_t n_targets,
+                                                 const double* t_target, const uint8_t* dev_active_mask,
+                                                 void* const* outs, int32_t* dev_spec_count, uint8_t* dev_rearm_mask,
+                                                 void* stream);
+
+/*
  * Close a reference step: push t_ref into each masked sample's reference history and raise its
  * reference count. Host state only. Errors: STATE if some entry has not been updated for
  * exactly the masked samples since the last commit, or no update is pending.

@@ -29,7 +29,7 @@ SPECA_MAX_ORDER, SPECA_MAX_BATCH, SPECA_MAX_ENTRIES, SPECA_MAX_HORIZON = 4, 64, 
 
 EXPORTS = [
     "speca_cache_arena_bytes", "speca_cache_create", "speca_cache_destroy", "speca_cache_reset",
-    "speca_cache_update", "speca_cache_update_activate", "speca_cache_update_forecast", "speca_cache_commit_step", "speca_forecast", "speca_verify",
+    "speca_cache_update", "speca_cache_update_activate", "speca_cache_update_forecast", "speca_cache_update_forecast_multi", "speca_cache_commit_step", "speca_forecast", "speca_verify",
     "speca_select_adaptive", "speca_activate", "speca_tau", "speca_cache_state", "speca_cache_plane",
     "speca_cache_launch_count", "speca_cache_stats", "speca_cache_check", "speca_cache_next_slot", "speca_forecast_weights", "speca_status_string", "speca_last_error", "speca_version",
     "speca_verify_pred_static", "speca_forecast_multi", "speca_verify_metric",
@@ -87,6 +87,7 @@ def _lib() -> ctypes.CDLL:
     L.speca_cache_update.argtypes = [vp, vp, vp, vp, vp]
     L.speca_cache_update_activate.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.speca_cache_update_forecast.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.speca_cache_update_forecast_multi.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
     L.speca_cache_commit_step.argtypes = [vp]
     L.speca_forecast.argtypes = [vp, vp, vp, vp, vp]
     L.speca_forecast_sum.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]
@@ -229,6 +230,15 @@ def speca_cache_update_forecast(cache, feats, t_ref, host_sample_mask, t_target,
     _check(_lib().speca_cache_update_forecast(cache, _ptr_array(feats), _doubles(t_ref), _bytes(host_sample_mask),
                                               _doubles(t_target), _dev_ptr(dev_active_mask), _ptr_array(outs),
                                               _dev_ptr(dev_spec_count), _dev_ptr(dev_rearm_mask), _stream_ptr(stream)), cache)
+
+
+def speca_cache_update_forecast_multi(cache, feats, t_ref, host_sample_mask, t_targets, dev_active_mask, outs,
+                                      dev_spec_count=None, dev_rearm_mask=None, stream=None) -> None:
+    """The same with K speculative times: t_targets is K lists of B times, outs[e] a [K, B, N_e, D] tensor."""
+    flat = [t for row in t_targets for t in row]
+    _check(_lib().speca_cache_update_forecast_multi(cache, _ptr_array(feats), _doubles(t_ref), _bytes(host_sample_mask),
+                                                    len(t_targets), _doubles(flat), _dev_ptr(dev_active_mask), _ptr_array(outs),
+                                                    _dev_ptr(dev_spec_count), _dev_ptr(dev_rearm_mask), _stream_ptr(stream)), cache)
 
 
 def speca_cache_commit_step(cache) -> None:
@@ -429,6 +439,10 @@ class SpecaCache:
     def update_forecast(self, feats, t_ref, t_target, outs, mask=None, active=None, spec_count=None, rearm=None, stream=None):
         """A whole reference step and the first forecast after it in one launch (commits the step)."""
         speca_cache_update_forecast(self.handle, feats, t_ref, mask, t_target, active, outs, spec_count, rearm, stream)
+
+    def update_forecast_multi(self, feats, t_ref, t_targets, outs, mask=None, active=None, spec_count=None, rearm=None, stream=None):
+        """The same for K speculative times: outs[e] is [K, B, N_e, D]."""
+        speca_cache_update_forecast_multi(self.handle, feats, t_ref, mask, t_targets, active, outs, spec_count, rearm, stream)
 
     def commit_step(self):
         speca_cache_commit_step(self.handle)

@@ -541,9 +541,19 @@ speca_status_t speca_cache_update_forecast(speca_cache_t* c, const void* const* 
                                            const uint8_t* host_sample_mask, const double* t_target,
                                            const uint8_t* dev_active_mask, void* const* outs, int32_t* dev_spec_count,
                                            uint8_t* dev_rearm_mask, void* stream) {
+    return speca_cache_update_forecast_multi(c, feats, t_ref, host_sample_mask, 1, t_target, dev_active_mask, outs,
+                                             dev_spec_count, dev_rearm_mask, stream);
+}
+
+speca_status_t speca_cache_update_forecast_multi(speca_cache_t* c, const void* const* feats, const double* t_ref,
+                                                 const uint8_t* host_sample_mask, int32_t n_targets, const double* t_target,
+                                                 const uint8_t* dev_active_mask, void* const* outs, int32_t* dev_spec_count,
+                                                 uint8_t* dev_rearm_mask, void* stream) {
     if (c == nullptr) return SPECA_ERR_INVALID_ARG;
     if (feats == nullptr || t_ref == nullptr || t_target == nullptr || outs == nullptr)
         return fail(c, SPECA_ERR_INVALID_ARG, "update_forecast: null argument");
+    if (n_targets < 1 || n_targets > SPECA_MAX_HORIZON)
+        return fail(c, SPECA_ERR_INVALID_ARG, "update_forecast: n_targets must be 1..%d", SPECA_MAX_HORIZON);
     if ((dev_spec_count == nullptr) != (dev_rearm_mask == nullptr))
         return fail(c, SPECA_ERR_INVALID_ARG, "update_forecast: give both re-arming buffers or neither");
     if (reinterpret_cast<uintptr_t>(dev_spec_count) % 4 != 0)
@@ -557,9 +567,11 @@ speca_status_t speca_cache_update_forecast(speca_cache_t* c, const void* const* 
         mask[b] = (host_sample_mask == nullptr || host_sample_mask[b] != 0) ? 1 : 0;
         any_sample |= mask[b] != 0;
         if (mask[b] && !std::isfinite(t_ref[b])) return fail(c, SPECA_ERR_INVALID_ARG, "update_forecast: t_ref[%d] not finite", b);
-        if (!std::isfinite(t_target[b])) return fail(c, SPECA_ERR_INVALID_ARG, "update_forecast: t_target[%d] not finite", b);
+        for (int k = 0; k < n_targets; ++k)
+            if (!std::isfinite(t_target[static_cast<size_t>(k) * c->B + b]))
+                return fail(c, SPECA_ERR_INVALID_ARG, "update_forecast: t_target[%d][%d] not finite", k, b);
     }
-    static thread_local FusedParams q;  // 10 KB: kept off the stack
+    static thread_local FusedParams q;  // 20 KB: kept off the stack
     std::memset(&q, 0, sizeof q);
     StreamParams& p = q.up;
     uint64_t bits = 0;
@@ -602,9 +614,12 @@ speca_status_t speca_cache_update_forecast(speca_cache_t* c, const void* const* 
         c->n_refs[b] += 1;
     }
     bool any_forecast = false;
+    q.n_targets = n_targets;
+    q.batch = c->B;
     for (int b = 0; b < c->B; ++b) {
-        int order;
-        forecast_scalars(c, b, t_target[b], &order, q.fc_coef[b]);
+        int order = -1;
+        for (int k = 0; k < n_targets; ++k)
+            forecast_scalars(c, b, t_target[static_cast<size_t>(k) * c->B + b], &order, q.fc_coef[k][b]);
         if (order < 0 && dev_active_mask == nullptr && any_out) {
             roll_back();
             return fail(c, SPECA_ERR_STATE, "update_forecast: sample %d has no reference, in this step or before", b);

@@ -88,8 +88,10 @@ struct FusedParams {
     StreamParams up;                  // the update half: io = features, order / coef as for an update
     const uint8_t* fc_mask;           // device, per sample, may be null: consulted for samples NOT updated here
     int8_t fc_order[SPECA_MAX_BATCH]; // order of the forecast after this step (-1: nothing to forecast)
-    float fc_coef[SPECA_MAX_BATCH][kCoef];  // Horner multipliers relative to the history after this step
-    void* out[SPECA_MAX_ENTRIES];     // per entry: forecast output; null = update only
+    int32_t n_targets;                // K speculative times forecast in this pass (1..SPECA_MAX_HORIZON)
+    int32_t batch;
+    float fc_coef[SPECA_MAX_HORIZON][SPECA_MAX_BATCH][kCoef];  // per target: Horner multipliers relative to the history after this step
+    void* out[SPECA_MAX_ENTRIES];     // per entry: [K, B, N_e, D] forecast output; null = update only
 };
 
 // Arguments of the multi-horizon forecast: K targets evaluated from one read of the table.

@@ -349,10 +349,14 @@ __device__ __forceinline__ void update_tile(char* __restrict__ plane0, uint64_t 
 // table again. Reads f and planes 0..V-1, writes planes 0..V and the forecast: 2V + 3 words per element
 // instead of (2V + 2) + (V + 2). The forecast is evaluated from the ROUNDED planes, exactly as a
 // forecast launch would find them in memory, so the result is bit for bit that of the two calls.
+// With several speculative times (mu[k] per target, outputs target_stride bytes apart) the planes stay
+// in registers and only the Horner pass and the store repeat: 2V + 2 + K words per element.
 template <int DT, int V, int W, int NT, int U>
 __device__ __forceinline__ void update_forecast_tile(char* __restrict__ plane0, uint64_t stride,
-                                                     const char* __restrict__ feat, char* __restrict__ out, uint32_t cnt,
-                                                     const float (&r)[kCoef], const float (&mu)[kCoef]) {
+                                                     const char* __restrict__ feat, char* __restrict__ out,
+                                                     uint64_t target_stride, int n_targets, uint32_t cnt,
+                                                     const float (&r)[kCoef],
+                                                     const float (*__restrict__ mu)[SPECA_MAX_BATCH][kCoef], uint32_t sample) {
     constexpr int EPV = W / Elem<DT>::kBytes;
     const uint32_t nvec = cnt / EPV;
     Vec<W> fv[U];
@@ -384,23 +388,35 @@ __device__ __forceinline__ void update_forecast_tile(char* __restrict__ plane0, 
 #pragma unroll
             for (int i = 0; i < V; ++i)
                 store_vec<W>(plane0 + (i + 1) * stride + static_cast<size_t>(idx) * W, d[i][u]);
-            // Horner over the stored values: acc = D_V; acc = D_{i-1} + acc * mu_i
-            float acc[EPV];
-            if constexpr (V > 0)
-                unpack_vec<DT, W>(d[V - 1][u], acc);
-            else
-                unpack_vec<DT, W>(fv[u], acc);
+        }
+    }
+    // Horner over the stored values, once per target: acc = D_V; acc = D_{i-1} + acc * mu_i
+#pragma unroll 1
+    for (int t = 0; t < n_targets; ++t) {
+        float m[kCoef];
 #pragma unroll
-            for (int i = V; i >= 1; --i) {
-                float lo[EPV];
-                if (i == 1)
-                    unpack_vec<DT, W>(fv[u], lo);
+        for (int i = 0; i < kCoef; ++i) m[i] = mu[t][sample][i];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t idx = u * NT + threadIdx.x;
+            if (idx < nvec) {
+                float acc[EPV];
+                if constexpr (V > 0)
+                    unpack_vec<DT, W>(d[V - 1][u], acc);
                 else
-                    unpack_vec<DT, W>(d[i - 2 >= 0 ? i - 2 : 0][u], lo);
+                    unpack_vec<DT, W>(fv[u], acc);
 #pragma unroll
-                for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], mu[i - 1], lo[k]);
+                for (int i = V; i >= 1; --i) {
+                    float lo[EPV];
+                    if (i == 1)
+                        unpack_vec<DT, W>(fv[u], lo);
+                    else
+                        unpack_vec<DT, W>(d[i - 2 >= 0 ? i - 2 : 0][u], lo);
+#pragma unroll
+                    for (int k = 0; k < EPV; ++k) acc[k] = fmaf(acc[k], m[i - 1], lo[k]);
+                }
+                store_vec<W>(out + t * target_stride + static_cast<size_t>(idx) * W, pack_vec<DT, W>(acc));
             }
-            store_vec<W>(out + static_cast<size_t>(idx) * W, pack_vec<DT, W>(acc));
         }
     }
     for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += NT) {
@@ -416,10 +432,12 @@ __device__ __forceinline__ void update_forecast_tile(char* __restrict__ plane0, 
             store_scalar<DT>(plane0 + (i + 1) * stride, j, c);
             neu[i + 1] = round_storage<DT>(c);
         }
-        float acc = neu[V];
+        for (int t = 0; t < n_targets; ++t) {
+            float acc = neu[V];
 #pragma unroll
-        for (int i = V; i >= 1; --i) acc = fmaf(acc, mu[i - 1], neu[i - 1]);
-        store_scalar<DT>(out, j, acc);
+            for (int i = V; i >= 1; --i) acc = fmaf(acc, mu[t][sample][i - 1], neu[i - 1]);
+            store_scalar<DT>(out + t * target_stride, j, acc);
+        }
     }
 }
 
@@ -592,84 +610,6 @@ __global__ void __launch_bounds__(NT, MINB) stream_kernel(const __grid_constant_
     }
 }
 
-// The fused reference step: stream_kernel's walk over the update's tile list with, per tile, one of
-//   sample updated, output given      -> update_forecast_tile
-//   sample updated, no output         -> update_tile
-//   sample not updated but forecast   -> forecast_tile from its unchanged planes
-// Launch shape: the update's for the order (the mix is write-heavy: V + 2 of 2V + 3 streams are stores).
-template <int DT, int V, int W, int NT, int U, int C, int MINB>
-__global__ void __launch_bounds__(NT, MINB) update_forecast_kernel(const __grid_constant__ FusedParams q) {
-    constexpr uint32_t kChunk = static_cast<uint32_t>(NT) * U * W / Elem<DT>::kBytes;  // elements
-    constexpr uint32_t kTile = kChunk * C;
-    const StreamParams& p = q.up;
-    if (p.act_active != nullptr && blockIdx.x == 0 && threadIdx.x < SPECA_MAX_BATCH && ((p.act_bits >> threadIdx.x) & 1ull)) {
-        p.act_active[threadIdx.x] = 1;
-        p.act_spec[threadIdx.x] = 0;
-    }
-    uint32_t seg = p.seg_lo, seg_first = 0, seg_end = 0;
-    SegDesc sd = {};
-    int v_up = -1, v_fc = -1;
-    char* in = nullptr;
-    char* out = nullptr;
-    float r[kCoef] = {}, mu[kCoef] = {};
-    for (uint32_t tile = p.tile_lo + blockIdx.x; tile < p.tile_hi; tile += gridDim.x) {
-        if (tile >= seg_end) {
-            seg = next_segment(p.tile_start, seg, p.seg_hi, tile, seg_first, seg_end);
-            sd = p.segs[seg];
-            v_up = p.order[sd.sample];
-            v_fc = q.fc_order[sd.sample];
-            in = static_cast<char*>(p.io[sd.entry]);
-            out = static_cast<char*>(q.out[sd.entry]);
-            // a sample that is not updated here is forecast only if it is still speculating
-            if (v_up < 0 && q.fc_mask != nullptr && q.fc_mask[sd.sample] == 0) v_fc = -1;
-#pragma unroll
-            for (int i = 0; i < kCoef; ++i) {
-                r[i] = p.coef[sd.sample][i];
-                mu[i] = q.fc_coef[sd.sample][i];
-            }
-        }
-        const bool do_up = v_up >= 0 && in != nullptr, do_fc = v_fc >= 0 && out != nullptr;
-        if (!do_up && !do_fc) continue;
-        const uint32_t elem0 = (tile - seg_first) * kTile;
-        const uint32_t cnt = min(kTile, sd.n_elems - elem0);
-        const uint64_t byte0 = static_cast<uint64_t>(elem0) * Elem<DT>::kBytes;
-        char* plane0 = p.arena + sd.plane0_off + byte0;
-        char* frow = do_up ? in + sd.io_off + byte0 : nullptr;
-        char* orow = do_fc ? out + sd.io_off + byte0 : nullptr;
-        const bool aligned = ((reinterpret_cast<uintptr_t>(frow) | reinterpret_cast<uintptr_t>(orow)) & (W - 1)) == 0;
-        if (do_up && do_fc && v_up == V && v_fc == V && aligned) {
-            for (uint32_t done = 0; done < cnt; done += kChunk) {
-                const size_t off = static_cast<size_t>(done) * Elem<DT>::kBytes;
-                update_forecast_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, frow + off, orow + off,
-                                                      min(kChunk, cnt - done), r, mu);
-            }
-            continue;
-        }
-        // the rare shapes: halves done one after the other by the single-purpose routines
-        if (do_up) {
-            if (v_up == V && (reinterpret_cast<uintptr_t>(frow) & (W - 1)) == 0) {
-                for (uint32_t done = 0; done < cnt; done += kChunk) {
-                    const size_t off = static_cast<size_t>(done) * Elem<DT>::kBytes;
-                    update_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, frow + off, min(kChunk, cnt - done), r);
-                }
-            } else {
-                update_tile_any<DT>(plane0, sd.plane_stride, frow, cnt, v_up, r);
-            }
-        }
-        if (do_fc) {
-            if (do_up) __syncthreads();  // the forecast may read a plane element another thread of the CTA has just written
-            if (v_fc == V && (reinterpret_cast<uintptr_t>(orow) & (W - 1)) == 0) {
-                for (uint32_t done = 0; done < cnt; done += kChunk) {
-                    const size_t off = static_cast<size_t>(done) * Elem<DT>::kBytes;
-                    forecast_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, orow + off, min(kChunk, cnt - done), mu, false);
-                }
-            } else {
-                forecast_tile_any<DT>(plane0, sd.plane_stride, orow, cnt, v_fc, mu);
-            }
-        }
-    }
-}
-
 // ------------------------------------------------------------------------------------------------
 // multi-horizon forecast: Eq. 2 for K speculative steps from one read of the table
 // ------------------------------------------------------------------------------------------------
@@ -781,6 +721,94 @@ __global__ void __launch_bounds__(NT, MINB) forecast_multi_kernel(const __grid_c
 #pragma unroll
                 for (int i = 0; i < kCoef; ++i) m[i] = p.coef[k][sd.sample][i];
                 forecast_tile_any<DT>(plane0, sd.plane_stride, row + k * target_stride, cnt, v, m, p.weighted != 0);
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// fused reference step: Eq. 3 and the forecasts that follow it, one pass over the tables
+// ------------------------------------------------------------------------------------------------
+// The fused reference step: stream_kernel's walk over the update's tile list with, per tile, one of
+//   sample updated, output given      -> update_forecast_tile (K forecasts from the planes just formed)
+//   sample updated, no output         -> update_tile
+//   sample not updated but forecast   -> forecast_multi_tile from its unchanged planes
+// Launch shape: the update's for the order (the mix is write-heavy: V + 2 of 2V + 3 streams are stores).
+template <int DT, int V, int W, int NT, int U, int C, int MINB>
+__global__ void __launch_bounds__(NT, MINB) update_forecast_kernel(const __grid_constant__ FusedParams q) {
+    constexpr uint32_t kChunk = static_cast<uint32_t>(NT) * U * W / Elem<DT>::kBytes;  // elements
+    constexpr uint32_t kTile = kChunk * C;
+    const StreamParams& p = q.up;
+    if (p.act_active != nullptr && blockIdx.x == 0 && threadIdx.x < SPECA_MAX_BATCH && ((p.act_bits >> threadIdx.x) & 1ull)) {
+        p.act_active[threadIdx.x] = 1;
+        p.act_spec[threadIdx.x] = 0;
+    }
+    const int K = q.n_targets;
+    uint32_t seg = p.seg_lo, seg_first = 0, seg_end = 0;
+    SegDesc sd = {};
+    int v_up = -1, v_fc = -1;
+    char* in = nullptr;
+    char* out = nullptr;
+    uint64_t target_stride = 0;  // bytes between consecutive targets of this entry's output
+    float r[kCoef] = {};
+    for (uint32_t tile = p.tile_lo + blockIdx.x; tile < p.tile_hi; tile += gridDim.x) {
+        if (tile >= seg_end) {
+            seg = next_segment(p.tile_start, seg, p.seg_hi, tile, seg_first, seg_end);
+            sd = p.segs[seg];
+            v_up = p.order[sd.sample];
+            v_fc = q.fc_order[sd.sample];
+            in = static_cast<char*>(p.io[sd.entry]);
+            out = static_cast<char*>(q.out[sd.entry]);
+            target_stride = static_cast<uint64_t>(q.batch) * sd.n_elems * Elem<DT>::kBytes;
+            // a sample that is not updated here is forecast only if it is still speculating
+            if (v_up < 0 && q.fc_mask != nullptr && q.fc_mask[sd.sample] == 0) v_fc = -1;
+#pragma unroll
+            for (int i = 0; i < kCoef; ++i) r[i] = p.coef[sd.sample][i];
+        }
+        const bool do_up = v_up >= 0 && in != nullptr, do_fc = v_fc >= 0 && out != nullptr;
+        if (!do_up && !do_fc) continue;
+        const uint32_t elem0 = (tile - seg_first) * kTile;
+        const uint32_t cnt = min(kTile, sd.n_elems - elem0);
+        const uint64_t byte0 = static_cast<uint64_t>(elem0) * Elem<DT>::kBytes;
+        char* plane0 = p.arena + sd.plane0_off + byte0;
+        char* frow = do_up ? in + sd.io_off + byte0 : nullptr;
+        char* orow = do_fc ? out + sd.io_off + byte0 : nullptr;
+        const bool out_aligned = ((reinterpret_cast<uintptr_t>(orow) | (K > 1 ? target_stride : 0)) & (W - 1)) == 0;
+        const bool in_aligned = (reinterpret_cast<uintptr_t>(frow) & (W - 1)) == 0;
+        if (do_up && do_fc && v_up == V && v_fc == V && in_aligned && out_aligned) {
+            for (uint32_t done = 0; done < cnt; done += kChunk) {
+                const size_t off = static_cast<size_t>(done) * Elem<DT>::kBytes;
+                update_forecast_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, frow + off, orow + off, target_stride, K,
+                                                      min(kChunk, cnt - done), r, q.fc_coef, sd.sample);
+            }
+            continue;
+        }
+        // the rare shapes: halves done one after the other by the single-purpose routines
+        if (do_up) {
+            if (v_up == V && in_aligned) {
+                for (uint32_t done = 0; done < cnt; done += kChunk) {
+                    const size_t off = static_cast<size_t>(done) * Elem<DT>::kBytes;
+                    update_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, frow + off, min(kChunk, cnt - done), r);
+                }
+            } else {
+                update_tile_any<DT>(plane0, sd.plane_stride, frow, cnt, v_up, r);
+            }
+        }
+        if (do_fc) {
+            if (do_up) __syncthreads();  // the forecast may read a plane element another thread of the CTA has just written
+            if (v_fc == V && out_aligned) {
+                for (uint32_t done = 0; done < cnt; done += kChunk) {
+                    const size_t off = static_cast<size_t>(done) * Elem<DT>::kBytes;
+                    forecast_multi_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, orow + off, target_stride, K,
+                                                         min(kChunk, cnt - done), q.fc_coef, sd.sample, false);
+                }
+            } else {
+                for (int t = 0; t < K; ++t) {
+                    float m[kCoef];
+#pragma unroll
+                    for (int i = 0; i < kCoef; ++i) m[i] = q.fc_coef[t][sd.sample][i];
+                    forecast_tile_any<DT>(plane0, sd.plane_stride, orow + t * target_stride, cnt, v_fc, m);
+                }
             }
         }
     }
@@ -1633,13 +1661,14 @@ __global__ void __launch_bounds__(kThreads, V <= 2 ? SPECA_VERIFY_MINB : 2) veri
 
     // Last cluster to arrive. A sample's partials sit side by side in the scratch ([sample][cluster]).
     // A group of L lanes adds one sample's partials: with few samples each has many partials and a
-    // whole warp takes one sample; with many samples each has few and a warp takes four at a time.
+    // whole warp takes one sample; with many samples each has few and a warp takes four or eight at a
+    // time, so that the CTA's eight warps cover the batch in one pass.
     // Per sample the order is fixed (lane l adds clusters q_lo + l, q_lo + l + L, ..., then a shuffle
     // tree over the group), four loads per lane are in flight at once, and the sums are fp64.
     // the continuation rule's own inputs are asked for now and used after the sums
     SelectIn sel_in = {};
     if (p.sel_active != nullptr && warp == 0) sel_in = select_load(p.batch, p.sel_spec, p.dev_mask);
-    const uint32_t L = n_active > 8 ? 8 : 32, per_warp = 32 / L;
+    const uint32_t L = n_active <= 8 ? 32 : (n_active <= 32 ? 8 : 4), per_warp = 32 / L;
     const uint32_t g = lane / L, l = lane % L;
     const bool holes = Q > T;  // more clusters than tiles: some clusters in a sample's span own nothing
     for (uint32_t a0 = 0; a0 < n_active; a0 += kWarps * per_warp) {  // uniform over the CTA

@@ -65,6 +65,7 @@ int main(void) {
         CHECK(speca_cache_stats(NULL, &st) == SPECA_ERR_INVALID_ARG);
     }
     CHECK(speca_cache_update_forecast(NULL, NULL, NULL, NULL, NULL, NULL, NULL, NULL, NULL, NULL) == SPECA_ERR_INVALID_ARG);
+    CHECK(speca_cache_update_forecast_multi(NULL, NULL, NULL, NULL, 2, NULL, NULL, NULL, NULL, NULL, NULL) == SPECA_ERR_INVALID_ARG);
     CHECK(speca_cache_check(NULL, NULL) == SPECA_ERR_INVALID_ARG);
     CHECK(speca_verify_decide(SPECA_METRIC_L2, NULL, 1, NULL, 0.f, NULL, NULL, NULL, NULL) == SPECA_ERR_INVALID_ARG);
     CHECK(speca_verify_pred_static(NULL, NULL, 8, 1, SPECA_BF16, NULL, 0.f, NULL, NULL, NULL, 0, NULL) ==

@@ -180,3 +180,55 @@ def test_fused_reference_step_at_full_size(S):
         del feats
     a.close()
     b.close()
+
+
+@pytest.mark.parametrize("dtype,tdt", [(1, torch.bfloat16), (0, torch.float32)])
+@pytest.mark.parametrize("m,K", [(0, 2), (1, 8), (2, 3), (2, 8), (3, 2), (4, 5)])
+def test_fused_reference_step_with_several_targets_equals_update_commit_forecast_multi(S, dtype, tdt, m, K):
+    """K speculative times forecast in the reference step's own pass: tables and all K forecasts bit for bit
+    those of update + commit + speca_forecast_multi (which the multi-horizon tests hold against the oracle),
+    with warm-up orders, a sample that skips a step and keeps speculating, one that has dropped out, and an
+    entry that is only updated."""
+    B, ne = 3, len(ENTRIES)
+    a = S.SpecaCache(ENTRIES, B, m, dtype, DEV)
+    b = S.SpecaCache(ENTRIES, B, m, dtype, DEV)
+    gen = torch.Generator(device=DEV).manual_seed(7 * m + K)
+    active = torch.tensor([1, 1, 1], dtype=torch.uint8, device=DEV)
+    active_b = active.clone()
+    spec_a, spec_b = torch.zeros(B, dtype=torch.int32, device=DEV), torch.zeros(B, dtype=torch.int32, device=DEV)
+    t = 1.0
+    for k, mask in enumerate([[1, 1, 1]] * (m + 1) + [[1, 0, 1], [0, 1, 1], [1, 1, 1]]):
+        t -= 0.04
+        t_ref = [t - 0.002 * s for s in range(B)]
+        targets = [[x - 0.006 * (j + 1) for x in t_ref] for j in range(K)]
+        if k == m + 2:
+            active[0] = 0                                    # sample 0 skips this step AND has dropped out: no forecast
+            active_b[0] = 0                                  # (the next step, which it takes, re-arms it)
+        feats = [torch.randn(B, n, d, generator=gen, device=DEV).to(tdt) for n, d in ENTRIES]
+        outs_a = [torch.full((K, B, n, d), 7.0, dtype=tdt, device=DEV) for n, d in ENTRIES]
+        outs_b = [torch.full((K, B, n, d), 7.0, dtype=tdt, device=DEV) for n, d in ENTRIES]
+        skip = k % ne
+        give_a = [None if e == skip else o for e, o in enumerate(outs_a)]
+        give_b = [None if e == skip else o for e, o in enumerate(outs_b)]
+        a.update_forecast_multi(feats, t_ref, targets, give_a, mask=mask, active=active, spec_count=spec_a, rearm=active)
+        b.update_activate(feats, t_ref, mask, spec_b, active_b)
+        b.commit_step()
+        b.forecast_multi(targets, give_b, active_b)
+        torch.cuda.synchronize()
+        assert torch.equal(active, active_b) and torch.equal(spec_a, spec_b)
+        refs = a.state()[0]
+        assert refs == b.state()[0]
+        for e in range(ne):
+            for s in range(B):
+                live = min(m, refs[s] - 1) + 1
+                assert torch.equal(bits(a.plane_tensor(e, s)[:live]), bits(b.plane_tensor(e, s)[:live])), ("planes", k, e, s)
+            assert torch.equal(bits(outs_a[e]), bits(outs_b[e])), ("forecasts", k, e)
+            if e == skip:
+                assert bool((outs_a[e].float() == 7.0).all())
+        if k == m + 2:
+            assert bool((outs_a[(skip + 1) % ne][:, 0].float() == 7.0).all())     # the dropped-out sample's rows are untouched
+    assert a.stats()["update_forecast_launches"] == m + 4
+    with pytest.raises(S.SpecaError):
+        a.update_forecast_multi(feats, [t - 1.0] * B, [[0.0] * B] * 9, give_a)   # more targets than SPECA_MAX_HORIZON
+    a.close()
+    b.close()
