@@ -381,6 +381,42 @@ def time_fused_reference_step(h: Harness, peak: float, reps: int = 20):
             "traffic_saved_vs_two_launches": 1.0 - nbytes / float(ab["update"] + ab["forecast"])}
 
 
+def time_fused_reference_step_multi(h: Harness, peak: float, K: int = 4, reps: int = 10):
+    """The same with K speculative times forecast in the reference step's pass (speca_cache_update_forecast_multi):
+    2 * order + 2 + K words per element against (2 * order + 2) + (order + 1 + K) for update + speca_forecast_multi."""
+    w, dev = h.w, h.device
+    m, eb = w.max_order, w.elem_bytes
+    outs = [torch.empty(K, h.B, n, d, dtype=w.torch_dtype, device=dev) for n, d in w.entries]
+    nbytes = (2 * m + 2 + K) * eb * w.elems_per_order
+    two_bytes = ((2 * m + 2) + (m + 1 + K)) * eb * w.elems_per_order
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    res = {}
+    for name in ("fused", "two_launches"):
+        total = 0.0
+        for r in range(reps + 3):
+            j = h.j
+            h.j += 1
+            t_ref, _ = h.times_for(j)
+            targets = [[t_ref[0] - 0.003 * (k + 1)] * h.B for k in range(K)]
+            e0.record()
+            if name == "fused":
+                h.cache.update_forecast_multi(h.feats[j & 1], t_ref, targets, outs)
+            else:
+                h.cache.update(h.feats[j & 1], t_ref)
+                h.cache.commit_step()
+                h.cache.forecast_multi(targets, outs)
+            e1.record()
+            torch.cuda.synchronize(dev)
+            if r >= 3:
+                total += e0.elapsed_time(e1)
+        res[name + "_ms"] = total / reps
+    del outs
+    torch.cuda.empty_cache()
+    gbs = nbytes / (res["fused_ms"] * 1e-3) / 1e9
+    return dict(res, targets=K, algorithmic_bytes=nbytes, gbs=gbs, frac_of_measured_peak=gbs / peak,
+                bytes_of_the_two_launches=two_bytes, speedup_vs_two_launches=res["two_launches_ms"] / res["fused_ms"])
+
+
 def time_update_per_entry(h: Harness, reps: int = 5):
     """A model hands over one block output at a time: the same reference step as one launch per entry."""
     w, dev = h.w, h.device
@@ -1150,6 +1186,8 @@ def main(argv=None):
         detail["verify_metrics"] = time_metrics(h)
     if args.full and tables:
         detail["multi_horizon"] = time_multi_horizon(h, peak, per_ms["forecast"])
+        if path in (0, 3):
+            detail["fused_reference_step_4_targets"] = time_fused_reference_step_multi(h, peak)
         try:
             detail["speculative_run_as_cuda_graph"] = time_graph_replay(h)
         except Exception as exc:  # report, do not hide
