@@ -81,6 +81,14 @@ def test_nothing_is_written_outside_the_buffers(S, path, dtype, tdt, m):
             S.speca_cache_update_forecast(handle, [f.t for f in ffeats], [t_new] * B, [1, 0, 1], [t_new - 0.02] * B, active.t,
                                           [o.t for o in fouts], spec.t, active.t)
             fouts += ffeats
+            # and with two speculative times in the same pass
+            mf = [Guarded((2, B, n, d), tdt, offset=shift) for n, d in RAGGED]
+            for f in ffeats:
+                f.t.copy_(torch.randn(f.t.shape, generator=gen, device=DEV).to(tdt))
+            S.speca_cache_update_forecast_multi(handle, [f.t for f in ffeats], [t_new - 0.03] * B, [0, 1, 1],
+                                                [[t_new - 0.04] * B, [t_new - 0.05] * B], active.t, [o.t for o in mf],
+                                                spec.t, active.t)
+            fouts += mf
         torch.cuda.synchronize()
         for g in outs + mouts + fouts + [pred, err, acc, sums, total, spec, active, idx, n_act, arena]:
             assert g.intact(), "a guard zone was overwritten (path %d, dtype %d, order %d, shift %d)" % (path, dtype, m, shift)
