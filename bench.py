@@ -1123,7 +1123,7 @@ def main(argv=None):
                          "the last references (speca_layout_t)")
     ap.add_argument("--separate-select", action="store_true",
                     help="five launches per step (update, activate, forecast, verify, select) instead of the three fused ones")
-    ap.add_argument("--detail", default=os.path.join("gpurun_out", "bench_detail.json"),
+    ap.add_argument("--detail", default="bench_detail.json",
                     help="JSON file for everything that does not belong in the last line ('' = none)")
     ap.add_argument("--full", action="store_true",
                     help="also run the sweeps reported only in the detail file: multi-horizon and summed forecasts, "

@@ -37,7 +37,7 @@ def _canned_line(n_gpus=1):
                             config=bench.workload_config(w), roofline=roofline, cpu_baseline=cpu, e2e=e2e,
                             gpu_launches=600, clocks=clocks, kernels=kernels, forecast_verify_gbs=6800.123456,
                             speculative_steps_per_s=1040.123456, also=also,
-                            detail_path=os.path.join("gpurun_out", "bench_detail.json"))
+                            detail_path="bench_detail.json")
 
 
 def test_line_is_compact_and_carries_the_contract_keys():
