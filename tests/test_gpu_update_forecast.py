@@ -232,3 +232,43 @@ def test_fused_reference_step_with_several_targets_equals_update_commit_forecast
         a.update_forecast_multi(feats, [t - 1.0] * B, [[0.0] * B] * 9, give_a)   # more targets than SPECA_MAX_HORIZON
     a.close()
     b.close()
+
+
+def test_fused_reference_step_can_be_captured_into_a_cuda_graph(S):
+    """The call neither allocates nor synchronises: captured once into a CUDA graph (nothing runs during the
+    capture; the host-side history advances then) and replayed, it leaves the same tables and forecasts
+    as the eager call on a twin cache."""
+    entries = [(40, 1030), (301, 1152)]
+    B, m = 4, 2
+    gen = torch.Generator(device=DEV).manual_seed(91)
+    a = S.SpecaCache(entries, B, m, 1, DEV)
+    b = S.SpecaCache(entries, B, m, 1, DEV)
+    feats = [torch.randn(B, n, d, generator=gen, device=DEV).bfloat16() for n, d in entries]
+    for k, t in enumerate((1.0, 0.93)):                      # two ordinary reference steps on both
+        f0 = [torch.randn(B, n, d, generator=gen, device=DEV).bfloat16() for n, d in entries]
+        for c in (a, b):
+            c.update(f0, [t] * B)
+            c.commit_step()
+    outs_a = [torch.zeros(B, n, d, dtype=torch.bfloat16, device=DEV) for n, d in entries]
+    outs_b = [torch.zeros(B, n, d, dtype=torch.bfloat16, device=DEV) for n, d in entries]
+    act = torch.ones(B, dtype=torch.uint8, device=DEV)
+    a.update_forecast(feats, [0.9] * B, [0.87] * B, outs_a, mask=[1, 1, 0, 1], active=act)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream(DEV)
+    side.wait_stream(torch.cuda.current_stream(DEV))
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            b.update_forecast(feats, [0.9] * B, [0.87] * B, outs_b, mask=[1, 1, 0, 1], active=act)
+    torch.cuda.current_stream(DEV).wait_stream(side)
+    torch.cuda.synchronize()
+    assert all(bool((o == 0).all()) for o in outs_b)          # captured, not run
+    assert a.state()[0] == b.state()[0] == [3, 3, 2, 3]       # the history advanced at capture time
+    graph.replay()
+    torch.cuda.synchronize()
+    for e in range(len(entries)):
+        assert torch.equal(bits(outs_a[e]), bits(outs_b[e]))
+        for s in range(B):
+            assert torch.equal(bits(a.plane_tensor(e, s)), bits(b.plane_tensor(e, s)))
+    a.close()
+    b.close()
