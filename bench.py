@@ -153,7 +153,7 @@ class Harness:
                  layout: int = 0):
         from paper_2509_11628_b200 import binding as S
         self.S, self.w, self.device = S, w, torch.device(device)
-        self.fused_select = fused_select
+        self.fused_select, self.layout = fused_select, layout
         self.B, self.m = w.batch, w.max_order
         self.cache = S.SpecaCache(w.entries, w.batch, w.max_order, w.dtype, device, path=path, layout=layout)
         self.src = W.FeatureSource(w, device, seed_offset)
@@ -364,14 +364,17 @@ def time_fused_reference_step(h: Harness, peak: float, reps: int = 20):
     """A reference step and the first forecast after it as ONE launch (speca_cache_update_forecast): the
     forecast is evaluated from the planes the update has just formed, so the tables are not read again --
     2 * order + 3 words per element (order + 2 of them writes) instead of (2 * order + 2) + (order + 2).
+    A cache that keeps raw features copies the feature into its ring plane and sums the planes with the
+    feature still in registers: order + 3 words instead of 2 + (order + 2).
     The verification entry is only updated (its forecast comes out of the verification launch)."""
     w, dev = h.w, h.device
     others = list(h.outs)
     others[w.vidx] = None
     m, eb = w.max_order, w.elem_bytes
     n_ver = w.batch * w.entry_elems(w.vidx)
-    nbytes = (2 * m + 3) * eb * (w.elems_per_order - n_ver) + (2 * m + 2) * eb * n_ver
-    ab = algorithmic_bytes(w, m)
+    ab = algorithmic_bytes(w, m, layout=h.layout)
+    # the update's traffic, one more store where a forecast is written and, for raw features, the other planes' reads
+    nbytes = ab["update"] + (1 + (m if h.layout == 1 else 0)) * eb * (w.elems_per_order - n_ver)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     total = 0.0
     for r in range(reps + 3):
@@ -1188,7 +1191,7 @@ def main(argv=None):
 
     tables = solo and layout == 0      # these calls exist for the table layout only
     fused = None
-    if layout == 0 and path in (0, 3):
+    if path in (0, 3):
         fused = time_fused_reference_step(h, peak)
         fused["ms_of_the_two_launches"] = per_ms["update"] + per_ms["forecast"]
         fused["speedup_vs_two_launches"] = fused["ms_of_the_two_launches"] / fused["ms"]

@@ -243,7 +243,10 @@ speca_status_t speca_cache_update_activate(speca_cache_t* cache, const void* con
  *   dev_spec_count, dev_rearm_mask   both or neither: as speca_cache_update_activate, the samples
  *                    of host_sample_mask are marked active in dev_rearm_mask and their counters
  *                    cleared (dev_rearm_mask may be the buffer dev_active_mask names).
- * Difference-table caches (SPECA_LAYOUT_TABLES) on the default kernel path only. On error nothing is
+ * A cache that keeps raw features (SPECA_LAYOUT_HISTORY) takes the same call: the feature is copied into
+ * its ring plane and the weighted sum is formed with it still in registers, v + 3 words per element
+ * instead of 2 + (v + 2); an entry given as SPECA_FEATURE_IN_PLACE, or as the pointer speca_cache_next_slot
+ * returned, is not copied and only forecast. The default kernel path only. On error nothing is
  * enqueued and the history is unchanged. Errors: INVALID_ARG, ALIGNMENT, ZERO_GAP, STATE (a reference
  * step is open; or a sample has no reference and no device mask is given), UNSUPPORTED, CUDA.
  */

@@ -558,8 +558,8 @@ speca_status_t speca_cache_update_forecast_multi(speca_cache_t* c, const void* c
         return fail(c, SPECA_ERR_INVALID_ARG, "update_forecast: give both re-arming buffers or neither");
     if (reinterpret_cast<uintptr_t>(dev_spec_count) % 4 != 0)
         return fail(c, SPECA_ERR_ALIGNMENT, "update_forecast: dev_spec_count must be 4-byte aligned");
-    if (c->layout != SPECA_LAYOUT_TABLES || c->path != SPECA_PATH_WIDE)
-        return fail(c, SPECA_ERR_UNSUPPORTED, "update_forecast: difference-table caches on the default kernel path only");
+    if (c->path != SPECA_PATH_WIDE) return fail(c, SPECA_ERR_UNSUPPORTED, "update_forecast: the default kernel path only");
+    const bool hist = c->layout == SPECA_LAYOUT_HISTORY;
     if (c->pending) return fail(c, SPECA_ERR_STATE, "update_forecast: a reference step is open (commit it first)");
     uint8_t mask[SPECA_MAX_BATCH];
     bool any_sample = false;
@@ -586,16 +586,37 @@ speca_status_t speca_cache_update_forecast_multi(speca_cache_t* c, const void* c
             p.coef[b][i] = static_cast<float>(1.0 / gap);
         }
         p.order[b] = static_cast<int8_t>(v_new);
+        if (hist) {  // nothing is differenced: the feature goes into the ring plane after the latest one
+            p.order[b] = 0;
+            p.slot[b] = static_cast<uint8_t>(c->n_refs[b] % (c->m + 1));
+        }
     }
+    p.weighted = hist ? 1 : 0;
     const size_t esz = elem_size(c);
     bool any_out = false;
     for (int e = 0; e < c->n_entries; ++e) {
         if (feats[e] == nullptr) return fail(c, SPECA_ERR_INVALID_ARG, "update_forecast: feats[%d] is null (the call is a whole reference step)", e);
-        if (reinterpret_cast<uintptr_t>(feats[e]) % esz != 0 || reinterpret_cast<uintptr_t>(outs[e]) % esz != 0)
-            return fail(c, SPECA_ERR_ALIGNMENT, "update_forecast: feats[%d] / outs[%d] not aligned to the element size", e, e);
-        p.io[e] = const_cast<void*>(feats[e]);
+        if (reinterpret_cast<uintptr_t>(outs[e]) % esz != 0)
+            return fail(c, SPECA_ERR_ALIGNMENT, "update_forecast: outs[%d] not aligned to the element size", e);
         q.out[e] = outs[e];
         any_out |= outs[e] != nullptr;
+        if (feats[e] == SPECA_FEATURE_IN_PLACE) {
+            if (!hist) return fail(c, SPECA_ERR_INVALID_ARG, "update_forecast: SPECA_FEATURE_IN_PLACE needs a cache that keeps raw features");
+            continue;  // the features already sit in their ring planes: nothing to copy, the forecast reads them there
+        }
+        if (reinterpret_cast<uintptr_t>(feats[e]) % esz != 0)
+            return fail(c, SPECA_ERR_ALIGNMENT, "update_forecast: feats[%d] not aligned to the element size", e);
+        if (hist) {  // written straight into the next ring planes (speca_cache_next_slot): nothing to copy either
+            bool in_place = any_sample;
+            for (int b = 0; b < c->B && in_place; ++b) {
+                if (!mask[b]) continue;
+                const SegDesc& sg = c->L.segs[static_cast<size_t>(e) * c->B + b];
+                in_place = static_cast<const char*>(feats[e]) + sg.io_off ==
+                           c->arena + sg.plane0_off + static_cast<size_t>(p.slot[b]) * sg.plane_stride;
+            }
+            if (in_place) continue;
+        }
+        p.io[e] = const_cast<void*>(feats[e]);
     }
     // The forecast's scalars are those of the history AFTER this step: commit on a copy of the host
     // state, keep the copy if anything below fails.
@@ -619,7 +640,7 @@ speca_status_t speca_cache_update_forecast_multi(speca_cache_t* c, const void* c
     for (int b = 0; b < c->B; ++b) {
         int order = -1;
         for (int k = 0; k < n_targets; ++k)
-            forecast_scalars(c, b, t_target[static_cast<size_t>(k) * c->B + b], &order, q.fc_coef[k][b]);
+            forecast_coefficients(c, b, t_target[static_cast<size_t>(k) * c->B + b], &order, q.fc_coef[k][b]);
         if (order < 0 && dev_active_mask == nullptr && any_out) {
             roll_back();
             return fail(c, SPECA_ERR_STATE, "update_forecast: sample %d has no reference, in this step or before", b);
@@ -658,7 +679,7 @@ speca_status_t speca_cache_update_forecast_multi(speca_cache_t* c, const void* c
         const int vf = launch_order(q.fc_order, c->B);
         v = vf > v ? vf : v;
         const uint32_t n_tiles = p.tile_hi - p.tile_lo;
-        const uint32_t full = static_cast<uint32_t>(c->sm_count * fused_ctas_per_sm(v));
+        const uint32_t full = static_cast<uint32_t>(c->sm_count * fused_ctas_per_sm(v, hist));
         const int grid = static_cast<int>(n_tiles < full ? n_tiles : full);
         cudaError_t ce = launch_update_forecast(q, c->dtype, grid, static_cast<cudaStream_t>(stream));
         if (ce != cudaSuccess) {

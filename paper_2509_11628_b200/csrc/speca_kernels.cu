@@ -729,12 +729,85 @@ __global__ void __launch_bounds__(NT, MINB) forecast_multi_kernel(const __grid_c
 // ------------------------------------------------------------------------------------------------
 // fused reference step: Eq. 3 and the forecasts that follow it, one pass over the tables
 // ------------------------------------------------------------------------------------------------
+// The same fusion for a cache that keeps raw features: the reference step copies the feature into ring
+// plane `slot` and the forecast is the weighted sum of the ring's planes, of which plane `slot` is the
+// feature just loaded: V + 1 reads (feature and the V other planes) and 1 + K writes instead of
+// (1 + 1) + (V + 1 + K). Same order of operations as the weighted forecast tiles: acc = w_V * plane_V,
+// then acc += w_i * plane_i for i = V-1 .. 0.
+template <int DT, int V, int W, int NT, int U>
+__device__ __forceinline__ void history_update_forecast_tile(char* __restrict__ plane0, uint64_t stride,
+                                                             const char* __restrict__ feat, char* __restrict__ out,
+                                                             uint64_t target_stride, int n_targets, uint32_t cnt, int slot,
+                                                             const float (*__restrict__ mu)[SPECA_MAX_BATCH][kCoef],
+                                                             uint32_t sample) {
+    constexpr int EPV = W / Elem<DT>::kBytes;
+    const uint32_t nvec = cnt / EPV;
+    Vec<W> d[V + 1][U];  // d[slot] holds the feature
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint32_t idx = u * NT + threadIdx.x;
+        if (idx < nvec) {
+#pragma unroll
+            for (int i = 0; i <= V; ++i)
+                d[i][u] = load_vec<W>((i == slot ? feat : plane0 + i * stride) + static_cast<size_t>(idx) * W);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint32_t idx = u * NT + threadIdx.x;
+        if (idx < nvec) {
+#pragma unroll
+            for (int i = 0; i <= V; ++i)
+                if (i == slot) store_vec<W>(plane0 + i * stride + static_cast<size_t>(idx) * W, d[i][u]);
+        }
+    }
+#pragma unroll 1
+    for (int t = 0; t < n_targets; ++t) {
+        float m[kCoef];
+#pragma unroll
+        for (int i = 0; i < kCoef; ++i) m[i] = mu[t][sample][i];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t idx = u * NT + threadIdx.x;
+            if (idx < nvec) {
+                float acc[EPV];
+                unpack_vec<DT, W>(d[V][u], acc);
+#pragma unroll
+                for (int k = 0; k < EPV; ++k) acc[k] *= m[V];
+#pragma unroll
+                for (int i = V; i >= 1; --i) {
+                    float lo[EPV];
+                    unpack_vec<DT, W>(d[i - 1][u], lo);
+#pragma unroll
+                    for (int k = 0; k < EPV; ++k) acc[k] = fmaf(lo[k], m[i - 1], acc[k]);
+                }
+                store_vec<W>(out + t * target_stride + static_cast<size_t>(idx) * W, pack_vec<DT, W>(acc));
+            }
+        }
+    }
+    for (uint32_t j = nvec * EPV + threadIdx.x; j < cnt; j += NT) {
+        float val[V + 1];
+#pragma unroll
+        for (int i = 0; i <= V; ++i) val[i] = load_scalar<DT>(i == slot ? feat : plane0 + i * stride, j);
+#pragma unroll
+        for (int i = 0; i <= V; ++i)
+            if (i == slot) store_scalar<DT>(plane0 + i * stride, j, val[i]);
+        for (int t = 0; t < n_targets; ++t) {
+            float acc = val[V] * mu[t][sample][V];
+#pragma unroll
+            for (int i = V; i >= 1; --i) acc = fmaf(val[i - 1], mu[t][sample][i - 1], acc);
+            store_scalar<DT>(out + t * target_stride, j, acc);
+        }
+    }
+}
+
 // The fused reference step: stream_kernel's walk over the update's tile list with, per tile, one of
 //   sample updated, output given      -> update_forecast_tile (K forecasts from the planes just formed)
 //   sample updated, no output         -> update_tile
 //   sample not updated but forecast   -> forecast_multi_tile from its unchanged planes
-// Launch shape: the update's for the order (the mix is write-heavy: V + 2 of 2V + 3 streams are stores).
-template <int DT, int V, int W, int NT, int U, int C, int MINB>
+// HIST: a cache that keeps raw features; the update is then a copy into ring plane `slot` and the
+// forecasts are weighted sums (history_update_forecast_tile).
+template <int DT, int V, int W, int NT, int U, int C, int MINB, bool HIST>
 __global__ void __launch_bounds__(NT, MINB) update_forecast_kernel(const __grid_constant__ FusedParams q) {
     constexpr uint32_t kChunk = static_cast<uint32_t>(NT) * U * W / Elem<DT>::kBytes;  // elements
     constexpr uint32_t kTile = kChunk * C;
@@ -744,9 +817,10 @@ __global__ void __launch_bounds__(NT, MINB) update_forecast_kernel(const __grid_
         p.act_spec[threadIdx.x] = 0;
     }
     const int K = q.n_targets;
+    constexpr bool hist = HIST;
     uint32_t seg = p.seg_lo, seg_first = 0, seg_end = 0;
     SegDesc sd = {};
-    int v_up = -1, v_fc = -1;
+    int v_up = -1, v_fc = -1, slot = 0;
     char* in = nullptr;
     char* out = nullptr;
     uint64_t target_stride = 0;  // bytes between consecutive targets of this entry's output
@@ -760,6 +834,7 @@ __global__ void __launch_bounds__(NT, MINB) update_forecast_kernel(const __grid_
             in = static_cast<char*>(p.io[sd.entry]);
             out = static_cast<char*>(q.out[sd.entry]);
             target_stride = static_cast<uint64_t>(q.batch) * sd.n_elems * Elem<DT>::kBytes;
+            slot = p.slot[sd.sample];
             // a sample that is not updated here is forecast only if it is still speculating
             if (v_up < 0 && q.fc_mask != nullptr && q.fc_mask[sd.sample] == 0) v_fc = -1;
 #pragma unroll
@@ -775,17 +850,32 @@ __global__ void __launch_bounds__(NT, MINB) update_forecast_kernel(const __grid_
         char* orow = do_fc ? out + sd.io_off + byte0 : nullptr;
         const bool out_aligned = ((reinterpret_cast<uintptr_t>(orow) | (K > 1 ? target_stride : 0)) & (W - 1)) == 0;
         const bool in_aligned = (reinterpret_cast<uintptr_t>(frow) & (W - 1)) == 0;
-        if (do_up && do_fc && v_up == V && v_fc == V && in_aligned && out_aligned) {
+        if (do_up && do_fc && v_fc == V && (hist || v_up == V) && in_aligned && out_aligned) {
             for (uint32_t done = 0; done < cnt; done += kChunk) {
                 const size_t off = static_cast<size_t>(done) * Elem<DT>::kBytes;
-                update_forecast_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, frow + off, orow + off, target_stride, K,
-                                                      min(kChunk, cnt - done), r, q.fc_coef, sd.sample);
+                if (hist)
+                    history_update_forecast_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, frow + off, orow + off,
+                                                                  target_stride, K, min(kChunk, cnt - done), slot, q.fc_coef,
+                                                                  sd.sample);
+                else
+                    update_forecast_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, frow + off, orow + off, target_stride,
+                                                          K, min(kChunk, cnt - done), r, q.fc_coef, sd.sample);
             }
             continue;
         }
         // the rare shapes: halves done one after the other by the single-purpose routines
         if (do_up) {
-            if (v_up == V && in_aligned) {
+            if (hist) {  // a copy into the ring plane
+                char* dst = plane0 + static_cast<size_t>(slot) * sd.plane_stride;
+                if (in_aligned) {
+                    for (uint32_t done = 0; done < cnt; done += kChunk) {
+                        const size_t off = static_cast<size_t>(done) * Elem<DT>::kBytes;
+                        update_tile<DT, 0, W, NT, U>(dst + off, sd.plane_stride, frow + off, min(kChunk, cnt - done), r);
+                    }
+                } else {
+                    update_tile_any<DT>(dst, sd.plane_stride, frow, cnt, 0, r);
+                }
+            } else if (v_up == V && in_aligned) {
                 for (uint32_t done = 0; done < cnt; done += kChunk) {
                     const size_t off = static_cast<size_t>(done) * Elem<DT>::kBytes;
                     update_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, frow + off, min(kChunk, cnt - done), r);
@@ -800,14 +890,14 @@ __global__ void __launch_bounds__(NT, MINB) update_forecast_kernel(const __grid_
                 for (uint32_t done = 0; done < cnt; done += kChunk) {
                     const size_t off = static_cast<size_t>(done) * Elem<DT>::kBytes;
                     forecast_multi_tile<DT, V, W, NT, U>(plane0 + off, sd.plane_stride, orow + off, target_stride, K,
-                                                         min(kChunk, cnt - done), q.fc_coef, sd.sample, false);
+                                                         min(kChunk, cnt - done), q.fc_coef, sd.sample, hist);
                 }
             } else {
                 for (int t = 0; t < K; ++t) {
                     float m[kCoef];
 #pragma unroll
                     for (int i = 0; i < kCoef; ++i) m[i] = q.fc_coef[t][sd.sample][i];
-                    forecast_tile_any<DT>(plane0, sd.plane_stride, orow + t * target_stride, cnt, v_fc, m);
+                    forecast_tile_any<DT>(plane0, sd.plane_stride, orow + t * target_stride, cnt, v_fc, m, hist);
                 }
             }
         }
@@ -1914,37 +2004,57 @@ cudaError_t launch_forecast(const StreamParams& p, int dtype, int path, int grid
 #define SPECA_SHAPES_FUSED \
     {32, 256, 1, 4, 2}, {32, 256, 2, 2, 1}, {32, 256, 2, 2, 1}, {32, 256, 2, 2, 1}, { 32, 256, 2, 2, 1 }
 #endif
-__host__ __device__ constexpr Shape fused_shape(int v) {
+// Raw-feature caches: order + 1 loads and two stores per element. Measured on 20 FLUX-shaped entries
+// (bf16 / fp32, GB/s over order + 3 words): orders 0 and 1 want many small CTAs (6030 / 6260 and 6330 /
+// 6250 against 5200 / 5450 and 5640 / 5930 with the table layout's shape), order 2 one vector per thread
+// (6610 / 6550 against 6230 / 6560), orders 3 and 4 the table layout's shape (6600-6990).
+#ifndef SPECA_SHAPES_FUSED_HISTORY
+#define SPECA_SHAPES_FUSED_HISTORY \
+    {32, 128, 2, 4, 3}, {32, 128, 2, 4, 3}, {32, 512, 1, 2, 1}, {32, 256, 2, 2, 1}, { 32, 256, 2, 2, 1 }
+#endif
+__host__ __device__ constexpr Shape fused_shape(int v, bool hist = false) {
     constexpr Shape fs[SPECA_MAX_ORDER + 1] = {SPECA_SHAPES_FUSED};
-    return fs[v < 0 ? 0 : (v > SPECA_MAX_ORDER ? SPECA_MAX_ORDER : v)];
+    constexpr Shape fh[SPECA_MAX_ORDER + 1] = {SPECA_SHAPES_FUSED_HISTORY};
+    const int i = v < 0 ? 0 : (v > SPECA_MAX_ORDER ? SPECA_MAX_ORDER : v);
+    return hist ? fh[i] : fs[i];
 }
-static_assert(shape_tile_bytes(fused_shape(0)) == shape_tile_bytes(shape_for(SPECA_PATH_WIDE, true, 0, SPECA_BF16)) &&
-                  shape_tile_bytes(fused_shape(2)) == shape_tile_bytes(shape_for(SPECA_PATH_WIDE, true, 2, SPECA_BF16)) &&
-                  shape_tile_bytes(fused_shape(4)) == shape_tile_bytes(shape_for(SPECA_PATH_WIDE, true, 4, SPECA_BF16)),
-              "the fused kernel walks the update's tile table");
+constexpr bool fused_shapes_fit_the_update_tiles() {
+    for (int v = 0; v <= SPECA_MAX_ORDER; ++v)
+        for (int h = 0; h < 2; ++h)
+            if (shape_tile_bytes(fused_shape(v, h != 0)) != shape_tile_bytes(shape_for(SPECA_PATH_WIDE, true, v, SPECA_BF16)))
+                return false;
+    return true;
+}
+static_assert(fused_shapes_fit_the_update_tiles(), "the fused kernel walks the update's tile table");
 
-template <int DT>
+template <int DT, bool HIST>
 static const void* fused_kernel_for(int v) {
-    constexpr Shape s0 = fused_shape(0), s1 = fused_shape(1), s2 = fused_shape(2), s3 = fused_shape(3), s4 = fused_shape(4);
+    constexpr Shape s0 = fused_shape(0, HIST), s1 = fused_shape(1, HIST), s2 = fused_shape(2, HIST), s3 = fused_shape(3, HIST),
+                    s4 = fused_shape(4, HIST);
     switch (v) {
-        case 0: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 0, s0.w, s0.nt, s0.u, s0.chunks, s0.minb>);
-        case 1: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 1, s1.w, s1.nt, s1.u, s1.chunks, s1.minb>);
-        case 2: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 2, s2.w, s2.nt, s2.u, s2.chunks, s2.minb>);
-        case 3: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 3, s3.w, s3.nt, s3.u, s3.chunks, s3.minb>);
-        default: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 4, s4.w, s4.nt, s4.u, s4.chunks, s4.minb>);
+        case 0: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 0, s0.w, s0.nt, s0.u, s0.chunks, s0.minb, HIST>);
+        case 1: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 1, s1.w, s1.nt, s1.u, s1.chunks, s1.minb, HIST>);
+        case 2: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 2, s2.w, s2.nt, s2.u, s2.chunks, s2.minb, HIST>);
+        case 3: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 3, s3.w, s3.nt, s3.u, s3.chunks, s3.minb, HIST>);
+        default: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 4, s4.w, s4.nt, s4.u, s4.chunks, s4.minb, HIST>);
     }
 }
 
-int fused_ctas_per_sm(int order) { return fused_shape(order).minb; }
+int fused_ctas_per_sm(int order, bool raw_features) { return fused_shape(order, raw_features).minb; }
 
 // The kernel is compiled for the highest order any sample has in either half of the launch.
 cudaError_t launch_update_forecast(const FusedParams& p, int dtype, int grid, cudaStream_t stream) {
     int v = max_order(p.up.order);
     const int vf = max_order(p.fc_order);
     v = vf > v ? vf : v;
-    const void* fn = dtype == SPECA_BF16 ? fused_kernel_for<SPECA_BF16>(v) : fused_kernel_for<SPECA_F32>(v);
+    const bool hist = p.up.weighted != 0;
+    const void* fn;
+    if (hist)
+        fn = dtype == SPECA_BF16 ? fused_kernel_for<SPECA_BF16, true>(v) : fused_kernel_for<SPECA_F32, true>(v);
+    else
+        fn = dtype == SPECA_BF16 ? fused_kernel_for<SPECA_BF16, false>(v) : fused_kernel_for<SPECA_F32, false>(v);
     void* args[1] = {const_cast<FusedParams*>(&p)};
-    return cudaLaunchKernel(fn, dim3(grid), dim3(fused_shape(v).nt), args, 0, stream);
+    return cudaLaunchKernel(fn, dim3(grid), dim3(fused_shape(v, hist).nt), args, 0, stream);
 }
 
 template <int DT, int KCLASS>

@@ -173,8 +173,7 @@ class SpecaCacheBackend:
 
     def reference_step(self, feats, t_ref, mask, t_next=None):
         S = self.S
-        fused = (self.use_fused and t_next is not None and self.cache.layout == S.SPECA_LAYOUT_TABLES and
-                 self.cache.path in (S.SPECA_PATH_AUTO, S.SPECA_PATH_WIDE))
+        fused = self.use_fused and t_next is not None and self.cache.path in (S.SPECA_PATH_AUTO, S.SPECA_PATH_WIDE)
         if fused:
             # Eq. 3, the re-arming and Eq. 2 at the next step's time in one launch: samples that took this
             # step are forecast from the planes just written, the ones still speculating from theirs

@@ -65,9 +65,9 @@ def test_random_scenario(S, U, seed):
         path = int(rng.choice([0, 3]))        # which only the default kernels serve
     pair = U.Pair(entries, B, m, dtype, basis, verify_entry=vidx, path=path, layout=layout)
     nv, dv = entries[pair.vidx]
-    # a second cache takes every reference step through the fused call (where that call exists): its tables
+    # a second cache takes every reference step through the fused call (where that call exists): its planes
     # and its forecast must be, bit for bit, those of update + commit + forecast on the first one
-    shadow = S.SpecaCache(entries, B, m, dtype, DEV, basis, vidx, path=path) if layout == 0 and path in (0, 3) else None
+    shadow = S.SpecaCache(entries, B, m, dtype, DEV, basis, vidx, path=path, layout=layout) if path in (0, 3) else None
     ones = torch.ones(B, dtype=torch.uint8, device=DEV)
     what = "seed %d (B=%d m=%d dtype=%d basis=%d path=%d layout=%d entries=%s)" % (seed, B, m, dtype, basis, path, layout, entries)
 

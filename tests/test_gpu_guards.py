@@ -125,9 +125,18 @@ def test_nothing_is_written_outside_the_buffers_raw_feature_cache(S, dtype, tdt,
         cur, nxt = Guarded((B,), torch.uint8, fill=1), Guarded((B,), torch.uint8)
         spec, idx, n_act = Guarded((B,), torch.int32, fill=0), Guarded((B,), torch.int32), Guarded((1,), torch.int32)
         S.speca_verify_select(handle, 0, fresh, t, [0.1] * B, cur.t, nxt.t, pred.t, err.t, acc.t, 3, 1, spec.t, idx.t, n_act.t)
+        # the fused reference step: copy into the ring and two forecasts per entry in one launch
+        ffeats = [Guarded((B, n, d), tdt, offset=shift) for n, d in RAGGED]
+        for f in ffeats:
+            f.t.copy_(torch.randn(f.t.shape, generator=gen, device=DEV).to(tdt))
+        fouts = [Guarded((2, B, n, d), tdt, offset=shift) for n, d in RAGGED]
+        t_new = 0.05 - shift
+        S.speca_cache_update_forecast_multi(handle, [f.t for f in ffeats], [t_new] * B, [1, 1, 0],
+                                            [[t_new - 0.02] * B, [t_new - 0.04] * B], None, [o.t for o in fouts], None, None)
         torch.cuda.synchronize()
-        for g in outs + [pred, err, acc, cur, nxt, spec, idx, n_act, arena]:
+        for g in outs + fouts + ffeats + [pred, err, acc, cur, nxt, spec, idx, n_act, arena]:
             assert g.intact(), "a guard zone was overwritten (dtype %d, order %d, shift %d)" % (dtype, m, shift)
         assert not bool((outs[2].t.view(torch.uint8) == PATTERN).all())
+        assert not bool((fouts[1].t.view(torch.uint8) == PATTERN).all())
     S.speca_cache_destroy(handle)
     assert arena.intact()

@@ -70,14 +70,13 @@ def test_sampler_trace_matches_oracle(S, name, metric, layout):
     st = cache.stats()
     assert st["reference_steps"] == [f + r for f, _, r in (tr_gpu.counts(b) for b in range(w.batch))]
     n_spec_steps = sum(1 for row in tr_gpu.steps if any(x != SCH.FULL for x in row))
-    # a reference step hands over the next step's forecasts in the same launch (difference-table caches):
+    # a reference step hands over the next step's forecasts in the same launch (either layout):
     # a speculative step that follows one issues no forecast launch of its own
     took_ref = [any(x != SCH.ACCEPTED for x in row) for row in tr_gpu.steps]
-    handed_over = sum(1 for i in range(1, len(tr_gpu.steps)) if layout == 0 and took_ref[i - 1] and i >= 3
+    handed_over = sum(1 for i in range(1, len(tr_gpu.steps)) if took_ref[i - 1] and i >= 3
                       and any(x != SCH.FULL for x in tr_gpu.steps[i]))
     assert st["verify_launches"] == n_spec_steps and st["forecast_launches"] == n_spec_steps - handed_over
-    if layout == 0:
-        assert st["update_forecast_launches"] == sum(1 for i in range(len(tr_gpu.steps) - 1) if took_ref[i] and i + 1 >= 3)
+    assert st["update_forecast_launches"] == sum(1 for i in range(len(tr_gpu.steps) - 1) if took_ref[i] and i + 1 >= 3)
     assert st["select_launches"] == 0 and st["resets"] == [1] * w.batch
     assert sum(st[k] for k in st if k.endswith("_launches")) == cache.launches
     cache.close()

@@ -126,9 +126,6 @@ def test_fused_reference_step_refuses_what_it_cannot_do_and_leaves_the_history_a
             fn()
         return ei.value.status
 
-    hist = S.SpecaCache(entries, B, 2, 1, DEV, layout=S.SPECA_LAYOUT_HISTORY)
-    assert status(lambda: hist.update_forecast(feats, [1.0] * B, [0.9] * B, outs)) == S.SPECA_ERR_UNSUPPORTED
-    hist.close()
     bulk = S.SpecaCache(entries, B, 2, 1, DEV, path=S.SPECA_PATH_BULK)
     assert status(lambda: bulk.update_forecast(feats, [1.0] * B, [0.9] * B, outs)) == S.SPECA_ERR_UNSUPPORTED
     bulk.close()
@@ -268,7 +265,87 @@ def test_fused_reference_step_can_be_captured_into_a_cuda_graph(S):
     torch.cuda.synchronize()
     for e in range(len(entries)):
         assert torch.equal(bits(outs_a[e]), bits(outs_b[e]))
-        for s in range(B):
-            assert torch.equal(bits(a.plane_tensor(e, s)), bits(b.plane_tensor(e, s)))
+        for s, refs in enumerate(a.state()[0]):               # the planes that hold a difference (the rest is unwritten memory)
+            assert torch.equal(bits(a.plane_tensor(e, s)[:refs]), bits(b.plane_tensor(e, s)[:refs]))
+    a.close()
+    b.close()
+
+
+@pytest.mark.parametrize("dtype,tdt", [(1, torch.bfloat16), (0, torch.float32)])
+@pytest.mark.parametrize("basis", [0, 1, 2])
+@pytest.mark.parametrize("m,K", [(0, 1), (1, 2), (2, 1), (2, 3), (3, 1), (4, 2)])
+def test_fused_reference_step_on_a_raw_feature_cache(S, dtype, tdt, basis, m, K):
+    """SPECA_LAYOUT_HISTORY: the step copies the feature into its ring plane and forms the weighted sum with
+    the feature still in registers. Ring planes and forecasts bit for bit those of update + commit +
+    speca_forecast_multi on a twin cache (which the raw-feature tests hold against the oracle), through
+    the warm-up, past the ring's wrap, with a sample that skips a step and one that has dropped out."""
+    B, ne = 3, len(ENTRIES)
+    a = S.SpecaCache(ENTRIES, B, m, dtype, DEV, basis=basis, layout=S.SPECA_LAYOUT_HISTORY)
+    b = S.SpecaCache(ENTRIES, B, m, dtype, DEV, basis=basis, layout=S.SPECA_LAYOUT_HISTORY)
+    gen = torch.Generator(device=DEV).manual_seed(1000 + 10 * m + K)
+    act_a = torch.ones(B, dtype=torch.uint8, device=DEV)
+    act_b = torch.ones(B, dtype=torch.uint8, device=DEV)
+    spec_a, spec_b = torch.zeros(B, dtype=torch.int32, device=DEV), torch.zeros(B, dtype=torch.int32, device=DEV)
+    t = 1.0
+    plan = [[1, 1, 1]] * (m + 1) + [[1, 0, 1], [0, 1, 1], [1, 1, 1], [1, 1, 1]]
+    for k, mask in enumerate(plan):
+        t -= 0.04 + 0.003 * (k % 2)
+        t_ref = [t - 0.002 * s for s in range(B)]
+        targets = [[x - 0.007 * (j + 1) for x in t_ref] for j in range(K)]
+        if k == m + 2:
+            act_a[0] = 0
+            act_b[0] = 0
+        feats = [torch.randn(B, n, d, generator=gen, device=DEV).to(tdt) for n, d in ENTRIES]
+        outs_a = [torch.full((K, B, n, d), 7.0, dtype=tdt, device=DEV) for n, d in ENTRIES]
+        outs_b = [torch.full((K, B, n, d), 7.0, dtype=tdt, device=DEV) for n, d in ENTRIES]
+        skip = k % ne
+        give_a = [None if e == skip else o for e, o in enumerate(outs_a)]
+        give_b = [None if e == skip else o for e, o in enumerate(outs_b)]
+        a.update_forecast_multi(feats, t_ref, targets, give_a, mask=mask, active=act_a, spec_count=spec_a, rearm=act_a)
+        b.update_activate(feats, t_ref, mask, spec_b, act_b)
+        b.commit_step()
+        b.forecast_multi(targets, give_b, act_b)
+        torch.cuda.synchronize()
+        refs = a.state()[0]
+        assert refs == b.state()[0]
+        for e in range(ne):
+            for s in range(B):
+                live = min(m + 1, refs[s])                   # ring planes that hold a feature
+                assert torch.equal(bits(a.plane_tensor(e, s)[:live]), bits(b.plane_tensor(e, s)[:live])), ("ring", k, e, s)
+            assert torch.equal(bits(outs_a[e]), bits(outs_b[e])), ("forecasts", k, e)
+        assert torch.equal(act_a, act_b) and torch.equal(spec_a, spec_b)
+    a.close()
+    b.close()
+
+
+def test_fused_reference_step_with_features_already_in_their_ring_planes(S):
+    """A model that writes its block output straight into the next ring plane (speca_cache_next_slot) passes
+    that pointer, or SPECA_FEATURE_IN_PLACE: nothing is copied and the forecast reads the feature where it is."""
+    entries = [(64, 1024), (9, 1031)]
+    m = 2
+    a = S.SpecaCache(entries, 1, m, 1, DEV, layout=S.SPECA_LAYOUT_HISTORY)
+    b = S.SpecaCache(entries, 1, m, 1, DEV, layout=S.SPECA_LAYOUT_HISTORY)
+    gen = torch.Generator(device=DEV).manual_seed(5)
+    t = 1.0
+    for k in range(m + 3):
+        t -= 0.05
+        feats = [torch.randn(1, n, d, generator=gen, device=DEV).bfloat16() for n, d in entries]
+        slots = [a.next_slot_tensor(e) for e in range(len(entries))]
+        for sl, f in zip(slots, feats):
+            sl.copy_(f[0])
+        outs_a = [torch.full((1, n, d), 7.0, dtype=torch.bfloat16, device=DEV) for n, d in entries]
+        outs_b = [torch.full((1, n, d), 7.0, dtype=torch.bfloat16, device=DEV) for n, d in entries]
+        launches = a.launches
+        how = [slots[0], S.SPECA_FEATURE_IN_PLACE] if k % 2 else [S.SPECA_FEATURE_IN_PLACE, slots[1]]
+        a.update_forecast(how, [t], [t - 0.02], outs_a)
+        b.update(feats, [t])
+        b.commit_step()
+        b.forecast([t - 0.02], outs_b)
+        torch.cuda.synchronize()
+        assert a.launches == launches + 1
+        for e in range(len(entries)):
+            live = min(m + 1, k + 1)
+            assert torch.equal(bits(a.plane_tensor(e, 0)[:live]), bits(b.plane_tensor(e, 0)[:live])), (k, e)
+            assert torch.equal(bits(outs_a[e]), bits(outs_b[e])), (k, e)
     a.close()
     b.close()
