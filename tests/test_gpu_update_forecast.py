@@ -147,20 +147,22 @@ def test_fused_reference_step_refuses_what_it_cannot_do_and_leaves_the_history_a
     c.close()
 
 
-def test_fused_reference_step_at_full_size(S):
+@pytest.mark.parametrize("layout", [0, 1])
+def test_fused_reference_step_at_full_size(S, layout):
     """FLUX-shaped cache at full size, every entry in the one launch, the verification entry updated only:
-    every plane and every forecast bit for bit equal to the three calls."""
+    every plane and every forecast bit for bit equal to the three calls, for difference tables and for a
+    cache that keeps raw features (there one step further, past the ring's wrap)."""
     w = W.flux()
     B, m, ne = w.batch, w.max_order, len(w.entries)
     src = W.FeatureSource(w, DEV)
-    a = S.SpecaCache(w.entries, B, m, w.dtype, DEV)
-    b = S.SpecaCache(w.entries, B, m, w.dtype, DEV)
+    a = S.SpecaCache(w.entries, B, m, w.dtype, DEV, layout=layout)
+    b = S.SpecaCache(w.entries, B, m, w.dtype, DEV, layout=layout)
     outs_a = [torch.empty(B, n, d, dtype=w.torch_dtype, device=DEV) for n, d in w.entries]
     outs_b = [torch.empty(B, n, d, dtype=w.torch_dtype, device=DEV) for n, d in w.entries]
     give_a, give_b = list(outs_a), list(outs_b)
     give_a[w.vidx] = None
     give_b[w.vidx] = None
-    for step in range(m + 2):                                # orders 0, 1, 2 warming up, then steady state
+    for step in range(m + 2 + layout):                       # orders 0, 1, 2 warming up, then steady state
         t = [w.times[step]] * B
         t_tgt = [w.times[step + 1]] * B
         feats = [src.feature(e, step, t) for e in range(ne)]
