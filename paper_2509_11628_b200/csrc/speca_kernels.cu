@@ -2036,25 +2036,32 @@ cudaError_t launch_forecast(const StreamParams& p, int dtype, int path, int grid
 #define SPECA_SHAPES_FUSED_HISTORY \
     {32, 128, 2, 4, 3}, {32, 128, 2, 4, 3}, {32, 512, 1, 2, 1}, {32, 256, 2, 2, 1}, { 32, 256, 2, 2, 1 }
 #endif
-__host__ __device__ constexpr Shape fused_shape(int v, bool hist = false) {
+// One exception by storage type, measured like the others: order 1 on bf16 tables runs at 6300 GB/s with
+// one vector per thread against 5990 with two, while fp32 drops to 4520 with one (6320 with two).
+#ifndef SPECA_SHAPE_FUSED1_BF16
+#define SPECA_SHAPE_FUSED1_BF16 { 32, 256, 1, 4, 2 }
+#endif
+__host__ __device__ constexpr Shape fused_shape(int v, bool hist, int dtype) {
     constexpr Shape fs[SPECA_MAX_ORDER + 1] = {SPECA_SHAPES_FUSED};
     constexpr Shape fh[SPECA_MAX_ORDER + 1] = {SPECA_SHAPES_FUSED_HISTORY};
     const int i = v < 0 ? 0 : (v > SPECA_MAX_ORDER ? SPECA_MAX_ORDER : v);
+    if (!hist && i == 1 && dtype == SPECA_BF16) return Shape SPECA_SHAPE_FUSED1_BF16;
     return hist ? fh[i] : fs[i];
 }
 constexpr bool fused_shapes_fit_the_update_tiles() {
     for (int v = 0; v <= SPECA_MAX_ORDER; ++v)
         for (int h = 0; h < 2; ++h)
-            if (shape_tile_bytes(fused_shape(v, h != 0)) != shape_tile_bytes(shape_for(SPECA_PATH_WIDE, true, v, SPECA_BF16)))
-                return false;
+            for (int dt = 0; dt < 2; ++dt)
+                if (shape_tile_bytes(fused_shape(v, h != 0, dt)) != shape_tile_bytes(shape_for(SPECA_PATH_WIDE, true, v, dt)))
+                    return false;
     return true;
 }
 static_assert(fused_shapes_fit_the_update_tiles(), "the fused kernel walks the update's tile table");
 
 template <int DT, bool HIST>
 static const void* fused_kernel_for(int v) {
-    constexpr Shape s0 = fused_shape(0, HIST), s1 = fused_shape(1, HIST), s2 = fused_shape(2, HIST), s3 = fused_shape(3, HIST),
-                    s4 = fused_shape(4, HIST);
+    constexpr Shape s0 = fused_shape(0, HIST, DT), s1 = fused_shape(1, HIST, DT), s2 = fused_shape(2, HIST, DT),
+                    s3 = fused_shape(3, HIST, DT), s4 = fused_shape(4, HIST, DT);
     switch (v) {
         case 0: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 0, s0.w, s0.nt, s0.u, s0.chunks, s0.minb, HIST>);
         case 1: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 1, s1.w, s1.nt, s1.u, s1.chunks, s1.minb, HIST>);
@@ -2064,7 +2071,7 @@ static const void* fused_kernel_for(int v) {
     }
 }
 
-int fused_ctas_per_sm(int order, bool raw_features) { return fused_shape(order, raw_features).minb; }
+int fused_ctas_per_sm(int order, bool raw_features, int dtype) { return fused_shape(order, raw_features, dtype).minb; }
 
 // The kernel is compiled for the highest order any sample has in either half of the launch.
 cudaError_t launch_update_forecast(const FusedParams& p, int dtype, int grid, cudaStream_t stream) {
@@ -2078,7 +2085,7 @@ cudaError_t launch_update_forecast(const FusedParams& p, int dtype, int grid, cu
     else
         fn = dtype == SPECA_BF16 ? fused_kernel_for<SPECA_BF16, false>(v) : fused_kernel_for<SPECA_F32, false>(v);
     void* args[1] = {const_cast<FusedParams*>(&p)};
-    return cudaLaunchKernel(fn, dim3(grid), dim3(fused_shape(v, hist).nt), args, 0, stream);
+    return cudaLaunchKernel(fn, dim3(grid), dim3(fused_shape(v, hist, dtype).nt), args, 0, stream);
 }
 
 template <int DT, int KCLASS>
