@@ -726,10 +726,11 @@ def adaptive_sweep(device: str, peak: float, path: int, orders=(1, 2, 3), horizo
     return out
 
 
-def sampler_run(device: str, path: int, name: str, layout: int = 0):
+def sampler_run(device: str, path: int, name: str, layout: int = 0, horizon: int = 1):
     """The whole forecast-then-verify loop (50 sampler steps) over the library with the seeded feature
     generator standing in for the transformer: which steps each sample took in full, acceptance rate,
-    speed-up by the paper's cost model next to Eq. 8, and the device time the cache path itself took."""
+    speed-up by the paper's cost model next to Eq. 8, and the device time the cache path itself took.
+    With `horizon` > 1 a reference step of the whole batch forecasts that many coming steps in its pass."""
     from paper_2509_11628_b200 import binding as S
     from paper_2509_11628_b200 import scheduler as SCH
     w = W.flux_adaptive(max_order=2, batch=8) if name == "flux_adaptive" else W.BY_NAME[name]()
@@ -746,7 +747,7 @@ def sampler_run(device: str, path: int, name: str, layout: int = 0):
 
     class Timed(SCH.SpecaCacheBackend):
         def __init__(self, cache):
-            super().__init__(cache)
+            super().__init__(cache, horizon=horizon)
             self.spans = {"forecast": [], "verify+select": [], "update": []}
 
         def _timed(self, key, fn):
@@ -757,14 +758,14 @@ def sampler_run(device: str, path: int, name: str, layout: int = 0):
             self.spans[key].append((e0, e1))
             return out
 
-        def forecast(self, t):
-            return self._timed("forecast", lambda: SCH.SpecaCacheBackend.forecast(self, t))
+        def forecast(self, t, t_later=()):
+            return self._timed("forecast", lambda: SCH.SpecaCacheBackend.forecast(self, t, t_later))
 
         def verify_and_select(self, fresh, t, tau, period):
             return self._timed("verify+select", lambda: SCH.SpecaCacheBackend.verify_and_select(self, fresh, t, tau, period))
 
-        def reference_step(self, feats, t, mask, t_next=None):
-            return self._timed("update", lambda: SCH.SpecaCacheBackend.reference_step(self, feats, t, mask, t_next))
+        def reference_step(self, feats, t, mask, t_next=None, t_later=()):
+            return self._timed("update", lambda: SCH.SpecaCacheBackend.reference_step(self, feats, t, mask, t_next, t_later))
 
     be = Timed(cache)
     wall0 = time.perf_counter()
@@ -774,7 +775,7 @@ def sampler_run(device: str, path: int, name: str, layout: int = 0):
     ms = {k: [a.elapsed_time(b_) for a, b_ in v] for k, v in be.spans.items()}
     lib_ms = sum(sum(v) for v in ms.values())
     res = {
-        "workload": w.name, "sampler_steps": len(w.times), "period": w.period, "warm_refs": w.warm_refs, "gamma": gamma,
+        "workload": w.name, "horizon": horizon, "sampler_steps": len(w.times), "period": w.period, "warm_refs": w.warm_refs, "gamma": gamma,
         "sigma": w.sigma, "acceptance_rate": tr.acceptance_rate(), "speedup_cost_model": tr.speedup(),
         "speedup_eq8": tr.predicted_speedup(), "full_steps_histogram": tr.full_steps_histogram(),
         "per_sample": ["".join(row[b] for row in tr.steps) for b in range(w.batch)],
@@ -1276,9 +1277,15 @@ def main(argv=None):
         except Exception as exc:  # report, do not hide
             detail["adaptive"] = {"error": repr(exc)}
         detail["sampler"] = {}
-        for name in ("dit_xl2", "flux_adaptive"):
+        for name in ("dit_xl2", "flux", "flux_adaptive"):
             try:
                 detail["sampler"][name] = sampler_run(device, path, name)
+                if path in (0, 3) and name != "flux_adaptive":
+                    # batches whose samples stay in step: a reference step hands over the whole run that follows
+                    far = sampler_run(device, path, name, horizon=W.BY_NAME[name]().period)
+                    assert far["per_sample"] == detail["sampler"][name]["per_sample"]     # same decisions
+                    detail["sampler"][name]["with_horizon"] = {k: far[k] for k in (
+                        "horizon", "library_ms_total", "calls", "ms_mean", "sampler_steps_per_s_library_only")}
                 if path in (0, 3):   # the same run on a cache that keeps raw features: cache-path time only
                     hist = sampler_run(device, path, name, layout=1)
                     detail["sampler"][name]["history_layout"] = {k: hist[k] for k in (

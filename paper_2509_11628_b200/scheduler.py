@@ -86,8 +86,12 @@ def run_sampler(backend, model, times: Sequence[float], tau0: float, beta: float
         tau_i = backend.tau(tau0, beta, T - i, T)
         trace.tau.append(tau_i)
         attempted = [b for b in range(B) if active[b]] if i >= warm_refs else []
+        horizon = getattr(backend, "horizon", 1)
         if attempted:
-            backend.forecast(tt)                                   # forecasts for the active samples
+            if horizon > 1:                                        # this step's forecasts, and the following steps' with them
+                backend.forecast(tt, [[x] * B for x in times[i + 1:i + horizon]])
+            else:
+                backend.forecast(tt)                               # forecasts for the active samples
             fresh = model.verify_feature(i, tt)                    # the model computes the verify layer
             e, acc = backend.verify_and_select(fresh, tt, [tau_i] * B, period)
             for b in attempted:
@@ -101,7 +105,13 @@ def run_sampler(backend, model, times: Sequence[float], tau0: float, beta: float
             # the next step is speculative for everyone who is active after this one: a backend that can
             # may hand over that step's forecasts from the same pass over the tables
             t_next = [times[i + 1]] * B if i + 1 < len(times) and i + 1 >= warm_refs else None
-            backend.reference_step(feats, tt, need_full, t_next)
+            if horizon > 1 and t_next is not None:
+                # up to `period` speculative steps follow a reference step: a backend with a horizon forecasts
+                # them all from the one pass (Fig. 1: the draft predicts the next steps from one reference)
+                later = [[x] * B for x in times[i + 2:i + 1 + min(horizon, period)]]
+                backend.reference_step(feats, tt, need_full, t_next, later)
+            else:
+                backend.reference_step(feats, tt, need_full, t_next)
             active = backend.active_mask()
         trace.steps.append(row)
         trace.err.append(errs)
@@ -112,17 +122,30 @@ class SpecaCacheBackend:
     """The CUDA library as a scheduler backend. Device buffers are allocated once; one small
     device-to-host copy of the decisions per speculative step is the only synchronisation."""
 
-    def __init__(self, cache, metric=None, use_fused=True):
+    def __init__(self, cache, metric=None, use_fused=True, horizon=1):
+        """``horizon`` K > 1: a reference step that the whole batch takes forecasts the next K steps in its
+        own pass over the tables (2v + 2 + K words per element for all K, where K single forecasts would read
+        the tables K times), and the speculative steps that follow launch only their verification. Costs K
+        output buffers per entry. A handed-over step costs one word per element if the run ends before it and
+        saves v + 1 if it is reached, so the number handed over follows the runs seen: one more than the
+        speculative run that has just ended (the first time: K). While the samples of a batch are out of step
+        with one another (reference steps that only some samples take come every step or two) only the next
+        step is handed over."""
         import torch
         from . import binding as S
         self.S, self.torch, self.cache = S, torch, cache
         self.use_fused = use_fused      # reference steps also hand over the next step's forecasts (one launch)
-        self.forecast_for = None        # the times the output buffers already hold forecasts for
+        self.horizon = max(1, min(int(horizon), S.SPECA_MAX_HORIZON)) if use_fused else 1
+        self.handed = {}                # time of a coming step (per sample, as a tuple) -> row of `multi` that holds its forecasts
+        self.in_step = False            # the last reference step was taken by the whole batch
+        self.run = None                 # speculative steps the whole batch has passed since then (None: no run seen yet)
         self.batch = cache.batch
         dev = cache.device
         self.metric = metric
-        self.outs = [torch.empty(cache.batch, n, d, dtype=torch.bfloat16 if cache.dtype == S.SPECA_BF16 else torch.float32,
-                                 device=dev) for n, d in cache.entries]
+        tdt = torch.bfloat16 if cache.dtype == S.SPECA_BF16 else torch.float32
+        # [K, B, N_e, D] per entry; `outs` are the rows the current step's forecasts are in
+        self.multi = [torch.empty(self.horizon, cache.batch, n, d, dtype=tdt, device=dev) for n, d in cache.entries]
+        self.outs = [m[0] for m in self.multi]
         self.err = torch.zeros(self.batch, dtype=torch.float32, device=dev)
         self.accept = torch.zeros(self.batch, dtype=torch.uint8, device=dev)
         self.active = torch.zeros(self.batch, dtype=torch.uint8, device=dev)
@@ -137,7 +160,7 @@ class SpecaCacheBackend:
 
     def reset_run(self):
         self.cache.reset()
-        self.forecast_for = None
+        self.handed, self.in_step, self.run = {}, False, None
         self.active.zero_()
         self.spec.zero_()
         self.h_active.zero_()
@@ -152,12 +175,20 @@ class SpecaCacheBackend:
     def tau(self, tau0, beta, t, T):
         return self.S.speca_tau(tau0, beta, t, T)
 
-    def forecast(self, t_target):
-        if self.forecast_for is not None and list(t_target) == self.forecast_for:
-            self.forecast_for = None      # the reference step before this one already wrote these forecasts
+    def forecast(self, t_target, t_later=()):
+        row = self.handed.get(tuple(t_target))
+        if row is not None:               # an earlier call already wrote these forecasts
+            self.outs = [m[row] for m in self.multi]
             return
-        self.forecast_for = None
-        self.cache.forecast(t_target, self.outs, self.active)
+        targets = [list(t_target)]
+        if self.in_step:                  # a run longer than expected: its next stretch in one read of the tables
+            targets += [list(t) for t in t_later][:self._expected_run() - 1]
+        self.handed = {tuple(t): k for k, t in enumerate(targets)}
+        self.outs = [m[0] for m in self.multi]
+        if len(targets) == 1:
+            self.cache.forecast(t_target, self.outs, self.active)
+        else:                             # the following steps' forecasts from the same read of the tables
+            self.cache.forecast_multi(targets, [m[:len(targets)] for m in self.multi], self.active)
 
     def verify_and_select(self, fresh, t_target, tau, period):
         self.accept.zero_()
@@ -165,23 +196,37 @@ class SpecaCacheBackend:
         self.cache.verify_select(fresh, t_target, tau, self.err, self.accept, self.active, self.active_next, period, 1,
                                  self.spec, self.idx, self.n_active, metric=self.metric or 0)
         self.active, self.active_next = self.active_next, self.active
+        attempted = self.h_active.tolist()
         self._fetch(with_decisions=True)
-        return self.h_err.tolist(), self.h_accept.tolist()
+        accepted = self.h_accept.tolist()
+        if self.run is not None and all(a for a, on in zip(accepted, attempted) if on):
+            self.run += 1
+        return self.h_err.tolist(), accepted
+
+    def _expected_run(self):
+        """How many coming steps to forecast at once: one more than the run that is ending (or under way)."""
+        return self.horizon if self.run is None else max(1, min(self.horizon, self.run + 1))
 
     def active_mask(self):
         return self.h_active.tolist()
 
-    def reference_step(self, feats, t_ref, mask, t_next=None):
+    def reference_step(self, feats, t_ref, mask, t_next=None, t_later=()):
         S = self.S
         fused = self.use_fused and t_next is not None and self.cache.path in (S.SPECA_PATH_AUTO, S.SPECA_PATH_WIDE)
+        self.handed = {}                  # the tables change: forecasts handed over earlier are void for the updated samples
+        self.in_step = all(mask)
         if fused:
-            # Eq. 3, the re-arming and Eq. 2 at the next step's time in one launch: samples that took this
+            # Eq. 3, the re-arming and Eq. 2 at the coming steps' times in one launch: samples that took this
             # step are forecast from the planes just written, the ones still speculating from theirs
-            self.cache.update_forecast(feats, t_ref, t_next, self.outs, mask=mask, active=self.active,
-                                       spec_count=self.spec, rearm=self.active)
-            self.forecast_for = list(t_next)
+            targets = [list(t_next)]
+            if self.in_step:              # the speculative run that follows, as long as the last one was (and one more)
+                targets += [list(t) for t in t_later][:self._expected_run() - 1]
+            self.cache.update_forecast_multi(feats, t_ref, targets, [m[:len(targets)] for m in self.multi], mask=mask,
+                                             active=self.active, spec_count=self.spec, rearm=self.active)
+            self.handed = {tuple(t): k for k, t in enumerate(targets)}
         else:
             self.cache.update_activate(feats, t_ref, mask, self.spec, self.active)   # Eq. 3 and the re-arming, one launch
             self.cache.commit_step()
-            self.forecast_for = None
+        if fused:
+            self.run = 0                  # a new run starts (warm-up references, which forecast nothing, do not count)
         self._fetch(with_decisions=False)

@@ -80,3 +80,56 @@ def test_sampler_trace_matches_oracle(S, name, metric, layout):
     assert st["select_launches"] == 0 and st["resets"] == [1] * w.batch
     assert sum(st[k] for k in st if k.endswith("_launches")) == cache.launches
     cache.close()
+
+
+@pytest.mark.parametrize("name,layout,horizon,period", [("flux", 0, 4, 4), ("flux", 1, 3, 5), ("dit_xl2", 0, 4, 4), ("dit_xl2", 0, 8, 3)])
+def test_a_horizon_hands_over_the_whole_speculative_run(S, name, layout, horizon, period):
+    """SpecaCacheBackend(horizon=K): a reference step the whole batch takes forecasts the next K steps in its own
+    pass, the speculative steps that follow launch only their verification. Same trace and errors, bit for
+    bit, as the step-by-step backend (the verification never reads the handed-over buffers), and at every
+    speculative step the buffers the model would consume hold, bit for bit, what speca_forecast gives."""
+    w = W.scaled(W.BY_NAME[name](), max_entries=3, max_tokens=40)
+    if name == "dit_xl2":
+        w.batch = 5
+        w.sigma = [0.002, 0.01, 0.02, 0.05, 0.3]                     # samples drift apart: partial reference steps
+    w.times = w.times[:32]
+    gamma = 1.0 / 28
+
+    class Checked(SCH.SpecaCacheBackend):
+        checked = 0
+
+        def forecast(self, t_target, t_later=()):
+            super().forecast(t_target, t_later)
+            ref = [torch.full_like(o, 3.0) for o in self.outs]
+            got = [o.clone() for o in self.outs]
+            launches = self.cache.launches
+            self.cache.forecast(t_target, ref, self.active)
+            torch.cuda.synchronize()
+            on = self.active.bool()
+            for g, r in zip(got, ref):
+                assert torch.equal(g[on].view(torch.uint8), r[on].view(torch.uint8))
+            Checked.checked += 1
+            self.extra = getattr(self, "extra", 0) + self.cache.launches - launches
+
+    cache = S.SpecaCache(w.entries, w.batch, w.max_order, w.dtype, DEV, layout=layout)
+    far = Checked(cache, horizon=horizon)
+    tr_far = SCH.run_sampler(far, SU.GeneratorModel(w, DEV), w.times, w.tau0, w.beta, period, 3, gamma, total_steps=50)
+    st = cache.stats()
+    cache2 = S.SpecaCache(w.entries, w.batch, w.max_order, w.dtype, DEV, layout=layout)
+    near = SCH.SpecaCacheBackend(cache2)
+    tr_near = SCH.run_sampler(near, SU.GeneratorModel(w, DEV), w.times, w.tau0, w.beta, period, 3, gamma, total_steps=50)
+    assert tr_far.steps == tr_near.steps
+    for a, b in zip(tr_far.err, tr_near.err):
+        assert np.array_equal(np.array(a), np.array(b), equal_nan=True)
+    n_spec_steps = sum(1 for row in tr_far.steps if any(x != SCH.FULL for x in row))
+    assert Checked.checked == n_spec_steps and n_spec_steps > 10
+    # forecast launches of the backend itself (without this test's checking launches), single- and multi-target
+    own_forecasts = st["forecast_launches"] - far.extra + st["forecast_multi_launches"]
+    if w.batch == 1:
+        # one sample is always in step with itself: a run no longer than the one before it (and one step)
+        # rides on its reference step; a run that outgrows that takes one multi-target launch per stretch
+        assert own_forecasts < n_spec_steps / 2
+    else:
+        assert own_forecasts <= cache2.stats()["forecast_launches"]
+    cache.close()
+    cache2.close()

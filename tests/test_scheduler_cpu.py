@@ -86,3 +86,42 @@ def test_whole_run_on_the_oracle_adapts_to_sample_difficulty():
             elif kind == SCH.REJECTED:
                 assert not tr.err[i][b] <= tr.tau[i]
     assert tr.tau[0] == pytest.approx(0.3) and tr.tau[-1] < tr.tau[0]
+
+
+class HorizonScripted(SU.ScriptedBackend):
+    """A scripted backend that announces a horizon: records which future times the sampler offers it."""
+
+    def __init__(self, batch, script, horizon):
+        super().__init__(batch, script)
+        self.horizon = horizon
+
+    def forecast(self, t_target, t_later=()):
+        self.calls.append(("forecast", self.step, tuple(t_target), tuple(tuple(t) for t in t_later)))
+
+    def reference_step(self, feats, t_ref, mask, t_next=None, t_later=()):
+        self.calls.append(("offer", self.step, None if t_next is None else tuple(t_next), tuple(tuple(t) for t in t_later)))
+        super().reference_step(feats, t_ref, mask, t_next)
+
+
+def test_a_backend_with_a_horizon_is_offered_the_times_of_the_whole_speculative_run():
+    times = [1.0 - 0.05 * i for i in range(12)]
+    B, period, warm = 2, 3, 2
+    for horizon in (2, 3, 5):
+        be = HorizonScripted(B, {(4, 1): 0}, horizon)
+        tr = SCH.run_sampler(be, SU.NullModel(), times, 0.1, 0.5, period, warm, 0.05)
+        plain = SU.ScriptedBackend(B, {(4, 1): 0})
+        assert tr.steps == SCH.run_sampler(plain, SU.NullModel(), times, 0.1, 0.5, period, warm, 0.05).steps   # same control flow
+        k = min(horizon, period)
+        for c in be.calls:
+            if c[0] == "offer":
+                i = c[1]
+                if i + 1 < warm:
+                    assert c[2] is None and c[3] == ()             # the next step is a warm-up reference: nothing to forecast
+                    continue
+                assert c[2] == (times[i + 1],) * B if i + 1 < len(times) else c[2] is None
+                want = times[i + 2:i + 1 + k]                      # never more than a run can hold, never past the end
+                assert c[3] == tuple((x,) * B for x in want), (horizon, i)
+            elif c[0] == "forecast":
+                i = c[1]
+                assert c[2] == (times[i],) * B
+                assert c[3] == tuple((x,) * B for x in times[i + 1:i + horizon])
