@@ -146,30 +146,45 @@ class SpecaCacheBackend:
         # [K, B, N_e, D] per entry; `outs` are the rows the current step's forecasts are in
         self.multi = [torch.empty(self.horizon, cache.batch, n, d, dtype=tdt, device=dev) for n, d in cache.entries]
         self.outs = [m[0] for m in self.multi]
-        self.err = torch.zeros(self.batch, dtype=torch.float32, device=dev)
-        self.accept = torch.zeros(self.batch, dtype=torch.uint8, device=dev)
-        self.active = torch.zeros(self.batch, dtype=torch.uint8, device=dev)
-        self.active_next = torch.zeros(self.batch, dtype=torch.uint8, device=dev)   # the fused call's output mask
-        self.spec = torch.zeros(self.batch, dtype=torch.int32, device=dev)
-        self.idx = torch.zeros(self.batch, dtype=torch.int32, device=dev)
+        # What the host reads back every step sits in ONE device buffer with ONE pinned mirror, so that a step
+        # costs one small copy and one stream synchronisation: errors | accept flags | the two mask buffers
+        # that the fused verification alternates between (the next mask goes to the buffer that is not read).
+        B = self.batch
+        self.pack = torch.zeros(7 * B, dtype=torch.uint8, device=dev)
+        self.h_pack = torch.zeros(7 * B, dtype=torch.uint8).pin_memory()
+        self.err = self.pack[:4 * B].view(torch.float32)
+        self.accept = self.pack[4 * B:5 * B]
+        self.masks = [self.pack[5 * B:6 * B], self.pack[6 * B:7 * B]]
+        self.cur = 0                    # which of the two masks is the current one
+        self.spec = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.idx = torch.zeros(B, dtype=torch.int32, device=dev)
         self.n_active = torch.zeros(1, dtype=torch.int32, device=dev)
-        # pinned host mirrors: one stream synchronisation per step brings back errors, decisions and mask
-        self.h_err = torch.zeros(self.batch, dtype=torch.float32).pin_memory()
-        self.h_accept = torch.zeros(self.batch, dtype=torch.uint8).pin_memory()
-        self.h_active = torch.zeros(self.batch, dtype=torch.uint8).pin_memory()
+        self.h_err = self.h_pack[:4 * B].view(torch.float32)
+        self.h_accept = self.h_pack[4 * B:5 * B]
+
+    @property
+    def active(self):
+        """The device mask of the samples that are speculating (the current one of the two buffers)."""
+        return self.masks[self.cur]
+
+    @property
+    def active_next(self):
+        return self.masks[1 - self.cur]
+
+    @property
+    def h_active(self):
+        B = self.batch
+        return self.h_pack[(5 + self.cur) * B:(6 + self.cur) * B]
 
     def reset_run(self):
         self.cache.reset()
         self.handed, self.in_step, self.run = {}, False, None
-        self.active.zero_()
+        self.pack.zero_()
         self.spec.zero_()
-        self.h_active.zero_()
+        self.h_pack.zero_()
 
     def _fetch(self, with_decisions):
-        if with_decisions:
-            self.h_err.copy_(self.err, non_blocking=True)
-            self.h_accept.copy_(self.accept, non_blocking=True)
-        self.h_active.copy_(self.active, non_blocking=True)
+        self.h_pack.copy_(self.pack, non_blocking=True)
         self.torch.cuda.current_stream(self.cache.device).synchronize()
 
     def tau(self, tau0, beta, t, T):
@@ -195,8 +210,8 @@ class SpecaCacheBackend:
         # Eq. 4 and the continuation rule in one launch; the next mask arrives in the other buffer
         self.cache.verify_select(fresh, t_target, tau, self.err, self.accept, self.active, self.active_next, period, 1,
                                  self.spec, self.idx, self.n_active, metric=self.metric or 0)
-        self.active, self.active_next = self.active_next, self.active
         attempted = self.h_active.tolist()
+        self.cur = 1 - self.cur
         self._fetch(with_decisions=True)
         accepted = self.h_accept.tolist()
         if self.run is not None and all(a for a, on in zip(accepted, attempted) if on):
