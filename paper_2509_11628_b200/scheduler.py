@@ -206,14 +206,14 @@ class SpecaCacheBackend:
             self.cache.forecast_multi(targets, [m[:len(targets)] for m in self.multi], self.active)
 
     def verify_and_select(self, fresh, t_target, tau, period):
-        self.accept.zero_()
         # Eq. 4 and the continuation rule in one launch; the next mask arrives in the other buffer
         self.cache.verify_select(fresh, t_target, tau, self.err, self.accept, self.active, self.active_next, period, 1,
                                  self.spec, self.idx, self.n_active, metric=self.metric or 0)
         attempted = self.h_active.tolist()
         self.cur = 1 - self.cur
         self._fetch(with_decisions=True)
-        accepted = self.h_accept.tolist()
+        # the launch writes the flags of the samples it verified; the others' are stale and read as "no"
+        accepted = [int(a) if on else 0 for a, on in zip(self.h_accept.tolist(), attempted)]
         if self.run is not None and all(a for a, on in zip(accepted, attempted) if on):
             self.run += 1
         return self.h_err.tolist(), accepted
