@@ -9,7 +9,10 @@
  * forecast[e][B][N_e*D] for every entry; float err[B]; uint8 accept[B]; uint8 next_active[B]; int32
  * spec_count[B]; int32 n_active.
  *
- * usage: gpu_roundtrip <out-file> <basis>
+ * usage: gpu_roundtrip <out-file> <basis> [fused]
+ * With a third argument the last reference step and the forecast are ONE call
+ * (speca_cache_update_forecast) instead of speca_cache_update + speca_cache_commit_step + speca_forecast;
+ * the file must come out the same.
  */
 #include <speca.h>
 
@@ -52,13 +55,14 @@ int main(int argc, char** argv) {
     void* dev_feat[NE];
     void* dev_out[NE];
     void *dev_fresh = NULL, *dev_small = NULL;
-    int e, step;
+    int e, step, fused;
     size_t i;
     FILE* fp;
     int32_t header[5];
     cudaStream_t stream;
 
     if (argc < 3) return 2;
+    fused = argc > 3;
     memset(&cfg, 0, sizeof cfg);
     cfg.n_entries = NE;
     cfg.entries = kEntries;
@@ -93,12 +97,17 @@ int main(int argc, char** argv) {
             CK(cudaMemcpyAsync(dev_feat[e], host, elems[e] * sizeof(float), cudaMemcpyHostToDevice, stream) == cudaSuccess);
             CK(cudaStreamSynchronize(stream) == cudaSuccess); /* host[] is reused */
         }
+        if (step == 2 && fused) { /* the reference step and the forecast that follows it, one pass over the tables */
+            CK(speca_cache_update_forecast(cache, (const void* const*)dev_feat, kTimes[step], kMask2, kTarget, NULL,
+                                           (void* const*)dev_out, NULL, NULL, stream) == SPECA_OK);
+            continue;
+        }
         CK(speca_cache_update(cache, (const void* const*)dev_feat, kTimes[step], step == 2 ? kMask2 : NULL, stream) == SPECA_OK);
         CK(speca_cache_commit_step(cache) == SPECA_OK);
     }
 
     /* speculative step: forecast everything, verify the last entry against forecast + noise */
-    CK(speca_forecast(cache, kTarget, NULL, (void* const*)dev_out, stream) == SPECA_OK);
+    if (!fused) CK(speca_forecast(cache, kTarget, NULL, (void* const*)dev_out, stream) == SPECA_OK);
     {
         const size_t nv = elems[NE - 1];
         const float level[B] = {0.0f, 0.02f, 0.5f};
@@ -162,7 +171,11 @@ int main(int argc, char** argv) {
     {
         speca_cache_stats_t st;
         CK(speca_cache_stats(cache, &st) == SPECA_OK);
-        CK(st.update_launches >= 3 && st.forecast_launches == 1 && st.verify_launches == 1 && st.select_launches == 0);
+        CK(st.verify_launches == 1 && st.select_launches == 0);
+        if (fused)
+            CK(st.update_launches >= 2 && st.forecast_launches == 0 && st.update_forecast_launches == 1);
+        else
+            CK(st.update_launches >= 3 && st.forecast_launches == 1 && st.update_forecast_launches == 0);
         CK(st.reference_steps[0] == 3 && st.reference_steps[1] == 2 && st.reference_steps[2] == 3);
     }
     CK(speca_cache_destroy(cache) == SPECA_OK);

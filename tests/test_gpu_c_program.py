@@ -41,11 +41,13 @@ def exe(tmp_path_factory):
     return out
 
 
+@pytest.mark.parametrize("fused", [False, True])     # True: the last reference step and the forecast as one call
 @pytest.mark.parametrize("basis", [O.TAYLOR, O.NEWTON, O.ADAMS_BASHFORTH])
-def test_c_program_matches_oracle(exe, tmp_path, basis):
+def test_c_program_matches_oracle(exe, tmp_path, basis, fused):
     from tests import gpu_util as U
     path = str(tmp_path / "out.bin")
-    res = subprocess.run([exe, path, str(basis)], stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True, timeout=120)
+    res = subprocess.run([exe, path, str(basis)] + (["fused"] if fused else []), stdout=subprocess.PIPE,
+                         stderr=subprocess.STDOUT, text=True, timeout=120)
     assert res.returncode == 0 and res.stdout.strip().endswith("ok"), res.stdout
     raw = open(path, "rb").read()
     B, ne, m, basis_got, n_steps = np.frombuffer(raw, np.int32, 5)
