@@ -679,7 +679,7 @@ speca_status_t speca_cache_update_forecast_multi(speca_cache_t* c, const void* c
         const int vf = launch_order(q.fc_order, c->B);
         v = vf > v ? vf : v;
         const uint32_t n_tiles = p.tile_hi - p.tile_lo;
-        const uint32_t full = static_cast<uint32_t>(c->sm_count * fused_ctas_per_sm(v, hist, c->dtype));
+        const uint32_t full = static_cast<uint32_t>(c->sm_count * fused_ctas_per_sm(v, hist, c->dtype, n_targets));
         const int grid = static_cast<int>(n_tiles < full ? n_tiles : full);
         cudaError_t ce = launch_update_forecast(q, c->dtype, grid, static_cast<cudaStream_t>(stream));
         if (ce != cudaSuccess) {

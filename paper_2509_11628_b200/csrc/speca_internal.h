@@ -168,7 +168,7 @@ struct DecideParams {
 cudaError_t launch_update(const StreamParams& p, int dtype, int path, int grid, cudaStream_t stream);
 cudaError_t launch_forecast(const StreamParams& p, int dtype, int path, int grid, cudaStream_t stream);
 cudaError_t launch_update_forecast(const FusedParams& p, int dtype, int grid, cudaStream_t stream);
-int fused_ctas_per_sm(int order, bool raw_features, int dtype);
+int fused_ctas_per_sm(int order, bool raw_features, int dtype, int n_targets);
 cudaError_t launch_verify(const VerifyParams& p, int dtype, int grid, int cluster, cudaStream_t stream);
 cudaError_t launch_select(const uint8_t* accept, int32_t k_max, int32_t group, int32_t batch, int32_t* spec_count,
                           uint8_t* active, int32_t* idx, int32_t* n_active, cudaStream_t stream);

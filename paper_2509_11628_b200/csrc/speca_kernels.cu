@@ -2041,27 +2041,37 @@ cudaError_t launch_forecast(const StreamParams& p, int dtype, int path, int grid
 #ifndef SPECA_SHAPE_FUSED1_BF16
 #define SPECA_SHAPE_FUSED1_BF16 { 32, 256, 1, 4, 2 }
 #endif
-__host__ __device__ constexpr Shape fused_shape(int v, bool hist, int dtype) {
+// With three or more targets per pass the stores dominate whatever the order and the layout, and the
+// two-vector shape wins everywhere it was measured (bf16, 20 FLUX-shaped entries, K = 3 / 5 / 8: raw features,
+// order 2, 627 / 795 / 1105 us against 648 / 865 / 1179 with the one-target shape; order 1 with K = 4, 623
+// against 683 us, and 754 against 786 us on tables).
+#ifndef SPECA_SHAPE_FUSED_MANY
+#define SPECA_SHAPE_FUSED_MANY { 32, 256, 2, 2, 1 }
+#endif
+constexpr int kFusedManyTargets = 3;
+__host__ __device__ constexpr Shape fused_shape(int v, bool hist, int dtype, bool many) {
     constexpr Shape fs[SPECA_MAX_ORDER + 1] = {SPECA_SHAPES_FUSED};
     constexpr Shape fh[SPECA_MAX_ORDER + 1] = {SPECA_SHAPES_FUSED_HISTORY};
     const int i = v < 0 ? 0 : (v > SPECA_MAX_ORDER ? SPECA_MAX_ORDER : v);
+    if (many && i >= 1) return Shape SPECA_SHAPE_FUSED_MANY;
     if (!hist && i == 1 && dtype == SPECA_BF16) return Shape SPECA_SHAPE_FUSED1_BF16;
     return hist ? fh[i] : fs[i];
 }
 constexpr bool fused_shapes_fit_the_update_tiles() {
     for (int v = 0; v <= SPECA_MAX_ORDER; ++v)
-        for (int h = 0; h < 2; ++h)
+        for (int h = 0; h < 4; ++h)
             for (int dt = 0; dt < 2; ++dt)
-                if (shape_tile_bytes(fused_shape(v, h != 0, dt)) != shape_tile_bytes(shape_for(SPECA_PATH_WIDE, true, v, dt)))
+                if (shape_tile_bytes(fused_shape(v, (h & 1) != 0, dt, (h & 2) != 0)) !=
+                    shape_tile_bytes(shape_for(SPECA_PATH_WIDE, true, v, dt)))
                     return false;
     return true;
 }
 static_assert(fused_shapes_fit_the_update_tiles(), "the fused kernel walks the update's tile table");
 
-template <int DT, bool HIST>
+template <int DT, bool HIST, bool MANY>
 static const void* fused_kernel_for(int v) {
-    constexpr Shape s0 = fused_shape(0, HIST, DT), s1 = fused_shape(1, HIST, DT), s2 = fused_shape(2, HIST, DT),
-                    s3 = fused_shape(3, HIST, DT), s4 = fused_shape(4, HIST, DT);
+    constexpr Shape s0 = fused_shape(0, HIST, DT, MANY), s1 = fused_shape(1, HIST, DT, MANY), s2 = fused_shape(2, HIST, DT, MANY),
+                    s3 = fused_shape(3, HIST, DT, MANY), s4 = fused_shape(4, HIST, DT, MANY);
     switch (v) {
         case 0: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 0, s0.w, s0.nt, s0.u, s0.chunks, s0.minb, HIST>);
         case 1: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 1, s1.w, s1.nt, s1.u, s1.chunks, s1.minb, HIST>);
@@ -2070,22 +2080,28 @@ static const void* fused_kernel_for(int v) {
         default: return reinterpret_cast<const void*>(&update_forecast_kernel<DT, 4, s4.w, s4.nt, s4.u, s4.chunks, s4.minb, HIST>);
     }
 }
+template <int DT, bool HIST>
+static const void* fused_kernel_for(int v, bool many) {
+    return many ? fused_kernel_for<DT, HIST, true>(v) : fused_kernel_for<DT, HIST, false>(v);
+}
 
-int fused_ctas_per_sm(int order, bool raw_features, int dtype) { return fused_shape(order, raw_features, dtype).minb; }
+int fused_ctas_per_sm(int order, bool raw_features, int dtype, int n_targets) {
+    return fused_shape(order, raw_features, dtype, n_targets >= kFusedManyTargets).minb;
+}
 
 // The kernel is compiled for the highest order any sample has in either half of the launch.
 cudaError_t launch_update_forecast(const FusedParams& p, int dtype, int grid, cudaStream_t stream) {
     int v = max_order(p.up.order);
     const int vf = max_order(p.fc_order);
     v = vf > v ? vf : v;
-    const bool hist = p.up.weighted != 0;
+    const bool hist = p.up.weighted != 0, many = p.n_targets >= kFusedManyTargets;
     const void* fn;
     if (hist)
-        fn = dtype == SPECA_BF16 ? fused_kernel_for<SPECA_BF16, true>(v) : fused_kernel_for<SPECA_F32, true>(v);
+        fn = dtype == SPECA_BF16 ? fused_kernel_for<SPECA_BF16, true>(v, many) : fused_kernel_for<SPECA_F32, true>(v, many);
     else
-        fn = dtype == SPECA_BF16 ? fused_kernel_for<SPECA_BF16, false>(v) : fused_kernel_for<SPECA_F32, false>(v);
+        fn = dtype == SPECA_BF16 ? fused_kernel_for<SPECA_BF16, false>(v, many) : fused_kernel_for<SPECA_F32, false>(v, many);
     void* args[1] = {const_cast<FusedParams*>(&p)};
-    return cudaLaunchKernel(fn, dim3(grid), dim3(fused_shape(v, hist, dtype).nt), args, 0, stream);
+    return cudaLaunchKernel(fn, dim3(grid), dim3(fused_shape(v, hist, dtype, many).nt), args, 0, stream);
 }
 
 template <int DT, int KCLASS>
